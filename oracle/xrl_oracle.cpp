@@ -1,0 +1,396 @@
+// CPU oracle for the X-RLflow agent's per-step forward pass.
+//
+// TEST INFRASTRUCTURE, NOT PRODUCT CODE.  This file is the slow, plain statement of what
+// the path computes: per-node and per-edge loops in double precision, no blocking, no
+// fusion, no SIMD, no BLAS.  It shares nothing with the CUDA library (no header, no
+// helper, no table) and must never be called from it.  Only tests, the smoke check and
+// the benchmark's CPU-baseline leg may load it.
+//
+// What it follows (sections and equations of the X-RLflow paper):
+//   xo_pack          Section 3.3.2  "batch them into a meta-graph"
+//   xo_encode        Section 3.4    Eq. 6 (node update), Eq. 7 (k graph-attention layers,
+//                                   attention as in the GAT paper it cites), Eq. 8 (global update)
+//   xo_policy_value  Section 3.3.2  two-layer MLP heads, padded action space with a boolean
+//                                   mask, No-Op action; Section 3.3.3 invalid-action masking
+//   xo_sample        Section 3.3.2  "the action sampled from the categorical distribution";
+//                                   random words from Philox4x32-10 (Salmon et al., SC'11)
+// Readings of what the paper leaves open (activation = ReLU, LeakyReLU slope 0.2 inside the
+// attention score, in-neighbours plus self, heads concatenated, biases, a weight matrix in
+// Eq. 8, per-graph scoring for the policy) are listed in the design notes of the repository.
+//
+// Parity pins: every function below is pinned by tests that do not call it to produce
+// their expected values (dense-adjacency brute force in numpy, closed forms on chains and
+// stars, invariants, a third-party Philox).  Nothing here is "parity unpinned".
+//
+// Floating point: double everywhere.  mode 0 ("exact") rounds only the inputs and those
+// weights the bf16 model stores in bf16; mode 1 ("mirrored") additionally rounds Z and every
+// layer output to bf16, as a debugging aid.
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <vector>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+namespace {
+
+enum { XO_OK = 0, XO_INVALID_ARG = 1, XO_BAD_GRAPH = 2 };
+
+struct Model {
+  int32_t T, S, H, K, L, Hm, Dg, dtype;  // dtype: 0 fp32, 1 bf16 storage
+};
+
+// bfloat16 = the upper 16 bits of an IEEE binary32; round to nearest, ties to even.
+double round_bf16(double x) {
+  float f = static_cast<float>(x);
+  uint32_t u;
+  std::memcpy(&u, &f, 4);
+  if ((u & 0x7F800000u) == 0x7F800000u) return f;  // inf / nan unchanged
+  uint32_t lsb = (u >> 16) & 1u;
+  u += 0x7FFFu + lsb;
+  u &= 0xFFFF0000u;
+  std::memcpy(&f, &u, 4);
+  return f;
+}
+
+double relu(double x) { return x > 0.0 ? x : 0.0; }
+double leaky_relu(double x) { return x > 0.0 ? x : 0.2 * x; }
+
+// Offsets into the flat weight blob (matrices row-major [in x out]).
+struct Weights {
+  const float* W0; const float* b0;
+  std::vector<const float*> W, a_src, a_dst, b;
+  const float* Wg; const float* bg;
+  const float* pW1; const float* pb1; const float* pw2; const float* pb2;
+  const float* vW1; const float* vb1; const float* vw2; const float* vb2;
+};
+
+Weights slice(const Model& m, const float* blob) {
+  Weights w;
+  const float* p = blob;
+  auto take = [&](int64_t n) { const float* q = p; p += n; return q; };
+  w.W0 = take(int64_t(2 * m.S + m.T) * m.H);
+  w.b0 = take(m.H);
+  for (int l = 0; l < m.L; ++l) {
+    w.W.push_back(take(int64_t(m.H) * m.H));
+    w.a_src.push_back(take(m.H));
+    w.a_dst.push_back(take(m.H));
+    w.b.push_back(take(m.H));
+  }
+  w.Wg = take(int64_t(m.H + m.Dg) * m.H);
+  w.bg = take(m.H);
+  w.pW1 = take(int64_t(m.H) * m.Hm); w.pb1 = take(m.Hm); w.pw2 = take(m.Hm); w.pb2 = take(1);
+  w.vW1 = take(int64_t(2 * m.H) * m.Hm); w.vb1 = take(m.Hm); w.vw2 = take(m.Hm); w.vb2 = take(1);
+  return w;
+}
+
+// A weight as the model stores it: Eq. 6 and Eq. 7 matrices live in bf16 when dtype = 1.
+double stored(const Model& m, float w) { return m.dtype == 1 ? round_bf16(w) : double(w); }
+
+// Encode one graph (nodes [lo, hi) of the packed batch).  Writes its H-vector to `emb`.
+void encode_graph(const Model& m, const Weights& w, int32_t lo, int32_t hi,
+                  const int32_t* rowptr, const int32_t* col, const int32_t* op,
+                  const float* shape, const double* g_attr, int mode, double* emb,
+                  int dump_layer, double* node_dump, double* alpha_edge, double* alpha_self) {
+  const int S = m.S, T = m.T, H = m.H, K = m.K, d = m.H / m.K;
+  const int n = hi - lo;
+  const int F0 = 2 * S + T;
+  std::vector<double> h(size_t(n) * H), z(size_t(n) * H), hn(size_t(n) * H);
+  std::vector<double> s_src(size_t(n) * K), s_dst(size_t(n) * K);
+
+  auto dump = [&](int layer) {
+    if (node_dump && dump_layer == layer)
+      for (int i = 0; i < n; ++i)
+        for (int c = 0; c < H; ++c) node_dump[size_t(lo + i) * H + c] = h[size_t(i) * H + c];
+  };
+
+  // ---- Eq. 6: h'_i = sigma( W ( sum_{j in E_i} e_j  ||  h_i ) ).
+  // The attribute of edge j->i is the shape feature vector of its producer j; the node
+  // attribute is the one-hot operator id followed by the node's own shape features.
+  std::vector<double> x(F0), W0s(size_t(F0) * H);
+  for (size_t t = 0; t < W0s.size(); ++t) W0s[t] = stored(m, w.W0[t]);
+  for (int i = 0; i < n; ++i) {
+    const int gi = lo + i;
+    for (int s = 0; s < F0; ++s) x[s] = 0.0;
+    for (int e = rowptr[gi]; e < rowptr[gi + 1]; ++e)
+      for (int s = 0; s < S; ++s) x[s] += double(shape[size_t(col[e]) * S + s]);
+    x[S + op[gi]] = 1.0;
+    for (int s = 0; s < S; ++s) x[S + T + s] = double(shape[size_t(gi) * S + s]);
+    for (int c = 0; c < H; ++c) {
+      double acc = 0.0;
+      for (int s = 0; s < F0; ++s) acc += x[s] * W0s[size_t(s) * H + c];
+      acc += double(w.b0[c]);
+      acc = relu(acc);
+      h[size_t(i) * H + c] = (mode == 1 && m.dtype == 1) ? round_bf16(acc) : acc;
+    }
+  }
+  dump(0);
+
+  // ---- Eq. 7, k times: h'_i = sigma( sum_{j in N_i} alpha_ij W h_j ),  N_i = in(i) + {i}.
+  for (int l = 0; l < m.L; ++l) {
+    const float* W = w.W[l];
+    std::vector<double> Ws(size_t(H) * H);
+    for (size_t t = 0; t < Ws.size(); ++t) Ws[t] = stored(m, W[t]);
+    for (int i = 0; i < n; ++i) {   // z_i = W^T h_i, summed over the input index k in order
+      for (int c = 0; c < H; ++c) z[size_t(i) * H + c] = 0.0;
+      for (int k = 0; k < H; ++k)
+        for (int c = 0; c < H; ++c)
+          z[size_t(i) * H + c] += h[size_t(i) * H + k] * Ws[size_t(k) * H + c];
+    }
+    // attention half-scores per head: e_ij = LeakyReLU(a_dst . z_i + a_src . z_j), i.e. the GAT
+    // score a . [z_i || z_j] with a = [a_dst || a_src], i the receiving node
+    for (int i = 0; i < n; ++i)
+      for (int k = 0; k < K; ++k) {
+        double ss = 0.0, sd = 0.0;
+        for (int c = 0; c < d; ++c) {
+          ss += double(w.a_src[l][k * d + c]) * z[size_t(i) * H + k * d + c];
+          sd += double(w.a_dst[l][k * d + c]) * z[size_t(i) * H + k * d + c];
+        }
+        s_src[size_t(i) * K + k] = ss;
+        s_dst[size_t(i) * K + k] = sd;
+      }
+    if (mode == 1 && m.dtype == 1)
+      for (auto& v : z) v = round_bf16(v);
+
+    for (int i = 0; i < n; ++i) {
+      const int gi = lo + i;
+      const int e0 = rowptr[gi], e1 = rowptr[gi + 1];
+      const int deg = e1 - e0;
+      std::vector<double> sc(deg + 1), al(deg + 1);
+      for (int k = 0; k < K; ++k) {
+        double mx = -INFINITY;
+        for (int t = 0; t <= deg; ++t) {
+          const int j = (t < deg) ? col[e0 + t] - lo : i;   // last entry is the self term
+          sc[t] = leaky_relu(s_src[size_t(j) * K + k] + s_dst[size_t(i) * K + k]);
+          if (sc[t] > mx) mx = sc[t];
+        }
+        double sum = 0.0;
+        for (int t = 0; t <= deg; ++t) { al[t] = std::exp(sc[t] - mx); sum += al[t]; }
+        for (int t = 0; t <= deg; ++t) al[t] /= sum;
+        if (dump_layer == l + 1 && alpha_edge) {
+          for (int t = 0; t < deg; ++t) alpha_edge[size_t(e0 + t) * K + k] = al[t];
+          alpha_self[size_t(gi) * K + k] = al[deg];
+        }
+        for (int c = k * d; c < (k + 1) * d; ++c) {
+          double acc = 0.0;
+          for (int t = 0; t <= deg; ++t) {
+            const int j = (t < deg) ? col[e0 + t] - lo : i;
+            acc += al[t] * z[size_t(j) * H + c];
+          }
+          acc = relu(acc + double(w.b[l][c]));
+          hn[size_t(i) * H + c] = (mode == 1 && m.dtype == 1) ? round_bf16(acc) : acc;
+        }
+      }
+    }
+    h.swap(hn);
+    dump(l + 1);
+  }
+
+  // ---- Eq. 8: g' = sigma( W_g ( sum_N h  ||  g ) + b_g )
+  std::vector<double> u(H + m.Dg, 0.0);
+  for (int i = 0; i < n; ++i)
+    for (int c = 0; c < H; ++c) u[c] += h[size_t(i) * H + c];
+  for (int c = 0; c < m.Dg; ++c) u[H + c] = g_attr ? g_attr[c] : 0.0;
+  for (int c = 0; c < H; ++c) {
+    double acc = 0.0;
+    for (int k = 0; k < H + m.Dg; ++k) acc += u[k] * double(w.Wg[size_t(k) * H + c]);
+    emb[c] = relu(acc + double(w.bg[c]));
+  }
+}
+
+double mlp_scalar(const double* x, int in, int hid, const float* W1, const float* b1,
+                  const float* w2, const float* b2) {
+  double out = double(b2[0]);
+  for (int c = 0; c < hid; ++c) {
+    double acc = double(b1[c]);
+    for (int k = 0; k < in; ++k) acc += x[k] * double(W1[size_t(k) * hid + c]);
+    out += relu(acc) * double(w2[c]);
+  }
+  return out;
+}
+
+inline void mulhilo(uint32_t a, uint32_t b, uint32_t& hi, uint32_t& lo) {
+  uint64_t p = uint64_t(a) * uint64_t(b);
+  hi = uint32_t(p >> 32);
+  lo = uint32_t(p);
+}
+
+}  // namespace
+
+extern "C" {
+
+// Philox4x32 with 10 rounds, from its published definition (Salmon, Moraes, Dror, Shaw,
+// "Parallel random numbers: as easy as 1, 2, 3", SC'11): round = two 32x32->64 multiplies,
+// a word permutation and a key xor; the key is bumped by the Weyl constants between rounds.
+void xo_philox4x32_10(uint32_t k0, uint32_t k1, uint32_t c0, uint32_t c1, uint32_t c2,
+                      uint32_t c3, uint32_t* out) {
+  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+  const uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+  for (int r = 0; r < 10; ++r) {
+    uint32_t hi0, lo0, hi1, lo1;
+    mulhilo(M0, c0, hi0, lo0);
+    mulhilo(M1, c2, hi1, lo1);
+    uint32_t n0 = hi1 ^ c1 ^ k0, n1 = lo1, n2 = hi0 ^ c3 ^ k1, n3 = lo0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += W0; k1 += W1;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// Section 3.3.2: batch the B graphs into one meta-graph.  CSR by destination over global
+// node ids; inside a row the sources keep the order of the input edge list.
+int xo_pack(int32_t B, const int32_t* n_nodes, const int32_t* n_edges, const int32_t* edge_src,
+            const int32_t* edge_dst, int32_t num_envs, const int32_t* env_off,
+            int32_t* node_off, int32_t* edge_off, int32_t* seg_id, int32_t* graph_env,
+            int32_t* rowptr, int32_t* col) {
+  if (B < 0 || num_envs < 0) return XO_INVALID_ARG;
+  node_off[0] = 0; edge_off[0] = 0;
+  for (int g = 0; g < B; ++g) {
+    if (n_nodes[g] < 0 || n_edges[g] < 0) return XO_INVALID_ARG;
+    node_off[g + 1] = node_off[g] + n_nodes[g];
+    edge_off[g + 1] = edge_off[g] + n_edges[g];
+  }
+  if (env_off[0] != 0 || env_off[num_envs] != B) return XO_INVALID_ARG;
+  for (int e = 0; e < num_envs; ++e) {
+    if (env_off[e + 1] <= env_off[e]) return XO_INVALID_ARG;  // each env has its current graph
+    for (int g = env_off[e]; g < env_off[e + 1]; ++g) graph_env[g] = e;
+  }
+  const int32_t N = node_off[B];
+  for (int g = 0; g < B; ++g)
+    for (int i = node_off[g]; i < node_off[g + 1]; ++i) seg_id[i] = g;
+  for (int i = 0; i <= N; ++i) rowptr[i] = 0;
+  for (int g = 0; g < B; ++g)
+    for (int e = edge_off[g]; e < edge_off[g + 1]; ++e) {
+      const int32_t s = edge_src[e], t = edge_dst[e];
+      if (s < 0 || s >= n_nodes[g] || t < 0 || t >= n_nodes[g] || s == t) return XO_BAD_GRAPH;
+      rowptr[node_off[g] + t + 1] += 1;
+    }
+  for (int i = 0; i < N; ++i) rowptr[i + 1] += rowptr[i];
+  std::vector<int32_t> cursor(rowptr, rowptr + N);
+  for (int g = 0; g < B; ++g)
+    for (int e = edge_off[g]; e < edge_off[g + 1]; ++e) {
+      const int32_t t = node_off[g] + edge_dst[e];
+      col[cursor[t]++] = node_off[g] + edge_src[e];
+    }
+  return XO_OK;
+}
+
+// Section 3.4: Eq. 6 -> L x Eq. 7 -> Eq. 8 for the graphs listed in `sel` (all when null).
+// graph_emb is [n_sel x H].  node_dump (optional, [N x H]) receives the node features after
+// stage `dump_layer` (0 = Eq. 6, l = l-th attention layer) for the selected graphs;
+// alpha_edge [E x K] / alpha_self [N x K] (optional) receive that layer's attention weights.
+int xo_encode(const Model* m, const float* weights, int32_t B, const int32_t* node_off,
+              const int32_t* rowptr, const int32_t* col, const int32_t* op, const float* shape,
+              const double* g0, int32_t n_sel, const int32_t* sel, int32_t mode,
+              int32_t threads, double* graph_emb, int32_t dump_layer, double* node_dump,
+              double* alpha_edge, double* alpha_self) {
+  if (m->H % m->K != 0 || m->L < 0) return XO_INVALID_ARG;
+  const Weights w = slice(*m, weights);
+  const int count = sel ? n_sel : B;
+  int bad = 0;
+#ifdef _OPENMP
+  if (threads > 0) omp_set_num_threads(threads);
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+  for (int t = 0; t < count; ++t) {
+    const int g = sel ? sel[t] : t;
+    if (g < 0 || g >= B) { bad = 1; continue; }
+    encode_graph(*m, w, node_off[g], node_off[g + 1], rowptr, col, op, shape,
+                 g0 ? g0 + size_t(g) * m->Dg : nullptr, mode, graph_emb + size_t(t) * m->H,
+                 dump_layer, node_dump, alpha_edge, alpha_self);
+  }
+  (void)threads;
+  return bad ? XO_INVALID_ARG : XO_OK;
+}
+
+// Section 3.3.2 / 3.3.3: policy and value heads over the graph embeddings of each
+// environment.  graph env_off[e] is the current graph, the following ones its candidates.
+// logits/probs are [num_envs x (A_max+1)], the last column is No-Op (scored by the current
+// graph).  Invalid and padded actions get probability exactly 0 (logit reported as -inf).
+int xo_policy_value(const Model* m, const float* weights, int32_t num_envs,
+                    const int32_t* env_off, int32_t A_max, const double* graph_emb,
+                    const uint8_t* mask, double* logits, double* probs, double* value) {
+  const Weights w = slice(*m, weights);
+  const int H = m->H, A1 = A_max + 1;
+  for (int e = 0; e < num_envs; ++e) {
+    const int cur = env_off[e];
+    const int C = env_off[e + 1] - env_off[e] - 1;
+    if (C < 0 || C > A_max) return XO_INVALID_ARG;
+    for (int a = C; a < A_max; ++a)
+      if (mask[size_t(e) * A_max + a]) return XO_INVALID_ARG;
+    double* lg = logits + size_t(e) * A1;
+    double* pr = probs + size_t(e) * A1;
+    double mx = -INFINITY;
+    for (int a = 0; a < A1; ++a) {
+      const bool valid = (a == A_max) || mask[size_t(e) * A_max + a];
+      const int g = (a == A_max) ? cur : cur + 1 + a;
+      lg[a] = valid ? mlp_scalar(graph_emb + size_t(g) * H, H, m->Hm, w.pW1, w.pb1, w.pw2, w.pb2)
+                    : -INFINITY;
+      if (lg[a] > mx) mx = lg[a];
+    }
+    double sum = 0.0;
+    for (int a = 0; a < A1; ++a) {
+      pr[a] = (lg[a] == -INFINITY) ? 0.0 : std::exp(lg[a] - mx);
+      sum += pr[a];
+    }
+    for (int a = 0; a < A1; ++a) pr[a] /= sum;
+
+    // value: MLP over [ current graph || mean of the valid candidates ]
+    std::vector<double> u(2 * H, 0.0);
+    int nv = 0;
+    for (int c = 0; c < H; ++c) u[c] = graph_emb[size_t(cur) * H + c];
+    for (int a = 0; a < C; ++a)
+      if (mask[size_t(e) * A_max + a]) {
+        ++nv;
+        for (int c = 0; c < H; ++c) u[H + c] += graph_emb[size_t(cur + 1 + a) * H + c];
+      }
+    if (nv > 0)
+      for (int c = 0; c < H; ++c) u[H + c] /= double(nv);
+    value[e] = mlp_scalar(u.data(), 2 * H, m->Hm, w.vW1, w.vb1, w.vw2, w.vb2);
+  }
+  return XO_OK;
+}
+
+// Draw one action per environment from fp32 probabilities with integer arithmetic only.
+// q_a = floor(p_a * 2^32); Q = sum q_a; r = 64 random bits from Philox keyed by the seed with
+// counter (env, step lo, step hi, 0); t = floor(r * Q / 2^64); the action is the first index
+// whose inclusive prefix sum of q exceeds t.  Q = 0 yields No-Op (the last index).
+int xo_sample(int32_t num_envs, int32_t A1, const float* probs, uint64_t seed, uint64_t step,
+              int32_t* action) {
+  for (int e = 0; e < num_envs; ++e) {
+    uint32_t r[4];
+    xo_philox4x32_10(uint32_t(seed), uint32_t(seed >> 32), uint32_t(e), uint32_t(step),
+                     uint32_t(step >> 32), 0u, r);
+    const uint64_t r64 = uint64_t(r[0]) | (uint64_t(r[1]) << 32);
+    uint64_t Q = 0;
+    for (int a = 0; a < A1; ++a) {
+      const float p = probs[size_t(e) * A1 + a];
+      if (!(p >= 0.0f) || p > 1.0f) return XO_INVALID_ARG;
+      Q += uint64_t(std::floor(double(p) * 4294967296.0));
+    }
+    int32_t act = A1 - 1;
+    if (Q > 0) {
+      const uint64_t t = uint64_t((static_cast<unsigned __int128>(r64) * Q) >> 64);
+      uint64_t run = 0;
+      for (int a = 0; a < A1; ++a) {
+        run += uint64_t(std::floor(double(probs[size_t(e) * A1 + a]) * 4294967296.0));
+        if (run > t) { act = a; break; }
+      }
+    }
+    action[e] = act;
+  }
+  return XO_OK;
+}
+
+int xo_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+}  // extern "C"
