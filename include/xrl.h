@@ -1,0 +1,198 @@
+/* xrl -- the per-step forward pass of the X-RLflow agent on one NVIDIA B200 (sm_100a).
+ *
+ * At every rewrite step the agent observes the current computation graph together with all
+ * of its candidate rewritten graphs, encodes them with a graph neural network, reads out one
+ * vector per graph and evaluates an actor-critic policy head (masked categorical distribution
+ * over the candidates plus No-Op) and a value head (paper Sections 3.3.2, 3.3.3 and 3.4).
+ * This library is that path and nothing else:
+ *
+ *     xrl_pack / xrl_pack_flat   Section 3.3.2  batch the graphs into one meta-graph (CSR)
+ *     xrl_encode                 Section 3.4    Eq. 6 -> L x Eq. 7 -> Eq. 8
+ *     xrl_policy_value           Section 3.3.2  policy / value MLPs, padded action space,
+ *                                Section 3.3.3  invalid-action masking, No-Op, sampling
+ *
+ * Conventions
+ *  - Plain C ABI.  Every function returns an xrl_status; nothing throws, aborts or traps.
+ *  - "host" / "device" on every pointer says where the memory lives.  The caller owns every
+ *    buffer it passes in; the library owns xrl_ctx and xrl_batch objects.
+ *  - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default stream)
+ *    and is asynchronous.  Argument errors are returned before anything is enqueued.  Errors
+ *    found by kernels (malformed graph ids, bad masks, bounded waits that ran out) are written
+ *    to a device status word; read it with xrl_last_device_status after the stream is synced.
+ *  - A context is bound to one device and is not thread-safe; distinct contexts are independent.
+ *  - There is no CPU fallback: without a CUDA device xrl_create fails with XRL_ERR_CUDA.
+ *
+ * Readings of what the paper leaves open: ReLU for every sigma; LeakyReLU(0.2) inside the
+ * attention score (the GAT paper's choice); neighbourhood = producers of the node plus the
+ * node itself; K heads of width H/K concatenated in every layer; a bias in every dense map;
+ * Eq. 8 carries a weight matrix W_g; the policy scores each graph with one shared MLP and the
+ * current graph's score is the No-Op logit.
+ */
+#ifndef XRL_H_
+#define XRL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t xrl_status;
+enum {
+  XRL_OK = 0,
+  XRL_ERR_INVALID_ARG = 1, /* null pointer, negative size, inconsistent offsets, bad mask  */
+  XRL_ERR_BAD_GRAPH = 2,   /* edge endpoint outside [0, num_nodes), self edge, op id >= T   */
+  XRL_ERR_CAPACITY = 3,    /* batch larger than the capacities given to xrl_create          */
+  XRL_ERR_ALLOC = 4,       /* host or device allocation failed                              */
+  XRL_ERR_CUDA = 5,        /* a CUDA runtime call failed (also: no device)                  */
+  XRL_ERR_STATE = 6,       /* weights not set, batch not packed, batch of another context   */
+  XRL_ERR_TIMEOUT = 7,     /* a bounded device-side wait ran out                            */
+  XRL_ERR_UNSUPPORTED = 8  /* model shape outside what the kernels are built for            */
+};
+
+enum { XRL_FP32 = 0, XRL_BF16 = 1 };      /* storage type of features / Eq. 6-7 weights      */
+enum { XRL_MEM_HOST = 0, XRL_MEM_DEVICE = 1 };
+
+/* Model and capacity description (plain data, copied by xrl_create).
+ * Supported shapes: hidden a multiple of 32 in [32, 512]; hidden / heads a multiple of 8;
+ * num_shape_feats = 8; num_op_types <= 256; mlp_hidden in [1, 1024]; global_dim in [0, 16]. */
+typedef struct {
+  int32_t num_op_types;    /* T: size of the operator table (one-hot node attribute)          */
+  int32_t num_shape_feats; /* S: shape features per node (attribute of its outgoing edges)    */
+  int32_t hidden;          /* H                                                               */
+  int32_t heads;           /* K, must divide H                                                */
+  int32_t layers;          /* L: number of graph-attention layers (the paper's k), >= 0       */
+  int32_t mlp_hidden;      /* Hm: hidden width of both two-layer MLP heads                    */
+  int32_t global_dim;      /* Dg: width of the per-graph global attribute (paper: value 0)    */
+  int32_t dtype;           /* XRL_FP32, or XRL_BF16 = bf16 storage with fp32 accumulation     */
+  int32_t max_actions;     /* A_max: padded number of candidate slots; No-Op is index A_max   */
+  int32_t max_graphs;      /* capacity: graphs per batch                                      */
+  int32_t max_envs;        /* capacity: environments per batch                                */
+  int64_t max_nodes;       /* capacity: total nodes per batch (< 2^31)                        */
+  int64_t max_edges;       /* capacity: total edges per batch (< 2^31)                        */
+} xrl_model_config;
+
+/* One computation graph: nodes are tensor operators, an edge (src -> dst) is a tensor produced
+ * by src and consumed by dst.  All pointers HOST, read-only to the library. */
+typedef struct {
+  int32_t num_nodes, num_edges;
+  const int32_t* op;       /* [num_nodes]      operator id in [0, T)                           */
+  const void* shape;       /* [num_nodes x S]  float (XRL_FP32) or bf16 bits (XRL_BF16)        */
+  const int32_t* edge_src; /* [num_edges]      producer, local id                              */
+  const int32_t* edge_dst; /* [num_edges]      consumer, local id; src != dst; repeats allowed */
+} xrl_graph;
+
+typedef struct xrl_ctx xrl_ctx;
+typedef struct xrl_batch xrl_batch;
+
+/* ---- context and weights -------------------------------------------------------------- */
+
+/* Create a context on CUDA device `device`: validates the config, allocates the activation
+ * workspace for the stated capacities (about 3 * max_nodes * H * sizeof(storage) bytes plus
+ * 8 * heads bytes per node).  *out is HOST.  Errors: INVALID_ARG, UNSUPPORTED, CUDA, ALLOC. */
+xrl_status xrl_create(const xrl_model_config* cfg, int32_t device, xrl_ctx** out);
+void xrl_destroy(xrl_ctx* ctx);
+
+/* Size in bytes of the flat fp32 weight blob.  Order (matrices row-major [in x out]):
+ *   W0 [(S+T+S) x H], b0 [H]                       Eq. 6; input = [edge aggregate | one-hot op | own shape]
+ *   per layer: W [H x H], a_src [H], a_dst [H], b [H]   Eq. 7; a_* are K per-head vectors of width H/K
+ *   Wg [(H+Dg) x H], bg [H]                        Eq. 8; input = [node sum | global attribute]
+ *   policy: W1 [H x Hm], b1 [Hm], w2 [Hm], b2 [1]
+ *   value:  W1 [2H x Hm], b1 [Hm], w2 [Hm], b2 [1]      input = [current graph | mean of valid candidates] */
+xrl_status xrl_weights_size(const xrl_ctx* ctx, size_t* bytes);
+/* Upload the blob (HOST, fp32).  With XRL_BF16 the library rounds W0 and the layer matrices W
+ * to bf16 (nearest even) once; everything else stays fp32.  Synchronous. */
+xrl_status xrl_set_weights(xrl_ctx* ctx, const void* host_blob, size_t bytes);
+
+/* ---- (1) packer: Section 3.3.2, "batch them into a meta-graph" -------------------------- */
+
+/* graphs[env_off[e]] is the CURRENT graph of environment e and graphs[env_off[e]+1 ..
+ * env_off[e+1]-1] are its candidates in action order.  env_off is HOST, [num_envs + 1],
+ * env_off[0] = 0, strictly increasing, env_off[num_envs] = num_graphs.
+ * The batch holds, on the device: node_off[B+1], edge_off[B+1] (exclusive prefix sums),
+ * seg_id[N] (node -> graph), graph_env[B], CSR by consumer rowptr[N+1] / col[E] over global
+ * node ids (inside a row the producers keep the order of the input edge list), op[N],
+ * shape[N x S].  If *out is NULL a batch sized to the context's capacities is allocated;
+ * otherwise the existing batch is re-packed in place with no allocation.
+ * Graph validity (ids in range, no self edge, op < T) is checked on the device: a violation
+ * sets XRL_ERR_BAD_GRAPH in the device status word and the batch must not be encoded. */
+xrl_status xrl_pack(xrl_ctx* ctx, const xrl_graph* graphs, int32_t num_graphs,
+                    const int32_t* env_off, int32_t num_envs, void* stream, xrl_batch** out);
+
+/* Same operation on already concatenated arrays.  n_nodes, n_edges [num_graphs] and env_off
+ * are always HOST; op [N], shape [N x S], edge_src [E], edge_dst [E] (local ids, graphs back
+ * to back) are HOST or DEVICE according to `where` (XRL_MEM_*).  DEVICE arrays are read by the
+ * kernels directly and must stay valid until the stream has passed the call. */
+xrl_status xrl_pack_flat(xrl_ctx* ctx, int32_t where, int32_t num_graphs, const int32_t* n_nodes,
+                         const int32_t* n_edges, const int32_t* op, const void* shape,
+                         const int32_t* edge_src, const int32_t* edge_dst, const int32_t* env_off,
+                         int32_t num_envs, void* stream, xrl_batch** out);
+
+xrl_status xrl_batch_free(xrl_ctx* ctx, xrl_batch* batch);
+/* All four outputs HOST. */
+xrl_status xrl_batch_info(const xrl_batch* batch, int64_t* num_nodes, int64_t* num_edges,
+                          int32_t* num_graphs, int32_t* num_envs);
+/* Copy the packed index arrays to HOST buffers (any may be NULL); synchronises the stream the
+ * batch was packed on.  Sizes: rowptr [N+1], col [E], seg_id [N], node_off [B+1],
+ * edge_off [B+1], graph_env [B]. */
+xrl_status xrl_batch_export(const xrl_batch* batch, int32_t* rowptr, int32_t* col, int32_t* seg_id,
+                            int32_t* node_off, int32_t* edge_off, int32_t* graph_env);
+
+/* ---- (2) encoder: Section 3.4 ------------------------------------------------------------ */
+
+/* Eq. 6:  h0_i = ReLU(W0^T [ sum_{j -> i} shape_j | onehot(op_i) | shape_i ] + b0)
+ * Eq. 7 (L times):  z = W^T h;  e_ij = LeakyReLU_0.2(a_src . z_j + a_dst . z_i) per head over
+ *         j in producers(i) + {i};  alpha = softmax_j e_ij;  h'_i = ReLU(sum_j alpha_ij z_j + b)
+ * Eq. 8:  emb_g = ReLU(Wg^T [ sum_{i in g} h_i | g0_g ] + bg)
+ * g0: DEVICE fp32 [B x Dg] or NULL (= 0, the paper's initial value).
+ * graph_emb: DEVICE fp32 [B x H], written by the call. */
+xrl_status xrl_encode(xrl_ctx* ctx, const xrl_batch* batch, const float* g0, float* graph_emb,
+                      void* stream);
+
+/* Debug aid for parity tests: run Eq. 6 and the first `num_layers` attention layers
+ * (0 <= num_layers <= L) and copy the node features to HOST fp32 [N x H].  Synchronous. */
+xrl_status xrl_debug_node_features(xrl_ctx* ctx, const xrl_batch* batch, int32_t num_layers,
+                                   float* host_out, void* stream);
+
+/* ---- (3) heads: Sections 3.3.2 and 3.3.3 -------------------------------------------------- */
+
+/* Per graph g: logit_g = w2 . ReLU(W1^T emb_g + b1) + b2 (policy MLP).  Per environment e with
+ * C candidates: action a < C is candidate a, action A_max is No-Op and takes the current graph's
+ * logit; probs = softmax over { a : mask[e][a] = 1 } + { No-Op }, every other entry exactly 0.
+ * value_e = value MLP of [ emb(current) | mean of emb over the valid candidates ] (zero vector
+ * if there is none).
+ *   graph_emb DEVICE fp32 [B x H]            (the output of xrl_encode)
+ *   mask      DEVICE u8  [num_envs x A_max]  1 = valid; a set bit at a >= C raises
+ *                                            XRL_ERR_INVALID_ARG in the device status word
+ *   probs     DEVICE fp32 [num_envs x (A_max+1)], last column = No-Op
+ *   value     DEVICE fp32 [num_envs]
+ *   action    DEVICE int32 [num_envs], or NULL for no sampling.  The draw uses Philox4x32-10
+ *             keyed by `seed` with counter (env, step lo, step hi, 0): r = word0 | word1 << 32;
+ *             q_a = floor(p_a * 2^32); t = floor(r * sum(q) / 2^64); action = first index whose
+ *             inclusive prefix sum of q exceeds t (No-Op if sum(q) = 0).  Integer-exact given
+ *             the fp32 probabilities. */
+xrl_status xrl_policy_value(xrl_ctx* ctx, const xrl_batch* batch, const float* graph_emb,
+                            const uint8_t* mask, float* probs, float* value, int32_t* action,
+                            uint64_t seed, uint64_t step, void* stream);
+
+/* The sampling step alone on caller-supplied probabilities: probs DEVICE fp32
+ * [num_envs x num_actions] -> action DEVICE int32 [num_envs]; same draw as above. */
+xrl_status xrl_sample(xrl_ctx* ctx, const float* probs, int32_t num_envs, int32_t num_actions,
+                      uint64_t seed, uint64_t step, int32_t* action, void* stream);
+
+/* Read and clear the device status word.  Synchronises `stream`.  *status (HOST) receives the
+ * first error code any kernel recorded since the last call, or XRL_OK. */
+xrl_status xrl_last_device_status(xrl_ctx* ctx, void* stream, int32_t* status);
+
+/* Names of the kernels launched by the last xrl_encode / xrl_policy_value / xrl_pack call on
+ * this context and how many launches each call made (HOST outputs, any may be NULL). */
+xrl_status xrl_launch_counts(const xrl_ctx* ctx, int64_t* pack, int64_t* encode, int64_t* heads);
+
+/* Static description of the build ("sm_100a ...").  Never NULL. */
+const char* xrl_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XRL_H_ */

@@ -1,0 +1,337 @@
+"""ctypes binding of libxrl.so: one Python function per C entry point, same names.
+
+Only argument marshalling happens here.  Device buffers are torch CUDA tensors (torch is used
+for device memory and streams, nothing else); every function takes raw pointers from them.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libxrl.so")
+_lib = None
+
+STATUS_NAMES = {0: "XRL_OK", 1: "XRL_ERR_INVALID_ARG", 2: "XRL_ERR_BAD_GRAPH", 3: "XRL_ERR_CAPACITY",
+                4: "XRL_ERR_ALLOC", 5: "XRL_ERR_CUDA", 6: "XRL_ERR_STATE", 7: "XRL_ERR_TIMEOUT",
+                8: "XRL_ERR_UNSUPPORTED"}
+XRL_FP32, XRL_BF16 = 0, 1
+XRL_MEM_HOST, XRL_MEM_DEVICE = 0, 1
+
+EXPORTED_SYMBOLS = [
+    "xrl_create", "xrl_destroy", "xrl_weights_size", "xrl_set_weights", "xrl_pack", "xrl_pack_flat",
+    "xrl_batch_free", "xrl_batch_info", "xrl_batch_export", "xrl_encode", "xrl_debug_node_features",
+    "xrl_policy_value", "xrl_sample", "xrl_last_device_status", "xrl_launch_counts", "xrl_version",
+]
+
+
+class XrlError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = int(status)
+        super().__init__(f"{where}: {STATUS_NAMES.get(int(status), status)}")
+
+
+class _ModelConfig(C.Structure):
+    _fields_ = [("num_op_types", C.c_int32), ("num_shape_feats", C.c_int32), ("hidden", C.c_int32),
+                ("heads", C.c_int32), ("layers", C.c_int32), ("mlp_hidden", C.c_int32),
+                ("global_dim", C.c_int32), ("dtype", C.c_int32), ("max_actions", C.c_int32),
+                ("max_graphs", C.c_int32), ("max_envs", C.c_int32), ("max_nodes", C.c_int64),
+                ("max_edges", C.c_int64)]
+
+
+class _Graph(C.Structure):
+    _fields_ = [("num_nodes", C.c_int32), ("num_edges", C.c_int32), ("op", C.c_void_p),
+                ("shape", C.c_void_p), ("edge_src", C.c_void_p), ("edge_dst", C.c_void_p)]
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Load libxrl.so.  Raises if it has not been built: there is no fallback path."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(f"{_LIB_PATH} is missing: build it with "
+                          "`python -m paper_2304_14698_b200.build` (needs nvcc)")
+    lib = C.CDLL(_LIB_PATH)
+    vp, i32, i64, u64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64
+    sigs = {
+        "xrl_create": [C.POINTER(_ModelConfig), i32, C.POINTER(vp)],
+        "xrl_destroy": [vp],
+        "xrl_weights_size": [vp, C.POINTER(C.c_size_t)],
+        "xrl_set_weights": [vp, vp, C.c_size_t],
+        "xrl_pack": [vp, C.POINTER(_Graph), i32, vp, i32, vp, C.POINTER(vp)],
+        "xrl_pack_flat": [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, i32, vp, C.POINTER(vp)],
+        "xrl_batch_free": [vp, vp],
+        "xrl_batch_info": [vp, C.POINTER(i64), C.POINTER(i64), C.POINTER(i32), C.POINTER(i32)],
+        "xrl_batch_export": [vp, vp, vp, vp, vp, vp, vp],
+        "xrl_encode": [vp, vp, vp, vp, vp],
+        "xrl_debug_node_features": [vp, vp, i32, vp, vp],
+        "xrl_policy_value": [vp, vp, vp, vp, vp, vp, vp, u64, u64, vp],
+        "xrl_sample": [vp, vp, i32, i32, u64, u64, vp, vp],
+        "xrl_last_device_status": [vp, vp, C.POINTER(i32)],
+        "xrl_launch_counts": [vp, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64)],
+    }
+    for name, args in sigs.items():
+        fn = getattr(lib, name)
+        fn.argtypes = args
+        fn.restype = None if name == "xrl_destroy" else C.c_int32
+    lib.xrl_version.restype = C.c_char_p
+    lib.xrl_version.argtypes = []
+    _lib = lib
+    return lib
+
+
+def _check(st, where):
+    if st != 0:
+        raise XrlError(st, where)
+
+
+def _np_ptr(a):
+    return None if a is None else C.c_void_p(a.ctypes.data)
+
+
+def _dev_ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    return C.c_void_p(int(stream))
+
+
+def model_config(m, max_graphs, max_envs, max_nodes, max_edges):
+    """Build the C config from a dict with keys T, S, H, K, L, Hm, Dg, dtype, A_max."""
+    return _ModelConfig(m["T"], m["S"], m["H"], m["K"], m["L"], m["Hm"], m["Dg"],
+                        XRL_BF16 if m["dtype"] in ("bf16", XRL_BF16) else XRL_FP32, m["A_max"],
+                        int(max_graphs), int(max_envs), int(max_nodes), int(max_edges))
+
+
+def to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """float32 -> bfloat16 bit patterns (uint16), round to nearest even."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) >> 16
+    return u.astype(np.uint16).reshape(x.shape)
+
+
+# ---- one function per C entry point ---------------------------------------------------------
+
+def xrl_version() -> str:
+    return load_library().xrl_version().decode()
+
+
+def xrl_create(cfg: _ModelConfig, device: int = 0):
+    out = C.c_void_p()
+    _check(load_library().xrl_create(C.byref(cfg), device, C.byref(out)), "xrl_create")
+    return out
+
+
+def xrl_destroy(ctx):
+    load_library().xrl_destroy(ctx)
+
+
+def xrl_weights_size(ctx) -> int:
+    n = C.c_size_t()
+    _check(load_library().xrl_weights_size(ctx, C.byref(n)), "xrl_weights_size")
+    return int(n.value)
+
+
+def xrl_set_weights(ctx, blob: np.ndarray):
+    blob = np.ascontiguousarray(blob, dtype=np.float32)
+    _check(load_library().xrl_set_weights(ctx, _np_ptr(blob), blob.nbytes), "xrl_set_weights")
+
+
+def xrl_pack(ctx, graphs, env_off, dtype, stream=None, batch=None):
+    """graphs: list of dicts (op int32[n], shape float32[n,S], edge_src, edge_dst) in HOST memory."""
+    keep = []
+    arr = (_Graph * max(1, len(graphs)))()
+    for i, g in enumerate(graphs):
+        op = np.ascontiguousarray(g["op"], dtype=np.int32)
+        shp = np.ascontiguousarray(g["shape"], dtype=np.float32)
+        if dtype in ("bf16", XRL_BF16):
+            shp = to_bf16_bits(shp)
+        es = np.ascontiguousarray(g["edge_src"], dtype=np.int32)
+        ed = np.ascontiguousarray(g["edge_dst"], dtype=np.int32)
+        keep += [op, shp, es, ed]
+        arr[i] = _Graph(len(op), len(es), op.ctypes.data, shp.ctypes.data, es.ctypes.data, ed.ctypes.data)
+    env_off = np.ascontiguousarray(env_off, dtype=np.int32)
+    out = C.c_void_p(batch.value if batch is not None else None)
+    st = load_library().xrl_pack(ctx, arr, len(graphs), _np_ptr(env_off), len(env_off) - 1,
+                                 _stream(stream), C.byref(out))
+    _check(st, "xrl_pack")
+    return out
+
+
+def xrl_pack_flat(ctx, where, n_nodes, n_edges, op, shape, edge_src, edge_dst, env_off, stream=None,
+                  batch=None):
+    """Counts and env_off: numpy int32 (HOST).  Bulk arrays: numpy (where = HOST) or torch CUDA
+    tensors (where = DEVICE); shape must already have the storage type (float32 or bf16)."""
+    n_nodes = np.ascontiguousarray(n_nodes, dtype=np.int32)
+    n_edges = np.ascontiguousarray(n_edges, dtype=np.int32)
+    env_off = np.ascontiguousarray(env_off, dtype=np.int32)
+    ptr = _np_ptr if where == XRL_MEM_HOST else _dev_ptr
+    out = C.c_void_p(batch.value if batch is not None else None)
+    st = load_library().xrl_pack_flat(ctx, where, len(n_nodes), _np_ptr(n_nodes), _np_ptr(n_edges),
+                                      ptr(op), ptr(shape), ptr(edge_src), ptr(edge_dst),
+                                      _np_ptr(env_off), len(env_off) - 1, _stream(stream), C.byref(out))
+    _check(st, "xrl_pack_flat")
+    return out
+
+
+def xrl_batch_free(ctx, batch):
+    _check(load_library().xrl_batch_free(ctx, batch), "xrl_batch_free")
+
+
+def xrl_batch_info(batch):
+    n, e, b, ne = C.c_int64(), C.c_int64(), C.c_int32(), C.c_int32()
+    _check(load_library().xrl_batch_info(batch, C.byref(n), C.byref(e), C.byref(b), C.byref(ne)),
+           "xrl_batch_info")
+    return {"num_nodes": n.value, "num_edges": e.value, "num_graphs": b.value, "num_envs": ne.value}
+
+
+def xrl_batch_export(batch):
+    info = xrl_batch_info(batch)
+    N, E, B = info["num_nodes"], info["num_edges"], info["num_graphs"]
+    out = {"rowptr": np.zeros(N + 1, np.int32), "col": np.zeros(E, np.int32),
+           "seg_id": np.zeros(N, np.int32), "node_off": np.zeros(B + 1, np.int32),
+           "edge_off": np.zeros(B + 1, np.int32), "graph_env": np.zeros(B, np.int32)}
+    st = load_library().xrl_batch_export(batch, _np_ptr(out["rowptr"]), _np_ptr(out["col"]),
+                                         _np_ptr(out["seg_id"]), _np_ptr(out["node_off"]),
+                                         _np_ptr(out["edge_off"]), _np_ptr(out["graph_env"]))
+    _check(st, "xrl_batch_export")
+    return out
+
+
+def xrl_encode(ctx, batch, graph_emb, g0=None, stream=None):
+    """graph_emb: torch CUDA float32 [B, H] (written).  g0: torch CUDA float32 [B, Dg] or None."""
+    _check(load_library().xrl_encode(ctx, batch, _dev_ptr(g0), _dev_ptr(graph_emb), _stream(stream)),
+           "xrl_encode")
+    return graph_emb
+
+
+def xrl_debug_node_features(ctx, batch, num_layers, hidden, stream=None):
+    info = xrl_batch_info(batch)
+    out = np.zeros((info["num_nodes"], hidden), np.float32)
+    _check(load_library().xrl_debug_node_features(ctx, batch, num_layers, _np_ptr(out), _stream(stream)),
+           "xrl_debug_node_features")
+    return out
+
+
+def xrl_policy_value(ctx, batch, graph_emb, mask, probs, value, action=None, seed=0, step=0,
+                     stream=None):
+    st = load_library().xrl_policy_value(ctx, batch, _dev_ptr(graph_emb), _dev_ptr(mask), _dev_ptr(probs),
+                                         _dev_ptr(value), _dev_ptr(action), seed, step, _stream(stream))
+    _check(st, "xrl_policy_value")
+    return probs, value, action
+
+
+def xrl_sample(ctx, probs, action, seed, step, stream=None):
+    ne, a1 = probs.shape
+    _check(load_library().xrl_sample(ctx, _dev_ptr(probs), ne, a1, seed, step, _dev_ptr(action),
+                                     _stream(stream)), "xrl_sample")
+    return action
+
+
+def xrl_last_device_status(ctx, stream=None) -> int:
+    s = C.c_int32()
+    _check(load_library().xrl_last_device_status(ctx, _stream(stream), C.byref(s)),
+           "xrl_last_device_status")
+    return int(s.value)
+
+
+def xrl_launch_counts(ctx):
+    a, b, c = C.c_int64(), C.c_int64(), C.c_int64()
+    _check(load_library().xrl_launch_counts(ctx, C.byref(a), C.byref(b), C.byref(c)), "xrl_launch_counts")
+    return {"pack": a.value, "encode": b.value, "heads": c.value}
+
+
+# ---- the call a user makes --------------------------------------------------------------------
+
+class Agent:
+    """One model on one GPU: set weights once, then `step()` per rewrite step.
+
+    m: dict with keys T, S, H, K, L, Hm, Dg, dtype, A_max.  Capacities bound the batch size.
+    """
+
+    def __init__(self, m, max_graphs, max_envs, max_nodes, max_edges, device=0):
+        import torch
+        self.torch = torch
+        self.m = dict(m)
+        self.device = torch.device("cuda", device)
+        torch.cuda.set_device(self.device)
+        self.cfg = model_config(m, max_graphs, max_envs, max_nodes, max_edges)
+        self.ctx = xrl_create(self.cfg, device)
+        self.batch = None
+        self._out = {}
+
+    def close(self):
+        if self.ctx is not None:
+            if self.batch is not None:
+                xrl_batch_free(self.ctx, self.batch)
+                self.batch = None
+            xrl_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_weights(self, blob):
+        xrl_set_weights(self.ctx, blob)
+
+    def _buffers(self, B, Ne):
+        t = self.torch
+        key = (B, Ne)
+        if key not in self._out:
+            self._out = {key: dict(
+                emb=t.empty((B, self.m["H"]), dtype=t.float32, device=self.device),
+                probs=t.empty((Ne, self.m["A_max"] + 1), dtype=t.float32, device=self.device),
+                value=t.empty((Ne,), dtype=t.float32, device=self.device),
+                action=t.empty((Ne,), dtype=t.int32, device=self.device))}
+        return self._out[key]
+
+    def storage_shape(self, shape_f32):
+        """Host float32 shape features -> the array xrl_pack_flat expects for this model's dtype."""
+        return to_bf16_bits(shape_f32) if self.m["dtype"] == "bf16" else \
+            np.ascontiguousarray(shape_f32, dtype=np.float32)
+
+    def pack(self, batch):
+        """batch: flat dict (n_nodes, n_edges, op, shape, edge_src, edge_dst, env_off); bulk arrays
+        either numpy (host) or torch CUDA tensors (device, shape already in storage type)."""
+        on_dev = not isinstance(batch["op"], np.ndarray)
+        shape = batch["shape"] if on_dev else self.storage_shape(batch["shape"])
+        self.batch = xrl_pack_flat(self.ctx, XRL_MEM_DEVICE if on_dev else XRL_MEM_HOST,
+                                   batch["n_nodes"], batch["n_edges"], batch["op"], shape,
+                                   batch["edge_src"], batch["edge_dst"], batch["env_off"],
+                                   batch=self.batch)
+        return self.batch
+
+    def pack_graphs(self, graphs, env_off):
+        self.batch = xrl_pack(self.ctx, graphs, env_off, self.m["dtype"], batch=self.batch)
+        return self.batch
+
+    def forward(self, mask, sample=False, seed=0, step=0, g0=None):
+        """Encode the packed batch and evaluate the heads.  mask: torch CUDA uint8 [envs, A_max]."""
+        info = xrl_batch_info(self.batch)
+        o = self._buffers(info["num_graphs"], info["num_envs"])
+        xrl_encode(self.ctx, self.batch, o["emb"], g0)
+        xrl_policy_value(self.ctx, self.batch, o["emb"], mask, o["probs"], o["value"],
+                         o["action"] if sample else None, seed, step)
+        return o
+
+    def step(self, batch, mask, sample=False, seed=0, step=0):
+        """The whole path for one batch: pack -> encode -> policy/value (-> sample)."""
+        self.pack(batch)
+        return self.forward(mask, sample, seed, step)
+
+    def device_status(self):
+        return xrl_last_device_status(self.ctx)

@@ -1,0 +1,374 @@
+// Per-graph readout and global update (paper Eq. 8), the policy and value heads with
+// invalid-action masking and No-Op (Sections 3.3.2, 3.3.3), and the categorical draw.
+// Every reduction runs in a fixed order (no floating-point atomics), so results are
+// reproducible run to run.
+#include "xrl_internal.cuh"
+
+namespace xrl {
+
+namespace {
+
+constexpr int kRoThreads = 256;
+
+// ---- readout, stage 1: column sums of one chunk of consecutive rows of one graph -------------
+template <typename T>
+__global__ void __launch_bounds__(kRoThreads)
+k_readout(const T* __restrict__ h, const int32_t* __restrict__ chunk_row0,
+          const int32_t* __restrict__ chunk_row1, int32_t chunk_begin, float* __restrict__ partial,
+          int H, int32_t win_base) {
+  constexpr int VEC = VecOf<T>::N;
+  extern __shared__ float red[];                 // [RG][H]
+  const int NV = H / VEC;
+  const int RG = kRoThreads / NV;                // row groups working in parallel
+  const int32_t chunk = chunk_begin + blockIdx.x;
+  const int32_t r0 = chunk_row0[chunk], r1 = chunk_row1[chunk];
+  const int vi = threadIdx.x % NV, rg = threadIdx.x / NV;
+  float acc[VEC];
+#pragma unroll
+  for (int t = 0; t < VEC; ++t) acc[t] = 0.f;
+  if (rg < RG) {
+    int32_t r = r0 + rg;
+    for (; r + 3 * RG < r1; r += 4 * RG) {
+      float f[4][VEC];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        load_vec(h + size_t(r + u * RG - win_base) * H + vi * VEC, f[u]);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int t = 0; t < VEC; ++t) acc[t] += f[u][t];
+    }
+    for (; r < r1; r += RG) {
+      float f[VEC];
+      load_vec(h + size_t(r - win_base) * H + vi * VEC, f);
+#pragma unroll
+      for (int t = 0; t < VEC; ++t) acc[t] += f[t];
+    }
+#pragma unroll
+    for (int t = 0; t < VEC; ++t) red[rg * H + vi * VEC + t] = acc[t];
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < H; c += kRoThreads) {
+    float s = 0.f;
+    for (int g = 0; g < RG; ++g) s += red[g * H + c];
+    partial[size_t(chunk) * H + c] = s;
+  }
+}
+
+// ---- Eq. 8: emb_g = ReLU(Wg^T [ sum of the graph's chunk sums | g0_g ] + bg) -------------------
+__global__ void __launch_bounds__(256)
+k_global_update(const float* __restrict__ partial, const int32_t* __restrict__ graph_chunk_off,
+                const float* __restrict__ g0, const float* __restrict__ Wg,
+                const float* __restrict__ bg, float* __restrict__ emb, int H, int Dg) {
+  extern __shared__ float u[];                   // [H + Dg]
+  const int32_t g = blockIdx.x;
+  const int32_t c0 = graph_chunk_off[g], c1 = graph_chunk_off[g + 1];
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    float s = 0.f;
+    for (int32_t ch = c0; ch < c1; ++ch) s += partial[size_t(ch) * H + c];
+    u[c] = s;
+  }
+  for (int t = threadIdx.x; t < Dg; t += blockDim.x) u[H + t] = g0 ? g0[size_t(g) * Dg + t] : 0.f;
+  __syncthreads();
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    float acc = bg[c];
+    for (int k = 0; k < H + Dg; ++k) acc = fmaf(u[k], __ldg(Wg + size_t(k) * H + c), acc);
+    emb[size_t(g) * H + c] = fmaxf(acc, 0.f);
+  }
+}
+
+// Block-wide sum in a fixed order: every thread contributes v, thread 0's tree is the same for
+// the same blockDim.  `scratch` holds blockDim.x floats.
+__device__ float block_sum(float v, float* scratch) {
+  scratch[threadIdx.x] = v;
+  __syncthreads();
+  for (int s = blockDim.x >> 1; s > 0; s >>= 1) {
+    if (int(threadIdx.x) < s) scratch[threadIdx.x] += scratch[threadIdx.x + s];
+    __syncthreads();
+  }
+  const float r = scratch[0];
+  __syncthreads();
+  return r;
+}
+
+// out = w2 . ReLU(W1^T x + b1) + b2 with x (length `in`) in shared memory; all threads return it.
+__device__ float mlp_scalar(const float* x, int in, int hid, const float* __restrict__ W1,
+                            const float* __restrict__ b1, const float* __restrict__ w2,
+                            const float* __restrict__ b2, float* scratch) {
+  float contrib = 0.f;
+  for (int c = threadIdx.x; c < hid; c += blockDim.x) {
+    float acc = b1[c];
+    for (int k = 0; k < in; ++k) acc = fmaf(x[k], __ldg(W1 + size_t(k) * hid + c), acc);
+    contrib += fmaxf(acc, 0.f) * w2[c];
+  }
+  return block_sum(contrib, scratch) + b2[0];
+}
+
+// ---- policy MLP: one scalar score per graph -----------------------------------------------------
+__global__ void __launch_bounds__(256)
+k_policy_logit(const float* __restrict__ emb, const float* __restrict__ W1, const float* __restrict__ b1,
+               const float* __restrict__ w2, const float* __restrict__ b2, float* __restrict__ logit,
+               int H, int Hm) {
+  extern __shared__ float sm[];                  // [H] + [blockDim]
+  float* x = sm;
+  float* scratch = sm + H;
+  const int32_t g = blockIdx.x;
+  for (int c = threadIdx.x; c < H; c += blockDim.x) x[c] = emb[size_t(g) * H + c];
+  __syncthreads();
+  const float v = mlp_scalar(x, H, Hm, W1, b1, w2, b2, scratch);
+  if (threadIdx.x == 0) logit[g] = v;
+}
+
+// ---- Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) -----------------------------------------
+struct U4 { uint32_t x, y, z, w; };
+__device__ U4 philox4x32_10(uint32_t k0, uint32_t k1, U4 c) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t lo0 = 0xD2511F53u * c.x, hi0 = __umulhi(0xD2511F53u, c.x);
+    const uint32_t lo1 = 0xCD9E8D57u * c.z, hi1 = __umulhi(0xCD9E8D57u, c.z);
+    c = U4{hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0};
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return c;
+}
+
+__device__ unsigned long long block_sum_u64(unsigned long long v, unsigned long long* scratch) {
+  scratch[threadIdx.x] = v;
+  __syncthreads();
+  for (int s = blockDim.x >> 1; s > 0; s >>= 1) {
+    if (int(threadIdx.x) < s) scratch[threadIdx.x] += scratch[threadIdx.x + s];
+    __syncthreads();
+  }
+  const unsigned long long r = scratch[0];
+  __syncthreads();
+  return r;
+}
+
+// Categorical draw from fp32 probabilities p[0..A1) with integer arithmetic only.
+// scratch: blockDim.x + 1 unsigned 64-bit words.  Every thread returns the action.
+__device__ int32_t sample_row(const float* __restrict__ p, int A1, uint64_t seed, uint64_t step,
+                              uint32_t env, unsigned long long* scratch) {
+  const int tid = threadIdx.x, nt = blockDim.x;
+  // contiguous slice per thread so that prefix order = index order
+  const int per = (A1 + nt - 1) / nt;
+  const int a0 = min(A1, tid * per), a1 = min(A1, a0 + per);
+  unsigned long long mine = 0;
+  for (int a = a0; a < a1; ++a) mine += (unsigned long long)floorf(p[a] * 4294967296.0f);
+  const unsigned long long Q = block_sum_u64(mine, scratch);
+  if (Q == 0) return A1 - 1;
+  const U4 r = philox4x32_10(uint32_t(seed), uint32_t(seed >> 32),
+                             U4{env, uint32_t(step), uint32_t(step >> 32), 0u});
+  const unsigned long long r64 = (unsigned long long)r.x | ((unsigned long long)r.y << 32);
+  const unsigned long long t = __umul64hi(r64, Q);
+  // exclusive prefix of the per-thread totals (serial over threads by thread 0: nt <= 1024)
+  scratch[tid] = mine;
+  __syncthreads();
+  if (tid == 0) {
+    unsigned long long run = 0;
+    for (int i = 0; i < nt; ++i) { const unsigned long long v = scratch[i]; scratch[i] = run; run += v; }
+    scratch[nt] = (unsigned long long)(A1 - 1);
+  }
+  __syncthreads();
+  unsigned long long run = scratch[tid];
+  if (run <= t && t < run + mine) {              // exactly one thread owns t
+    for (int a = a0; a < a1; ++a) {
+      run += (unsigned long long)floorf(p[a] * 4294967296.0f);
+      if (run > t) { scratch[nt] = (unsigned long long)a; break; }
+    }
+  }
+  __syncthreads();
+  const int32_t act = int32_t(scratch[nt]);
+  __syncthreads();
+  return act;
+}
+
+// ---- per environment: masked softmax, candidate mean, value MLP, optional draw -----------------
+__global__ void __launch_bounds__(1024)
+k_env_policy(const float* __restrict__ emb, const float* __restrict__ logit,
+             const int32_t* __restrict__ env_off, const uint8_t* __restrict__ mask,
+             const float* __restrict__ vW1, const float* __restrict__ vb1,
+             const float* __restrict__ vw2, const float* __restrict__ vb2, float* __restrict__ probs,
+             float* __restrict__ value, int32_t* __restrict__ action, int H, int Hm, int A,
+             uint64_t seed, uint64_t step, int32_t* status) {
+  extern __shared__ unsigned long long sm64[];   // [nt + 1] u64, then floats
+  const int nt = blockDim.x, tid = threadIdx.x;
+  float* scratch = reinterpret_cast<float*>(sm64 + nt + 1);   // [nt]
+  float* u = scratch + nt;                                    // [2H]
+  float* part = u + 2 * H;                                    // [parts][H]
+  const int32_t e = blockIdx.x;
+  const int32_t cur = env_off[e];
+  const int32_t C = env_off[e + 1] - cur - 1;
+  const uint8_t* mk = mask + size_t(e) * A;
+  float* pr = probs + size_t(e) * (A + 1);
+
+  // masked softmax over the valid candidates and No-Op (index A, scored by the current graph)
+  float mx = -INFINITY;
+  for (int a = tid; a <= A; a += nt) {
+    bool valid = (a == A);
+    if (a < A && mk[a]) {
+      if (a >= C) raise(status, XRL_ERR_INVALID_ARG); else valid = true;
+    }
+    if (valid) mx = fmaxf(mx, logit[a == A ? cur : cur + 1 + a]);
+  }
+  scratch[tid] = mx;
+  __syncthreads();
+  for (int s = nt >> 1; s > 0; s >>= 1) {
+    if (tid < s) scratch[tid] = fmaxf(scratch[tid], scratch[tid + s]);
+    __syncthreads();
+  }
+  mx = scratch[0];
+  __syncthreads();
+  float se = 0.f;
+  for (int a = tid; a <= A; a += nt) {
+    const bool valid = (a == A) || (a < C && mk[a]);
+    const float ex = valid ? expf(logit[a == A ? cur : cur + 1 + a] - mx) : 0.f;
+    pr[a] = ex;
+    se += ex;
+  }
+  const float denom = block_sum(se, scratch);
+  for (int a = tid; a <= A; a += nt) pr[a] = pr[a] / denom;     // each thread rewrites its own entries
+
+  // value head input: [ emb(current) | mean of emb over the valid candidates ]
+  const int parts = nt / H > 0 ? nt / H : 1;
+  for (int c = tid; c < H; c += nt) u[c] = emb[size_t(cur) * H + c];
+  if (tid < parts * H) {
+    const int c = tid % H, p = tid / H;
+    float s = 0.f;
+    for (int a = p; a < C; a += parts)
+      if (mk[a]) s += emb[size_t(cur + 1 + a) * H + c];
+    part[p * H + c] = s;
+  }
+  float cnt = 0.f;
+  for (int a = tid; a < C; a += nt) cnt += mk[a] ? 1.f : 0.f;
+  const float nv = block_sum(cnt, scratch);      // also orders the writes to part[] before the reads
+  if (nt < H) {                                   // fewer threads than columns: plain loop
+    for (int c = tid; c < H; c += nt) {
+      float s = 0.f;
+      for (int a = 0; a < C; ++a)
+        if (mk[a]) s += emb[size_t(cur + 1 + a) * H + c];
+      u[H + c] = nv > 0.f ? s / nv : 0.f;
+    }
+  } else if (tid < H) {
+    float s = 0.f;
+    for (int p = 0; p < parts; ++p) s += part[p * H + tid];
+    u[H + tid] = nv > 0.f ? s / nv : 0.f;
+  }
+  __syncthreads();
+  const float v = mlp_scalar(u, 2 * H, Hm, vW1, vb1, vw2, vb2, scratch);
+  if (tid == 0) value[e] = v;
+
+  if (action != nullptr) {
+    __syncthreads();                              // probs of this row are written by this block
+    const int32_t act = sample_row(pr, A + 1, seed, step, uint32_t(e), sm64);
+    if (tid == 0) action[e] = act;
+  }
+}
+
+__global__ void __launch_bounds__(1024)
+k_sample(const float* __restrict__ probs, int A1, uint64_t seed, uint64_t step,
+         int32_t* __restrict__ action) {
+  extern __shared__ unsigned long long sm64[];
+  const int32_t e = blockIdx.x;
+  const int32_t act = sample_row(probs + size_t(e) * A1, A1, seed, step, uint32_t(e), sm64);
+  if (threadIdx.x == 0) action[e] = act;
+}
+
+__global__ void k_to_float_bf16(const bf16* __restrict__ src, float* __restrict__ dst, int64_t n) {
+  const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = __bfloat162float(src[i]);
+}
+
+// dst = storage-type copy of src [rows x cols]; dst_t (optional) = its transpose [cols x rows]
+template <typename T>
+__global__ void k_round_weights(const float* __restrict__ src, T* __restrict__ dst,
+                                T* __restrict__ dst_t, int rows, int cols) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= rows * cols) return;
+  const int r = i / cols, c = i - r * cols;
+  const T v = T(src[i]);
+  dst[i] = v;
+  if (dst_t != nullptr) dst_t[size_t(c) * rows + r] = v;
+}
+
+int pow2_threads(int want) {          // power of two in [32, 1024] (block_sum needs a power of two)
+  int t = 32;
+  while (t < want && t < 1024) t <<= 1;
+  return t;
+}
+
+}  // namespace
+
+int launch_readout(const Dims& d, const void* h, const int32_t* chunk_row0, const int32_t* chunk_row1,
+                   int32_t chunk_begin, int32_t chunk_end, float* partial, int32_t win_base,
+                   cudaStream_t st) {
+  const int n = chunk_end - chunk_begin;
+  if (n <= 0) return 0;
+  if (d.dtype == XRL_BF16) {
+    const int RG = kRoThreads / (d.H / 8);
+    k_readout<bf16><<<n, kRoThreads, sizeof(float) * size_t(RG) * d.H, st>>>(
+        static_cast<const bf16*>(h), chunk_row0, chunk_row1, chunk_begin, partial, d.H, win_base);
+  } else {
+    const int RG = kRoThreads / (d.H / 4);
+    k_readout<float><<<n, kRoThreads, sizeof(float) * size_t(RG) * d.H, st>>>(
+        static_cast<const float*>(h), chunk_row0, chunk_row1, chunk_begin, partial, d.H, win_base);
+  }
+  return 1;
+}
+
+int launch_global_update(const Dims& d, const float* partial, const int32_t* graph_chunk_off,
+                         const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st) {
+  if (B <= 0) return 0;
+  k_global_update<<<B, 256, sizeof(float) * size_t(d.H + d.Dg), st>>>(partial, graph_chunk_off, g0,
+                                                                      w.Wg, w.bg, emb, d.H, d.Dg);
+  return 1;
+}
+
+int launch_heads(const Dims& d, const DevWeights& w, const float* emb, const int32_t* env_off,
+                 const uint8_t* mask, int32_t B, int32_t num_envs, float* logit_ws, float* probs,
+                 float* value, int32_t* action, uint64_t seed, uint64_t step, int32_t* status,
+                 cudaStream_t st) {
+  if (B <= 0 || num_envs <= 0) return 0;
+  k_policy_logit<<<B, 256, sizeof(float) * size_t(d.H + 256), st>>>(emb, w.pW1, w.pb1, w.pw2, w.pb2,
+                                                                    logit_ws, d.H, d.Hm);
+  const int nt = pow2_threads(d.H > d.A + 1 ? d.H : d.A + 1);
+  const int parts = nt / d.H > 0 ? nt / d.H : 1;
+  const size_t smem = sizeof(unsigned long long) * size_t(nt + 1) +
+                      sizeof(float) * size_t(nt + 2 * d.H + parts * d.H);
+  k_env_policy<<<num_envs, nt, smem, st>>>(emb, logit_ws, env_off, mask, w.vW1, w.vb1, w.vw2, w.vb2,
+                                           probs, value, action, d.H, d.Hm, d.A, seed, step, status);
+  return 2;
+}
+
+int launch_sample(const float* probs, int32_t num_envs, int32_t A1, uint64_t seed, uint64_t step,
+                  int32_t* action, cudaStream_t st) {
+  if (num_envs <= 0) return 0;
+  const int nt = pow2_threads(A1);
+  k_sample<<<num_envs, nt, sizeof(unsigned long long) * size_t(nt + 1), st>>>(probs, A1, seed, step,
+                                                                              action);
+  return 1;
+}
+
+int launch_to_float(const void* src, int dtype, float* dst, int64_t n, cudaStream_t st) {
+  if (n <= 0) return 0;
+  if (dtype == XRL_BF16) {
+    k_to_float_bf16<<<unsigned((n + 255) / 256), 256, 0, st>>>(static_cast<const bf16*>(src), dst, n);
+    return 1;
+  }
+  cudaMemcpyAsync(dst, src, sizeof(float) * size_t(n), cudaMemcpyDeviceToDevice, st);
+  return 0;
+}
+
+int launch_round_weights(const float* src, void* dst, void* dst_t, int rows, int cols, int dtype,
+                         cudaStream_t st) {
+  const int n = rows * cols;
+  if (dtype == XRL_BF16)
+    k_round_weights<bf16><<<(n + 255) / 256, 256, 0, st>>>(src, static_cast<bf16*>(dst),
+                                                          static_cast<bf16*>(dst_t), rows, cols);
+  else
+    k_round_weights<float><<<(n + 255) / 256, 256, 0, st>>>(src, static_cast<float*>(dst),
+                                                           static_cast<float*>(dst_t), rows, cols);
+  return 1;
+}
+
+}  // namespace xrl

@@ -1,0 +1,238 @@
+// Meta-graph packer (paper Section 3.3.2: the current graph and its candidates are batched
+// into one graph).  Integer-only, deterministic: exclusive scans for the per-graph offsets,
+// segment ids, in-degree count, and a CSR-by-consumer fill that keeps, inside every row, the
+// order of the input edge list.
+#include "xrl_internal.cuh"
+
+namespace xrl {
+
+namespace {
+
+constexpr int kScanThreads = 256;
+constexpr int kScanItems = 8;                       // per thread
+constexpr int kScanTile = kScanThreads * kScanItems;
+
+// Exclusive scan of one tile; in[i] is taken as 0 for i >= n_in; writes out[i] for i < n_out.
+// If block_sums != nullptr the tile total goes there.
+__global__ void __launch_bounds__(kScanThreads)
+k_scan_tile(const int32_t* __restrict__ in, int32_t* __restrict__ out, int32_t n_in, int32_t n_out,
+            int32_t* __restrict__ block_sums) {
+  __shared__ int32_t warp_tot[kScanThreads / 32];
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int64_t base = int64_t(blockIdx.x) * kScanTile + int64_t(tid) * kScanItems;
+  int32_t v[kScanItems];
+  int32_t sum = 0;
+#pragma unroll
+  for (int t = 0; t < kScanItems; ++t) {
+    const int64_t i = base + t;
+    v[t] = (i < n_in) ? in[i] : 0;
+    sum += v[t];
+  }
+  int32_t incl = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) warp_tot[wid] = incl;
+  __syncthreads();
+  int32_t warp_base = 0, total = 0;
+#pragma unroll
+  for (int w = 0; w < kScanThreads / 32; ++w) {
+    if (w < wid) warp_base += warp_tot[w];
+    total += warp_tot[w];
+  }
+  int32_t run = warp_base + incl - sum;
+#pragma unroll
+  for (int t = 0; t < kScanItems; ++t) {
+    const int64_t i = base + t;
+    if (i < n_out) out[i] = run;
+    run += v[t];
+  }
+  if (block_sums != nullptr && tid == 0) block_sums[blockIdx.x] = total;
+}
+
+__global__ void __launch_bounds__(kScanThreads)
+k_scan_add(int32_t* __restrict__ out, int32_t n_out, const int32_t* __restrict__ block_offsets) {
+  const int32_t add = block_offsets[blockIdx.x];
+  const int64_t base = int64_t(blockIdx.x) * kScanTile + int64_t(threadIdx.x) * kScanItems;
+#pragma unroll
+  for (int t = 0; t < kScanItems; ++t)
+    if (base + t < n_out) out[base + t] += add;
+}
+
+int num_tiles(int64_t n) { return int((n + kScanTile - 1) / kScanTile); }
+
+// out[0..n_in] = exclusive scan of in[0..n_in) (n_in + 1 outputs, the last is the total).
+// ws holds the per-tile sums of every level.
+int exclusive_scan(const int32_t* in, int32_t* out, int32_t n_in, int32_t* ws, cudaStream_t st) {
+  const int32_t n_out = n_in + 1;
+  const int tiles = num_tiles(n_out);
+  int launches = 0;
+  if (tiles == 1) {
+    k_scan_tile<<<1, kScanThreads, 0, st>>>(in, out, n_in, n_out, nullptr);
+    return 1;
+  }
+  int32_t* sums = ws;
+  int32_t* sums_scanned = ws + tiles;
+  k_scan_tile<<<tiles, kScanThreads, 0, st>>>(in, out, n_in, n_out, sums);
+  ++launches;
+  // scan of the tile sums (tiles outputs are enough; the recursion writes tiles + 1)
+  launches += exclusive_scan(sums, sums_scanned, tiles, ws + 2 * tiles + 2, st);
+  k_scan_add<<<tiles, kScanThreads, 0, st>>>(out, n_out, sums_scanned);
+  return launches + 1;
+}
+
+__device__ __forceinline__ int32_t upper_segment(const int32_t* __restrict__ off, int32_t n_seg,
+                                                 int32_t x) {
+  // largest g in [0, n_seg) with off[g] <= x  (off is non-decreasing, off[0] = 0)
+  int32_t lo = 0, hi = n_seg;
+  while (hi - lo > 1) {
+    const int32_t mid = (lo + hi) >> 1;
+    if (__ldg(off + mid) <= x) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+__global__ void k_node_segments(const int32_t* __restrict__ node_off, int32_t B, int32_t N,
+                                const int32_t* __restrict__ op, int32_t T,
+                                int32_t* __restrict__ seg_id, int32_t* __restrict__ deg,
+                                int32_t* status) {
+  const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= N) return;
+  seg_id[i] = upper_segment(node_off, B, i);
+  deg[i] = 0;
+  const int32_t o = op[i];
+  if (o < 0 || o >= T) raise(status, XRL_ERR_BAD_GRAPH);
+}
+
+__global__ void k_graph_envs(const int32_t* __restrict__ env_off, int32_t num_envs, int32_t B,
+                             int32_t* __restrict__ graph_env) {
+  const int32_t g = blockIdx.x * blockDim.x + threadIdx.x;
+  if (g < B) graph_env[g] = upper_segment(env_off, num_envs, g);
+}
+
+// One thread per edge: validate, count the consumer's in-degree.
+__global__ void k_edge_count(const int32_t* __restrict__ edge_src, const int32_t* __restrict__ edge_dst,
+                             const int32_t* __restrict__ edge_off, const int32_t* __restrict__ node_off,
+                             int32_t B, int32_t E, int32_t* __restrict__ deg, int32_t* status) {
+  const int32_t e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= E) return;
+  const int32_t g = upper_segment(edge_off, B, e);
+  const int32_t n = node_off[g + 1] - node_off[g];
+  const int32_t s = edge_src[e], t = edge_dst[e];
+  if (s < 0 || s >= n || t < 0 || t >= n || s == t) { raise(status, XRL_ERR_BAD_GRAPH); return; }
+  atomicAdd(&deg[node_off[g] + t], 1);
+}
+
+// One thread per edge: drop the edge id into some slot of its consumer's row (order fixed later).
+__global__ void k_edge_scatter(const int32_t* __restrict__ edge_src, const int32_t* __restrict__ edge_dst,
+                               const int32_t* __restrict__ edge_off, const int32_t* __restrict__ node_off,
+                               const int32_t* __restrict__ rowptr, int32_t B, int32_t E,
+                               int32_t* __restrict__ cursor, int32_t* __restrict__ tmp_eid) {
+  const int32_t e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= E) return;
+  const int32_t g = upper_segment(edge_off, B, e);
+  const int32_t n = node_off[g + 1] - node_off[g];
+  const int32_t s = edge_src[e], t = edge_dst[e];
+  if (s < 0 || s >= n || t < 0 || t >= n || s == t) return;
+  const int32_t row = node_off[g] + t;
+  const int32_t slot = atomicAdd(&cursor[row], 1);
+  tmp_eid[rowptr[row] + slot] = e;
+}
+
+constexpr int kShortRow = 32;
+
+// One thread per row: place each edge at its rank among the row's edge ids, which restores
+// the input order whatever order the atomics handed the slots out in.
+__global__ void k_row_order(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ tmp_eid,
+                            const int32_t* __restrict__ edge_src, const int32_t* __restrict__ seg_id,
+                            const int32_t* __restrict__ node_off, int32_t N, int32_t* __restrict__ col,
+                            int32_t* __restrict__ long_rows, int32_t* __restrict__ long_count) {
+  const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= N) return;
+  const int32_t b = rowptr[i], n = rowptr[i + 1] - b;
+  if (n == 0) return;
+  if (n > kShortRow) { long_rows[atomicAdd(long_count, 1)] = i; return; }
+  const int32_t base = node_off[seg_id[i]];
+  for (int32_t a = 0; a < n; ++a) {
+    const int32_t ea = tmp_eid[b + a];
+    int32_t rank = 0;
+    for (int32_t c = 0; c < n; ++c) rank += (tmp_eid[b + c] < ea) ? 1 : 0;
+    col[b + rank] = base + edge_src[ea];
+  }
+}
+
+// Rows longer than kShortRow: one warp per row, the same rank computation spread over lanes.
+__global__ void __launch_bounds__(256)
+k_row_order_long(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ tmp_eid,
+                 const int32_t* __restrict__ edge_src, const int32_t* __restrict__ seg_id,
+                 const int32_t* __restrict__ node_off, int32_t* __restrict__ col,
+                 const int32_t* __restrict__ long_rows, const int32_t* __restrict__ long_count) {
+  const int lane = threadIdx.x & 31;
+  const int32_t warps = (gridDim.x * blockDim.x) >> 5;
+  const int32_t count = *long_count;
+  for (int32_t w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < count; w += warps) {
+    const int32_t i = long_rows[w];
+    const int32_t b = rowptr[i], n = rowptr[i + 1] - b;
+    const int32_t base = node_off[seg_id[i]];
+    for (int32_t a = lane; a < n; a += 32) {
+      const int32_t ea = tmp_eid[b + a];
+      int32_t rank = 0;
+      for (int32_t c = 0; c < n; ++c) rank += (tmp_eid[b + c] < ea) ? 1 : 0;
+      col[b + rank] = base + edge_src[ea];
+    }
+  }
+}
+
+}  // namespace
+
+size_t scan_workspace_ints(int64_t n) {
+  size_t total = 0;
+  int64_t m = n + 1;
+  while (true) {
+    const int64_t tiles = (m + kScanTile - 1) / kScanTile;
+    if (tiles <= 1) break;
+    total += size_t(2 * tiles + 2);
+    m = tiles + 1;
+  }
+  return total + 16;
+}
+
+int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cudaStream_t st) {
+  int launches = 0;
+  const int TB = 256;
+  launches += exclusive_scan(in.n_nodes, out.node_off, in.B, out.scan_ws, st);
+  launches += exclusive_scan(in.n_edges, out.edge_off, in.B, out.scan_ws, st);
+  if (in.B > 0) {
+    k_graph_envs<<<(in.B + TB - 1) / TB, TB, 0, st>>>(in.env_off, in.num_envs, in.B, out.graph_env);
+    ++launches;
+  }
+  if (in.N > 0) {
+    k_node_segments<<<(in.N + TB - 1) / TB, TB, 0, st>>>(out.node_off, in.B, in.N, in.op, T,
+                                                          out.seg_id, out.deg, status);
+    ++launches;
+  }
+  if (in.E > 0) {
+    k_edge_count<<<(in.E + TB - 1) / TB, TB, 0, st>>>(in.edge_src, in.edge_dst, out.edge_off,
+                                                       out.node_off, in.B, in.E, out.deg, status);
+    ++launches;
+  }
+  launches += exclusive_scan(out.deg, out.rowptr, in.N, out.scan_ws, st);
+  if (in.E > 0 && in.N > 0) {
+    cudaMemsetAsync(out.deg, 0, sizeof(int32_t) * size_t(in.N), st);      // reused as the row cursors
+    cudaMemsetAsync(out.long_count, 0, sizeof(int32_t), st);
+    k_edge_scatter<<<(in.E + TB - 1) / TB, TB, 0, st>>>(in.edge_src, in.edge_dst, out.edge_off,
+                                                         out.node_off, out.rowptr, in.B, in.E,
+                                                         out.deg, out.tmp_eid);
+    k_row_order<<<(in.N + TB - 1) / TB, TB, 0, st>>>(out.rowptr, out.tmp_eid, in.edge_src, out.seg_id,
+                                                      out.node_off, in.N, out.col, out.long_rows,
+                                                      out.long_count);
+    k_row_order_long<<<kNumSMs, 256, 0, st>>>(out.rowptr, out.tmp_eid, in.edge_src, out.seg_id,
+                                              out.node_off, out.col, out.long_rows, out.long_count);
+    launches += 3;
+  }
+  return launches;
+}
+
+}  // namespace xrl

@@ -1,0 +1,309 @@
+// Row-wise kernels of the encoder (paper Section 3.4): the node-update layer (Eq. 6), the
+// attention half-scores, and the edge-score / segment-softmax / weighted-aggregate step of a
+// graph-attention layer (Eq. 7).  One group of LPR lanes owns one destination row and moves it
+// as 16-byte vectors (VPL vectors per lane); 32 / LPR rows share a warp.
+#include "xrl_internal.cuh"
+
+namespace xrl {
+
+namespace {
+
+constexpr int kRowThreads = 256;
+
+__device__ __forceinline__ float leaky(float x) { return x > 0.f ? x : 0.2f * x; }
+
+// 8 shape features of one node as floats (all lanes of a group read the same address).
+__device__ __forceinline__ void load_shape(const float* shape, int32_t node, float (&f)[kS]) {
+  const float4 a = __ldg(reinterpret_cast<const float4*>(shape + size_t(node) * kS));
+  const float4 b = __ldg(reinterpret_cast<const float4*>(shape + size_t(node) * kS) + 1);
+  f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+}
+__device__ __forceinline__ void load_shape(const bf16* shape, int32_t node, float (&f)[kS]) {
+  unpack(__ldg(reinterpret_cast<const uint4*>(shape + size_t(node) * kS)), f);
+}
+
+// ---- Eq. 6: h0_i = ReLU(W0^T [ sum_{j->i} shape_j | onehot(op_i) | shape_i ] + b0) -----------
+// The one-hot block of the product is a row lookup of W0; the two shape blocks are a 16 x H
+// dense map kept in shared memory as fp32.
+template <typename T, int LPR, int VPL>
+__global__ void __launch_bounds__(kRowThreads)
+k_embed(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+        const int32_t* __restrict__ op, const T* __restrict__ shape, const T* __restrict__ W0,
+        const float* __restrict__ b0, T* __restrict__ h, int H, int Tn, Window win) {
+  constexpr int VEC = VecOf<T>::N;
+  constexpr int RPW = 32 / LPR;
+  extern __shared__ float smem[];
+  float* Wd = smem;                    // [2*kS][H]
+  float* bs = smem + 2 * kS * H;       // [H]
+  for (int t = threadIdx.x; t < 2 * kS * H; t += blockDim.x) {
+    const int s = t / H, c = t - s * H;
+    const int src_row = (s < kS) ? s : (kS + Tn + (s - kS));
+    Wd[t] = to_float(W0[size_t(src_row) * H + c]);
+  }
+  for (int t = threadIdx.x; t < H; t += blockDim.x) bs[t] = b0[t];
+  __syncthreads();
+
+  const int NV = H / VEC;
+  const int lane = threadIdx.x & 31, sub = lane / LPR, sl = lane % LPR;
+  const int warps_total = (gridDim.x * blockDim.x) >> 5;
+  const int warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * RPW; r0 < win.row_end;
+       r0 += int64_t(warps_total) * RPW) {
+    const int32_t row = int32_t(r0) + sub;
+    if (row >= win.row_end) continue;
+    float x[2 * kS];
+#pragma unroll
+    for (int s = 0; s < kS; ++s) x[s] = 0.f;
+    const int32_t e0 = __ldg(rowptr + row), e1 = __ldg(rowptr + row + 1);
+    for (int32_t e = e0; e < e1; ++e) {
+      float f[kS];
+      load_shape(shape, __ldg(col + e), f);
+#pragma unroll
+      for (int s = 0; s < kS; ++s) x[s] += f[s];
+    }
+    {
+      float f[kS];
+      load_shape(shape, row, f);
+#pragma unroll
+      for (int s = 0; s < kS; ++s) x[kS + s] = f[s];
+    }
+    const T* lookup = W0 + size_t(kS + __ldg(op + row)) * H;
+    T* out = h + size_t(row - win.win_base) * H;
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+      const int vi = v * LPR + sl;
+      if (vi < NV) {
+        const int c0 = vi * VEC;
+        float acc[VEC];
+        load_vec(lookup + c0, acc);
+#pragma unroll
+        for (int t = 0; t < VEC; ++t) acc[t] += bs[c0 + t];
+#pragma unroll
+        for (int s = 0; s < 2 * kS; ++s)
+#pragma unroll
+          for (int t = 0; t < VEC; ++t) acc[t] = fmaf(x[s], Wd[s * H + c0 + t], acc[t]);
+#pragma unroll
+        for (int t = 0; t < VEC; ++t) acc[t] = fmaxf(acc[t], 0.f);
+        store_vec(out + c0, acc);
+      }
+    }
+  }
+}
+
+// ---- attention half-scores from Z (used when the transform kernel does not emit them) ------
+// s_src[i,k] = a_src[k] . Z[i, head k],  s_dst[i,k] = a_dst[k] . Z[i, head k]
+template <typename T, int LPR, int VPL>
+__global__ void __launch_bounds__(kRowThreads)
+k_scores(const T* __restrict__ Z, const float* __restrict__ a_src, const float* __restrict__ a_dst,
+         float* __restrict__ s_src, float* __restrict__ s_dst, int H, int K, Window win) {
+  constexpr int VEC = VecOf<T>::N;
+  constexpr int RPW = 32 / LPR;
+  constexpr int WARPS = kRowThreads / 32;
+  __shared__ float part[WARPS][RPW][LPR * VPL][2];
+  const int NV = H / VEC, d = H / K, vec_per_head = d / VEC;
+  const int lane = threadIdx.x & 31, sub = lane / LPR, sl = lane % LPR, wib = threadIdx.x >> 5;
+  const int warps_total = (gridDim.x * blockDim.x) >> 5;
+  const int warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * RPW; r0 < win.row_end;
+       r0 += int64_t(warps_total) * RPW) {
+    const int32_t row = int32_t(r0) + sub;
+    const bool live = row < win.row_end;
+    if (live) {
+      const T* z = Z + size_t(row - win.win_base) * H;
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) {
+        const int vi = v * LPR + sl;
+        if (vi < NV) {
+          float f[VEC];
+          load_vec(z + vi * VEC, f);
+          float ps = 0.f, pd = 0.f;
+#pragma unroll
+          for (int t = 0; t < VEC; ++t) {
+            ps = fmaf(f[t], __ldg(a_src + vi * VEC + t), ps);
+            pd = fmaf(f[t], __ldg(a_dst + vi * VEC + t), pd);
+          }
+          part[wib][sub][vi][0] = ps;
+          part[wib][sub][vi][1] = pd;
+        }
+      }
+    }
+    __syncwarp();
+    if (live) {
+      for (int k = sl; k < K; k += LPR) {
+        float ss = 0.f, sd = 0.f;
+        for (int v = k * vec_per_head; v < (k + 1) * vec_per_head; ++v) {
+          ss += part[wib][sub][v][0];
+          sd += part[wib][sub][v][1];
+        }
+        s_src[size_t(row - win.win_base) * K + k] = ss;
+        s_dst[size_t(row - win.win_base) * K + k] = sd;
+      }
+    }
+    __syncwarp();
+  }
+}
+
+// ---- Eq. 7: edge scores, softmax over producers + self, weighted sum of Z rows, bias, ReLU ---
+// Single pass with a running maximum (the sum is rescaled whenever the maximum grows), so every
+// Z row and every score is read once.  Edges are taken four at a time to keep loads in flight.
+template <typename T, int LPR, int VPL>
+__global__ void __launch_bounds__(kRowThreads)
+k_aggregate(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+            const T* __restrict__ Z, const float* __restrict__ s_src, const float* __restrict__ s_dst,
+            const float* __restrict__ bias, T* __restrict__ h_out, int H, int K, Window win) {
+  constexpr int VEC = VecOf<T>::N;
+  constexpr int RPW = 32 / LPR;
+  constexpr int EB = 4;
+  const int NV = H / VEC, d = H / K;
+  const int lane = threadIdx.x & 31, sub = lane / LPR, sl = lane % LPR;
+  const int warps_total = (gridDim.x * blockDim.x) >> 5;
+  const int warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+
+  int head[VPL];
+  bool on[VPL];
+#pragma unroll
+  for (int v = 0; v < VPL; ++v) {
+    const int vi = v * LPR + sl;
+    on[v] = vi < NV;
+    head[v] = on[v] ? (vi * VEC) / d : 0;
+  }
+
+  for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * RPW; r0 < win.row_end;
+       r0 += int64_t(warps_total) * RPW) {
+    const int32_t row = int32_t(r0) + sub;
+    if (row >= win.row_end) continue;
+    const int32_t lrow = row - win.win_base;
+    const int32_t e0 = __ldg(rowptr + row), e1 = __ldg(rowptr + row + 1);
+
+    float m[VPL], l[VPL], sd[VPL], acc[VPL][VEC];
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+      if (on[v]) {
+        sd[v] = __ldg(s_dst + size_t(lrow) * K + head[v]);
+        m[v] = leaky(__ldg(s_src + size_t(lrow) * K + head[v]) + sd[v]);   // the self term
+        l[v] = 1.f;
+        load_vec(Z + size_t(lrow) * H + (v * LPR + sl) * VEC, acc[v]);
+      }
+    }
+    for (int32_t e = e0; e < e1; e += EB) {
+      int32_t j[EB];
+#pragma unroll
+      for (int b = 0; b < EB; ++b) j[b] = (e + b < e1) ? __ldg(col + e + b) - win.win_base : -1;
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) {
+        if (!on[v]) continue;
+        float sc[EB], z[EB][VEC];
+#pragma unroll
+        for (int b = 0; b < EB; ++b) {
+          if (j[b] >= 0) {
+            sc[b] = __ldg(s_src + size_t(j[b]) * K + head[v]);
+            load_vec(Z + size_t(j[b]) * H + (v * LPR + sl) * VEC, z[b]);
+          }
+        }
+#pragma unroll
+        for (int b = 0; b < EB; ++b) {
+          if (j[b] >= 0) {
+            const float ev = leaky(sc[b] + sd[v]);
+            if (ev > m[v]) {
+              const float scale = __expf(m[v] - ev);
+              l[v] *= scale;
+#pragma unroll
+              for (int t = 0; t < VEC; ++t) acc[v][t] *= scale;
+              m[v] = ev;
+            }
+            const float p = __expf(ev - m[v]);
+            l[v] += p;
+#pragma unroll
+            for (int t = 0; t < VEC; ++t) acc[v][t] = fmaf(p, z[b][t], acc[v][t]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+      if (!on[v]) continue;
+      const int c0 = (v * LPR + sl) * VEC;
+      const float inv = 1.f / l[v];
+      float o[VEC];
+#pragma unroll
+      for (int t = 0; t < VEC; ++t) o[t] = fmaxf(fmaf(acc[v][t], inv, __ldg(bias + c0 + t)), 0.f);
+      store_vec(h_out + size_t(lrow) * H + c0, o);
+    }
+  }
+}
+
+// ---- dispatch on the row geometry ------------------------------------------------------------
+struct RowGeom { int lpr, vpl; };
+
+template <typename T>
+RowGeom row_geom(int H) {
+  const int nv = H / VecOf<T>::N;
+  if (nv <= 8) return {8, 1};
+  if (nv == 16) return {16, 1};
+  const int vpl = (nv + 31) / 32;
+  return {32, vpl <= 1 ? 1 : (vpl == 2 ? 2 : 4)};
+}
+
+int row_grid(int64_t rows, int rpw) {
+  const int64_t warps = (rows + rpw - 1) / rpw;
+  const int64_t blocks = (warps + (kRowThreads / 32) - 1) / (kRowThreads / 32);
+  const int64_t cap = int64_t(kNumSMs) * 8;
+  return int(blocks < 1 ? 1 : (blocks > cap ? cap : blocks));
+}
+
+#define XRL_ROW_DISPATCH(TY_, H, CALL)                                         \
+  do {                                                                       \
+    const RowGeom g_ = row_geom<TY_>(H);                                       \
+    if (g_.lpr == 8) { CALL(TY_, 8, 1); }                                      \
+    else if (g_.lpr == 16) { CALL(TY_, 16, 1); }                               \
+    else if (g_.vpl == 1) { CALL(TY_, 32, 1); }                                \
+    else if (g_.vpl == 2) { CALL(TY_, 32, 2); }                                \
+    else { CALL(TY_, 32, 4); }                                                 \
+  } while (0)
+
+}  // namespace
+
+int launch_embed(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op,
+                 const void* shape, const DevWeights& w, void* h, Window win, cudaStream_t st) {
+  const int64_t rows = int64_t(win.row_end) - win.row_begin;
+  if (rows <= 0) return 0;
+  const size_t smem = sizeof(float) * size_t(2 * kS + 1) * d.H;
+#define CALL(TY_, LPR, VPL)                                                                        \
+  k_embed<TY_, LPR, VPL><<<row_grid(rows, 32 / LPR), kRowThreads, smem, st>>>(                     \
+      rowptr, col, op, static_cast<const TY_*>(shape), static_cast<const TY_*>(w.W0), w.b0,   \
+      static_cast<TY_*>(h), d.H, d.T, win)
+  if (d.dtype == XRL_BF16) XRL_ROW_DISPATCH(bf16, d.H, CALL);
+  else XRL_ROW_DISPATCH(float, d.H, CALL);
+#undef CALL
+  return 1;
+}
+
+int launch_scores(const Dims& d, const void* Z, const LayerWeights& lw, float* s_src, float* s_dst,
+                  Window win, cudaStream_t st) {
+  const int64_t rows = int64_t(win.row_end) - win.row_begin;
+  if (rows <= 0) return 0;
+#define CALL(TY_, LPR, VPL)                                                                        \
+  k_scores<TY_, LPR, VPL><<<row_grid(rows, 32 / LPR), kRowThreads, 0, st>>>(                       \
+      static_cast<const TY_*>(Z), lw.a_src, lw.a_dst, s_src, s_dst, d.H, d.K, win)
+  if (d.dtype == XRL_BF16) XRL_ROW_DISPATCH(bf16, d.H, CALL);
+  else XRL_ROW_DISPATCH(float, d.H, CALL);
+#undef CALL
+  return 1;
+}
+
+int launch_aggregate(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z,
+                     const float* s_src, const float* s_dst, const float* bias, void* h_out,
+                     Window win, cudaStream_t st) {
+  const int64_t rows = int64_t(win.row_end) - win.row_begin;
+  if (rows <= 0) return 0;
+#define CALL(TY_, LPR, VPL)                                                                        \
+  k_aggregate<TY_, LPR, VPL><<<row_grid(rows, 32 / LPR), kRowThreads, 0, st>>>(                    \
+      rowptr, col, static_cast<const TY_*>(Z), s_src, s_dst, bias, static_cast<TY_*>(h_out), d.H,   \
+      d.K, win)
+  if (d.dtype == XRL_BF16) XRL_ROW_DISPATCH(bf16, d.H, CALL);
+  else XRL_ROW_DISPATCH(float, d.H, CALL);
+#undef CALL
+  return 1;
+}
+
+}  // namespace xrl

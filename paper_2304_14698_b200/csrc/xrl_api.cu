@@ -1,0 +1,554 @@
+// C-ABI layer of libxrl: contexts, weights, batches and the three calls of the path
+// (xrl_pack, xrl_encode, xrl_policy_value).  Host code here only validates arguments, moves
+// bytes and sequences kernel launches; every step of the method runs in the kernels.
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "xrl_internal.cuh"
+
+using namespace xrl;
+
+namespace {
+
+constexpr int32_t kReadoutChunkRows = 512;
+
+struct DeviceBuf {
+  void* p = nullptr;
+  size_t bytes = 0;
+  cudaError_t alloc(size_t n) {
+    bytes = n;
+    return cudaMalloc(&p, n ? n : 1);
+  }
+  void release() { if (p) cudaFree(p); p = nullptr; }
+  template <typename T> T* as() const { return static_cast<T*>(p); }
+};
+
+size_t storage_bytes(int dtype) { return dtype == XRL_BF16 ? 2 : 4; }
+
+}  // namespace
+
+struct xrl_ctx {
+  xrl_model_config cfg;
+  Dims dims;
+  int device = 0;
+  bool weights_set = false;
+  size_t weight_floats = 0;
+  DeviceBuf w_f32;          // the fp32 blob
+  DeviceBuf w_store;        // storage-type copies of W0 and the layer matrices (+ transposes)
+  DevWeights dw;
+  DeviceBuf h, Z, s_src, s_dst, partial, logits, status;
+  int32_t max_chunks = 0;
+  int64_t launches_pack = 0, launches_encode = 0, launches_heads = 0;
+};
+
+struct xrl_batch {
+  xrl_ctx* ctx = nullptr;
+  bool packed = false;
+  int32_t B = 0, num_envs = 0, N = 0, E = 0, num_chunks = 0;
+  cudaStream_t stream = nullptr;
+  // device
+  DeviceBuf meta;           // n_nodes[B] n_edges[B] env_off[Ne+1] graph_chunk_off[B+1] chunk_row0[] chunk_row1[]
+  DeviceBuf node_off, edge_off, seg_id, graph_env, rowptr, col, op, shape;
+  DeviceBuf edge_src, edge_dst, deg, tmp_eid, long_rows, long_count, scan_ws;
+  const int32_t *d_n_nodes = nullptr, *d_n_edges = nullptr, *d_env_off = nullptr,
+                *d_graph_chunk_off = nullptr, *d_chunk_row0 = nullptr, *d_chunk_row1 = nullptr;
+  // pinned host staging (allocated on the first pack from host memory)
+  int32_t* h_meta = nullptr;
+  size_t h_meta_ints = 0;
+  char* h_bulk = nullptr;
+  size_t h_bulk_bytes = 0;
+  cudaEvent_t staged = nullptr;   // the last upload out of the staging buffers has completed
+};
+
+namespace {
+
+xrl_status check_config(const xrl_model_config& c) {
+  if (c.num_op_types < 1 || c.hidden < 1 || c.heads < 1 || c.layers < 0 || c.mlp_hidden < 1 ||
+      c.global_dim < 0 || c.max_actions < 0 || c.max_graphs < 1 || c.max_envs < 1 ||
+      c.max_nodes < 1 || c.max_edges < 0)
+    return XRL_ERR_INVALID_ARG;
+  if (c.dtype != XRL_FP32 && c.dtype != XRL_BF16) return XRL_ERR_INVALID_ARG;
+  if (c.hidden % c.heads != 0) return XRL_ERR_INVALID_ARG;
+  if (c.max_nodes >= (int64_t(1) << 31) - 1 || c.max_edges >= (int64_t(1) << 31) - 1)
+    return XRL_ERR_INVALID_ARG;
+  if (c.num_shape_feats != kS || c.num_op_types > 256) return XRL_ERR_UNSUPPORTED;
+  if (c.hidden % 32 != 0 || c.hidden > 512 || (c.hidden / c.heads) % 8 != 0) return XRL_ERR_UNSUPPORTED;
+  if (c.layers > 64 || c.mlp_hidden > 1024 || c.global_dim > 16) return XRL_ERR_UNSUPPORTED;
+  if (c.max_actions > (1 << 20)) return XRL_ERR_UNSUPPORTED;
+  return XRL_OK;
+}
+
+size_t weight_float_count(const xrl_model_config& c) {
+  const size_t S = c.num_shape_feats, T = c.num_op_types, H = c.hidden, L = c.layers,
+               Hm = c.mlp_hidden, Dg = c.global_dim;
+  return (2 * S + T) * H + H + L * (H * H + 3 * H) + (H + Dg) * H + H + (H * Hm + 2 * Hm + 1) +
+         (2 * H * Hm + 2 * Hm + 1);
+}
+
+#define XRL_CUDA(call)                      \
+  do {                                      \
+    if ((call) != cudaSuccess) {            \
+      cudaGetLastError();                   \
+      return XRL_ERR_CUDA;                  \
+    }                                       \
+  } while (0)
+#define XRL_ALLOC(call)                     \
+  do {                                      \
+    if ((call) != cudaSuccess) {            \
+      cudaGetLastError();                   \
+      return XRL_ERR_ALLOC;                 \
+    }                                       \
+  } while (0)
+
+xrl_status alloc_batch(xrl_ctx* ctx, xrl_batch** out) {
+  xrl_batch* b = new (std::nothrow) xrl_batch();
+  if (!b) return XRL_ERR_ALLOC;
+  b->ctx = ctx;
+  const xrl_model_config& c = ctx->cfg;
+  const size_t N = size_t(c.max_nodes), E = size_t(c.max_edges), B = size_t(c.max_graphs),
+               Ne = size_t(c.max_envs);
+  const size_t sb = storage_bytes(c.dtype);
+  b->h_meta_ints = 2 * B + (Ne + 1) + (B + 1) + 2 * size_t(ctx->max_chunks);
+  cudaError_t e = cudaSuccess;
+  auto A = [&](DeviceBuf& d, size_t bytes) { if (e == cudaSuccess) e = d.alloc(bytes); };
+  A(b->meta, 4 * b->h_meta_ints);
+  A(b->node_off, 4 * (B + 1)); A(b->edge_off, 4 * (B + 1));
+  A(b->seg_id, 4 * N); A(b->graph_env, 4 * B);
+  A(b->rowptr, 4 * (N + 1)); A(b->col, 4 * E);
+  A(b->op, 4 * N); A(b->shape, sb * N * kS);
+  A(b->edge_src, 4 * E); A(b->edge_dst, 4 * E);
+  A(b->deg, 4 * N); A(b->tmp_eid, 4 * E);
+  A(b->long_rows, 4 * (E / 32 + 1)); A(b->long_count, 4);
+  A(b->scan_ws, 4 * scan_workspace_ints(int64_t(N > B ? N : B) + 1));
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&b->staged, cudaEventDisableTiming);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    xrl_batch_free(ctx, b);
+    return XRL_ERR_ALLOC;
+  }
+  *out = b;
+  return XRL_OK;
+}
+
+xrl_status ensure_staging(xrl_batch* b) {
+  if (b->h_meta == nullptr)
+    XRL_ALLOC(cudaHostAlloc(reinterpret_cast<void**>(&b->h_meta), 4 * b->h_meta_ints, cudaHostAllocDefault));
+  return XRL_OK;
+}
+
+xrl_status ensure_bulk_staging(xrl_batch* b) {
+  if (b->h_bulk == nullptr) {
+    const xrl_model_config& c = b->ctx->cfg;
+    b->h_bulk_bytes = size_t(c.max_nodes) * (4 + storage_bytes(c.dtype) * kS) + size_t(c.max_edges) * 8;
+    XRL_ALLOC(cudaHostAlloc(reinterpret_cast<void**>(&b->h_bulk), b->h_bulk_bytes ? b->h_bulk_bytes : 1,
+                            cudaHostAllocDefault));
+  }
+  return XRL_OK;
+}
+
+// Shared tail of both pack entry points.  `graphs` non-null: gather from per-graph host arrays.
+xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int32_t num_graphs,
+                       const int32_t* n_nodes, const int32_t* n_edges, const int32_t* op,
+                       const void* shape, const int32_t* edge_src, const int32_t* edge_dst,
+                       const int32_t* env_off, int32_t num_envs, void* stream, xrl_batch** out) {
+  if (!ctx || !out || !env_off || num_graphs < 0 || num_envs < 0) return XRL_ERR_INVALID_ARG;
+  if (!graphs && (where != XRL_MEM_HOST && where != XRL_MEM_DEVICE)) return XRL_ERR_INVALID_ARG;
+  if (!graphs && num_graphs > 0 && (!n_nodes || !n_edges)) return XRL_ERR_INVALID_ARG;
+  const xrl_model_config& c = ctx->cfg;
+  if (num_graphs > c.max_graphs || num_envs > c.max_envs) return XRL_ERR_CAPACITY;
+  if (env_off[0] != 0 || env_off[num_envs] != num_graphs) return XRL_ERR_INVALID_ARG;
+  for (int32_t e = 0; e < num_envs; ++e) {
+    if (env_off[e + 1] <= env_off[e]) return XRL_ERR_INVALID_ARG;
+    if (env_off[e + 1] - env_off[e] - 1 > c.max_actions) return XRL_ERR_CAPACITY;
+  }
+  int64_t N = 0, E = 0;
+  for (int32_t g = 0; g < num_graphs; ++g) {
+    const int32_t n = graphs ? graphs[g].num_nodes : n_nodes[g];
+    const int32_t m = graphs ? graphs[g].num_edges : n_edges[g];
+    if (n < 0 || m < 0) return XRL_ERR_INVALID_ARG;
+    if (graphs && ((n > 0 && (!graphs[g].op || !graphs[g].shape)) ||
+                   (m > 0 && (!graphs[g].edge_src || !graphs[g].edge_dst))))
+      return XRL_ERR_INVALID_ARG;
+    N += n; E += m;
+  }
+  if (N > c.max_nodes || E > c.max_edges) return XRL_ERR_CAPACITY;
+  if (!graphs && ((N > 0 && (!op || !shape)) || (E > 0 && (!edge_src || !edge_dst))))
+    return XRL_ERR_INVALID_ARG;
+
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  xrl_batch* b = *out;
+  if (b == nullptr) {
+    const xrl_status s = alloc_batch(ctx, &b);
+    if (s != XRL_OK) return s;
+  } else if (b->ctx != ctx) {
+    return XRL_ERR_STATE;
+  }
+  xrl_status s = ensure_staging(b);
+  if (s == XRL_OK && (graphs || where == XRL_MEM_HOST)) s = ensure_bulk_staging(b);
+  if (s != XRL_OK) { if (*out == nullptr) xrl_batch_free(ctx, b); return s; }
+  *out = b;
+  b->packed = false;
+  // the previous upload out of the staging buffers must have finished before they are rewritten
+  XRL_CUDA(cudaEventSynchronize(b->staged));
+
+  // ---- metadata: counts, env offsets, readout chunk list --------------------------------------
+  const size_t Bz = size_t(c.max_graphs), Nez = size_t(c.max_envs);
+  int32_t* m_nn = b->h_meta;
+  int32_t* m_ne = m_nn + Bz;
+  int32_t* m_env = m_ne + Bz;
+  int32_t* m_gco = m_env + (Nez + 1);
+  int32_t* m_c0 = m_gco + (Bz + 1);
+  int32_t* m_c1 = m_c0 + ctx->max_chunks;
+  int32_t chunks = 0, row = 0;
+  for (int32_t g = 0; g < num_graphs; ++g) {
+    const int32_t n = graphs ? graphs[g].num_nodes : n_nodes[g];
+    m_nn[g] = n;
+    m_ne[g] = graphs ? graphs[g].num_edges : n_edges[g];
+    m_gco[g] = chunks;
+    for (int32_t r = 0; r < n; r += kReadoutChunkRows) {
+      m_c0[chunks] = row + r;
+      m_c1[chunks] = row + (r + kReadoutChunkRows < n ? r + kReadoutChunkRows : n);
+      ++chunks;
+    }
+    row += n;
+  }
+  m_gco[num_graphs] = chunks;
+  memcpy(m_env, env_off, sizeof(int32_t) * size_t(num_envs + 1));
+  XRL_CUDA(cudaMemcpyAsync(b->meta.p, b->h_meta, 4 * b->h_meta_ints, cudaMemcpyHostToDevice, st));
+  const int32_t* dm = b->meta.as<int32_t>();
+  b->d_n_nodes = dm; b->d_n_edges = dm + Bz; b->d_env_off = dm + 2 * Bz;
+  b->d_graph_chunk_off = dm + 2 * Bz + (Nez + 1);
+  b->d_chunk_row0 = b->d_graph_chunk_off + (Bz + 1);
+  b->d_chunk_row1 = b->d_chunk_row0 + ctx->max_chunks;
+
+  // ---- bulk arrays -------------------------------------------------------------------------------
+  const size_t sb = storage_bytes(c.dtype);
+  const int32_t *d_src, *d_dst;
+  if (graphs || where == XRL_MEM_HOST) {
+    char* p_op = b->h_bulk;
+    char* p_shape = p_op + 4 * size_t(N);
+    char* p_src = p_shape + sb * kS * size_t(N);
+    char* p_dst = p_src + 4 * size_t(E);
+    if (graphs) {
+      size_t no = 0, eo = 0;
+      for (int32_t g = 0; g < num_graphs; ++g) {
+        const size_t n = size_t(graphs[g].num_nodes), m = size_t(graphs[g].num_edges);
+        if (n) {
+          memcpy(p_op + 4 * no, graphs[g].op, 4 * n);
+          memcpy(p_shape + sb * kS * no, graphs[g].shape, sb * kS * n);
+        }
+        if (m) {
+          memcpy(p_src + 4 * eo, graphs[g].edge_src, 4 * m);
+          memcpy(p_dst + 4 * eo, graphs[g].edge_dst, 4 * m);
+        }
+        no += n; eo += m;
+      }
+    } else {
+      if (N) { memcpy(p_op, op, 4 * size_t(N)); memcpy(p_shape, shape, sb * kS * size_t(N)); }
+      if (E) { memcpy(p_src, edge_src, 4 * size_t(E)); memcpy(p_dst, edge_dst, 4 * size_t(E)); }
+    }
+    if (N) {
+      XRL_CUDA(cudaMemcpyAsync(b->op.p, p_op, 4 * size_t(N), cudaMemcpyHostToDevice, st));
+      XRL_CUDA(cudaMemcpyAsync(b->shape.p, p_shape, sb * kS * size_t(N), cudaMemcpyHostToDevice, st));
+    }
+    if (E) {
+      XRL_CUDA(cudaMemcpyAsync(b->edge_src.p, p_src, 4 * size_t(E), cudaMemcpyHostToDevice, st));
+      XRL_CUDA(cudaMemcpyAsync(b->edge_dst.p, p_dst, 4 * size_t(E), cudaMemcpyHostToDevice, st));
+    }
+    d_src = b->edge_src.as<int32_t>();
+    d_dst = b->edge_dst.as<int32_t>();
+  } else {
+    if (N) {
+      XRL_CUDA(cudaMemcpyAsync(b->op.p, op, 4 * size_t(N), cudaMemcpyDeviceToDevice, st));
+      XRL_CUDA(cudaMemcpyAsync(b->shape.p, shape, sb * kS * size_t(N), cudaMemcpyDeviceToDevice, st));
+    }
+    d_src = edge_src;
+    d_dst = edge_dst;
+  }
+  XRL_CUDA(cudaEventRecord(b->staged, st));
+
+  PackIn in;
+  in.B = num_graphs; in.num_envs = num_envs; in.N = int32_t(N); in.E = int32_t(E);
+  in.n_nodes = b->d_n_nodes; in.n_edges = b->d_n_edges; in.env_off = b->d_env_off;
+  in.op = b->op.as<int32_t>(); in.edge_src = d_src; in.edge_dst = d_dst;
+  PackOut po;
+  po.node_off = b->node_off.as<int32_t>(); po.edge_off = b->edge_off.as<int32_t>();
+  po.seg_id = b->seg_id.as<int32_t>(); po.graph_env = b->graph_env.as<int32_t>();
+  po.rowptr = b->rowptr.as<int32_t>(); po.col = b->col.as<int32_t>();
+  po.deg = b->deg.as<int32_t>(); po.tmp_eid = b->tmp_eid.as<int32_t>();
+  po.long_rows = b->long_rows.as<int32_t>(); po.long_count = b->long_count.as<int32_t>();
+  po.scan_ws = b->scan_ws.as<int32_t>();
+  ctx->launches_pack = launch_pack(in, po, c.num_op_types, ctx->status.as<int32_t>(), st);
+  XRL_CUDA(cudaGetLastError());
+
+  b->B = num_graphs; b->num_envs = num_envs; b->N = int32_t(N); b->E = int32_t(E);
+  b->num_chunks = chunks; b->stream = st; b->packed = true;
+  return XRL_OK;
+}
+
+// Eq. 6 and the first `layers` attention layers over the whole batch; features end up in ctx->h.
+int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t st) {
+  const Dims& d = ctx->dims;
+  const Window win{0, b->N, 0};
+  int n = launch_embed(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), b->op.as<int32_t>(),
+                       b->shape.p, ctx->dw, ctx->h.p, win, st);
+  for (int l = 0; l < layers; ++l) {
+    n += launch_xform_simt(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->s_src.as<float>(),
+                           ctx->s_dst.as<float>(), win, st);
+    n += launch_aggregate(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), ctx->Z.p,
+                          ctx->s_src.as<float>(), ctx->s_dst.as<float>(), ctx->dw.layer[l].b,
+                          ctx->h.p, win, st);
+  }
+  return n;
+}
+
+xrl_status check_batch(const xrl_ctx* ctx, const xrl_batch* b) {
+  if (!ctx || !b) return XRL_ERR_INVALID_ARG;
+  if (b->ctx != ctx || !b->packed || !ctx->weights_set) return XRL_ERR_STATE;
+  return XRL_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* xrl_version(void) { return "xrl 0.1 (sm_100a, CUDA C-ABI)"; }
+
+xrl_status xrl_create(const xrl_model_config* cfg, int32_t device, xrl_ctx** out) {
+  if (!cfg || !out) return XRL_ERR_INVALID_ARG;
+  *out = nullptr;
+  const xrl_status s = check_config(*cfg);
+  if (s != XRL_OK) return s;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+    cudaGetLastError();
+    return XRL_ERR_CUDA;
+  }
+  XRL_CUDA(cudaSetDevice(device));
+  xrl_ctx* ctx = new (std::nothrow) xrl_ctx();
+  if (!ctx) return XRL_ERR_ALLOC;
+  ctx->cfg = *cfg;
+  ctx->device = device;
+  ctx->dims = Dims{cfg->num_op_types, cfg->hidden, cfg->heads, cfg->layers, cfg->mlp_hidden,
+                   cfg->global_dim, cfg->max_actions, cfg->dtype};
+  ctx->weight_floats = weight_float_count(*cfg);
+  ctx->max_chunks = int32_t(cfg->max_graphs + cfg->max_nodes / kReadoutChunkRows + 1);
+  const size_t sb = storage_bytes(cfg->dtype), N = size_t(cfg->max_nodes), H = size_t(cfg->hidden);
+  const size_t F0 = size_t(2 * kS + cfg->num_op_types);
+  cudaError_t e = cudaSuccess;
+  auto A = [&](DeviceBuf& d, size_t bytes) { if (e == cudaSuccess) e = d.alloc(bytes); };
+  A(ctx->w_f32, 4 * ctx->weight_floats);
+  A(ctx->w_store, sb * (F0 * H + 2 * size_t(cfg->layers) * H * H));
+  A(ctx->h, sb * N * H);
+  A(ctx->Z, sb * N * H);
+  A(ctx->s_src, 4 * N * size_t(cfg->heads));
+  A(ctx->s_dst, 4 * N * size_t(cfg->heads));
+  A(ctx->partial, 4 * size_t(ctx->max_chunks) * H);
+  A(ctx->logits, 4 * size_t(cfg->max_graphs));
+  A(ctx->status, 4);
+  if (e == cudaSuccess) e = cudaMemset(ctx->status.p, 0, 4);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    xrl_destroy(ctx);
+    return XRL_ERR_ALLOC;
+  }
+  *out = ctx;
+  return XRL_OK;
+}
+
+void xrl_destroy(xrl_ctx* ctx) {
+  if (!ctx) return;
+  cudaSetDevice(ctx->device);
+  cudaDeviceSynchronize();
+  DeviceBuf* bufs[] = {&ctx->w_f32, &ctx->w_store, &ctx->h, &ctx->Z, &ctx->s_src, &ctx->s_dst,
+                       &ctx->partial, &ctx->logits, &ctx->status};
+  for (DeviceBuf* d : bufs) d->release();
+  delete ctx;
+}
+
+xrl_status xrl_weights_size(const xrl_ctx* ctx, size_t* bytes) {
+  if (!ctx || !bytes) return XRL_ERR_INVALID_ARG;
+  *bytes = 4 * ctx->weight_floats;
+  return XRL_OK;
+}
+
+xrl_status xrl_set_weights(xrl_ctx* ctx, const void* host_blob, size_t bytes) {
+  if (!ctx || !host_blob) return XRL_ERR_INVALID_ARG;
+  if (bytes != 4 * ctx->weight_floats) return XRL_ERR_INVALID_ARG;
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  XRL_CUDA(cudaMemcpy(ctx->w_f32.p, host_blob, bytes, cudaMemcpyHostToDevice));
+  const xrl_model_config& c = ctx->cfg;
+  const size_t H = size_t(c.hidden), Hm = size_t(c.mlp_hidden), Dg = size_t(c.global_dim);
+  const size_t F0 = size_t(2 * kS + c.num_op_types), sb = storage_bytes(c.dtype);
+  const float* p = ctx->w_f32.as<float>();
+  char* store = ctx->w_store.as<char>();
+  auto take = [&](size_t n) { const float* q = p; p += n; return q; };
+  DevWeights& w = ctx->dw;
+  const float* W0 = take(F0 * H);
+  launch_round_weights(W0, store, nullptr, int(F0), int(H), c.dtype, nullptr);
+  w.W0 = store; store += sb * F0 * H;
+  w.b0 = take(H);
+  for (int l = 0; l < c.layers; ++l) {
+    const float* W = take(H * H);
+    launch_round_weights(W, store, store + sb * H * H, int(H), int(H), c.dtype, nullptr);
+    w.layer[l].W = store;
+    w.layer[l].Wt = store + sb * H * H;
+    store += 2 * sb * H * H;
+    w.layer[l].a_src = take(H);
+    w.layer[l].a_dst = take(H);
+    w.layer[l].b = take(H);
+  }
+  w.Wg = take((H + Dg) * H); w.bg = take(H);
+  w.pW1 = take(H * Hm); w.pb1 = take(Hm); w.pw2 = take(Hm); w.pb2 = take(1);
+  w.vW1 = take(2 * H * Hm); w.vb1 = take(Hm); w.vw2 = take(Hm); w.vb2 = take(1);
+  XRL_CUDA(cudaDeviceSynchronize());
+  XRL_CUDA(cudaGetLastError());
+  ctx->weights_set = true;
+  return XRL_OK;
+}
+
+xrl_status xrl_pack(xrl_ctx* ctx, const xrl_graph* graphs, int32_t num_graphs, const int32_t* env_off,
+                    int32_t num_envs, void* stream, xrl_batch** out) {
+  if (num_graphs > 0 && !graphs) return XRL_ERR_INVALID_ARG;
+  static const xrl_graph none = {0, 0, nullptr, nullptr, nullptr, nullptr};
+  return pack_common(ctx, graphs ? graphs : &none, XRL_MEM_HOST, num_graphs, nullptr, nullptr, nullptr,
+                     nullptr, nullptr, nullptr, env_off, num_envs, stream, out);
+}
+
+xrl_status xrl_pack_flat(xrl_ctx* ctx, int32_t where, int32_t num_graphs, const int32_t* n_nodes,
+                         const int32_t* n_edges, const int32_t* op, const void* shape,
+                         const int32_t* edge_src, const int32_t* edge_dst, const int32_t* env_off,
+                         int32_t num_envs, void* stream, xrl_batch** out) {
+  return pack_common(ctx, nullptr, where, num_graphs, n_nodes, n_edges, op, shape, edge_src, edge_dst,
+                     env_off, num_envs, stream, out);
+}
+
+xrl_status xrl_batch_free(xrl_ctx* ctx, xrl_batch* b) {
+  if (!b) return XRL_OK;
+  if (ctx && b->ctx != ctx) return XRL_ERR_STATE;
+  cudaSetDevice(b->ctx->device);
+  cudaDeviceSynchronize();
+  DeviceBuf* bufs[] = {&b->meta, &b->node_off, &b->edge_off, &b->seg_id, &b->graph_env, &b->rowptr,
+                       &b->col, &b->op, &b->shape, &b->edge_src, &b->edge_dst, &b->deg, &b->tmp_eid,
+                       &b->long_rows, &b->long_count, &b->scan_ws};
+  for (DeviceBuf* d : bufs) d->release();
+  if (b->h_meta) cudaFreeHost(b->h_meta);
+  if (b->h_bulk) cudaFreeHost(b->h_bulk);
+  if (b->staged) cudaEventDestroy(b->staged);
+  delete b;
+  return XRL_OK;
+}
+
+xrl_status xrl_batch_info(const xrl_batch* b, int64_t* num_nodes, int64_t* num_edges,
+                          int32_t* num_graphs, int32_t* num_envs) {
+  if (!b) return XRL_ERR_INVALID_ARG;
+  if (!b->packed) return XRL_ERR_STATE;
+  if (num_nodes) *num_nodes = b->N;
+  if (num_edges) *num_edges = b->E;
+  if (num_graphs) *num_graphs = b->B;
+  if (num_envs) *num_envs = b->num_envs;
+  return XRL_OK;
+}
+
+xrl_status xrl_batch_export(const xrl_batch* b, int32_t* rowptr, int32_t* col, int32_t* seg_id,
+                            int32_t* node_off, int32_t* edge_off, int32_t* graph_env) {
+  if (!b) return XRL_ERR_INVALID_ARG;
+  if (!b->packed) return XRL_ERR_STATE;
+  XRL_CUDA(cudaSetDevice(b->ctx->device));
+  XRL_CUDA(cudaStreamSynchronize(b->stream));
+  const size_t N = size_t(b->N), E = size_t(b->E), B = size_t(b->B);
+  if (rowptr) XRL_CUDA(cudaMemcpy(rowptr, b->rowptr.p, 4 * (N + 1), cudaMemcpyDeviceToHost));
+  if (col && E) XRL_CUDA(cudaMemcpy(col, b->col.p, 4 * E, cudaMemcpyDeviceToHost));
+  if (seg_id && N) XRL_CUDA(cudaMemcpy(seg_id, b->seg_id.p, 4 * N, cudaMemcpyDeviceToHost));
+  if (node_off) XRL_CUDA(cudaMemcpy(node_off, b->node_off.p, 4 * (B + 1), cudaMemcpyDeviceToHost));
+  if (edge_off) XRL_CUDA(cudaMemcpy(edge_off, b->edge_off.p, 4 * (B + 1), cudaMemcpyDeviceToHost));
+  if (graph_env && B) XRL_CUDA(cudaMemcpy(graph_env, b->graph_env.p, 4 * B, cudaMemcpyDeviceToHost));
+  return XRL_OK;
+}
+
+xrl_status xrl_encode(xrl_ctx* ctx, const xrl_batch* b, const float* g0, float* graph_emb, void* stream) {
+  const xrl_status s = check_batch(ctx, b);
+  if (s != XRL_OK) return s;
+  if (!graph_emb && b->B > 0) return XRL_ERR_INVALID_ARG;
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int n = run_node_layers(ctx, b, ctx->cfg.layers, st);
+  n += launch_readout(ctx->dims, ctx->h.p, b->d_chunk_row0, b->d_chunk_row1, 0, b->num_chunks,
+                      ctx->partial.as<float>(), 0, st);
+  n += launch_global_update(ctx->dims, ctx->partial.as<float>(), b->d_graph_chunk_off, g0, ctx->dw,
+                            graph_emb, b->B, st);
+  ctx->launches_encode = n;
+  XRL_CUDA(cudaGetLastError());
+  return XRL_OK;
+}
+
+xrl_status xrl_debug_node_features(xrl_ctx* ctx, const xrl_batch* b, int32_t num_layers,
+                                   float* host_out, void* stream) {
+  const xrl_status s = check_batch(ctx, b);
+  if (s != XRL_OK) return s;
+  if (num_layers < 0 || num_layers > ctx->cfg.layers || (!host_out && b->N > 0)) return XRL_ERR_INVALID_ARG;
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  run_node_layers(ctx, b, num_layers, st);
+  const int64_t n = int64_t(b->N) * ctx->cfg.hidden;
+  if (n == 0) return XRL_OK;
+  float* tmp = nullptr;
+  XRL_ALLOC(cudaMalloc(&tmp, sizeof(float) * size_t(n)));
+  launch_to_float(ctx->h.p, ctx->cfg.dtype, tmp, n, st);
+  cudaError_t e = cudaStreamSynchronize(st);
+  if (e == cudaSuccess) e = cudaMemcpy(host_out, tmp, sizeof(float) * size_t(n), cudaMemcpyDeviceToHost);
+  cudaFree(tmp);
+  XRL_CUDA(e);
+  XRL_CUDA(cudaGetLastError());
+  return XRL_OK;
+}
+
+xrl_status xrl_policy_value(xrl_ctx* ctx, const xrl_batch* b, const float* graph_emb,
+                            const uint8_t* mask, float* probs, float* value, int32_t* action,
+                            uint64_t seed, uint64_t step, void* stream) {
+  const xrl_status s = check_batch(ctx, b);
+  if (s != XRL_OK) return s;
+  if (b->num_envs > 0 && (!graph_emb || !probs || !value || (!mask && ctx->cfg.max_actions > 0)))
+    return XRL_ERR_INVALID_ARG;
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ctx->launches_heads = launch_heads(ctx->dims, ctx->dw, graph_emb, b->d_env_off, mask, b->B, b->num_envs,
+                                     ctx->logits.as<float>(), probs, value, action, seed, step,
+                                     ctx->status.as<int32_t>(), st);
+  XRL_CUDA(cudaGetLastError());
+  return XRL_OK;
+}
+
+xrl_status xrl_sample(xrl_ctx* ctx, const float* probs, int32_t num_envs, int32_t num_actions,
+                      uint64_t seed, uint64_t step, int32_t* action, void* stream) {
+  if (!ctx || num_envs < 0 || num_actions < 1) return XRL_ERR_INVALID_ARG;
+  if (num_envs > 0 && (!probs || !action)) return XRL_ERR_INVALID_ARG;
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  launch_sample(probs, num_envs, num_actions, seed, step, action, static_cast<cudaStream_t>(stream));
+  XRL_CUDA(cudaGetLastError());
+  return XRL_OK;
+}
+
+xrl_status xrl_last_device_status(xrl_ctx* ctx, void* stream, int32_t* status) {
+  if (!ctx || !status) return XRL_ERR_INVALID_ARG;
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  XRL_CUDA(cudaStreamSynchronize(st));
+  XRL_CUDA(cudaMemcpy(status, ctx->status.p, 4, cudaMemcpyDeviceToHost));
+  XRL_CUDA(cudaMemset(ctx->status.p, 0, 4));
+  return XRL_OK;
+}
+
+xrl_status xrl_launch_counts(const xrl_ctx* ctx, int64_t* pack, int64_t* encode, int64_t* heads) {
+  if (!ctx) return XRL_ERR_INVALID_ARG;
+  if (pack) *pack = ctx->launches_pack;
+  if (encode) *encode = ctx->launches_encode;
+  if (heads) *heads = ctx->launches_heads;
+  return XRL_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,123 @@
+// Internal declarations shared by the kernels and the C-ABI layer of libxrl.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "xrl.h"
+
+namespace xrl {
+
+constexpr int kS = 8;            // shape features per node (compile-time in the kernels)
+constexpr int kNumSMs = 148;     // B200
+
+typedef __nv_bfloat16 bf16;
+
+// First error wins; kernels never trap.
+__device__ __forceinline__ void raise(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
+
+// ---- 16-byte vectors of the storage type ------------------------------------------------
+template <typename T> struct VecOf;
+template <> struct VecOf<float> { static constexpr int N = 4; };
+template <> struct VecOf<bf16> { static constexpr int N = 8; };
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t hi16) { return __uint_as_float(hi16 << 16); }
+
+__device__ __forceinline__ void unpack(const uint4& v, float (&f)[4]) {
+  f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+  f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+}
+__device__ __forceinline__ void unpack(const uint4& v, float (&f)[8]) {
+  f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xFFFF0000u);
+  f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xFFFF0000u);
+  f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xFFFF0000u);
+  f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xFFFF0000u);
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);   // .x = lo (low 16 bits), .y = hi
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+__device__ __forceinline__ uint4 pack(const float (&f)[4]) {
+  return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]),
+                    __float_as_uint(f[3]));
+}
+__device__ __forceinline__ uint4 pack(const float (&f)[8]) {
+  return make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]),
+                    pack_bf16x2(f[6], f[7]));
+}
+template <typename T>
+__device__ __forceinline__ void load_vec(const T* p, float (&f)[VecOf<T>::N]) {
+  unpack(__ldg(reinterpret_cast<const uint4*>(p)), f);
+}
+template <typename T>
+__device__ __forceinline__ void store_vec(T* p, const float (&f)[VecOf<T>::N]) {
+  *reinterpret_cast<uint4*>(p) = pack(f);
+}
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(bf16 x) { return __bfloat162float(x); }
+
+// ---- device-side weights ------------------------------------------------------------------
+struct LayerWeights {
+  const void* W;        // storage type, [H x H] row-major [in x out]
+  const void* Wt;       // bf16 only: transpose [out x in] (K-major B operand of the tensor-core path)
+  const float* a_src;   // [H]
+  const float* a_dst;   // [H]
+  const float* b;       // [H]
+};
+struct DevWeights {
+  const void* W0;       // storage type, [(2S+T) x H]
+  const float* b0;
+  LayerWeights layer[64];
+  const float* Wg; const float* bg;
+  const float *pW1, *pb1, *pw2, *pb2;
+  const float *vW1, *vb1, *vw2, *vb2;
+};
+
+struct Dims {
+  int T, H, K, L, Hm, Dg, A;
+  int dtype;
+};
+
+// ---- launchers (each returns the number of kernels it launched; errors via cudaGetLastError) --
+struct PackIn {
+  int32_t B, num_envs, N, E;
+  const int32_t *n_nodes, *n_edges, *env_off;     // device copies of the metadata
+  const int32_t *op, *edge_src, *edge_dst;        // device
+};
+struct PackOut {
+  int32_t *node_off, *edge_off, *seg_id, *graph_env, *rowptr, *col;
+  int32_t *deg, *tmp_eid, *long_rows, *long_count, *scan_ws;   // scratch
+};
+int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cudaStream_t st);
+size_t scan_workspace_ints(int64_t n);
+
+// Row windows: kernels process global rows [row_begin, row_end); activation buffers (h, Z,
+// scores) are indexed by (row - win_base), CSR / op / shape arrays by the global row id.
+struct Window { int32_t row_begin, row_end, win_base; };
+
+int launch_embed(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op,
+                 const void* shape, const DevWeights& w, void* h, Window win, cudaStream_t st);
+int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* s_src,
+                      float* s_dst, Window win, cudaStream_t st);
+int launch_scores(const Dims& d, const void* Z, const LayerWeights& lw, float* s_src, float* s_dst,
+                  Window win, cudaStream_t st);
+int launch_aggregate(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z,
+                     const float* s_src, const float* s_dst, const float* bias, void* h_out,
+                     Window win, cudaStream_t st);
+int launch_readout(const Dims& d, const void* h, const int32_t* chunk_row0, const int32_t* chunk_row1,
+                   int32_t chunk_begin, int32_t chunk_end, float* partial, int32_t win_base,
+                   cudaStream_t st);
+int launch_global_update(const Dims& d, const float* partial, const int32_t* graph_chunk_off,
+                         const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st);
+int launch_heads(const Dims& d, const DevWeights& w, const float* emb, const int32_t* env_off,
+                 const uint8_t* mask, int32_t B, int32_t num_envs, float* logit_ws, float* probs,
+                 float* value, int32_t* action, uint64_t seed, uint64_t step, int32_t* status,
+                 cudaStream_t st);
+int launch_sample(const float* probs, int32_t num_envs, int32_t A1, uint64_t seed, uint64_t step,
+                  int32_t* action, cudaStream_t st);
+int launch_to_float(const void* src, int dtype, float* dst, int64_t n, cudaStream_t st);
+int launch_round_weights(const float* src, void* dst, void* dst_t, int rows, int cols, int dtype,
+                         cudaStream_t st);
+
+}  // namespace xrl

@@ -1,0 +1,154 @@
+"""GPU parity of the encoder and heads (Sections 3.3.2-3.4) against the CPU oracle."""
+import numpy as np
+import pytest
+
+from workloads import configs, dags
+import gpu_util
+
+pytestmark = pytest.mark.gpu
+
+CASES = [(1, {}), (2, {}), (3, dict(candidates=15)), (4, dict(candidates=7)),
+         (5, dict(candidates=7, envs=3))]
+
+
+def _oracle(xo, batch, blob, **kw):
+    st, packed = xo.pack(batch)
+    assert st == 0
+    return packed, xo.encode(batch["model"], blob, batch, packed, **kw)
+
+
+@pytest.mark.parametrize("cfg,kw", CASES)
+def test_node_features_after_each_stage(xo, cfg, kw):
+    """Eq. 6 and each attention layer, node by node."""
+    import paper_2304_14698_b200 as xrl
+    batch = configs.make_batch(cfg, **kw)
+    m = batch["model"]
+    blob, _ = gpu_util.default_weights(batch, 1000 + cfg)
+    ag = gpu_util.make_agent(batch)
+    try:
+        ag.set_weights(blob)
+        ag.pack(batch)
+        for layer in range(m["L"] + 1):
+            got = xrl.xrl_debug_node_features(ag.ctx, ag.batch, layer, m["H"])
+            _, want = _oracle(xo, batch, blob, dump_layer=layer, want_nodes=True)
+            gpu_util.assert_close(got, want["nodes"], m["dtype"], f"cfg{cfg} nodes after stage {layer}")
+        assert ag.device_status() == 0
+    finally:
+        ag.close()
+
+
+@pytest.mark.parametrize("where", ["host", "device"])
+@pytest.mark.parametrize("cfg,kw", CASES)
+def test_step_outputs(xo, cfg, kw, where):
+    """graph_emb, probs, value of the whole step; structural properties of probs."""
+    batch = configs.make_batch(cfg, **kw)
+    m = batch["model"]
+    blob, _ = gpu_util.default_weights(batch, 1000 + cfg)
+    got = gpu_util.run_gpu(batch, blob, where=where)
+    assert got["status"] == 0
+    want = xo.forward(m, blob, batch)
+    gpu_util.assert_close(got["emb"], want["emb"], m["dtype"], "graph_emb")
+    gpu_util.assert_close(got["probs"], want["probs"], m["dtype"], "probs")
+    gpu_util.assert_close(got["value"], want["value"], m["dtype"], "value")
+    assert np.all(got["probs"][want["probs"] == 0] == 0.0)       # masked / padded: exactly zero
+    assert np.all(np.abs(got["probs"].sum(axis=1) - 1) < 1e-5)
+    assert np.all(got["probs"][:, -1] > 0)
+
+
+def test_policy_with_spread_logits(xo):
+    """Head weights scaled so that the candidates get clearly different probabilities."""
+    batch = configs.make_batch(2, candidates=31)
+    m = batch["model"]
+    blob, W = gpu_util.default_weights(batch, 77)
+    W["pw2"] *= 400.0
+    blob = configs.pack_weights(m, W)
+    got = gpu_util.run_gpu(batch, blob)
+    want = xo.forward(m, blob, batch)
+    assert want["probs"][0, :31].max() / want["probs"][0, :31].min() > 1.5
+    gpu_util.assert_close(got["probs"], want["probs"], "fp32", "probs")
+
+
+def test_global_attribute_input(xo):
+    import torch
+    import paper_2304_14698_b200 as xrl
+    batch = configs.make_batch(1)
+    m = dict(batch["model"], Dg=3)
+    batch["model"] = m
+    blob, _ = gpu_util.default_weights(batch, 5)
+    g0 = np.random.default_rng(0).normal(size=(8, 3))
+    _, want = _oracle(xo, batch, blob, g0=g0)
+    ag = gpu_util.make_agent(batch)
+    try:
+        ag.set_weights(blob)
+        ag.pack(batch)
+        emb = torch.empty((8, m["H"]), device="cuda")
+        xrl.xrl_encode(ag.ctx, ag.batch, emb, torch.from_numpy(g0.astype(np.float32)).cuda())
+        gpu_util.assert_close(emb.cpu().numpy(), want["emb"], "fp32", "emb with g0")
+    finally:
+        ag.close()
+
+
+@pytest.mark.parametrize("H,K,dtype,L", [(32, 1, "fp32", 1), (32, 4, "bf16", 1), (96, 3, "fp32", 2),
+                                          (96, 2, "bf16", 2), (256, 8, "fp32", 1), (512, 8, "fp32", 1),
+                                          (512, 16, "bf16", 1), (64, 8, "bf16", 0), (128, 2, "bf16", 2)])
+def test_model_shapes(xo, H, K, dtype, L):
+    """Every row geometry of the row-wise kernels (lanes per row, vectors per lane), L = 0."""
+    batch = configs.make_batch(1)
+    if dtype == "bf16":
+        batch["shape"] = dags.round_to_bf16_grid(batch["shape"])
+    m = dict(batch["model"], H=H, K=K, dtype=dtype, L=L, Hm=40)
+    batch["model"] = m
+    blob, _ = gpu_util.default_weights(batch, 9)
+    got = gpu_util.run_gpu(batch, blob)
+    want = xo.forward(m, blob, batch)
+    assert got["status"] == 0
+    gpu_util.assert_close(got["emb"], want["emb"], dtype, "graph_emb")
+    gpu_util.assert_close(got["probs"], want["probs"], dtype, "probs")
+    gpu_util.assert_close(got["value"], want["value"], dtype, "value")
+
+
+def test_degenerate_batches(xo):
+    """Environment without candidates, fully masked environment, empty graph, isolated nodes,
+    a consumer with hundreds of producers, padded action slots."""
+    rng = dags.make_rng(11)
+    n = 400
+    star = {"op": rng.integers(0, 32, n).astype(np.int32), "shape": dags.shape_features(rng, n, 8, False),
+            "edge_src": np.arange(n - 1, dtype=np.int32), "edge_dst": np.full(n - 1, n - 1, np.int32)}
+    iso = {"op": rng.integers(0, 32, 7).astype(np.int32), "shape": dags.shape_features(rng, 7, 8, False),
+           "edge_src": np.zeros(0, np.int32), "edge_dst": np.zeros(0, np.int32)}
+    empty = {"op": np.zeros(0, np.int32), "shape": np.zeros((0, 8), np.float32),
+             "edge_src": np.zeros(0, np.int32), "edge_dst": np.zeros(0, np.int32)}
+    g = [dags.random_dag(rng, 30) for _ in range(4)]
+    graphs = [g[0],                 # env 0: no candidates
+              g[1], star, iso,      # env 1: two candidates, both masked below
+              g[2], empty, g[3], star]   # env 2
+    b = dags.flatten(graphs, [0, 1, 4, 8], 5)
+    b["mask"][1, :] = 0
+    b["model"] = dict(configs.MODEL[1], A_max=5)
+    blob, _ = configs.make_weights(b["model"], 3, readout_scale=0.02)
+    got = gpu_util.run_gpu(b, blob)
+    want = xo.forward(b["model"], blob, b)
+    assert got["status"] == 0
+    gpu_util.assert_close(got["emb"], want["emb"], "fp32", "graph_emb")
+    gpu_util.assert_close(got["probs"], want["probs"], "fp32", "probs")
+    gpu_util.assert_close(got["value"], want["value"], "fp32", "value")
+    assert got["probs"][0, -1] == 1.0 and got["probs"][1, -1] == 1.0
+    assert np.all(got["probs"][want["probs"] == 0] == 0.0)
+
+
+def test_mask_beyond_candidates_raises_device_status():
+    batch = configs.make_batch(1, candidates=5)
+    blob, _ = gpu_util.default_weights(batch, 2)
+    batch["mask"][0, 6] = 1
+    got = gpu_util.run_gpu(batch, blob)
+    assert got["status"] == 1
+    assert got["probs"][0, 6] == 0.0
+
+
+def test_results_are_bitwise_reproducible():
+    batch = configs.make_batch(3, candidates=15)
+    blob, _ = gpu_util.default_weights(batch, 4)
+    a = gpu_util.run_gpu(batch, blob, sample=True, seed=3, step=9)
+    b = gpu_util.run_gpu(batch, blob, sample=True, seed=3, step=9, where="device")
+    for k in ("emb", "probs", "value", "action"):
+        assert np.array_equal(a[k], b[k]), k

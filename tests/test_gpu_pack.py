@@ -1,0 +1,135 @@
+"""GPU parity of the packer (Section 3.3.2): bit-exact against the oracle."""
+import numpy as np
+import pytest
+
+from workloads import configs, dags
+import gpu_util
+
+pytestmark = pytest.mark.gpu
+
+KEYS = ("node_off", "edge_off", "seg_id", "graph_env", "rowptr", "col")
+
+
+def _compare(xo, batch, via):
+    import torch
+    import paper_2304_14698_b200 as xrl
+    st, want = xo.pack(batch)
+    assert st == 0
+    ag = gpu_util.make_agent(batch)
+    try:
+        if via == "graphs":
+            ag.pack_graphs(dags.split(batch), batch["env_off"])
+        elif via == "flat_host":
+            ag.pack(batch)
+        else:
+            dev = {k: batch[k] for k in ("n_nodes", "n_edges", "env_off")}
+            for k in ("op", "edge_src", "edge_dst"):
+                dev[k] = torch.from_numpy(batch[k]).cuda()
+            shp = torch.from_numpy(batch["shape"]).cuda()
+            dev["shape"] = shp.to(torch.bfloat16) if batch["model"]["dtype"] == "bf16" else shp
+            ag.pack(dev)
+        got = xrl.xrl_batch_export(ag.batch)
+        assert ag.device_status() == 0
+        info = xrl.xrl_batch_info(ag.batch)
+        assert info["num_nodes"] == batch["n_nodes"].sum() and info["num_edges"] == batch["n_edges"].sum()
+        for k in KEYS:
+            assert np.array_equal(got[k], want[k]), k
+    finally:
+        ag.close()
+
+
+@pytest.mark.parametrize("via", ["graphs", "flat_host", "flat_device"])
+@pytest.mark.parametrize("cfg,kw", [(1, {}), (2, {}), (3, dict(candidates=31)), (4, dict(candidates=15)),
+                                    (5, dict(candidates=7, envs=5))])
+def test_pack_bit_exact(xo, cfg, kw, via):
+    _compare(xo, configs.make_batch(cfg, **kw), via)
+
+
+def test_pack_shuffled_edges_long_rows_and_empty_graphs(xo):
+    rng = np.random.default_rng(0)
+    n = 700
+    star = {"op": np.zeros(n, np.int32), "shape": np.zeros((n, 8), np.float32),
+            # 3 consumers with 40, 33 and 600 producers (rows beyond the one-thread path), repeats included
+            "edge_src": np.concatenate([rng.integers(0, 50, 40), rng.integers(0, 50, 33),
+                                        rng.integers(0, 690, 600)]).astype(np.int32),
+            "edge_dst": np.concatenate([np.full(40, 697), np.full(33, 698), np.full(600, 699)]).astype(np.int32)}
+    perm = rng.permutation(len(star["edge_src"]))
+    star["edge_src"], star["edge_dst"] = star["edge_src"][perm], star["edge_dst"][perm]
+    empty = {"op": np.zeros(0, np.int32), "shape": np.zeros((0, 8), np.float32),
+             "edge_src": np.zeros(0, np.int32), "edge_dst": np.zeros(0, np.int32)}
+    iso = {"op": np.ones(5, np.int32), "shape": np.zeros((5, 8), np.float32),
+           "edge_src": np.zeros(0, np.int32), "edge_dst": np.zeros(0, np.int32)}
+    small = dags.random_dag(dags.make_rng(1), 64)
+    p2 = rng.permutation(len(small["edge_src"]))
+    small["edge_src"], small["edge_dst"] = small["edge_src"][p2], small["edge_dst"][p2]
+    b = dags.flatten([small, empty, star, iso, empty], [0, 2, 5], 4)
+    b["model"] = dict(configs.MODEL[1], A_max=4)
+    for via in ("graphs", "flat_device"):
+        _compare(xo, b, via)
+
+
+def test_pack_large_scan_spans_many_tiles(xo):
+    # > 2048 graphs and > 2048*... nodes so that both scans take the multi-level path
+    rng = dags.make_rng(3)
+    graphs = [dags.random_dag(rng, int(rng.integers(1, 40)), 32, 8, False, window=8) for _ in range(2500)]
+    b = dags.flatten(graphs, [0, 1000, 2500], 1600)
+    b["model"] = dict(configs.MODEL[1], A_max=1600)
+    _compare(xo, b, "flat_host")
+
+
+def test_pack_reports_bad_graphs_in_the_device_status(xo):
+    import paper_2304_14698_b200 as xrl
+    base = configs.make_batch(1)
+    for k, idx, val in [("edge_src", 3, 64), ("edge_dst", 10, -1), ("op", 5, 32), ("self", 7, 0)]:
+        b = {kk: (v.copy() if isinstance(v, np.ndarray) else v) for kk, v in base.items()}
+        if k == "self":
+            b["edge_src"][idx] = b["edge_dst"][idx]
+        else:
+            b[k][idx] = val
+        ag = gpu_util.make_agent(b)
+        try:
+            ag.pack(b)
+            assert ag.device_status() == 2
+            assert ag.device_status() == 0        # reading clears it
+        finally:
+            ag.close()
+
+
+def test_pack_argument_and_capacity_errors():
+    import paper_2304_14698_b200 as xrl
+    b = configs.make_batch(1)
+    ag = gpu_util.make_agent(b)
+    try:
+        with pytest.raises(xrl.XrlError) as e:
+            ag.pack(dict(b, env_off=np.array([0, 9], np.int32)))
+        assert e.value.status == 1
+        big = configs.make_batch(1, candidates=8)
+        with pytest.raises(xrl.XrlError) as e:
+            ag.pack(big)
+        assert e.value.status == 3
+        # encode before weights are set
+        ag.pack(b)
+        import torch
+        with pytest.raises(xrl.XrlError) as e:
+            xrl.xrl_encode(ag.ctx, ag.batch, torch.empty((8, 64), device="cuda"))
+        assert e.value.status == 6
+    finally:
+        ag.close()
+
+
+def test_repack_in_place_reuses_the_batch(xo):
+    import paper_2304_14698_b200 as xrl
+    b1 = configs.make_batch(2, candidates=9, seed=5)
+    b2 = configs.make_batch(2, candidates=9, seed=6)
+    ag = gpu_util.make_agent(b1, slack=64)
+    try:
+        ag.pack(b1)
+        h1 = ag.batch.value
+        ag.pack(b2)
+        assert ag.batch.value == h1
+        got = xrl.xrl_batch_export(ag.batch)
+        _, want = xo.pack(b2)
+        for k in KEYS:
+            assert np.array_equal(got[k], want[k]), k
+    finally:
+        ag.close()
