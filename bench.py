@@ -1,0 +1,352 @@
+#!/usr/bin/env python
+"""Benchmark of the agent's per-step forward pass (pack -> encode -> policy/value -> sample).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl reference]
+
+One step = one pass of the whole path over one synthetic batch.  Prints ONE JSON line.
+With --impl reference the CPU oracle is timed instead (a deliberately plain program).
+Under torchrun each rank runs its own batch (no data-path collective: graphs of different
+environments never interact); the time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workloads import configs  # noqa: E402
+
+FALLBACK_HBM_GBS = 6650.0
+
+
+def rank_info():
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")),
+            int(os.environ.get("WORLD_SIZE", "1")))
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def algorithmic_bytes(family, m, N, E):
+    """Compulsory HBM bytes of one launch of a kernel family (gathers of a row beyond its first
+    touch are counted as L2 traffic, not HBM)."""
+    b = 2 if m["dtype"] == "bf16" else 4
+    H, K, S = m["H"], m["K"], m["S"]
+    if family == "transform":        # read h, write Z, write both half-scores
+        return N * (2 * H * b + 2 * K * 4)
+    if family == "aggregate":        # read Z once, write h', rowptr, both half-scores, col per edge
+        return N * (2 * H * b + 4 + 2 * K * 4) + 4 * E
+    if family == "node_update":      # read shape + op + rowptr, write h0, col per edge
+        return N * (S * b + 4 + 4 + H * b) + 4 * E
+    if family == "readout":
+        return N * H * b
+    if family == "pack":             # read edge lists twice + op, write col/seg_id/rowptr/tmp
+        return E * (2 * 8 + 4 + 4 + 4) + N * (4 + 4 + 4 + 4)
+    return 0
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(mx)) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample_run(batch, blob, graphs, threads):
+    """Time the CPU oracle (as it stands) on `graphs` whole graphs of the workload.  Returns
+    (seconds, threads used).  The heads are evaluated on the sampled graphs' environment only if
+    the sample covers it; the encoder dominates either way."""
+    from oracle import xrl_oracle as xo
+    m = batch["model"]
+    st, packed = xo.pack(batch)
+    assert st == 0
+    sel = np.arange(min(graphs, batch["num_graphs"]), dtype=np.int32)
+    t0 = time.perf_counter()
+    xo.encode(m, blob, batch, packed, sel=sel, threads=threads)
+    dt = time.perf_counter() - t0
+    return dt, len(sel)
+
+
+def run_reference(args, cfg_id):
+    """--impl reference: the CPU oracle on a bounded sample of the same workload."""
+    rank, _, world = rank_info()
+    if rank != 0:
+        return
+    from oracle import xrl_oracle as xo
+    cores = os.cpu_count() or 1
+    threads = min(cores, xo.num_threads())
+    sample_graphs = {1: 8, 2: 64, 3: 64, 4: max(16, 2 * threads), 5: max(32, 2 * threads)}[cfg_id]
+    cand = max(1, sample_graphs - 1)
+    batch = configs.make_batch(cfg_id, candidates=min(cand, configs.FULL[cfg_id][0]), envs=1)
+    m = batch["model"]
+    blob, _ = configs.make_weights(m, 1000 + cfg_id, readout_scale=1.0 / float(batch["n_nodes"].mean()))
+    E_sample = int(batch["n_edges"].sum())
+    def one_step():
+        t0 = time.perf_counter()
+        xo.forward(m, blob, batch, threads=threads)         # pack -> encode -> heads
+        return time.perf_counter() - t0
+
+    for _ in range(min(args.warmup, 1)):
+        one_step()
+    times = [one_step() for _ in range(args.steps)]
+    t = float(np.mean(times))
+    gps = batch["num_graphs"] / t
+    sample = (f"{batch['num_graphs']} whole graphs of workload {configs.NAME[cfg_id]} "
+              f"({int(batch['n_nodes'].sum())} nodes, {E_sample} edges) per step, whole path")
+    line = {
+        "impl": "reference", "metric": "graphs_encoded_per_s", "value": gps, "unit": "graphs/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "edges_per_s": E_sample / t,
+        "config": {"workload": configs.NAME[cfg_id], "sample": sample},
+        "cpu_baseline": {"value": gps, "unit": "graphs/s", "cores": threads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": gps, "unit": "graphs/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=4, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--impl", default="xrl", choices=["xrl", "reference"])
+    ap.add_argument("--candidates", type=int, default=None, help="shrink the workload (profiling)")
+    ap.add_argument("--envs", type=int, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    cfg_id = args.config
+    rank, local_rank, world = rank_info()
+
+    if args.impl == "reference":
+        run_reference(args, cfg_id)
+        return
+
+    warmup = max(3, args.warmup)
+    batch = configs.make_batch(cfg_id, candidates=args.candidates, envs=args.envs, seed=cfg_id + 100 * rank)
+    m = batch["model"]
+    N, E, B = int(batch["n_nodes"].sum()), int(batch["n_edges"].sum()), int(batch["num_graphs"])
+    Ne = len(batch["env_off"]) - 1
+    blob, _ = configs.make_weights(m, 1000 + cfg_id, readout_scale=1.0 / float(batch["n_nodes"].mean()))
+
+    # ---- CPU baseline first (before the first CUDA call): the oracle on a bounded sample ----------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import xrl_oracle as xo
+        threads = min(os.cpu_count() or 1, xo.num_threads())
+        n_s = min(B, {1: 8, 2: 64, 3: 64}.get(cfg_id, max(16, 2 * threads)))
+        dt, g = oracle_sample_run(batch, blob, n_s, threads)
+        no = np.concatenate([[0], np.cumsum(batch["n_nodes"])]); eo = np.concatenate([[0], np.cumsum(batch["n_edges"])])
+        cpu = {"value": g / dt, "unit": "graphs/s", "cores": threads, "kind": "oracle",
+               "sample": f"first {g} graphs of the same batch ({int(no[g])} nodes, {int(eo[g])} edges), "
+                         f"encoder + readout, {dt:.1f} s", "edges_per_s": float(eo[g]) / dt}
+
+    import torch
+    import paper_2304_14698_b200 as xrl
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    agent = xrl.Agent(m, B, Ne, N, E, device=local_rank)
+    agent.set_weights(blob)
+    bf16 = m["dtype"] == "bf16"
+    dev = {k: batch[k] for k in ("n_nodes", "n_edges", "env_off")}
+    dev["op"] = torch.from_numpy(batch["op"]).cuda()
+    shp = torch.from_numpy(batch["shape"]).cuda()
+    dev["shape"] = shp.to(torch.bfloat16) if bf16 else shp
+    dev["edge_src"] = torch.from_numpy(batch["edge_src"]).cuda()
+    dev["edge_dst"] = torch.from_numpy(batch["edge_dst"]).cuda()
+    mask_d = torch.from_numpy(batch["mask"]).cuda()
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def device_step(i):
+        return agent.step(dev, mask_d, sample=True, seed=cfg_id, step=i)
+
+    for i in range(warmup):
+        device_step(i)
+    torch.cuda.synchronize()
+    assert agent.device_status() == 0, "device status after warm-up"
+
+    # ---- timed region: device-resident inputs -----------------------------------------------------
+    xrl.xrl_profile(agent.ctx, True)
+    clocks = ClockSampler(local_rank)
+    clocks.start()
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for i in range(args.steps):
+        device_step(warmup + i)
+    ev1.record(stream)
+    barrier()
+    elapsed_ms = ev0.elapsed_time(ev1)
+    clock_info = clocks.stop()
+    prof = xrl.xrl_profile_read(agent.ctx)
+    xrl.xrl_profile(agent.ctx, False)
+    launches = xrl.xrl_launch_counts(agent.ctx)
+    status = agent.device_status()
+    assert status == 0, f"device status {status}"
+
+    # ---- end to end: host buffers in, results out, through the public call ---------------------------
+    e2e = None
+    if not args.no_e2e:
+        host = {k: batch[k] for k in ("n_nodes", "n_edges", "env_off", "op", "edge_src", "edge_dst")}
+        host["shape"] = agent.storage_shape(batch["shape"])
+        mask_h = torch.from_numpy(batch["mask"]).pin_memory()
+        h2d = sum(host[k].nbytes for k in ("op", "edge_src", "edge_dst", "shape", "n_nodes", "n_edges",
+                                           "env_off")) + batch["mask"].nbytes
+        outs_h = None
+
+        def host_step(i):
+            nonlocal outs_h
+            agent.batch = xrl.xrl_pack_flat(agent.ctx, 0, host["n_nodes"], host["n_edges"], host["op"],
+                                            host["shape"], host["edge_src"], host["edge_dst"],
+                                            host["env_off"], batch=agent.batch)
+            md = mask_h.cuda(non_blocking=True)
+            o = agent.forward(md, sample=True, seed=cfg_id, step=i)
+            outs_h = (o["probs"].cpu(), o["value"].cpu(), o["action"].cpu())   # device -> host, syncs
+
+        e2e_steps = max(1, min(args.steps, 5))
+        for i in range(2):
+            host_step(i)
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            host_step(i)
+        barrier()
+        e2e_s = (time.perf_counter() - t0) / e2e_steps
+        d2h = sum(t.numel() * t.element_size() for t in outs_h)
+        e2e = {"s_per_step": e2e_s, "h2d": int(h2d), "d2h": int(d2h)}
+
+    # ---- reduce over ranks -----------------------------------------------------------------------------
+    tot_graphs, tot_edges, tot_nodes = B, E, N
+    if world > 1:
+        t = torch.tensor([elapsed_ms, e2e["s_per_step"] if e2e else 0.0], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t[0]);
+        if e2e:
+            e2e["s_per_step"] = float(t[1])
+        c = torch.tensor([B, E, N], device="cuda", dtype=torch.int64)
+        dist.all_reduce(c, op=dist.ReduceOp.SUM)
+        tot_graphs, tot_edges, tot_nodes = (int(v) for v in c)
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    ms_per_step = elapsed_ms / args.steps
+    peak, peak_kind = measured_peaks()
+    fam_ms = {f: (v["ms"] / args.steps) for f, v in prof.items()}
+    dominant = max(("transform", "aggregate", "node_update", "readout", "pack"), key=lambda f: fam_ms[f])
+    per_step_launches = max(1, prof[dominant]["launches"] // args.steps)
+    dom_ms = fam_ms[dominant] / per_step_launches
+    alg = algorithmic_bytes(dominant, m, N, E)
+    achieved = alg / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
+    step_alg = (algorithmic_bytes("pack", m, N, E) + algorithmic_bytes("node_update", m, N, E) +
+                m["L"] * (algorithmic_bytes("transform", m, N, E) + algorithmic_bytes("aggregate", m, N, E)) +
+                algorithmic_bytes("readout", m, N, E))
+    line = {
+        "metric": "graphs_encoded_per_s", "value": tot_graphs / (ms_per_step * 1e-3), "unit": "graphs/s",
+        "n_gpus": world, "steps": args.steps, "warmup": warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
+        "edges_per_s": tot_edges / (ms_per_step * 1e-3),
+        "config": {"workload": configs.NAME[cfg_id], "graphs": B, "envs": Ne, "nodes": N, "edges": E,
+                   "hidden": m["H"], "heads": m["K"], "gat_layers": m["L"], "actions": m["A_max"] + 1,
+                   "per_rank": world > 1, "l2": "inputs and activations larger than L2 (no flush needed)"
+                   if N * m["H"] * (2 if bf16 else 4) > 200e6 else "working set below L2 size"},
+        "clocks": clock_info,
+        "gpu_launches": int(args.steps * (launches["pack"] + launches["encode"] + launches["heads"])),
+        "kernel_ms_per_step": {f: round(v, 4) for f, v in fam_ms.items()},
+        "step_hbm_frac": step_alg / (ms_per_step * 1e-3) / 1e9 / peak,
+        "roofline": {"kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peak,
+                     "peak_source": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": TRAFFIC.get((cfg_id, dominant)) if args.candidates is None else None,
+                     "algorithmic_bytes": int(alg), "launch_ms": dom_ms},
+    }
+    if e2e:
+        line["e2e"] = {"value": tot_graphs / e2e["s_per_step"], "unit": "graphs/s",
+                       "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                       "ms_per_step": e2e["s_per_step"] * 1e3}
+    if cpu:
+        line["cpu_baseline"] = cpu
+    print(json.dumps(line))
+    agent.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from the
+# ncu capture summarised under profiles/; filled in once a capture of the current kernel exists.
+TRAFFIC = {}
+
+if __name__ == "__main__":
+    main()

@@ -189,6 +189,16 @@ xrl_status xrl_last_device_status(xrl_ctx* ctx, void* stream, int32_t* status);
  * this context and how many launches each call made (HOST outputs, any may be NULL). */
 xrl_status xrl_launch_counts(const xrl_ctx* ctx, int64_t* pack, int64_t* encode, int64_t* heads);
 
+/* Per-step timing of the path's steps with CUDA events on the launching stream (off by
+ * default).  Families: 0 pack (Section 3.3.2), 1 node update (Eq. 6), 2 transform and 3
+ * score/softmax/aggregate (Eq. 7), 4 readout (Eq. 8 sum), 5 global update + heads.
+ * xrl_profile(ctx, 1) starts recording (synchronises the device, drops earlier records);
+ * xrl_profile_read synchronises the device, fills total_ms / launches (HOST,
+ * [num_families]) with the time and kernel count accumulated per family since the last read,
+ * and clears the records. */
+xrl_status xrl_profile(xrl_ctx* ctx, int32_t enable);
+xrl_status xrl_profile_read(xrl_ctx* ctx, double* total_ms, int64_t* launches, int32_t num_families);
+
 /* Static description of the build ("sm_100a ...").  Never NULL. */
 const char* xrl_version(void);
 

@@ -24,7 +24,9 @@ EXPORTED_SYMBOLS = [
     "xrl_create", "xrl_destroy", "xrl_weights_size", "xrl_set_weights", "xrl_pack", "xrl_pack_flat",
     "xrl_batch_free", "xrl_batch_info", "xrl_batch_export", "xrl_encode", "xrl_debug_node_features",
     "xrl_policy_value", "xrl_sample", "xrl_last_device_status", "xrl_launch_counts", "xrl_version",
+    "xrl_profile", "xrl_profile_read",
 ]
+PROFILE_FAMILIES = ["pack", "node_update", "transform", "aggregate", "readout", "heads"]
 
 
 class XrlError(RuntimeError):
@@ -76,6 +78,8 @@ def load_library():
         "xrl_sample": [vp, vp, i32, i32, u64, u64, vp, vp],
         "xrl_last_device_status": [vp, vp, C.POINTER(i32)],
         "xrl_launch_counts": [vp, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64)],
+        "xrl_profile": [vp, i32],
+        "xrl_profile_read": [vp, C.POINTER(C.c_double), C.POINTER(i64), i32],
     }
     for name, args in sigs.items():
         fn = getattr(lib, name)
@@ -250,6 +254,18 @@ def xrl_launch_counts(ctx):
     a, b, c = C.c_int64(), C.c_int64(), C.c_int64()
     _check(load_library().xrl_launch_counts(ctx, C.byref(a), C.byref(b), C.byref(c)), "xrl_launch_counts")
     return {"pack": a.value, "encode": b.value, "heads": c.value}
+
+
+def xrl_profile(ctx, enable: bool):
+    _check(load_library().xrl_profile(ctx, 1 if enable else 0), "xrl_profile")
+
+
+def xrl_profile_read(ctx):
+    n = len(PROFILE_FAMILIES)
+    ms = (C.c_double * n)()
+    cnt = (C.c_int64 * n)()
+    _check(load_library().xrl_profile_read(ctx, ms, cnt, n), "xrl_profile_read")
+    return {f: {"ms": ms[i], "launches": cnt[i]} for i, f in enumerate(PROFILE_FAMILIES)}
 
 
 # ---- the call a user makes --------------------------------------------------------------------

@@ -30,7 +30,38 @@ size_t storage_bytes(int dtype) { return dtype == XRL_BF16 ? 2 : 4; }
 
 }  // namespace
 
+// Optional per-kernel-family timing: CUDA events recorded on the launching stream around every
+// launcher call.  Families index the steps of the path.
+enum { FAM_PACK = 0, FAM_EMBED, FAM_XFORM, FAM_AGG, FAM_READOUT, FAM_HEADS, FAM_COUNT };
+
+struct Profiler {
+  bool on = false;
+  std::vector<cudaEvent_t> pool;
+  size_t used = 0;
+  struct Rec { int fam; size_t a, b; int launches; };
+  std::vector<Rec> recs;
+  size_t begin(cudaStream_t st) {
+    if (!on) return 0;
+    if (used + 2 > pool.size()) {
+      cudaEvent_t e0, e1;
+      if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) { on = false; return 0; }
+      pool.push_back(e0); pool.push_back(e1);
+    }
+    cudaEventRecord(pool[used], st);
+    used += 2;
+    return used - 2;
+  }
+  void end(int fam, size_t slot, int launches, cudaStream_t st) {
+    if (!on) return;
+    cudaEventRecord(pool[slot + 1], st);
+    recs.push_back(Rec{fam, slot, slot + 1, launches});
+  }
+  void clear() { used = 0; recs.clear(); }
+  void release() { for (cudaEvent_t e : pool) cudaEventDestroy(e); pool.clear(); clear(); }
+};
+
 struct xrl_ctx {
+  Profiler prof;
   xrl_model_config cfg;
   Dims dims;
   int device = 0;
@@ -282,7 +313,11 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
   po.deg = b->deg.as<int32_t>(); po.tmp_eid = b->tmp_eid.as<int32_t>();
   po.long_rows = b->long_rows.as<int32_t>(); po.long_count = b->long_count.as<int32_t>();
   po.scan_ws = b->scan_ws.as<int32_t>();
-  ctx->launches_pack = launch_pack(in, po, c.num_op_types, ctx->status.as<int32_t>(), st);
+  {
+    const size_t slot = ctx->prof.begin(st);
+    ctx->launches_pack = launch_pack(in, po, c.num_op_types, ctx->status.as<int32_t>(), st);
+    ctx->prof.end(FAM_PACK, slot, int(ctx->launches_pack), st);
+  }
   XRL_CUDA(cudaGetLastError());
 
   b->B = num_graphs; b->num_envs = num_envs; b->N = int32_t(N); b->E = int32_t(E);
@@ -294,14 +329,24 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
 int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t st) {
   const Dims& d = ctx->dims;
   const Window win{0, b->N, 0};
-  int n = launch_embed(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), b->op.as<int32_t>(),
+  Profiler& pf = ctx->prof;
+  size_t slot = pf.begin(st);
+  int k = launch_embed(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), b->op.as<int32_t>(),
                        b->shape.p, ctx->dw, ctx->h.p, win, st);
+  pf.end(FAM_EMBED, slot, k, st);
+  int n = k;
   for (int l = 0; l < layers; ++l) {
-    n += launch_xform_simt(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->s_src.as<float>(),
-                           ctx->s_dst.as<float>(), win, st);
-    n += launch_aggregate(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), ctx->Z.p,
-                          ctx->s_src.as<float>(), ctx->s_dst.as<float>(), ctx->dw.layer[l].b,
-                          ctx->h.p, win, st);
+    slot = pf.begin(st);
+    k = launch_xform_simt(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->s_src.as<float>(),
+                          ctx->s_dst.as<float>(), win, st);
+    pf.end(FAM_XFORM, slot, k, st);
+    n += k;
+    slot = pf.begin(st);
+    k = launch_aggregate(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), ctx->Z.p,
+                         ctx->s_src.as<float>(), ctx->s_dst.as<float>(), ctx->dw.layer[l].b,
+                         ctx->h.p, win, st);
+    pf.end(FAM_AGG, slot, k, st);
+    n += k;
   }
   return n;
 }
@@ -367,6 +412,7 @@ void xrl_destroy(xrl_ctx* ctx) {
   DeviceBuf* bufs[] = {&ctx->w_f32, &ctx->w_store, &ctx->h, &ctx->Z, &ctx->s_src, &ctx->s_dst,
                        &ctx->partial, &ctx->logits, &ctx->status};
   for (DeviceBuf* d : bufs) d->release();
+  ctx->prof.release();
   delete ctx;
 }
 
@@ -477,10 +523,16 @@ xrl_status xrl_encode(xrl_ctx* ctx, const xrl_batch* b, const float* g0, float* 
   XRL_CUDA(cudaSetDevice(ctx->device));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int n = run_node_layers(ctx, b, ctx->cfg.layers, st);
-  n += launch_readout(ctx->dims, ctx->h.p, b->d_chunk_row0, b->d_chunk_row1, 0, b->num_chunks,
-                      ctx->partial.as<float>(), 0, st);
-  n += launch_global_update(ctx->dims, ctx->partial.as<float>(), b->d_graph_chunk_off, g0, ctx->dw,
-                            graph_emb, b->B, st);
+  size_t slot = ctx->prof.begin(st);
+  int k = launch_readout(ctx->dims, ctx->h.p, b->d_chunk_row0, b->d_chunk_row1, 0, b->num_chunks,
+                         ctx->partial.as<float>(), 0, st);
+  ctx->prof.end(FAM_READOUT, slot, k, st);
+  n += k;
+  slot = ctx->prof.begin(st);
+  k = launch_global_update(ctx->dims, ctx->partial.as<float>(), b->d_graph_chunk_off, g0, ctx->dw,
+                           graph_emb, b->B, st);
+  ctx->prof.end(FAM_HEADS, slot, k, st);
+  n += k;
   ctx->launches_encode = n;
   XRL_CUDA(cudaGetLastError());
   return XRL_OK;
@@ -516,9 +568,11 @@ xrl_status xrl_policy_value(xrl_ctx* ctx, const xrl_batch* b, const float* graph
     return XRL_ERR_INVALID_ARG;
   XRL_CUDA(cudaSetDevice(ctx->device));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t slot = ctx->prof.begin(st);
   ctx->launches_heads = launch_heads(ctx->dims, ctx->dw, graph_emb, b->d_env_off, mask, b->B, b->num_envs,
                                      ctx->logits.as<float>(), probs, value, action, seed, step,
                                      ctx->status.as<int32_t>(), st);
+  ctx->prof.end(FAM_HEADS, slot, int(ctx->launches_heads), st);
   XRL_CUDA(cudaGetLastError());
   return XRL_OK;
 }
@@ -540,6 +594,29 @@ xrl_status xrl_last_device_status(xrl_ctx* ctx, void* stream, int32_t* status) {
   XRL_CUDA(cudaStreamSynchronize(st));
   XRL_CUDA(cudaMemcpy(status, ctx->status.p, 4, cudaMemcpyDeviceToHost));
   XRL_CUDA(cudaMemset(ctx->status.p, 0, 4));
+  return XRL_OK;
+}
+
+xrl_status xrl_profile(xrl_ctx* ctx, int32_t enable) {
+  if (!ctx) return XRL_ERR_INVALID_ARG;
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  XRL_CUDA(cudaDeviceSynchronize());
+  ctx->prof.clear();
+  ctx->prof.on = enable != 0;
+  return XRL_OK;
+}
+
+xrl_status xrl_profile_read(xrl_ctx* ctx, double* total_ms, int64_t* launches, int32_t num_families) {
+  if (!ctx || !total_ms || !launches || num_families < 0) return XRL_ERR_INVALID_ARG;
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  XRL_CUDA(cudaDeviceSynchronize());
+  for (int f = 0; f < num_families; ++f) { total_ms[f] = 0.0; launches[f] = 0; }
+  for (const Profiler::Rec& r : ctx->prof.recs) {
+    float ms = 0.f;
+    XRL_CUDA(cudaEventElapsedTime(&ms, ctx->prof.pool[r.a], ctx->prof.pool[r.b]));
+    if (r.fam < num_families) { total_ms[r.fam] += ms; launches[r.fam] += r.launches; }
+  }
+  ctx->prof.clear();
   return XRL_OK;
 }
 
