@@ -189,6 +189,48 @@ xrl_status xrl_last_device_status(xrl_ctx* ctx, void* stream, int32_t* status);
  * this context and how many launches each call made (HOST outputs, any may be NULL). */
 xrl_status xrl_launch_counts(const xrl_ctx* ctx, int64_t* pack, int64_t* encode, int64_t* heads);
 
+/* ---- packing for callers that must not allocate ------------------------------------------------ */
+
+/* (No counterpart in the paper: this is a deployment variant of the packer above.)
+ *
+ * Some programs that embed this library are not allowed to ask CUDA for memory while they run:
+ * an inference server whose own pool already holds the whole GPU (a cudaMalloc there fails, or
+ * stalls every stream while the driver synchronises the device), a control loop with a latency
+ * budget that a device-wide synchronisation would break, or a plug-in whose host forbids driver
+ * allocations from callbacks.  xrl_create / xrl_pack allocate (context workspace, batch, pinned
+ * staging), so those programs cannot use them.  This call builds the same packed index arrays
+ * with NO allocation of any kind: no context, no batch object, and the packer's scratch (in-degree
+ * counters, row cursors, the unsorted edge slots, scan partial sums, a device copy of the counts)
+ * sits in a fixed array inside the library image, about 2.7 MB that every GPU loading the library
+ * keeps until the process exits.  The price is a size limit:
+ *     num_graphs <= XRL_STATIC_PACK_MAX_GRAPHS, num_envs <= XRL_STATIC_PACK_MAX_ENVS,
+ *     total nodes <= XRL_STATIC_PACK_MAX_NODES, total edges <= XRL_STATIC_PACK_MAX_EDGES;
+ * anything larger is refused with XRL_ERR_CAPACITY before any work is queued (the paper's own
+ * steps, 13-50 candidates of a few hundred to a few thousand operators, fit).
+ *
+ * Arguments: n_nodes, n_edges [num_graphs] and env_off [num_envs + 1] are HOST (read before the
+ * call returns); op [N], edge_src [E], edge_dst [E] are DEVICE inputs with the meaning they have
+ * in xrl_pack_flat; node_off [B+1], edge_off [B+1], seg_id [N], graph_env [B], rowptr [N+1],
+ * col [E] and device_status [1] are DEVICE outputs owned by the caller.  device_status receives
+ * XRL_OK or XRL_ERR_BAD_GRAPH once the stream has run the work.  `device` is the CUDA device the
+ * pointers belong to; the call makes it current.
+ *
+ * The first call on each device looks up the device address of the built-in array once
+ * (cudaGetSymbolAddress); make that first call before you begin any stream capture.  All calls on
+ * a device share the one array and it keeps whatever the previous call left there (the kernels
+ * re-zero the counters they need), so two calls must never overlap on the GPU: issue them on one
+ * stream, or order them with events.  Overlapping calls race and corrupt each other's result. */
+#define XRL_STATIC_PACK_MAX_GRAPHS 4096
+#define XRL_STATIC_PACK_MAX_ENVS 1024
+#define XRL_STATIC_PACK_MAX_NODES 131072
+#define XRL_STATIC_PACK_MAX_EDGES 524288
+xrl_status xrl_pack_csr_static(int32_t device, int32_t num_op_types, int32_t num_graphs,
+                               const int32_t* n_nodes, const int32_t* n_edges, const int32_t* op,
+                               const int32_t* edge_src, const int32_t* edge_dst,
+                               const int32_t* env_off, int32_t num_envs, int32_t* node_off,
+                               int32_t* edge_off, int32_t* seg_id, int32_t* graph_env,
+                               int32_t* rowptr, int32_t* col, int32_t* device_status, void* stream);
+
 /* Per-step timing of the path's steps with CUDA events on the launching stream (off by
  * default).  Families: 0 pack (Section 3.3.2), 1 node update (Eq. 6), 2 transform and 3
  * score/softmax/aggregate (Eq. 7), 4 readout (Eq. 8 sum), 5 global update + heads.

@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = [
     "xrl_create", "xrl_destroy", "xrl_weights_size", "xrl_set_weights", "xrl_pack", "xrl_pack_flat",
     "xrl_batch_free", "xrl_batch_info", "xrl_batch_export", "xrl_encode", "xrl_debug_node_features",
     "xrl_policy_value", "xrl_sample", "xrl_last_device_status", "xrl_launch_counts", "xrl_version",
-    "xrl_profile", "xrl_profile_read",
+    "xrl_profile", "xrl_profile_read", "xrl_pack_csr_static",
 ]
 PROFILE_FAMILIES = ["pack", "node_update", "transform", "aggregate", "readout", "heads"]
 
@@ -79,6 +79,7 @@ def load_library():
         "xrl_last_device_status": [vp, vp, C.POINTER(i32)],
         "xrl_launch_counts": [vp, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64)],
         "xrl_profile": [vp, i32],
+        "xrl_pack_csr_static": [i32, i32, i32] + [vp] * 6 + [i32] + [vp] * 8,
         "xrl_profile_read": [vp, C.POINTER(C.c_double), C.POINTER(i64), i32],
     }
     for name, args in sigs.items():
@@ -266,6 +267,26 @@ def xrl_profile_read(ctx):
     cnt = (C.c_int64 * n)()
     _check(load_library().xrl_profile_read(ctx, ms, cnt, n), "xrl_profile_read")
     return {f: {"ms": ms[i], "launches": cnt[i]} for i, f in enumerate(PROFILE_FAMILIES)}
+
+
+def xrl_pack_csr_static(device, num_op_types, n_nodes, n_edges, op, edge_src, edge_dst, env_off,
+                        node_off, edge_off, seg_id, graph_env, rowptr, col, device_status, stream=None):
+    """Packer variant for callers that may not allocate device memory (see include/xrl.h).
+
+    Counts and env_off are numpy int32 (host); every other array is a torch CUDA int32 tensor the
+    caller allocated beforehand (inputs op/edge_src/edge_dst, outputs the packed arrays and a
+    one-element status).  Nothing is allocated by the call; batches beyond the XRL_STATIC_PACK_MAX_*
+    limits raise XrlError(XRL_ERR_CAPACITY).  Calls share one built-in scratch array per GPU, so
+    keep them on one stream."""
+    n_nodes = np.ascontiguousarray(n_nodes, dtype=np.int32)
+    n_edges = np.ascontiguousarray(n_edges, dtype=np.int32)
+    env_off = np.ascontiguousarray(env_off, dtype=np.int32)
+    st = load_library().xrl_pack_csr_static(
+        device, num_op_types, len(n_nodes), _np_ptr(n_nodes), _np_ptr(n_edges), _dev_ptr(op),
+        _dev_ptr(edge_src), _dev_ptr(edge_dst), _np_ptr(env_off), len(env_off) - 1, _dev_ptr(node_off),
+        _dev_ptr(edge_off), _dev_ptr(seg_id), _dev_ptr(graph_env), _dev_ptr(rowptr), _dev_ptr(col),
+        _dev_ptr(device_status), _stream(stream))
+    _check(st, "xrl_pack_csr_static")
 
 
 # ---- the call a user makes --------------------------------------------------------------------

@@ -236,3 +236,87 @@ int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cu
 }
 
 }  // namespace xrl
+
+// ---- packing without any allocation -----------------------------------------------------------
+// Scratch for xrl_pack_csr_static lives in the library image instead of in memory obtained at run
+// time.  Layout (int32 words): n_nodes[G] n_edges[G] env_off[V+1] deg[N] tmp_eid[E] long_rows[E/32+1]
+// long_count[1] scan workspace[kStaticScanInts], with G/V/N/E the maxima below.
+namespace {
+
+constexpr int64_t kStG = XRL_STATIC_PACK_MAX_GRAPHS, kStV = XRL_STATIC_PACK_MAX_ENVS,
+                  kStN = XRL_STATIC_PACK_MAX_NODES, kStE = XRL_STATIC_PACK_MAX_EDGES;
+constexpr int64_t kStaticScanInts = 1024;
+constexpr int64_t kOffNn = 0, kOffNe = kOffNn + kStG, kOffEnv = kOffNe + kStG, kOffDeg = kOffEnv + kStV + 1,
+                  kOffTmp = kOffDeg + kStN, kOffLong = kOffTmp + kStE, kOffCount = kOffLong + kStE / 32 + 1,
+                  kOffScan = kOffCount + 1, kStaticInts = kOffScan + kStaticScanInts;
+
+static __device__ __align__(256) int32_t g_pack_scratch[kStaticInts];
+
+constexpr int kMaxDevices = 64;
+int32_t* g_pack_scratch_addr[kMaxDevices] = {};   // device address of the array, per device
+
+}  // namespace
+
+extern "C" xrl_status xrl_pack_csr_static(int32_t device, int32_t num_op_types, int32_t num_graphs,
+                                          const int32_t* n_nodes, const int32_t* n_edges,
+                                          const int32_t* op, const int32_t* edge_src,
+                                          const int32_t* edge_dst, const int32_t* env_off,
+                                          int32_t num_envs, int32_t* node_off, int32_t* edge_off,
+                                          int32_t* seg_id, int32_t* graph_env, int32_t* rowptr,
+                                          int32_t* col, int32_t* device_status, void* stream) {
+  using namespace xrl;
+  if (device < 0 || device >= kMaxDevices || num_op_types < 1 || num_graphs < 0 || num_envs < 0 ||
+      !env_off || !node_off || !edge_off || !rowptr || !device_status ||
+      (num_graphs > 0 && (!n_nodes || !n_edges || !graph_env)))
+    return XRL_ERR_INVALID_ARG;
+  if (num_graphs > kStG || num_envs > kStV) return XRL_ERR_CAPACITY;
+  if (env_off[0] != 0 || env_off[num_envs] != num_graphs) return XRL_ERR_INVALID_ARG;
+  for (int32_t e = 0; e < num_envs; ++e)
+    if (env_off[e + 1] <= env_off[e]) return XRL_ERR_INVALID_ARG;
+  int64_t N = 0, E = 0;
+  for (int32_t g = 0; g < num_graphs; ++g) {
+    if (n_nodes[g] < 0 || n_edges[g] < 0) return XRL_ERR_INVALID_ARG;
+    N += n_nodes[g]; E += n_edges[g];
+  }
+  if (N > kStN || E > kStE) return XRL_ERR_CAPACITY;          // beyond the built-in scratch
+  if ((N > 0 && (!op || !seg_id)) || (E > 0 && (!edge_src || !edge_dst || !col))) return XRL_ERR_INVALID_ARG;
+  if (scan_workspace_ints((N > num_graphs ? N : num_graphs) + 1) > size_t(kStaticScanInts))
+    return XRL_ERR_CAPACITY;
+
+  if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return XRL_ERR_CUDA; }
+  if (g_pack_scratch_addr[device] == nullptr) {
+    // one-time set-up on this device: the array's name is only a host-side handle, kernels need
+    // the address the device sees
+    int32_t* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_pack_scratch) != cudaSuccess || p == nullptr) {
+      cudaGetLastError();
+      return XRL_ERR_CUDA;
+    }
+    g_pack_scratch_addr[device] = p;
+  }
+  int32_t* sc = g_pack_scratch_addr[device];
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemsetAsync(device_status, 0, sizeof(int32_t), st);
+  if (e == cudaSuccess && num_graphs > 0) {
+    e = cudaMemcpyAsync(sc + kOffNn, n_nodes, 4 * size_t(num_graphs), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(sc + kOffNe, n_edges, 4 * size_t(num_graphs), cudaMemcpyHostToDevice, st);
+  }
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(sc + kOffEnv, env_off, 4 * size_t(num_envs + 1), cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) { cudaGetLastError(); return XRL_ERR_CUDA; }
+
+  PackIn in;
+  in.B = num_graphs; in.num_envs = num_envs; in.N = int32_t(N); in.E = int32_t(E);
+  in.n_nodes = sc + kOffNn; in.n_edges = sc + kOffNe; in.env_off = sc + kOffEnv;
+  in.op = op; in.edge_src = edge_src; in.edge_dst = edge_dst;
+  PackOut out;
+  out.node_off = node_off; out.edge_off = edge_off; out.seg_id = seg_id; out.graph_env = graph_env;
+  out.rowptr = rowptr; out.col = col;
+  out.deg = sc + kOffDeg; out.tmp_eid = sc + kOffTmp; out.long_rows = sc + kOffLong;
+  out.long_count = sc + kOffCount; out.scan_ws = sc + kOffScan;
+  // the pack kernels zero what they count into (deg, the row cursors, long_count) themselves
+  launch_pack(in, out, num_op_types, device_status, st);
+  if (cudaGetLastError() != cudaSuccess) return XRL_ERR_CUDA;
+  return XRL_OK;
+}
