@@ -66,6 +66,7 @@ struct xrl_ctx {
   Dims dims;
   int device = 0;
   bool weights_set = false;
+  bool use_umma = false;    // bf16 transform on the tensor cores (hidden 128 or 256)
   size_t weight_floats = 0;
   DeviceBuf w_f32;          // the fp32 blob
   DeviceBuf w_store;        // storage-type copies of W0 and the layer matrices (+ transposes)
@@ -337,8 +338,13 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
   int n = k;
   for (int l = 0; l < layers; ++l) {
     slot = pf.begin(st);
-    k = launch_xform_simt(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->s_src.as<float>(),
-                          ctx->s_dst.as<float>(), win, st);
+    k = -1;
+    if (ctx->use_umma)
+      k = launch_xform_umma(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->s_src.as<float>(),
+                            ctx->s_dst.as<float>(), win, ctx->status.as<int32_t>(), st);
+    if (k < 0)
+      k = launch_xform_simt(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->s_src.as<float>(),
+                            ctx->s_dst.as<float>(), win, st);
     pf.end(FAM_XFORM, slot, k, st);
     n += k;
     slot = pf.begin(st);
@@ -381,6 +387,8 @@ xrl_status xrl_create(const xrl_model_config* cfg, int32_t device, xrl_ctx** out
   ctx->dims = Dims{cfg->num_op_types, cfg->hidden, cfg->heads, cfg->layers, cfg->mlp_hidden,
                    cfg->global_dim, cfg->max_actions, cfg->dtype};
   ctx->weight_floats = weight_float_count(*cfg);
+  // XRL_FORCE_SIMT_TRANSFORM=1 keeps the CUDA-core transform for every shape (debugging aid)
+  ctx->use_umma = xform_umma_supported(ctx->dims) && getenv("XRL_FORCE_SIMT_TRANSFORM") == nullptr;
   ctx->max_chunks = int32_t(cfg->max_graphs + cfg->max_nodes / kReadoutChunkRows + 1);
   const size_t sb = storage_bytes(cfg->dtype), N = size_t(cfg->max_nodes), H = size_t(cfg->hidden);
   const size_t F0 = size_t(2 * kS + cfg->num_op_types);

@@ -100,6 +100,9 @@ int launch_embed(const Dims& d, const int32_t* rowptr, const int32_t* col, const
                  const void* shape, const DevWeights& w, void* h, Window win, cudaStream_t st);
 int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* s_src,
                       float* s_dst, Window win, cudaStream_t st);
+bool xform_umma_supported(const Dims& d);
+int launch_xform_umma(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* s_src,
+                      float* s_dst, Window win, int32_t* status, cudaStream_t st);
 int launch_scores(const Dims& d, const void* Z, const LayerWeights& lw, float* s_src, float* s_dst,
                   Window win, cudaStream_t st);
 int launch_aggregate(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z,
