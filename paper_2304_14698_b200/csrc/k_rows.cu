@@ -10,8 +10,6 @@ namespace {
 
 constexpr int kRowThreads = 256;
 
-__device__ __forceinline__ float leaky(float x) { return x > 0.f ? x : 0.2f * x; }
-
 // 8 shape features of one node as floats (all lanes of a group read the same address).
 __device__ __forceinline__ void load_shape(const float* shape, int32_t node, float (&f)[kS]) {
   const float4 a = __ldg(reinterpret_cast<const float4*>(shape + size_t(node) * kS));
@@ -144,90 +142,114 @@ k_scores(const T* __restrict__ Z, const float* __restrict__ a_src, const float* 
 }
 
 // ---- Eq. 7: edge scores, softmax over producers + self, weighted sum of Z rows, bias, ReLU ---
-// Single pass with a running maximum (the sum is rescaled whenever the maximum grows), so every
-// Z row and every score is read once.  Edges are taken four at a time to keep loads in flight.
+// A warp takes blocks of 32 consecutive destination rows: row pointers and producer ids of the
+// whole block are fetched with a few coalesced loads into shared memory, so that the per-row work
+// starts straight at the gathers of Z.  Softmax in a single pass with a running maximum (the sum
+// is rescaled when the maximum grows): every Z row and every score is read once.
+constexpr int kAggBlockRows = 32;
+constexpr int kAggColCap = 192;       // cached producer ids per block; rows beyond read col directly
+
+template <int VEC>
+__device__ __forceinline__ void softmax_accumulate(float sc, float sd, const float (&z)[VEC], float& m,
+                                                   float& l, float (&acc)[VEC]) {
+  const float ev = fmaxf(sc + sd, 0.2f * (sc + sd));          // LeakyReLU, slope 0.2
+  if (ev > m) {
+    const float scale = __expf(m - ev);
+    l *= scale;
+#pragma unroll
+    for (int t = 0; t < VEC; ++t) acc[t] *= scale;
+    m = ev;
+  }
+  const float p = __expf(ev - m);
+  l += p;
+#pragma unroll
+  for (int t = 0; t < VEC; ++t) acc[t] = fmaf(p, z[t], acc[t]);
+}
+
 template <typename T, int LPR, int VPL>
-__global__ void __launch_bounds__(kRowThreads)
+__global__ void __launch_bounds__(kRowThreads, (VPL == 1 ? 4 : 2))
 k_aggregate(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
             const T* __restrict__ Z, const float* __restrict__ s_src, const float* __restrict__ s_dst,
             const float* __restrict__ bias, T* __restrict__ h_out, int H, int K, Window win) {
   constexpr int VEC = VecOf<T>::N;
   constexpr int RPW = 32 / LPR;
+  constexpr int WARPS = kRowThreads / 32;
   constexpr int EB = 4;
+  __shared__ int32_t s_rp[WARPS][kAggBlockRows + 1];
+  __shared__ int32_t s_col[WARPS][kAggColCap];
   const int NV = H / VEC, d = H / K;
-  const int lane = threadIdx.x & 31, sub = lane / LPR, sl = lane % LPR;
+  const int lane = threadIdx.x & 31, sub = lane / LPR, sl = lane % LPR, wib = threadIdx.x >> 5;
   const int warps_total = (gridDim.x * blockDim.x) >> 5;
   const int warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nrows = int64_t(win.row_end) - win.row_begin;
+  const int64_t nblocks = (nrows + kAggBlockRows - 1) / kAggBlockRows;
 
-  int head[VPL];
+  int head[VPL], c0[VPL];
   bool on[VPL];
+  float bs[VPL][VEC];
 #pragma unroll
   for (int v = 0; v < VPL; ++v) {
     const int vi = v * LPR + sl;
     on[v] = vi < NV;
-    head[v] = on[v] ? (vi * VEC) / d : 0;
+    c0[v] = on[v] ? vi * VEC : 0;
+    head[v] = c0[v] / d;
+#pragma unroll
+    for (int t = 0; t < VEC; ++t) bs[v][t] = __ldg(bias + c0[v] + t);
   }
 
-  for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * RPW; r0 < win.row_end;
-       r0 += int64_t(warps_total) * RPW) {
-    const int32_t row = int32_t(r0) + sub;
-    if (row >= win.row_end) continue;
-    const int32_t lrow = row - win.win_base;
-    const int32_t e0 = __ldg(rowptr + row), e1 = __ldg(rowptr + row + 1);
+  for (int64_t blk = warp_id; blk < nblocks; blk += warps_total) {
+    const int32_t r0 = win.row_begin + int32_t(blk) * kAggBlockRows;
+    const int nr = min(kAggBlockRows, win.row_end - r0);
+    __syncwarp();                                   // the previous block's reads are done
+    if (lane < nr) s_rp[wib][lane] = __ldg(rowptr + r0 + lane);
+    if (lane == 0) s_rp[wib][nr] = __ldg(rowptr + r0 + nr);
+    __syncwarp();
+    const int32_t eb = s_rp[wib][0];
+    const int ne = min(s_rp[wib][nr] - eb, kAggColCap);
+    for (int t = lane; t < ne; t += 32) s_col[wib][t] = __ldg(col + eb + t);
+    __syncwarp();
 
-    float m[VPL], l[VPL], sd[VPL], acc[VPL][VEC];
-#pragma unroll
-    for (int v = 0; v < VPL; ++v) {
-      if (on[v]) {
-        sd[v] = __ldg(s_dst + size_t(lrow) * K + head[v]);
-        m[v] = leaky(__ldg(s_src + size_t(lrow) * K + head[v]) + sd[v]);   // the self term
-        l[v] = 1.f;
-        load_vec(Z + size_t(lrow) * H + (v * LPR + sl) * VEC, acc[v]);
-      }
-    }
-    for (int32_t e = e0; e < e1; e += EB) {
-      int32_t j[EB];
-#pragma unroll
-      for (int b = 0; b < EB; ++b) j[b] = (e + b < e1) ? __ldg(col + e + b) - win.win_base : -1;
+    for (int rr = sub; rr < nr; rr += RPW) {
+      const int32_t lrow = r0 + rr - win.win_base;
+      const int32_t e0 = s_rp[wib][rr] - eb;          // edge offsets relative to the block
+      const int n = s_rp[wib][rr + 1] - eb - e0;
+      auto producer = [&](int t) -> int32_t {         // t-th producer of this row, window-relative
+        const int idx = e0 + t;
+        return (idx < kAggColCap ? s_col[wib][idx] : __ldg(col + eb + idx)) - win.win_base;
+      };
 #pragma unroll
       for (int v = 0; v < VPL; ++v) {
         if (!on[v]) continue;
-        float sc[EB], z[EB][VEC];
+        const float sd = __ldg(s_dst + size_t(lrow) * K + head[v]);
+        float m = __ldg(s_src + size_t(lrow) * K + head[v]) + sd;
+        m = fmaxf(m, 0.2f * m);                       // the self term opens the running softmax
+        float l = 1.f, acc[VEC];
+        load_vec(Z + size_t(lrow) * H + c0[v], acc);
+        for (int t = 0; t < n; t += EB) {
+          // n is the same for all lanes of a row group: these branches do not diverge inside it
+          float sc[EB];
+          uint4 raw[EB];                              // kept packed until used: fewer live registers
 #pragma unroll
-        for (int b = 0; b < EB; ++b) {
-          if (j[b] >= 0) {
-            sc[b] = __ldg(s_src + size_t(j[b]) * K + head[v]);
-            load_vec(Z + size_t(j[b]) * H + (v * LPR + sl) * VEC, z[b]);
-          }
-        }
-#pragma unroll
-        for (int b = 0; b < EB; ++b) {
-          if (j[b] >= 0) {
-            const float ev = leaky(sc[b] + sd[v]);
-            if (ev > m[v]) {
-              const float scale = __expf(m[v] - ev);
-              l[v] *= scale;
-#pragma unroll
-              for (int t = 0; t < VEC; ++t) acc[v][t] *= scale;
-              m[v] = ev;
+          for (int b = 0; b < EB; ++b)
+            if (t + b < n) {
+              const int32_t j = producer(t + b);
+              sc[b] = __ldg(s_src + size_t(j) * K + head[v]);
+              raw[b] = __ldg(reinterpret_cast<const uint4*>(Z + size_t(j) * H + c0[v]));
             }
-            const float p = __expf(ev - m[v]);
-            l[v] += p;
 #pragma unroll
-            for (int t = 0; t < VEC; ++t) acc[v][t] = fmaf(p, z[b][t], acc[v][t]);
-          }
+          for (int b = 0; b < EB; ++b)
+            if (t + b < n) {
+              float z[VEC];
+              unpack(raw[b], z);
+              softmax_accumulate<VEC>(sc[b], sd, z, m, l, acc);
+            }
         }
+        const float inv = __frcp_rn(l);
+        float o[VEC];
+#pragma unroll
+        for (int t = 0; t < VEC; ++t) o[t] = fmaxf(fmaf(acc[t], inv, bs[v][t]), 0.f);
+        store_vec(h_out + size_t(lrow) * H + c0[v], o);
       }
-    }
-#pragma unroll
-    for (int v = 0; v < VPL; ++v) {
-      if (!on[v]) continue;
-      const int c0 = (v * LPR + sl) * VEC;
-      const float inv = 1.f / l[v];
-      float o[VEC];
-#pragma unroll
-      for (int t = 0; t < VEC; ++t) o[t] = fmaxf(fmaf(acc[v][t], inv, __ldg(bias + c0 + t)), 0.f);
-      store_vec(h_out + size_t(lrow) * H + c0, o);
     }
   }
 }
@@ -297,7 +319,7 @@ int launch_aggregate(const Dims& d, const int32_t* rowptr, const int32_t* col, c
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   if (rows <= 0) return 0;
 #define CALL(TY_, LPR, VPL)                                                                        \
-  k_aggregate<TY_, LPR, VPL><<<row_grid(rows, 32 / LPR), kRowThreads, 0, st>>>(                    \
+  k_aggregate<TY_, LPR, VPL><<<row_grid(rows, kAggBlockRows), kRowThreads, 0, st>>>(                \
       rowptr, col, static_cast<const TY_*>(Z), s_src, s_dst, bias, static_cast<TY_*>(h_out), d.H,   \
       d.K, win)
   if (d.dtype == XRL_BF16) XRL_ROW_DISPATCH(bf16, d.H, CALL);
