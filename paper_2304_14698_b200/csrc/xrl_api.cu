@@ -67,6 +67,8 @@ struct xrl_ctx {
   int device = 0;
   bool weights_set = false;
   bool use_umma = false;    // bf16 transform on the tensor cores (hidden 128 or 256)
+  bool use_umma_embed = false;   // bf16 node update on the tensor cores
+  DeviceBuf w0ext;          // W0 extended and transposed for the tensor-core node update
   size_t weight_floats = 0;
   DeviceBuf w_f32;          // the fp32 blob
   DeviceBuf w_store;        // storage-type copies of W0 and the layer matrices (+ transposes)
@@ -332,8 +334,13 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
   const Window win{0, b->N, 0};
   Profiler& pf = ctx->prof;
   size_t slot = pf.begin(st);
-  int k = launch_embed(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), b->op.as<int32_t>(),
-                       b->shape.p, ctx->dw, ctx->h.p, win, st);
+  int k = -1;
+  if (ctx->use_umma_embed)
+    k = launch_embed_umma(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), b->op.as<int32_t>(),
+                          b->shape.p, ctx->w0ext.p, ctx->h.p, win, ctx->status.as<int32_t>(), st);
+  if (k < 0)
+    k = launch_embed(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), b->op.as<int32_t>(),
+                     b->shape.p, ctx->dw, ctx->h.p, win, st);
   pf.end(FAM_EMBED, slot, k, st);
   int n = k;
   for (int l = 0; l < layers; ++l) {
@@ -389,6 +396,7 @@ xrl_status xrl_create(const xrl_model_config* cfg, int32_t device, xrl_ctx** out
   ctx->weight_floats = weight_float_count(*cfg);
   // XRL_FORCE_SIMT_TRANSFORM=1 keeps the CUDA-core transform for every shape (debugging aid)
   ctx->use_umma = xform_umma_supported(ctx->dims) && getenv("XRL_FORCE_SIMT_TRANSFORM") == nullptr;
+  ctx->use_umma_embed = embed_umma_supported(ctx->dims) && getenv("XRL_FORCE_SIMT_TRANSFORM") == nullptr;
   ctx->max_chunks = int32_t(cfg->max_graphs + cfg->max_nodes / kReadoutChunkRows + 1);
   const size_t sb = storage_bytes(cfg->dtype), N = size_t(cfg->max_nodes), H = size_t(cfg->hidden);
   const size_t F0 = size_t(2 * kS + cfg->num_op_types);
@@ -396,6 +404,7 @@ xrl_status xrl_create(const xrl_model_config* cfg, int32_t device, xrl_ctx** out
   auto A = [&](DeviceBuf& d, size_t bytes) { if (e == cudaSuccess) e = d.alloc(bytes); };
   A(ctx->w_f32, 4 * ctx->weight_floats);
   A(ctx->w_store, sb * (F0 * H + 2 * size_t(cfg->layers) * H * H));
+  A(ctx->w0ext, ctx->use_umma_embed ? 2 * H * size_t(embed_umma_kpad(ctx->dims)) : 0);
   A(ctx->h, sb * N * H);
   A(ctx->Z, sb * N * H);
   A(ctx->s_src, 4 * N * size_t(cfg->heads));
@@ -417,7 +426,7 @@ void xrl_destroy(xrl_ctx* ctx) {
   if (!ctx) return;
   cudaSetDevice(ctx->device);
   cudaDeviceSynchronize();
-  DeviceBuf* bufs[] = {&ctx->w_f32, &ctx->w_store, &ctx->h, &ctx->Z, &ctx->s_src, &ctx->s_dst,
+  DeviceBuf* bufs[] = {&ctx->w0ext, &ctx->w_f32, &ctx->w_store, &ctx->h, &ctx->Z, &ctx->s_src, &ctx->s_dst,
                        &ctx->partial, &ctx->logits, &ctx->status};
   for (DeviceBuf* d : bufs) d->release();
   ctx->prof.release();
@@ -446,6 +455,7 @@ xrl_status xrl_set_weights(xrl_ctx* ctx, const void* host_blob, size_t bytes) {
   launch_round_weights(W0, store, nullptr, int(F0), int(H), c.dtype, nullptr);
   w.W0 = store; store += sb * F0 * H;
   w.b0 = take(H);
+  if (ctx->use_umma_embed) build_w0ext(ctx->dims, w.W0, w.b0, ctx->w0ext.p, nullptr);
   for (int l = 0; l < c.layers; ++l) {
     const float* W = take(H * H);
     launch_round_weights(W, store, store + sb * H * H, int(H), int(H), c.dtype, nullptr);

@@ -100,6 +100,12 @@ int launch_embed(const Dims& d, const int32_t* rowptr, const int32_t* col, const
                  const void* shape, const DevWeights& w, void* h, Window win, cudaStream_t st);
 int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* s_src,
                       float* s_dst, Window win, cudaStream_t st);
+bool embed_umma_supported(const Dims& d);
+int embed_umma_kpad(const Dims& d);
+void build_w0ext(const Dims& d, const void* W0_store, const float* b0, void* out, cudaStream_t st);
+int launch_embed_umma(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op,
+                      const void* shape, const void* w0ext_t, void* h, Window win, int32_t* status,
+                      cudaStream_t st);
 bool xform_umma_supported(const Dims& d);
 int launch_xform_umma(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* s_src,
                       float* s_dst, Window win, int32_t* status, cudaStream_t st);
