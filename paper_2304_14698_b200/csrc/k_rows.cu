@@ -89,7 +89,8 @@ k_embed(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
 }
 
 // ---- attention half-scores from Z (used when the transform kernel does not emit them) ------
-// s_src[i,k] = a_src[k] . Z[i, head k],  s_dst[i,k] = a_dst[k] . Z[i, head k]
+// s_src[i,k] = log2(e) a_src[k] . Z[i, head k],  s_dst[i,k] = log2(e) a_dst[k] . Z[i, head k]
+// (stored pre-multiplied by log2(e): the aggregate kernel then needs exp2 only)
 template <typename T, int LPR, int VPL>
 __global__ void __launch_bounds__(kRowThreads)
 k_scores(const T* __restrict__ Z, const float* __restrict__ a_src, const float* __restrict__ a_dst,
@@ -133,8 +134,8 @@ k_scores(const T* __restrict__ Z, const float* __restrict__ a_src, const float* 
           ss += part[wib][sub][v][0];
           sd += part[wib][sub][v][1];
         }
-        s_src[size_t(row - win.win_base) * K + k] = ss;
-        s_dst[size_t(row - win.win_base) * K + k] = sd;
+        s_src[size_t(row - win.win_base) * K + k] = ss * kLog2e;
+        s_dst[size_t(row - win.win_base) * K + k] = sd * kLog2e;
       }
     }
     __syncwarp();
@@ -144,26 +145,55 @@ k_scores(const T* __restrict__ Z, const float* __restrict__ a_src, const float* 
 // ---- Eq. 7: edge scores, softmax over producers + self, weighted sum of Z rows, bias, ReLU ---
 // A warp takes blocks of 32 consecutive destination rows: row pointers and producer ids of the
 // whole block are fetched with a few coalesced loads into shared memory, so that the per-row work
-// starts straight at the gathers of Z.  Softmax in a single pass with a running maximum (the sum
-// is rescaled when the maximum grows): every Z row and every score is read once.
+// starts straight at the gathers of Z.  The half-scores arrive already multiplied by log2(e)
+// (LeakyReLU commutes with a positive factor), so the softmax weights are plain exp2.  Producers
+// are taken in groups of up to four: all their loads are issued first, the running maximum is
+// updated once per group and the partial sum rescaled only if it grew.  Every Z row and every
+// score is read once.
 constexpr int kAggBlockRows = 32;
-constexpr int kAggColCap = 192;       // cached producer ids per block; rows beyond read col directly
+constexpr int kAggColCap = 224;       // producer ids cached per block of rows
 
-template <int VEC>
-__device__ __forceinline__ void softmax_accumulate(float sc, float sd, const float (&z)[VEC], float& m,
-                                                   float& l, float (&acc)[VEC]) {
-  const float ev = fmaxf(sc + sd, 0.2f * (sc + sd));          // LeakyReLU, slope 0.2
-  if (ev > m) {
-    const float scale = __expf(m - ev);
+__device__ __forceinline__ float lrelu(float x) { return fmaxf(x, 0.2f * x); }
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// One group of NB (1..4) producers of a row: loads, then maximum, weights, accumulation.
+template <typename T, int NB>
+__device__ __forceinline__ void agg_group(const int32_t* __restrict__ js, int32_t win_base,
+                                          const T* __restrict__ zlane, const float* __restrict__ slane,
+                                          int H, int K, float sd, float& m, float& l,
+                                          float (&acc)[VecOf<T>::N]) {
+  constexpr int VEC = VecOf<T>::N;
+  float ev[NB];
+  uint4 raw[NB];
+#pragma unroll
+  for (int b = 0; b < NB; ++b) {
+    const int32_t j = js[b] - win_base;
+    ev[b] = __ldg(slane + size_t(j) * K);
+    raw[b] = __ldg(reinterpret_cast<const uint4*>(zlane + size_t(j) * H));
+  }
+  float mx = m;
+#pragma unroll
+  for (int b = 0; b < NB; ++b) { ev[b] = lrelu(ev[b] + sd); mx = fmaxf(mx, ev[b]); }
+  if (mx > m) {
+    const float scale = fast_exp2(m - mx);
     l *= scale;
 #pragma unroll
     for (int t = 0; t < VEC; ++t) acc[t] *= scale;
-    m = ev;
+    m = mx;
   }
-  const float p = __expf(ev - m);
-  l += p;
 #pragma unroll
-  for (int t = 0; t < VEC; ++t) acc[t] = fmaf(p, z[t], acc[t]);
+  for (int b = 0; b < NB; ++b) {
+    const float p = fast_exp2(ev[b] - m);
+    l += p;
+    float z[VEC];
+    unpack(raw[b], z);
+#pragma unroll
+    for (int t = 0; t < VEC; ++t) acc[t] = fmaf(p, z[t], acc[t]);
+  }
 }
 
 template <typename T, int LPR, int VPL>
@@ -174,17 +204,14 @@ k_aggregate(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
   constexpr int VEC = VecOf<T>::N;
   constexpr int RPW = 32 / LPR;
   constexpr int WARPS = kRowThreads / 32;
-  constexpr int EB = 4;
   __shared__ int32_t s_rp[WARPS][kAggBlockRows + 1];
   __shared__ int32_t s_col[WARPS][kAggColCap];
   const int NV = H / VEC, d = H / K;
   const int lane = threadIdx.x & 31, sub = lane / LPR, sl = lane % LPR, wib = threadIdx.x >> 5;
   const int warps_total = (gridDim.x * blockDim.x) >> 5;
   const int warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int64_t nrows = int64_t(win.row_end) - win.row_begin;
-  const int64_t nblocks = (nrows + kAggBlockRows - 1) / kAggBlockRows;
 
-  int head[VPL], c0[VPL];
+  int c0[VPL], head[VPL];
   bool on[VPL];
   float bs[VPL][VEC];
 #pragma unroll
@@ -197,9 +224,11 @@ k_aggregate(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
     for (int t = 0; t < VEC; ++t) bs[v][t] = __ldg(bias + c0[v] + t);
   }
 
-  for (int64_t blk = warp_id; blk < nblocks; blk += warps_total) {
-    const int32_t r0 = win.row_begin + int32_t(blk) * kAggBlockRows;
-    const int nr = min(kAggBlockRows, win.row_end - r0);
+  // blocks of rows: as many rows (up to 32) as keep the block's producer ids within the cache;
+  // a single row with more producers than that is walked straight from global memory
+  int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * kAggBlockRows;
+  while (r0 < win.row_end) {
+    const int nr = int(min(int64_t(kAggBlockRows), win.row_end - r0));
     __syncwarp();                                   // the previous block's reads are done
     if (lane < nr) s_rp[wib][lane] = __ldg(rowptr + r0 + lane);
     if (lane == 0) s_rp[wib][nr] = __ldg(rowptr + r0 + nr);
@@ -210,47 +239,34 @@ k_aggregate(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
     __syncwarp();
 
     for (int rr = sub; rr < nr; rr += RPW) {
-      const int32_t lrow = r0 + rr - win.win_base;
-      const int32_t e0 = s_rp[wib][rr] - eb;          // edge offsets relative to the block
+      const int32_t lrow = int32_t(r0) + rr - win.win_base;
+      const int e0 = s_rp[wib][rr] - eb;              // edge offsets relative to the block
       const int n = s_rp[wib][rr + 1] - eb - e0;
-      auto producer = [&](int t) -> int32_t {         // t-th producer of this row, window-relative
-        const int idx = e0 + t;
-        return (idx < kAggColCap ? s_col[wib][idx] : __ldg(col + eb + idx)) - win.win_base;
-      };
+      const bool cached = e0 + n <= kAggColCap;
+      const int32_t* js = cached ? &s_col[wib][e0] : col + eb + e0;
 #pragma unroll
       for (int v = 0; v < VPL; ++v) {
         if (!on[v]) continue;
+        const T* zlane = Z + c0[v];
+        const float* slane = s_src + head[v];
         const float sd = __ldg(s_dst + size_t(lrow) * K + head[v]);
-        float m = __ldg(s_src + size_t(lrow) * K + head[v]) + sd;
-        m = fmaxf(m, 0.2f * m);                       // the self term opens the running softmax
+        float m = lrelu(__ldg(slane + size_t(lrow) * K) + sd);     // the self term opens the softmax
         float l = 1.f, acc[VEC];
-        load_vec(Z + size_t(lrow) * H + c0[v], acc);
-        for (int t = 0; t < n; t += EB) {
-          // n is the same for all lanes of a row group: these branches do not diverge inside it
-          float sc[EB];
-          uint4 raw[EB];                              // kept packed until used: fewer live registers
-#pragma unroll
-          for (int b = 0; b < EB; ++b)
-            if (t + b < n) {
-              const int32_t j = producer(t + b);
-              sc[b] = __ldg(s_src + size_t(j) * K + head[v]);
-              raw[b] = __ldg(reinterpret_cast<const uint4*>(Z + size_t(j) * H + c0[v]));
-            }
-#pragma unroll
-          for (int b = 0; b < EB; ++b)
-            if (t + b < n) {
-              float z[VEC];
-              unpack(raw[b], z);
-              softmax_accumulate<VEC>(sc[b], sd, z, m, l, acc);
-            }
-        }
-        const float inv = __frcp_rn(l);
+        load_vec(zlane + size_t(lrow) * H, acc);
+        int t = 0;
+        for (; t + 4 <= n; t += 4) agg_group<T, 4>(js + t, win.win_base, zlane, slane, H, K, sd, m, l, acc);
+        const int rem = n - t;                          // the same for all lanes of a row group
+        if (rem == 1) agg_group<T, 1>(js + t, win.win_base, zlane, slane, H, K, sd, m, l, acc);
+        else if (rem == 2) agg_group<T, 2>(js + t, win.win_base, zlane, slane, H, K, sd, m, l, acc);
+        else if (rem == 3) agg_group<T, 3>(js + t, win.win_base, zlane, slane, H, K, sd, m, l, acc);
+        const float inv = __fdividef(1.f, l);
         float o[VEC];
 #pragma unroll
-        for (int t = 0; t < VEC; ++t) o[t] = fmaxf(fmaf(acc[t], inv, bs[v][t]), 0.f);
+        for (int t2 = 0; t2 < VEC; ++t2) o[t2] = fmaxf(fmaf(acc[t2], inv, bs[v][t2]), 0.f);
         store_vec(h_out + size_t(lrow) * H + c0[v], o);
       }
     }
+    r0 += int64_t(warps_total) * kAggBlockRows;
   }
 }
 

@@ -73,7 +73,8 @@ k_xform_umma(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
-  for (int t = threadIdx.x; t < H; t += kThreads) { avec[t] = a_src[t]; avec[H + t] = a_dst[t]; }
+  // attention vectors pre-multiplied by log2(e): the half-scores are consumed by an exp2 softmax
+  for (int t = threadIdx.x; t < H; t += kThreads) { avec[t] = a_src[t] * kLog2e; avec[H + t] = a_dst[t] * kLog2e; }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(tmem_slot)), "r"(uint32_t(C::TMEM_COLS)) : "memory");

@@ -11,6 +11,7 @@ namespace xrl {
 
 constexpr int kS = 8;            // shape features per node (compile-time in the kernels)
 constexpr int kNumSMs = 148;     // B200
+constexpr float kLog2e = 1.4426950408889634f;   // half-scores are stored multiplied by log2(e)
 
 typedef __nv_bfloat16 bf16;
 
