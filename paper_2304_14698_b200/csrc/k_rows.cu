@@ -94,7 +94,7 @@ k_embed(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
 template <typename T, int LPR, int VPL>
 __global__ void __launch_bounds__(kRowThreads)
 k_scores(const T* __restrict__ Z, const float* __restrict__ a_src, const float* __restrict__ a_dst,
-         float* __restrict__ s_src, float* __restrict__ s_dst, int H, int K, Window win) {
+         float2* __restrict__ scores, int H, int K, Window win) {
   constexpr int VEC = VecOf<T>::N;
   constexpr int RPW = 32 / LPR;
   constexpr int WARPS = kRowThreads / 32;
@@ -134,8 +134,7 @@ k_scores(const T* __restrict__ Z, const float* __restrict__ a_src, const float* 
           ss += part[wib][sub][v][0];
           sd += part[wib][sub][v][1];
         }
-        s_src[size_t(row - win.win_base) * K + k] = ss * kLog2e;
-        s_dst[size_t(row - win.win_base) * K + k] = sd * kLog2e;
+        scores[size_t(row - win.win_base) * K + k] = make_float2(ss * kLog2e, sd * kLog2e);
       }
     }
     __syncwarp();
@@ -163,7 +162,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
 // One group of NB (1..4) producers of a row: loads, then maximum, weights, accumulation.
 template <typename T, int NB>
 __device__ __forceinline__ void agg_group(const int32_t* __restrict__ js, int32_t win_base,
-                                          const T* __restrict__ zlane, const float* __restrict__ slane,
+                                          const T* __restrict__ zlane, const float2* __restrict__ slane,
                                           int H, int K, float sd, float& m, float& l,
                                           float (&acc)[VecOf<T>::N]) {
   constexpr int VEC = VecOf<T>::N;
@@ -172,7 +171,7 @@ __device__ __forceinline__ void agg_group(const int32_t* __restrict__ js, int32_
 #pragma unroll
   for (int b = 0; b < NB; ++b) {
     const int32_t j = js[b] - win_base;
-    ev[b] = __ldg(slane + size_t(j) * K);
+    ev[b] = __ldg(&slane[size_t(j) * K].x);
     raw[b] = __ldg(reinterpret_cast<const uint4*>(zlane + size_t(j) * H));
   }
   float mx = m;
@@ -199,7 +198,7 @@ __device__ __forceinline__ void agg_group(const int32_t* __restrict__ js, int32_
 template <typename T, int LPR, int VPL>
 __global__ void __launch_bounds__(kRowThreads, (VPL == 1 ? 4 : 2))
 k_aggregate(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
-            const T* __restrict__ Z, const float* __restrict__ s_src, const float* __restrict__ s_dst,
+            const T* __restrict__ Z, const float2* __restrict__ scores,
             const float* __restrict__ bias, T* __restrict__ h_out, int H, int K, Window win) {
   constexpr int VEC = VecOf<T>::N;
   constexpr int RPW = 32 / LPR;
@@ -248,9 +247,10 @@ k_aggregate(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
       for (int v = 0; v < VPL; ++v) {
         if (!on[v]) continue;
         const T* zlane = Z + c0[v];
-        const float* slane = s_src + head[v];
-        const float sd = __ldg(s_dst + size_t(lrow) * K + head[v]);
-        float m = lrelu(__ldg(slane + size_t(lrow) * K) + sd);     // the self term opens the softmax
+        const float2* slane = scores + head[v];
+        const float2 self = __ldg(slane + size_t(lrow) * K);
+        const float sd = self.y;
+        float m = lrelu(self.x + sd);                               // the self term opens the softmax
         float l = 1.f, acc[VEC];
         load_vec(zlane + size_t(lrow) * H, acc);
         int t = 0;
@@ -267,6 +267,153 @@ k_aggregate(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
       }
     }
     r0 += int64_t(warps_total) * kAggBlockRows;
+  }
+}
+
+// ---- Eq. 7 for 512-byte rows (hidden 256 in bf16, 128 in fp32): gathers through a cp.async ring ---
+// Same arithmetic as k_aggregate with one producer per softmax update.  The vectors a warp has to
+// gather for a block of rows (each row's own Z vector, then its producers') form one sequence;
+// every lane copies its 16 bytes of vector i + kRing - 1 (and its head's pair of half-scores) into
+// a private shared-memory slot with cp.async while it consumes vector i, so that several gathers
+// per warp are always in flight without holding them in registers.
+constexpr int kRing = 6;
+constexpr int kRingItems = kAggBlockRows + kAggColCap;
+
+__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(uint32_t(__cvta_generic_to_shared(dst))), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async8(void* dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(uint32_t(__cvta_generic_to_shared(dst))), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kRowThreads, 4)
+k_aggregate_ring(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+                 const T* __restrict__ Z, const float2* __restrict__ scores,
+                 const float* __restrict__ bias, T* __restrict__ h_out, int K, Window win) {
+  constexpr int VEC = VecOf<T>::N;
+  constexpr int H = 32 * VEC;
+  constexpr int WARPS = kRowThreads / 32;
+  __shared__ int32_t s_rp[WARPS][kAggBlockRows + 1];
+  __shared__ int32_t s_item[WARPS][kRingItems];
+  __shared__ uint4 s_z[WARPS][kRing][32];
+  __shared__ float2 s_sc[WARPS][kRing][32];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const int warps_total = (gridDim.x * blockDim.x) >> 5;
+  const int warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int c0 = lane * VEC;
+  const T* zlane = Z + c0;
+  const float2* slane = scores + c0 / (H / K);
+  float bs[VEC];
+#pragma unroll
+  for (int t = 0; t < VEC; ++t) bs[t] = __ldg(bias + c0 + t);
+  int32_t* item = s_item[wib];
+  uint4* ring_z = &s_z[wib][0][lane];
+  float2* ring_s = &s_sc[wib][0][lane];
+
+  auto issue = [&](int i, int total, int slot) {
+    if (i < total) {
+      const int32_t idx = item[i];
+      cp_async16(ring_z + slot * 32, zlane + size_t(idx) * H);
+      cp_async8(ring_s + slot * 32, slane + size_t(idx) * K);
+    }
+    cp_async_commit();                    // an empty group keeps the group count in step
+  };
+
+  for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * kAggBlockRows; r0 < win.row_end;
+       r0 += int64_t(warps_total) * kAggBlockRows) {
+    const int nr = int(min(int64_t(kAggBlockRows), win.row_end - r0));
+    __syncwarp();
+    if (lane < nr) s_rp[wib][lane] = __ldg(rowptr + r0 + lane);
+    if (lane == 0) s_rp[wib][nr] = __ldg(rowptr + r0 + nr);
+    __syncwarp();
+    int rs = 0;
+    while (rs < nr) {
+      // as many rows from rs on as keep (rows + producers) within the item list
+      const int32_t eb = s_rp[wib][rs];
+      const bool fits = (rs + lane < nr) && (lane + 1 + s_rp[wib][rs + lane + 1] - eb <= kRingItems);
+      const uint32_t fmask = __ballot_sync(0xFFFFFFFFu, fits);
+      const int cnt = __ffs(~fmask) - 1 < 0 ? 32 : __ffs(~fmask) - 1;      // leading run of fitting rows
+      if (cnt == 0) {
+        // a single row with more producers than the list holds: walk it straight from global memory
+        const int32_t lrow = int32_t(r0) + rs - win.win_base;
+        const int n = s_rp[wib][rs + 1] - eb;
+        const float2 self = __ldg(slane + size_t(lrow) * K);
+        const float sd = self.y;
+        float m = lrelu(self.x + sd), l = 1.f, acc[VEC];
+        load_vec(zlane + size_t(lrow) * H, acc);
+        int t = 0;
+        for (; t + 4 <= n; t += 4) agg_group<T, 4>(col + eb + t, win.win_base, zlane, slane, H, K, sd, m, l, acc);
+        for (; t < n; ++t) agg_group<T, 1>(col + eb + t, win.win_base, zlane, slane, H, K, sd, m, l, acc);
+        const float inv = __fdividef(1.f, l);
+        float o[VEC];
+#pragma unroll
+        for (int t2 = 0; t2 < VEC; ++t2) o[t2] = fmaxf(fmaf(acc[t2], inv, bs[t2]), 0.f);
+        store_vec(h_out + size_t(lrow) * H + c0, o);
+        rs += 1;
+        continue;
+      }
+      // item list: for each row its own index, then its producers', all window-relative
+      __syncwarp();
+      if (lane < cnt) {
+        const int e0 = s_rp[wib][rs + lane] - eb, n = s_rp[wib][rs + lane + 1] - eb - e0;
+        int pos = lane + e0;
+        item[pos++] = int32_t(r0) + rs + lane - win.win_base;
+        for (int t = 0; t < n; ++t) item[pos++] = __ldg(col + eb + e0 + t) - win.win_base;
+      }
+      __syncwarp();
+      const int total = cnt + (s_rp[wib][rs + cnt] - eb);
+#pragma unroll
+      for (int i = 0; i < kRing - 1; ++i) issue(i, total, i);
+      int i = 0, cslot = 0, pslot = kRing - 1;
+      for (int rr = 0; rr < cnt; ++rr) {
+        const int n = s_rp[wib][rs + rr + 1] - s_rp[wib][rs + rr];
+        const int32_t lrow = int32_t(r0) + rs + rr - win.win_base;
+        // the row's own vector opens the running softmax
+        cp_async_wait<kRing - 2>();
+        uint4 raw = ring_z[cslot * 32];
+        float2 sc = ring_s[cslot * 32];
+        asm volatile("" ::: "memory");
+        issue(i + kRing - 1, total, pslot);
+        ++i; cslot = cslot + 1 == kRing ? 0 : cslot + 1; pslot = pslot + 1 == kRing ? 0 : pslot + 1;
+        const float sd = sc.y;
+        float m = lrelu(sc.x + sd), l = 1.f, acc[VEC];
+        unpack(raw, acc);
+        for (int t = 0; t < n; ++t) {
+          cp_async_wait<kRing - 2>();
+          raw = ring_z[cslot * 32];
+          sc = ring_s[cslot * 32];
+          asm volatile("" ::: "memory");
+          issue(i + kRing - 1, total, pslot);
+          ++i; cslot = cslot + 1 == kRing ? 0 : cslot + 1; pslot = pslot + 1 == kRing ? 0 : pslot + 1;
+          const float ev = lrelu(sc.x + sd);
+          if (ev > m) {
+            const float scale = fast_exp2(m - ev);
+            l *= scale;
+#pragma unroll
+            for (int t2 = 0; t2 < VEC; ++t2) acc[t2] *= scale;
+            m = ev;
+          }
+          const float p = fast_exp2(ev - m);
+          l += p;
+          float z[VEC];
+          unpack(raw, z);
+#pragma unroll
+          for (int t2 = 0; t2 < VEC; ++t2) acc[t2] = fmaf(p, z[t2], acc[t2]);
+        }
+        const float inv = __fdividef(1.f, l);
+        float o[VEC];
+#pragma unroll
+        for (int t2 = 0; t2 < VEC; ++t2) o[t2] = fmaxf(fmaf(acc[t2], inv, bs[t2]), 0.f);
+        store_vec(h_out + size_t(lrow) * H + c0, o);
+      }
+      cp_async_wait<0>();
+      rs += cnt;
+    }
   }
 }
 
@@ -316,13 +463,13 @@ int launch_embed(const Dims& d, const int32_t* rowptr, const int32_t* col, const
   return 1;
 }
 
-int launch_scores(const Dims& d, const void* Z, const LayerWeights& lw, float* s_src, float* s_dst,
-                  Window win, cudaStream_t st) {
+int launch_scores(const Dims& d, const void* Z, const LayerWeights& lw, float* scores, Window win,
+                  cudaStream_t st) {
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   if (rows <= 0) return 0;
 #define CALL(TY_, LPR, VPL)                                                                        \
   k_scores<TY_, LPR, VPL><<<row_grid(rows, 32 / LPR), kRowThreads, 0, st>>>(                       \
-      static_cast<const TY_*>(Z), lw.a_src, lw.a_dst, s_src, s_dst, d.H, d.K, win)
+      static_cast<const TY_*>(Z), lw.a_src, lw.a_dst, reinterpret_cast<float2*>(scores), d.H, d.K, win)
   if (d.dtype == XRL_BF16) XRL_ROW_DISPATCH(bf16, d.H, CALL);
   else XRL_ROW_DISPATCH(float, d.H, CALL);
 #undef CALL
@@ -330,14 +477,26 @@ int launch_scores(const Dims& d, const void* Z, const LayerWeights& lw, float* s
 }
 
 int launch_aggregate(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z,
-                     const float* s_src, const float* s_dst, const float* bias, void* h_out,
+                     const float* scores, const float* bias, void* h_out,
                      Window win, cudaStream_t st) {
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   if (rows <= 0) return 0;
+  if (d.dtype == XRL_BF16 && d.H == 256) {
+    k_aggregate_ring<bf16><<<row_grid(rows, kAggBlockRows), kRowThreads, 0, st>>>(
+        rowptr, col, static_cast<const bf16*>(Z), reinterpret_cast<const float2*>(scores), bias,
+        static_cast<bf16*>(h_out), d.K, win);
+    return 1;
+  }
+  if (d.dtype == XRL_FP32 && d.H == 128) {
+    k_aggregate_ring<float><<<row_grid(rows, kAggBlockRows), kRowThreads, 0, st>>>(
+        rowptr, col, static_cast<const float*>(Z), reinterpret_cast<const float2*>(scores), bias,
+        static_cast<float*>(h_out), d.K, win);
+    return 1;
+  }
 #define CALL(TY_, LPR, VPL)                                                                        \
   k_aggregate<TY_, LPR, VPL><<<row_grid(rows, kAggBlockRows), kRowThreads, 0, st>>>(                \
-      rowptr, col, static_cast<const TY_*>(Z), s_src, s_dst, bias, static_cast<TY_*>(h_out), d.H,   \
-      d.K, win)
+      rowptr, col, static_cast<const TY_*>(Z), reinterpret_cast<const float2*>(scores), bias,       \
+      static_cast<TY_*>(h_out), d.H, d.K, win)
   if (d.dtype == XRL_BF16) XRL_ROW_DISPATCH(bf16, d.H, CALL);
   else XRL_ROW_DISPATCH(float, d.H, CALL);
 #undef CALL

@@ -71,8 +71,8 @@ k_xform_simt(const T* __restrict__ h, const T* __restrict__ W, T* __restrict__ Z
 
 }  // namespace
 
-int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* s_src,
-                      float* s_dst, Window win, cudaStream_t st) {
+int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* scores,
+                      Window win, cudaStream_t st) {
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   if (rows <= 0) return 0;
   const size_t off = size_t(win.row_begin - win.win_base) * d.H;
@@ -85,7 +85,7 @@ int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void
     k_xform_simt<float><<<grid, 256, 0, st>>>(static_cast<const float*>(h) + off,
                                              static_cast<const float*>(lw.W),
                                              static_cast<float*>(Z) + off, d.H, int(rows));
-  return 1 + launch_scores(d, Z, lw, s_src, s_dst, win, st);
+  return 1 + launch_scores(d, Z, lw, scores, win, st);
 }
 
 }  // namespace xrl

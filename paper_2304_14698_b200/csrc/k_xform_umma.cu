@@ -44,7 +44,7 @@ template <int H>
 __global__ void __launch_bounds__(kThreads, 1)
 k_xform_umma(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w,
              const __grid_constant__ CUtensorMap map_z, const float* __restrict__ a_src,
-             const float* __restrict__ a_dst, float* __restrict__ s_src, float* __restrict__ s_dst,
+             const float* __restrict__ a_dst, float2* __restrict__ scores,
              int rows, int K, int32_t* status) {
   using C = Cfg<H>;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -186,7 +186,7 @@ k_xform_umma(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ 
           ss = fmaf(__uint_as_float(z[7]), s1.w, ss); sd = fmaf(__uint_as_float(z[7]), d1.w, sd);
           left -= 8;
           if (left == 0) {
-            if (live) { s_src[grow * K + head] = ss; s_dst[grow * K + head] = sd; }
+            if (live) scores[grow * K + head] = make_float2(ss, sd);
             ss = 0.f; sd = 0.f; ++head; left = d;
           }
         }
@@ -227,7 +227,7 @@ k_xform_umma(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ 
 }
 
 template <int H>
-int launch_h(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* s_src, float* s_dst,
+int launch_h(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* scores,
              Window win, int32_t* status, cudaStream_t st) {
   using C = Cfg<H>;
   static bool attr_set = false;
@@ -249,8 +249,9 @@ int launch_h(const Dims& d, const void* h, const LayerWeights& lw, void* Z, floa
     return -1;
   const int tiles = int((rows + BM - 1) / BM);
   const int grid = tiles < kNumSMs ? tiles : kNumSMs;
-  k_xform_umma<H><<<grid, kThreads, C::SMEM_BYTES, st>>>(mh, mw, mz, lw.a_src, lw.a_dst, s_src + off * d.K,
-                                                         s_dst + off * d.K, int(rows), d.K, status);
+  k_xform_umma<H><<<grid, kThreads, C::SMEM_BYTES, st>>>(mh, mw, mz, lw.a_src, lw.a_dst,
+                                                         reinterpret_cast<float2*>(scores) + off * d.K,
+                                                         int(rows), d.K, status);
   return 1;
 }
 
@@ -261,11 +262,11 @@ bool xform_umma_supported(const Dims& d) {
 }
 
 // Returns the number of kernels launched, or -1 if the tensor maps could not be built.
-int launch_xform_umma(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* s_src,
-                      float* s_dst, Window win, int32_t* status, cudaStream_t st) {
+int launch_xform_umma(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* scores,
+                      Window win, int32_t* status, cudaStream_t st) {
   if (int64_t(win.row_end) - win.row_begin <= 0) return 0;
-  if (d.H == 256) return launch_h<256>(d, h, lw, Z, s_src, s_dst, win, status, st);
-  return launch_h<128>(d, h, lw, Z, s_src, s_dst, win, status, st);
+  if (d.H == 256) return launch_h<256>(d, h, lw, Z, scores, win, status, st);
+  return launch_h<128>(d, h, lw, Z, scores, win, status, st);
 }
 
 }  // namespace xrl

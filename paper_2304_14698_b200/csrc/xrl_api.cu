@@ -73,7 +73,7 @@ struct xrl_ctx {
   DeviceBuf w_f32;          // the fp32 blob
   DeviceBuf w_store;        // storage-type copies of W0 and the layer matrices (+ transposes)
   DevWeights dw;
-  DeviceBuf h, Z, s_src, s_dst, partial, logits, status;
+  DeviceBuf h, Z, scores, partial, logits, status;
   int32_t max_chunks = 0;
   int64_t launches_pack = 0, launches_encode = 0, launches_heads = 0;
 };
@@ -347,16 +347,16 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
     slot = pf.begin(st);
     k = -1;
     if (ctx->use_umma)
-      k = launch_xform_umma(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->s_src.as<float>(),
-                            ctx->s_dst.as<float>(), win, ctx->status.as<int32_t>(), st);
+      k = launch_xform_umma(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), win,
+                            ctx->status.as<int32_t>(), st);
     if (k < 0)
-      k = launch_xform_simt(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->s_src.as<float>(),
-                            ctx->s_dst.as<float>(), win, st);
+      k = launch_xform_simt(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), win,
+                            st);
     pf.end(FAM_XFORM, slot, k, st);
     n += k;
     slot = pf.begin(st);
     k = launch_aggregate(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), ctx->Z.p,
-                         ctx->s_src.as<float>(), ctx->s_dst.as<float>(), ctx->dw.layer[l].b,
+                         ctx->scores.as<float>(), ctx->dw.layer[l].b,
                          ctx->h.p, win, st);
     pf.end(FAM_AGG, slot, k, st);
     n += k;
@@ -407,8 +407,7 @@ xrl_status xrl_create(const xrl_model_config* cfg, int32_t device, xrl_ctx** out
   A(ctx->w0ext, ctx->use_umma_embed ? 2 * H * size_t(embed_umma_kpad(ctx->dims)) : 0);
   A(ctx->h, sb * N * H);
   A(ctx->Z, sb * N * H);
-  A(ctx->s_src, 4 * N * size_t(cfg->heads));
-  A(ctx->s_dst, 4 * N * size_t(cfg->heads));
+  A(ctx->scores, 8 * N * size_t(cfg->heads));
   A(ctx->partial, 4 * size_t(ctx->max_chunks) * H);
   A(ctx->logits, 4 * size_t(cfg->max_graphs));
   A(ctx->status, 4);
@@ -426,7 +425,7 @@ void xrl_destroy(xrl_ctx* ctx) {
   if (!ctx) return;
   cudaSetDevice(ctx->device);
   cudaDeviceSynchronize();
-  DeviceBuf* bufs[] = {&ctx->w0ext, &ctx->w_f32, &ctx->w_store, &ctx->h, &ctx->Z, &ctx->s_src, &ctx->s_dst,
+  DeviceBuf* bufs[] = {&ctx->w0ext, &ctx->w_f32, &ctx->w_store, &ctx->h, &ctx->Z, &ctx->scores,
                        &ctx->partial, &ctx->logits, &ctx->status};
   for (DeviceBuf* d : bufs) d->release();
   ctx->prof.release();

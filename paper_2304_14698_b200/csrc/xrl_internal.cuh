@@ -99,8 +99,9 @@ struct Window { int32_t row_begin, row_end, win_base; };
 
 int launch_embed(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op,
                  const void* shape, const DevWeights& w, void* h, Window win, cudaStream_t st);
-int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* s_src,
-                      float* s_dst, Window win, cudaStream_t st);
+// scores: [N][K] pairs {s_src, s_dst} (float2), both already multiplied by log2(e)
+int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* scores,
+                      Window win, cudaStream_t st);
 bool embed_umma_supported(const Dims& d);
 int embed_umma_kpad(const Dims& d);
 void build_w0ext(const Dims& d, const void* W0_store, const float* b0, void* out, cudaStream_t st);
@@ -108,12 +109,12 @@ int launch_embed_umma(const Dims& d, const int32_t* rowptr, const int32_t* col, 
                       const void* shape, const void* w0ext_t, void* h, Window win, int32_t* status,
                       cudaStream_t st);
 bool xform_umma_supported(const Dims& d);
-int launch_xform_umma(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* s_src,
-                      float* s_dst, Window win, int32_t* status, cudaStream_t st);
-int launch_scores(const Dims& d, const void* Z, const LayerWeights& lw, float* s_src, float* s_dst,
-                  Window win, cudaStream_t st);
+int launch_xform_umma(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* scores,
+                      Window win, int32_t* status, cudaStream_t st);
+int launch_scores(const Dims& d, const void* Z, const LayerWeights& lw, float* scores, Window win,
+                  cudaStream_t st);
 int launch_aggregate(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z,
-                     const float* s_src, const float* s_dst, const float* bias, void* h_out,
+                     const float* scores, const float* bias, void* h_out,
                      Window win, cudaStream_t st);
 int launch_readout(const Dims& d, const void* h, const int32_t* chunk_row0, const int32_t* chunk_row1,
                    int32_t chunk_begin, int32_t chunk_end, float* partial, int32_t win_base,
