@@ -33,6 +33,21 @@ def rank_info():
             int(os.environ.get("WORLD_SIZE", "1")))
 
 
+def rank_seed(cfg_id, rank):
+    """Each rank encodes its own batch (weak scaling): a different seed per rank."""
+    return cfg_id + 100 * rank
+
+
+def reduce_over_ranks(elapsed_ms, graphs, edges, nodes, dist, device):
+    """Max of the per-rank times, sums of the per-rank work.  Only these scalars cross ranks."""
+    import torch
+    t = torch.tensor([elapsed_ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    c = torch.tensor([graphs, edges, nodes], device=device, dtype=torch.int64)
+    dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    return float(t[0]), int(c[0]), int(c[1]), int(c[2])
+
+
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -75,7 +90,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -169,7 +184,7 @@ def run_reference(args, cfg_id):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=4, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--impl", default="xrl", choices=["xrl", "reference"])
@@ -186,7 +201,7 @@ def main():
         return
 
     warmup = max(3, args.warmup)
-    batch = configs.make_batch(cfg_id, candidates=args.candidates, envs=args.envs, seed=cfg_id + 100 * rank)
+    batch = configs.make_batch(cfg_id, candidates=args.candidates, envs=args.envs, seed=rank_seed(cfg_id, rank))
     m = batch["model"]
     N, E, B = int(batch["n_nodes"].sum()), int(batch["n_edges"].sum()), int(batch["num_graphs"])
     Ne = len(batch["env_off"]) - 1
@@ -197,7 +212,7 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import xrl_oracle as xo
         threads = min(os.cpu_count() or 1, xo.num_threads())
-        n_s = min(B, {1: 8, 2: 64, 3: 64}.get(cfg_id, max(16, 2 * threads)))
+        n_s = min(B, {1: 8, 2: 64, 3: 256}.get(cfg_id, 24 * threads))     # ~10-20 s of CPU work on cfg 4/5
         dt, g = oracle_sample_run(batch, blob, n_s, threads)
         no = np.concatenate([[0], np.cumsum(batch["n_nodes"])]); eo = np.concatenate([[0], np.cumsum(batch["n_edges"])])
         cpu = {"value": g / dt, "unit": "graphs/s", "cores": threads, "kind": "oracle",
@@ -289,14 +304,9 @@ def main():
     # ---- reduce over ranks -----------------------------------------------------------------------------
     tot_graphs, tot_edges, tot_nodes = B, E, N
     if world > 1:
-        t = torch.tensor([elapsed_ms, e2e["s_per_step"] if e2e else 0.0], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t[0]);
+        elapsed_ms, tot_graphs, tot_edges, tot_nodes = reduce_over_ranks(elapsed_ms, B, E, N, dist, "cuda")
         if e2e:
-            e2e["s_per_step"] = float(t[1])
-        c = torch.tensor([B, E, N], device="cuda", dtype=torch.int64)
-        dist.all_reduce(c, op=dist.ReduceOp.SUM)
-        tot_graphs, tot_edges, tot_nodes = (int(v) for v in c)
+            e2e["s_per_step"] = reduce_over_ranks(e2e["s_per_step"], 0, 0, 0, dist, "cuda")[0]
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
