@@ -270,81 +270,78 @@ k_aggregate(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
   }
 }
 
-// ---- Eq. 7 for 512-byte rows (hidden 256 in bf16, 128 in fp32) ---------------------------------
-// Same arithmetic as k_aggregate, organised to spend few instructions per gathered vector.
-// A warp takes a block of up to 32 consecutive rows and lists the vectors it has to gather (each
-// row's own Z vector, then its producers').
-//   Phase 1 (weights): the half-scores of all listed nodes are fetched with coalesced loads into
-//     shared memory; then lane r runs the softmax of row r for every head and leaves the
-//     unnormalised weights exp2(e - max) in place plus one reciprocal sum per (row, head).
-//   Phase 2 (vectors): every lane copies its 16 bytes of vector i + kRing - 1 into a private
-//     shared-memory slot with cp.async while it multiplies vector i by its head's weight, so several
-//     gathers per warp are in flight without being held in registers.
+// ---- Eq. 7 for 512-byte rows (hidden 256 in bf16, 128 in fp32): gathers through a cp.async ring ---
+// Same arithmetic as k_aggregate with one producer per softmax update.  The vectors a warp has to
+// gather for a block of rows (each row's own Z vector, then its producers') form one sequence;
+// every lane copies its 16 bytes of vector i + kRing - 1 (and its head's pair of half-scores) into
+// a private shared-memory slot with cp.async while it consumes vector i, so that several gathers
+// per warp are always in flight without holding them in registers.
 constexpr int kRing = 6;
-constexpr int kRingRows = 32;
-constexpr int kRingItems = 128;          // vectors listed per pass: rows + producers
-constexpr int kRingWarps = 4;
+constexpr int kRingItems = kAggBlockRows + kAggColCap;
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(uint32_t(__cvta_generic_to_shared(dst))), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async8(void* dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(uint32_t(__cvta_generic_to_shared(dst))), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-  uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-  return v;
-}
 
-template <int K> struct RingSmem {
-  int32_t rp[kRingRows + 1];
-  int32_t item[kRingItems + kRing];      // padded: the prefetch runs kRing - 1 entries ahead
-  float w[kRingItems * K];               // half-scores, then softmax weights, per (vector, head)
-  float inv[kRingRows * K];              // 1 / sum per (row, head)
-  uint4 z[kRing][32];
-};
-
-template <typename T, int K>
-__global__ void __launch_bounds__(kRingWarps * 32, 4)
+template <typename T>
+__global__ void __launch_bounds__(kRowThreads, 4)
 k_aggregate_ring(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
                  const T* __restrict__ Z, const float2* __restrict__ scores,
-                 const float* __restrict__ bias, T* __restrict__ h_out, Window win) {
+                 const float* __restrict__ bias, T* __restrict__ h_out, int K, Window win) {
   constexpr int VEC = VecOf<T>::N;
   constexpr int H = 32 * VEC;
-  extern __shared__ __align__(16) uint8_t ring_smem_raw[];
-  RingSmem<K>& sm = reinterpret_cast<RingSmem<K>*>(ring_smem_raw)[threadIdx.x >> 5];
-  const int lane = threadIdx.x & 31;
+  constexpr int WARPS = kRowThreads / 32;
+  __shared__ int32_t s_rp[WARPS][kAggBlockRows + 1];
+  __shared__ int32_t s_item[WARPS][kRingItems];
+  __shared__ uint4 s_z[WARPS][kRing][32];
+  __shared__ float2 s_sc[WARPS][kRing][32];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
   const int warps_total = (gridDim.x * blockDim.x) >> 5;
   const int warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int c0 = lane * VEC;
-  const int head = c0 / (H / K);
   const T* zlane = Z + c0;
+  const float2* slane = scores + c0 / (H / K);
   float bs[VEC];
 #pragma unroll
   for (int t = 0; t < VEC; ++t) bs[t] = __ldg(bias + c0 + t);
-  const uint32_t zring = uint32_t(__cvta_generic_to_shared(&sm.z[0][lane]));
+  int32_t* item = s_item[wib];
+  uint4* ring_z = &s_z[wib][0][lane];
+  float2* ring_s = &s_sc[wib][0][lane];
 
-  for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * kRingRows; r0 < win.row_end;
-       r0 += int64_t(warps_total) * kRingRows) {
-    const int nr = int(min(int64_t(kRingRows), win.row_end - r0));
+  auto issue = [&](int i, int total, int slot) {
+    if (i < total) {
+      const int32_t idx = item[i];
+      cp_async16(ring_z + slot * 32, zlane + size_t(idx) * H);
+      cp_async8(ring_s + slot * 32, slane + size_t(idx) * K);
+    }
+    cp_async_commit();                    // an empty group keeps the group count in step
+  };
+
+  for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * kAggBlockRows; r0 < win.row_end;
+       r0 += int64_t(warps_total) * kAggBlockRows) {
+    const int nr = int(min(int64_t(kAggBlockRows), win.row_end - r0));
     __syncwarp();
-    if (lane < nr) sm.rp[lane] = __ldg(rowptr + r0 + lane);
-    if (lane == 0) sm.rp[nr] = __ldg(rowptr + r0 + nr);
+    if (lane < nr) s_rp[wib][lane] = __ldg(rowptr + r0 + lane);
+    if (lane == 0) s_rp[wib][nr] = __ldg(rowptr + r0 + nr);
     __syncwarp();
     int rs = 0;
     while (rs < nr) {
-      // as many rows from rs on as keep (rows + producers) within the list
-      const int32_t eb = sm.rp[rs];
-      const bool fits = (rs + lane < nr) && (lane + 1 + sm.rp[rs + lane + 1] - eb <= kRingItems);
+      // as many rows from rs on as keep (rows + producers) within the item list
+      const int32_t eb = s_rp[wib][rs];
+      const bool fits = (rs + lane < nr) && (lane + 1 + s_rp[wib][rs + lane + 1] - eb <= kRingItems);
       const uint32_t fmask = __ballot_sync(0xFFFFFFFFu, fits);
-      const int cnt = (fmask == 0xFFFFFFFFu) ? 32 : __ffs(~fmask) - 1;   // leading run of fitting rows
+      const int cnt = __ffs(~fmask) - 1 < 0 ? 32 : __ffs(~fmask) - 1;      // leading run of fitting rows
       if (cnt == 0) {
-        // one row with more producers than the list holds: walk it straight from global memory
+        // a single row with more producers than the list holds: walk it straight from global memory
         const int32_t lrow = int32_t(r0) + rs - win.win_base;
-        const int n = sm.rp[rs + 1] - eb;
-        const float2* slane = scores + head;
+        const int n = s_rp[wib][rs + 1] - eb;
         const float2 self = __ldg(slane + size_t(lrow) * K);
         const float sd = self.y;
         float m = lrelu(self.x + sd), l = 1.f, acc[VEC];
@@ -360,122 +357,64 @@ k_aggregate_ring(const int32_t* __restrict__ rowptr, const int32_t* __restrict__
         rs += 1;
         continue;
       }
-      // ---- the list: for each row its own index, then its producers', all window-relative ----------
+      // item list: for each row its own index, then its producers', all window-relative
       __syncwarp();
-      const int total = cnt + (sm.rp[rs + cnt] - eb);
-      int my_e0 = 0, my_n = 0;
       if (lane < cnt) {
-        my_e0 = sm.rp[rs + lane] - eb;
-        my_n = sm.rp[rs + lane + 1] - eb - my_e0;
-        int pos = lane + my_e0;
-        sm.item[pos++] = int32_t(r0) + rs + lane - win.win_base;
-        for (int t = 0; t < my_n; ++t) sm.item[pos++] = __ldg(col + eb + my_e0 + t) - win.win_base;
+        const int e0 = s_rp[wib][rs + lane] - eb, n = s_rp[wib][rs + lane + 1] - eb - e0;
+        int pos = lane + e0;
+        item[pos++] = int32_t(r0) + rs + lane - win.win_base;
+        for (int t = 0; t < n; ++t) item[pos++] = __ldg(col + eb + e0 + t) - win.win_base;
       }
-      if (lane < kRing) sm.item[total + lane] = int32_t(r0) + rs - win.win_base;   // padding: any valid row
       __syncwarp();
-      // start the vector gathers now: they fly while the weights are computed
+      const int total = cnt + (s_rp[wib][rs + cnt] - eb);
 #pragma unroll
-      for (int i = 0; i < kRing - 1; ++i) {
-        cp_async16(zring + i * 512, zlane + size_t(sm.item[i]) * H);
-        cp_async_commit();
-      }
-      // ---- phase 1a: half-scores s_src of every listed node -> shared memory ---------------------------
-      {
-        constexpr int CH = (K + 1) / 2;                      // 16-byte chunks (two {src, dst} pairs) per node
-        for (int q = lane; q < total * CH; q += 32) {
-          const int it = q / CH, ch = q - it * CH;
-          if (K == 1) {
-            sm.w[it] = __ldg(&scores[size_t(sm.item[it])].x);
-          } else {
-            const float4 pr = __ldg(reinterpret_cast<const float4*>(scores + size_t(sm.item[it]) * K) + ch);
-            sm.w[it * K + 2 * ch] = pr.x;
-            sm.w[it * K + 2 * ch + 1] = pr.z;
-          }
-        }
-      }
-      __syncwarp();
-      // ---- phase 1b: lane r owns row r: softmax weights of its own vector and its producers ------------
-      if (lane < cnt) {
-        const int p0 = lane + my_e0;                          // list position of the row's own vector
-        const float2* self = scores + size_t(sm.item[p0]) * K;
-#pragma unroll
-        for (int k = 0; k < K; ++k) {
-          const float sd = __ldg(&self[k].y);
-          float mx = -INFINITY;
-          for (int t = 0; t <= my_n; ++t) {
-            const float e = lrelu(sm.w[(p0 + t) * K + k] + sd);
-            sm.w[(p0 + t) * K + k] = e;
-            mx = fmaxf(mx, e);
-          }
-          float sum = 0.f;
-          for (int t = 0; t <= my_n; ++t) {
-            const float pw = fast_exp2(sm.w[(p0 + t) * K + k] - mx);
-            sm.w[(p0 + t) * K + k] = pw;
-            sum += pw;
-          }
-          sm.inv[lane * K + k] = __fdividef(1.f, sum);
-        }
-      }
-      __syncwarp();
-      // ---- phase 2: weighted sums, one vector per step --------------------------------------------------
+      for (int i = 0; i < kRing - 1; ++i) issue(i, total, i);
       int i = 0, cslot = 0, pslot = kRing - 1;
       for (int rr = 0; rr < cnt; ++rr) {
-        const int n = sm.rp[rs + rr + 1] - sm.rp[rs + rr];
-        float acc[VEC];
-#pragma unroll
-        for (int t2 = 0; t2 < VEC; ++t2) acc[t2] = 0.f;
-        for (int t = 0; t <= n; ++t) {
+        const int n = s_rp[wib][rs + rr + 1] - s_rp[wib][rs + rr];
+        const int32_t lrow = int32_t(r0) + rs + rr - win.win_base;
+        // the row's own vector opens the running softmax
+        cp_async_wait<kRing - 2>();
+        uint4 raw = ring_z[cslot * 32];
+        float2 sc = ring_s[cslot * 32];
+        asm volatile("" ::: "memory");
+        issue(i + kRing - 1, total, pslot);
+        ++i; cslot = cslot + 1 == kRing ? 0 : cslot + 1; pslot = pslot + 1 == kRing ? 0 : pslot + 1;
+        const float sd = sc.y;
+        float m = lrelu(sc.x + sd), l = 1.f, acc[VEC];
+        unpack(raw, acc);
+        for (int t = 0; t < n; ++t) {
           cp_async_wait<kRing - 2>();
-          const uint4 raw = lds128(zring + cslot * 512);
-          const float pw = sm.w[i * K + head];
-          cp_async16(zring + pslot * 512, zlane + size_t(sm.item[i + kRing - 1]) * H);
-          cp_async_commit();
-          ++i;
-          cslot = cslot + 1 == kRing ? 0 : cslot + 1;
-          pslot = pslot + 1 == kRing ? 0 : pslot + 1;
+          raw = ring_z[cslot * 32];
+          sc = ring_s[cslot * 32];
+          asm volatile("" ::: "memory");
+          issue(i + kRing - 1, total, pslot);
+          ++i; cslot = cslot + 1 == kRing ? 0 : cslot + 1; pslot = pslot + 1 == kRing ? 0 : pslot + 1;
+          const float ev = lrelu(sc.x + sd);
+          if (ev > m) {
+            const float scale = fast_exp2(m - ev);
+            l *= scale;
+#pragma unroll
+            for (int t2 = 0; t2 < VEC; ++t2) acc[t2] *= scale;
+            m = ev;
+          }
+          const float p = fast_exp2(ev - m);
+          l += p;
           float z[VEC];
           unpack(raw, z);
 #pragma unroll
-          for (int t2 = 0; t2 < VEC; ++t2) acc[t2] = fmaf(pw, z[t2], acc[t2]);
+          for (int t2 = 0; t2 < VEC; ++t2) acc[t2] = fmaf(p, z[t2], acc[t2]);
         }
-        const float inv = sm.inv[rr * K + head];
+        const float inv = __fdividef(1.f, l);
         float o[VEC];
 #pragma unroll
         for (int t2 = 0; t2 < VEC; ++t2) o[t2] = fmaxf(fmaf(acc[t2], inv, bs[t2]), 0.f);
-        store_vec(h_out + size_t(int32_t(r0) + rs + rr - win.win_base) * H + c0, o);
+        store_vec(h_out + size_t(lrow) * H + c0, o);
       }
       cp_async_wait<0>();
       rs += cnt;
     }
   }
-}
-
-template <typename T>
-bool launch_ring(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z,
-                 const float* scores, const float* bias, void* h_out, Window win, int64_t rows,
-                 cudaStream_t st) {
-  int64_t nb = (rows + kRingRows * kRingWarps - 1) / (kRingRows * kRingWarps);
-  if (nb > int64_t(kNumSMs) * 6) nb = int64_t(kNumSMs) * 6;
-  const int blocks_needed = int(nb);
-#define RING_CASE(KK)                                                                               \
-  case KK: {                                                                                        \
-    static bool attr = false;                                                                       \
-    const size_t smem = sizeof(RingSmem<KK>) * kRingWarps;                                          \
-    if (!attr) {                                                                                    \
-      if (cudaFuncSetAttribute(k_aggregate_ring<T, KK>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                               int(smem)) != cudaSuccess) { cudaGetLastError(); return false; }     \
-      attr = true;                                                                                  \
-    }                                                                                               \
-    k_aggregate_ring<T, KK><<<blocks_needed, kRingWarps * 32, smem, st>>>(                          \
-        rowptr, col, static_cast<const T*>(Z), reinterpret_cast<const float2*>(scores), bias,       \
-        static_cast<T*>(h_out), win);                                                               \
-    return true;                                                                                    \
-  }
-  switch (d.K) {
-    RING_CASE(1) RING_CASE(2) RING_CASE(4) RING_CASE(8)
-    default: return false;
-  }
-#undef RING_CASE
 }
 
 // ---- dispatch on the row geometry ------------------------------------------------------------
@@ -542,10 +481,18 @@ int launch_aggregate(const Dims& d, const int32_t* rowptr, const int32_t* col, c
                      Window win, cudaStream_t st) {
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   if (rows <= 0) return 0;
-  if (d.dtype == XRL_BF16 && d.H == 256 &&
-      launch_ring<bf16>(d, rowptr, col, Z, scores, bias, h_out, win, rows, st)) return 1;
-  if (d.dtype == XRL_FP32 && d.H == 128 &&
-      launch_ring<float>(d, rowptr, col, Z, scores, bias, h_out, win, rows, st)) return 1;
+  if (d.dtype == XRL_BF16 && d.H == 256) {
+    k_aggregate_ring<bf16><<<row_grid(rows, kAggBlockRows), kRowThreads, 0, st>>>(
+        rowptr, col, static_cast<const bf16*>(Z), reinterpret_cast<const float2*>(scores), bias,
+        static_cast<bf16*>(h_out), d.K, win);
+    return 1;
+  }
+  if (d.dtype == XRL_FP32 && d.H == 128) {
+    k_aggregate_ring<float><<<row_grid(rows, kAggBlockRows), kRowThreads, 0, st>>>(
+        rowptr, col, static_cast<const float*>(Z), reinterpret_cast<const float2*>(scores), bias,
+        static_cast<float*>(h_out), d.K, win);
+    return 1;
+  }
 #define CALL(TY_, LPR, VPL)                                                                        \
   k_aggregate<TY_, LPR, VPL><<<row_grid(rows, kAggBlockRows), kRowThreads, 0, st>>>(                \
       rowptr, col, static_cast<const TY_*>(Z), reinterpret_cast<const float2*>(scores), bias,       \
