@@ -1,0 +1,285 @@
+// Edge score / segment softmax / weighted aggregate of a graph-attention layer (paper Eq. 7) for
+// 512-byte feature rows (hidden 256 in bf16, 128 in fp32), with the gathers done by the TMA engine.
+//
+// A warp takes a block of up to 32 consecutive destination rows and lists the rows of Z it needs
+// (each destination's own row, then its producers').  One lane hands the list to the TMA unit four
+// rows at a time (cp.async.bulk.tensor ... tile::gather4, one instruction per four 512-byte rows,
+// a second one for the four rows of half-score pairs); the data lands in a small per-warp ring in
+// shared memory and completion is signalled on an mbarrier.  The 32 lanes then only read their
+// 16 bytes of each row from shared memory and do the arithmetic: LeakyReLU score, running-maximum
+// softmax with exp2 (the half-scores are stored multiplied by log2 e), fp32 accumulation, bias,
+// ReLU.  No lane spends instructions on gather addresses.
+//
+// Every wait is bounded; on expiry the warp records XRL_ERR_TIMEOUT and stops.
+#include "xrl_umma.cuh"
+
+namespace xrl {
+
+using namespace umma;
+
+namespace {
+
+constexpr int TW = 4;            // warps per CTA
+constexpr int G = 4;             // gather groups (of four rows) in flight per warp
+constexpr int BR = 32;           // destination rows per block
+constexpr int ITEMS = 160;       // list capacity, a multiple of 4
+
+template <int K> struct alignas(128) WarpSmem {
+  uint4 z[G][4][32];             // four gathered rows of 512 bytes per group
+  float2 sc[G][4][K];            // their {s_src, s_dst} pairs
+  unsigned long long bar[G];
+  int32_t rp[BR + 1];
+  int32_t item[ITEMS + 4];
+};
+
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, int r0, int r1, int r2,
+                                            int r3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+      ::"r"(dst), "l"(map), "r"(0), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float2 lds64(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float lrelu(float x) { return fmaxf(x, 0.2f * x); }
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+template <typename T, int K>
+__global__ void __launch_bounds__(TW * 32, 5)
+k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant__ CUtensorMap map_s,
+                const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+                const float* __restrict__ bias, T* __restrict__ h_out, Window win, int32_t* status) {
+  constexpr int VEC = VecOf<T>::N;
+  constexpr int H = 32 * VEC;
+  constexpr uint32_t GROUP_BYTES = 4 * 512 + 4 * K * 8;
+  extern __shared__ __align__(128) uint8_t tma_smem_raw[];
+  WarpSmem<K>& sm = reinterpret_cast<WarpSmem<K>*>(tma_smem_raw)[threadIdx.x >> 5];
+  const int lane = threadIdx.x & 31;
+  const int warps_total = (gridDim.x * blockDim.x) >> 5;
+  const int warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int c0 = lane * VEC;
+  const int head = c0 / (H / K);
+  float bs[VEC];
+#pragma unroll
+  for (int t = 0; t < VEC; ++t) bs[t] = __ldg(bias + c0 + t);
+  const uint32_t z_addr = smem_u32(&sm.z[0][0][lane]);       // + slot * 2048 + w * 512
+  const uint32_t s_addr = smem_u32(&sm.sc[0][0][head]);      // + slot * 32 K + w * 8 K
+  const uint32_t z_base = smem_u32(&sm.z[0][0][0]);
+  const uint32_t s_base = smem_u32(&sm.sc[0][0][0]);
+  const uint32_t bar_base = smem_u32(&sm.bar[0]);
+
+  if (lane == 0) {
+    for (int g = 0; g < G; ++g) mbar_init(bar_base + 8 * g, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  __syncwarp();
+  uint32_t q_base = 0;              // gather groups issued (and consumed) by this warp so far
+
+  auto issue = [&](int gi) {        // lane 0 only: group gi of the current list
+    const uint32_t q = q_base + gi;
+    const uint32_t s = q % G;
+    const int32_t* it = &sm.item[gi * 4];
+    mbar_expect_tx(bar_base + 8 * s, GROUP_BYTES);
+    tma_gather4(z_base + s * 2048, &map_z, it[0], it[1], it[2], it[3], bar_base + 8 * s);
+    tma_gather4(s_base + s * (32 * K), &map_s, it[0], it[1], it[2], it[3], bar_base + 8 * s);
+  };
+
+  bool alive = true;
+  for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * BR; r0 < win.row_end && alive;
+       r0 += int64_t(warps_total) * BR) {
+    const int nr = int(min(int64_t(BR), win.row_end - r0));
+    __syncwarp();
+    if (lane < nr) sm.rp[lane] = __ldg(rowptr + r0 + lane);
+    if (lane == 0) sm.rp[nr] = __ldg(rowptr + r0 + nr);
+    __syncwarp();
+    int rs = 0;
+    while (rs < nr && alive) {
+      // as many rows from rs on as keep (rows + producers) within the list; at least one
+      const int32_t eb = sm.rp[rs];
+      const bool fits = (rs + lane < nr) && (lane + 1 + sm.rp[rs + lane + 1] - eb <= ITEMS);
+      const uint32_t fmask = __ballot_sync(0xFFFFFFFFu, fits);
+      int cnt = (fmask == 0xFFFFFFFFu) ? 32 : __ffs(~fmask) - 1;
+      // a row with more producers than the list holds is taken alone, its producers in list-sized parts
+      const bool huge = (cnt == 0);
+      if (huge) cnt = 1;
+      const int n_first = sm.rp[rs + 1] - eb;                  // producers of row rs (used when huge)
+      float m = 0.f, l = 0.f, sd = 0.f, acc[VEC];
+      int part_begin = 0;                                       // huge rows: producers already done
+      bool row_open = false;
+      do {
+        // ---- the list ---------------------------------------------------------------------------------
+        __syncwarp();
+        int total;
+        if (!huge) {
+          total = cnt + (sm.rp[rs + cnt] - eb);
+          if (lane < cnt) {
+            const int e0 = sm.rp[rs + lane] - eb, n = sm.rp[rs + lane + 1] - eb - e0;
+            int pos = lane + e0;
+            sm.item[pos++] = int32_t(r0) + rs + lane - win.win_base;
+            for (int t = 0; t < n; ++t) sm.item[pos++] = __ldg(col + eb + e0 + t) - win.win_base;
+          }
+        } else {
+          const int first = part_begin == 0 ? 1 : 0;            // the row's own vector opens the first part
+          const int np = min(n_first - part_begin, ITEMS - first);
+          total = np + first;
+          if (first && lane == 0) sm.item[0] = int32_t(r0) + rs - win.win_base;
+          for (int t = lane; t < np; t += 32) sm.item[first + t] = __ldg(col + eb + part_begin + t) - win.win_base;
+        }
+        __syncwarp();
+        if (lane < 4) sm.item[total + lane] = sm.item[0];        // pad the last group with a valid row
+        __syncwarp();
+        const int ngroups = (total + 3) >> 2;
+        if (lane == 0)
+          for (int gi = 0; gi < min(G, ngroups); ++gi) issue(gi);
+
+        // ---- consume ----------------------------------------------------------------------------------
+        int i = 0;
+        auto next_vector = [&](uint4& raw, float2& sc) -> bool {
+          const int gi = i >> 2, w = i & 3;
+          const uint32_t q = q_base + gi, s = q % G;
+          if (w == 0) {
+            uint32_t ok = 1;
+            if (lane == 0) ok = mbar_wait(bar_base + 8 * s, (q / G) & 1) ? 1u : 0u;
+            ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+            if (ok && lane != 0) ok = mbar_try(bar_base + 8 * s, (q / G) & 1) ? 1u : 0u;
+            if (!__all_sync(0xFFFFFFFFu, ok != 0)) return false;
+          }
+          raw = lds128(z_addr + s * 2048 + w * 512);
+          sc = lds64(s_addr + s * (32 * K) + w * (8 * K));
+          ++i;
+          if (w == 3 || i == total) {                            // group finished: refill its slot
+            __syncwarp();
+            if (lane == 0 && gi + G < ngroups) issue(gi + G);
+          }
+          return true;
+        };
+        const int rows_here = cnt;
+        for (int rr = 0; rr < rows_here && alive; ++rr) {
+          int n;
+          if (!huge) n = sm.rp[rs + rr + 1] - sm.rp[rs + rr];
+          else n = total - (part_begin == 0 ? 1 : 0);
+          uint4 raw;
+          float2 sc;
+          if (!huge || part_begin == 0) {                        // the row's own vector opens the softmax
+            if (!next_vector(raw, sc)) { alive = false; break; }
+            sd = sc.y;
+            m = lrelu(sc.x + sd);
+            l = 1.f;
+            unpack(raw, acc);
+            row_open = true;
+          }
+          for (int t = 0; t < n; ++t) {
+            if (!next_vector(raw, sc)) { alive = false; break; }
+            const float ev = lrelu(sc.x + sd);
+            if (ev > m) {
+              const float scale = fast_exp2(m - ev);
+              l *= scale;
+#pragma unroll
+              for (int t2 = 0; t2 < VEC; ++t2) acc[t2] *= scale;
+              m = ev;
+            }
+            const float p = fast_exp2(ev - m);
+            l += p;
+            float z[VEC];
+            unpack(raw, z);
+#pragma unroll
+            for (int t2 = 0; t2 < VEC; ++t2) acc[t2] = fmaf(p, z[t2], acc[t2]);
+          }
+          if (!alive) break;
+          const bool row_done = !huge || (part_begin + n >= n_first);
+          if (row_done && row_open) {
+            const float inv = __fdividef(1.f, l);
+            float o[VEC];
+#pragma unroll
+            for (int t2 = 0; t2 < VEC; ++t2) o[t2] = fmaxf(fmaf(acc[t2], inv, bs[t2]), 0.f);
+            store_vec(h_out + size_t(int32_t(r0) + rs + rr - win.win_base) * H + c0, o);
+            row_open = false;
+          }
+          if (huge) part_begin += n;
+        }
+        q_base += ngroups;
+      } while (alive && huge && part_begin < n_first);
+      rs += cnt;
+    }
+  }
+  if (!alive) {
+    if (lane == 0) raise(status, XRL_ERR_TIMEOUT);
+    for (int t = 0; t < 100; ++t) __nanosleep(10000);     // give copies still in flight time to land
+  }
+}
+
+bool make_row_map(CUtensorMap* m, const void* ptr, CUtensorMapDataType dt, uint32_t elem_bytes,
+                  uint64_t rows, uint32_t cols) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {uint64_t(cols) * elem_bytes};
+  cuuint32_t box[2] = {cols, 1};                 // gather4 takes boxes one row high
+  cuuint32_t estr[2] = {1, 1};
+  return fn(m, dt, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <typename T, int K>
+int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const float* scores, const float* bias,
+             void* h_out, Window win, int64_t buf_rows, int32_t* status, cudaStream_t st) {
+  static bool attr = false;
+  const size_t smem = sizeof(WarpSmem<K>) * TW;
+  if (!attr) {
+    if (cudaFuncSetAttribute(k_aggregate_tma<T, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) !=
+        cudaSuccess) {
+      cudaGetLastError();
+      return -1;
+    }
+    attr = true;
+  }
+  constexpr bool is_bf16 = sizeof(T) == 2;
+  CUtensorMap mz, ms;
+  if (!make_row_map(&mz, Z, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                    sizeof(T), uint64_t(buf_rows), is_bf16 ? 256 : 128) ||
+      !make_row_map(&ms, scores, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, uint64_t(buf_rows), 2 * K))
+    return -1;
+  const int64_t rows = int64_t(win.row_end) - win.row_begin;
+  int64_t nb = (rows + BR * TW - 1) / (BR * TW);
+  if (nb > int64_t(kNumSMs) * 5) nb = int64_t(kNumSMs) * 5;
+  k_aggregate_tma<T, K><<<int(nb), TW * 32, smem, st>>>(mz, ms, rowptr, col, bias, static_cast<T*>(h_out),
+                                                        win, status);
+  return 1;
+}
+
+}  // namespace
+
+// buf_rows: rows of the Z / scores buffers reachable from this window (indices are window-relative).
+// Returns kernels launched, or -1 when this shape is not handled here.
+int launch_aggregate_tma(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z,
+                         const float* scores, const float* bias, void* h_out, Window win, int64_t buf_rows,
+                         int32_t* status, cudaStream_t st) {
+  if (encode_fn() == nullptr) return -1;
+  const bool bf = d.dtype == XRL_BF16 && d.H == 256, fp = d.dtype == XRL_FP32 && d.H == 128;
+  if (!bf && !fp) return -1;
+#define TMA_CASE(KK)                                                                                     \
+  case KK:                                                                                               \
+    return bf ? launch_k<bf16, KK>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, status, st)       \
+              : launch_k<float, KK>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, status, st);
+  switch (d.K) {
+    TMA_CASE(4) TMA_CASE(8) TMA_CASE(16)
+    default: return -1;
+  }
+#undef TMA_CASE
+}
+
+}  // namespace xrl

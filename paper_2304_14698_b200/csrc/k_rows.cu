@@ -2,6 +2,8 @@
 // attention half-scores, and the edge-score / segment-softmax / weighted-aggregate step of a
 // graph-attention layer (Eq. 7).  One group of LPR lanes owns one destination row and moves it
 // as 16-byte vectors (VPL vectors per lane); 32 / LPR rows share a warp.
+#include <stdlib.h>
+
 #include "xrl_internal.cuh"
 
 namespace xrl {
@@ -478,16 +480,22 @@ int launch_scores(const Dims& d, const void* Z, const LayerWeights& lw, float* s
 
 int launch_aggregate(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z,
                      const float* scores, const float* bias, void* h_out,
-                     Window win, cudaStream_t st) {
+                     Window win, int64_t buf_rows, int32_t* status, cudaStream_t st) {
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   if (rows <= 0) return 0;
-  if (d.dtype == XRL_BF16 && d.H == 256) {
+  static const char* mode = getenv("XRL_AGG");            // "ring" / "plain": bypass the TMA gather kernel
+  if (mode == nullptr) {
+    const int k = launch_aggregate_tma(d, rowptr, col, Z, scores, bias, h_out, win, buf_rows, status, st);
+    if (k >= 0) return k;
+  }
+  const bool plain = mode != nullptr && mode[0] == 'p';
+  if (!plain && d.dtype == XRL_BF16 && d.H == 256) {
     k_aggregate_ring<bf16><<<row_grid(rows, kAggBlockRows), kRowThreads, 0, st>>>(
         rowptr, col, static_cast<const bf16*>(Z), reinterpret_cast<const float2*>(scores), bias,
         static_cast<bf16*>(h_out), d.K, win);
     return 1;
   }
-  if (d.dtype == XRL_FP32 && d.H == 128) {
+  if (!plain && d.dtype == XRL_FP32 && d.H == 128) {
     k_aggregate_ring<float><<<row_grid(rows, kAggBlockRows), kRowThreads, 0, st>>>(
         rowptr, col, static_cast<const float*>(Z), reinterpret_cast<const float2*>(scores), bias,
         static_cast<float*>(h_out), d.K, win);

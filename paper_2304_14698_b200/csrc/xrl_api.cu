@@ -357,7 +357,7 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
     slot = pf.begin(st);
     k = launch_aggregate(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), ctx->Z.p,
                          ctx->scores.as<float>(), ctx->dw.layer[l].b,
-                         ctx->h.p, win, st);
+                         ctx->h.p, win, b->N, ctx->status.as<int32_t>(), st);
     pf.end(FAM_AGG, slot, k, st);
     n += k;
   }

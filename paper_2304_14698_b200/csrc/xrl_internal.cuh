@@ -115,7 +115,10 @@ int launch_scores(const Dims& d, const void* Z, const LayerWeights& lw, float* s
                   cudaStream_t st);
 int launch_aggregate(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z,
                      const float* scores, const float* bias, void* h_out,
-                     Window win, cudaStream_t st);
+                     Window win, int64_t buf_rows, int32_t* status, cudaStream_t st);
+int launch_aggregate_tma(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z,
+                         const float* scores, const float* bias, void* h_out, Window win, int64_t buf_rows,
+                         int32_t* status, cudaStream_t st);
 int launch_readout(const Dims& d, const void* h, const int32_t* chunk_row0, const int32_t* chunk_row1,
                    int32_t chunk_begin, int32_t chunk_end, float* partial, int32_t win_base,
                    cudaStream_t st);
