@@ -29,7 +29,7 @@ template <int K> struct alignas(128) WarpSmem {
   float2 sc[G][4][K];            // their {s_src, s_dst} pairs
   unsigned long long bar[G];
   int32_t rp[BR + 1];
-  int32_t item[ITEMS + 4];
+  alignas(16) int32_t item[ITEMS + 4];
 };
 
 __device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, int r0, int r1, int r2,
@@ -56,14 +56,23 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// Bounded wait executed by every lane (each lane must observe the phase itself to see the data).
+__device__ __forceinline__ bool wait_all_lanes(uint32_t bar, uint32_t parity) {
+  for (int it = 0; it < (1 << 20); ++it)
+    if (mbar_try(bar, parity)) return true;
+  return false;
+}
+
 template <typename T, int K>
 __global__ void __launch_bounds__(TW * 32, 5)
 k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant__ CUtensorMap map_s,
                 const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+                const T* __restrict__ Z, const float2* __restrict__ scores,
                 const float* __restrict__ bias, T* __restrict__ h_out, Window win, int32_t* status) {
   constexpr int VEC = VecOf<T>::N;
   constexpr int H = 32 * VEC;
   constexpr uint32_t GROUP_BYTES = 4 * 512 + 4 * K * 8;
+  constexpr uint32_t ZG = 2048, SG = 32 * K;          // bytes per group in the two rings
   extern __shared__ __align__(128) uint8_t tma_smem_raw[];
   WarpSmem<K>& sm = reinterpret_cast<WarpSmem<K>*>(tma_smem_raw)[threadIdx.x >> 5];
   const int lane = threadIdx.x & 31;
@@ -74,8 +83,8 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
   float bs[VEC];
 #pragma unroll
   for (int t = 0; t < VEC; ++t) bs[t] = __ldg(bias + c0 + t);
-  const uint32_t z_addr = smem_u32(&sm.z[0][0][lane]);       // + slot * 2048 + w * 512
-  const uint32_t s_addr = smem_u32(&sm.sc[0][0][head]);      // + slot * 32 K + w * 8 K
+  const uint32_t z_lane = smem_u32(&sm.z[0][0][lane]);       // this lane's 16 bytes of slot 0, row 0
+  const uint32_t s_lane = smem_u32(&sm.sc[0][0][head]);      // this lane's head in slot 0, row 0
   const uint32_t z_base = smem_u32(&sm.z[0][0][0]);
   const uint32_t s_base = smem_u32(&sm.sc[0][0][0]);
   const uint32_t bar_base = smem_u32(&sm.bar[0]);
@@ -86,18 +95,20 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
     fence_async_smem();
   }
   __syncwarp();
-  uint32_t q_base = 0;              // gather groups issued (and consumed) by this warp so far
 
-  auto issue = [&](int gi) {        // lane 0 only: group gi of the current list
-    const uint32_t q = q_base + gi;
-    const uint32_t s = q % G;
-    const int32_t* it = &sm.item[gi * 4];
-    mbar_expect_tx(bar_base + 8 * s, GROUP_BYTES);
-    tma_gather4(z_base + s * 2048, &map_z, it[0], it[1], it[2], it[3], bar_base + 8 * s);
-    tma_gather4(s_base + s * (32 * K), &map_s, it[0], it[1], it[2], it[3], bar_base + 8 * s);
+  // ring state, carried across lists: slot and phase parity of the next group to consume
+  uint32_t slot = 0, par = 0;
+  bool alive = true;
+
+  // lane 0: hand group `gi` of the current list (list rows item[4 gi .. 4 gi + 3]) to slot `s`
+  auto issue = [&](int gi, uint32_t s) {
+    const int4 it = *reinterpret_cast<const int4*>(&sm.item[gi * 4]);
+    const uint32_t bar = bar_base + 8 * s;
+    mbar_expect_tx(bar, GROUP_BYTES);
+    tma_gather4(z_base + s * ZG, &map_z, it.x, it.y, it.z, it.w, bar);
+    tma_gather4(s_base + s * SG, &map_s, it.x, it.y, it.z, it.w, bar);
   };
 
-  bool alive = true;
   for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * BR; r0 < win.row_end && alive;
        r0 += int64_t(warps_total) * BR) {
     const int nr = int(min(int64_t(BR), win.row_end - r0));
@@ -107,111 +118,111 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
     __syncwarp();
     int rs = 0;
     while (rs < nr && alive) {
-      // as many rows from rs on as keep (rows + producers) within the list; at least one
+      // as many rows from rs on as keep (rows + producers) within the list
       const int32_t eb = sm.rp[rs];
       const bool fits = (rs + lane < nr) && (lane + 1 + sm.rp[rs + lane + 1] - eb <= ITEMS);
       const uint32_t fmask = __ballot_sync(0xFFFFFFFFu, fits);
-      int cnt = (fmask == 0xFFFFFFFFu) ? 32 : __ffs(~fmask) - 1;
-      // a row with more producers than the list holds is taken alone, its producers in list-sized parts
-      const bool huge = (cnt == 0);
-      if (huge) cnt = 1;
-      const int n_first = sm.rp[rs + 1] - eb;                  // producers of row rs (used when huge)
-      float m = 0.f, l = 0.f, sd = 0.f, acc[VEC];
-      int part_begin = 0;                                       // huge rows: producers already done
-      bool row_open = false;
-      do {
-        // ---- the list ---------------------------------------------------------------------------------
-        __syncwarp();
-        int total;
-        if (!huge) {
-          total = cnt + (sm.rp[rs + cnt] - eb);
-          if (lane < cnt) {
-            const int e0 = sm.rp[rs + lane] - eb, n = sm.rp[rs + lane + 1] - eb - e0;
-            int pos = lane + e0;
-            sm.item[pos++] = int32_t(r0) + rs + lane - win.win_base;
-            for (int t = 0; t < n; ++t) sm.item[pos++] = __ldg(col + eb + e0 + t) - win.win_base;
+      const int cnt = (fmask == 0xFFFFFFFFu) ? 32 : __ffs(~fmask) - 1;
+      if (cnt == 0) {
+        // a row with more producers than the list holds: plain loads, one producer at a time
+        const int32_t lrow = int32_t(r0) + rs - win.win_base;
+        const int n = sm.rp[rs + 1] - eb;
+        const float2 self = __ldg(scores + size_t(lrow) * K + head);
+        const float sd = self.y;
+        float m = lrelu(self.x + sd), l = 1.f, acc[VEC];
+        load_vec(Z + size_t(lrow) * H + c0, acc);
+        for (int t = 0; t < n; ++t) {
+          const int32_t j = __ldg(col + eb + t) - win.win_base;
+          const float ev = lrelu(__ldg(&scores[size_t(j) * K + head].x) + sd);
+          float z[VEC];
+          load_vec(Z + size_t(j) * H + c0, z);
+          if (ev > m) {
+            const float scale = fast_exp2(m - ev);
+            l *= scale;
+#pragma unroll
+            for (int t2 = 0; t2 < VEC; ++t2) acc[t2] *= scale;
+            m = ev;
           }
-        } else {
-          const int first = part_begin == 0 ? 1 : 0;            // the row's own vector opens the first part
-          const int np = min(n_first - part_begin, ITEMS - first);
-          total = np + first;
-          if (first && lane == 0) sm.item[0] = int32_t(r0) + rs - win.win_base;
-          for (int t = lane; t < np; t += 32) sm.item[first + t] = __ldg(col + eb + part_begin + t) - win.win_base;
+          const float p = fast_exp2(ev - m);
+          l += p;
+#pragma unroll
+          for (int t2 = 0; t2 < VEC; ++t2) acc[t2] = fmaf(p, z[t2], acc[t2]);
         }
-        __syncwarp();
-        if (lane < 4) sm.item[total + lane] = sm.item[0];        // pad the last group with a valid row
-        __syncwarp();
-        const int ngroups = (total + 3) >> 2;
-        if (lane == 0)
-          for (int gi = 0; gi < min(G, ngroups); ++gi) issue(gi);
+        const float inv = __fdividef(1.f, l);
+        float o[VEC];
+#pragma unroll
+        for (int t2 = 0; t2 < VEC; ++t2) o[t2] = fmaxf(fmaf(acc[t2], inv, bs[t2]), 0.f);
+        store_vec(h_out + size_t(lrow) * H + c0, o);
+        rs += 1;
+        continue;
+      }
+      // ---- the list: for each row its own index, then its producers', all window-relative ----------
+      __syncwarp();
+      const int total = cnt + (sm.rp[rs + cnt] - eb);
+      if (lane < cnt) {
+        const int e0 = sm.rp[rs + lane] - eb, n = sm.rp[rs + lane + 1] - eb - e0;
+        int pos = lane + e0;
+        sm.item[pos++] = int32_t(r0) + rs + lane - win.win_base;
+        for (int t = 0; t < n; ++t) sm.item[pos++] = __ldg(col + eb + e0 + t) - win.win_base;
+      }
+      if (lane < 4) sm.item[total + lane] = int32_t(r0) + rs - win.win_base;   // pad the last group
+      __syncwarp();
+      const int ngroups = (total + 3) >> 2;
+      if (lane == 0) {
+        uint32_t s = slot;
+        for (int gi = 0; gi < min(G, ngroups); ++gi) { issue(gi, s); s = (s + 1 == G) ? 0 : s + 1; }
+      }
 
-        // ---- consume ----------------------------------------------------------------------------------
-        int i = 0;
-        auto next_vector = [&](uint4& raw, float2& sc) -> bool {
-          const int gi = i >> 2, w = i & 3;
-          const uint32_t q = q_base + gi, s = q % G;
-          if (w == 0) {
-            uint32_t ok = 1;
-            if (lane == 0) ok = mbar_wait(bar_base + 8 * s, (q / G) & 1) ? 1u : 0u;
-            ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-            if (ok && lane != 0) ok = mbar_try(bar_base + 8 * s, (q / G) & 1) ? 1u : 0u;
-            if (!__all_sync(0xFFFFFFFFu, ok != 0)) return false;
-          }
-          raw = lds128(z_addr + s * 2048 + w * 512);
-          sc = lds64(s_addr + s * (32 * K) + w * (8 * K));
-          ++i;
-          if (w == 3 || i == total) {                            // group finished: refill its slot
-            __syncwarp();
-            if (lane == 0 && gi + G < ngroups) issue(gi + G);
-          }
-          return true;
-        };
-        const int rows_here = cnt;
-        for (int rr = 0; rr < rows_here && alive; ++rr) {
-          int n;
-          if (!huge) n = sm.rp[rs + rr + 1] - sm.rp[rs + rr];
-          else n = total - (part_begin == 0 ? 1 : 0);
-          uint4 raw;
-          float2 sc;
-          if (!huge || part_begin == 0) {                        // the row's own vector opens the softmax
-            if (!next_vector(raw, sc)) { alive = false; break; }
-            sd = sc.y;
-            m = lrelu(sc.x + sd);
-            l = 1.f;
-            unpack(raw, acc);
-            row_open = true;
-          }
-          for (int t = 0; t < n; ++t) {
-            if (!next_vector(raw, sc)) { alive = false; break; }
-            const float ev = lrelu(sc.x + sd);
-            if (ev > m) {
-              const float scale = fast_exp2(m - ev);
-              l *= scale;
+      // ---- consume: rows in order, vectors in list order ----------------------------------------------
+      int left = total;                       // vectors not yet consumed
+      int gi = 0, w = 0;                      // current group of the list, position inside it
+      uint32_t zp = z_lane + slot * ZG, sp = s_lane + slot * SG;
+      uint4 raw;
+      float2 sc;
+#define XRL_NEXT_VECTOR()                                                                          \
+  do {                                                                                             \
+    if (w == 0 && alive && !wait_all_lanes(bar_base + 8 * slot, par)) alive = false;               \
+    raw = lds128(zp);                                                                              \
+    sc = lds64(sp);                                                                                \
+    zp += 512; sp += 8 * K; ++w; --left;                                                           \
+    if (w == 4 || left == 0) {              /* group finished: refill its slot, move to the next */ \
+      __syncwarp();                                                                                \
+      if (lane == 0 && gi + G < ngroups) issue(gi + G, slot);                                      \
+      w = 0; ++gi;                                                                                 \
+      if (++slot == G) { slot = 0; par ^= 1; }                                                     \
+      zp = z_lane + slot * ZG; sp = s_lane + slot * SG;                                            \
+    }                                                                                              \
+  } while (0)
+      for (int rr = 0; rr < cnt; ++rr) {
+        const int n = sm.rp[rs + rr + 1] - sm.rp[rs + rr];
+        XRL_NEXT_VECTOR();                    // the row's own vector opens the running softmax
+        const float sd = sc.y;
+        float m = lrelu(sc.x + sd), l = 1.f, acc[VEC];
+        unpack(raw, acc);
+        for (int t = 0; t < n; ++t) {
+          XRL_NEXT_VECTOR();
+          const float ev = lrelu(sc.x + sd);
+          if (ev > m) {
+            const float scale = fast_exp2(m - ev);
+            l *= scale;
 #pragma unroll
-              for (int t2 = 0; t2 < VEC; ++t2) acc[t2] *= scale;
-              m = ev;
-            }
-            const float p = fast_exp2(ev - m);
-            l += p;
-            float z[VEC];
-            unpack(raw, z);
-#pragma unroll
-            for (int t2 = 0; t2 < VEC; ++t2) acc[t2] = fmaf(p, z[t2], acc[t2]);
+            for (int t2 = 0; t2 < VEC; ++t2) acc[t2] *= scale;
+            m = ev;
           }
-          if (!alive) break;
-          const bool row_done = !huge || (part_begin + n >= n_first);
-          if (row_done && row_open) {
-            const float inv = __fdividef(1.f, l);
-            float o[VEC];
+          const float p = fast_exp2(ev - m);
+          l += p;
+          float z[VEC];
+          unpack(raw, z);
 #pragma unroll
-            for (int t2 = 0; t2 < VEC; ++t2) o[t2] = fmaxf(fmaf(acc[t2], inv, bs[t2]), 0.f);
-            store_vec(h_out + size_t(int32_t(r0) + rs + rr - win.win_base) * H + c0, o);
-            row_open = false;
-          }
-          if (huge) part_begin += n;
+          for (int t2 = 0; t2 < VEC; ++t2) acc[t2] = fmaf(p, z[t2], acc[t2]);
         }
-        q_base += ngroups;
-      } while (alive && huge && part_begin < n_first);
+        const float inv = __fdividef(1.f, l);
+        float o[VEC];
+#pragma unroll
+        for (int t2 = 0; t2 < VEC; ++t2) o[t2] = fmaxf(fmaf(acc[t2], inv, bs[t2]), 0.f);
+        if (alive) store_vec(h_out + size_t(int32_t(r0) + rs + rr - win.win_base) * H + c0, o);
+      }
+#undef XRL_NEXT_VECTOR
       rs += cnt;
     }
   }
@@ -256,8 +267,9 @@ int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const flo
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   int64_t nb = (rows + BR * TW - 1) / (BR * TW);
   if (nb > int64_t(kNumSMs) * 5) nb = int64_t(kNumSMs) * 5;
-  k_aggregate_tma<T, K><<<int(nb), TW * 32, smem, st>>>(mz, ms, rowptr, col, bias, static_cast<T*>(h_out),
-                                                        win, status);
+  k_aggregate_tma<T, K><<<int(nb), TW * 32, smem, st>>>(mz, ms, rowptr, col, static_cast<const T*>(Z),
+                                                        reinterpret_cast<const float2*>(scores), bias,
+                                                        static_cast<T*>(h_out), win, status);
   return 1;
 }
 
