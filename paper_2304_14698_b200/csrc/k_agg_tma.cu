@@ -63,6 +63,77 @@ __device__ __forceinline__ bool wait_all_lanes(uint32_t bar, uint32_t parity) {
   return false;
 }
 
+// Two fp32 lanes per instruction (sm_100): acc = p * z + acc on register pairs.
+struct F2 { unsigned long long v; };
+__device__ __forceinline__ F2 make_f2(float lo, float hi) {
+  F2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r.v) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void split_f2(F2 a, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(a.v));
+}
+__device__ __forceinline__ void fma2(F2& acc, F2 p, F2 z) {
+  asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc.v) : "l"(p.v), "l"(z.v));
+}
+__device__ __forceinline__ void mul2(F2& acc, F2 p) {
+  asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(acc.v) : "l"(p.v));
+}
+
+// Per-lane accumulator of one destination row: NP register pairs.
+template <int VEC> struct Acc { F2 a[VEC / 2]; };
+
+// bf16: a 32-bit word holds elements (2t, 2t+1); fp32: words are the elements themselves.
+__device__ __forceinline__ void to_pairs(const uint4& raw, F2 (&z)[4]) {        // 8 bf16
+  z[0] = make_f2(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xFFFF0000u));
+  z[1] = make_f2(__uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xFFFF0000u));
+  z[2] = make_f2(__uint_as_float(raw.z << 16), __uint_as_float(raw.z & 0xFFFF0000u));
+  z[3] = make_f2(__uint_as_float(raw.w << 16), __uint_as_float(raw.w & 0xFFFF0000u));
+}
+__device__ __forceinline__ void to_pairs(const uint4& raw, F2 (&z)[2]) {        // 4 fp32
+  z[0] = make_f2(__uint_as_float(raw.x), __uint_as_float(raw.y));
+  z[1] = make_f2(__uint_as_float(raw.z), __uint_as_float(raw.w));
+}
+
+// out = ReLU(acc * inv + bias), stored in the feature type
+__device__ __forceinline__ void finish_row(bf16* dst, const F2 (&acc)[4], float inv, const float (&bs)[8]) {
+  uint32_t w[4];
+#pragma unroll
+  for (int t = 0; t < 4; ++t) {
+    float lo, hi;
+    split_f2(acc[t], lo, hi);
+    lo = fmaf(lo, inv, bs[2 * t]);
+    hi = fmaf(hi, inv, bs[2 * t + 1]);
+    asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(w[t]) : "f"(hi), "f"(lo));   // ReLU inside the rounding
+  }
+  *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+}
+__device__ __forceinline__ void finish_row(float* dst, const F2 (&acc)[2], float inv, const float (&bs)[4]) {
+  float o[4];
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    float lo, hi;
+    split_f2(acc[t], lo, hi);
+    o[2 * t] = fmaxf(fmaf(lo, inv, bs[2 * t]), 0.f);
+    o[2 * t + 1] = fmaxf(fmaf(hi, inv, bs[2 * t + 1]), 0.f);
+  }
+  *reinterpret_cast<float4*>(dst) = make_float4(o[0], o[1], o[2], o[3]);
+}
+
+// Rare path of the running softmax: the reference exponent is moved up only when a score exceeds
+// it by more than 32 (so every weight stays below 2^32 and nothing overflows); kept a real branch so
+// that the common path carries no rescaling arithmetic.
+template <int NP>
+__device__ __forceinline__ void raise_reference(float ev, float& m, float& l, F2 (&acc)[NP]) {
+  asm volatile("" ::: "memory");          // keeps this a real (rarely taken) branch, not predicated code
+  const float scale = fast_exp2(m - ev);
+  l *= scale;
+  const F2 s2 = make_f2(scale, scale);
+#pragma unroll
+  for (int t = 0; t < NP; ++t) mul2(acc[t], s2);
+  m = ev;
+}
+
 template <typename T, int K>
 __global__ void __launch_bounds__(TW * 32, 5)
 k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant__ CUtensorMap map_s,
@@ -70,6 +141,7 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
                 const T* __restrict__ Z, const float2* __restrict__ scores,
                 const float* __restrict__ bias, T* __restrict__ h_out, Window win, int32_t* status) {
   constexpr int VEC = VecOf<T>::N;
+  constexpr int NP = VEC / 2;
   constexpr int H = 32 * VEC;
   constexpr uint32_t GROUP_BYTES = 4 * 512 + 4 * K * 8;
   constexpr uint32_t ZG = 2048, SG = 32 * K;          // bytes per group in the two rings
@@ -129,30 +201,22 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
         const int n = sm.rp[rs + 1] - eb;
         const float2 self = __ldg(scores + size_t(lrow) * K + head);
         const float sd = self.y;
-        float m = lrelu(self.x + sd), l = 1.f, acc[VEC];
-        load_vec(Z + size_t(lrow) * H + c0, acc);
+        float m = lrelu(self.x + sd), l = 1.f;
+        F2 acc[NP];
+        to_pairs(__ldg(reinterpret_cast<const uint4*>(Z + size_t(lrow) * H + c0)), acc);
         for (int t = 0; t < n; ++t) {
           const int32_t j = __ldg(col + eb + t) - win.win_base;
           const float ev = lrelu(__ldg(&scores[size_t(j) * K + head].x) + sd);
-          float z[VEC];
-          load_vec(Z + size_t(j) * H + c0, z);
-          if (ev > m) {
-            const float scale = fast_exp2(m - ev);
-            l *= scale;
-#pragma unroll
-            for (int t2 = 0; t2 < VEC; ++t2) acc[t2] *= scale;
-            m = ev;
-          }
+          F2 z[NP];
+          to_pairs(__ldg(reinterpret_cast<const uint4*>(Z + size_t(j) * H + c0)), z);
+          if (ev > m + 32.f) raise_reference<NP>(ev, m, l, acc);
           const float p = fast_exp2(ev - m);
           l += p;
+          const F2 p2 = make_f2(p, p);
 #pragma unroll
-          for (int t2 = 0; t2 < VEC; ++t2) acc[t2] = fmaf(p, z[t2], acc[t2]);
+          for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], p2, z[t2]);
         }
-        const float inv = __fdividef(1.f, l);
-        float o[VEC];
-#pragma unroll
-        for (int t2 = 0; t2 < VEC; ++t2) o[t2] = fmaxf(fmaf(acc[t2], inv, bs[t2]), 0.f);
-        store_vec(h_out + size_t(lrow) * H + c0, o);
+        finish_row(h_out + size_t(lrow) * H + c0, acc, __fdividef(1.f, l), bs);
         rs += 1;
         continue;
       }
@@ -174,55 +238,52 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
       }
 
       // ---- consume: rows in order, vectors in list order ----------------------------------------------
-      int left = total;                       // vectors not yet consumed
-      int gi = 0, w = 0;                      // current group of the list, position inside it
+      int gi = 0, w = 4;                      // current group of the list, vectors left in it
       uint32_t zp = z_lane + slot * ZG, sp = s_lane + slot * SG;
-      uint4 raw;
-      float2 sc;
-#define XRL_NEXT_VECTOR()                                                                          \
-  do {                                                                                             \
-    if (w == 0 && alive && !wait_all_lanes(bar_base + 8 * slot, par)) alive = false;               \
-    raw = lds128(zp);                                                                              \
-    sc = lds64(sp);                                                                                \
-    zp += 512; sp += 8 * K; ++w; --left;                                                           \
-    if (w == 4 || left == 0) {              /* group finished: refill its slot, move to the next */ \
-      __syncwarp();                                                                                \
-      if (lane == 0 && gi + G < ngroups) issue(gi + G, slot);                                      \
-      w = 0; ++gi;                                                                                 \
-      if (++slot == G) { slot = 0; par ^= 1; }                                                     \
-      zp = z_lane + slot * ZG; sp = s_lane + slot * SG;                                            \
-    }                                                                                              \
-  } while (0)
+      if (!wait_all_lanes(bar_base + 8 * slot, par)) alive = false;
+      // group finished: refill its slot with group gi + G, move on, wait for the next one
+      auto advance = [&]() {
+        __syncwarp();
+        if (lane == 0 && gi + G < ngroups) issue(gi + G, slot);
+        ++gi;
+        if (++slot == G) { slot = 0; par ^= 1; }
+        zp = z_lane + slot * ZG;
+        sp = s_lane + slot * SG;
+        w = 4;
+        if (gi < ngroups && alive && !wait_all_lanes(bar_base + 8 * slot, par)) alive = false;
+      };
       for (int rr = 0; rr < cnt; ++rr) {
         const int n = sm.rp[rs + rr + 1] - sm.rp[rs + rr];
-        XRL_NEXT_VECTOR();                    // the row's own vector opens the running softmax
+        // the row's own vector opens the running softmax: reference exponent = its score, weight 1
+        uint4 raw = lds128(zp);
+        float2 sc = lds64(sp);
+        zp += 512; sp += 8 * K;
+        if (--w == 0) advance();
         const float sd = sc.y;
-        float m = lrelu(sc.x + sd), l = 1.f, acc[VEC];
-        unpack(raw, acc);
+        float m = lrelu(sc.x + sd), l = 1.f;
+        F2 acc[NP];
+        to_pairs(raw, acc);
         for (int t = 0; t < n; ++t) {
-          XRL_NEXT_VECTOR();
+          raw = lds128(zp);
+          sc = lds64(sp);
+          zp += 512; sp += 8 * K;
+          if (--w == 0) advance();
           const float ev = lrelu(sc.x + sd);
-          if (ev > m) {
-            const float scale = fast_exp2(m - ev);
-            l *= scale;
-#pragma unroll
-            for (int t2 = 0; t2 < VEC; ++t2) acc[t2] *= scale;
-            m = ev;
-          }
+          if (ev > m + 32.f) raise_reference<NP>(ev, m, l, acc);
           const float p = fast_exp2(ev - m);
           l += p;
-          float z[VEC];
-          unpack(raw, z);
+          F2 z[NP];
+          to_pairs(raw, z);
+          const F2 p2 = make_f2(p, p);
 #pragma unroll
-          for (int t2 = 0; t2 < VEC; ++t2) acc[t2] = fmaf(p, z[t2], acc[t2]);
+          for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], p2, z[t2]);
         }
-        const float inv = __fdividef(1.f, l);
-        float o[VEC];
-#pragma unroll
-        for (int t2 = 0; t2 < VEC; ++t2) o[t2] = fmaxf(fmaf(acc[t2], inv, bs[t2]), 0.f);
-        if (alive) store_vec(h_out + size_t(int32_t(r0) + rs + rr - win.win_base) * H + c0, o);
+        finish_row(h_out + size_t(int32_t(r0) + rs + rr - win.win_base) * H + c0, acc, __fdividef(1.f, l), bs);
       }
-#undef XRL_NEXT_VECTOR
+      if (w != 4) {                            // the list ended inside a group: retire it without waiting
+        __syncwarp();
+        if (++slot == G) { slot = 0; par ^= 1; }
+      }
       rs += cnt;
     }
   }
