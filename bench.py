@@ -273,8 +273,19 @@ def main():
     # ---- end to end: host buffers in, results out, through the public call ---------------------------
     e2e = None
     if not args.no_e2e:
-        host = {k: batch[k] for k in ("n_nodes", "n_edges", "env_off", "op", "edge_src", "edge_dst")}
-        host["shape"] = agent.storage_shape(batch["shape"])
+        # host inputs live in page-locked memory (the library then copies straight out of them)
+        pinned = {}
+
+        def pin(a):
+            t = torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+            pinned[id(t)] = t
+            return t.numpy()
+
+        host = {k: batch[k] for k in ("n_nodes", "n_edges", "env_off")}
+        for k in ("op", "edge_src", "edge_dst"):
+            host[k] = pin(batch[k])
+        host["shape"] = pin(agent.storage_shape(batch["shape"]).view(np.int16) if bf16
+                            else agent.storage_shape(batch["shape"]))
         mask_h = torch.from_numpy(batch["mask"]).pin_memory()
         h2d = sum(host[k].nbytes for k in ("op", "edge_src", "edge_dst", "shape", "n_nodes", "n_edges",
                                            "env_off")) + batch["mask"].nbytes

@@ -123,7 +123,10 @@ xrl_status xrl_pack(xrl_ctx* ctx, const xrl_graph* graphs, int32_t num_graphs,
 /* Same operation on already concatenated arrays.  n_nodes, n_edges [num_graphs] and env_off
  * are always HOST; op [N], shape [N x S], edge_src [E], edge_dst [E] (local ids, graphs back
  * to back) are HOST or DEVICE according to `where` (XRL_MEM_*).  DEVICE arrays are read by the
- * kernels directly and must stay valid until the stream has passed the call. */
+ * kernels directly and must stay valid until the stream has passed the call.  HOST arrays in
+ * pageable memory are staged through a pinned buffer before the call returns; HOST arrays that are
+ * all page-locked (cudaHostAlloc / cudaHostRegister) are copied asynchronously straight from the
+ * caller's memory and must then also stay valid until the stream has passed the call. */
 xrl_status xrl_pack_flat(xrl_ctx* ctx, int32_t where, int32_t num_graphs, const int32_t* n_nodes,
                          const int32_t* n_edges, const int32_t* op, const void* shape,
                          const int32_t* edge_src, const int32_t* edge_dst, const int32_t* env_off,

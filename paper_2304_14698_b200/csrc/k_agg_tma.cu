@@ -20,7 +20,13 @@ using namespace umma;
 namespace {
 
 constexpr int TW = 4;            // warps per CTA
-constexpr int G = 4;             // gather groups (of four rows) in flight per warp
+#ifndef XRL_AGG_GROUPS
+#define XRL_AGG_GROUPS 4
+#endif
+#ifndef XRL_AGG_CTAS
+#define XRL_AGG_CTAS 5
+#endif
+constexpr int G = XRL_AGG_GROUPS;   // gather groups (of four rows) in flight per warp
 constexpr int BR = 32;           // destination rows per block
 constexpr int ITEMS = 160;       // list capacity, a multiple of 4
 
@@ -135,7 +141,7 @@ __device__ __forceinline__ void raise_reference(float ev, float& m, float& l, F2
 }
 
 template <typename T, int K>
-__global__ void __launch_bounds__(TW * 32, 5)
+__global__ void __launch_bounds__(TW * 32, XRL_AGG_CTAS)
 k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant__ CUtensorMap map_s,
                 const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
                 const T* __restrict__ Z, const float2* __restrict__ scores,
@@ -327,7 +333,7 @@ int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const flo
     return -1;
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   int64_t nb = (rows + BR * TW - 1) / (BR * TW);
-  if (nb > int64_t(kNumSMs) * 5) nb = int64_t(kNumSMs) * 5;
+  if (nb > int64_t(kNumSMs) * XRL_AGG_CTAS) nb = int64_t(kNumSMs) * XRL_AGG_CTAS;
   k_aggregate_tma<T, K><<<int(nb), TW * 32, smem, st>>>(mz, ms, rowptr, col, static_cast<const T*>(Z),
                                                         reinterpret_cast<const float2*>(scores), bias,
                                                         static_cast<T*>(h_out), win, status);

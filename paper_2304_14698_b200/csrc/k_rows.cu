@@ -2,8 +2,6 @@
 // attention half-scores, and the edge-score / segment-softmax / weighted-aggregate step of a
 // graph-attention layer (Eq. 7).  One group of LPR lanes owns one destination row and moves it
 // as 16-byte vectors (VPL vectors per lane); 32 / LPR rows share a warp.
-#include <stdlib.h>
-
 #include "xrl_internal.cuh"
 
 namespace xrl {
@@ -272,153 +270,6 @@ k_aggregate(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
   }
 }
 
-// ---- Eq. 7 for 512-byte rows (hidden 256 in bf16, 128 in fp32): gathers through a cp.async ring ---
-// Same arithmetic as k_aggregate with one producer per softmax update.  The vectors a warp has to
-// gather for a block of rows (each row's own Z vector, then its producers') form one sequence;
-// every lane copies its 16 bytes of vector i + kRing - 1 (and its head's pair of half-scores) into
-// a private shared-memory slot with cp.async while it consumes vector i, so that several gathers
-// per warp are always in flight without holding them in registers.
-constexpr int kRing = 6;
-constexpr int kRingItems = kAggBlockRows + kAggColCap;
-
-__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(uint32_t(__cvta_generic_to_shared(dst))), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async8(void* dst, const void* src) {
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(uint32_t(__cvta_generic_to_shared(dst))), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-
-template <typename T>
-__global__ void __launch_bounds__(kRowThreads, 4)
-k_aggregate_ring(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
-                 const T* __restrict__ Z, const float2* __restrict__ scores,
-                 const float* __restrict__ bias, T* __restrict__ h_out, int K, Window win) {
-  constexpr int VEC = VecOf<T>::N;
-  constexpr int H = 32 * VEC;
-  constexpr int WARPS = kRowThreads / 32;
-  __shared__ int32_t s_rp[WARPS][kAggBlockRows + 1];
-  __shared__ int32_t s_item[WARPS][kRingItems];
-  __shared__ uint4 s_z[WARPS][kRing][32];
-  __shared__ float2 s_sc[WARPS][kRing][32];
-  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-  const int warps_total = (gridDim.x * blockDim.x) >> 5;
-  const int warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int c0 = lane * VEC;
-  const T* zlane = Z + c0;
-  const float2* slane = scores + c0 / (H / K);
-  float bs[VEC];
-#pragma unroll
-  for (int t = 0; t < VEC; ++t) bs[t] = __ldg(bias + c0 + t);
-  int32_t* item = s_item[wib];
-  uint4* ring_z = &s_z[wib][0][lane];
-  float2* ring_s = &s_sc[wib][0][lane];
-
-  auto issue = [&](int i, int total, int slot) {
-    if (i < total) {
-      const int32_t idx = item[i];
-      cp_async16(ring_z + slot * 32, zlane + size_t(idx) * H);
-      cp_async8(ring_s + slot * 32, slane + size_t(idx) * K);
-    }
-    cp_async_commit();                    // an empty group keeps the group count in step
-  };
-
-  for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * kAggBlockRows; r0 < win.row_end;
-       r0 += int64_t(warps_total) * kAggBlockRows) {
-    const int nr = int(min(int64_t(kAggBlockRows), win.row_end - r0));
-    __syncwarp();
-    if (lane < nr) s_rp[wib][lane] = __ldg(rowptr + r0 + lane);
-    if (lane == 0) s_rp[wib][nr] = __ldg(rowptr + r0 + nr);
-    __syncwarp();
-    int rs = 0;
-    while (rs < nr) {
-      // as many rows from rs on as keep (rows + producers) within the item list
-      const int32_t eb = s_rp[wib][rs];
-      const bool fits = (rs + lane < nr) && (lane + 1 + s_rp[wib][rs + lane + 1] - eb <= kRingItems);
-      const uint32_t fmask = __ballot_sync(0xFFFFFFFFu, fits);
-      const int cnt = __ffs(~fmask) - 1 < 0 ? 32 : __ffs(~fmask) - 1;      // leading run of fitting rows
-      if (cnt == 0) {
-        // a single row with more producers than the list holds: walk it straight from global memory
-        const int32_t lrow = int32_t(r0) + rs - win.win_base;
-        const int n = s_rp[wib][rs + 1] - eb;
-        const float2 self = __ldg(slane + size_t(lrow) * K);
-        const float sd = self.y;
-        float m = lrelu(self.x + sd), l = 1.f, acc[VEC];
-        load_vec(zlane + size_t(lrow) * H, acc);
-        int t = 0;
-        for (; t + 4 <= n; t += 4) agg_group<T, 4>(col + eb + t, win.win_base, zlane, slane, H, K, sd, m, l, acc);
-        for (; t < n; ++t) agg_group<T, 1>(col + eb + t, win.win_base, zlane, slane, H, K, sd, m, l, acc);
-        const float inv = __fdividef(1.f, l);
-        float o[VEC];
-#pragma unroll
-        for (int t2 = 0; t2 < VEC; ++t2) o[t2] = fmaxf(fmaf(acc[t2], inv, bs[t2]), 0.f);
-        store_vec(h_out + size_t(lrow) * H + c0, o);
-        rs += 1;
-        continue;
-      }
-      // item list: for each row its own index, then its producers', all window-relative
-      __syncwarp();
-      if (lane < cnt) {
-        const int e0 = s_rp[wib][rs + lane] - eb, n = s_rp[wib][rs + lane + 1] - eb - e0;
-        int pos = lane + e0;
-        item[pos++] = int32_t(r0) + rs + lane - win.win_base;
-        for (int t = 0; t < n; ++t) item[pos++] = __ldg(col + eb + e0 + t) - win.win_base;
-      }
-      __syncwarp();
-      const int total = cnt + (s_rp[wib][rs + cnt] - eb);
-#pragma unroll
-      for (int i = 0; i < kRing - 1; ++i) issue(i, total, i);
-      int i = 0, cslot = 0, pslot = kRing - 1;
-      for (int rr = 0; rr < cnt; ++rr) {
-        const int n = s_rp[wib][rs + rr + 1] - s_rp[wib][rs + rr];
-        const int32_t lrow = int32_t(r0) + rs + rr - win.win_base;
-        // the row's own vector opens the running softmax
-        cp_async_wait<kRing - 2>();
-        uint4 raw = ring_z[cslot * 32];
-        float2 sc = ring_s[cslot * 32];
-        asm volatile("" ::: "memory");
-        issue(i + kRing - 1, total, pslot);
-        ++i; cslot = cslot + 1 == kRing ? 0 : cslot + 1; pslot = pslot + 1 == kRing ? 0 : pslot + 1;
-        const float sd = sc.y;
-        float m = lrelu(sc.x + sd), l = 1.f, acc[VEC];
-        unpack(raw, acc);
-        for (int t = 0; t < n; ++t) {
-          cp_async_wait<kRing - 2>();
-          raw = ring_z[cslot * 32];
-          sc = ring_s[cslot * 32];
-          asm volatile("" ::: "memory");
-          issue(i + kRing - 1, total, pslot);
-          ++i; cslot = cslot + 1 == kRing ? 0 : cslot + 1; pslot = pslot + 1 == kRing ? 0 : pslot + 1;
-          const float ev = lrelu(sc.x + sd);
-          if (ev > m) {
-            const float scale = fast_exp2(m - ev);
-            l *= scale;
-#pragma unroll
-            for (int t2 = 0; t2 < VEC; ++t2) acc[t2] *= scale;
-            m = ev;
-          }
-          const float p = fast_exp2(ev - m);
-          l += p;
-          float z[VEC];
-          unpack(raw, z);
-#pragma unroll
-          for (int t2 = 0; t2 < VEC; ++t2) acc[t2] = fmaf(p, z[t2], acc[t2]);
-        }
-        const float inv = __fdividef(1.f, l);
-        float o[VEC];
-#pragma unroll
-        for (int t2 = 0; t2 < VEC; ++t2) o[t2] = fmaxf(fmaf(acc[t2], inv, bs[t2]), 0.f);
-        store_vec(h_out + size_t(lrow) * H + c0, o);
-      }
-      cp_async_wait<0>();
-      rs += cnt;
-    }
-  }
-}
-
 // ---- dispatch on the row geometry ------------------------------------------------------------
 struct RowGeom { int lpr, vpl; };
 
@@ -483,23 +334,9 @@ int launch_aggregate(const Dims& d, const int32_t* rowptr, const int32_t* col, c
                      Window win, int64_t buf_rows, int32_t* status, cudaStream_t st) {
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   if (rows <= 0) return 0;
-  static const char* mode = getenv("XRL_AGG");            // "ring" / "plain": bypass the TMA gather kernel
-  if (mode == nullptr) {
+  {   // 512-byte rows with 4 | K: gathers by the TMA engine
     const int k = launch_aggregate_tma(d, rowptr, col, Z, scores, bias, h_out, win, buf_rows, status, st);
     if (k >= 0) return k;
-  }
-  const bool plain = mode != nullptr && mode[0] == 'p';
-  if (!plain && d.dtype == XRL_BF16 && d.H == 256) {
-    k_aggregate_ring<bf16><<<row_grid(rows, kAggBlockRows), kRowThreads, 0, st>>>(
-        rowptr, col, static_cast<const bf16*>(Z), reinterpret_cast<const float2*>(scores), bias,
-        static_cast<bf16*>(h_out), d.K, win);
-    return 1;
-  }
-  if (!plain && d.dtype == XRL_FP32 && d.H == 128) {
-    k_aggregate_ring<float><<<row_grid(rows, kAggBlockRows), kRowThreads, 0, st>>>(
-        rowptr, col, static_cast<const float*>(Z), reinterpret_cast<const float2*>(scores), bias,
-        static_cast<float*>(h_out), d.K, win);
-    return 1;
   }
 #define CALL(TY_, LPR, VPL)                                                                        \
   k_aggregate<TY_, LPR, VPL><<<row_grid(rows, kAggBlockRows), kRowThreads, 0, st>>>(                \

@@ -183,6 +183,15 @@ xrl_status ensure_bulk_staging(xrl_batch* b) {
   return XRL_OK;
 }
 
+// True if p is page-locked host memory (cudaHostAlloc / cudaHostRegister): asynchronous copies can
+// then read it directly.  A null pointer counts as pinned (nothing to copy).
+bool pinned(const void* p) {
+  if (p == nullptr) return true;
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, p) != cudaSuccess) { cudaGetLastError(); return false; }
+  return a.type == cudaMemoryTypeHost;
+}
+
 // Shared tail of both pack entry points.  `graphs` non-null: gather from per-graph host arrays.
 xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int32_t num_graphs,
                        const int32_t* n_nodes, const int32_t* n_edges, const int32_t* op,
@@ -222,7 +231,9 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
     return XRL_ERR_STATE;
   }
   xrl_status s = ensure_staging(b);
-  if (s == XRL_OK && (graphs || where == XRL_MEM_HOST)) s = ensure_bulk_staging(b);
+  const bool direct = !graphs && where == XRL_MEM_HOST && pinned(op) && pinned(shape) &&
+                      pinned(edge_src) && pinned(edge_dst);
+  if (s == XRL_OK && (graphs || where == XRL_MEM_HOST) && !direct) s = ensure_bulk_staging(b);
   if (s != XRL_OK) { if (*out == nullptr) xrl_batch_free(ctx, b); return s; }
   *out = b;
   b->packed = false;
@@ -262,7 +273,19 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
   // ---- bulk arrays -------------------------------------------------------------------------------
   const size_t sb = storage_bytes(c.dtype);
   const int32_t *d_src, *d_dst;
-  if (graphs || where == XRL_MEM_HOST) {
+  if (direct) {
+    // page-locked caller memory: copy straight from it, no staging pass
+    if (N) {
+      XRL_CUDA(cudaMemcpyAsync(b->op.p, op, 4 * size_t(N), cudaMemcpyHostToDevice, st));
+      XRL_CUDA(cudaMemcpyAsync(b->shape.p, shape, sb * kS * size_t(N), cudaMemcpyHostToDevice, st));
+    }
+    if (E) {
+      XRL_CUDA(cudaMemcpyAsync(b->edge_src.p, edge_src, 4 * size_t(E), cudaMemcpyHostToDevice, st));
+      XRL_CUDA(cudaMemcpyAsync(b->edge_dst.p, edge_dst, 4 * size_t(E), cudaMemcpyHostToDevice, st));
+    }
+    d_src = b->edge_src.as<int32_t>();
+    d_dst = b->edge_dst.as<int32_t>();
+  } else if (graphs || where == XRL_MEM_HOST) {
     char* p_op = b->h_bulk;
     char* p_shape = p_op + 4 * size_t(N);
     char* p_src = p_shape + sb * kS * size_t(N);

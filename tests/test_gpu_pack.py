@@ -21,6 +21,14 @@ def _compare(xo, batch, via):
             ag.pack_graphs(dags.split(batch), batch["env_off"])
         elif via == "flat_host":
             ag.pack(batch)
+        elif via == "flat_pinned":          # page-locked host arrays: copied without staging
+            keep = {k: torch.from_numpy(batch[k]).pin_memory() for k in ("op", "edge_src", "edge_dst")}
+            shp = ag.storage_shape(batch["shape"])
+            keep["shape"] = torch.from_numpy(shp.view(np.int16) if shp.dtype == np.uint16 else shp).pin_memory()
+            ag.batch = xrl.xrl_pack_flat(ag.ctx, 0, batch["n_nodes"], batch["n_edges"], keep["op"].numpy(),
+                                         keep["shape"].numpy(), keep["edge_src"].numpy(),
+                                         keep["edge_dst"].numpy(), batch["env_off"], batch=ag.batch)
+            torch.cuda.synchronize()
         else:
             dev = {k: batch[k] for k in ("n_nodes", "n_edges", "env_off")}
             for k in ("op", "edge_src", "edge_dst"):
@@ -38,7 +46,7 @@ def _compare(xo, batch, via):
         ag.close()
 
 
-@pytest.mark.parametrize("via", ["graphs", "flat_host", "flat_device"])
+@pytest.mark.parametrize("via", ["graphs", "flat_host", "flat_pinned", "flat_device"])
 @pytest.mark.parametrize("cfg,kw", [(1, {}), (2, {}), (3, dict(candidates=31)), (4, dict(candidates=15)),
                                     (5, dict(candidates=7, envs=5))])
 def test_pack_bit_exact(xo, cfg, kw, via):
