@@ -367,7 +367,7 @@ def main():
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from the
 # ncu capture summarised under profiles/; filled in once a capture of the current kernel exists.
-TRAFFIC = {(4, "aggregate"): 4.62e9}   # 577 MB on the 128-graph capture, scaled by the node count
+TRAFFIC = {(4, "aggregate"): 4.65e9}   # 581.5 MB on the 128-graph capture, scaled by the node count
 
 if __name__ == "__main__":
     main()
