@@ -126,6 +126,19 @@ __device__ __forceinline__ void finish_row(float* dst, const F2 (&acc)[2], float
   *reinterpret_cast<float4*>(dst) = make_float4(o[0], o[1], o[2], o[3]);
 }
 
+// out = ReLU(acc * inv + bias) kept in fp32 (for the fused per-graph readout)
+template <int NP>
+__device__ __forceinline__ void finish_row_f32(const F2 (&acc)[NP], float inv, const float (&bs)[2 * NP],
+                                               float (&o)[2 * NP]) {
+#pragma unroll
+  for (int t = 0; t < NP; ++t) {
+    float lo, hi;
+    split_f2(acc[t], lo, hi);
+    o[2 * t] = fmaxf(fmaf(lo, inv, bs[2 * t]), 0.f);
+    o[2 * t + 1] = fmaxf(fmaf(hi, inv, bs[2 * t + 1]), 0.f);
+  }
+}
+
 // Rare path of the running softmax: the reference exponent is moved up only when a score exceeds
 // it by more than 32 (so every weight stays below 2^32 and nothing overflows); kept a real branch so
 // that the common path carries no rescaling arithmetic.
@@ -140,12 +153,20 @@ __device__ __forceinline__ void raise_reference(float ev, float& m, float& l, F2
   m = ev;
 }
 
-template <typename T, int K>
+// READOUT = true is the last attention layer fused with the per-graph sum of Eq. 8: the layer output
+// is not stored; each warp adds the rows of its 32-row block per graph, in row order, and writes
+//   partial[b]           the rows of block b that belong to the graph of the block's first row
+//   partial[nblocks + g] the rows of graph g inside the block in which g starts, when that is not at
+//                        the block's first row
+// (k_global_update_blocks adds them per graph in a fixed order).  Needs row_begin = win_base = 0.
+template <typename T, int K, bool READOUT>
 __global__ void __launch_bounds__(TW * 32, XRL_AGG_CTAS)
 k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant__ CUtensorMap map_s,
                 const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
                 const T* __restrict__ Z, const float2* __restrict__ scores,
-                const float* __restrict__ bias, T* __restrict__ h_out, Window win, int32_t* status) {
+                const float* __restrict__ bias, T* __restrict__ h_out, Window win,
+                const int32_t* __restrict__ seg_id, float* __restrict__ partial, int32_t nblocks,
+                int32_t* status) {
   constexpr int VEC = VecOf<T>::N;
   constexpr int NP = VEC / 2;
   constexpr int H = 32 * VEC;
@@ -194,6 +215,35 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
     if (lane < nr) sm.rp[lane] = __ldg(rowptr + r0 + lane);
     if (lane == 0) sm.rp[nr] = __ldg(rowptr + r0 + nr);
     __syncwarp();
+    // fused readout: running per-graph sum of this block's rows
+    int32_t myseg = 0, cur_g = -1;
+    bool first_seg = true;
+    float rsum[VEC];
+    if (READOUT) {
+      myseg = (lane < nr) ? __ldg(seg_id + r0 + lane) : 0;
+#pragma unroll
+      for (int t = 0; t < VEC; ++t) rsum[t] = 0.f;
+    }
+    auto flush = [&]() {
+      float* dst = partial + size_t(first_seg ? int32_t(r0 / BR) : nblocks + cur_g) * H + c0;
+#pragma unroll
+      for (int t = 0; t < VEC; t += 4)
+        *reinterpret_cast<float4*>(dst + t) = make_float4(rsum[t], rsum[t + 1], rsum[t + 2], rsum[t + 3]);
+    };
+    auto add_row = [&](int row_in_block, const float (&o)[VEC]) {
+      const int32_t g = __shfl_sync(0xFFFFFFFFu, myseg, row_in_block);
+      if (g != cur_g) {
+        if (cur_g >= 0) {
+          flush();
+          first_seg = false;
+#pragma unroll
+          for (int t = 0; t < VEC; ++t) rsum[t] = 0.f;
+        }
+        cur_g = g;
+      }
+#pragma unroll
+      for (int t = 0; t < VEC; ++t) rsum[t] += o[t];
+    };
     int rs = 0;
     while (rs < nr && alive) {
       // as many rows from rs on as keep (rows + producers) within the list
@@ -222,7 +272,13 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
 #pragma unroll
           for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], p2, z[t2]);
         }
-        finish_row(h_out + size_t(lrow) * H + c0, acc, __fdividef(1.f, l), bs);
+        if (READOUT) {
+          float o[VEC];
+          finish_row_f32<NP>(acc, __fdividef(1.f, l), bs, o);
+          add_row(rs, o);
+        } else {
+          finish_row(h_out + size_t(lrow) * H + c0, acc, __fdividef(1.f, l), bs);
+        }
         rs += 1;
         continue;
       }
@@ -284,7 +340,13 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
 #pragma unroll
           for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], p2, z[t2]);
         }
-        finish_row(h_out + size_t(int32_t(r0) + rs + rr - win.win_base) * H + c0, acc, __fdividef(1.f, l), bs);
+        if (READOUT) {
+          float o[VEC];
+          finish_row_f32<NP>(acc, __fdividef(1.f, l), bs, o);
+          add_row(rs + rr, o);
+        } else {
+          finish_row(h_out + size_t(int32_t(r0) + rs + rr - win.win_base) * H + c0, acc, __fdividef(1.f, l), bs);
+        }
       }
       if (w != 4) {                            // the list ended inside a group: retire it without waiting
         __syncwarp();
@@ -292,6 +354,7 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
       }
       rs += cnt;
     }
+    if (READOUT && cur_g >= 0) flush();
   }
   if (!alive) {
     if (lane == 0) raise(status, XRL_ERR_TIMEOUT);
@@ -312,14 +375,15 @@ bool make_row_map(CUtensorMap* m, const void* ptr, CUtensorMapDataType dt, uint3
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <typename T, int K>
+template <typename T, int K, bool READOUT>
 int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const float* scores, const float* bias,
-             void* h_out, Window win, int64_t buf_rows, int32_t* status, cudaStream_t st) {
+             void* h_out, Window win, int64_t buf_rows, const int32_t* seg_id, float* partial,
+             int32_t* status, cudaStream_t st) {
   static bool attr = false;
   const size_t smem = sizeof(WarpSmem<K>) * TW;
   if (!attr) {
-    if (cudaFuncSetAttribute(k_aggregate_tma<T, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) !=
-        cudaSuccess) {
+    if (cudaFuncSetAttribute(k_aggregate_tma<T, K, READOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             int(smem)) != cudaSuccess) {
       cudaGetLastError();
       return -1;
     }
@@ -332,33 +396,47 @@ int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const flo
       !make_row_map(&ms, scores, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, uint64_t(buf_rows), 2 * K))
     return -1;
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
+  const int64_t nblocks = (rows + BR - 1) / BR;
   int64_t nb = (rows + BR * TW - 1) / (BR * TW);
   if (nb > int64_t(kNumSMs) * XRL_AGG_CTAS) nb = int64_t(kNumSMs) * XRL_AGG_CTAS;
-  k_aggregate_tma<T, K><<<int(nb), TW * 32, smem, st>>>(mz, ms, rowptr, col, static_cast<const T*>(Z),
-                                                        reinterpret_cast<const float2*>(scores), bias,
-                                                        static_cast<T*>(h_out), win, status);
+  k_aggregate_tma<T, K, READOUT><<<int(nb), TW * 32, smem, st>>>(
+      mz, ms, rowptr, col, static_cast<const T*>(Z), reinterpret_cast<const float2*>(scores), bias,
+      static_cast<T*>(h_out), win, seg_id, partial, int32_t(nblocks), status);
   return 1;
 }
 
 }  // namespace
 
 // buf_rows: rows of the Z / scores buffers reachable from this window (indices are window-relative).
-// Returns kernels launched, or -1 when this shape is not handled here.
+// partial != nullptr selects the variant fused with the per-graph sum (then h_out is not written and
+// the window must start at row 0).  Returns kernels launched, or -1 when this shape is not handled here.
 int launch_aggregate_tma(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z,
                          const float* scores, const float* bias, void* h_out, Window win, int64_t buf_rows,
-                         int32_t* status, cudaStream_t st) {
+                         const int32_t* seg_id, float* partial, int32_t* status, cudaStream_t st) {
   if (encode_fn() == nullptr) return -1;
   const bool bf = d.dtype == XRL_BF16 && d.H == 256, fp = d.dtype == XRL_FP32 && d.H == 128;
   if (!bf && !fp) return -1;
-#define TMA_CASE(KK)                                                                                     \
-  case KK:                                                                                               \
-    return bf ? launch_k<bf16, KK>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, status, st)       \
-              : launch_k<float, KK>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, status, st);
+  if (partial != nullptr && (win.row_begin != 0 || win.win_base != 0)) return -1;
+#define TMA_CASE(KK)                                                                                       \
+  case KK:                                                                                                 \
+    if (partial != nullptr)                                                                                \
+      return bf ? launch_k<bf16, KK, true>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, seg_id,     \
+                                           partial, status, st)                                            \
+                : launch_k<float, KK, true>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, seg_id,    \
+                                            partial, status, st);                                          \
+    return bf ? launch_k<bf16, KK, false>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, seg_id,      \
+                                          partial, status, st)                                             \
+              : launch_k<float, KK, false>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, seg_id,     \
+                                           partial, status, st);
   switch (d.K) {
     TMA_CASE(4) TMA_CASE(8) TMA_CASE(16)
     default: return -1;
   }
 #undef TMA_CASE
 }
+
+// Partial-sum slots the fused variant writes for `rows` rows and B graphs.
+int64_t aggregate_readout_slots(int64_t rows, int64_t B) { return (rows + BR - 1) / BR + B; }
+int32_t aggregate_readout_blocks(int64_t rows) { return int32_t((rows + BR - 1) / BR); }
 
 }  // namespace xrl

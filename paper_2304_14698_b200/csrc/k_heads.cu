@@ -77,6 +77,35 @@ k_global_update(const float* __restrict__ partial, const int32_t* __restrict__ g
   }
 }
 
+// Eq. 8 from the partial sums written by the aggregate kernel fused with the readout: per graph, the
+// partial of the block in which the graph starts (if it does not start at the block's first row), then
+// the partials of the following 32-row blocks whose first row belongs to the graph, in order.
+__global__ void __launch_bounds__(256)
+k_global_update_blocks(const float* __restrict__ partial, const int32_t* __restrict__ node_off,
+                       int32_t nblocks, const float* __restrict__ g0, const float* __restrict__ Wg,
+                       const float* __restrict__ bg, float* __restrict__ emb, int H, int Dg) {
+  extern __shared__ float u[];                   // [H + Dg]
+  const int32_t g = blockIdx.x;
+  const int32_t start = node_off[g], end = node_off[g + 1];
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    float s = 0.f;
+    if (end > start) {
+      int32_t b0 = start >> 5;
+      if (start & 31) { s += partial[size_t(nblocks + g) * H + c]; ++b0; }
+      const int32_t b1 = (end - 1) >> 5;
+      for (int32_t b = b0; b <= b1; ++b) s += partial[size_t(b) * H + c];
+    }
+    u[c] = s;
+  }
+  for (int t = threadIdx.x; t < Dg; t += blockDim.x) u[H + t] = g0 ? g0[size_t(g) * Dg + t] : 0.f;
+  __syncthreads();
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    float acc = bg[c];
+    for (int k = 0; k < H + Dg; ++k) acc = fmaf(u[k], __ldg(Wg + size_t(k) * H + c), acc);
+    emb[size_t(g) * H + c] = fmaxf(acc, 0.f);
+  }
+}
+
 // Block-wide sum in a fixed order: every thread contributes v, thread 0's tree is the same for
 // the same blockDim.  `scratch` holds blockDim.x floats.
 __device__ float block_sum(float v, float* scratch) {
@@ -183,9 +212,35 @@ __device__ int32_t sample_row(const float* __restrict__ p, int A1, uint64_t seed
   return act;
 }
 
+// ---- sum of the valid candidates' embeddings of one environment, 32 columns per CTA ---------------
+// 1024 threads = 32 columns x 32 parts; part p adds candidates p, p + 32, ... in order, the parts are
+// then added in order: a fixed summation order, so the result is reproducible.
+__global__ void __launch_bounds__(1024)
+k_candidate_sum(const float* __restrict__ emb, const int32_t* __restrict__ env_off,
+                const uint8_t* __restrict__ mask, float* __restrict__ cand_sum, int H, int A) {
+  __shared__ float part[32][33];
+  const int32_t e = blockIdx.x;
+  const int c = blockIdx.y * 32 + (threadIdx.x & 31), p = threadIdx.x >> 5;
+  const int32_t cur = env_off[e];
+  const int32_t C = env_off[e + 1] - cur - 1;
+  const uint8_t* mk = mask + size_t(e) * A;
+  float s = 0.f;
+  if (c < H)
+    for (int a = p; a < C; a += 32)
+      if (mk[a]) s += emb[size_t(cur + 1 + a) * H + c];
+  part[p][threadIdx.x & 31] = s;
+  __syncthreads();
+  if (p == 0 && c < H) {
+    float t = 0.f;
+    for (int q = 0; q < 32; ++q) t += part[q][threadIdx.x & 31];
+    cand_sum[size_t(e) * H + c] = t;
+  }
+}
+
 // ---- per environment: masked softmax, candidate mean, value MLP, optional draw -----------------
 __global__ void __launch_bounds__(1024)
 k_env_policy(const float* __restrict__ emb, const float* __restrict__ logit,
+             const float* __restrict__ cand_sum,
              const int32_t* __restrict__ env_off, const uint8_t* __restrict__ mask,
              const float* __restrict__ vW1, const float* __restrict__ vb1,
              const float* __restrict__ vw2, const float* __restrict__ vb2, float* __restrict__ probs,
@@ -195,7 +250,6 @@ k_env_policy(const float* __restrict__ emb, const float* __restrict__ logit,
   const int nt = blockDim.x, tid = threadIdx.x;
   float* scratch = reinterpret_cast<float*>(sm64 + nt + 1);   // [nt]
   float* u = scratch + nt;                                    // [2H]
-  float* part = u + 2 * H;                                    // [parts][H]
   const int32_t e = blockIdx.x;
   const int32_t cur = env_off[e];
   const int32_t C = env_off[e + 1] - cur - 1;
@@ -230,30 +284,11 @@ k_env_policy(const float* __restrict__ emb, const float* __restrict__ logit,
   for (int a = tid; a <= A; a += nt) pr[a] = pr[a] / denom;     // each thread rewrites its own entries
 
   // value head input: [ emb(current) | mean of emb over the valid candidates ]
-  const int parts = nt / H > 0 ? nt / H : 1;
   for (int c = tid; c < H; c += nt) u[c] = emb[size_t(cur) * H + c];
-  if (tid < parts * H) {
-    const int c = tid % H, p = tid / H;
-    float s = 0.f;
-    for (int a = p; a < C; a += parts)
-      if (mk[a]) s += emb[size_t(cur + 1 + a) * H + c];
-    part[p * H + c] = s;
-  }
   float cnt = 0.f;
   for (int a = tid; a < C; a += nt) cnt += mk[a] ? 1.f : 0.f;
-  const float nv = block_sum(cnt, scratch);      // also orders the writes to part[] before the reads
-  if (nt < H) {                                   // fewer threads than columns: plain loop
-    for (int c = tid; c < H; c += nt) {
-      float s = 0.f;
-      for (int a = 0; a < C; ++a)
-        if (mk[a]) s += emb[size_t(cur + 1 + a) * H + c];
-      u[H + c] = nv > 0.f ? s / nv : 0.f;
-    }
-  } else if (tid < H) {
-    float s = 0.f;
-    for (int p = 0; p < parts; ++p) s += part[p * H + tid];
-    u[H + tid] = nv > 0.f ? s / nv : 0.f;
-  }
+  const float nv = block_sum(cnt, scratch);
+  for (int c = tid; c < H; c += nt) u[H + c] = nv > 0.f ? cand_sum[size_t(e) * H + c] / nv : 0.f;
   __syncthreads();
   const float v = mlp_scalar(u, 2 * H, Hm, vW1, vb1, vw2, vb2, scratch);
   if (tid == 0) value[e] = v;
@@ -324,6 +359,14 @@ int launch_global_update(const Dims& d, const float* partial, const int32_t* gra
   return 1;
 }
 
+int launch_global_update_blocks(const Dims& d, const float* partial, const int32_t* node_off, int32_t nblocks,
+                                const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st) {
+  if (B <= 0) return 0;
+  k_global_update_blocks<<<B, 256, sizeof(float) * size_t(d.H + d.Dg), st>>>(partial, node_off, nblocks, g0,
+                                                                             w.Wg, w.bg, emb, d.H, d.Dg);
+  return 1;
+}
+
 int launch_heads(const Dims& d, const DevWeights& w, const float* emb, const int32_t* env_off,
                  const uint8_t* mask, int32_t B, int32_t num_envs, float* logit_ws, float* probs,
                  float* value, int32_t* action, uint64_t seed, uint64_t step, int32_t* status,
@@ -331,13 +374,13 @@ int launch_heads(const Dims& d, const DevWeights& w, const float* emb, const int
   if (B <= 0 || num_envs <= 0) return 0;
   k_policy_logit<<<B, 256, sizeof(float) * size_t(d.H + 256), st>>>(emb, w.pW1, w.pb1, w.pw2, w.pb2,
                                                                     logit_ws, d.H, d.Hm);
+  float* cand_sum = logit_ws + B;                 // [num_envs x H], behind the per-graph logits
+  k_candidate_sum<<<dim3(num_envs, (d.H + 31) / 32), 1024, 0, st>>>(emb, env_off, mask, cand_sum, d.H, d.A);
   const int nt = pow2_threads(d.H > d.A + 1 ? d.H : d.A + 1);
-  const int parts = nt / d.H > 0 ? nt / d.H : 1;
-  const size_t smem = sizeof(unsigned long long) * size_t(nt + 1) +
-                      sizeof(float) * size_t(nt + 2 * d.H + parts * d.H);
-  k_env_policy<<<num_envs, nt, smem, st>>>(emb, logit_ws, env_off, mask, w.vW1, w.vb1, w.vw2, w.vb2,
-                                           probs, value, action, d.H, d.Hm, d.A, seed, step, status);
-  return 2;
+  const size_t smem = sizeof(unsigned long long) * size_t(nt + 1) + sizeof(float) * size_t(nt + 2 * d.H);
+  k_env_policy<<<num_envs, nt, smem, st>>>(emb, logit_ws, cand_sum, env_off, mask, w.vW1, w.vb1, w.vw2,
+                                           w.vb2, probs, value, action, d.H, d.Hm, d.A, seed, step, status);
+  return 3;
 }
 
 int launch_sample(const float* probs, int32_t num_envs, int32_t A1, uint64_t seed, uint64_t step,

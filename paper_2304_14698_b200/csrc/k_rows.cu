@@ -335,7 +335,7 @@ int launch_aggregate(const Dims& d, const int32_t* rowptr, const int32_t* col, c
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   if (rows <= 0) return 0;
   {   // 512-byte rows with 4 | K: gathers by the TMA engine
-    const int k = launch_aggregate_tma(d, rowptr, col, Z, scores, bias, h_out, win, buf_rows, status, st);
+    const int k = launch_aggregate_tma(d, rowptr, col, Z, scores, bias, h_out, win, buf_rows, nullptr, nullptr, status, st);
     if (k >= 0) return k;
   }
 #define CALL(TY_, LPR, VPL)                                                                        \

@@ -352,7 +352,10 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
 }
 
 // Eq. 6 and the first `layers` attention layers over the whole batch; features end up in ctx->h.
-int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t st) {
+// With fuse_readout the last of the `layers` attention layers may leave per-graph partial sums in
+// ctx->partial instead of node features in ctx->h; *fused tells whether it did.
+int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t st, bool fuse_readout = false,
+                    bool* fused = nullptr) {
   const Dims& d = ctx->dims;
   const Window win{0, b->N, 0};
   Profiler& pf = ctx->prof;
@@ -378,9 +381,18 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
     pf.end(FAM_XFORM, slot, k, st);
     n += k;
     slot = pf.begin(st);
-    k = launch_aggregate(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), ctx->Z.p,
-                         ctx->scores.as<float>(), ctx->dw.layer[l].b,
-                         ctx->h.p, win, b->N, ctx->status.as<int32_t>(), st);
+    k = -1;
+    if (fuse_readout && l == layers - 1) {
+      k = launch_aggregate_tma(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), ctx->Z.p,
+                               ctx->scores.as<float>(), ctx->dw.layer[l].b, ctx->h.p, win, b->N,
+                               b->seg_id.as<int32_t>(), ctx->partial.as<float>(),
+                               ctx->status.as<int32_t>(), st);
+      if (k >= 0 && fused) *fused = true;
+    }
+    if (k < 0)
+      k = launch_aggregate(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), ctx->Z.p,
+                           ctx->scores.as<float>(), ctx->dw.layer[l].b,
+                           ctx->h.p, win, b->N, ctx->status.as<int32_t>(), st);
     pf.end(FAM_AGG, slot, k, st);
     n += k;
   }
@@ -431,8 +443,12 @@ xrl_status xrl_create(const xrl_model_config* cfg, int32_t device, xrl_ctx** out
   A(ctx->h, sb * N * H);
   A(ctx->Z, sb * N * H);
   A(ctx->scores, 8 * N * size_t(cfg->heads));
-  A(ctx->partial, 4 * size_t(ctx->max_chunks) * H);
-  A(ctx->logits, 4 * size_t(cfg->max_graphs));
+  {
+    const size_t slots_fused = size_t(aggregate_readout_slots(cfg->max_nodes, cfg->max_graphs));
+    const size_t slots = slots_fused > size_t(ctx->max_chunks) ? slots_fused : size_t(ctx->max_chunks);
+    A(ctx->partial, 4 * slots * H);
+  }
+  A(ctx->logits, 4 * (size_t(cfg->max_graphs) + size_t(cfg->max_envs) * H));   // logits, then candidate sums
   A(ctx->status, 4);
   if (e == cudaSuccess) e = cudaMemset(ctx->status.p, 0, 4);
   if (e != cudaSuccess) {
@@ -562,15 +578,24 @@ xrl_status xrl_encode(xrl_ctx* ctx, const xrl_batch* b, const float* g0, float* 
   if (!graph_emb && b->B > 0) return XRL_ERR_INVALID_ARG;
   XRL_CUDA(cudaSetDevice(ctx->device));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  int n = run_node_layers(ctx, b, ctx->cfg.layers, st);
-  size_t slot = ctx->prof.begin(st);
-  int k = launch_readout(ctx->dims, ctx->h.p, b->d_chunk_row0, b->d_chunk_row1, 0, b->num_chunks,
-                         ctx->partial.as<float>(), 0, st);
-  ctx->prof.end(FAM_READOUT, slot, k, st);
-  n += k;
+  bool fused = false;
+  int n = run_node_layers(ctx, b, ctx->cfg.layers, st, true, &fused);
+  size_t slot;
+  int k;
+  if (!fused) {
+    slot = ctx->prof.begin(st);
+    k = launch_readout(ctx->dims, ctx->h.p, b->d_chunk_row0, b->d_chunk_row1, 0, b->num_chunks,
+                       ctx->partial.as<float>(), 0, st);
+    ctx->prof.end(FAM_READOUT, slot, k, st);
+    n += k;
+  }
   slot = ctx->prof.begin(st);
-  k = launch_global_update(ctx->dims, ctx->partial.as<float>(), b->d_graph_chunk_off, g0, ctx->dw,
-                           graph_emb, b->B, st);
+  if (fused)
+    k = launch_global_update_blocks(ctx->dims, ctx->partial.as<float>(), b->node_off.as<int32_t>(),
+                                    aggregate_readout_blocks(b->N), g0, ctx->dw, graph_emb, b->B, st);
+  else
+    k = launch_global_update(ctx->dims, ctx->partial.as<float>(), b->d_graph_chunk_off, g0, ctx->dw,
+                             graph_emb, b->B, st);
   ctx->prof.end(FAM_HEADS, slot, k, st);
   n += k;
   ctx->launches_encode = n;
