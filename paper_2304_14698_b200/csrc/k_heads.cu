@@ -10,6 +10,22 @@ namespace {
 
 constexpr int kRoThreads = 256;
 
+// sum_k x[k] * W[k * ld + c]: the weight loads are issued eight at a time so that their latencies
+// overlap; the additions keep the order k = 0, 1, 2, ...
+__device__ __forceinline__ float column_dot(const float* x, int in, const float* __restrict__ W, int ld,
+                                            int c, float acc) {
+  int k = 0;
+  for (; k + 8 <= in; k += 8) {
+    float w[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) w[t] = __ldg(W + size_t(k + t) * ld + c);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) acc = fmaf(x[k + t], w[t], acc);
+  }
+  for (; k < in; ++k) acc = fmaf(x[k], __ldg(W + size_t(k) * ld + c), acc);
+  return acc;
+}
+
 // ---- readout, stage 1: column sums of one chunk of consecutive rows of one graph -------------
 template <typename T>
 __global__ void __launch_bounds__(kRoThreads)
@@ -71,9 +87,7 @@ k_global_update(const float* __restrict__ partial, const int32_t* __restrict__ g
   for (int t = threadIdx.x; t < Dg; t += blockDim.x) u[H + t] = g0 ? g0[size_t(g) * Dg + t] : 0.f;
   __syncthreads();
   for (int c = threadIdx.x; c < H; c += blockDim.x) {
-    float acc = bg[c];
-    for (int k = 0; k < H + Dg; ++k) acc = fmaf(u[k], __ldg(Wg + size_t(k) * H + c), acc);
-    emb[size_t(g) * H + c] = fmaxf(acc, 0.f);
+    emb[size_t(g) * H + c] = fmaxf(column_dot(u, H + Dg, Wg, H, c, bg[c]), 0.f);
   }
 }
 
@@ -100,9 +114,7 @@ k_global_update_blocks(const float* __restrict__ partial, const int32_t* __restr
   for (int t = threadIdx.x; t < Dg; t += blockDim.x) u[H + t] = g0 ? g0[size_t(g) * Dg + t] : 0.f;
   __syncthreads();
   for (int c = threadIdx.x; c < H; c += blockDim.x) {
-    float acc = bg[c];
-    for (int k = 0; k < H + Dg; ++k) acc = fmaf(u[k], __ldg(Wg + size_t(k) * H + c), acc);
-    emb[size_t(g) * H + c] = fmaxf(acc, 0.f);
+    emb[size_t(g) * H + c] = fmaxf(column_dot(u, H + Dg, Wg, H, c, bg[c]), 0.f);
   }
 }
 
@@ -126,9 +138,7 @@ __device__ float mlp_scalar(const float* x, int in, int hid, const float* __rest
                             const float* __restrict__ b2, float* scratch) {
   float contrib = 0.f;
   for (int c = threadIdx.x; c < hid; c += blockDim.x) {
-    float acc = b1[c];
-    for (int k = 0; k < in; ++k) acc = fmaf(x[k], __ldg(W1 + size_t(k) * hid + c), acc);
-    contrib += fmaxf(acc, 0.f) * w2[c];
+    contrib += fmaxf(column_dot(x, in, W1, hid, c, b1[c]), 0.f) * w2[c];
   }
   return block_sum(contrib, scratch) + b2[0];
 }
@@ -190,13 +200,24 @@ __device__ int32_t sample_row(const float* __restrict__ p, int A1, uint64_t seed
                              U4{env, uint32_t(step), uint32_t(step >> 32), 0u});
   const unsigned long long r64 = (unsigned long long)r.x | ((unsigned long long)r.y << 32);
   const unsigned long long t = __umul64hi(r64, Q);
-  // exclusive prefix of the per-thread totals (serial over threads by thread 0: nt <= 1024)
-  scratch[tid] = mine;
-  __syncthreads();
-  if (tid == 0) {
-    unsigned long long run = 0;
-    for (int i = 0; i < nt; ++i) { const unsigned long long v = scratch[i]; scratch[i] = run; run += v; }
-    scratch[nt] = (unsigned long long)(A1 - 1);
+  // exclusive prefix of the per-thread totals: scan inside each warp, then over the warp totals
+  // (integer sums: any association gives the same result)
+  {
+    const int lane = tid & 31, wid = tid >> 5, nw = nt >> 5;
+    unsigned long long incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    __syncthreads();                            // scratch is free again after block_sum_u64
+    if (lane == 31) scratch[wid] = incl;
+    __syncthreads();
+    unsigned long long wbase = 0;
+    for (int w = 0; w < wid && w < nw; ++w) wbase += scratch[w];
+    __syncthreads();
+    scratch[tid] = wbase + incl - mine;
+    if (tid == 0) scratch[nt] = (unsigned long long)(A1 - 1);
   }
   __syncthreads();
   unsigned long long run = scratch[tid];
