@@ -21,17 +21,16 @@ namespace {
 
 constexpr int TW = 4;            // warps per CTA
 #ifndef XRL_AGG_GROUPS
-#define XRL_AGG_GROUPS 2
+#define XRL_AGG_GROUPS 4
 #endif
 #ifndef XRL_AGG_CTAS
-#define XRL_AGG_CTAS 4
+#define XRL_AGG_CTAS 5
 #endif
-constexpr int G = XRL_AGG_GROUPS;   // gather groups (of four rows) in flight per half-warp
-constexpr int BR = 16;           // destination rows per half-warp block
-constexpr int ITEMS = 96;        // list capacity per half-warp, a multiple of 4
+constexpr int G = XRL_AGG_GROUPS;   // gather groups (of four rows) in flight per warp
+constexpr int BR = 32;           // destination rows per block
+constexpr int ITEMS = 160;       // list capacity, a multiple of 4
 
-// One per half-warp: the two halves of a warp work on different row blocks with rings of their own.
-template <int K> struct alignas(128) HalfSmem {
+template <int K> struct alignas(128) WarpSmem {
   uint4 z[G][4][32];             // four gathered rows of 512 bytes per group
   float2 sc[G][4][K];            // their {s_src, s_dst} pairs
   unsigned long long bar[G];
@@ -102,6 +101,31 @@ __device__ __forceinline__ void to_pairs(const uint4& raw, F2 (&z)[2]) {        
   z[1] = make_f2(__uint_as_float(raw.z), __uint_as_float(raw.w));
 }
 
+// out = ReLU(acc * inv + bias), stored in the feature type
+__device__ __forceinline__ void finish_row(bf16* dst, const F2 (&acc)[4], float inv, const float (&bs)[8]) {
+  uint32_t w[4];
+#pragma unroll
+  for (int t = 0; t < 4; ++t) {
+    float lo, hi;
+    split_f2(acc[t], lo, hi);
+    lo = fmaf(lo, inv, bs[2 * t]);
+    hi = fmaf(hi, inv, bs[2 * t + 1]);
+    asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(w[t]) : "f"(hi), "f"(lo));   // ReLU inside the rounding
+  }
+  *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+}
+__device__ __forceinline__ void finish_row(float* dst, const F2 (&acc)[2], float inv, const float (&bs)[4]) {
+  float o[4];
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    float lo, hi;
+    split_f2(acc[t], lo, hi);
+    o[2 * t] = fmaxf(fmaf(lo, inv, bs[2 * t]), 0.f);
+    o[2 * t + 1] = fmaxf(fmaf(hi, inv, bs[2 * t + 1]), 0.f);
+  }
+  *reinterpret_cast<float4*>(dst) = make_float4(o[0], o[1], o[2], o[3]);
+}
+
 // out = ReLU(acc * inv + bias) kept in fp32 (for the fused per-graph readout)
 template <int NP>
 __device__ __forceinline__ void finish_row_f32(const F2 (&acc)[NP], float inv, const float (&bs)[2 * NP],
@@ -113,41 +137,6 @@ __device__ __forceinline__ void finish_row_f32(const F2 (&acc)[NP], float inv, c
     o[2 * t] = fmaxf(fmaf(lo, inv, bs[2 * t]), 0.f);
     o[2 * t + 1] = fmaxf(fmaf(hi, inv, bs[2 * t + 1]), 0.f);
   }
-}
-
-// 32 bytes per lane = two 16-byte vectors
-template <int NP>
-__device__ __forceinline__ void to_pairs2(const uint4& a, const uint4& b, F2 (&z)[2 * NP]) {
-  F2 lo[NP], hi[NP];
-  to_pairs(a, lo);
-  to_pairs(b, hi);
-#pragma unroll
-  for (int t = 0; t < NP; ++t) { z[t] = lo[t]; z[NP + t] = hi[t]; }
-}
-template <typename T, int NP2>
-__device__ __forceinline__ void load_pairs2(const T* p, F2 (&z)[NP2]) {
-  const uint4 a = __ldg(reinterpret_cast<const uint4*>(p));
-  const uint4 b = __ldg(reinterpret_cast<const uint4*>(p) + 1);
-  to_pairs2<NP2 / 2>(a, b, z);
-}
-__device__ __forceinline__ void finish_row2(bf16* dst, const F2 (&acc)[8], float inv, const float (&bs)[16]) {
-  uint32_t w[8];
-#pragma unroll
-  for (int t = 0; t < 8; ++t) {
-    float lo, hi;
-    split_f2(acc[t], lo, hi);
-    lo = fmaf(lo, inv, bs[2 * t]);
-    hi = fmaf(hi, inv, bs[2 * t + 1]);
-    asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(w[t]) : "f"(hi), "f"(lo));   // ReLU inside the rounding
-  }
-  reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
-  reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
-}
-__device__ __forceinline__ void finish_row2(float* dst, const F2 (&acc)[4], float inv, const float (&bs)[8]) {
-  float o[8];
-  finish_row_f32<4>(acc, inv, bs, o);
-  reinterpret_cast<float4*>(dst)[0] = make_float4(o[0], o[1], o[2], o[3]);
-  reinterpret_cast<float4*>(dst)[1] = make_float4(o[4], o[5], o[6], o[7]);
 }
 
 // Rare path of the running softmax: the reference exponent is moved up only when a score exceeds
@@ -165,15 +154,11 @@ __device__ __forceinline__ void raise_reference(float ev, float& m, float& l, F2
 }
 
 // READOUT = true is the last attention layer fused with the per-graph sum of Eq. 8: the layer output
-// is not stored; each half-warp adds the rows of its 16-row block per graph, in row order, and writes
+// is not stored; each warp adds the rows of its 32-row block per graph, in row order, and writes
 //   partial[b]           the rows of block b that belong to the graph of the block's first row
 //   partial[nblocks + g] the rows of graph g inside the block in which g starts, when that is not at
 //                        the block's first row
 // (k_global_update_blocks adds them per graph in a fixed order).  Needs row_begin = win_base = 0.
-//
-// Work split: a destination row is owned by 16 lanes, 32 bytes (16 bf16 / 8 fp32, inside one head)
-// per lane; the two half-warps of a warp run the same code on different 16-row blocks, so the
-// per-vector bookkeeping (loop control, ring pointers, score arithmetic) is paid once per two rows.
 template <typename T, int K, bool READOUT>
 __global__ void __launch_bounds__(TW * 32, XRL_AGG_CTAS)
 k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant__ CUtensorMap map_s,
@@ -182,41 +167,39 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
                 const float* __restrict__ bias, T* __restrict__ h_out, Window win,
                 const int32_t* __restrict__ seg_id, float* __restrict__ partial, int32_t nblocks,
                 int32_t* status) {
-  constexpr int VEC = VecOf<T>::N;          // elements per 16 bytes
-  constexpr int NP = VEC / 2;               // register pairs per 16 bytes
-  constexpr int LV = 2 * VEC;               // elements per lane (32 bytes)
+  constexpr int VEC = VecOf<T>::N;
+  constexpr int NP = VEC / 2;
   constexpr int H = 32 * VEC;
   constexpr uint32_t GROUP_BYTES = 4 * 512 + 4 * K * 8;
   constexpr uint32_t ZG = 2048, SG = 32 * K;          // bytes per group in the two rings
   extern __shared__ __align__(128) uint8_t tma_smem_raw[];
-  const int lane = threadIdx.x & 31, half = lane >> 4, hl = lane & 15;
-  const uint32_t hmask = 0xFFFFu << (16 * half);
-  HalfSmem<K>& sm = reinterpret_cast<HalfSmem<K>*>(tma_smem_raw)[(threadIdx.x >> 5) * 2 + half];
-  const int64_t halves_total = int64_t(gridDim.x) * (blockDim.x >> 4);
-  const int64_t half_id = (int64_t(blockIdx.x) * blockDim.x + threadIdx.x) >> 4;
-  const int c0 = hl * LV;
+  WarpSmem<K>& sm = reinterpret_cast<WarpSmem<K>*>(tma_smem_raw)[threadIdx.x >> 5];
+  const int lane = threadIdx.x & 31;
+  const int warps_total = (gridDim.x * blockDim.x) >> 5;
+  const int warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int c0 = lane * VEC;
   const int head = c0 / (H / K);
-  float bs[LV];
+  float bs[VEC];
 #pragma unroll
-  for (int t = 0; t < LV; ++t) bs[t] = __ldg(bias + c0 + t);
-  const uint32_t z_lane = smem_u32(&sm.z[0][0][2 * hl]);     // this lane's 32 bytes of slot 0, row 0
+  for (int t = 0; t < VEC; ++t) bs[t] = __ldg(bias + c0 + t);
+  const uint32_t z_lane = smem_u32(&sm.z[0][0][lane]);       // this lane's 16 bytes of slot 0, row 0
   const uint32_t s_lane = smem_u32(&sm.sc[0][0][head]);      // this lane's head in slot 0, row 0
   const uint32_t z_base = smem_u32(&sm.z[0][0][0]);
   const uint32_t s_base = smem_u32(&sm.sc[0][0][0]);
   const uint32_t bar_base = smem_u32(&sm.bar[0]);
 
-  if (hl == 0) {
+  if (lane == 0) {
     for (int g = 0; g < G; ++g) mbar_init(bar_base + 8 * g, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
   __syncwarp();
 
-  // ring state of this half-warp, carried across lists
+  // ring state, carried across lists: slot and phase parity of the next group to consume
   uint32_t slot = 0, par = 0;
   bool alive = true;
 
-  // leader of the half-warp: hand group `gi` of the current list to slot `s`
+  // lane 0: hand group `gi` of the current list (list rows item[4 gi .. 4 gi + 3]) to slot `s`
   auto issue = [&](int gi, uint32_t s) {
     const int4 it = *reinterpret_cast<const int4*>(&sm.item[gi * 4]);
     const uint32_t bar = bar_base + 8 * s;
@@ -225,64 +208,49 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
     tma_gather4(s_base + s * SG, &map_s, it.x, it.y, it.z, it.w, bar);
   };
 
-  // both halves run the same number of outer iterations (a half without rows idles through them)
-  const int64_t nblk = (int64_t(win.row_end) - win.row_begin + BR - 1) / BR;
-  const int64_t iters = (nblk + halves_total - 1) / halves_total;
-  for (int64_t itn = 0; itn < iters; ++itn) {
-    const int64_t blk = itn * halves_total + half_id;
-    const int64_t r0 = int64_t(win.row_begin) + blk * BR;
-    const int nr = (blk < nblk && alive) ? int(min(int64_t(BR), win.row_end - r0)) : 0;
-    __syncwarp(hmask);
-    if (hl < nr) sm.rp[hl] = __ldg(rowptr + r0 + hl);
-    if (hl == 0 && nr > 0) sm.rp[nr] = __ldg(rowptr + r0 + nr);
-    __syncwarp(hmask);
+  for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * BR; r0 < win.row_end && alive;
+       r0 += int64_t(warps_total) * BR) {
+    const int nr = int(min(int64_t(BR), win.row_end - r0));
+    __syncwarp();
+    if (lane < nr) sm.rp[lane] = __ldg(rowptr + r0 + lane);
+    if (lane == 0) sm.rp[nr] = __ldg(rowptr + r0 + nr);
+    __syncwarp();
     // fused readout: running per-graph sum of this block's rows
     int32_t myseg = 0, cur_g = -1;
     bool first_seg = true;
-    float rsum[LV];
+    float rsum[VEC];
     if (READOUT) {
-      myseg = (hl < nr) ? __ldg(seg_id + r0 + hl) : 0;
+      myseg = (lane < nr) ? __ldg(seg_id + r0 + lane) : 0;
 #pragma unroll
-      for (int t = 0; t < LV; ++t) rsum[t] = 0.f;
+      for (int t = 0; t < VEC; ++t) rsum[t] = 0.f;
     }
     auto flush = [&]() {
-      float* dst = partial + size_t(first_seg ? int32_t(blk) : nblocks + cur_g) * H + c0;
+      float* dst = partial + size_t(first_seg ? int32_t(r0 / BR) : nblocks + cur_g) * H + c0;
 #pragma unroll
-      for (int t = 0; t < LV; t += 4)
+      for (int t = 0; t < VEC; t += 4)
         *reinterpret_cast<float4*>(dst + t) = make_float4(rsum[t], rsum[t + 1], rsum[t + 2], rsum[t + 3]);
     };
-    auto add_row = [&](int row_in_block, const float (&o)[LV]) {
-      const int32_t g = __shfl_sync(hmask, myseg, row_in_block, 16);
+    auto add_row = [&](int row_in_block, const float (&o)[VEC]) {
+      const int32_t g = __shfl_sync(0xFFFFFFFFu, myseg, row_in_block);
       if (g != cur_g) {
         if (cur_g >= 0) {
           flush();
           first_seg = false;
 #pragma unroll
-          for (int t = 0; t < LV; ++t) rsum[t] = 0.f;
+          for (int t = 0; t < VEC; ++t) rsum[t] = 0.f;
         }
         cur_g = g;
       }
 #pragma unroll
-      for (int t = 0; t < LV; ++t) rsum[t] += o[t];
+      for (int t = 0; t < VEC; ++t) rsum[t] += o[t];
     };
-    auto finish = [&](int row_in_block, const F2 (&acc)[2 * NP], float inv) {
-      if (READOUT) {
-        float o[LV];
-        finish_row_f32<2 * NP>(acc, inv, bs, o);
-        add_row(row_in_block, o);
-      } else {
-        T* dst = h_out + size_t(int32_t(r0) + row_in_block - win.win_base) * H + c0;
-        finish_row2(dst, acc, inv, bs);
-      }
-    };
-
     int rs = 0;
-    while (rs < nr) {
+    while (rs < nr && alive) {
       // as many rows from rs on as keep (rows + producers) within the list
       const int32_t eb = sm.rp[rs];
-      const bool fits = (rs + hl < nr) && (hl + 1 + sm.rp[rs + hl + 1] - eb <= ITEMS);
-      const uint32_t fmask = (__ballot_sync(hmask, fits) >> (16 * half)) & 0xFFFFu;
-      const int cnt = (fmask == 0xFFFFu) ? 16 : __ffs(~fmask) - 1;
+      const bool fits = (rs + lane < nr) && (lane + 1 + sm.rp[rs + lane + 1] - eb <= ITEMS);
+      const uint32_t fmask = __ballot_sync(0xFFFFFFFFu, fits);
+      const int cnt = (fmask == 0xFFFFFFFFu) ? 32 : __ffs(~fmask) - 1;
       if (cnt == 0) {
         // a row with more producers than the list holds: plain loads, one producer at a time
         const int32_t lrow = int32_t(r0) + rs - win.win_base;
@@ -290,37 +258,43 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
         const float2 self = __ldg(scores + size_t(lrow) * K + head);
         const float sd = self.y;
         float m = lrelu(self.x + sd), l = 1.f;
-        F2 acc[2 * NP];
-        load_pairs2(Z + size_t(lrow) * H + c0, acc);
+        F2 acc[NP];
+        to_pairs(__ldg(reinterpret_cast<const uint4*>(Z + size_t(lrow) * H + c0)), acc);
         for (int t = 0; t < n; ++t) {
           const int32_t j = __ldg(col + eb + t) - win.win_base;
           const float ev = lrelu(__ldg(&scores[size_t(j) * K + head].x) + sd);
-          F2 z[2 * NP];
-          load_pairs2(Z + size_t(j) * H + c0, z);
-          if (ev > m + 32.f) raise_reference<2 * NP>(ev, m, l, acc);
+          F2 z[NP];
+          to_pairs(__ldg(reinterpret_cast<const uint4*>(Z + size_t(j) * H + c0)), z);
+          if (ev > m + 32.f) raise_reference<NP>(ev, m, l, acc);
           const float p = fast_exp2(ev - m);
           l += p;
           const F2 p2 = make_f2(p, p);
 #pragma unroll
-          for (int t2 = 0; t2 < 2 * NP; ++t2) fma2(acc[t2], p2, z[t2]);
+          for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], p2, z[t2]);
         }
-        finish(rs, acc, __fdividef(1.f, l));
+        if (READOUT) {
+          float o[VEC];
+          finish_row_f32<NP>(acc, __fdividef(1.f, l), bs, o);
+          add_row(rs, o);
+        } else {
+          finish_row(h_out + size_t(lrow) * H + c0, acc, __fdividef(1.f, l), bs);
+        }
         rs += 1;
         continue;
       }
       // ---- the list: for each row its own index, then its producers', all window-relative ----------
-      __syncwarp(hmask);
+      __syncwarp();
       const int total = cnt + (sm.rp[rs + cnt] - eb);
-      if (hl < cnt) {
-        const int e0 = sm.rp[rs + hl] - eb, n = sm.rp[rs + hl + 1] - eb - e0;
-        int pos = hl + e0;
-        sm.item[pos++] = int32_t(r0) + rs + hl - win.win_base;
+      if (lane < cnt) {
+        const int e0 = sm.rp[rs + lane] - eb, n = sm.rp[rs + lane + 1] - eb - e0;
+        int pos = lane + e0;
+        sm.item[pos++] = int32_t(r0) + rs + lane - win.win_base;
         for (int t = 0; t < n; ++t) sm.item[pos++] = __ldg(col + eb + e0 + t) - win.win_base;
       }
-      if (hl < 4) sm.item[total + hl] = int32_t(r0) + rs - win.win_base;   // pad the last group
-      __syncwarp(hmask);
+      if (lane < 4) sm.item[total + lane] = int32_t(r0) + rs - win.win_base;   // pad the last group
+      __syncwarp();
       const int ngroups = (total + 3) >> 2;
-      if (hl == 0) {
+      if (lane == 0) {
         uint32_t s = slot;
         for (int gi = 0; gi < min(G, ngroups); ++gi) { issue(gi, s); s = (s + 1 == G) ? 0 : s + 1; }
       }
@@ -331,8 +305,8 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
       if (!wait_all_lanes(bar_base + 8 * slot, par)) alive = false;
       // group finished: refill its slot with group gi + G, move on, wait for the next one
       auto advance = [&]() {
-        __syncwarp(hmask);
-        if (hl == 0 && gi + G < ngroups) issue(gi + G, slot);
+        __syncwarp();
+        if (lane == 0 && gi + G < ngroups) issue(gi + G, slot);
         ++gi;
         if (++slot == G) { slot = 0; par ^= 1; }
         zp = z_lane + slot * ZG;
@@ -343,33 +317,39 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
       for (int rr = 0; rr < cnt; ++rr) {
         const int n = sm.rp[rs + rr + 1] - sm.rp[rs + rr];
         // the row's own vector opens the running softmax: reference exponent = its score, weight 1
-        uint4 ra = lds128(zp), rb = lds128(zp + 16);
+        uint4 raw = lds128(zp);
         float2 sc = lds64(sp);
         zp += 512; sp += 8 * K;
         if (--w == 0) advance();
         const float sd = sc.y;
         float m = lrelu(sc.x + sd), l = 1.f;
-        F2 acc[2 * NP];
-        to_pairs2<NP>(ra, rb, acc);
+        F2 acc[NP];
+        to_pairs(raw, acc);
         for (int t = 0; t < n; ++t) {
-          ra = lds128(zp); rb = lds128(zp + 16);
+          raw = lds128(zp);
           sc = lds64(sp);
           zp += 512; sp += 8 * K;
           if (--w == 0) advance();
           const float ev = lrelu(sc.x + sd);
-          if (ev > m + 32.f) raise_reference<2 * NP>(ev, m, l, acc);
+          if (ev > m + 32.f) raise_reference<NP>(ev, m, l, acc);
           const float p = fast_exp2(ev - m);
           l += p;
-          F2 z[2 * NP];
-          to_pairs2<NP>(ra, rb, z);
+          F2 z[NP];
+          to_pairs(raw, z);
           const F2 p2 = make_f2(p, p);
 #pragma unroll
-          for (int t2 = 0; t2 < 2 * NP; ++t2) fma2(acc[t2], p2, z[t2]);
+          for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], p2, z[t2]);
         }
-        finish(rs + rr, acc, __fdividef(1.f, l));
+        if (READOUT) {
+          float o[VEC];
+          finish_row_f32<NP>(acc, __fdividef(1.f, l), bs, o);
+          add_row(rs + rr, o);
+        } else {
+          finish_row(h_out + size_t(int32_t(r0) + rs + rr - win.win_base) * H + c0, acc, __fdividef(1.f, l), bs);
+        }
       }
       if (w != 4) {                            // the list ended inside a group: retire it without waiting
-        __syncwarp(hmask);
+        __syncwarp();
         if (++slot == G) { slot = 0; par ^= 1; }
       }
       rs += cnt;
@@ -377,7 +357,7 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
     if (READOUT && cur_g >= 0) flush();
   }
   if (!alive) {
-    if (hl == 0) raise(status, XRL_ERR_TIMEOUT);
+    if (lane == 0) raise(status, XRL_ERR_TIMEOUT);
     for (int t = 0; t < 100; ++t) __nanosleep(10000);     // give copies still in flight time to land
   }
 }
@@ -400,7 +380,7 @@ int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const flo
              void* h_out, Window win, int64_t buf_rows, const int32_t* seg_id, float* partial,
              int32_t* status, cudaStream_t st) {
   static bool attr = false;
-  const size_t smem = sizeof(HalfSmem<K>) * TW * 2;
+  const size_t smem = sizeof(WarpSmem<K>) * TW;
   if (!attr) {
     if (cudaFuncSetAttribute(k_aggregate_tma<T, K, READOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              int(smem)) != cudaSuccess) {
@@ -417,7 +397,7 @@ int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const flo
     return -1;
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   const int64_t nblocks = (rows + BR - 1) / BR;
-  int64_t nb = (rows + BR * TW * 2 - 1) / (BR * TW * 2);
+  int64_t nb = (rows + BR * TW - 1) / (BR * TW);
   if (nb > int64_t(kNumSMs) * XRL_AGG_CTAS) nb = int64_t(kNumSMs) * XRL_AGG_CTAS;
   k_aggregate_tma<T, K, READOUT><<<int(nb), TW * 32, smem, st>>>(
       mz, ms, rowptr, col, static_cast<const T*>(Z), reinterpret_cast<const float2*>(scores), bias,
@@ -458,6 +438,5 @@ int launch_aggregate_tma(const Dims& d, const int32_t* rowptr, const int32_t* co
 // Partial-sum slots the fused variant writes for `rows` rows and B graphs.
 int64_t aggregate_readout_slots(int64_t rows, int64_t B) { return (rows + BR - 1) / BR + B; }
 int32_t aggregate_readout_blocks(int64_t rows) { return int32_t((rows + BR - 1) / BR); }
-int aggregate_readout_shift() { static_assert(BR == 16, "block rows"); return 4; }
 
 }  // namespace xrl

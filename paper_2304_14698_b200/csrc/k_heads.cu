@@ -93,10 +93,10 @@ k_global_update(const float* __restrict__ partial, const int32_t* __restrict__ g
 
 // Eq. 8 from the partial sums written by the aggregate kernel fused with the readout: per graph, the
 // partial of the block in which the graph starts (if it does not start at the block's first row), then
-// the partials of the following 2^shift-row blocks whose first row belongs to the graph, in order.
+// the partials of the following 32-row blocks whose first row belongs to the graph, in order.
 __global__ void __launch_bounds__(256)
 k_global_update_blocks(const float* __restrict__ partial, const int32_t* __restrict__ node_off,
-                       int32_t nblocks, int shift, const float* __restrict__ g0, const float* __restrict__ Wg,
+                       int32_t nblocks, const float* __restrict__ g0, const float* __restrict__ Wg,
                        const float* __restrict__ bg, float* __restrict__ emb, int H, int Dg) {
   extern __shared__ float u[];                   // [H + Dg]
   const int32_t g = blockIdx.x;
@@ -104,9 +104,9 @@ k_global_update_blocks(const float* __restrict__ partial, const int32_t* __restr
   for (int c = threadIdx.x; c < H; c += blockDim.x) {
     float s = 0.f;
     if (end > start) {
-      int32_t b0 = start >> shift;
-      if (start & ((1 << shift) - 1)) { s += partial[size_t(nblocks + g) * H + c]; ++b0; }
-      const int32_t b1 = (end - 1) >> shift;
+      int32_t b0 = start >> 5;
+      if (start & 31) { s += partial[size_t(nblocks + g) * H + c]; ++b0; }
+      const int32_t b1 = (end - 1) >> 5;
       for (int32_t b = b0; b <= b1; ++b) s += partial[size_t(b) * H + c];
     }
     u[c] = s;
@@ -381,9 +381,9 @@ int launch_global_update(const Dims& d, const float* partial, const int32_t* gra
 }
 
 int launch_global_update_blocks(const Dims& d, const float* partial, const int32_t* node_off, int32_t nblocks,
-                                int shift, const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st) {
+                                const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st) {
   if (B <= 0) return 0;
-  k_global_update_blocks<<<B, 256, sizeof(float) * size_t(d.H + d.Dg), st>>>(partial, node_off, nblocks, shift, g0,
+  k_global_update_blocks<<<B, 256, sizeof(float) * size_t(d.H + d.Dg), st>>>(partial, node_off, nblocks, g0,
                                                                              w.Wg, w.bg, emb, d.H, d.Dg);
   return 1;
 }

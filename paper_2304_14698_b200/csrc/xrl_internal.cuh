@@ -121,9 +121,8 @@ int launch_aggregate_tma(const Dims& d, const int32_t* rowptr, const int32_t* co
                          const int32_t* seg_id, float* partial, int32_t* status, cudaStream_t st);
 int64_t aggregate_readout_slots(int64_t rows, int64_t B);
 int32_t aggregate_readout_blocks(int64_t rows);
-int aggregate_readout_shift();
 int launch_global_update_blocks(const Dims& d, const float* partial, const int32_t* node_off, int32_t nblocks,
-                                int shift, const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st);
+                                const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st);
 int launch_readout(const Dims& d, const void* h, const int32_t* chunk_row0, const int32_t* chunk_row1,
                    int32_t chunk_begin, int32_t chunk_end, float* partial, int32_t win_base,
                    cudaStream_t st);
