@@ -203,8 +203,9 @@ xrl_status xrl_launch_counts(const xrl_ctx* ctx, int64_t* pack, int64_t* encode,
  * allocations from callbacks.  xrl_create / xrl_pack allocate (context workspace, batch, pinned
  * staging), so those programs cannot use them.  This call builds the same packed index arrays
  * with NO allocation of any kind: no context, no batch object, and the packer's scratch (in-degree
- * counters, row cursors, the unsorted edge slots, scan partial sums, a device copy of the counts)
- * sits in a fixed array inside the library image, about 2.7 MB that every GPU loading the library
+ * counters, row cursors, the unsorted (edge id, producer) slots, scan partial sums, a device copy of
+ * the counts)
+ * sits in a fixed array inside the library image, about 4.8 MB that every GPU loading the library
  * keeps until the process exits.  The price is a size limit:
  *     num_graphs <= XRL_STATIC_PACK_MAX_GRAPHS, num_envs <= XRL_STATIC_PACK_MAX_ENVS,
  *     total nodes <= XRL_STATIC_PACK_MAX_NODES, total edges <= XRL_STATIC_PACK_MAX_EDGES;

@@ -94,6 +94,21 @@ __device__ __forceinline__ int32_t upper_segment(const int32_t* __restrict__ off
   return lo;
 }
 
+// Graph of every 1024-th edge: lets the per-edge kernels find their graph with a short forward walk
+// instead of a binary search.
+constexpr int kCoarseShift = 10;
+__global__ void k_edge_coarse(const int32_t* __restrict__ edge_off, int32_t B, int32_t E,
+                              int32_t* __restrict__ coarse) {
+  const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  if ((int64_t(i) << kCoarseShift) < E) coarse[i] = upper_segment(edge_off, B, i << kCoarseShift);
+}
+__device__ __forceinline__ int32_t graph_of_edge(const int32_t* __restrict__ edge_off,
+                                                 const int32_t* __restrict__ coarse, int32_t B, int32_t e) {
+  int32_t g = __ldg(coarse + (e >> kCoarseShift));
+  while (g + 1 < B && __ldg(edge_off + g + 1) <= e) ++g;      // skips empty graphs as well
+  return g;
+}
+
 __global__ void k_node_segments(const int32_t* __restrict__ node_off, int32_t B, int32_t N,
                                 const int32_t* __restrict__ op, int32_t T,
                                 int32_t* __restrict__ seg_id, int32_t* __restrict__ deg,
@@ -115,72 +130,72 @@ __global__ void k_graph_envs(const int32_t* __restrict__ env_off, int32_t num_en
 // One thread per edge: validate, count the consumer's in-degree.
 __global__ void k_edge_count(const int32_t* __restrict__ edge_src, const int32_t* __restrict__ edge_dst,
                              const int32_t* __restrict__ edge_off, const int32_t* __restrict__ node_off,
-                             int32_t B, int32_t E, int32_t* __restrict__ deg, int32_t* status) {
+                             const int32_t* __restrict__ coarse, int32_t B, int32_t E,
+                             int32_t* __restrict__ deg, int32_t* status) {
   const int32_t e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= E) return;
-  const int32_t g = upper_segment(edge_off, B, e);
+  const int32_t g = graph_of_edge(edge_off, coarse, B, e);
   const int32_t n = node_off[g + 1] - node_off[g];
   const int32_t s = edge_src[e], t = edge_dst[e];
   if (s < 0 || s >= n || t < 0 || t >= n || s == t) { raise(status, XRL_ERR_BAD_GRAPH); return; }
   atomicAdd(&deg[node_off[g] + t], 1);
 }
 
-// One thread per edge: drop the edge id into some slot of its consumer's row (order fixed later).
+// One thread per edge: drop (edge id, global producer id) into some slot of its consumer's row
+// (the order inside the row is fixed later from the edge ids).
 __global__ void k_edge_scatter(const int32_t* __restrict__ edge_src, const int32_t* __restrict__ edge_dst,
                                const int32_t* __restrict__ edge_off, const int32_t* __restrict__ node_off,
-                               const int32_t* __restrict__ rowptr, int32_t B, int32_t E,
-                               int32_t* __restrict__ cursor, int32_t* __restrict__ tmp_eid) {
+                               const int32_t* __restrict__ coarse, const int32_t* __restrict__ rowptr,
+                               int32_t B, int32_t E, int32_t* __restrict__ cursor,
+                               int2* __restrict__ tmp) {
   const int32_t e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= E) return;
-  const int32_t g = upper_segment(edge_off, B, e);
+  const int32_t g = graph_of_edge(edge_off, coarse, B, e);
   const int32_t n = node_off[g + 1] - node_off[g];
   const int32_t s = edge_src[e], t = edge_dst[e];
   if (s < 0 || s >= n || t < 0 || t >= n || s == t) return;
   const int32_t row = node_off[g] + t;
   const int32_t slot = atomicAdd(&cursor[row], 1);
-  tmp_eid[rowptr[row] + slot] = e;
+  tmp[rowptr[row] + slot] = make_int2(e, node_off[g] + s);
 }
 
 constexpr int kShortRow = 32;
 
-// One thread per row: place each edge at its rank among the row's edge ids, which restores
-// the input order whatever order the atomics handed the slots out in.
-__global__ void k_row_order(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ tmp_eid,
-                            const int32_t* __restrict__ edge_src, const int32_t* __restrict__ seg_id,
-                            const int32_t* __restrict__ node_off, int32_t N, int32_t* __restrict__ col,
-                            int32_t* __restrict__ long_rows, int32_t* __restrict__ long_count) {
+// One thread per row: place each producer at the rank of its edge id among the row's edge ids, which
+// restores the input order whatever order the atomics handed the slots out in.
+__global__ void k_row_order(const int32_t* __restrict__ rowptr, const int2* __restrict__ tmp, int32_t N,
+                            int32_t* __restrict__ col, int32_t* __restrict__ long_rows,
+                            int32_t* __restrict__ long_count) {
   const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= N) return;
   const int32_t b = rowptr[i], n = rowptr[i + 1] - b;
   if (n == 0) return;
+  if (n == 1) { col[b] = tmp[b].y; return; }
   if (n > kShortRow) { long_rows[atomicAdd(long_count, 1)] = i; return; }
-  const int32_t base = node_off[seg_id[i]];
   for (int32_t a = 0; a < n; ++a) {
-    const int32_t ea = tmp_eid[b + a];
+    const int2 ea = tmp[b + a];
     int32_t rank = 0;
-    for (int32_t c = 0; c < n; ++c) rank += (tmp_eid[b + c] < ea) ? 1 : 0;
-    col[b + rank] = base + edge_src[ea];
+    for (int32_t c = 0; c < n; ++c) rank += (tmp[b + c].x < ea.x) ? 1 : 0;
+    col[b + rank] = ea.y;
   }
 }
 
 // Rows longer than kShortRow: one warp per row, the same rank computation spread over lanes.
 __global__ void __launch_bounds__(256)
-k_row_order_long(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ tmp_eid,
-                 const int32_t* __restrict__ edge_src, const int32_t* __restrict__ seg_id,
-                 const int32_t* __restrict__ node_off, int32_t* __restrict__ col,
-                 const int32_t* __restrict__ long_rows, const int32_t* __restrict__ long_count) {
+k_row_order_long(const int32_t* __restrict__ rowptr, const int2* __restrict__ tmp,
+                 int32_t* __restrict__ col, const int32_t* __restrict__ long_rows,
+                 const int32_t* __restrict__ long_count) {
   const int lane = threadIdx.x & 31;
   const int32_t warps = (gridDim.x * blockDim.x) >> 5;
   const int32_t count = *long_count;
   for (int32_t w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < count; w += warps) {
     const int32_t i = long_rows[w];
     const int32_t b = rowptr[i], n = rowptr[i + 1] - b;
-    const int32_t base = node_off[seg_id[i]];
     for (int32_t a = lane; a < n; a += 32) {
-      const int32_t ea = tmp_eid[b + a];
+      const int2 ea = tmp[b + a];
       int32_t rank = 0;
-      for (int32_t c = 0; c < n; ++c) rank += (tmp_eid[b + c] < ea) ? 1 : 0;
-      col[b + rank] = base + edge_src[ea];
+      for (int32_t c = 0; c < n; ++c) rank += (tmp[b + c].x < ea.x) ? 1 : 0;
+      col[b + rank] = ea.y;
     }
   }
 }
@@ -214,22 +229,23 @@ int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cu
     ++launches;
   }
   if (in.E > 0) {
+    const int nc = (in.E >> kCoarseShift) + 1;
+    k_edge_coarse<<<(nc + TB - 1) / TB, TB, 0, st>>>(out.edge_off, in.B, in.E, out.coarse);
     k_edge_count<<<(in.E + TB - 1) / TB, TB, 0, st>>>(in.edge_src, in.edge_dst, out.edge_off,
-                                                       out.node_off, in.B, in.E, out.deg, status);
-    ++launches;
+                                                       out.node_off, out.coarse, in.B, in.E, out.deg, status);
+    launches += 2;
   }
   launches += exclusive_scan(out.deg, out.rowptr, in.N, out.scan_ws, st);
   if (in.E > 0 && in.N > 0) {
     cudaMemsetAsync(out.deg, 0, sizeof(int32_t) * size_t(in.N), st);      // reused as the row cursors
     cudaMemsetAsync(out.long_count, 0, sizeof(int32_t), st);
+    int2* tmp = reinterpret_cast<int2*>(out.tmp_eid);
     k_edge_scatter<<<(in.E + TB - 1) / TB, TB, 0, st>>>(in.edge_src, in.edge_dst, out.edge_off,
-                                                         out.node_off, out.rowptr, in.B, in.E,
-                                                         out.deg, out.tmp_eid);
-    k_row_order<<<(in.N + TB - 1) / TB, TB, 0, st>>>(out.rowptr, out.tmp_eid, in.edge_src, out.seg_id,
-                                                      out.node_off, in.N, out.col, out.long_rows,
+                                                         out.node_off, out.coarse, out.rowptr, in.B, in.E,
+                                                         out.deg, tmp);
+    k_row_order<<<(in.N + TB - 1) / TB, TB, 0, st>>>(out.rowptr, tmp, in.N, out.col, out.long_rows,
                                                       out.long_count);
-    k_row_order_long<<<kNumSMs, 256, 0, st>>>(out.rowptr, out.tmp_eid, in.edge_src, out.seg_id,
-                                              out.node_off, out.col, out.long_rows, out.long_count);
+    k_row_order_long<<<kNumSMs, 256, 0, st>>>(out.rowptr, tmp, out.col, out.long_rows, out.long_count);
     launches += 3;
   }
   return launches;
@@ -239,16 +255,18 @@ int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cu
 
 // ---- packing without any allocation -----------------------------------------------------------
 // Scratch for xrl_pack_csr_static lives in the library image instead of in memory obtained at run
-// time.  Layout (int32 words): n_nodes[G] n_edges[G] env_off[V+1] deg[N] tmp_eid[E] long_rows[E/32+1]
-// long_count[1] scan workspace[kStaticScanInts], with G/V/N/E the maxima below.
+// time.  Layout (int32 words): n_nodes[G] n_edges[G] env_off[V+1] deg[N] tmp[2E] long_rows[E/32+1]
+// long_count[1] scan workspace[kStaticScanInts] coarse[E/1024+1], with G/V/N/E the maxima below.
 namespace {
 
 constexpr int64_t kStG = XRL_STATIC_PACK_MAX_GRAPHS, kStV = XRL_STATIC_PACK_MAX_ENVS,
                   kStN = XRL_STATIC_PACK_MAX_NODES, kStE = XRL_STATIC_PACK_MAX_EDGES;
 constexpr int64_t kStaticScanInts = 1024;
 constexpr int64_t kOffNn = 0, kOffNe = kOffNn + kStG, kOffEnv = kOffNe + kStG, kOffDeg = kOffEnv + kStV + 1,
-                  kOffTmp = kOffDeg + kStN, kOffLong = kOffTmp + kStE, kOffCount = kOffLong + kStE / 32 + 1,
-                  kOffScan = kOffCount + 1, kStaticInts = kOffScan + kStaticScanInts;
+                  kOffTmp = (kOffDeg + kStN + 1) & ~int64_t(1) /* 8-byte aligned pairs */,
+                  kOffLong = kOffTmp + 2 * kStE,
+                  kOffCount = kOffLong + kStE / 32 + 1, kOffScan = kOffCount + 1,
+                  kOffCoarse = kOffScan + kStaticScanInts, kStaticInts = kOffCoarse + (kStE >> 10) + 1;
 
 static __device__ __align__(256) int32_t g_pack_scratch[kStaticInts];
 
@@ -314,7 +332,7 @@ extern "C" xrl_status xrl_pack_csr_static(int32_t device, int32_t num_op_types, 
   out.node_off = node_off; out.edge_off = edge_off; out.seg_id = seg_id; out.graph_env = graph_env;
   out.rowptr = rowptr; out.col = col;
   out.deg = sc + kOffDeg; out.tmp_eid = sc + kOffTmp; out.long_rows = sc + kOffLong;
-  out.long_count = sc + kOffCount; out.scan_ws = sc + kOffScan;
+  out.long_count = sc + kOffCount; out.scan_ws = sc + kOffScan; out.coarse = sc + kOffCoarse;
   // the pack kernels zero what they count into (deg, the row cursors, long_count) themselves
   launch_pack(in, out, num_op_types, device_status, st);
   if (cudaGetLastError() != cudaSuccess) return XRL_ERR_CUDA;

@@ -86,7 +86,7 @@ struct xrl_batch {
   // device
   DeviceBuf meta;           // n_nodes[B] n_edges[B] env_off[Ne+1] graph_chunk_off[B+1] chunk_row0[] chunk_row1[]
   DeviceBuf node_off, edge_off, seg_id, graph_env, rowptr, col, op, shape;
-  DeviceBuf edge_src, edge_dst, deg, tmp_eid, long_rows, long_count, scan_ws;
+  DeviceBuf edge_src, edge_dst, deg, tmp_eid, long_rows, long_count, scan_ws, coarse;
   const int32_t *d_n_nodes = nullptr, *d_n_edges = nullptr, *d_env_off = nullptr,
                 *d_graph_chunk_off = nullptr, *d_chunk_row0 = nullptr, *d_chunk_row1 = nullptr;
   // pinned host staging (allocated on the first pack from host memory)
@@ -154,8 +154,8 @@ xrl_status alloc_batch(xrl_ctx* ctx, xrl_batch** out) {
   A(b->rowptr, 4 * (N + 1)); A(b->col, 4 * E);
   A(b->op, 4 * N); A(b->shape, sb * N * kS);
   A(b->edge_src, 4 * E); A(b->edge_dst, 4 * E);
-  A(b->deg, 4 * N); A(b->tmp_eid, 4 * E);
-  A(b->long_rows, 4 * (E / 32 + 1)); A(b->long_count, 4);
+  A(b->deg, 4 * N); A(b->tmp_eid, 8 * E + 8);
+  A(b->long_rows, 4 * (E / 32 + 1)); A(b->long_count, 4); A(b->coarse, 4 * (E / 1024 + 2));
   A(b->scan_ws, 4 * scan_workspace_ints(int64_t(N > B ? N : B) + 1));
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&b->staged, cudaEventDisableTiming);
   if (e != cudaSuccess) {
@@ -338,7 +338,7 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
   po.rowptr = b->rowptr.as<int32_t>(); po.col = b->col.as<int32_t>();
   po.deg = b->deg.as<int32_t>(); po.tmp_eid = b->tmp_eid.as<int32_t>();
   po.long_rows = b->long_rows.as<int32_t>(); po.long_count = b->long_count.as<int32_t>();
-  po.scan_ws = b->scan_ws.as<int32_t>();
+  po.scan_ws = b->scan_ws.as<int32_t>(); po.coarse = b->coarse.as<int32_t>();
   {
     const size_t slot = ctx->prof.begin(st);
     ctx->launches_pack = launch_pack(in, po, c.num_op_types, ctx->status.as<int32_t>(), st);
@@ -536,7 +536,7 @@ xrl_status xrl_batch_free(xrl_ctx* ctx, xrl_batch* b) {
   cudaDeviceSynchronize();
   DeviceBuf* bufs[] = {&b->meta, &b->node_off, &b->edge_off, &b->seg_id, &b->graph_env, &b->rowptr,
                        &b->col, &b->op, &b->shape, &b->edge_src, &b->edge_dst, &b->deg, &b->tmp_eid,
-                       &b->long_rows, &b->long_count, &b->scan_ws};
+                       &b->long_rows, &b->long_count, &b->scan_ws, &b->coarse};
   for (DeviceBuf* d : bufs) d->release();
   if (b->h_meta) cudaFreeHost(b->h_meta);
   if (b->h_bulk) cudaFreeHost(b->h_bulk);

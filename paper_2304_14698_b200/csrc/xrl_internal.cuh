@@ -88,7 +88,7 @@ struct PackIn {
 };
 struct PackOut {
   int32_t *node_off, *edge_off, *seg_id, *graph_env, *rowptr, *col;
-  int32_t *deg, *tmp_eid, *long_rows, *long_count, *scan_ws;   // scratch
+  int32_t *deg, *tmp_eid /* [2E]: (edge id, producer) pairs */, *long_rows, *long_count, *scan_ws, *coarse;   // scratch
 };
 int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cudaStream_t st);
 size_t scan_workspace_ints(int64_t n);
