@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = [
     "xrl_policy_value", "xrl_sample", "xrl_last_device_status", "xrl_launch_counts", "xrl_version",
     "xrl_profile", "xrl_profile_read", "xrl_pack_csr_static",
 ]
-PROFILE_FAMILIES = ["pack", "node_update", "transform", "aggregate", "readout", "heads"]
+PROFILE_FAMILIES = ["pack", "node_update", "transform", "aggregate", "readout", "heads", "aggregate_readout"]
 
 
 class XrlError(RuntimeError):

@@ -32,7 +32,7 @@ size_t storage_bytes(int dtype) { return dtype == XRL_BF16 ? 2 : 4; }
 
 // Optional per-kernel-family timing: CUDA events recorded on the launching stream around every
 // launcher call.  Families index the steps of the path.
-enum { FAM_PACK = 0, FAM_EMBED, FAM_XFORM, FAM_AGG, FAM_READOUT, FAM_HEADS, FAM_COUNT };
+enum { FAM_PACK = 0, FAM_EMBED, FAM_XFORM, FAM_AGG, FAM_READOUT, FAM_HEADS, FAM_AGG_READOUT, FAM_COUNT };
 
 struct Profiler {
   bool on = false;
@@ -382,18 +382,19 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
     n += k;
     slot = pf.begin(st);
     k = -1;
+    bool fused_here = false;
     if (fuse_readout && l == layers - 1) {
       k = launch_aggregate_tma(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), ctx->Z.p,
                                ctx->scores.as<float>(), ctx->dw.layer[l].b, ctx->h.p, win, b->N,
                                b->seg_id.as<int32_t>(), ctx->partial.as<float>(),
                                ctx->status.as<int32_t>(), st);
-      if (k >= 0 && fused) *fused = true;
+      if (k >= 0) { fused_here = true; if (fused) *fused = true; }
     }
     if (k < 0)
       k = launch_aggregate(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), ctx->Z.p,
                            ctx->scores.as<float>(), ctx->dw.layer[l].b,
                            ctx->h.p, win, b->N, ctx->status.as<int32_t>(), st);
-    pf.end(FAM_AGG, slot, k, st);
+    pf.end(fused_here ? FAM_AGG_READOUT : FAM_AGG, slot, k, st);
     n += k;
   }
   return n;
