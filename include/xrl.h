@@ -153,6 +153,26 @@ xrl_status xrl_batch_export(const xrl_batch* batch, int32_t* rowptr, int32_t* co
 xrl_status xrl_encode(xrl_ctx* ctx, const xrl_batch* batch, const float* g0, float* graph_emb,
                       void* stream);
 
+/* Delta encoding: same result as xrl_encode (within rounding), computed only where it can differ.
+ * The candidates of a step are the current graph with one rewrite applied at one location (paper
+ * Sections 3.2, 3.3.1), so almost every candidate node equals a node of the current graph.  A candidate
+ * node with the same operator, shape features and producers as a current-graph node, whose producers are
+ * unchanged too, has that node's features after Eq. 6; a change reaches a node one attention layer after
+ * it reached one of its producers (Eq. 7 looks at producers only).  Per layer the library lists the rows
+ * a change has reached, runs the encoder kernels on those rows only (current graphs are always computed
+ * in full) and lets every other candidate node read its current-graph twin.
+ *   base_id  DEVICE int32 [N], or NULL: for node i of a candidate graph, the global (packed) id of the node
+ *            of its environment's current graph that it corresponds to, or -1.  It is a HINT: the library
+ *            verifies operator, shape features and producer lists on the device and recomputes whatever
+ *            does not check out, so a wrong hint costs time, never correctness.  Entries of current-graph
+ *            nodes are ignored.
+ * The call synchronises `stream` once per layer (it reads the number of listed rows back).
+ * xrl_delta_rows reports, for the last call, the rows computed at Eq. 6 and after each attention layer
+ * (HOST int64 [count], count <= L + 1). */
+xrl_status xrl_encode_delta(xrl_ctx* ctx, const xrl_batch* batch, const int32_t* base_id, const float* g0,
+                            float* graph_emb, void* stream);
+xrl_status xrl_delta_rows(const xrl_ctx* ctx, int64_t* rows, int32_t count);
+
 /* Debug aid for parity tests: run Eq. 6 and the first `num_layers` attention layers
  * (0 <= num_layers <= L) and copy the node features to HOST fp32 [N x H].  Synchronous. */
 xrl_status xrl_debug_node_features(xrl_ctx* ctx, const xrl_batch* batch, int32_t num_layers,

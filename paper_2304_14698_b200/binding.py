@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = [
     "xrl_create", "xrl_destroy", "xrl_weights_size", "xrl_set_weights", "xrl_pack", "xrl_pack_flat",
     "xrl_batch_free", "xrl_batch_info", "xrl_batch_export", "xrl_encode", "xrl_debug_node_features",
     "xrl_policy_value", "xrl_sample", "xrl_last_device_status", "xrl_launch_counts", "xrl_version",
-    "xrl_profile", "xrl_profile_read", "xrl_pack_csr_static",
+    "xrl_profile", "xrl_profile_read", "xrl_pack_csr_static", "xrl_encode_delta", "xrl_delta_rows",
 ]
 PROFILE_FAMILIES = ["pack", "node_update", "transform", "aggregate", "readout", "heads", "aggregate_readout"]
 
@@ -79,6 +79,8 @@ def load_library():
         "xrl_last_device_status": [vp, vp, C.POINTER(i32)],
         "xrl_launch_counts": [vp, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64)],
         "xrl_profile": [vp, i32],
+        "xrl_encode_delta": [vp, vp, vp, vp, vp, vp],
+        "xrl_delta_rows": [vp, C.POINTER(i64), i32],
         "xrl_pack_csr_static": [i32, i32, i32] + [vp] * 6 + [i32] + [vp] * 8,
         "xrl_profile_read": [vp, C.POINTER(C.c_double), C.POINTER(i64), i32],
     }
@@ -221,6 +223,20 @@ def xrl_encode(ctx, batch, graph_emb, g0=None, stream=None):
     return graph_emb
 
 
+def xrl_encode_delta(ctx, batch, base_id, graph_emb, g0=None, stream=None):
+    """Like xrl_encode, recomputing only what a candidate's rewrite can change.  base_id: torch CUDA int32
+    [N] hint (packed id of the equal node of the env's current graph, or -1), or None."""
+    _check(load_library().xrl_encode_delta(ctx, batch, _dev_ptr(base_id), _dev_ptr(g0), _dev_ptr(graph_emb),
+                                           _stream(stream)), "xrl_encode_delta")
+    return graph_emb
+
+
+def xrl_delta_rows(ctx, layers):
+    rows = (C.c_int64 * (layers + 1))()
+    _check(load_library().xrl_delta_rows(ctx, rows, layers + 1), "xrl_delta_rows")
+    return [int(v) for v in rows]
+
+
 def xrl_debug_node_features(ctx, batch, num_layers, hidden, stream=None):
     info = xrl_batch_info(batch)
     out = np.zeros((info["num_nodes"], hidden), np.float32)
@@ -356,19 +372,23 @@ class Agent:
         self.batch = xrl_pack(self.ctx, graphs, env_off, self.m["dtype"], batch=self.batch)
         return self.batch
 
-    def forward(self, mask, sample=False, seed=0, step=0, g0=None):
-        """Encode the packed batch and evaluate the heads.  mask: torch CUDA uint8 [envs, A_max]."""
+    def forward(self, mask, sample=False, seed=0, step=0, g0=None, base_id=None):
+        """Encode the packed batch and evaluate the heads.  mask: torch CUDA uint8 [envs, A_max].
+        base_id (torch CUDA int32 [N]) switches to delta encoding of the candidates."""
         info = xrl_batch_info(self.batch)
         o = self._buffers(info["num_graphs"], info["num_envs"])
-        xrl_encode(self.ctx, self.batch, o["emb"], g0)
+        if base_id is None:
+            xrl_encode(self.ctx, self.batch, o["emb"], g0)
+        else:
+            xrl_encode_delta(self.ctx, self.batch, base_id, o["emb"], g0)
         xrl_policy_value(self.ctx, self.batch, o["emb"], mask, o["probs"], o["value"],
                          o["action"] if sample else None, seed, step)
         return o
 
-    def step(self, batch, mask, sample=False, seed=0, step=0):
+    def step(self, batch, mask, sample=False, seed=0, step=0, base_id=None):
         """The whole path for one batch: pack -> encode -> policy/value (-> sample)."""
         self.pack(batch)
-        return self.forward(mask, sample, seed, step)
+        return self.forward(mask, sample, seed, step, base_id=base_id)
 
     def device_status(self):
         return xrl_last_device_status(self.ctx)

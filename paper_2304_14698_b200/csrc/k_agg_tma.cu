@@ -166,7 +166,7 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
                 const T* __restrict__ Z, const float2* __restrict__ scores,
                 const float* __restrict__ bias, T* __restrict__ h_out, Window win,
                 const int32_t* __restrict__ seg_id, float* __restrict__ partial, int32_t nblocks,
-                int32_t* status) {
+                const int32_t* __restrict__ self_idx, int32_t* status) {
   constexpr int VEC = VecOf<T>::N;
   constexpr int NP = VEC / 2;
   constexpr int H = 32 * VEC;
@@ -255,11 +255,12 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
         // a row with more producers than the list holds: plain loads, one producer at a time
         const int32_t lrow = int32_t(r0) + rs - win.win_base;
         const int n = sm.rp[rs + 1] - eb;
-        const float2 self = __ldg(scores + size_t(lrow) * K + head);
+        const int32_t srow = self_idx ? __ldg(self_idx + int32_t(r0) + rs) : lrow;
+        const float2 self = __ldg(scores + size_t(srow) * K + head);
         const float sd = self.y;
         float m = lrelu(self.x + sd), l = 1.f;
         F2 acc[NP];
-        to_pairs(__ldg(reinterpret_cast<const uint4*>(Z + size_t(lrow) * H + c0)), acc);
+        to_pairs(__ldg(reinterpret_cast<const uint4*>(Z + size_t(srow) * H + c0)), acc);
         for (int t = 0; t < n; ++t) {
           const int32_t j = __ldg(col + eb + t) - win.win_base;
           const float ev = lrelu(__ldg(&scores[size_t(j) * K + head].x) + sd);
@@ -288,7 +289,8 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
       if (lane < cnt) {
         const int e0 = sm.rp[rs + lane] - eb, n = sm.rp[rs + lane + 1] - eb - e0;
         int pos = lane + e0;
-        sm.item[pos++] = int32_t(r0) + rs + lane - win.win_base;
+        sm.item[pos++] = self_idx ? __ldg(self_idx + int32_t(r0) + rs + lane)       // where the row's own Z lives
+                                  : int32_t(r0) + rs + lane - win.win_base;
         for (int t = 0; t < n; ++t) sm.item[pos++] = __ldg(col + eb + e0 + t) - win.win_base;
       }
       if (lane < 4) sm.item[total + lane] = int32_t(r0) + rs - win.win_base;   // pad the last group
@@ -378,7 +380,7 @@ bool make_row_map(CUtensorMap* m, const void* ptr, CUtensorMapDataType dt, uint3
 template <typename T, int K, bool READOUT>
 int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const float* scores, const float* bias,
              void* h_out, Window win, int64_t buf_rows, const int32_t* seg_id, float* partial,
-             int32_t* status, cudaStream_t st) {
+             const int32_t* self_idx, int32_t* status, cudaStream_t st) {
   static bool attr = false;
   const size_t smem = sizeof(WarpSmem<K>) * TW;
   if (!attr) {
@@ -401,7 +403,7 @@ int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const flo
   if (nb > int64_t(kNumSMs) * XRL_AGG_CTAS) nb = int64_t(kNumSMs) * XRL_AGG_CTAS;
   k_aggregate_tma<T, K, READOUT><<<int(nb), TW * 32, smem, st>>>(
       mz, ms, rowptr, col, static_cast<const T*>(Z), reinterpret_cast<const float2*>(scores), bias,
-      static_cast<T*>(h_out), win, seg_id, partial, int32_t(nblocks), status);
+      static_cast<T*>(h_out), win, seg_id, partial, int32_t(nblocks), self_idx, status);
   return 1;
 }
 
@@ -412,7 +414,8 @@ int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const flo
 // the window must start at row 0).  Returns kernels launched, or -1 when this shape is not handled here.
 int launch_aggregate_tma(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z,
                          const float* scores, const float* bias, void* h_out, Window win, int64_t buf_rows,
-                         const int32_t* seg_id, float* partial, int32_t* status, cudaStream_t st) {
+                         const int32_t* seg_id, float* partial, int32_t* status, cudaStream_t st,
+                         const int32_t* self_idx) {
   if (encode_fn() == nullptr) return -1;
   const bool bf = d.dtype == XRL_BF16 && d.H == 256, fp = d.dtype == XRL_FP32 && d.H == 128;
   if (!bf && !fp) return -1;
@@ -421,13 +424,13 @@ int launch_aggregate_tma(const Dims& d, const int32_t* rowptr, const int32_t* co
   case KK:                                                                                                 \
     if (partial != nullptr)                                                                                \
       return bf ? launch_k<bf16, KK, true>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, seg_id,     \
-                                           partial, status, st)                                            \
+                                           partial, self_idx, status, st)                                            \
                 : launch_k<float, KK, true>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, seg_id,    \
-                                            partial, status, st);                                          \
+                                            partial, self_idx, status, st);                                          \
     return bf ? launch_k<bf16, KK, false>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, seg_id,      \
-                                          partial, status, st)                                             \
+                                          partial, self_idx, status, st)                                             \
               : launch_k<float, KK, false>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, seg_id,     \
-                                           partial, status, st);
+                                           partial, self_idx, status, st);
   switch (d.K) {
     TMA_CASE(4) TMA_CASE(8) TMA_CASE(16)
     default: return -1;

@@ -44,8 +44,9 @@ template <int H>
 __global__ void __launch_bounds__(kThreads, 1)
 k_embed_umma(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_h,
              const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
-             const int32_t* __restrict__ op, const bf16* __restrict__ shape, int row_begin, int rows,
-             int op_pieces, int ksteps, int32_t* status) {
+             const int32_t* __restrict__ op, const bf16* __restrict__ shape,
+             const int32_t* __restrict__ row_list, int row_begin, int rows, int op_pieces, int ksteps,
+             int32_t* status) {
   using C = ECfg<H>;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t base = smem_u32(smem);
@@ -170,7 +171,7 @@ k_embed_umma(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ 
       uint4 own = make_uint4(0, 0, 0, 0);
       int o = -1;
       if (lrow < rows) {
-        const int32_t row = row_begin + lrow;
+        const int32_t row = row_list ? __ldg(row_list + lrow) : row_begin + lrow;   // listed rows are written densely
         const int32_t e0 = __ldg(rowptr + row), e1 = __ldg(rowptr + row + 1);
         own = __ldg(reinterpret_cast<const uint4*>(shape + size_t(row) * kS));
         o = __ldg(op + row);
@@ -238,8 +239,8 @@ __global__ void k_build_w0ext(const bf16* __restrict__ W0, const float* __restri
 
 template <int H>
 int launch_h(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op,
-             const void* shape, const void* w0ext_t, void* h, Window win, int32_t* status,
-             cudaStream_t st) {
+             const void* shape, const void* w0ext_t, void* h, Window win, const int32_t* row_list,
+             int32_t* status, cudaStream_t st) {
   using C = ECfg<H>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -260,8 +261,8 @@ int launch_h(const Dims& d, const int32_t* rowptr, const int32_t* col, const int
   const int tiles = int((rows + BM - 1) / BM);
   const int grid = tiles < kNumSMs ? tiles : kNumSMs;
   k_embed_umma<H><<<grid, kThreads, C::SMEM_BYTES, st>>>(mw, mh, rowptr, col, op,
-                                                         static_cast<const bf16*>(shape), win.row_begin,
-                                                         int(rows), op_pieces, ksteps, status);
+                                                         static_cast<const bf16*>(shape), row_list,
+                                                         win.row_begin, int(rows), op_pieces, ksteps, status);
   return 1;
 }
 
@@ -285,10 +286,10 @@ void build_w0ext(const Dims& d, const void* W0_store, const float* b0, void* out
 
 int launch_embed_umma(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op,
                       const void* shape, const void* w0ext_t, void* h, Window win, int32_t* status,
-                      cudaStream_t st) {
+                      cudaStream_t st, const int32_t* row_list) {
   if (int64_t(win.row_end) - win.row_begin <= 0) return 0;
-  if (d.H == 256) return launch_h<256>(d, rowptr, col, op, shape, w0ext_t, h, win, status, st);
-  return launch_h<128>(d, rowptr, col, op, shape, w0ext_t, h, win, status, st);
+  if (d.H == 256) return launch_h<256>(d, rowptr, col, op, shape, w0ext_t, h, win, row_list, status, st);
+  return launch_h<128>(d, rowptr, col, op, shape, w0ext_t, h, win, row_list, status, st);
 }
 
 }  // namespace xrl

@@ -31,7 +31,7 @@ template <typename T>
 __global__ void __launch_bounds__(kRoThreads)
 k_readout(const T* __restrict__ h, const int32_t* __restrict__ chunk_row0,
           const int32_t* __restrict__ chunk_row1, int32_t chunk_begin, float* __restrict__ partial,
-          int H, int32_t win_base) {
+          int H, int32_t win_base, const int32_t* __restrict__ remap) {
   constexpr int VEC = VecOf<T>::N;
   extern __shared__ float red[];                 // [RG][H]
   const int NV = H / VEC;
@@ -48,7 +48,7 @@ k_readout(const T* __restrict__ h, const int32_t* __restrict__ chunk_row0,
       float f[4][VEC];
 #pragma unroll
       for (int u = 0; u < 4; ++u)
-        load_vec(h + size_t(r + u * RG - win_base) * H + vi * VEC, f[u]);
+        load_vec(h + size_t(remap ? __ldg(remap + r + u * RG) : r + u * RG - win_base) * H + vi * VEC, f[u]);
 #pragma unroll
       for (int u = 0; u < 4; ++u)
 #pragma unroll
@@ -56,7 +56,7 @@ k_readout(const T* __restrict__ h, const int32_t* __restrict__ chunk_row0,
     }
     for (; r < r1; r += RG) {
       float f[VEC];
-      load_vec(h + size_t(r - win_base) * H + vi * VEC, f);
+      load_vec(h + size_t(remap ? __ldg(remap + r) : r - win_base) * H + vi * VEC, f);
 #pragma unroll
       for (int t = 0; t < VEC; ++t) acc[t] += f[t];
     }
@@ -357,17 +357,17 @@ int pow2_threads(int want) {          // power of two in [32, 1024] (block_sum n
 
 int launch_readout(const Dims& d, const void* h, const int32_t* chunk_row0, const int32_t* chunk_row1,
                    int32_t chunk_begin, int32_t chunk_end, float* partial, int32_t win_base,
-                   cudaStream_t st) {
+                   cudaStream_t st, const int32_t* remap) {
   const int n = chunk_end - chunk_begin;
   if (n <= 0) return 0;
   if (d.dtype == XRL_BF16) {
     const int RG = kRoThreads / (d.H / 8);
     k_readout<bf16><<<n, kRoThreads, sizeof(float) * size_t(RG) * d.H, st>>>(
-        static_cast<const bf16*>(h), chunk_row0, chunk_row1, chunk_begin, partial, d.H, win_base);
+        static_cast<const bf16*>(h), chunk_row0, chunk_row1, chunk_begin, partial, d.H, win_base, remap);
   } else {
     const int RG = kRoThreads / (d.H / 4);
     k_readout<float><<<n, kRoThreads, sizeof(float) * size_t(RG) * d.H, st>>>(
-        static_cast<const float*>(h), chunk_row0, chunk_row1, chunk_begin, partial, d.H, win_base);
+        static_cast<const float*>(h), chunk_row0, chunk_row1, chunk_begin, partial, d.H, win_base, remap);
   }
   return 1;
 }

@@ -202,6 +202,10 @@ k_row_order_long(const int32_t* __restrict__ rowptr, const int2* __restrict__ tm
 
 }  // namespace
 
+int launch_exclusive_scan(const int32_t* in, int32_t* out, int32_t n_in, int32_t* ws, cudaStream_t st) {
+  return exclusive_scan(in, out, n_in, ws, st);
+}
+
 size_t scan_workspace_ints(int64_t n) {
   size_t total = 0;
   int64_t m = n + 1;

@@ -27,7 +27,8 @@ template <typename T, int LPR, int VPL>
 __global__ void __launch_bounds__(kRowThreads)
 k_embed(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
         const int32_t* __restrict__ op, const T* __restrict__ shape, const T* __restrict__ W0,
-        const float* __restrict__ b0, T* __restrict__ h, int H, int Tn, Window win) {
+        const float* __restrict__ b0, T* __restrict__ h, int H, int Tn, Window win,
+        const int32_t* __restrict__ row_list) {
   constexpr int VEC = VecOf<T>::N;
   constexpr int RPW = 32 / LPR;
   extern __shared__ float smem[];
@@ -47,8 +48,9 @@ k_embed(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
   const int warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * RPW; r0 < win.row_end;
        r0 += int64_t(warps_total) * RPW) {
-    const int32_t row = int32_t(r0) + sub;
-    if (row >= win.row_end) continue;
+    const int32_t out_row = int32_t(r0) + sub;
+    if (out_row >= win.row_end) continue;
+    const int32_t row = row_list ? __ldg(row_list + out_row) : out_row;   // listed rows are written densely
     float x[2 * kS];
 #pragma unroll
     for (int s = 0; s < kS; ++s) x[s] = 0.f;
@@ -66,7 +68,7 @@ k_embed(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
       for (int s = 0; s < kS; ++s) x[kS + s] = f[s];
     }
     const T* lookup = W0 + size_t(kS + __ldg(op + row)) * H;
-    T* out = h + size_t(row - win.win_base) * H;
+    T* out = h + size_t(out_row - win.win_base) * H;
 #pragma unroll
     for (int v = 0; v < VPL; ++v) {
       const int vi = v * LPR + sl;
@@ -199,7 +201,8 @@ template <typename T, int LPR, int VPL>
 __global__ void __launch_bounds__(kRowThreads, (VPL == 1 ? 4 : 2))
 k_aggregate(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
             const T* __restrict__ Z, const float2* __restrict__ scores,
-            const float* __restrict__ bias, T* __restrict__ h_out, int H, int K, Window win) {
+            const float* __restrict__ bias, T* __restrict__ h_out, int H, int K, Window win,
+            const int32_t* __restrict__ self_idx) {
   constexpr int VEC = VecOf<T>::N;
   constexpr int RPW = 32 / LPR;
   constexpr int WARPS = kRowThreads / 32;
@@ -248,11 +251,12 @@ k_aggregate(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
         if (!on[v]) continue;
         const T* zlane = Z + c0[v];
         const float2* slane = scores + head[v];
-        const float2 self = __ldg(slane + size_t(lrow) * K);
+        const int32_t srow = self_idx ? __ldg(self_idx + int32_t(r0) + rr) : lrow;   // where the row's own Z lives
+        const float2 self = __ldg(slane + size_t(srow) * K);
         const float sd = self.y;
         float m = lrelu(self.x + sd);                               // the self term opens the softmax
         float l = 1.f, acc[VEC];
-        load_vec(zlane + size_t(lrow) * H, acc);
+        load_vec(zlane + size_t(srow) * H, acc);
         int t = 0;
         for (; t + 4 <= n; t += 4) agg_group<T, 4>(js + t, win.win_base, zlane, slane, H, K, sd, m, l, acc);
         const int rem = n - t;                          // the same for all lanes of a row group
@@ -302,14 +306,15 @@ int row_grid(int64_t rows, int rpw) {
 }  // namespace
 
 int launch_embed(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op,
-                 const void* shape, const DevWeights& w, void* h, Window win, cudaStream_t st) {
+                 const void* shape, const DevWeights& w, void* h, Window win, cudaStream_t st,
+                 const int32_t* row_list) {
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   if (rows <= 0) return 0;
   const size_t smem = sizeof(float) * size_t(2 * kS + 1) * d.H;
 #define CALL(TY_, LPR, VPL)                                                                        \
   k_embed<TY_, LPR, VPL><<<row_grid(rows, 32 / LPR), kRowThreads, smem, st>>>(                     \
       rowptr, col, op, static_cast<const TY_*>(shape), static_cast<const TY_*>(w.W0), w.b0,   \
-      static_cast<TY_*>(h), d.H, d.T, win)
+      static_cast<TY_*>(h), d.H, d.T, win, row_list)
   if (d.dtype == XRL_BF16) XRL_ROW_DISPATCH(bf16, d.H, CALL);
   else XRL_ROW_DISPATCH(float, d.H, CALL);
 #undef CALL
@@ -331,17 +336,19 @@ int launch_scores(const Dims& d, const void* Z, const LayerWeights& lw, float* s
 
 int launch_aggregate(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z,
                      const float* scores, const float* bias, void* h_out,
-                     Window win, int64_t buf_rows, int32_t* status, cudaStream_t st) {
+                     Window win, int64_t buf_rows, int32_t* status, cudaStream_t st,
+                     const int32_t* self_idx) {
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   if (rows <= 0) return 0;
   {   // 512-byte rows with 4 | K: gathers by the TMA engine
-    const int k = launch_aggregate_tma(d, rowptr, col, Z, scores, bias, h_out, win, buf_rows, nullptr, nullptr, status, st);
+    const int k = launch_aggregate_tma(d, rowptr, col, Z, scores, bias, h_out, win, buf_rows, nullptr, nullptr, status, st,
+                                       self_idx);
     if (k >= 0) return k;
   }
 #define CALL(TY_, LPR, VPL)                                                                        \
   k_aggregate<TY_, LPR, VPL><<<row_grid(rows, kAggBlockRows), kRowThreads, 0, st>>>(                \
       rowptr, col, static_cast<const TY_*>(Z), reinterpret_cast<const float2*>(scores), bias,       \
-      static_cast<TY_*>(h_out), d.H, d.K, win)
+      static_cast<TY_*>(h_out), d.H, d.K, win, self_idx)
   if (d.dtype == XRL_BF16) XRL_ROW_DISPATCH(bf16, d.H, CALL);
   else XRL_ROW_DISPATCH(float, d.H, CALL);
 #undef CALL

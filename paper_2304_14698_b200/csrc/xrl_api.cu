@@ -76,6 +76,10 @@ struct xrl_ctx {
   DeviceBuf h, Z, scores, partial, logits, status;
   int32_t max_chunks = 0;
   int64_t launches_pack = 0, launches_encode = 0, launches_heads = 0;
+  // delta encoding workspace (allocated on the first xrl_encode_delta)
+  DeviceBuf dl_ints, dl_col, dl_scan;
+  int32_t* dl_host = nullptr;      // pinned: row counts read back per layer
+  int64_t delta_rows[65] = {0};    // rows computed per layer by the last xrl_encode_delta
 };
 
 struct xrl_batch {
@@ -469,6 +473,8 @@ void xrl_destroy(xrl_ctx* ctx) {
                        &ctx->partial, &ctx->logits, &ctx->status};
   for (DeviceBuf* d : bufs) d->release();
   ctx->prof.release();
+  ctx->dl_ints.release(); ctx->dl_col.release(); ctx->dl_scan.release();
+  if (ctx->dl_host) cudaFreeHost(ctx->dl_host);
   delete ctx;
 }
 
@@ -601,6 +607,129 @@ xrl_status xrl_encode(xrl_ctx* ctx, const xrl_batch* b, const float* g0, float* 
   n += k;
   ctx->launches_encode = n;
   XRL_CUDA(cudaGetLastError());
+  return XRL_OK;
+}
+
+xrl_status xrl_encode_delta(xrl_ctx* ctx, const xrl_batch* b, const int32_t* base_id, const float* g0,
+                            float* graph_emb, void* stream) {
+  const xrl_status s = check_batch(ctx, b);
+  if (s != XRL_OK) return s;
+  if (!graph_emb && b->B > 0) return XRL_ERR_INVALID_ARG;
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t Ncap = size_t(ctx->cfg.max_nodes) + 1, Ecap = size_t(ctx->cfg.max_edges) + 1;
+  if (ctx->dl_ints.p == nullptr) {
+    XRL_ALLOC(ctx->dl_ints.alloc(4 * 11 * Ncap));
+    XRL_ALLOC(ctx->dl_col.alloc(4 * Ecap));
+    XRL_ALLOC(ctx->dl_scan.alloc(4 * scan_workspace_ints(int64_t(Ncap))));
+    XRL_ALLOC(cudaHostAlloc(reinterpret_cast<void**>(&ctx->dl_host), 4 * 4, cudaHostAllocDefault));
+  }
+  int32_t* I = ctx->dl_ints.as<int32_t>();
+  int32_t *valid = I, *base = I + Ncap, *flag_prev = I + 2 * Ncap, *flag_cur = I + 3 * Ncap,
+          *rank_prev = I + 4 * Ncap, *rank_cur = I + 5 * Ncap, *list = I + 6 * Ncap, *deg = I + 7 * Ncap,
+          *rowptr_c = I + 8 * Ncap, *self_c = I + 9 * Ncap, *remap = I + 10 * Ncap;
+  int32_t* col_c = ctx->dl_col.as<int32_t>();
+  int32_t* scan_ws = ctx->dl_scan.as<int32_t>();
+  const Dims& d = ctx->dims;
+  const int N = b->N;
+
+  DeltaIn in;
+  in.N = N; in.E = b->E;
+  in.seg_id = b->seg_id.as<int32_t>(); in.graph_env = b->graph_env.as<int32_t>();
+  in.env_off = b->d_env_off; in.node_off = b->node_off.as<int32_t>();
+  in.rowptr = b->rowptr.as<int32_t>(); in.col = b->col.as<int32_t>(); in.op = b->op.as<int32_t>();
+  in.shape = b->shape.p; in.shape_bytes = int(storage_bytes(d.dtype)) * kS;
+  in.base_id = base_id;
+
+  // rows of rank[N] read back: the launches of a layer are sized by its number of dirty rows
+  auto count_of = [&](const int32_t* rank, int32_t* out) -> xrl_status {
+    XRL_CUDA(cudaMemcpyAsync(ctx->dl_host, rank + N, 4, cudaMemcpyDeviceToHost, st));
+    XRL_CUDA(cudaStreamSynchronize(st));
+    *out = ctx->dl_host[0];
+    return XRL_OK;
+  };
+  Profiler& pf = ctx->prof;
+  int n_launch = 0;
+  size_t slot = pf.begin(st);
+  int k = launch_delta_init(in, valid, base, flag_prev, st);
+  k += launch_exclusive_scan(flag_prev, rank_prev, N, scan_ws, st);
+  k += launch_delta_list(N, flag_prev, rank_prev, list, st);
+  pf.end(FAM_PACK, slot, k, st);
+  n_launch += k;
+  int32_t n_prev = 0;
+  xrl_status rs = count_of(rank_prev, &n_prev);
+  if (rs != XRL_OK) return rs;
+  ctx->delta_rows[0] = n_prev;
+
+  // Eq. 6 on the listed rows, written densely
+  slot = pf.begin(st);
+  const Window w0{0, n_prev, 0};
+  k = -1;
+  if (ctx->use_umma_embed)
+    k = launch_embed_umma(d, in.rowptr, in.col, in.op, b->shape.p, ctx->w0ext.p, ctx->h.p, w0,
+                          ctx->status.as<int32_t>(), st, list);
+  if (k < 0) k = launch_embed(d, in.rowptr, in.col, in.op, b->shape.p, ctx->dw, ctx->h.p, w0, st, list);
+  pf.end(FAM_EMBED, slot, k, st);
+  n_launch += k;
+
+  for (int l = 0; l < d.L; ++l) {
+    // transform of the rows recomputed so far (dense)
+    slot = pf.begin(st);
+    const Window wp{0, n_prev, 0};
+    k = -1;
+    if (ctx->use_umma)
+      k = launch_xform_umma(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), wp,
+                            ctx->status.as<int32_t>(), st);
+    if (k < 0) k = launch_xform_simt(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), wp, st);
+    pf.end(FAM_XFORM, slot, k, st);
+    n_launch += k;
+    // rows reached by the change after this layer, their list and compact CSR
+    slot = pf.begin(st);
+    k = launch_delta_propagate(in, flag_prev, flag_cur, st);
+    k += launch_exclusive_scan(flag_cur, rank_cur, N, scan_ws, st);
+    k += launch_delta_list(N, flag_cur, rank_cur, list, st);
+    pf.end(FAM_PACK, slot, k, st);
+    n_launch += k;
+    int32_t n_cur = 0;
+    rs = count_of(rank_cur, &n_cur);
+    if (rs != XRL_OK) return rs;
+    ctx->delta_rows[l + 1] = n_cur;
+    slot = pf.begin(st);
+    k = launch_delta_degrees(in, n_cur, list, deg, st);
+    k += launch_exclusive_scan(deg, rowptr_c, n_cur, scan_ws, st);
+    k += launch_delta_fill(in, n_cur, list, rowptr_c, flag_prev, rank_prev, base, col_c, self_c, st);
+    pf.end(FAM_PACK, slot, k, st);
+    n_launch += k;
+    // aggregate on the compact CSR: producers and the row's own vector come from the dense Z buffer
+    slot = pf.begin(st);
+    const Window wc{0, n_cur, 0};
+    k = launch_aggregate(d, rowptr_c, col_c, ctx->Z.p, ctx->scores.as<float>(), ctx->dw.layer[l].b, ctx->h.p,
+                         wc, n_prev > 0 ? n_prev : 1, ctx->status.as<int32_t>(), st, self_c);
+    pf.end(FAM_AGG, slot, k, st);
+    n_launch += k;
+    int32_t* t = flag_prev; flag_prev = flag_cur; flag_cur = t;
+    t = rank_prev; rank_prev = rank_cur; rank_cur = t;
+    n_prev = n_cur;
+  }
+  // Eq. 8: every node adds the dense row that holds its features (its own or its base node's)
+  slot = pf.begin(st);
+  k = launch_delta_remap(N, flag_prev, rank_prev, base, remap, st);
+  k += launch_readout(d, ctx->h.p, b->d_chunk_row0, b->d_chunk_row1, 0, b->num_chunks,
+                      ctx->partial.as<float>(), 0, st, remap);
+  pf.end(FAM_READOUT, slot, k, st);
+  n_launch += k;
+  slot = pf.begin(st);
+  k = launch_global_update(d, ctx->partial.as<float>(), b->d_graph_chunk_off, g0, ctx->dw, graph_emb, b->B, st);
+  pf.end(FAM_HEADS, slot, k, st);
+  n_launch += k;
+  ctx->launches_encode = n_launch;
+  XRL_CUDA(cudaGetLastError());
+  return XRL_OK;
+}
+
+xrl_status xrl_delta_rows(const xrl_ctx* ctx, int64_t* rows, int32_t count) {
+  if (!ctx || !rows || count < 0) return XRL_ERR_INVALID_ARG;
+  for (int32_t i = 0; i < count; ++i) rows[i] = (i <= ctx->cfg.layers && i < 65) ? ctx->delta_rows[i] : 0;
   return XRL_OK;
 }
 

@@ -92,13 +92,19 @@ struct PackOut {
 };
 int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cudaStream_t st);
 size_t scan_workspace_ints(int64_t n);
+// out[0..n_in] = exclusive prefix sums of in[0..n_in) (n_in + 1 outputs); ws: scan_workspace_ints(n_in) ints
+int launch_exclusive_scan(const int32_t* in, int32_t* out, int32_t n_in, int32_t* ws, cudaStream_t st);
 
+// Row lists (delta encoding): `row_list` makes the node-update kernels read node row_list[r] and write
+// row r of a dense buffer; `self_idx` tells the aggregate kernels where row r's own Z row lives (its
+// producers come from the compact CSR it is given).
 // Row windows: kernels process global rows [row_begin, row_end); activation buffers (h, Z,
 // scores) are indexed by (row - win_base), CSR / op / shape arrays by the global row id.
 struct Window { int32_t row_begin, row_end, win_base; };
 
 int launch_embed(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op,
-                 const void* shape, const DevWeights& w, void* h, Window win, cudaStream_t st);
+                 const void* shape, const DevWeights& w, void* h, Window win, cudaStream_t st,
+                 const int32_t* row_list = nullptr);
 // scores: [N][K] pairs {s_src, s_dst} (float2), both already multiplied by log2(e)
 int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* scores,
                       Window win, cudaStream_t st);
@@ -107,7 +113,7 @@ int embed_umma_kpad(const Dims& d);
 void build_w0ext(const Dims& d, const void* W0_store, const float* b0, void* out, cudaStream_t st);
 int launch_embed_umma(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op,
                       const void* shape, const void* w0ext_t, void* h, Window win, int32_t* status,
-                      cudaStream_t st);
+                      cudaStream_t st, const int32_t* row_list = nullptr);
 bool xform_umma_supported(const Dims& d);
 int launch_xform_umma(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* scores,
                       Window win, int32_t* status, cudaStream_t st);
@@ -115,17 +121,37 @@ int launch_scores(const Dims& d, const void* Z, const LayerWeights& lw, float* s
                   cudaStream_t st);
 int launch_aggregate(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z,
                      const float* scores, const float* bias, void* h_out,
-                     Window win, int64_t buf_rows, int32_t* status, cudaStream_t st);
+                     Window win, int64_t buf_rows, int32_t* status, cudaStream_t st,
+                     const int32_t* self_idx = nullptr);
 int launch_aggregate_tma(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z,
                          const float* scores, const float* bias, void* h_out, Window win, int64_t buf_rows,
-                         const int32_t* seg_id, float* partial, int32_t* status, cudaStream_t st);
+                         const int32_t* seg_id, float* partial, int32_t* status, cudaStream_t st,
+                         const int32_t* self_idx = nullptr);
 int64_t aggregate_readout_slots(int64_t rows, int64_t B);
 int32_t aggregate_readout_blocks(int64_t rows);
 int launch_global_update_blocks(const Dims& d, const float* partial, const int32_t* node_off, int32_t nblocks,
                                 const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st);
 int launch_readout(const Dims& d, const void* h, const int32_t* chunk_row0, const int32_t* chunk_row1,
                    int32_t chunk_begin, int32_t chunk_end, float* partial, int32_t win_base,
-                   cudaStream_t st);
+                   cudaStream_t st, const int32_t* remap = nullptr);
+
+// ---- delta encoding: candidates reuse the rows of their environment's current graph ---------------
+struct DeltaIn {
+  int32_t N, E;
+  const int32_t *seg_id, *graph_env, *env_off, *node_off, *rowptr, *col, *op;
+  const void* shape;
+  int shape_bytes;                 // bytes of one node's shape features
+  const int32_t* base_id;          // caller's hint
+};
+int launch_delta_init(const DeltaIn& in, int32_t* valid, int32_t* base, int32_t* flag0, cudaStream_t st);
+int launch_delta_propagate(const DeltaIn& in, const int32_t* flag_in, int32_t* flag_out, cudaStream_t st);
+int launch_delta_list(int32_t N, const int32_t* flag, const int32_t* rank, int32_t* list, cudaStream_t st);
+int launch_delta_degrees(const DeltaIn& in, int32_t n, const int32_t* list, int32_t* deg, cudaStream_t st);
+int launch_delta_fill(const DeltaIn& in, int32_t n, const int32_t* list, const int32_t* rowptr_c,
+                      const int32_t* flag_prev, const int32_t* rank_prev, const int32_t* base,
+                      int32_t* col_c, int32_t* self_c, cudaStream_t st);
+int launch_delta_remap(int32_t N, const int32_t* flag, const int32_t* rank, const int32_t* base,
+                       int32_t* remap, cudaStream_t st);
 int launch_global_update(const Dims& d, const float* partial, const int32_t* graph_chunk_off,
                          const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st);
 int launch_heads(const Dims& d, const DevWeights& w, const float* emb, const int32_t* env_off,

@@ -187,7 +187,10 @@ def local_rewrite(rng, g, T, bf16=False, max_region=6, max_new=6):
         for p in rng.choice(pool, size=deg, replace=False):
             add_s.append(int(p)); add_d.append(s + k)
 
+    # which node of the original each node of the candidate is (-1 for the fresh ones)
+    twin = np.concatenate([np.arange(s), np.full(r, -1), np.arange(e, n)]).astype(np.int32)
     return {
+        "twin": twin,
         "op": np.concatenate([op[:s], rng.integers(0, T, size=r).astype(np.int32), op[e:]]),
         "shape": np.concatenate([shp[:s], shape_features(rng, r, S, bf16), shp[e:]]),
         "edge_src": np.concatenate([new_src, np.asarray(add_s, dtype=np.int32)]).astype(np.int32),
@@ -204,7 +207,17 @@ def flatten(graphs, env_off, A_max, mask=None):
         for e in range(num_envs):
             mask[e, : env_off[e + 1] - env_off[e] - 1] = 1
     S = graphs[0]["shape"].shape[1]
+    # base_id: packed id of the current-graph node a candidate node was copied from (-1: none)
+    node_off = np.concatenate([[0], np.cumsum([len(g["op"]) for g in graphs])])
+    base_id = np.full(int(node_off[-1]), -1, dtype=np.int32)
+    for e in range(num_envs):
+        cur = int(env_off[e])
+        for gi in range(cur + 1, int(env_off[e + 1])):
+            tw = graphs[gi].get("twin")
+            if tw is not None:
+                base_id[node_off[gi]:node_off[gi + 1]] = np.where(tw >= 0, tw + node_off[cur], -1)
     return {
+        "base_id": base_id,
         "num_graphs": len(graphs),
         "n_nodes": np.array([len(g["op"]) for g in graphs], dtype=np.int32),
         "n_edges": np.array([len(g["edge_src"]) for g in graphs], dtype=np.int32),
