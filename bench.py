@@ -194,6 +194,7 @@ def main():
     ap.add_argument("--envs", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-delta", action="store_true")
     args = ap.parse_args()
     cfg_id = args.config
     rank, local_rank, world = rank_info()
@@ -271,6 +272,28 @@ def main():
     launches = xrl.xrl_launch_counts(agent.ctx)
     status = agent.device_status()
     assert status == 0, f"device status {status}"
+
+    # ---- delta encoding of the candidates (same outputs, work only where a rewrite can reach) --------
+    delta = None
+    if not args.no_delta and cfg_id != 1:
+        base_d = torch.from_numpy(batch["base_id"]).cuda()
+        for i in range(3):
+            agent.step(dev, mask_d, sample=True, seed=cfg_id, step=i, base_id=base_d)
+        torch.cuda.synchronize()
+        xrl.xrl_profile(agent.ctx, True)
+        barrier()
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record(stream)
+        for i in range(args.steps):
+            agent.step(dev, mask_d, sample=True, seed=cfg_id, step=warmup + i, base_id=base_d)
+        d1.record(stream)
+        barrier()
+        dprof = xrl.xrl_profile_read(agent.ctx)
+        xrl.xrl_profile(agent.ctx, False)
+        assert agent.device_status() == 0
+        dms = d0.elapsed_time(d1) / args.steps
+        delta = {"ms_per_step": dms, "rows_per_layer": xrl.xrl_delta_rows(agent.ctx, m["L"]),
+                 "kernel_ms_per_step": {f: round(v["ms"] / args.steps, 4) for f, v in dprof.items()}}
 
     # ---- end to end: host buffers in, results out, through the public call ---------------------------
     e2e = None
@@ -360,6 +383,13 @@ def main():
         line["e2e"] = {"value": tot_graphs / e2e["s_per_step"], "unit": "graphs/s",
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                        "ms_per_step": e2e["s_per_step"] * 1e3}
+    if delta:
+        if world > 1:
+            delta["ms_per_step"] = reduce_over_ranks(delta["ms_per_step"], 0, 0, 0, dist, "cuda")[0]
+        delta["value"] = tot_graphs / (delta["ms_per_step"] * 1e-3)
+        delta["unit"] = "graphs/s"
+        delta["note"] = "xrl_encode_delta: same outputs, candidates reuse the current graph's unchanged rows"
+        line["delta"] = delta
     if cpu:
         line["cpu_baseline"] = cpu
     print(json.dumps(line))

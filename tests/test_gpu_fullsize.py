@@ -11,7 +11,7 @@ import gpu_util
 pytestmark = pytest.mark.gpu
 
 
-def _run_full(batch, blob, seed, step):
+def _run_full(batch, blob, seed, step, delta=False):
     import torch
     import paper_2304_14698_b200 as xrl
     ag = gpu_util.make_agent(batch)
@@ -24,7 +24,8 @@ def _run_full(batch, blob, seed, step):
         dev["edge_src"] = torch.from_numpy(batch["edge_src"]).cuda()
         dev["edge_dst"] = torch.from_numpy(batch["edge_dst"]).cuda()
         mask = torch.from_numpy(batch["mask"]).cuda()
-        out = ag.step(dev, mask, sample=True, seed=seed, step=step)
+        bid = torch.from_numpy(batch["base_id"]).cuda() if delta else None
+        out = ag.step(dev, mask, sample=True, seed=seed, step=step, base_id=bid)
         torch.cuda.synchronize()
         res = {k: v.cpu().numpy() for k, v in out.items()}
         res["status"] = ag.device_status()
@@ -34,11 +35,11 @@ def _run_full(batch, blob, seed, step):
         ag.close()
 
 
-def _check(xo, cfg_id, n_sample):
+def _check(xo, cfg_id, n_sample, delta=False):
     batch = configs.make_batch(cfg_id)
     m = batch["model"]
     blob, _ = gpu_util.default_weights(batch, 1000 + cfg_id)
-    got = _run_full(batch, blob, seed=cfg_id, step=3)
+    got = _run_full(batch, blob, seed=cfg_id, step=3, delta=delta)
     assert got["status"] == 0
 
     st, packed = xo.pack(batch)
@@ -83,6 +84,14 @@ def test_large_step_full_size(xo):
 
 def test_rollout_batch_full_size(xo):
     _check(xo, 5, 6)
+
+
+def test_large_step_full_size_delta_encoding(xo):
+    _check(xo, 4, 6, delta=True)
+
+
+def test_rollout_batch_full_size_delta_encoding(xo):
+    _check(xo, 5, 6, delta=True)
 
 
 def test_cnn_step_full_size_every_output(xo):
