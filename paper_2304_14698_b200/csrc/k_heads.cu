@@ -94,76 +94,64 @@ k_readout(const T* __restrict__ h, const int32_t* __restrict__ chunk_row0,
 }
 
 // ---- Eq. 8: emb_g = ReLU(Wg^T [ sum of the graph's chunk sums | g0_g ] + bg) -------------------
-// Sum of one graph's partial rows: warp w adds slots first + w, first + w + 8, ... (32 consecutive
-// columns per load), the eight warp sums are then added in warp order.  `extra` (or -1) is one more slot,
-// taken first by warp 0.  Fixed order, so reproducible.
-__device__ void sum_slots(const float* __restrict__ partial, int32_t extra, int32_t first, int32_t last,
-                          float* __restrict__ out, int H, float* red /* [8][H] */) {
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  float acc[16];                                   // H <= 512: up to 16 columns per lane
-#pragma unroll
-  for (int t = 0; t < 16; ++t) acc[t] = 0.f;
-  if (w == 0 && extra >= 0) {
-#pragma unroll
-    for (int t = 0; t < 16; ++t)
-      if (lane + 32 * t < H) acc[t] += partial[size_t(extra) * H + lane + 32 * t];
-  }
-  for (int32_t sl = first + w; sl <= last; sl += 8) {
-#pragma unroll
-    for (int t = 0; t < 16; ++t)
-      if (lane + 32 * t < H) acc[t] += partial[size_t(sl) * H + lane + 32 * t];
-  }
-#pragma unroll
-  for (int t = 0; t < 16; ++t)
-    if (lane + 32 * t < H) red[w * H + lane + 32 * t] = acc[t];
-  __syncthreads();
-  for (int c = threadIdx.x; c < H; c += blockDim.x) {
-    float sres = 0.f;
-    for (int q = 0; q < 8; ++q) sres += red[q * H + c];
-    out[c] = sres;
-  }
-}
-
-// per-graph readout sums r[B][H] from the chunk sums of k_readout
+// GB graphs per CTA: sums of the graphs' partials into shared memory, then the dense map.
 __global__ void __launch_bounds__(256)
-k_sum_chunks(const float* __restrict__ partial, const int32_t* __restrict__ graph_chunk_off,
-             float* __restrict__ r, int H) {
-  extern __shared__ float red[];
-  const int32_t g = blockIdx.x;
-  sum_slots(partial, -1, graph_chunk_off[g], graph_chunk_off[g + 1] - 1, r + size_t(g) * H, H, red);
-}
-
-// per-graph readout sums from the partial sums written by the aggregate kernel fused with the readout:
-// the partial of the block in which the graph starts (if it does not start at the block's first row),
-// then the partials of the following 32-row blocks whose first row belongs to the graph.
-__global__ void __launch_bounds__(256)
-k_sum_blocks(const float* __restrict__ partial, const int32_t* __restrict__ node_off, int32_t nblocks,
-             float* __restrict__ r, int H) {
-  extern __shared__ float red[];
-  const int32_t g = blockIdx.x;
-  const int32_t start = node_off[g], end = node_off[g + 1];
-  int32_t extra = -1, b0 = 0, b1 = -1;
-  if (end > start) {
-    b0 = start >> 5;
-    if (start & 31) { extra = nblocks + g; ++b0; }
-    b1 = (end - 1) >> 5;
-  }
-  sum_slots(partial, extra, b0, b1, r + size_t(g) * H, H, red);
-}
-
-// Eq. 8: emb_g = ReLU(Wg^T [ r_g | g0_g ] + bg), GB graphs per CTA
-__global__ void __launch_bounds__(256)
-k_global_update(const float* __restrict__ r, const float* __restrict__ g0, const float* __restrict__ Wg,
+k_global_update(const float* __restrict__ partial, const int32_t* __restrict__ graph_chunk_off,
+                const float* __restrict__ g0, const float* __restrict__ Wg,
                 const float* __restrict__ bg, float* __restrict__ emb, int H, int Dg, int32_t B) {
   extern __shared__ float u[];                   // [GB][H + Dg]
   const int xs = H + Dg;
   const int32_t gb = blockIdx.x * GB;
-  for (int t = threadIdx.x; t < GB * xs; t += blockDim.x) {
-    const int q = t / xs, k = t - q * xs;
+  for (int q = 0; q < GB; ++q) {
     const int32_t g = gb + q;
-    float v = 0.f;
-    if (g < B) v = (k < H) ? r[size_t(g) * H + k] : (g0 ? g0[size_t(g) * Dg + (k - H)] : 0.f);
-    u[t] = v;
+    const bool live = g < B;
+    const int32_t c0 = live ? graph_chunk_off[g] : 0, c1 = live ? graph_chunk_off[g + 1] : 0;
+    for (int c = threadIdx.x; c < H; c += blockDim.x) {
+      float s = 0.f;
+      for (int32_t ch = c0; ch < c1; ++ch) s += partial[size_t(ch) * H + c];
+      u[q * xs + c] = s;
+    }
+    for (int t = threadIdx.x; t < Dg; t += blockDim.x)
+      u[q * xs + H + t] = (live && g0) ? g0[size_t(g) * Dg + t] : 0.f;
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    float acc[GB];
+#pragma unroll
+    for (int q = 0; q < GB; ++q) acc[q] = bg[c];
+    column_dot_multi(u, xs, xs, Wg, H, c, acc);
+#pragma unroll
+    for (int q = 0; q < GB; ++q)
+      if (gb + q < B) emb[size_t(gb + q) * H + c] = fmaxf(acc[q], 0.f);
+  }
+}
+
+// Eq. 8 from the partial sums written by the aggregate kernel fused with the readout: per graph, the
+// partial of the block in which the graph starts (if it does not start at the block's first row), then
+// the partials of the following 32-row blocks whose first row belongs to the graph, in order.
+__global__ void __launch_bounds__(256)
+k_global_update_blocks(const float* __restrict__ partial, const int32_t* __restrict__ node_off,
+                       int32_t nblocks, const float* __restrict__ g0, const float* __restrict__ Wg,
+                       const float* __restrict__ bg, float* __restrict__ emb, int H, int Dg, int32_t B) {
+  extern __shared__ float u[];                   // [GB][H + Dg]
+  const int xs = H + Dg;
+  const int32_t gb = blockIdx.x * GB;
+  for (int q = 0; q < GB; ++q) {
+    const int32_t g = gb + q;
+    const bool live = g < B;
+    const int32_t start = live ? node_off[g] : 0, end = live ? node_off[g + 1] : 0;
+    for (int c = threadIdx.x; c < H; c += blockDim.x) {
+      float s = 0.f;
+      if (end > start) {
+        int32_t b0 = start >> 5;
+        if (start & 31) { s += partial[size_t(nblocks + g) * H + c]; ++b0; }
+        const int32_t b1 = (end - 1) >> 5;
+        for (int32_t b = b0; b <= b1; ++b) s += partial[size_t(b) * H + c];
+      }
+      u[q * xs + c] = s;
+    }
+    for (int t = threadIdx.x; t < Dg; t += blockDim.x)
+      u[q * xs + H + t] = (live && g0) ? g0[size_t(g) * Dg + t] : 0.f;
   }
   __syncthreads();
   for (int c = threadIdx.x; c < H; c += blockDim.x) {
@@ -450,23 +438,19 @@ int launch_readout(const Dims& d, const void* h, const int32_t* chunk_row0, cons
 }
 
 int launch_global_update(const Dims& d, const float* partial, const int32_t* graph_chunk_off,
-                         const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st,
-                         float* r_ws) {
+                         const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st) {
   if (B <= 0) return 0;
-  k_sum_chunks<<<B, 256, sizeof(float) * 8 * size_t(d.H), st>>>(partial, graph_chunk_off, r_ws, d.H);
   k_global_update<<<(B + GB - 1) / GB, 256, sizeof(float) * size_t(GB) * size_t(d.H + d.Dg), st>>>(
-      r_ws, g0, w.Wg, w.bg, emb, d.H, d.Dg, B);
-  return 2;
+      partial, graph_chunk_off, g0, w.Wg, w.bg, emb, d.H, d.Dg, B);
+  return 1;
 }
 
 int launch_global_update_blocks(const Dims& d, const float* partial, const int32_t* node_off, int32_t nblocks,
-                                const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st,
-                                float* r_ws) {
+                                const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st) {
   if (B <= 0) return 0;
-  k_sum_blocks<<<B, 256, sizeof(float) * 8 * size_t(d.H), st>>>(partial, node_off, nblocks, r_ws, d.H);
-  k_global_update<<<(B + GB - 1) / GB, 256, sizeof(float) * size_t(GB) * size_t(d.H + d.Dg), st>>>(
-      r_ws, g0, w.Wg, w.bg, emb, d.H, d.Dg, B);
-  return 2;
+  k_global_update_blocks<<<(B + GB - 1) / GB, 256, sizeof(float) * size_t(GB) * size_t(d.H + d.Dg), st>>>(
+      partial, node_off, nblocks, g0, w.Wg, w.bg, emb, d.H, d.Dg, B);
+  return 1;
 }
 
 int launch_heads(const Dims& d, const DevWeights& w, const float* emb, const int32_t* env_off,

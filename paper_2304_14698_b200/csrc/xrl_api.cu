@@ -73,7 +73,7 @@ struct xrl_ctx {
   DeviceBuf w_f32;          // the fp32 blob
   DeviceBuf w_store;        // storage-type copies of W0 and the layer matrices (+ transposes)
   DevWeights dw;
-  DeviceBuf h, Z, scores, partial, logits, status, rsum;
+  DeviceBuf h, Z, scores, partial, logits, status;
   int32_t max_chunks = 0;
   int64_t launches_pack = 0, launches_encode = 0, launches_heads = 0;
   // delta encoding workspace (allocated on the first xrl_encode_delta)
@@ -455,7 +455,6 @@ xrl_status xrl_create(const xrl_model_config* cfg, int32_t device, xrl_ctx** out
   }
   A(ctx->logits, 4 * (size_t(cfg->max_graphs) + size_t(cfg->max_envs) * H));   // logits, then candidate sums
   A(ctx->status, 4);
-  A(ctx->rsum, 4 * size_t(cfg->max_graphs) * H);
   if (e == cudaSuccess) e = cudaMemset(ctx->status.p, 0, 4);
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -471,7 +470,7 @@ void xrl_destroy(xrl_ctx* ctx) {
   cudaSetDevice(ctx->device);
   cudaDeviceSynchronize();
   DeviceBuf* bufs[] = {&ctx->w0ext, &ctx->w_f32, &ctx->w_store, &ctx->h, &ctx->Z, &ctx->scores,
-                       &ctx->partial, &ctx->logits, &ctx->status, &ctx->rsum};
+                       &ctx->partial, &ctx->logits, &ctx->status};
   for (DeviceBuf* d : bufs) d->release();
   ctx->prof.release();
   ctx->dl_ints.release(); ctx->dl_col.release(); ctx->dl_scan.release();
@@ -600,11 +599,10 @@ xrl_status xrl_encode(xrl_ctx* ctx, const xrl_batch* b, const float* g0, float* 
   slot = ctx->prof.begin(st);
   if (fused)
     k = launch_global_update_blocks(ctx->dims, ctx->partial.as<float>(), b->node_off.as<int32_t>(),
-                                    aggregate_readout_blocks(b->N), g0, ctx->dw, graph_emb, b->B, st,
-                                    ctx->rsum.as<float>());
+                                    aggregate_readout_blocks(b->N), g0, ctx->dw, graph_emb, b->B, st);
   else
     k = launch_global_update(ctx->dims, ctx->partial.as<float>(), b->d_graph_chunk_off, g0, ctx->dw,
-                             graph_emb, b->B, st, ctx->rsum.as<float>());
+                             graph_emb, b->B, st);
   ctx->prof.end(FAM_HEADS, slot, k, st);
   n += k;
   ctx->launches_encode = n;
@@ -721,8 +719,7 @@ xrl_status xrl_encode_delta(xrl_ctx* ctx, const xrl_batch* b, const int32_t* bas
   pf.end(FAM_READOUT, slot, k, st);
   n_launch += k;
   slot = pf.begin(st);
-  k = launch_global_update(d, ctx->partial.as<float>(), b->d_graph_chunk_off, g0, ctx->dw, graph_emb, b->B, st,
-                           ctx->rsum.as<float>());
+  k = launch_global_update(d, ctx->partial.as<float>(), b->d_graph_chunk_off, g0, ctx->dw, graph_emb, b->B, st);
   pf.end(FAM_HEADS, slot, k, st);
   n_launch += k;
   ctx->launches_encode = n_launch;

@@ -130,8 +130,7 @@ int launch_aggregate_tma(const Dims& d, const int32_t* rowptr, const int32_t* co
 int64_t aggregate_readout_slots(int64_t rows, int64_t B);
 int32_t aggregate_readout_blocks(int64_t rows);
 int launch_global_update_blocks(const Dims& d, const float* partial, const int32_t* node_off, int32_t nblocks,
-                                const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st,
-                         float* r_ws /* [B x H] scratch */);
+                                const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st);
 int launch_readout(const Dims& d, const void* h, const int32_t* chunk_row0, const int32_t* chunk_row1,
                    int32_t chunk_begin, int32_t chunk_end, float* partial, int32_t win_base,
                    cudaStream_t st, const int32_t* remap = nullptr);
@@ -154,8 +153,7 @@ int launch_delta_fill(const DeltaIn& in, int32_t n, const int32_t* list, const i
 int launch_delta_remap(int32_t N, const int32_t* flag, const int32_t* rank, const int32_t* base,
                        int32_t* remap, cudaStream_t st);
 int launch_global_update(const Dims& d, const float* partial, const int32_t* graph_chunk_off,
-                         const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st,
-                         float* r_ws /* [B x H] scratch */);
+                         const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st);
 int launch_heads(const Dims& d, const DevWeights& w, const float* emb, const int32_t* env_off,
                  const uint8_t* mask, int32_t B, int32_t num_envs, float* logit_ws, float* probs,
                  float* value, int32_t* action, uint64_t seed, uint64_t step, int32_t* status,
