@@ -26,28 +26,6 @@ __device__ __forceinline__ float column_dot(const float* x, int in, const float*
   return acc;
 }
 
-// The same for GB input vectors x[g][0..in) (row stride xs) at once: each weight is loaded once and
-// used GB times (a CTA handles GB graphs, so the weight matrix is read GB times less often).
-constexpr int GB = 8;
-__device__ __forceinline__ void column_dot_multi(const float* x, int xs, int in, const float* __restrict__ W,
-                                                 int ld, int c, float (&acc)[GB]) {
-  int k = 0;
-  for (; k + 4 <= in; k += 4) {
-    float w[4];
-#pragma unroll
-    for (int t = 0; t < 4; ++t) w[t] = __ldg(W + size_t(k + t) * ld + c);
-#pragma unroll
-    for (int t = 0; t < 4; ++t)
-#pragma unroll
-      for (int g = 0; g < GB; ++g) acc[g] = fmaf(x[g * xs + k + t], w[t], acc[g]);
-  }
-  for (; k < in; ++k) {
-    const float w = __ldg(W + size_t(k) * ld + c);
-#pragma unroll
-    for (int g = 0; g < GB; ++g) acc[g] = fmaf(x[g * xs + k], w, acc[g]);
-  }
-}
-
 // ---- readout, stage 1: column sums of one chunk of consecutive rows of one graph -------------
 template <typename T>
 __global__ void __launch_bounds__(kRoThreads)
@@ -94,35 +72,22 @@ k_readout(const T* __restrict__ h, const int32_t* __restrict__ chunk_row0,
 }
 
 // ---- Eq. 8: emb_g = ReLU(Wg^T [ sum of the graph's chunk sums | g0_g ] + bg) -------------------
-// GB graphs per CTA: sums of the graphs' partials into shared memory, then the dense map.
 __global__ void __launch_bounds__(256)
 k_global_update(const float* __restrict__ partial, const int32_t* __restrict__ graph_chunk_off,
                 const float* __restrict__ g0, const float* __restrict__ Wg,
-                const float* __restrict__ bg, float* __restrict__ emb, int H, int Dg, int32_t B) {
-  extern __shared__ float u[];                   // [GB][H + Dg]
-  const int xs = H + Dg;
-  const int32_t gb = blockIdx.x * GB;
-  for (int q = 0; q < GB; ++q) {
-    const int32_t g = gb + q;
-    const bool live = g < B;
-    const int32_t c0 = live ? graph_chunk_off[g] : 0, c1 = live ? graph_chunk_off[g + 1] : 0;
-    for (int c = threadIdx.x; c < H; c += blockDim.x) {
-      float s = 0.f;
-      for (int32_t ch = c0; ch < c1; ++ch) s += partial[size_t(ch) * H + c];
-      u[q * xs + c] = s;
-    }
-    for (int t = threadIdx.x; t < Dg; t += blockDim.x)
-      u[q * xs + H + t] = (live && g0) ? g0[size_t(g) * Dg + t] : 0.f;
+                const float* __restrict__ bg, float* __restrict__ emb, int H, int Dg) {
+  extern __shared__ float u[];                   // [H + Dg]
+  const int32_t g = blockIdx.x;
+  const int32_t c0 = graph_chunk_off[g], c1 = graph_chunk_off[g + 1];
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    float s = 0.f;
+    for (int32_t ch = c0; ch < c1; ++ch) s += partial[size_t(ch) * H + c];
+    u[c] = s;
   }
+  for (int t = threadIdx.x; t < Dg; t += blockDim.x) u[H + t] = g0 ? g0[size_t(g) * Dg + t] : 0.f;
   __syncthreads();
   for (int c = threadIdx.x; c < H; c += blockDim.x) {
-    float acc[GB];
-#pragma unroll
-    for (int q = 0; q < GB; ++q) acc[q] = bg[c];
-    column_dot_multi(u, xs, xs, Wg, H, c, acc);
-#pragma unroll
-    for (int q = 0; q < GB; ++q)
-      if (gb + q < B) emb[size_t(gb + q) * H + c] = fmaxf(acc[q], 0.f);
+    emb[size_t(g) * H + c] = fmaxf(column_dot(u, H + Dg, Wg, H, c, bg[c]), 0.f);
   }
 }
 
@@ -132,36 +97,24 @@ k_global_update(const float* __restrict__ partial, const int32_t* __restrict__ g
 __global__ void __launch_bounds__(256)
 k_global_update_blocks(const float* __restrict__ partial, const int32_t* __restrict__ node_off,
                        int32_t nblocks, const float* __restrict__ g0, const float* __restrict__ Wg,
-                       const float* __restrict__ bg, float* __restrict__ emb, int H, int Dg, int32_t B) {
-  extern __shared__ float u[];                   // [GB][H + Dg]
-  const int xs = H + Dg;
-  const int32_t gb = blockIdx.x * GB;
-  for (int q = 0; q < GB; ++q) {
-    const int32_t g = gb + q;
-    const bool live = g < B;
-    const int32_t start = live ? node_off[g] : 0, end = live ? node_off[g + 1] : 0;
-    for (int c = threadIdx.x; c < H; c += blockDim.x) {
-      float s = 0.f;
-      if (end > start) {
-        int32_t b0 = start >> 5;
-        if (start & 31) { s += partial[size_t(nblocks + g) * H + c]; ++b0; }
-        const int32_t b1 = (end - 1) >> 5;
-        for (int32_t b = b0; b <= b1; ++b) s += partial[size_t(b) * H + c];
-      }
-      u[q * xs + c] = s;
+                       const float* __restrict__ bg, float* __restrict__ emb, int H, int Dg) {
+  extern __shared__ float u[];                   // [H + Dg]
+  const int32_t g = blockIdx.x;
+  const int32_t start = node_off[g], end = node_off[g + 1];
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    float s = 0.f;
+    if (end > start) {
+      int32_t b0 = start >> 5;
+      if (start & 31) { s += partial[size_t(nblocks + g) * H + c]; ++b0; }
+      const int32_t b1 = (end - 1) >> 5;
+      for (int32_t b = b0; b <= b1; ++b) s += partial[size_t(b) * H + c];
     }
-    for (int t = threadIdx.x; t < Dg; t += blockDim.x)
-      u[q * xs + H + t] = (live && g0) ? g0[size_t(g) * Dg + t] : 0.f;
+    u[c] = s;
   }
+  for (int t = threadIdx.x; t < Dg; t += blockDim.x) u[H + t] = g0 ? g0[size_t(g) * Dg + t] : 0.f;
   __syncthreads();
   for (int c = threadIdx.x; c < H; c += blockDim.x) {
-    float acc[GB];
-#pragma unroll
-    for (int q = 0; q < GB; ++q) acc[q] = bg[c];
-    column_dot_multi(u, xs, xs, Wg, H, c, acc);
-#pragma unroll
-    for (int q = 0; q < GB; ++q)
-      if (gb + q < B) emb[size_t(gb + q) * H + c] = fmaxf(acc[q], 0.f);
+    emb[size_t(g) * H + c] = fmaxf(column_dot(u, H + Dg, Wg, H, c, bg[c]), 0.f);
   }
 }
 
@@ -194,33 +147,15 @@ __device__ float mlp_scalar(const float* x, int in, int hid, const float* __rest
 __global__ void __launch_bounds__(256)
 k_policy_logit(const float* __restrict__ emb, const float* __restrict__ W1, const float* __restrict__ b1,
                const float* __restrict__ w2, const float* __restrict__ b2, float* __restrict__ logit,
-               int H, int Hm, int32_t B) {
-  extern __shared__ float sm[];                  // [GB][H] + [blockDim]
+               int H, int Hm) {
+  extern __shared__ float sm[];                  // [H] + [blockDim]
   float* x = sm;
-  float* scratch = sm + GB * H;
-  const int32_t gb = blockIdx.x * GB;
-  for (int t = threadIdx.x; t < GB * H; t += blockDim.x) {
-    const int q = t / H;
-    x[t] = (gb + q < B) ? emb[size_t(gb) * H + t] : 0.f;
-  }
+  float* scratch = sm + H;
+  const int32_t g = blockIdx.x;
+  for (int c = threadIdx.x; c < H; c += blockDim.x) x[c] = emb[size_t(g) * H + c];
   __syncthreads();
-  float contrib[GB];
-#pragma unroll
-  for (int q = 0; q < GB; ++q) contrib[q] = 0.f;
-  for (int c = threadIdx.x; c < Hm; c += blockDim.x) {
-    float acc[GB];
-#pragma unroll
-    for (int q = 0; q < GB; ++q) acc[q] = b1[c];
-    column_dot_multi(x, H, H, W1, Hm, c, acc);
-    const float wc = w2[c];
-#pragma unroll
-    for (int q = 0; q < GB; ++q) contrib[q] += fmaxf(acc[q], 0.f) * wc;
-  }
-#pragma unroll
-  for (int q = 0; q < GB; ++q) {
-    const float v = block_sum(contrib[q], scratch) + b2[0];
-    if (threadIdx.x == 0 && gb + q < B) logit[gb + q] = v;
-  }
+  const float v = mlp_scalar(x, H, Hm, W1, b1, w2, b2, scratch);
+  if (threadIdx.x == 0) logit[g] = v;
 }
 
 // ---- Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) -----------------------------------------
@@ -440,16 +375,16 @@ int launch_readout(const Dims& d, const void* h, const int32_t* chunk_row0, cons
 int launch_global_update(const Dims& d, const float* partial, const int32_t* graph_chunk_off,
                          const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st) {
   if (B <= 0) return 0;
-  k_global_update<<<(B + GB - 1) / GB, 256, sizeof(float) * size_t(GB) * size_t(d.H + d.Dg), st>>>(
-      partial, graph_chunk_off, g0, w.Wg, w.bg, emb, d.H, d.Dg, B);
+  k_global_update<<<B, 256, sizeof(float) * size_t(d.H + d.Dg), st>>>(partial, graph_chunk_off, g0,
+                                                                      w.Wg, w.bg, emb, d.H, d.Dg);
   return 1;
 }
 
 int launch_global_update_blocks(const Dims& d, const float* partial, const int32_t* node_off, int32_t nblocks,
                                 const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st) {
   if (B <= 0) return 0;
-  k_global_update_blocks<<<(B + GB - 1) / GB, 256, sizeof(float) * size_t(GB) * size_t(d.H + d.Dg), st>>>(
-      partial, node_off, nblocks, g0, w.Wg, w.bg, emb, d.H, d.Dg, B);
+  k_global_update_blocks<<<B, 256, sizeof(float) * size_t(d.H + d.Dg), st>>>(partial, node_off, nblocks, g0,
+                                                                             w.Wg, w.bg, emb, d.H, d.Dg);
   return 1;
 }
 
@@ -458,8 +393,8 @@ int launch_heads(const Dims& d, const DevWeights& w, const float* emb, const int
                  float* value, int32_t* action, uint64_t seed, uint64_t step, int32_t* status,
                  cudaStream_t st) {
   if (B <= 0 || num_envs <= 0) return 0;
-  k_policy_logit<<<(B + GB - 1) / GB, 256, sizeof(float) * size_t(GB * d.H + 256), st>>>(
-      emb, w.pW1, w.pb1, w.pw2, w.pb2, logit_ws, d.H, d.Hm, B);
+  k_policy_logit<<<B, 256, sizeof(float) * size_t(d.H + 256), st>>>(emb, w.pW1, w.pb1, w.pw2, w.pb2,
+                                                                    logit_ws, d.H, d.Hm);
   float* cand_sum = logit_ws + B;                 // [num_envs x H], behind the per-graph logits
   k_candidate_sum<<<dim3(num_envs, (d.H + 31) / 32), 1024, 0, st>>>(emb, env_off, mask, cand_sum, d.H, d.A);
   const int nt = pow2_threads(d.H > d.A + 1 ? d.H : d.A + 1);
