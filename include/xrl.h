@@ -166,7 +166,7 @@ xrl_status xrl_encode(xrl_ctx* ctx, const xrl_batch* batch, const float* g0, flo
  *            verifies operator, shape features and producer lists on the device and recomputes whatever
  *            does not check out, so a wrong hint costs time, never correctness.  Entries of current-graph
  *            nodes are ignored.
- * The call synchronises `stream` once per layer (it reads the number of listed rows back).
+ * The call synchronises `stream` once (it reads the number of rows per layer back).
  * xrl_delta_rows reports, for the last call, the rows computed at Eq. 6 and after each attention layer
  * (HOST int64 [count], count <= L + 1). */
 xrl_status xrl_encode_delta(xrl_ctx* ctx, const xrl_batch* batch, const int32_t* base_id, const float* g0,

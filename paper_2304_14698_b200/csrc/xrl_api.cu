@@ -619,19 +619,19 @@ xrl_status xrl_encode_delta(xrl_ctx* ctx, const xrl_batch* b, const int32_t* bas
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t Ncap = size_t(ctx->cfg.max_nodes) + 1, Ecap = size_t(ctx->cfg.max_edges) + 1;
   if (ctx->dl_ints.p == nullptr) {
-    XRL_ALLOC(ctx->dl_ints.alloc(4 * 11 * Ncap));
+    XRL_ALLOC(ctx->dl_ints.alloc(4 * (10 * Ncap + 256)));
     XRL_ALLOC(ctx->dl_col.alloc(4 * Ecap));
     XRL_ALLOC(ctx->dl_scan.alloc(4 * scan_workspace_ints(int64_t(Ncap))));
-    XRL_ALLOC(cudaHostAlloc(reinterpret_cast<void**>(&ctx->dl_host), 4 * 4, cudaHostAllocDefault));
+    XRL_ALLOC(cudaHostAlloc(reinterpret_cast<void**>(&ctx->dl_host), 4 * 128, cudaHostAllocDefault));
   }
   int32_t* I = ctx->dl_ints.as<int32_t>();
-  int32_t *valid = I, *base = I + Ncap, *flag_prev = I + 2 * Ncap, *flag_cur = I + 3 * Ncap,
-          *rank_prev = I + 4 * Ncap, *rank_cur = I + 5 * Ncap, *list = I + 6 * Ncap, *deg = I + 7 * Ncap,
-          *rowptr_c = I + 8 * Ncap, *self_c = I + 9 * Ncap, *remap = I + 10 * Ncap;
+  int32_t *valid = I, *base = I + Ncap, *level_a = I + 2 * Ncap, *level_b = I + 3 * Ncap,
+          *rank = I + 4 * Ncap, *list = I + 5 * Ncap, *deg = I + 6 * Ncap, *rowptr_c = I + 7 * Ncap,
+          *self_c = I + 8 * Ncap, *remap = I + 9 * Ncap, *counts = I + 10 * Ncap, *cursor = counts + 128;
   int32_t* col_c = ctx->dl_col.as<int32_t>();
   int32_t* scan_ws = ctx->dl_scan.as<int32_t>();
   const Dims& d = ctx->dims;
-  const int N = b->N;
+  const int N = b->N, L = d.L;
 
   DeltaIn in;
   in.N = N; in.E = b->E;
@@ -641,29 +641,37 @@ xrl_status xrl_encode_delta(xrl_ctx* ctx, const xrl_batch* b, const int32_t* bas
   in.shape = b->shape.p; in.shape_bytes = int(storage_bytes(d.dtype)) * kS;
   in.base_id = base_id;
 
-  // rows of rank[N] read back: the launches of a layer are sized by its number of dirty rows
-  auto count_of = [&](const int32_t* rank, int32_t* out) -> xrl_status {
-    XRL_CUDA(cudaMemcpyAsync(ctx->dl_host, rank + N, 4, cudaMemcpyDeviceToHost, st));
-    XRL_CUDA(cudaStreamSynchronize(st));
-    *out = ctx->dl_host[0];
-    return XRL_OK;
-  };
+  // ---- levels, dense rows (ordered by level) and the row list ---------------------------------------
   Profiler& pf = ctx->prof;
   int n_launch = 0;
   size_t slot = pf.begin(st);
-  int k = launch_delta_init(in, valid, base, flag_prev, st);
-  k += launch_exclusive_scan(flag_prev, rank_prev, N, scan_ws, st);
-  k += launch_delta_list(N, flag_prev, rank_prev, list, st);
+  int k = launch_delta_level0(in, valid, base, level_a, st);
+  int32_t* level = level_a;
+  int32_t* other = level_b;
+  for (int t = 1; t <= L; ++t) {
+    k += launch_delta_propagate(in, t, level, other, st);
+    int32_t* tmp = level; level = other; other = tmp;
+  }
+  k += launch_delta_count(N, L, level, counts, cursor, st);
+  k += launch_delta_assign(N, L, level, counts, cursor, rank, list, st);
   pf.end(FAM_PACK, slot, k, st);
   n_launch += k;
-  int32_t n_prev = 0;
-  xrl_status rs = count_of(rank_prev, &n_prev);
-  if (rs != XRL_OK) return rs;
-  ctx->delta_rows[0] = n_prev;
-
-  // Eq. 6 on the listed rows, written densely
+  // the only read-back: rows per level, which size the launches of every layer
+  XRL_CUDA(cudaMemcpyAsync(ctx->dl_host, counts, 4 * size_t(L + 1), cudaMemcpyDeviceToHost, st));
+  XRL_CUDA(cudaStreamSynchronize(st));
+  int32_t n_at[66];
+  int32_t run = 0;
+  for (int t = 0; t <= L; ++t) { run += ctx->dl_host[t]; n_at[t] = run; ctx->delta_rows[t] = run; }
+  const int32_t n_all = n_at[L];
   slot = pf.begin(st);
-  const Window w0{0, n_prev, 0};
+  k = launch_delta_degrees(in, n_all, list, deg, st);
+  k += launch_exclusive_scan(deg, rowptr_c, n_all, scan_ws, st);
+  pf.end(FAM_PACK, slot, k, st);
+  n_launch += k;
+
+  // Eq. 6 on the level-0 rows, written densely
+  slot = pf.begin(st);
+  const Window w0{0, n_at[0], 0};
   k = -1;
   if (ctx->use_umma_embed)
     k = launch_embed_umma(d, in.rowptr, in.col, in.op, b->shape.p, ctx->w0ext.p, ctx->h.p, w0,
@@ -672,8 +680,9 @@ xrl_status xrl_encode_delta(xrl_ctx* ctx, const xrl_batch* b, const int32_t* bas
   pf.end(FAM_EMBED, slot, k, st);
   n_launch += k;
 
-  for (int l = 0; l < d.L; ++l) {
-    // transform of the rows recomputed so far (dense)
+  for (int l = 0; l < L; ++l) {
+    const int32_t n_prev = n_at[l], n_cur = n_at[l + 1];
+    // transform of the rows reached so far (dense)
     slot = pf.begin(st);
     const Window wp{0, n_prev, 0};
     k = -1;
@@ -683,37 +692,21 @@ xrl_status xrl_encode_delta(xrl_ctx* ctx, const xrl_batch* b, const int32_t* bas
     if (k < 0) k = launch_xform_simt(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), wp, st);
     pf.end(FAM_XFORM, slot, k, st);
     n_launch += k;
-    // rows reached by the change after this layer, their list and compact CSR
+    // compact CSR of the rows this layer reaches: producers and the row's own vector by dense row
     slot = pf.begin(st);
-    k = launch_delta_propagate(in, flag_prev, flag_cur, st);
-    k += launch_exclusive_scan(flag_cur, rank_cur, N, scan_ws, st);
-    k += launch_delta_list(N, flag_cur, rank_cur, list, st);
+    k = launch_delta_fill(in, n_cur, l + 1, list, rowptr_c, level, rank, base, col_c, self_c, st);
     pf.end(FAM_PACK, slot, k, st);
     n_launch += k;
-    int32_t n_cur = 0;
-    rs = count_of(rank_cur, &n_cur);
-    if (rs != XRL_OK) return rs;
-    ctx->delta_rows[l + 1] = n_cur;
-    slot = pf.begin(st);
-    k = launch_delta_degrees(in, n_cur, list, deg, st);
-    k += launch_exclusive_scan(deg, rowptr_c, n_cur, scan_ws, st);
-    k += launch_delta_fill(in, n_cur, list, rowptr_c, flag_prev, rank_prev, base, col_c, self_c, st);
-    pf.end(FAM_PACK, slot, k, st);
-    n_launch += k;
-    // aggregate on the compact CSR: producers and the row's own vector come from the dense Z buffer
     slot = pf.begin(st);
     const Window wc{0, n_cur, 0};
     k = launch_aggregate(d, rowptr_c, col_c, ctx->Z.p, ctx->scores.as<float>(), ctx->dw.layer[l].b, ctx->h.p,
                          wc, n_prev > 0 ? n_prev : 1, ctx->status.as<int32_t>(), st, self_c);
     pf.end(FAM_AGG, slot, k, st);
     n_launch += k;
-    int32_t* t = flag_prev; flag_prev = flag_cur; flag_cur = t;
-    t = rank_prev; rank_prev = rank_cur; rank_cur = t;
-    n_prev = n_cur;
   }
   // Eq. 8: every node adds the dense row that holds its features (its own or its base node's)
   slot = pf.begin(st);
-  k = launch_delta_remap(N, flag_prev, rank_prev, base, remap, st);
+  k = launch_delta_remap(N, L, level, rank, base, remap, st);
   k += launch_readout(d, ctx->h.p, b->d_chunk_row0, b->d_chunk_row1, 0, b->num_chunks,
                       ctx->partial.as<float>(), 0, st, remap);
   pf.end(FAM_READOUT, slot, k, st);

@@ -143,14 +143,18 @@ struct DeltaIn {
   int shape_bytes;                 // bytes of one node's shape features
   const int32_t* base_id;          // caller's hint
 };
-int launch_delta_init(const DeltaIn& in, int32_t* valid, int32_t* base, int32_t* flag0, cudaStream_t st);
-int launch_delta_propagate(const DeltaIn& in, const int32_t* flag_in, int32_t* flag_out, cudaStream_t st);
-int launch_delta_list(int32_t N, const int32_t* flag, const int32_t* rank, int32_t* list, cudaStream_t st);
+int launch_delta_level0(const DeltaIn& in, int32_t* valid, int32_t* base, int32_t* level, cudaStream_t st);
+int launch_delta_propagate(const DeltaIn& in, int32_t t, const int32_t* level_in, int32_t* level_out,
+                           cudaStream_t st);
+int launch_delta_count(int32_t N, int32_t L, const int32_t* level, int32_t* counts, int32_t* cursor,
+                       cudaStream_t st);
+int launch_delta_assign(int32_t N, int32_t L, const int32_t* level, const int32_t* counts, int32_t* cursor,
+                        int32_t* rank, int32_t* list, cudaStream_t st);
 int launch_delta_degrees(const DeltaIn& in, int32_t n, const int32_t* list, int32_t* deg, cudaStream_t st);
-int launch_delta_fill(const DeltaIn& in, int32_t n, const int32_t* list, const int32_t* rowptr_c,
-                      const int32_t* flag_prev, const int32_t* rank_prev, const int32_t* base,
-                      int32_t* col_c, int32_t* self_c, cudaStream_t st);
-int launch_delta_remap(int32_t N, const int32_t* flag, const int32_t* rank, const int32_t* base,
+int launch_delta_fill(const DeltaIn& in, int32_t n, int32_t t, const int32_t* list, const int32_t* rowptr_c,
+                      const int32_t* level, const int32_t* rank, const int32_t* base, int32_t* col_c,
+                      int32_t* self_c, cudaStream_t st);
+int launch_delta_remap(int32_t N, int32_t L, const int32_t* level, const int32_t* rank, const int32_t* base,
                        int32_t* remap, cudaStream_t st);
 int launch_global_update(const Dims& d, const float* partial, const int32_t* graph_chunk_off,
                          const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st);
