@@ -105,7 +105,7 @@ xrl_status xrl_weights_size(const xrl_ctx* ctx, size_t* bytes);
  * to bf16 (nearest even) once; everything else stays fp32.  Synchronous. */
 xrl_status xrl_set_weights(xrl_ctx* ctx, const void* host_blob, size_t bytes);
 
-/* ---- (1) packer: Section 3.3.2, "batch them into a meta-graph" -------------------------- */
+/* ---- (1) packer: Section 3.3.2, the current graph and its candidates become one meta-graph ---- */
 
 /* graphs[env_off[e]] is the CURRENT graph of environment e and graphs[env_off[e]+1 ..
  * env_off[e+1]-1] are its candidates in action order.  env_off is HOST, [num_envs + 1],

@@ -7,12 +7,12 @@
 // the benchmark's CPU-baseline leg may load it.
 //
 // What it follows (sections and equations of the X-RLflow paper):
-//   xo_pack          Section 3.3.2  "batch them into a meta-graph"
+//   xo_pack          Section 3.3.2  the current graph and its candidates batched into one meta-graph
 //   xo_encode        Section 3.4    Eq. 6 (node update), Eq. 7 (k graph-attention layers,
 //                                   attention as in the GAT paper it cites), Eq. 8 (global update)
 //   xo_policy_value  Section 3.3.2  two-layer MLP heads, padded action space with a boolean
 //                                   mask, No-Op action; Section 3.3.3 invalid-action masking
-//   xo_sample        Section 3.3.2  "the action sampled from the categorical distribution";
+//   xo_sample        Section 3.3.2  the action is drawn from the categorical distribution;
 //                                   random words from Philox4x32-10 (Salmon et al., SC'11)
 // Readings of what the paper leaves open (activation = ReLU, LeakyReLU slope 0.2 inside the
 // attention score, in-neighbours plus self, heads concatenated, biases, a weight matrix in

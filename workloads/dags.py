@@ -21,7 +21,7 @@ from __future__ import annotations
 
 import numpy as np
 
-# A small operator table (the paper speaks of "around 40" tensor operators).
+# A small operator table (the paper's table has about forty tensor operators, Section 3.3.2).
 OP_INPUT, OP_WEIGHT, OP_MATMUL, OP_ADD, OP_SOFTMAX, OP_LAYERNORM, OP_TRANSPOSE, \
     OP_RESHAPE, OP_SCALE, OP_GELU, OP_CONV, OP_BATCHNORM, OP_RELU, OP_CONCAT, \
     OP_SPLIT, OP_POOL = range(16)
