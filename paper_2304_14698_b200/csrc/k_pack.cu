@@ -200,6 +200,101 @@ k_row_order_long(const int32_t* __restrict__ rowptr, const int2* __restrict__ tm
   }
 }
 
+// ---- one CTA per graph: the whole CSR of a graph built in shared memory ---------------------------
+// For graphs whose counters and edge slots fit in shared memory: in-degrees by shared-memory atomics, a
+// block scan, a scatter of (edge id, producer) pairs into the rows and the per-row rank restore all stay
+// on chip; global memory sees each edge once on the way in and each output once on the way out.  Rows of
+// graph g occupy col[edge_off[g] .. edge_off[g+1]), so no scan over all nodes is needed.
+constexpr int kGraphThreads = 512;
+
+__global__ void __launch_bounds__(kGraphThreads)
+k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ edge_off,
+             const int32_t* __restrict__ op, const int32_t* __restrict__ edge_src,
+             const int32_t* __restrict__ edge_dst, int32_t T, int32_t B, int32_t cap_n,
+             int32_t* __restrict__ seg_id, int32_t* __restrict__ rowptr, int32_t* __restrict__ col,
+             int32_t* status) {
+  extern __shared__ __align__(16) int32_t psm[];
+  int32_t* deg = psm;                         // [cap_n + 1] in-degree, then exclusive row starts
+  int32_t* cur = psm + cap_n + 1;             // [cap_n]     row cursors
+  int32_t* wsum = cur + cap_n;                // [kGraphThreads / 32 + 1]
+  int2* tmp = reinterpret_cast<int2*>(wsum + kGraphThreads / 32 + 3);   // word 2 cap_n + 20: 8-byte aligned
+  const int32_t g = blockIdx.x;
+  const int32_t nb = node_off[g], n = node_off[g + 1] - nb;
+  const int32_t eb = edge_off[g], m = edge_off[g + 1] - eb;
+  const int tid = threadIdx.x;
+
+  for (int32_t i = tid; i < n; i += kGraphThreads) {
+    deg[i] = 0;
+    cur[i] = 0;
+    seg_id[nb + i] = g;
+    const int32_t o = op[nb + i];
+    if (o < 0 || o >= T) raise(status, XRL_ERR_BAD_GRAPH);
+  }
+  __syncthreads();
+  for (int32_t e = tid; e < m; e += kGraphThreads) {
+    const int32_t s = edge_src[eb + e], t = edge_dst[eb + e];
+    if (s < 0 || s >= n || t < 0 || t >= n || s == t) raise(status, XRL_ERR_BAD_GRAPH);
+    else atomicAdd(&deg[t], 1);
+  }
+  __syncthreads();
+  // exclusive scan of deg[0..n): each thread scans a contiguous slice, warp / block offsets on top
+  const int32_t per = (n + kGraphThreads - 1) / kGraphThreads;
+  const int32_t a0 = min(n, tid * per), a1 = min(n, a0 + per);
+  int32_t sum = 0;
+  for (int32_t i = a0; i < a1; ++i) sum += deg[i];
+  int32_t incl = sum;
+  const int lane = tid & 31, wid = tid >> 5;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) wsum[wid] = incl;
+  __syncthreads();
+  int32_t wbase = 0;
+  for (int w = 0; w < wid; ++w) wbase += wsum[w];
+  int32_t run = wbase + incl - sum;
+  for (int32_t i = a0; i < a1; ++i) { const int32_t dgr = deg[i]; deg[i] = run; run += dgr; }
+  if (tid == kGraphThreads - 1) deg[n] = run;          // valid edges of the graph
+  __syncthreads();
+  for (int32_t i = tid; i < n; i += kGraphThreads) rowptr[nb + i] = eb + deg[i];
+  if (g == B - 1 && tid == 0) rowptr[nb + n] = eb + deg[n];
+  // scatter (edge id, global producer) into the rows, slot order as the atomics hand it out
+  for (int32_t e = tid; e < m; e += kGraphThreads) {
+    const int32_t s = edge_src[eb + e], t = edge_dst[eb + e];
+    if (s < 0 || s >= n || t < 0 || t >= n || s == t) continue;
+    tmp[deg[t] + atomicAdd(&cur[t], 1)] = make_int2(e, nb + s);
+  }
+  __syncthreads();
+  // rank of each edge id inside its row restores the input order; short rows by one thread ...
+  for (int32_t i = tid; i < n; i += kGraphThreads) {
+    const int32_t b = deg[i], k = deg[i + 1] - b;
+    if (k == 1) col[eb + b] = tmp[b].y;
+    else if (k > 1 && k <= kShortRow)
+      for (int32_t a = 0; a < k; ++a) {
+        const int2 ea = tmp[b + a];
+        int32_t rank = 0;
+        for (int32_t c = 0; c < k; ++c) rank += (tmp[b + c].x < ea.x) ? 1 : 0;
+        col[eb + b + rank] = ea.y;
+      }
+  }
+  // ... long rows by one warp each
+  for (int32_t i = wid; i < n; i += kGraphThreads / 32) {
+    const int32_t b = deg[i], k = deg[i + 1] - b;
+    if (k <= kShortRow) continue;
+    for (int32_t a = lane; a < k; a += 32) {
+      const int2 ea = tmp[b + a];
+      int32_t rank = 0;
+      for (int32_t c = 0; c < k; ++c) rank += (tmp[b + c].x < ea.x) ? 1 : 0;
+      col[eb + b + rank] = ea.y;
+    }
+  }
+}
+
+size_t pack_graph_smem(int32_t cap_n, int32_t cap_m) {
+  return 4 * size_t(2 * cap_n + 1 + kGraphThreads / 32 + 3) + 8 * size_t(cap_m) + 16;
+}
+
 }  // namespace
 
 int launch_exclusive_scan(const int32_t* in, int32_t* out, int32_t n_in, int32_t* ws, cudaStream_t st) {
@@ -226,6 +321,18 @@ int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cu
   if (in.B > 0) {
     k_graph_envs<<<(in.B + TB - 1) / TB, TB, 0, st>>>(in.env_off, in.num_envs, in.B, out.graph_env);
     ++launches;
+  }
+  // graphs small enough for shared memory: one CTA builds the whole CSR of a graph
+  if (in.B > 0 && in.max_n > 0 && in.max_n <= 16384 && pack_graph_smem(in.max_n, in.max_m) <= 160 * 1024) {
+    static bool attr = false;
+    if (!attr) {
+      cudaFuncSetAttribute(k_pack_graph, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+      attr = true;
+    }
+    k_pack_graph<<<in.B, kGraphThreads, pack_graph_smem(in.max_n, in.max_m), st>>>(
+        out.node_off, out.edge_off, in.op, in.edge_src, in.edge_dst, T, in.B, in.max_n, out.seg_id,
+        out.rowptr, out.col, status);
+    return launches + 1;
   }
   if (in.N > 0) {
     k_node_segments<<<(in.N + TB - 1) / TB, TB, 0, st>>>(out.node_off, in.B, in.N, in.op, T,
@@ -296,9 +403,12 @@ extern "C" xrl_status xrl_pack_csr_static(int32_t device, int32_t num_op_types, 
   for (int32_t e = 0; e < num_envs; ++e)
     if (env_off[e + 1] <= env_off[e]) return XRL_ERR_INVALID_ARG;
   int64_t N = 0, E = 0;
+  int32_t max_n = 0, max_m = 0;
   for (int32_t g = 0; g < num_graphs; ++g) {
     if (n_nodes[g] < 0 || n_edges[g] < 0) return XRL_ERR_INVALID_ARG;
     N += n_nodes[g]; E += n_edges[g];
+    if (n_nodes[g] > max_n) max_n = n_nodes[g];
+    if (n_edges[g] > max_m) max_m = n_edges[g];
   }
   if (N > kStN || E > kStE) return XRL_ERR_CAPACITY;          // beyond the built-in scratch
   if ((N > 0 && (!op || !seg_id)) || (E > 0 && (!edge_src || !edge_dst || !col))) return XRL_ERR_INVALID_ARG;
@@ -330,6 +440,7 @@ extern "C" xrl_status xrl_pack_csr_static(int32_t device, int32_t num_op_types, 
 
   PackIn in;
   in.B = num_graphs; in.num_envs = num_envs; in.N = int32_t(N); in.E = int32_t(E);
+  in.max_n = max_n; in.max_m = max_m;
   in.n_nodes = sc + kOffNn; in.n_edges = sc + kOffNe; in.env_off = sc + kOffEnv;
   in.op = op; in.edge_src = edge_src; in.edge_dst = edge_dst;
   PackOut out;

@@ -212,10 +212,13 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
     if (env_off[e + 1] - env_off[e] - 1 > c.max_actions) return XRL_ERR_CAPACITY;
   }
   int64_t N = 0, E = 0;
+  int32_t max_n = 0, max_m = 0;
   for (int32_t g = 0; g < num_graphs; ++g) {
     const int32_t n = graphs ? graphs[g].num_nodes : n_nodes[g];
     const int32_t m = graphs ? graphs[g].num_edges : n_edges[g];
     if (n < 0 || m < 0) return XRL_ERR_INVALID_ARG;
+    if (n > max_n) max_n = n;
+    if (m > max_m) max_m = m;
     if (graphs && ((n > 0 && (!graphs[g].op || !graphs[g].shape)) ||
                    (m > 0 && (!graphs[g].edge_src || !graphs[g].edge_dst))))
       return XRL_ERR_INVALID_ARG;
@@ -334,6 +337,7 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
 
   PackIn in;
   in.B = num_graphs; in.num_envs = num_envs; in.N = int32_t(N); in.E = int32_t(E);
+  in.max_n = max_n; in.max_m = max_m;
   in.n_nodes = b->d_n_nodes; in.n_edges = b->d_n_edges; in.env_off = b->d_env_off;
   in.op = b->op.as<int32_t>(); in.edge_src = d_src; in.edge_dst = d_dst;
   PackOut po;

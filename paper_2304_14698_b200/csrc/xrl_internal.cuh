@@ -83,6 +83,7 @@ struct Dims {
 // ---- launchers (each returns the number of kernels it launched; errors via cudaGetLastError) --
 struct PackIn {
   int32_t B, num_envs, N, E;
+  int32_t max_n, max_m;                           // largest node / edge count of one graph
   const int32_t *n_nodes, *n_edges, *env_off;     // device copies of the metadata
   const int32_t *op, *edge_src, *edge_dst;        // device
 };
