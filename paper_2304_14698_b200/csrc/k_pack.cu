@@ -231,10 +231,21 @@ k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ e
     if (o < 0 || o >= T) raise(status, XRL_ERR_BAD_GRAPH);
   }
   __syncthreads();
-  for (int32_t e = tid; e < m; e += kGraphThreads) {
-    const int32_t s = edge_src[eb + e], t = edge_dst[eb + e];
-    if (s < 0 || s >= n || t < 0 || t >= n || s == t) raise(status, XRL_ERR_BAD_GRAPH);
-    else atomicAdd(&deg[t], 1);
+  // edges four at a time per thread: the loads of a batch are issued before any of them is used
+  for (int32_t e0 = tid; e0 < m; e0 += 4 * kGraphThreads) {
+    int32_t s[4], t[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int32_t e = e0 + u * kGraphThreads;
+      s[u] = e < m ? __ldg(edge_src + eb + e) : 0;
+      t[u] = e < m ? __ldg(edge_dst + eb + e) : -2;          // -2: no edge here
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (t[u] == -2) continue;
+      if (s[u] < 0 || s[u] >= n || t[u] < 0 || t[u] >= n || s[u] == t[u]) raise(status, XRL_ERR_BAD_GRAPH);
+      else atomicAdd(&deg[t[u]], 1);
+    }
   }
   __syncthreads();
   // exclusive scan of deg[0..n): each thread scans a contiguous slice, warp / block offsets on top
@@ -260,10 +271,19 @@ k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ e
   for (int32_t i = tid; i < n; i += kGraphThreads) rowptr[nb + i] = eb + deg[i];
   if (g == B - 1 && tid == 0) rowptr[nb + n] = eb + deg[n];
   // scatter (edge id, global producer) into the rows, slot order as the atomics hand it out
-  for (int32_t e = tid; e < m; e += kGraphThreads) {
-    const int32_t s = edge_src[eb + e], t = edge_dst[eb + e];
-    if (s < 0 || s >= n || t < 0 || t >= n || s == t) continue;
-    tmp[deg[t] + atomicAdd(&cur[t], 1)] = make_int2(e, nb + s);
+  for (int32_t e0 = tid; e0 < m; e0 += 4 * kGraphThreads) {
+    int32_t s[4], t[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int32_t e = e0 + u * kGraphThreads;
+      s[u] = e < m ? __ldg(edge_src + eb + e) : 0;
+      t[u] = e < m ? __ldg(edge_dst + eb + e) : -2;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (t[u] == -2 || s[u] < 0 || s[u] >= n || t[u] < 0 || t[u] >= n || s[u] == t[u]) continue;
+      tmp[deg[t[u]] + atomicAdd(&cur[t[u]], 1)] = make_int2(e0 + u * kGraphThreads, nb + s[u]);
+    }
   }
   __syncthreads();
   // rank of each edge id inside its row restores the input order; short rows by one thread ...
