@@ -201,9 +201,7 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
 
   // lane 0: hand group `gi` of the current list (list rows item[4 gi .. 4 gi + 3]) to slot `s`
   auto issue = [&](int gi, uint32_t s) {
-    int4 it = *reinterpret_cast<const int4*>(&sm.item[gi * 4]);
-    it.x = it.x < 0 ? ~it.x : it.x; it.y = it.y < 0 ? ~it.y : it.y;      // row starts are stored complemented
-    it.z = it.z < 0 ? ~it.z : it.z; it.w = it.w < 0 ? ~it.w : it.w;
+    const int4 it = *reinterpret_cast<const int4*>(&sm.item[gi * 4]);
     const uint32_t bar = bar_base + 8 * s;
     mbar_expect_tx(bar, GROUP_BYTES);
     tma_gather4(z_base + s * ZG, &map_z, it.x, it.y, it.z, it.w, bar);
@@ -285,18 +283,17 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
         rs += 1;
         continue;
       }
-      // ---- the list: for each row its own index (stored complemented: negative marks a row start),
-      // then its producers', all window-relative ------------------------------------------------------
+      // ---- the list: for each row its own index, then its producers', all window-relative ----------
       __syncwarp();
       const int total = cnt + (sm.rp[rs + cnt] - eb);
       if (lane < cnt) {
         const int e0 = sm.rp[rs + lane] - eb, n = sm.rp[rs + lane + 1] - eb - e0;
         int pos = lane + e0;
-        sm.item[pos++] = ~(self_idx ? __ldg(self_idx + int32_t(r0) + rs + lane)      // where the row's own Z lives
-                                    : int32_t(r0) + rs + lane - win.win_base);
+        sm.item[pos++] = self_idx ? __ldg(self_idx + int32_t(r0) + rs + lane)       // where the row's own Z lives
+                                  : int32_t(r0) + rs + lane - win.win_base;
         for (int t = 0; t < n; ++t) sm.item[pos++] = __ldg(col + eb + e0 + t) - win.win_base;
       }
-      if (lane < 4) sm.item[total + lane] = ~(int32_t(r0) + rs - win.win_base);  // padding: row starts never finished
+      if (lane < 4) sm.item[total + lane] = int32_t(r0) + rs - win.win_base;   // pad the last group
       __syncwarp();
       const int ngroups = (total + 3) >> 2;
       if (lane == 0) {
@@ -304,58 +301,59 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
         for (int gi = 0; gi < min(G, ngroups); ++gi) { issue(gi, s); s = (s + 1 == G) ? 0 : s + 1; }
       }
 
-      // ---- consume group by group; a negative list entry closes the row in progress and opens the next ---
-      int rr = 0;                              // rows of this list finished so far
-      bool open = false;
-      float sd = 0.f, m = 0.f, l = 1.f;
-      F2 acc[NP];
-      auto close_row = [&]() {
-        if (rr < cnt) {                        // padding entries open rows that are never closed for real
-          if (READOUT) {
-            float o[VEC];
-            finish_row_f32<NP>(acc, __fdividef(1.f, l), bs, o);
-            add_row(rs + rr, o);
-          } else {
-            finish_row(h_out + size_t(int32_t(r0) + rs + rr - win.win_base) * H + c0, acc, __fdividef(1.f, l), bs);
-          }
-        }
-        ++rr;
-      };
-      for (int gi = 0; gi < ngroups; ++gi) {
-        if (alive && !wait_all_lanes(bar_base + 8 * slot, par)) alive = false;
-        const int4 it = *reinterpret_cast<const int4*>(&sm.item[gi * 4]);
-        const int32_t flags[4] = {it.x, it.y, it.z, it.w};
-        const uint32_t zp = z_lane + slot * ZG, sp = s_lane + slot * SG;
-#pragma unroll
-        for (int w = 0; w < 4; ++w) {
-          const uint4 raw = lds128(zp + w * 512);
-          const float2 sc = lds64(sp + w * (8 * K));
-          if (flags[w] < 0) {
-            // the row's own vector opens the running softmax: reference exponent = its score, weight 1
-            if (open) close_row();
-            open = true;
-            sd = sc.y;
-            m = lrelu(sc.x + sd);
-            l = 1.f;
-            to_pairs(raw, acc);
-          } else {
-            const float ev = lrelu(sc.x + sd);
-            if (ev > m + 32.f) raise_reference<NP>(ev, m, l, acc);
-            const float p = fast_exp2(ev - m);
-            l += p;
-            F2 z[NP];
-            to_pairs(raw, z);
-            const F2 p2 = make_f2(p, p);
-#pragma unroll
-            for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], p2, z[t2]);
-          }
-        }
-        // group finished: refill its slot with group gi + G, move on
+      // ---- consume: rows in order, vectors in list order ----------------------------------------------
+      int gi = 0, w = 4;                      // current group of the list, vectors left in it
+      uint32_t zp = z_lane + slot * ZG, sp = s_lane + slot * SG;
+      if (!wait_all_lanes(bar_base + 8 * slot, par)) alive = false;
+      // group finished: refill its slot with group gi + G, move on, wait for the next one
+      auto advance = [&]() {
         __syncwarp();
         if (lane == 0 && gi + G < ngroups) issue(gi + G, slot);
+        ++gi;
+        if (++slot == G) { slot = 0; par ^= 1; }
+        zp = z_lane + slot * ZG;
+        sp = s_lane + slot * SG;
+        w = 4;
+        if (gi < ngroups && alive && !wait_all_lanes(bar_base + 8 * slot, par)) alive = false;
+      };
+      for (int rr = 0; rr < cnt; ++rr) {
+        const int n = sm.rp[rs + rr + 1] - sm.rp[rs + rr];
+        // the row's own vector opens the running softmax: reference exponent = its score, weight 1
+        uint4 raw = lds128(zp);
+        float2 sc = lds64(sp);
+        zp += 512; sp += 8 * K;
+        if (--w == 0) advance();
+        const float sd = sc.y;
+        float m = lrelu(sc.x + sd), l = 1.f;
+        F2 acc[NP];
+        to_pairs(raw, acc);
+        for (int t = 0; t < n; ++t) {
+          raw = lds128(zp);
+          sc = lds64(sp);
+          zp += 512; sp += 8 * K;
+          if (--w == 0) advance();
+          const float ev = lrelu(sc.x + sd);
+          if (ev > m + 32.f) raise_reference<NP>(ev, m, l, acc);
+          const float p = fast_exp2(ev - m);
+          l += p;
+          F2 z[NP];
+          to_pairs(raw, z);
+          const F2 p2 = make_f2(p, p);
+#pragma unroll
+          for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], p2, z[t2]);
+        }
+        if (READOUT) {
+          float o[VEC];
+          finish_row_f32<NP>(acc, __fdividef(1.f, l), bs, o);
+          add_row(rs + rr, o);
+        } else {
+          finish_row(h_out + size_t(int32_t(r0) + rs + rr - win.win_base) * H + c0, acc, __fdividef(1.f, l), bs);
+        }
+      }
+      if (w != 4) {                            // the list ended inside a group: retire it without waiting
+        __syncwarp();
         if (++slot == G) { slot = 0; par ^= 1; }
       }
-      if (open) close_row();
       rs += cnt;
     }
     if (READOUT && cur_g >= 0) flush();
