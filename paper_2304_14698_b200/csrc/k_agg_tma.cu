@@ -381,16 +381,9 @@ template <typename T, int K, bool READOUT>
 int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const float* scores, const float* bias,
              void* h_out, Window win, int64_t buf_rows, const int32_t* seg_id, float* partial,
              const int32_t* self_idx, int32_t* status, cudaStream_t st) {
-  static bool attr = false;
+  static bool attr[64] = {};
   const size_t smem = sizeof(WarpSmem<K>) * TW;
-  if (!attr) {
-    if (cudaFuncSetAttribute(k_aggregate_tma<T, K, READOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             int(smem)) != cudaSuccess) {
-      cudaGetLastError();
-      return -1;
-    }
-    attr = true;
-  }
+  if (!ensure_dynamic_smem(k_aggregate_tma<T, K, READOUT>, int(smem), attr)) return -1;
   constexpr bool is_bf16 = sizeof(T) == 2;
   CUtensorMap mz, ms;
   if (!make_row_map(&mz, Z, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,

@@ -242,15 +242,8 @@ int launch_h(const Dims& d, const int32_t* rowptr, const int32_t* col, const int
              const void* shape, const void* w0ext_t, void* h, Window win, const int32_t* row_list,
              int32_t* status, cudaStream_t st) {
   using C = ECfg<H>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(k_embed_umma<H>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) !=
-        cudaSuccess) {
-      cudaGetLastError();
-      return -1;
-    }
-    attr_set = true;
-  }
+  static bool attr_set[64] = {};
+  if (!ensure_dynamic_smem(k_embed_umma<H>, C::SMEM_BYTES, attr_set)) return -1;
   const int op_pieces = (d.T + 7) / 8;
   const int ksteps = (4 + op_pieces + 1) / 2;
   const int kpad = ((ksteps + 3) / 4) * KCH;

@@ -344,11 +344,8 @@ int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cu
   }
   // graphs small enough for shared memory: one CTA builds the whole CSR of a graph
   if (in.B > 0 && in.max_n > 0 && in.max_n <= 16384 && pack_graph_smem(in.max_n, in.max_m) <= 160 * 1024) {
-    static bool attr = false;
-    if (!attr) {
-      cudaFuncSetAttribute(k_pack_graph, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-      attr = true;
-    }
+    static bool attr[64] = {};
+    ensure_dynamic_smem(k_pack_graph, 160 * 1024, attr);
     k_pack_graph<<<in.B, kGraphThreads, pack_graph_smem(in.max_n, in.max_m), st>>>(
         out.node_off, out.edge_off, in.op, in.edge_src, in.edge_dst, T, in.B, in.max_n, out.seg_id,
         out.rowptr, out.col, status);

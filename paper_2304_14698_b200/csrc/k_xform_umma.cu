@@ -230,15 +230,8 @@ template <int H>
 int launch_h(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* scores,
              Window win, int32_t* status, cudaStream_t st) {
   using C = Cfg<H>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(k_xform_umma<H>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) !=
-        cudaSuccess) {
-      cudaGetLastError();
-      return -1;
-    }
-    attr_set = true;
-  }
+  static bool attr_set[64] = {};
+  if (!ensure_dynamic_smem(k_xform_umma<H>, C::SMEM_BYTES, attr_set)) return -1;
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   const size_t off = size_t(win.row_begin - win.win_base);
   const bf16* hp = static_cast<const bf16*>(h) + off * H;

@@ -80,6 +80,20 @@ struct Dims {
   int dtype;
 };
 
+// Opt-in to large dynamic shared memory is a per-device function attribute: remember it per device.
+template <typename Kernel>
+inline bool ensure_dynamic_smem(Kernel kernel, int bytes, bool (&done)[64]) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return false; }
+  if (done[dev]) return true;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  done[dev] = true;
+  return true;
+}
+
 // ---- launchers (each returns the number of kernels it launched; errors via cudaGetLastError) --
 struct PackIn {
   int32_t B, num_envs, N, E;
