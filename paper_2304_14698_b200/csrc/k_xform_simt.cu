@@ -69,6 +69,87 @@ k_xform_simt(const T* __restrict__ h, const T* __restrict__ W, T* __restrict__ Z
   }
 }
 
+// Larger register tile for batches with many rows: 128 x 128 outputs per CTA, 8 x 8 per thread (as two
+// 4-wide column groups and two 4-high row groups so that the shared-memory reads are conflict-free
+// 16-byte loads), K advanced 8 at a time with the next slice prefetched into registers.
+constexpr int TM = 128, TN = 128, TK = 8;
+
+template <typename T>
+__device__ __forceinline__ void load4(const T* p, bool ok, float (&v)[4]);
+template <>
+__device__ __forceinline__ void load4<float>(const float* p, bool ok, float (&v)[4]) {
+  const float4 t = ok ? __ldg(reinterpret_cast<const float4*>(p)) : make_float4(0.f, 0.f, 0.f, 0.f);
+  v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+}
+template <>
+__device__ __forceinline__ void load4<bf16>(const bf16* p, bool ok, float (&v)[4]) {
+  const uint2 t = ok ? __ldg(reinterpret_cast<const uint2*>(p)) : make_uint2(0u, 0u);
+  v[0] = __uint_as_float(t.x << 16); v[1] = __uint_as_float(t.x & 0xFFFF0000u);
+  v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xFFFF0000u);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+k_xform_simt128(const T* __restrict__ h, const T* __restrict__ W, T* __restrict__ Z, int H, int rows) {
+  __shared__ __align__(16) float As[TK][TM];
+  __shared__ __align__(16) float Bs[TK][TN];
+  const int tid = threadIdx.x;
+  const int ty = tid >> 4, tx = tid & 15;
+  const int64_t row0 = int64_t(blockIdx.x) * TM;
+  const int col0 = blockIdx.y * TN;
+  float acc[8][8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+
+  const int a_row = tid >> 1, a_k = (tid & 1) * 4;      // 128 rows x 8 k: one 4-vector per thread
+  const int b_k = tid >> 5, b_c = (tid & 31) * 4;       // 8 k x 128 cols
+  const bool a_ok = row0 + a_row < rows;
+  const T* a_ptr = h + size_t(a_ok ? row0 + a_row : 0) * H + a_k;
+  const bool b_ok = col0 + b_c < H;                     // H is a multiple of 4
+  const T* b_ptr = W + size_t(b_k) * H + (b_ok ? col0 + b_c : 0);
+  float ra[4], rb[4];
+  load4<T>(a_ptr, a_ok, ra);
+  load4<T>(b_ptr, b_ok, rb);
+  for (int k0 = 0; k0 < H; k0 += TK) {
+#pragma unroll
+    for (int t = 0; t < 4; ++t) As[a_k + t][a_row] = ra[t];
+    *reinterpret_cast<float4*>(&Bs[b_k][b_c]) = make_float4(rb[0], rb[1], rb[2], rb[3]);
+    __syncthreads();
+    if (k0 + TK < H) {                                    // next slice in flight during the arithmetic
+      load4<T>(a_ptr + k0 + TK, a_ok, ra);
+      load4<T>(b_ptr + size_t(k0 + TK) * H, b_ok, rb);
+    }
+#pragma unroll
+    for (int k = 0; k < TK; ++k) {
+      const float4 a0 = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&As[k][64 + ty * 4]);
+      const float4 b0 = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
+      const float4 b1 = *reinterpret_cast<const float4*>(&Bs[k][64 + tx * 4]);
+      const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int64_t r = row0 + (i < 4 ? ty * 4 + i : 64 + ty * 4 + (i - 4));
+    if (r >= rows) continue;
+#pragma unroll
+    for (int jg = 0; jg < 2; ++jg) {
+      const int c = col0 + jg * 64 + tx * 4;
+      if (c >= H) continue;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) Z[size_t(r) * H + c + j] = T(acc[i][jg * 4 + j]);
+    }
+  }
+}
+
 }  // namespace
 
 int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* scores,
@@ -76,6 +157,18 @@ int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   if (rows <= 0) return 0;
   const size_t off = size_t(win.row_begin - win.win_base) * d.H;
+  if (rows >= 8192) {
+    dim3 g128(unsigned((rows + TM - 1) / TM), unsigned((d.H + TN - 1) / TN));
+    if (d.dtype == XRL_BF16)
+      k_xform_simt128<bf16><<<g128, 256, 0, st>>>(static_cast<const bf16*>(h) + off,
+                                                  static_cast<const bf16*>(lw.W),
+                                                  static_cast<bf16*>(Z) + off, d.H, int(rows));
+    else
+      k_xform_simt128<float><<<g128, 256, 0, st>>>(static_cast<const float*>(h) + off,
+                                                   static_cast<const float*>(lw.W),
+                                                   static_cast<float*>(Z) + off, d.H, int(rows));
+    return 1 + launch_scores(d, Z, lw, scores, win, st);
+  }
   dim3 grid(unsigned((rows + BM - 1) / BM), unsigned((d.H + BN - 1) / BN));
   if (d.dtype == XRL_BF16)
     k_xform_simt<bf16><<<grid, 256, 0, st>>>(static_cast<const bf16*>(h) + off,

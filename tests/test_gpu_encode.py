@@ -107,6 +107,23 @@ def test_model_shapes(xo, H, K, dtype, L):
     gpu_util.assert_close(got["value"], want["value"], dtype, "value")
 
 
+@pytest.mark.parametrize("H,K,dtype", [(96, 3, "bf16"), (160, 5, "fp32"), (64, 2, "fp32")])
+def test_cuda_core_transform_on_many_rows(xo, H, K, dtype):
+    """Row counts large enough for the 128 x 128 tile of the CUDA-core transform, sizes the tensor-core
+    kernel does not take."""
+    batch = configs.make_batch(2, candidates=19)
+    if dtype == "bf16":
+        batch["shape"] = dags.round_to_bf16_grid(batch["shape"])
+    m = dict(batch["model"], H=H, K=K, dtype=dtype, L=2, Hm=32)
+    batch["model"] = m
+    blob, _ = gpu_util.default_weights(batch, 12)
+    got = gpu_util.run_gpu(batch, blob)
+    want = xo.forward(m, blob, batch)
+    assert got["status"] == 0
+    gpu_util.assert_close(got["emb"], want["emb"], dtype, "graph_emb")
+    gpu_util.assert_close(got["probs"], want["probs"], dtype, "probs")
+
+
 def test_degenerate_batches(xo):
     """Environment without candidates, fully masked environment, empty graph, isolated nodes,
     a consumer with hundreds of producers, padded action slots."""
