@@ -343,6 +343,8 @@ def main():
         elapsed_ms, tot_graphs, tot_edges, tot_nodes = reduce_over_ranks(elapsed_ms, B, E, N, dist, "cuda")
         if e2e:
             e2e["s_per_step"] = reduce_over_ranks(e2e["s_per_step"], 0, 0, 0, dist, "cuda")[0]
+        if delta:
+            delta["ms_per_step"] = reduce_over_ranks(delta["ms_per_step"], 0, 0, 0, dist, "cuda")[0]
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -384,8 +386,6 @@ def main():
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                        "ms_per_step": e2e["s_per_step"] * 1e3}
     if delta:
-        if world > 1:
-            delta["ms_per_step"] = reduce_over_ranks(delta["ms_per_step"], 0, 0, 0, dist, "cuda")[0]
         delta["value"] = tot_graphs / (delta["ms_per_step"] * 1e-3)
         delta["unit"] = "graphs/s"
         delta["note"] = "xrl_encode_delta: same outputs, candidates reuse the current graph's unchanged rows"
