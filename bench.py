@@ -224,10 +224,18 @@ def main():
 
     import torch
     import paper_2304_14698_b200 as xrl
+    ndev = torch.cuda.device_count()
+    shared_gpu = world > ndev                  # more ranks than GPUs (testing only): ranks share devices
+    local_rank = local_rank % max(1, ndev)
     torch.cuda.set_device(local_rank)
+    red_dev = "cuda"
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        if shared_gpu:                         # NCCL cannot put two ranks on one GPU: reduce the scalars over gloo
+            dist.init_process_group("gloo")
+            red_dev = "cpu"
+        else:
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     agent = xrl.Agent(m, B, Ne, N, E, device=local_rank)
     agent.set_weights(blob)
@@ -340,11 +348,11 @@ def main():
     # ---- reduce over ranks -----------------------------------------------------------------------------
     tot_graphs, tot_edges, tot_nodes = B, E, N
     if world > 1:
-        elapsed_ms, tot_graphs, tot_edges, tot_nodes = reduce_over_ranks(elapsed_ms, B, E, N, dist, "cuda")
+        elapsed_ms, tot_graphs, tot_edges, tot_nodes = reduce_over_ranks(elapsed_ms, B, E, N, dist, red_dev)
         if e2e:
-            e2e["s_per_step"] = reduce_over_ranks(e2e["s_per_step"], 0, 0, 0, dist, "cuda")[0]
+            e2e["s_per_step"] = reduce_over_ranks(e2e["s_per_step"], 0, 0, 0, dist, red_dev)[0]
         if delta:
-            delta["ms_per_step"] = reduce_over_ranks(delta["ms_per_step"], 0, 0, 0, dist, "cuda")[0]
+            delta["ms_per_step"] = reduce_over_ranks(delta["ms_per_step"], 0, 0, 0, dist, red_dev)[0]
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
