@@ -1,0 +1,75 @@
+"""The pins must be sharp: each plausible slip planted in a copy of the oracle (on the CPU, in a scratch
+directory) has to make the dense brute-force comparison or a heads/pack check fail."""
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+import pytest
+
+import dense_ref
+from workloads import configs, dags
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+SRC = os.path.join(os.path.dirname(HERE), "oracle", "xrl_oracle.cpp")
+
+MUTATIONS = [
+    ("LeakyReLU slope", "return x > 0.0 ? x : 0.2 * x;", "return x > 0.0 ? x : 0.1 * x;"),
+    ("half-scores swapped", "s_src[size_t(j) * K + k] + s_dst[size_t(i) * K + k]",
+     "s_src[size_t(i) * K + k] + s_dst[size_t(j) * K + k]"),
+    ("one-hot offset", "x[S + op[gi]] = 1.0;", "x[S + op[gi] + 1 < F0 ? S + op[gi] + 1 : S] = 1.0;"),
+    ("layer bias dropped", "acc = relu(acc + double(w.b[l][c]));", "acc = relu(acc);"),
+    ("self term dropped", "for (int t = 0; t <= deg; ++t) { al[t] = std::exp(sc[t] - mx); sum += al[t]; }",
+     "for (int t = 0; t <= deg; ++t) { al[t] = (t < deg || deg == 0) ? std::exp(sc[t] - mx) : 0.0; sum += al[t]; }"),
+    ("own shape block dropped", "x[S + T + s] = double(shape[size_t(gi) * S + s]);", "x[S + T + s] = 0.0;"),
+    ("edge aggregate takes the consumer's shape", "x[s] += double(shape[size_t(col[e]) * S + s]);",
+     "x[s] += double(shape[size_t(gi) * S + s]);"),
+    ("readout mean instead of sum", "for (int c = 0; c < m.Dg; ++c) u[H + c] = g_attr ? g_attr[c] : 0.0;",
+     "for (int c = 0; c < H; ++c) u[c] /= double(n > 0 ? n : 1);\n  for (int c = 0; c < m.Dg; ++c) u[H + c] = g_attr ? g_attr[c] : 0.0;"),
+    ("global attribute ignored", "u[H + c] = g_attr ? g_attr[c] : 0.0;", "u[H + c] = 0.0;"),
+    ("bf16 truncation instead of rounding", "u += 0x7FFFu + lsb;", "u += 0u * lsb;"),
+]
+
+
+def _build(tmp_path, name, old, new):
+    src = open(SRC).read()
+    assert old in src, f"mutation target for '{name}' not found: the oracle changed, update this test"
+    path = tmp_path / "mut.cpp"
+    path.write_text(src.replace(old, new))
+    so = tmp_path / "libmut.so"
+    subprocess.run(["g++", "-std=c++17", "-O1", "-fPIC", "-shared", "-fopenmp", "-o", str(so), str(path)], check=True)
+    return ctypes.CDLL(str(so))
+
+
+def _pins_hold(xo):
+    """A condensed version of the brute-force pins; returns False as soon as one breaks."""
+    for dtype in ("fp32", "bf16"):
+        m = dict(T=6, S=8, H=16, K=2, L=2, Hm=8, Dg=2, dtype=dtype, A_max=4)
+        _, W = configs.make_weights(m, 11)
+        rng = dags.make_rng(5)
+        graphs = [dags.random_dag(rng, 12, 6, 8, dtype == "bf16", window=6) for _ in range(4)]
+        b = dags.flatten(graphs, [0, len(graphs)], 4)
+        st, p = xo.pack(b)
+        if st != 0:
+            return False
+        g0 = np.random.default_rng(1).normal(size=(len(graphs), 2))
+        # weights that are not on the bf16 grid exercise the rounding of the stored matrices
+        out = xo.encode(m, configs.pack_weights(m, W), b, p, g0=g0)
+        for gi, g in enumerate(graphs):
+            want = dense_ref.encode_graph(g, W, m, g0[gi])
+            if not np.allclose(out["emb"][gi], want, rtol=1e-10, atol=1e-11):
+                return False
+    return True
+
+
+@pytest.mark.parametrize("name,old,new", MUTATIONS, ids=[m[0] for m in MUTATIONS])
+def test_planted_mistake_is_caught(xo, tmp_path, name, old, new):
+    assert _pins_hold(xo), "the unmodified oracle must pass"
+    mutant = _build(tmp_path, name, old, new)
+    mutant.xo_philox4x32_10.restype = None
+    saved = xo._lib
+    try:
+        xo._lib = mutant
+        assert not _pins_hold(xo), f"mutation '{name}' went unnoticed"
+    finally:
+        xo._lib = saved
