@@ -89,8 +89,10 @@ typedef struct xrl_batch xrl_batch;
 /* ---- context and weights -------------------------------------------------------------- */
 
 /* Create a context on CUDA device `device`: validates the config, allocates the activation
- * workspace for the stated capacities (about 3 * max_nodes * H * sizeof(storage) bytes plus
- * 8 * heads bytes per node).  *out is HOST.  Errors: INVALID_ARG, UNSUPPORTED, CUDA, ALLOC. */
+ * workspace for the stated capacities: two feature buffers of max_nodes * H * sizeof(storage) bytes,
+ * 8 * heads bytes of half-scores per node, 4 * H bytes of readout partial sums per 32 nodes (the first
+ * xrl_encode_delta call adds about 40 bytes per node and 4 per edge).  *out is HOST.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA, ALLOC. */
 xrl_status xrl_create(const xrl_model_config* cfg, int32_t device, xrl_ctx** out);
 void xrl_destroy(xrl_ctx* ctx);
 

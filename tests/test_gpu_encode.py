@@ -124,6 +124,19 @@ def test_cuda_core_transform_on_many_rows(xo, H, K, dtype):
     gpu_util.assert_close(got["probs"], want["probs"], dtype, "probs")
 
 
+def test_cuda_core_kernels_on_tensor_core_shapes(xo, monkeypatch):
+    """XRL_FORCE_SIMT_TRANSFORM keeps Eq. 6 and the transform on the CUDA cores for shapes the tensor-core
+    kernels normally take: both paths must agree with the oracle."""
+    monkeypatch.setenv("XRL_FORCE_SIMT_TRANSFORM", "1")
+    batch = configs.make_batch(4, candidates=3)
+    blob, _ = gpu_util.default_weights(batch, 1004)
+    got = gpu_util.run_gpu(batch, blob)
+    want = xo.forward(batch["model"], blob, batch)
+    assert got["status"] == 0
+    gpu_util.assert_close(got["emb"], want["emb"], "bf16", "graph_emb")
+    gpu_util.assert_close(got["probs"], want["probs"], "bf16", "probs")
+
+
 def test_degenerate_batches(xo):
     """Environment without candidates, fully masked environment, empty graph, isolated nodes,
     a consumer with hundreds of producers, padded action slots."""
