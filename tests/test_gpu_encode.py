@@ -137,6 +137,33 @@ def test_cuda_core_kernels_on_tensor_core_shapes(xo, monkeypatch):
     gpu_util.assert_close(got["probs"], want["probs"], "bf16", "probs")
 
 
+@pytest.mark.parametrize("cfg,kw", [(4, dict(candidates=3)), (2, dict(candidates=7)), (3, dict(candidates=7))])
+def test_large_attention_scores(xo, cfg, kw):
+    """Attention vectors scaled up until the scores of one row differ by hundreds: the running softmax
+    has to move its reference exponent (a rarely taken branch) and must neither overflow nor lose the
+    dominant producer."""
+    batch = configs.make_batch(cfg, **kw)
+    m = batch["model"]
+    _, W = gpu_util.default_weights(batch, 31)
+    for l in range(1, m["L"] + 1):
+        W[f"a_src{l}"] *= 300.0
+        W[f"a_dst{l}"] *= 300.0
+    blob = configs.pack_weights(m, W)
+    got = gpu_util.run_gpu(batch, blob)
+    st, packed = xo.pack(batch)
+    enc = xo.encode(m, blob, batch, packed, dump_layer=1, want_nodes=True, want_alpha=True)
+    assert np.nanmax(enc["alpha_edge"]) > 0.999 and np.nanmin(enc["alpha_edge"]) < 1e-30   # really saturated
+    assert got["status"] == 0
+    assert np.all(np.isfinite(got["emb"]))
+    if m["dtype"] == "fp32":
+        gpu_util.assert_close(got["emb"], enc["emb"], "fp32", "graph_emb")
+    else:
+        # with saturated attention a bf16 rounding of Z can flip which producer wins: compare the bulk
+        err = np.abs(got["emb"] - enc["emb"])
+        bound = 2e-2 + 2e-2 * np.abs(enc["emb"])
+        assert (err <= bound).mean() > 0.97
+
+
 def test_degenerate_batches(xo):
     """Environment without candidates, fully masked environment, empty graph, isolated nodes,
     a consumer with hundreds of producers, padded action slots."""
