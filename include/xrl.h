@@ -106,6 +106,9 @@ xrl_status xrl_weights_size(const xrl_ctx* ctx, size_t* bytes);
 /* Upload the blob (HOST, fp32).  With XRL_BF16 the library rounds W0 and the layer matrices W
  * to bf16 (nearest even) once; everything else stays fp32.  Synchronous. */
 xrl_status xrl_set_weights(xrl_ctx* ctx, const void* host_blob, size_t bytes);
+/* Read the fp32 blob back (HOST, same layout and size; the master copy, not the bf16-rounded one):
+ * together with xrl_set_weights this is the checkpoint / restore of a model.  Synchronous. */
+xrl_status xrl_get_weights(const xrl_ctx* ctx, void* host_blob, size_t bytes);
 
 /* ---- (1) packer: Section 3.3.2, the current graph and its candidates become one meta-graph ---- */
 

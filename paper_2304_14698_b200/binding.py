@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = [
     "xrl_create", "xrl_destroy", "xrl_weights_size", "xrl_set_weights", "xrl_pack", "xrl_pack_flat",
     "xrl_batch_free", "xrl_batch_info", "xrl_batch_export", "xrl_encode", "xrl_debug_node_features",
     "xrl_policy_value", "xrl_sample", "xrl_last_device_status", "xrl_launch_counts", "xrl_version",
-    "xrl_profile", "xrl_profile_read", "xrl_pack_csr_static", "xrl_encode_delta", "xrl_delta_rows",
+    "xrl_profile", "xrl_profile_read", "xrl_pack_csr_static", "xrl_encode_delta", "xrl_delta_rows", "xrl_get_weights",
 ]
 PROFILE_FAMILIES = ["pack", "node_update", "transform", "aggregate", "readout", "heads", "aggregate_readout"]
 
@@ -67,6 +67,7 @@ def load_library():
         "xrl_destroy": [vp],
         "xrl_weights_size": [vp, C.POINTER(C.c_size_t)],
         "xrl_set_weights": [vp, vp, C.c_size_t],
+        "xrl_get_weights": [vp, vp, C.c_size_t],
         "xrl_pack": [vp, C.POINTER(_Graph), i32, vp, i32, vp, C.POINTER(vp)],
         "xrl_pack_flat": [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, i32, vp, C.POINTER(vp)],
         "xrl_batch_free": [vp, vp],
@@ -153,6 +154,12 @@ def xrl_weights_size(ctx) -> int:
 def xrl_set_weights(ctx, blob: np.ndarray):
     blob = np.ascontiguousarray(blob, dtype=np.float32)
     _check(load_library().xrl_set_weights(ctx, _np_ptr(blob), blob.nbytes), "xrl_set_weights")
+
+
+def xrl_get_weights(ctx) -> np.ndarray:
+    blob = np.zeros(xrl_weights_size(ctx) // 4, np.float32)
+    _check(load_library().xrl_get_weights(ctx, _np_ptr(blob), blob.nbytes), "xrl_get_weights")
+    return blob
 
 
 def xrl_pack(ctx, graphs, env_off, dtype, stream=None, batch=None):

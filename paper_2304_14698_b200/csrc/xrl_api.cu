@@ -524,6 +524,15 @@ xrl_status xrl_set_weights(xrl_ctx* ctx, const void* host_blob, size_t bytes) {
   return XRL_OK;
 }
 
+xrl_status xrl_get_weights(const xrl_ctx* ctx, void* host_blob, size_t bytes) {
+  if (!ctx || !host_blob) return XRL_ERR_INVALID_ARG;
+  if (bytes != 4 * ctx->weight_floats) return XRL_ERR_INVALID_ARG;
+  if (!ctx->weights_set) return XRL_ERR_STATE;
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  XRL_CUDA(cudaMemcpy(host_blob, ctx->w_f32.p, bytes, cudaMemcpyDeviceToHost));
+  return XRL_OK;
+}
+
 xrl_status xrl_pack(xrl_ctx* ctx, const xrl_graph* graphs, int32_t num_graphs, const int32_t* env_off,
                     int32_t num_envs, void* stream, xrl_batch** out) {
   if (num_graphs > 0 && !graphs) return XRL_ERR_INVALID_ARG;

@@ -125,6 +125,22 @@ def test_pack_argument_and_capacity_errors():
         ag.close()
 
 
+def test_weights_round_trip():
+    import paper_2304_14698_b200 as xrl
+    b = configs.make_batch(3, candidates=1)
+    blob, _ = configs.make_weights(b["model"], 3)
+    ag = gpu_util.make_agent(b)
+    try:
+        assert xrl.xrl_weights_size(ag.ctx) == blob.nbytes == 4 * configs.weight_count(b["model"])
+        with pytest.raises(xrl.XrlError) as e:
+            xrl.xrl_get_weights(ag.ctx)
+        assert e.value.status == 6            # nothing set yet
+        ag.set_weights(blob)
+        assert np.array_equal(xrl.xrl_get_weights(ag.ctx), blob)     # the fp32 master copy, bit for bit
+    finally:
+        ag.close()
+
+
 def test_repack_in_place_reuses_the_batch(xo):
     import paper_2304_14698_b200 as xrl
     b1 = configs.make_batch(2, candidates=9, seed=5)
