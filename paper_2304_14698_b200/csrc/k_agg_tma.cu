@@ -30,9 +30,12 @@ constexpr int G = XRL_AGG_GROUPS;   // gather groups (of four rows) in flight pe
 constexpr int BR = 32;           // destination rows per block
 constexpr int ITEMS = 160;       // list capacity, a multiple of 4
 
-template <int K> struct alignas(128) WarpSmem {
-  uint4 z[G][4][32];             // four gathered rows of 512 bytes per group
-  float2 sc[G][4][K];            // their {s_src, s_dst} pairs
+// MERGED: the rows of Z carry their K {s_src, s_dst} pairs behind the 512 feature bytes, so one gather
+// per group brings both; otherwise the pairs come from a second gather into `sc`.
+template <int K, bool MERGED> struct alignas(128) WarpSmem {
+  static constexpr int ROW = MERGED ? 512 + 8 * K : 512;     // bytes per gathered row
+  uint8_t z[G][4][ROW];          // four gathered rows per group
+  float2 sc[MERGED ? 1 : G][4][K];   // their {s_src, s_dst} pairs (separate gather only)
   unsigned long long bar[G];
   int32_t rp[BR + 1];
   alignas(16) int32_t item[ITEMS + 4];
@@ -159,7 +162,7 @@ __device__ __forceinline__ void raise_reference(float ev, float& m, float& l, F2
 //   partial[nblocks + g] the rows of graph g inside the block in which g starts, when that is not at
 //                        the block's first row
 // (k_global_update_blocks adds them per graph in a fixed order).  Needs row_begin = win_base = 0.
-template <typename T, int K, bool READOUT>
+template <typename T, int K, bool READOUT, bool MERGED>
 __global__ void __launch_bounds__(TW * 32, XRL_AGG_CTAS)
 k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant__ CUtensorMap map_s,
                 const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
@@ -170,10 +173,14 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
   constexpr int VEC = VecOf<T>::N;
   constexpr int NP = VEC / 2;
   constexpr int H = 32 * VEC;
+  using Smem = WarpSmem<K, MERGED>;
+  constexpr uint32_t ZR = Smem::ROW;                  // bytes per gathered row
+  constexpr uint32_t SR = MERGED ? ZR : 8 * K;        // distance between consecutive rows' pairs
   constexpr uint32_t GROUP_BYTES = 4 * 512 + 4 * K * 8;
-  constexpr uint32_t ZG = 2048, SG = 32 * K;          // bytes per group in the two rings
+  constexpr uint32_t ZG = 4 * ZR, SG = 4 * SR;        // bytes per group in the ring(s)
+  constexpr int ZS = int(ZR / sizeof(T));             // elements between rows of the Z buffer (slow path)
   extern __shared__ __align__(128) uint8_t tma_smem_raw[];
-  WarpSmem<K>& sm = reinterpret_cast<WarpSmem<K>*>(tma_smem_raw)[threadIdx.x >> 5];
+  Smem& sm = reinterpret_cast<Smem*>(tma_smem_raw)[threadIdx.x >> 5];
   const int lane = threadIdx.x & 31;
   const int warps_total = (gridDim.x * blockDim.x) >> 5;
   const int warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -182,10 +189,11 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
   float bs[VEC];
 #pragma unroll
   for (int t = 0; t < VEC; ++t) bs[t] = __ldg(bias + c0 + t);
-  const uint32_t z_lane = smem_u32(&sm.z[0][0][lane]);       // this lane's 16 bytes of slot 0, row 0
-  const uint32_t s_lane = smem_u32(&sm.sc[0][0][head]);      // this lane's head in slot 0, row 0
   const uint32_t z_base = smem_u32(&sm.z[0][0][0]);
   const uint32_t s_base = smem_u32(&sm.sc[0][0][0]);
+  const uint32_t z_lane = z_base + lane * 16;                // this lane's 16 bytes of slot 0, row 0
+  const uint32_t s_lane = MERGED ? z_base + 512 + head * 8   // this lane's head in slot 0, row 0
+                                 : s_base + head * 8;
   const uint32_t bar_base = smem_u32(&sm.bar[0]);
 
   if (lane == 0) {
@@ -205,7 +213,7 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
     const uint32_t bar = bar_base + 8 * s;
     mbar_expect_tx(bar, GROUP_BYTES);
     tma_gather4(z_base + s * ZG, &map_z, it.x, it.y, it.z, it.w, bar);
-    tma_gather4(s_base + s * SG, &map_s, it.x, it.y, it.z, it.w, bar);
+    if (!MERGED) tma_gather4(s_base + s * SG, &map_s, it.x, it.y, it.z, it.w, bar);
   };
 
   for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * BR; r0 < win.row_end && alive;
@@ -256,16 +264,21 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
         const int32_t lrow = int32_t(r0) + rs - win.win_base;
         const int n = sm.rp[rs + 1] - eb;
         const int32_t srow = self_idx ? __ldg(self_idx + int32_t(r0) + rs) : lrow;
-        const float2 self = __ldg(scores + size_t(srow) * K + head);
+        // pairs of node v: behind its Z row when merged, else in the separate array
+        auto pair_of = [&](int32_t v) -> const float2* {
+          return MERGED ? reinterpret_cast<const float2*>(Z + size_t(v) * ZS + H) + head
+                        : scores + size_t(v) * K + head;
+        };
+        const float2 self = __ldg(pair_of(srow));
         const float sd = self.y;
         float m = lrelu(self.x + sd), l = 1.f;
         F2 acc[NP];
-        to_pairs(__ldg(reinterpret_cast<const uint4*>(Z + size_t(srow) * H + c0)), acc);
+        to_pairs(__ldg(reinterpret_cast<const uint4*>(Z + size_t(srow) * ZS + c0)), acc);
         for (int t = 0; t < n; ++t) {
           const int32_t j = __ldg(col + eb + t) - win.win_base;
-          const float ev = lrelu(__ldg(&scores[size_t(j) * K + head].x) + sd);
+          const float ev = lrelu(__ldg(&pair_of(j)->x) + sd);
           F2 z[NP];
-          to_pairs(__ldg(reinterpret_cast<const uint4*>(Z + size_t(j) * H + c0)), z);
+          to_pairs(__ldg(reinterpret_cast<const uint4*>(Z + size_t(j) * ZS + c0)), z);
           if (ev > m + 32.f) raise_reference<NP>(ev, m, l, acc);
           const float p = fast_exp2(ev - m);
           l += p;
@@ -321,7 +334,7 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
         // the row's own vector opens the running softmax: reference exponent = its score, weight 1
         uint4 raw = lds128(zp);
         float2 sc = lds64(sp);
-        zp += 512; sp += 8 * K;
+        zp += ZR; sp += SR;
         if (--w == 0) advance();
         const float sd = sc.y;
         float m = lrelu(sc.x + sd), l = 1.f;
@@ -330,7 +343,7 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
         for (int t = 0; t < n; ++t) {
           raw = lds128(zp);
           sc = lds64(sp);
-          zp += 512; sp += 8 * K;
+          zp += ZR; sp += SR;
           if (--w == 0) advance();
           const float ev = lrelu(sc.x + sd);
           if (ev > m + 32.f) raise_reference<NP>(ev, m, l, acc);
@@ -377,24 +390,40 @@ bool make_row_map(CUtensorMap* m, const void* ptr, CUtensorMapDataType dt, uint3
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <typename T, int K, bool READOUT>
+bool make_merged_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint32_t row_bytes) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {row_bytes / 4, rows};      // rows of 32-bit words: features, then the pairs
+  cuuint64_t strides[1] = {row_bytes};
+  cuuint32_t box[2] = {row_bytes / 4, 1};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <typename T, int K, bool READOUT, bool MERGED>
 int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const float* scores, const float* bias,
              void* h_out, Window win, int64_t buf_rows, const int32_t* seg_id, float* partial,
              const int32_t* self_idx, int32_t* status, cudaStream_t st) {
   static bool attr[64] = {};
-  const size_t smem = sizeof(WarpSmem<K>) * TW;
-  if (!ensure_dynamic_smem(k_aggregate_tma<T, K, READOUT>, int(smem), attr)) return -1;
+  const size_t smem = sizeof(WarpSmem<K, MERGED>) * TW;
+  if (!ensure_dynamic_smem(k_aggregate_tma<T, K, READOUT, MERGED>, int(smem), attr)) return -1;
   constexpr bool is_bf16 = sizeof(T) == 2;
   CUtensorMap mz, ms;
-  if (!make_row_map(&mz, Z, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
-                    sizeof(T), uint64_t(buf_rows), is_bf16 ? 256 : 128) ||
-      !make_row_map(&ms, scores, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, uint64_t(buf_rows), 2 * K))
+  if (MERGED) {
+    if (!make_merged_map(&mz, Z, uint64_t(buf_rows), 512 + 8 * K)) return -1;
+    ms = mz;
+  } else if (!make_row_map(&mz, Z, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                           sizeof(T), uint64_t(buf_rows), is_bf16 ? 256 : 128) ||
+             !make_row_map(&ms, scores, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, uint64_t(buf_rows), 2 * K)) {
     return -1;
+  }
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   const int64_t nblocks = (rows + BR - 1) / BR;
   int64_t nb = (rows + BR * TW - 1) / (BR * TW);
   if (nb > int64_t(kNumSMs) * XRL_AGG_CTAS) nb = int64_t(kNumSMs) * XRL_AGG_CTAS;
-  k_aggregate_tma<T, K, READOUT><<<int(nb), TW * 32, smem, st>>>(
+  k_aggregate_tma<T, K, READOUT, MERGED><<<int(nb), TW * 32, smem, st>>>(
       mz, ms, rowptr, col, static_cast<const T*>(Z), reinterpret_cast<const float2*>(scores), bias,
       static_cast<T*>(h_out), win, seg_id, partial, int32_t(nblocks), self_idx, status);
   return 1;
@@ -412,23 +441,28 @@ int launch_aggregate_tma(const Dims& d, const int32_t* rowptr, const int32_t* co
   if (encode_fn() == nullptr) return -1;
   const bool bf = d.dtype == XRL_BF16 && d.H == 256, fp = d.dtype == XRL_FP32 && d.H == 128;
   if (!bf && !fp) return -1;
+  if (d.zmerged && !bf) return -1;
   if (partial != nullptr && (win.row_begin != 0 || win.win_base != 0)) return -1;
-#define TMA_CASE(KK)                                                                                       \
-  case KK:                                                                                                 \
-    if (partial != nullptr)                                                                                \
-      return bf ? launch_k<bf16, KK, true>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, seg_id,     \
-                                           partial, self_idx, status, st)                                            \
-                : launch_k<float, KK, true>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, seg_id,    \
-                                            partial, self_idx, status, st);                                          \
-    return bf ? launch_k<bf16, KK, false>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, seg_id,      \
-                                          partial, self_idx, status, st)                                             \
-              : launch_k<float, KK, false>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, seg_id,     \
-                                           partial, self_idx, status, st);
+#define TMA_ARGS rowptr, col, Z, scores, bias, h_out, win, buf_rows, seg_id, partial, self_idx, status, st
+#define TMA_CASE(KK)                                                                                   \
+  case KK:                                                                                             \
+    if (d.zmerged)                                                                                     \
+      return partial ? launch_k<bf16, KK, true, true>(TMA_ARGS) : launch_k<bf16, KK, false, true>(TMA_ARGS); \
+    if (partial != nullptr)                                                                            \
+      return bf ? launch_k<bf16, KK, true, false>(TMA_ARGS) : launch_k<float, KK, true, false>(TMA_ARGS);    \
+    return bf ? launch_k<bf16, KK, false, false>(TMA_ARGS) : launch_k<float, KK, false, false>(TMA_ARGS);
   switch (d.K) {
     TMA_CASE(4) TMA_CASE(8) TMA_CASE(16)
     default: return -1;
   }
+#undef TMA_ARGS
 #undef TMA_CASE
+}
+
+// Shapes this kernel takes (512-byte feature rows, 4 | K).
+bool aggregate_tma_shape(const Dims& d) {
+  const bool bf = d.dtype == XRL_BF16 && d.H == 256, fp = d.dtype == XRL_FP32 && d.H == 128;
+  return (bf || fp) && (d.K == 4 || d.K == 8 || d.K == 16) && encode_fn() != nullptr;
 }
 
 // Partial-sum slots the fused variant writes for `rows` rows and B graphs.

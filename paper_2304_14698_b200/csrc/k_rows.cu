@@ -343,7 +343,7 @@ int launch_aggregate(const Dims& d, const int32_t* rowptr, const int32_t* col, c
   {   // 512-byte rows with 4 | K: gathers by the TMA engine
     const int k = launch_aggregate_tma(d, rowptr, col, Z, scores, bias, h_out, win, buf_rows, nullptr, nullptr, status, st,
                                        self_idx);
-    if (k >= 0) return k;
+    if (k >= 0 || d.zmerged) return k;       // with merged rows there is no other kernel to fall back to
   }
 #define CALL(TY_, LPR, VPL)                                                                        \
   k_aggregate<TY_, LPR, VPL><<<row_grid(rows, kAggBlockRows), kRowThreads, 0, st>>>(                \

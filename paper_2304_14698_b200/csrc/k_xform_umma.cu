@@ -44,7 +44,7 @@ template <int H>
 __global__ void __launch_bounds__(kThreads, 1)
 k_xform_umma(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w,
              const __grid_constant__ CUtensorMap map_z, const float* __restrict__ a_src,
-             const float* __restrict__ a_dst, float2* __restrict__ scores,
+             const float* __restrict__ a_dst, float2* __restrict__ scores, int score_stride,
              int rows, int K, int32_t* status) {
   using C = Cfg<H>;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -186,7 +186,7 @@ k_xform_umma(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ 
           ss = fmaf(__uint_as_float(z[7]), s1.w, ss); sd = fmaf(__uint_as_float(z[7]), d1.w, sd);
           left -= 8;
           if (left == 0) {
-            if (live) scores[grow * K + head] = make_float2(ss, sd);
+            if (live) scores[grow * score_stride + head] = make_float2(ss, sd);
             ss = 0.f; sd = 0.f; ++head; left = d;
           }
         }
@@ -235,15 +235,18 @@ int launch_h(const Dims& d, const void* h, const LayerWeights& lw, void* Z, floa
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   const size_t off = size_t(win.row_begin - win.win_base);
   const bf16* hp = static_cast<const bf16*>(h) + off * H;
-  bf16* zp = static_cast<bf16*>(Z) + off * H;
+  const size_t zrow = z_row_bytes(d);                    // H * 2, or H * 2 + 8 K when the pairs follow the row
+  char* zp = static_cast<char*>(Z) + off * zrow;
+  float2* sc = d.zmerged ? reinterpret_cast<float2*>(zp + size_t(H) * 2)
+                         : reinterpret_cast<float2*>(scores) + off * d.K;
+  const int sc_stride = d.zmerged ? int(zrow / 8) : d.K;
   CUtensorMap mh, mw, mz;
   if (!make_map(&mh, hp, uint64_t(rows), H, BM) || !make_map(&mw, lw.Wt, H, H, H) ||
-      !make_map(&mz, zp, uint64_t(rows), H, BM))
+      !make_map(&mz, zp, uint64_t(rows), H, BM, zrow))
     return -1;
   const int tiles = int((rows + BM - 1) / BM);
   const int grid = tiles < kNumSMs ? tiles : kNumSMs;
-  k_xform_umma<H><<<grid, kThreads, C::SMEM_BYTES, st>>>(mh, mw, mz, lw.a_src, lw.a_dst,
-                                                         reinterpret_cast<float2*>(scores) + off * d.K,
+  k_xform_umma<H><<<grid, kThreads, C::SMEM_BYTES, st>>>(mh, mw, mz, lw.a_src, lw.a_dst, sc, sc_stride,
                                                          int(rows), d.K, status);
   return 1;
 }

@@ -383,9 +383,10 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
     if (ctx->use_umma)
       k = launch_xform_umma(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), win,
                             ctx->status.as<int32_t>(), st);
-    if (k < 0)
+    if (k < 0 && !d.zmerged)
       k = launch_xform_simt(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), win,
                             st);
+    if (k < 0) return -1;                       // merged rows: only the tensor-core transform writes them
     pf.end(FAM_XFORM, slot, k, st);
     n += k;
     slot = pf.begin(st);
@@ -402,6 +403,7 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
       k = launch_aggregate(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), ctx->Z.p,
                            ctx->scores.as<float>(), ctx->dw.layer[l].b,
                            ctx->h.p, win, b->N, ctx->status.as<int32_t>(), st);
+    if (k < 0) return -1;
     pf.end(fused_here ? FAM_AGG_READOUT : FAM_AGG, slot, k, st);
     n += k;
   }
@@ -436,11 +438,13 @@ xrl_status xrl_create(const xrl_model_config* cfg, int32_t device, xrl_ctx** out
   ctx->cfg = *cfg;
   ctx->device = device;
   ctx->dims = Dims{cfg->num_op_types, cfg->hidden, cfg->heads, cfg->layers, cfg->mlp_hidden,
-                   cfg->global_dim, cfg->max_actions, cfg->dtype};
+                   cfg->global_dim, cfg->max_actions, cfg->dtype, 0};
   ctx->weight_floats = weight_float_count(*cfg);
   // XRL_FORCE_SIMT_TRANSFORM=1 keeps the CUDA-core transform for every shape (debugging aid)
   ctx->use_umma = xform_umma_supported(ctx->dims) && getenv("XRL_FORCE_SIMT_TRANSFORM") == nullptr;
   ctx->use_umma_embed = embed_umma_supported(ctx->dims) && getenv("XRL_FORCE_SIMT_TRANSFORM") == nullptr;
+  // Z rows carry their half-score pairs when both kernels that touch them support it
+  ctx->dims.zmerged = (ctx->use_umma && cfg->dtype == XRL_BF16 && aggregate_tma_shape(ctx->dims)) ? 1 : 0;
   ctx->max_chunks = int32_t(cfg->max_graphs + cfg->max_nodes / kReadoutChunkRows + 1);
   const size_t sb = storage_bytes(cfg->dtype), N = size_t(cfg->max_nodes), H = size_t(cfg->hidden);
   const size_t F0 = size_t(2 * kS + cfg->num_op_types);
@@ -450,7 +454,7 @@ xrl_status xrl_create(const xrl_model_config* cfg, int32_t device, xrl_ctx** out
   A(ctx->w_store, sb * (F0 * H + 2 * size_t(cfg->layers) * H * H));
   A(ctx->w0ext, ctx->use_umma_embed ? 2 * H * size_t(embed_umma_kpad(ctx->dims)) : 0);
   A(ctx->h, sb * N * H);
-  A(ctx->Z, sb * N * H);
+  A(ctx->Z, N * z_row_bytes(ctx->dims));
   A(ctx->scores, 8 * N * size_t(cfg->heads));
   {
     const size_t slots_fused = size_t(aggregate_readout_slots(cfg->max_nodes, cfg->max_graphs));
@@ -600,6 +604,7 @@ xrl_status xrl_encode(xrl_ctx* ctx, const xrl_batch* b, const float* g0, float* 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   bool fused = false;
   int n = run_node_layers(ctx, b, ctx->cfg.layers, st, true, &fused);
+  if (n < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
   size_t slot;
   int k;
   if (!fused) {
@@ -702,7 +707,9 @@ xrl_status xrl_encode_delta(xrl_ctx* ctx, const xrl_batch* b, const int32_t* bas
     if (ctx->use_umma)
       k = launch_xform_umma(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), wp,
                             ctx->status.as<int32_t>(), st);
-    if (k < 0) k = launch_xform_simt(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), wp, st);
+    if (k < 0 && !d.zmerged)
+      k = launch_xform_simt(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), wp, st);
+    if (k < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
     pf.end(FAM_XFORM, slot, k, st);
     n_launch += k;
     // compact CSR of the rows this layer reaches: producers and the row's own vector by dense row
@@ -714,6 +721,7 @@ xrl_status xrl_encode_delta(xrl_ctx* ctx, const xrl_batch* b, const int32_t* bas
     const Window wc{0, n_cur, 0};
     k = launch_aggregate(d, rowptr_c, col_c, ctx->Z.p, ctx->scores.as<float>(), ctx->dw.layer[l].b, ctx->h.p,
                          wc, n_prev > 0 ? n_prev : 1, ctx->status.as<int32_t>(), st, self_c);
+    if (k < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
     pf.end(FAM_AGG, slot, k, st);
     n_launch += k;
   }
@@ -746,7 +754,7 @@ xrl_status xrl_debug_node_features(xrl_ctx* ctx, const xrl_batch* b, int32_t num
   if (num_layers < 0 || num_layers > ctx->cfg.layers || (!host_out && b->N > 0)) return XRL_ERR_INVALID_ARG;
   XRL_CUDA(cudaSetDevice(ctx->device));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  run_node_layers(ctx, b, num_layers, st);
+  if (run_node_layers(ctx, b, num_layers, st) < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
   const int64_t n = int64_t(b->N) * ctx->cfg.hidden;
   if (n == 0) return XRL_OK;
   float* tmp = nullptr;

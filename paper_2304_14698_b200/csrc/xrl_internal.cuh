@@ -78,7 +78,15 @@ struct DevWeights {
 struct Dims {
   int T, H, K, L, Hm, Dg, A;
   int dtype;
+  // 1: each row of the Z buffer is followed by the node's K {s_src, s_dst} pairs (row stride
+  // H * sizeof(storage) + 8 K bytes), so that one gather brings both; set only when the tensor-core
+  // transform and the TMA aggregate kernel handle the shape (the `scores` arguments are then unused)
+  int zmerged;
 };
+inline size_t z_row_bytes(const Dims& d) {
+  return size_t(d.H) * (d.dtype == XRL_BF16 ? 2 : 4) + (d.zmerged ? size_t(8) * d.K : 0);
+}
+bool aggregate_tma_shape(const Dims& d);
 
 // Opt-in to large dynamic shared memory is a per-device function attribute: remember it per device.
 template <typename Kernel>

@@ -123,11 +123,12 @@ inline EncodeTiledFn encode_fn() {
 }
 
 // 2-D bf16 tensor [rows x cols] row-major, box [box_rows x 64 columns], 128-byte swizzle.
-inline bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+inline bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                     uint64_t row_stride_bytes = 0) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 2};
+  cuuint64_t strides[1] = {row_stride_bytes ? row_stride_bytes : cols * 2};
   cuuint32_t box[2] = {KCH, box_rows};
   cuuint32_t estr[2] = {1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
