@@ -164,6 +164,33 @@ def test_large_attention_scores(xo, cfg, kw):
         assert (err <= bound).mean() > 0.97
 
 
+@pytest.mark.parametrize("cfg", [2, 4])
+def test_one_context_many_batches(xo, cfg):
+    """A context and its batch object are reused for steps of different sizes (the candidate set shrinks and
+    grows between rewrite steps): nothing may leak from one step into the next, in either encoder."""
+    import torch
+    big = configs.make_batch(cfg, candidates=9, seed=50)
+    m = big["model"]
+    blob, _ = gpu_util.default_weights(big, 77)
+    ag = gpu_util.make_agent(big, slack=64)
+    try:
+        ag.set_weights(blob)
+        for step, cands in enumerate([9, 2, 7, 0, 5]):
+            batch = configs.make_batch(cfg, candidates=cands, seed=60 + step)
+            want = xo.forward(m, blob, batch)
+            mask = torch.from_numpy(batch["mask"]).cuda()
+            for mode in ("full", "delta"):
+                bid = torch.from_numpy(batch["base_id"]).cuda() if mode == "delta" else None
+                o = ag.step(batch, mask, sample=True, seed=1, step=step, base_id=bid)
+                torch.cuda.synchronize()
+                assert ag.device_status() == 0
+                gpu_util.assert_close(o["emb"].cpu().numpy(), want["emb"], m["dtype"], f"step {step} {mode} emb")
+                gpu_util.assert_close(o["probs"].cpu().numpy(), want["probs"], m["dtype"], f"step {step} {mode} probs")
+                gpu_util.assert_close(o["value"].cpu().numpy(), want["value"], m["dtype"], f"step {step} {mode} value")
+    finally:
+        ag.close()
+
+
 def test_degenerate_batches(xo):
     """Environment without candidates, fully masked environment, empty graph, isolated nodes,
     a consumer with hundreds of producers, padded action slots."""
