@@ -26,6 +26,31 @@ __device__ __forceinline__ float column_dot(const float* x, int in, const float*
   return acc;
 }
 
+// y[c] = bias[c] + sum_k x[k] W[k * ld + c] for c < ncols, for every thread block shape: with fewer columns
+// than threads the k range is cut into P = blockDim / CP contiguous parts (CP = columns per pass, a power of
+// two), the parts are computed by different thread groups and added in part order.  Every thread of the
+// block calls it; `part` is blockDim floats of scratch; emit(c, y) runs once per column.
+template <typename Emit>
+__device__ __forceinline__ void dense_columns(const float* x, int in, const float* __restrict__ W, int ld,
+                                              int ncols, const float* __restrict__ bias, float* part, Emit emit) {
+  const int nt = blockDim.x, tid = threadIdx.x;
+  int CP = 32;
+  while (CP < ncols && CP < nt) CP <<= 1;
+  const int P = nt / CP, cl = tid % CP, p = tid / CP;
+  const int k0 = int((int64_t(in) * p) / P), k1 = int((int64_t(in) * (p + 1)) / P);
+  for (int c0 = 0; c0 < ncols; c0 += CP) {
+    const int c = c0 + cl;
+    part[tid] = (c < ncols) ? column_dot(x + k0, k1 - k0, W + size_t(k0) * ld, ld, c, 0.f) : 0.f;
+    __syncthreads();
+    if (p == 0 && c < ncols) {
+      float y = bias[c];
+      for (int q = 0; q < P; ++q) y += part[q * CP + cl];
+      emit(c, y);
+    }
+    __syncthreads();
+  }
+}
+
 // ---- readout, stage 1: column sums of one chunk of consecutive rows of one graph -------------
 template <typename T>
 __global__ void __launch_bounds__(kRoThreads)
@@ -76,7 +101,8 @@ __global__ void __launch_bounds__(256)
 k_global_update(const float* __restrict__ partial, const int32_t* __restrict__ graph_chunk_off,
                 const float* __restrict__ g0, const float* __restrict__ Wg,
                 const float* __restrict__ bg, float* __restrict__ emb, int H, int Dg) {
-  extern __shared__ float u[];                   // [H + Dg]
+  extern __shared__ float u[];                   // [H + Dg], then blockDim floats of scratch
+  float* part = u + H + Dg;
   const int32_t g = blockIdx.x;
   const int32_t c0 = graph_chunk_off[g], c1 = graph_chunk_off[g + 1];
   for (int c = threadIdx.x; c < H; c += blockDim.x) {
@@ -86,9 +112,8 @@ k_global_update(const float* __restrict__ partial, const int32_t* __restrict__ g
   }
   for (int t = threadIdx.x; t < Dg; t += blockDim.x) u[H + t] = g0 ? g0[size_t(g) * Dg + t] : 0.f;
   __syncthreads();
-  for (int c = threadIdx.x; c < H; c += blockDim.x) {
-    emb[size_t(g) * H + c] = fmaxf(column_dot(u, H + Dg, Wg, H, c, bg[c]), 0.f);
-  }
+  dense_columns(u, H + Dg, Wg, H, H, bg, part,
+                [&](int c, float y) { emb[size_t(g) * H + c] = fmaxf(y, 0.f); });
 }
 
 // Eq. 8 from the partial sums written by the aggregate kernel fused with the readout: per graph, the
@@ -98,7 +123,8 @@ __global__ void __launch_bounds__(256)
 k_global_update_blocks(const float* __restrict__ partial, const int32_t* __restrict__ node_off,
                        int32_t nblocks, const float* __restrict__ g0, const float* __restrict__ Wg,
                        const float* __restrict__ bg, float* __restrict__ emb, int H, int Dg) {
-  extern __shared__ float u[];                   // [H + Dg]
+  extern __shared__ float u[];                   // [H + Dg], then blockDim floats of scratch
+  float* part = u + H + Dg;
   const int32_t g = blockIdx.x;
   const int32_t start = node_off[g], end = node_off[g + 1];
   for (int c = threadIdx.x; c < H; c += blockDim.x) {
@@ -113,9 +139,8 @@ k_global_update_blocks(const float* __restrict__ partial, const int32_t* __restr
   }
   for (int t = threadIdx.x; t < Dg; t += blockDim.x) u[H + t] = g0 ? g0[size_t(g) * Dg + t] : 0.f;
   __syncthreads();
-  for (int c = threadIdx.x; c < H; c += blockDim.x) {
-    emb[size_t(g) * H + c] = fmaxf(column_dot(u, H + Dg, Wg, H, c, bg[c]), 0.f);
-  }
+  dense_columns(u, H + Dg, Wg, H, H, bg, part,
+                [&](int c, float y) { emb[size_t(g) * H + c] = fmaxf(y, 0.f); });
 }
 
 // Block-wide sum in a fixed order: every thread contributes v, thread 0's tree is the same for
@@ -137,9 +162,7 @@ __device__ float mlp_scalar(const float* x, int in, int hid, const float* __rest
                             const float* __restrict__ b1, const float* __restrict__ w2,
                             const float* __restrict__ b2, float* scratch) {
   float contrib = 0.f;
-  for (int c = threadIdx.x; c < hid; c += blockDim.x) {
-    contrib += fmaxf(column_dot(x, in, W1, hid, c, b1[c]), 0.f) * w2[c];
-  }
+  dense_columns(x, in, W1, hid, hid, b1, scratch, [&](int c, float y) { contrib += fmaxf(y, 0.f) * w2[c]; });
   return block_sum(contrib, scratch) + b2[0];
 }
 
@@ -375,7 +398,7 @@ int launch_readout(const Dims& d, const void* h, const int32_t* chunk_row0, cons
 int launch_global_update(const Dims& d, const float* partial, const int32_t* graph_chunk_off,
                          const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st) {
   if (B <= 0) return 0;
-  k_global_update<<<B, 256, sizeof(float) * size_t(d.H + d.Dg), st>>>(partial, graph_chunk_off, g0,
+  k_global_update<<<B, 256, sizeof(float) * size_t(d.H + d.Dg + 256), st>>>(partial, graph_chunk_off, g0,
                                                                       w.Wg, w.bg, emb, d.H, d.Dg);
   return 1;
 }
@@ -383,7 +406,7 @@ int launch_global_update(const Dims& d, const float* partial, const int32_t* gra
 int launch_global_update_blocks(const Dims& d, const float* partial, const int32_t* node_off, int32_t nblocks,
                                 const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st) {
   if (B <= 0) return 0;
-  k_global_update_blocks<<<B, 256, sizeof(float) * size_t(d.H + d.Dg), st>>>(partial, node_off, nblocks, g0,
+  k_global_update_blocks<<<B, 256, sizeof(float) * size_t(d.H + d.Dg + 256), st>>>(partial, node_off, nblocks, g0,
                                                                              w.Wg, w.bg, emb, d.H, d.Dg);
   return 1;
 }
@@ -397,7 +420,9 @@ int launch_heads(const Dims& d, const DevWeights& w, const float* emb, const int
                                                                     logit_ws, d.H, d.Hm);
   float* cand_sum = logit_ws + B;                 // [num_envs x H], behind the per-graph logits
   k_candidate_sum<<<dim3(num_envs, (d.H + 31) / 32), 1024, 0, st>>>(emb, env_off, mask, cand_sum, d.H, d.A);
-  const int nt = pow2_threads(d.H > d.A + 1 ? d.H : d.A + 1);
+  int want = d.H > d.A + 1 ? d.H : d.A + 1;
+  if (want < 256) want = 256;               // enough threads to split the value head's dense map
+  const int nt = pow2_threads(want);
   const size_t smem = sizeof(unsigned long long) * size_t(nt + 1) + sizeof(float) * size_t(nt + 2 * d.H);
   k_env_policy<<<num_envs, nt, smem, st>>>(emb, logit_ws, cand_sum, env_off, mask, w.vW1, w.vb1, w.vw2,
                                            w.vb2, probs, value, action, d.H, d.Hm, d.A, seed, step, status);

@@ -202,7 +202,7 @@ __global__ void __launch_bounds__(kRowThreads, (VPL == 1 ? 4 : 2))
 k_aggregate(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
             const T* __restrict__ Z, const float2* __restrict__ scores,
             const float* __restrict__ bias, T* __restrict__ h_out, int H, int K, Window win,
-            const int32_t* __restrict__ self_idx) {
+            const int32_t* __restrict__ self_idx, int block_rows) {
   constexpr int VEC = VecOf<T>::N;
   constexpr int RPW = 32 / LPR;
   constexpr int WARPS = kRowThreads / 32;
@@ -228,9 +228,11 @@ k_aggregate(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
 
   // blocks of rows: as many rows (up to 32) as keep the block's producer ids within the cache;
   // a single row with more producers than that is walked straight from global memory
-  int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * kAggBlockRows;
+  // block_rows <= kAggBlockRows rows per warp and pass: fewer when the batch is small, so that every
+  // warp of the grid has work
+  int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * block_rows;
   while (r0 < win.row_end) {
-    const int nr = int(min(int64_t(kAggBlockRows), win.row_end - r0));
+    const int nr = int(min(int64_t(block_rows), win.row_end - r0));
     __syncwarp();                                   // the previous block's reads are done
     if (lane < nr) s_rp[wib][lane] = __ldg(rowptr + r0 + lane);
     if (lane == 0) s_rp[wib][nr] = __ldg(rowptr + r0 + nr);
@@ -270,7 +272,7 @@ k_aggregate(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
         store_vec(h_out + size_t(lrow) * H + c0[v], o);
       }
     }
-    r0 += int64_t(warps_total) * kAggBlockRows;
+    r0 += int64_t(warps_total) * block_rows;
   }
 }
 
@@ -345,10 +347,19 @@ int launch_aggregate(const Dims& d, const int32_t* rowptr, const int32_t* col, c
                                        self_idx);
     if (k >= 0 || d.zmerged) return k;       // with merged rows there is no other kernel to fall back to
   }
+  // rows per warp and pass: the 32 of a full block, fewer for small batches (a multiple of the rows a
+  // warp holds at once)
+  const int64_t warps_avail = int64_t(kNumSMs) * 8 * (kRowThreads / 32);
 #define CALL(TY_, LPR, VPL)                                                                        \
-  k_aggregate<TY_, LPR, VPL><<<row_grid(rows, kAggBlockRows), kRowThreads, 0, st>>>(                \
-      rowptr, col, static_cast<const TY_*>(Z), reinterpret_cast<const float2*>(scores), bias,       \
-      static_cast<TY_*>(h_out), d.H, d.K, win, self_idx)
+  do {                                                                                             \
+    const int rpw_ = 32 / LPR;                                                                     \
+    int64_t br_ = (rows + warps_avail - 1) / warps_avail;                                          \
+    br_ = ((br_ + rpw_ - 1) / rpw_) * rpw_;                                                        \
+    if (br_ > kAggBlockRows) br_ = kAggBlockRows;                                                  \
+    k_aggregate<TY_, LPR, VPL><<<row_grid(rows, int(br_)), kRowThreads, 0, st>>>(                  \
+        rowptr, col, static_cast<const TY_*>(Z), reinterpret_cast<const float2*>(scores), bias,    \
+        static_cast<TY_*>(h_out), d.H, d.K, win, self_idx, int(br_));                              \
+  } while (0)
   if (d.dtype == XRL_BF16) XRL_ROW_DISPATCH(bf16, d.H, CALL);
   else XRL_ROW_DISPATCH(float, d.H, CALL);
 #undef CALL
