@@ -37,6 +37,10 @@ __device__ __forceinline__ void dense_columns(const float* x, int in, const floa
   int CP = 32;
   while (CP < ncols && CP < nt) CP <<= 1;
   const int P = nt / CP, cl = tid % CP, p = tid / CP;
+  if (P == 1) {                                  // as many columns as threads (or more): no split, no barriers
+    for (int c = tid; c < ncols; c += nt) emit(c, column_dot(x, in, W, ld, c, bias[c]));
+    return;
+  }
   const int k0 = int((int64_t(in) * p) / P), k1 = int((int64_t(in) * (p + 1)) / P);
   for (int c0 = 0; c0 < ncols; c0 += CP) {
     const int c = c0 + cl;
