@@ -131,17 +131,17 @@ class ClockSampler:
 
 def oracle_sample_run(batch, blob, graphs, threads):
     """Time the CPU oracle (as it stands) on `graphs` whole graphs of the workload.  Returns
-    (seconds, threads used).  The heads are evaluated on the sampled graphs' environment only if
-    the sample covers it; the encoder dominates either way."""
+    (seconds, graphs, their embeddings).  The heads are evaluated on the sampled graphs' environment
+    only if the sample covers it; the encoder dominates either way."""
     from oracle import xrl_oracle as xo
     m = batch["model"]
     st, packed = xo.pack(batch)
     assert st == 0
     sel = np.arange(min(graphs, batch["num_graphs"]), dtype=np.int32)
     t0 = time.perf_counter()
-    xo.encode(m, blob, batch, packed, sel=sel, threads=threads)
+    out = xo.encode(m, blob, batch, packed, sel=sel, threads=threads)
     dt = time.perf_counter() - t0
-    return dt, len(sel)
+    return dt, len(sel), out["emb"]
 
 
 def run_reference(args, cfg_id):
@@ -211,12 +211,12 @@ def main():
     blob, _ = configs.make_weights(m, 1000 + cfg_id, readout_scale=1.0 / float(batch["n_nodes"].mean()))
 
     # ---- CPU baseline first (before the first CUDA call): the oracle on a bounded sample ----------
-    cpu = None
+    cpu, cpu_emb = None, None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import xrl_oracle as xo
         threads = min(os.cpu_count() or 1, xo.num_threads())
         n_s = min(B, {1: 8, 2: 64, 3: 256}.get(cfg_id, 24 * threads))     # ~10-20 s of CPU work on cfg 4/5
-        dt, g = oracle_sample_run(batch, blob, n_s, threads)
+        dt, g, cpu_emb = oracle_sample_run(batch, blob, n_s, threads)
         no = np.concatenate([[0], np.cumsum(batch["n_nodes"])]); eo = np.concatenate([[0], np.cumsum(batch["n_edges"])])
         cpu = {"value": g / dt, "unit": "graphs/s", "cores": threads, "kind": "oracle",
                "sample": f"first {g} graphs of the same batch ({int(no[g])} nodes, {int(eo[g])} edges), "
@@ -280,6 +280,15 @@ def main():
     launches = xrl.xrl_launch_counts(agent.ctx)
     status = agent.device_status()
     assert status == 0, f"device status {status}"
+    # observed error of the timed configuration against the oracle's embeddings of the sampled graphs
+    parity = None
+    if cpu_emb is not None:
+        got = device_step(0)["emb"][:len(cpu_emb)].double().cpu().numpy()
+        atol, rtol = (2e-2, 2e-2) if bf16 else (1e-4, 1e-3)
+        err = np.abs(got - cpu_emb)
+        parity = {"graphs": int(len(cpu_emb)), "output": "graph_emb", "max_abs_err": float(err.max()),
+                  "max_err_over_tol": float((err / (atol + rtol * np.abs(cpu_emb))).max()),
+                  "atol": atol, "rtol": rtol}
 
     # ---- delta encoding of the candidates (same outputs, work only where a rewrite can reach) --------
     delta = None
@@ -400,6 +409,8 @@ def main():
         line["delta"] = delta
     if cpu:
         line["cpu_baseline"] = cpu
+    if parity:
+        line["parity"] = parity
     print(json.dumps(line))
     agent.close()
     if world > 1:

@@ -220,6 +220,32 @@ def test_degenerate_batches(xo):
     assert np.all(got["probs"][want["probs"] == 0] == 0.0)
 
 
+@pytest.mark.parametrize("H,K,dtype", [(256, 8, "bf16"), (256, 4, "bf16"), (256, 16, "bf16"), (128, 4, "fp32")])
+def test_busy_consumers_on_512_byte_rows(xo, H, K, dtype):
+    """Consumers with more producers than the gather list of the 512-byte-row aggregate holds (160 entries
+    per 32 rows), alone and next to ordinary rows, on every row geometry that kernel takes; with the last
+    attention layer fused with the per-graph sum (L = 2) and without it (intermediate layer)."""
+    rng = dags.make_rng(23)
+    bf = dtype == "bf16"
+    n = 700
+    # node n - 1 has 400 producers, node n - 2 has 170, node 300 has 161 (with repeats), the rest few
+    src = [np.arange(0, 400), np.arange(100, 270), rng.integers(0, 299, 161)]
+    dst = [np.full(400, n - 1), np.full(170, n - 2), np.full(161, 300)]
+    base = dags.random_dag(rng, n, 32, 8, bf, window=12)
+    busy = dict(base, edge_src=np.concatenate([base["edge_src"]] + src).astype(np.int32),
+                edge_dst=np.concatenate([base["edge_dst"]] + dst).astype(np.int32))
+    graphs = [busy, dags.random_dag(rng, 90, 32, 8, bf), busy]
+    b = dags.flatten(graphs, [0, 3], 2)
+    b["model"] = dict(configs.MODEL[1], H=H, K=K, dtype=dtype, L=2, Hm=48, A_max=2)
+    blob, _ = configs.make_weights(b["model"], 5, readout_scale=1.0 / 500.0)
+    got = gpu_util.run_gpu(b, blob)
+    want = xo.forward(b["model"], blob, b)
+    assert got["status"] == 0
+    gpu_util.assert_close(got["emb"], want["emb"], dtype, "graph_emb")
+    gpu_util.assert_close(got["probs"], want["probs"], dtype, "probs")
+    gpu_util.assert_close(got["value"], want["value"], dtype, "value")
+
+
 def test_mask_beyond_candidates_raises_device_status():
     batch = configs.make_batch(1, candidates=5)
     blob, _ = gpu_util.default_weights(batch, 2)
