@@ -41,6 +41,7 @@ enum { XO_OK = 0, XO_INVALID_ARG = 1, XO_BAD_GRAPH = 2 };
 
 struct Model {
   int32_t T, S, H, K, L, Hm, Dg, dtype;  // dtype: 0 fp32, 1 bf16 storage
+  int32_t Hm2;                           // second hidden width of the heads' MLPs, 0 = one hidden layer
 };
 
 // bfloat16 = the upper 16 bits of an IEEE binary32; round to nearest, ties to even.
@@ -64,8 +65,8 @@ struct Weights {
   const float* W0; const float* b0;
   std::vector<const float*> W, a_src, a_dst, b;
   const float* Wg; const float* bg;
-  const float* pW1; const float* pb1; const float* pw2; const float* pb2;
-  const float* vW1; const float* vb1; const float* vw2; const float* vb2;
+  const float* pW1; const float* pb1; const float* pWh; const float* pbh; const float* pw2; const float* pb2;
+  const float* vW1; const float* vb1; const float* vWh; const float* vbh; const float* vw2; const float* vb2;
 };
 
 Weights slice(const Model& m, const float* blob) {
@@ -82,8 +83,14 @@ Weights slice(const Model& m, const float* blob) {
   }
   w.Wg = take(int64_t(m.H + m.Dg) * m.H);
   w.bg = take(m.H);
-  w.pW1 = take(int64_t(m.H) * m.Hm); w.pb1 = take(m.Hm); w.pw2 = take(m.Hm); w.pb2 = take(1);
-  w.vW1 = take(int64_t(2 * m.H) * m.Hm); w.vb1 = take(m.Hm); w.vw2 = take(m.Hm); w.vb2 = take(1);
+  // heads: Linear(in, Hm), ReLU, [Linear(Hm, Hm2), ReLU,] Linear(last hidden, 1)
+  const int last = m.Hm2 > 0 ? m.Hm2 : m.Hm;
+  w.pW1 = take(int64_t(m.H) * m.Hm); w.pb1 = take(m.Hm);
+  w.pWh = take(int64_t(m.Hm) * m.Hm2); w.pbh = take(m.Hm2);
+  w.pw2 = take(last); w.pb2 = take(1);
+  w.vW1 = take(int64_t(2 * m.H) * m.Hm); w.vb1 = take(m.Hm);
+  w.vWh = take(int64_t(m.Hm) * m.Hm2); w.vbh = take(m.Hm2);
+  w.vw2 = take(last); w.vb2 = take(1);
   return w;
 }
 
@@ -201,12 +208,24 @@ void encode_graph(const Model& m, const Weights& w, int32_t lo, int32_t hi,
   }
 }
 
-double mlp_scalar(const double* x, int in, int hid, const float* W1, const float* b1,
-                  const float* w2, const float* b2) {
-  double out = double(b2[0]);
+// The heads' MLP (Section 3.3.2: "two layers"; the hyper-parameter table lists hidden sizes [256, 64]):
+// y1 = ReLU(W1^T x + b1); with a second hidden width, y2 = ReLU(Wh^T y1 + bh); out = w2 . y_last + b2.
+double mlp_scalar(const double* x, int in, int hid, int hid2, const float* W1, const float* b1,
+                  const float* Wh, const float* bh, const float* w2, const float* b2) {
+  std::vector<double> y1(hid);
   for (int c = 0; c < hid; ++c) {
     double acc = double(b1[c]);
     for (int k = 0; k < in; ++k) acc += x[k] * double(W1[size_t(k) * hid + c]);
+    y1[c] = relu(acc);
+  }
+  double out = double(b2[0]);
+  if (hid2 <= 0) {
+    for (int c = 0; c < hid; ++c) out += y1[c] * double(w2[c]);
+    return out;
+  }
+  for (int c = 0; c < hid2; ++c) {
+    double acc = double(bh[c]);
+    for (int k = 0; k < hid; ++k) acc += y1[k] * double(Wh[size_t(k) * hid2 + c]);
     out += relu(acc) * double(w2[c]);
   }
   return out;
@@ -327,7 +346,7 @@ int xo_policy_value(const Model* m, const float* weights, int32_t num_envs,
     for (int a = 0; a < A1; ++a) {
       const bool valid = (a == A_max) || mask[size_t(e) * A_max + a];
       const int g = (a == A_max) ? cur : cur + 1 + a;
-      lg[a] = valid ? mlp_scalar(graph_emb + size_t(g) * H, H, m->Hm, w.pW1, w.pb1, w.pw2, w.pb2)
+      lg[a] = valid ? mlp_scalar(graph_emb + size_t(g) * H, H, m->Hm, m->Hm2, w.pW1, w.pb1, w.pWh, w.pbh, w.pw2, w.pb2)
                     : -INFINITY;
       if (lg[a] > mx) mx = lg[a];
     }
@@ -349,7 +368,7 @@ int xo_policy_value(const Model* m, const float* weights, int32_t num_envs,
       }
     if (nv > 0)
       for (int c = 0; c < H; ++c) u[H + c] /= double(nv);
-    value[e] = mlp_scalar(u.data(), 2 * H, m->Hm, w.vW1, w.vb1, w.vw2, w.vb2);
+    value[e] = mlp_scalar(u.data(), 2 * H, m->Hm, m->Hm2, w.vW1, w.vb1, w.vWh, w.vbh, w.vw2, w.vb2);
   }
   return XO_OK;
 }

@@ -72,5 +72,8 @@ def encode_graph(g, W, m, g_attr=None):
     return global_update(h, W, m, g_attr)
 
 
-def mlp(x, W1, b1, w2, b2):
-    return float(np.maximum(x @ W1.astype(np.float64) + b1, 0.0) @ w2.astype(np.float64) + b2[0])
+def mlp(x, W1, b1, w2, b2, Wh=None, bh=None):
+    y = np.maximum(x @ W1.astype(np.float64) + b1, 0.0)
+    if Wh is not None:                      # second hidden layer
+        y = np.maximum(y @ Wh.astype(np.float64) + bh, 0.0)
+    return float(y @ w2.astype(np.float64) + b2[0])

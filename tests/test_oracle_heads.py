@@ -1,5 +1,6 @@
 """Pins for the oracle's policy / value heads and masked softmax (Sections 3.3.2, 3.3.3)."""
 import numpy as np
+import pytest
 
 import dense_ref
 from workloads import configs
@@ -7,8 +8,8 @@ from workloads import configs
 M = dict(T=6, S=8, H=16, K=2, L=1, Hm=12, Dg=1, dtype="fp32", A_max=6)
 
 
-def _setup(num_envs, cands, seed=0, A=6):
-    m = dict(M, A_max=A)
+def _setup(num_envs, cands, seed=0, A=6, Hm2=0):
+    m = dict(M, A_max=A, Hm2=Hm2)
     blob, W = configs.make_weights(m, 30 + seed)
     rng = np.random.default_rng(seed)
     env_off = np.concatenate([[0], np.cumsum([c + 1 for c in cands])]).astype(np.int32)
@@ -20,8 +21,14 @@ def _setup(num_envs, cands, seed=0, A=6):
     return m, blob, W, batch, emb
 
 
-def test_policy_matches_bruteforce_mlp_and_softmax(xo):
-    m, blob, W, batch, emb = _setup(2, [4, 6])
+def _second(W, p):
+    """The optional second hidden layer of head `p` as keyword arguments of dense_ref.mlp."""
+    return dict(Wh=W[p + "Wh"], bh=W[p + "bh"]) if (p + "Wh") in W else {}
+
+
+@pytest.mark.parametrize("Hm2", [0, 5])
+def test_policy_matches_bruteforce_mlp_and_softmax(xo, Hm2):
+    m, blob, W, batch, emb = _setup(2, [4, 6], Hm2=Hm2)
     batch["mask"][0, 1] = 0
     st, logits, probs, value = xo.policy_value(m, blob, batch, emb)
     assert st == 0
@@ -32,8 +39,8 @@ def test_policy_matches_bruteforce_mlp_and_softmax(xo):
         ell = {}
         for a in range(C):
             if batch["mask"][e, a]:
-                ell[a] = dense_ref.mlp(emb[cur + 1 + a], W["pW1"], W["pb1"], W["pw2"], W["pb2"])
-        ell[A] = dense_ref.mlp(emb[cur], W["pW1"], W["pb1"], W["pw2"], W["pb2"])
+                ell[a] = dense_ref.mlp(emb[cur + 1 + a], W["pW1"], W["pb1"], W["pw2"], W["pb2"], **_second(W, "p"))
+        ell[A] = dense_ref.mlp(emb[cur], W["pW1"], W["pb1"], W["pw2"], W["pb2"], **_second(W, "p"))
         z = sum(np.exp(v) for v in ell.values())
         for a in range(A + 1):
             if a in ell:
@@ -46,7 +53,40 @@ def test_policy_matches_bruteforce_mlp_and_softmax(xo):
         # value: [current || mean of valid candidates] through the value MLP
         valid = [a for a in range(C) if batch["mask"][e, a]]
         u = np.concatenate([emb[cur], np.mean([emb[cur + 1 + a] for a in valid], axis=0)])
-        assert abs(value[e] - dense_ref.mlp(u, W["vW1"], W["vb1"], W["vw2"], W["vb2"])) < 1e-12
+        assert abs(value[e] - dense_ref.mlp(u, W["vW1"], W["vb1"], W["vw2"], W["vb2"], **_second(W, "v"))) < 1e-12
+
+
+def test_second_hidden_layer_reduces_to_one_layer_when_it_is_the_identity(xo):
+    """Hidden sizes [Hm, Hm] with Wh = I, bh = 0: the first layer's outputs are >= 0, so the second
+    layer passes them through and the heads equal the one-hidden-layer heads with the same w2, b2.
+    With Wh = 0 the output is the constant w2 . ReLU(bh) + b2 whatever the input."""
+    m1, blob1, W1, batch, emb = _setup(2, [3, 5], seed=4)
+    Hm = m1["Hm"]
+    m2 = dict(m1, Hm2=Hm)
+    _, W2 = configs.make_weights(m2, 99)
+    for k in W1:
+        W2[k] = W1[k]
+    for p in "pv":
+        W2[p + "Wh"] = np.eye(Hm, dtype=np.float32)
+        W2[p + "bh"] = np.zeros(Hm, np.float32)
+    blob2 = np.concatenate([W2[n].ravel() for n, _ in configs.weight_layout(m2)]).astype(np.float32)
+    _, lg1, p1, v1 = xo.policy_value(m1, blob1, batch, emb)
+    _, lg2, p2, v2 = xo.policy_value(m2, blob2, batch, emb)
+    np.testing.assert_allclose(lg2, lg1, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(p2, p1, rtol=0, atol=1e-15)
+    np.testing.assert_allclose(v2, v1, rtol=0, atol=1e-13)
+    for p in "pv":
+        W2[p + "Wh"] = np.zeros((Hm, Hm), np.float32)
+        W2[p + "bh"] = np.linspace(-1, 1, Hm).astype(np.float32)
+    blob3 = np.concatenate([W2[n].ravel() for n, _ in configs.weight_layout(m2)]).astype(np.float32)
+    _, lg3, p3, v3 = xo.policy_value(m2, blob3, batch, emb)
+    const_p = float(np.maximum(W2["pbh"].astype(np.float64), 0) @ W2["pw2"].astype(np.float64) + W2["pb2"][0])
+    const_v = float(np.maximum(W2["vbh"].astype(np.float64), 0) @ W2["vw2"].astype(np.float64) + W2["vb2"][0])
+    assert np.all(np.abs(lg3[np.isfinite(lg3)] - const_p) < 1e-13)
+    assert np.all(np.abs(v3 - const_v) < 1e-13)
+    # equal logits: the valid actions and No-Op share the probability evenly
+    for e, c in enumerate([3, 5]):
+        np.testing.assert_allclose(p3[e][p3[e] > 0], 1.0 / (c + 1), rtol=1e-13)
 
 
 def test_identical_candidates_and_permutation(xo):

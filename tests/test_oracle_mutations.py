@@ -28,6 +28,12 @@ MUTATIONS = [
      "for (int c = 0; c < H; ++c) u[c] /= double(n > 0 ? n : 1);\n  for (int c = 0; c < m.Dg; ++c) u[H + c] = g_attr ? g_attr[c] : 0.0;"),
     ("global attribute ignored", "u[H + c] = g_attr ? g_attr[c] : 0.0;", "u[H + c] = 0.0;"),
     ("bf16 truncation instead of rounding", "u += 0x7FFFu + lsb;", "u += 0u * lsb;"),
+    ("second hidden layer without its ReLU", "out += relu(acc) * double(w2[c]);", "out += acc * double(w2[c]);"),
+    ("second hidden layer's bias dropped", "double acc = double(bh[c]);", "double acc = 0.0;"),
+    ("second hidden layer reads the first layer transposed", "acc += y1[k] * double(Wh[size_t(k) * hid2 + c]);",
+     "acc += y1[k] * double(Wh[size_t(c) * hid + k]);"),
+    ("masked candidates counted in the value head's mean", "if (mask[size_t(e) * A_max + a]) {\n        ++nv;",
+     "{\n        ++nv;"),
 ]
 
 
@@ -59,6 +65,20 @@ def _pins_hold(xo):
             want = dense_ref.encode_graph(g, W, m, g0[gi])
             if not np.allclose(out["emb"][gi], want, rtol=1e-10, atol=1e-11):
                 return False
+    # heads with two hidden layers (widths 7 and 7) against the brute-force MLP, one candidate masked
+    m = dict(T=6, S=8, H=16, K=2, L=0, Hm=7, Hm2=7, Dg=1, dtype="fp32", A_max=3)
+    blob, W = configs.make_weights(m, 17)
+    emb = np.random.default_rng(2).random((4, 16)) * 2.0
+    hb = {"env_off": np.array([0, 4], np.int32), "mask": np.array([[1, 0, 1]], np.uint8)}
+    st, logits, probs, value = xo.policy_value(m, blob, hb, emb)
+    if st != 0:
+        return False
+    ell = [dense_ref.mlp(emb[g], W["pW1"], W["pb1"], W["pw2"], W["pb2"], W["pWh"], W["pbh"]) for g in (1, 3, 0)]
+    if not np.allclose(logits[0, [0, 2, 3]], ell, rtol=1e-12, atol=1e-12):
+        return False
+    u = np.concatenate([emb[0], (emb[1] + emb[3]) / 2.0])
+    if abs(value[0] - dense_ref.mlp(u, W["vW1"], W["vb1"], W["vw2"], W["vb2"], W["vWh"], W["vbh"])) > 1e-12:
+        return False
     return True
 
 

@@ -78,17 +78,20 @@ def make_batch(cfg_id, candidates=None, envs=None, seed=None, mask_fraction=None
 #   W0 [(S+T+S) x H], b0 [H]
 #   per layer: W [H x H], a_src [H], a_dst [H], b [H]
 #   Wg [(H+Dg) x H], bg [H]
-#   policy: W1 [H x Hm], b1 [Hm], w2 [Hm], b2 [1]
-#   value : W1 [2H x Hm], b1 [Hm], w2 [Hm], b2 [1]
+#   policy: W1 [H x Hm], b1 [Hm], (Wh [Hm x Hm2], bh [Hm2] if Hm2 > 0), w2 [last hidden], b2 [1]
+#   value : W1 [2H x Hm], b1 [Hm], (Wh [Hm x Hm2], bh [Hm2] if Hm2 > 0), w2 [last hidden], b2 [1]
 def weight_layout(m):
     S, T, H, K, L, Hm, Dg = m["S"], m["T"], m["H"], m["K"], m["L"], m["Hm"], m["Dg"]
+    Hm2 = int(m.get("Hm2", 0))
+    last = Hm2 if Hm2 > 0 else Hm
+    second = lambda p: [(p + "Wh", (Hm, Hm2)), (p + "bh", (Hm2,))] if Hm2 > 0 else []
     items = [("W0", (2 * S + T, H)), ("b0", (H,))]
     for l in range(L):
         items += [(f"W{l + 1}", (H, H)), (f"a_src{l + 1}", (H,)), (f"a_dst{l + 1}", (H,)),
                   (f"b{l + 1}", (H,))]
     items += [("Wg", (H + Dg, H)), ("bg", (H,)),
-              ("pW1", (H, Hm)), ("pb1", (Hm,)), ("pw2", (Hm,)), ("pb2", (1,)),
-              ("vW1", (2 * H, Hm)), ("vb1", (Hm,)), ("vw2", (Hm,)), ("vb2", (1,))]
+              ("pW1", (H, Hm)), ("pb1", (Hm,))] + second("p") + [("pw2", (last,)), ("pb2", (1,)),
+              ("vW1", (2 * H, Hm)), ("vb1", (Hm,))] + second("v") + [("vw2", (last,)), ("vb2", (1,))]
     return items
 
 
