@@ -152,7 +152,7 @@ def run_reference(args, cfg_id):
     from oracle import xrl_oracle as xo
     cores = os.cpu_count() or 1
     threads = min(cores, xo.num_threads())
-    sample_graphs = {1: 8, 2: 64, 3: 64, 4: max(16, 2 * threads), 5: max(32, 2 * threads)}[cfg_id]
+    sample_graphs = {1: 8, 2: 64, 3: 64, 4: max(16, 2 * threads), 5: max(32, 2 * threads), 6: 27}[cfg_id]
     cand = max(1, sample_graphs - 1)
     batch = configs.make_batch(cfg_id, candidates=min(cand, configs.FULL[cfg_id][0]), envs=1)
     m = batch["model"]
@@ -188,7 +188,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--config", type=int, default=4, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--config", type=int, default=4, choices=[1, 2, 3, 4, 5, 6])
     ap.add_argument("--impl", default="xrl", choices=["xrl", "reference"])
     ap.add_argument("--candidates", type=int, default=None, help="shrink the workload (profiling)")
     ap.add_argument("--envs", type=int, default=None)

@@ -56,14 +56,19 @@ enum { XRL_MEM_HOST = 0, XRL_MEM_DEVICE = 1 };
 
 /* Model and capacity description (plain data, copied by xrl_create).
  * Supported shapes: hidden a multiple of 32 in [32, 512]; hidden / heads a multiple of 8;
- * num_shape_feats = 8; num_op_types <= 256; mlp_hidden in [1, 1024]; global_dim in [0, 16]. */
+ * num_shape_feats = 8; num_op_types <= 256; mlp_hidden in [1, 1024]; mlp_hidden2 in [0, 1024];
+ * global_dim in [0, 16]. */
 typedef struct {
   int32_t num_op_types;    /* T: size of the operator table (one-hot node attribute)          */
   int32_t num_shape_feats; /* S: shape features per node (attribute of its outgoing edges)    */
   int32_t hidden;          /* H                                                               */
   int32_t heads;           /* K, must divide H                                                */
   int32_t layers;          /* L: number of graph-attention layers (the paper's k), >= 0       */
-  int32_t mlp_hidden;      /* Hm: hidden width of both two-layer MLP heads                    */
+  int32_t mlp_hidden;      /* Hm: (first) hidden width of the policy and value MLPs           */
+  int32_t mlp_hidden2;     /* Hm2: second hidden width, 0 = none.  Section 3.3.2 describes the heads
+                              as two-layer MLPs, the hyper-parameter table lists hidden sizes
+                              [256, 64]: (Hm, Hm2) = (256, 64) is that table's model, Hm2 = 0 the
+                              one-hidden-layer reading                                             */
   int32_t global_dim;      /* Dg: width of the per-graph global attribute (paper: value 0)    */
   int32_t dtype;           /* XRL_FP32, or XRL_BF16 = bf16 storage with fp32 accumulation     */
   int32_t max_actions;     /* A_max: padded number of candidate slots; No-Op is index A_max   */
@@ -100,8 +105,10 @@ void xrl_destroy(xrl_ctx* ctx);
  *   W0 [(S+T+S) x H], b0 [H]                       Eq. 6; input = [edge aggregate | one-hot op | own shape]
  *   per layer: W [H x H], a_src [H], a_dst [H], b [H]   Eq. 7; a_* are K per-head vectors of width H/K
  *   Wg [(H+Dg) x H], bg [H]                        Eq. 8; input = [node sum | global attribute]
- *   policy: W1 [H x Hm], b1 [Hm], w2 [Hm], b2 [1]
- *   value:  W1 [2H x Hm], b1 [Hm], w2 [Hm], b2 [1]      input = [current graph | mean of valid candidates] */
+ *   policy: W1 [H x Hm], b1 [Hm], (Wh [Hm x Hm2], bh [Hm2] when Hm2 > 0), w2 [last hidden width], b2 [1]
+ *   value:  W1 [2H x Hm], b1 [Hm], (Wh, bh likewise), w2 [last hidden width], b2 [1]
+ *           input = [current graph | mean of valid candidates]
+ *   A head computes w2 . ReLU(Wh^T ReLU(W1^T x + b1) + bh) + b2, without the middle map when Hm2 = 0. */
 xrl_status xrl_weights_size(const xrl_ctx* ctx, size_t* bytes);
 /* Upload the blob (HOST, fp32).  With XRL_BF16 the library rounds W0 and the layer matrices W
  * to bf16 (nearest even) once; everything else stays fp32.  Synchronous. */

@@ -38,7 +38,7 @@ class XrlError(RuntimeError):
 class _ModelConfig(C.Structure):
     _fields_ = [("num_op_types", C.c_int32), ("num_shape_feats", C.c_int32), ("hidden", C.c_int32),
                 ("heads", C.c_int32), ("layers", C.c_int32), ("mlp_hidden", C.c_int32),
-                ("global_dim", C.c_int32), ("dtype", C.c_int32), ("max_actions", C.c_int32),
+                ("mlp_hidden2", C.c_int32), ("global_dim", C.c_int32), ("dtype", C.c_int32), ("max_actions", C.c_int32),
                 ("max_graphs", C.c_int32), ("max_envs", C.c_int32), ("max_nodes", C.c_int64),
                 ("max_edges", C.c_int64)]
 
@@ -116,8 +116,9 @@ def _stream(stream):
 
 
 def model_config(m, max_graphs, max_envs, max_nodes, max_edges):
-    """Build the C config from a dict with keys T, S, H, K, L, Hm, Dg, dtype, A_max."""
-    return _ModelConfig(m["T"], m["S"], m["H"], m["K"], m["L"], m["Hm"], m["Dg"],
+    """Build the C config from a dict with keys T, S, H, K, L, Hm, Dg, dtype, A_max and, optionally,
+    Hm2 (second hidden width of the heads' MLPs, default 0 = one hidden layer)."""
+    return _ModelConfig(m["T"], m["S"], m["H"], m["K"], m["L"], m["Hm"], int(m.get("Hm2", 0)), m["Dg"],
                         XRL_BF16 if m["dtype"] in ("bf16", XRL_BF16) else XRL_FP32, m["A_max"],
                         int(max_graphs), int(max_envs), int(max_nodes), int(max_edges))
 
@@ -317,7 +318,8 @@ def xrl_pack_csr_static(device, num_op_types, n_nodes, n_edges, op, edge_src, ed
 class Agent:
     """One model on one GPU: set weights once, then `step()` per rewrite step.
 
-    m: dict with keys T, S, H, K, L, Hm, Dg, dtype, A_max.  Capacities bound the batch size.
+    m: dict with keys T, S, H, K, L, Hm, Dg, dtype, A_max (and optionally Hm2).  Capacities bound the
+    batch size.
     """
 
     def __init__(self, m, max_graphs, max_envs, max_nodes, max_edges, device=0):

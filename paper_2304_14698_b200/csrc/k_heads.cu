@@ -161,27 +161,34 @@ __device__ float block_sum(float v, float* scratch) {
   return r;
 }
 
-// out = w2 . ReLU(W1^T x + b1) + b2 with x (length `in`) in shared memory; all threads return it.
-__device__ float mlp_scalar(const float* x, int in, int hid, const float* __restrict__ W1,
-                            const float* __restrict__ b1, const float* __restrict__ w2,
-                            const float* __restrict__ b2, float* scratch) {
+// A head's MLP (Section 3.3.2): out = w2 . ReLU(W1^T x + b1) + b2, or with a second hidden width hid2 > 0
+// out = w2 . ReLU(Wh^T ReLU(W1^T x + b1) + bh) + b2.  x (length `in`) and y1 (hid floats, used only when
+// hid2 > 0) are in shared memory; all threads return the result.
+struct Mlp { const float *W1, *b1, *Wh, *bh, *w2, *b2; int hid, hid2; };
+__device__ float mlp_scalar(const float* x, int in, const Mlp& m, float* y1, float* scratch) {
   float contrib = 0.f;
-  dense_columns(x, in, W1, hid, hid, b1, scratch, [&](int c, float y) { contrib += fmaxf(y, 0.f) * w2[c]; });
-  return block_sum(contrib, scratch) + b2[0];
+  if (m.hid2 <= 0) {
+    dense_columns(x, in, m.W1, m.hid, m.hid, m.b1, scratch, [&](int c, float y) { contrib += fmaxf(y, 0.f) * m.w2[c]; });
+  } else {
+    dense_columns(x, in, m.W1, m.hid, m.hid, m.b1, scratch, [&](int c, float y) { y1[c] = fmaxf(y, 0.f); });
+    __syncthreads();
+    dense_columns(y1, m.hid, m.Wh, m.hid2, m.hid2, m.bh, scratch,
+                  [&](int c, float y) { contrib += fmaxf(y, 0.f) * m.w2[c]; });
+  }
+  return block_sum(contrib, scratch) + m.b2[0];
 }
 
 // ---- policy MLP: one scalar score per graph -----------------------------------------------------
 __global__ void __launch_bounds__(256)
-k_policy_logit(const float* __restrict__ emb, const float* __restrict__ W1, const float* __restrict__ b1,
-               const float* __restrict__ w2, const float* __restrict__ b2, float* __restrict__ logit,
-               int H, int Hm) {
-  extern __shared__ float sm[];                  // [H] + [blockDim]
+k_policy_logit(const float* __restrict__ emb, const Mlp mlp, float* __restrict__ logit, int H) {
+  extern __shared__ float sm[];                  // [H] + [blockDim] + [hid]
   float* x = sm;
   float* scratch = sm + H;
+  float* y1 = scratch + blockDim.x;
   const int32_t g = blockIdx.x;
   for (int c = threadIdx.x; c < H; c += blockDim.x) x[c] = emb[size_t(g) * H + c];
   __syncthreads();
-  const float v = mlp_scalar(x, H, Hm, W1, b1, w2, b2, scratch);
+  const float v = mlp_scalar(x, H, mlp, y1, scratch);
   if (threadIdx.x == 0) logit[g] = v;
 }
 
@@ -290,14 +297,14 @@ __global__ void __launch_bounds__(1024)
 k_env_policy(const float* __restrict__ emb, const float* __restrict__ logit,
              const float* __restrict__ cand_sum,
              const int32_t* __restrict__ env_off, const uint8_t* __restrict__ mask,
-             const float* __restrict__ vW1, const float* __restrict__ vb1,
-             const float* __restrict__ vw2, const float* __restrict__ vb2, float* __restrict__ probs,
-             float* __restrict__ value, int32_t* __restrict__ action, int H, int Hm, int A,
+             const Mlp vmlp, float* __restrict__ probs,
+             float* __restrict__ value, int32_t* __restrict__ action, int H, int A,
              uint64_t seed, uint64_t step, int32_t* status) {
   extern __shared__ unsigned long long sm64[];   // [nt + 1] u64, then floats
   const int nt = blockDim.x, tid = threadIdx.x;
   float* scratch = reinterpret_cast<float*>(sm64 + nt + 1);   // [nt]
   float* u = scratch + nt;                                    // [2H]
+  float* y1 = u + 2 * H;                                      // [hid]
   const int32_t e = blockIdx.x;
   const int32_t cur = env_off[e];
   const int32_t C = env_off[e + 1] - cur - 1;
@@ -338,7 +345,7 @@ k_env_policy(const float* __restrict__ emb, const float* __restrict__ logit,
   const float nv = block_sum(cnt, scratch);
   for (int c = tid; c < H; c += nt) u[H + c] = nv > 0.f ? cand_sum[size_t(e) * H + c] / nv : 0.f;
   __syncthreads();
-  const float v = mlp_scalar(u, 2 * H, Hm, vW1, vb1, vw2, vb2, scratch);
+  const float v = mlp_scalar(u, 2 * H, vmlp, y1, scratch);
   if (tid == 0) value[e] = v;
 
   if (action != nullptr) {
@@ -420,16 +427,17 @@ int launch_heads(const Dims& d, const DevWeights& w, const float* emb, const int
                  float* value, int32_t* action, uint64_t seed, uint64_t step, int32_t* status,
                  cudaStream_t st) {
   if (B <= 0 || num_envs <= 0) return 0;
-  k_policy_logit<<<B, 256, sizeof(float) * size_t(d.H + 256), st>>>(emb, w.pW1, w.pb1, w.pw2, w.pb2,
-                                                                    logit_ws, d.H, d.Hm);
+  const Mlp pm{w.pW1, w.pb1, w.pWh, w.pbh, w.pw2, w.pb2, d.Hm, d.Hm2};
+  const Mlp vm{w.vW1, w.vb1, w.vWh, w.vbh, w.vw2, w.vb2, d.Hm, d.Hm2};
+  k_policy_logit<<<B, 256, sizeof(float) * size_t(d.H + 256 + d.Hm), st>>>(emb, pm, logit_ws, d.H);
   float* cand_sum = logit_ws + B;                 // [num_envs x H], behind the per-graph logits
   k_candidate_sum<<<dim3(num_envs, (d.H + 31) / 32), 1024, 0, st>>>(emb, env_off, mask, cand_sum, d.H, d.A);
   int want = d.H > d.A + 1 ? d.H : d.A + 1;
   if (want < 256) want = 256;               // enough threads to split the value head's dense map
   const int nt = pow2_threads(want);
-  const size_t smem = sizeof(unsigned long long) * size_t(nt + 1) + sizeof(float) * size_t(nt + 2 * d.H);
-  k_env_policy<<<num_envs, nt, smem, st>>>(emb, logit_ws, cand_sum, env_off, mask, w.vW1, w.vb1, w.vw2,
-                                           w.vb2, probs, value, action, d.H, d.Hm, d.A, seed, step, status);
+  const size_t smem = sizeof(unsigned long long) * size_t(nt + 1) + sizeof(float) * size_t(nt + 2 * d.H + d.Hm);
+  k_env_policy<<<num_envs, nt, smem, st>>>(emb, logit_ws, cand_sum, env_off, mask, vm, probs, value, action,
+                                           d.H, d.A, seed, step, status);
   return 3;
 }
 

@@ -114,16 +114,18 @@ xrl_status check_config(const xrl_model_config& c) {
     return XRL_ERR_INVALID_ARG;
   if (c.num_shape_feats != kS || c.num_op_types > 256) return XRL_ERR_UNSUPPORTED;
   if (c.hidden % 32 != 0 || c.hidden > 512 || (c.hidden / c.heads) % 8 != 0) return XRL_ERR_UNSUPPORTED;
-  if (c.layers > 64 || c.mlp_hidden > 1024 || c.global_dim > 16) return XRL_ERR_UNSUPPORTED;
+  if (c.mlp_hidden2 < 0) return XRL_ERR_INVALID_ARG;
+  if (c.layers > 64 || c.mlp_hidden > 1024 || c.mlp_hidden2 > 1024 || c.global_dim > 16) return XRL_ERR_UNSUPPORTED;
   if (c.max_actions > (1 << 20)) return XRL_ERR_UNSUPPORTED;
   return XRL_OK;
 }
 
 size_t weight_float_count(const xrl_model_config& c) {
   const size_t S = c.num_shape_feats, T = c.num_op_types, H = c.hidden, L = c.layers,
-               Hm = c.mlp_hidden, Dg = c.global_dim;
-  return (2 * S + T) * H + H + L * (H * H + 3 * H) + (H + Dg) * H + H + (H * Hm + 2 * Hm + 1) +
-         (2 * H * Hm + 2 * Hm + 1);
+               Hm = c.mlp_hidden, Hm2 = c.mlp_hidden2, Dg = c.global_dim;
+  const size_t last = Hm2 > 0 ? Hm2 : Hm, second = Hm * Hm2 + Hm2;     // optional second hidden layer
+  return (2 * S + T) * H + H + L * (H * H + 3 * H) + (H + Dg) * H + H + (H * Hm + Hm + second + last + 1) +
+         (2 * H * Hm + Hm + second + last + 1);
 }
 
 #define XRL_CUDA(call)                      \
@@ -438,7 +440,7 @@ xrl_status xrl_create(const xrl_model_config* cfg, int32_t device, xrl_ctx** out
   ctx->cfg = *cfg;
   ctx->device = device;
   ctx->dims = Dims{cfg->num_op_types, cfg->hidden, cfg->heads, cfg->layers, cfg->mlp_hidden,
-                   cfg->global_dim, cfg->max_actions, cfg->dtype, 0};
+                   cfg->global_dim, cfg->max_actions, cfg->dtype, cfg->mlp_hidden2, 0};
   ctx->weight_floats = weight_float_count(*cfg);
   // XRL_FORCE_SIMT_TRANSFORM=1 keeps the CUDA-core transform for every shape (debugging aid)
   ctx->use_umma = xform_umma_supported(ctx->dims) && getenv("XRL_FORCE_SIMT_TRANSFORM") == nullptr;
@@ -498,7 +500,8 @@ xrl_status xrl_set_weights(xrl_ctx* ctx, const void* host_blob, size_t bytes) {
   XRL_CUDA(cudaSetDevice(ctx->device));
   XRL_CUDA(cudaMemcpy(ctx->w_f32.p, host_blob, bytes, cudaMemcpyHostToDevice));
   const xrl_model_config& c = ctx->cfg;
-  const size_t H = size_t(c.hidden), Hm = size_t(c.mlp_hidden), Dg = size_t(c.global_dim);
+  const size_t H = size_t(c.hidden), Hm = size_t(c.mlp_hidden), Hm2 = size_t(c.mlp_hidden2), Dg = size_t(c.global_dim);
+  const size_t last = Hm2 > 0 ? Hm2 : Hm;
   const size_t F0 = size_t(2 * kS + c.num_op_types), sb = storage_bytes(c.dtype);
   const float* p = ctx->w_f32.as<float>();
   char* store = ctx->w_store.as<char>();
@@ -520,8 +523,10 @@ xrl_status xrl_set_weights(xrl_ctx* ctx, const void* host_blob, size_t bytes) {
     w.layer[l].b = take(H);
   }
   w.Wg = take((H + Dg) * H); w.bg = take(H);
-  w.pW1 = take(H * Hm); w.pb1 = take(Hm); w.pw2 = take(Hm); w.pb2 = take(1);
-  w.vW1 = take(2 * H * Hm); w.vb1 = take(Hm); w.vw2 = take(Hm); w.vb2 = take(1);
+  w.pW1 = take(H * Hm); w.pb1 = take(Hm); w.pWh = take(Hm * Hm2); w.pbh = take(Hm2);
+  w.pw2 = take(last); w.pb2 = take(1);
+  w.vW1 = take(2 * H * Hm); w.vb1 = take(Hm); w.vWh = take(Hm * Hm2); w.vbh = take(Hm2);
+  w.vw2 = take(last); w.vb2 = take(1);
   XRL_CUDA(cudaDeviceSynchronize());
   XRL_CUDA(cudaGetLastError());
   ctx->weights_set = true;

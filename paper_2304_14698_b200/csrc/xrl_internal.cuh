@@ -71,13 +71,14 @@ struct DevWeights {
   const float* b0;
   LayerWeights layer[64];
   const float* Wg; const float* bg;
-  const float *pW1, *pb1, *pw2, *pb2;
-  const float *vW1, *vb1, *vw2, *vb2;
+  const float *pW1, *pb1, *pWh, *pbh, *pw2, *pb2;     // Wh, bh: second hidden layer (Hm2 > 0)
+  const float *vW1, *vb1, *vWh, *vbh, *vw2, *vb2;
 };
 
 struct Dims {
   int T, H, K, L, Hm, Dg, A;
   int dtype;
+  int Hm2;            // second hidden width of the heads' MLPs, 0 = none
   // 1: each row of the Z buffer is followed by the node's K {s_src, s_dst} pairs (row stride
   // H * sizeof(storage) + 8 K bytes), so that one gather brings both; set only when the tensor-core
   // transform and the TMA aggregate kernel handle the shape (the `scores` arguments are then unused)

@@ -8,7 +8,7 @@ import gpu_util
 pytestmark = pytest.mark.gpu
 
 CASES = [(1, {}), (2, {}), (3, dict(candidates=15)), (4, dict(candidates=7)),
-         (5, dict(candidates=7, envs=3))]
+         (5, dict(candidates=7, envs=3)), (6, {})]     # 6: the paper's hyper-parameter table (k = 5, heads [256, 64])
 
 
 def _oracle(xo, batch, blob, **kw):
@@ -86,6 +86,25 @@ def test_global_attribute_input(xo):
         gpu_util.assert_close(emb.cpu().numpy(), want["emb"], "fp32", "emb with g0")
     finally:
         ag.close()
+
+
+@pytest.mark.parametrize("Hm,Hm2", [(256, 64), (64, 256), (1, 1), (1024, 1024), (33, 7)])
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_heads_with_two_hidden_layers(xo, Hm, Hm2, dtype):
+    """Policy and value MLPs with a second hidden layer: widths below, at and above the thread-block
+    size, several environments, masked candidates, sampling."""
+    batch = configs.make_batch(5, candidates=5, envs=3, nodes_scale=0.2)
+    batch["mask"][1, 2] = 0
+    m = dict(batch["model"], H=64, K=2, L=1, Hm=Hm, Hm2=Hm2, dtype=dtype)
+    batch["model"] = m
+    blob, _ = gpu_util.default_weights(batch, 31)
+    got = gpu_util.run_gpu(batch, blob, sample=True, seed=9, step=4)
+    want = xo.forward(m, blob, batch)
+    assert got["status"] == 0
+    gpu_util.assert_close(got["emb"], want["emb"], dtype, "graph_emb")
+    gpu_util.assert_close(got["probs"], want["probs"], dtype, "probs")
+    gpu_util.assert_close(got["value"], want["value"], dtype, "value")
+    assert np.array_equal(got["action"], xo.sample(got["probs"], 9, 4))
 
 
 @pytest.mark.parametrize("H,K,dtype,L", [(32, 1, "fp32", 1), (32, 4, "bf16", 1), (96, 3, "fp32", 2),

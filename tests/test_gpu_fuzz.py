@@ -17,6 +17,7 @@ def _random_case(seed):
     dtype = "bf16" if rng.random() < 0.5 else "fp32"
     T = int(rng.choice([3, 17, 32, 64]))
     m = dict(T=T, S=8, H=H, K=K, L=int(rng.integers(0, 4)), Hm=int(rng.integers(1, 70)),
+             Hm2=int(rng.integers(1, 50)) if rng.random() < 0.4 else 0,
              Dg=int(rng.integers(0, 4)), dtype=dtype, A_max=0)
     nenv = int(rng.integers(1, 4))
     graphs, env_off = [], [0]

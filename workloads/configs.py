@@ -3,7 +3,11 @@ plus seeded weight blobs.  No arithmetic of the encoded method lives here.
 
 model config keys: T (operator types), S (shape features), H (hidden), K (heads),
 L (graph-attention layers), Hm (MLP hidden), Dg (global attribute width),
-dtype ("fp32" | "bf16"), A_max (padded candidate slots).
+dtype ("fp32" | "bf16"), A_max (padded candidate slots); optional Hm2 (second MLP hidden width).
+
+Workload 6 is not one of the benchmark's five: it carries the values of the paper's hyper-parameter
+table (5 attention layers, MLP heads with hidden sizes [256, 64], about 40 operator types) on a step
+of the size its workload table reports for BERT (26 candidates of a transformer-shaped graph).
 """
 from __future__ import annotations
 
@@ -17,17 +21,19 @@ MODEL = {
     3: dict(T=32, S=8, H=128, K=4, L=3, Hm=128, Dg=1, dtype="bf16", A_max=256),
     4: dict(T=64, S=8, H=256, K=8, L=4, Hm=256, Dg=1, dtype="bf16", A_max=1024),
     5: dict(T=64, S=8, H=256, K=8, L=4, Hm=256, Dg=1, dtype="bf16", A_max=128),
+    6: dict(T=40, S=8, H=256, K=8, L=5, Hm=256, Hm2=64, Dg=1, dtype="bf16", A_max=32),
 }
 # candidates per environment and number of environments at full size
-FULL = {1: (7, 1), 2: (63, 1), 3: (255, 1), 4: (1023, 1), 5: (127, 64)}
-NAME = {1: "tiny_step", 2: "transformer_step", 3: "cnn_step", 4: "large_step", 5: "rollout_batch"}
+FULL = {1: (7, 1), 2: (63, 1), 3: (255, 1), 4: (1023, 1), 5: (127, 64), 6: (26, 1)}
+NAME = {1: "tiny_step", 2: "transformer_step", 3: "cnn_step", 4: "large_step", 5: "rollout_batch",
+        6: "paper_step"}
 
 
 def _base_graph(cfg_id, rng, env, m, nodes_scale=1.0):
     bf16 = m["dtype"] == "bf16"
     if cfg_id == 1:
         return dags.random_dag(rng, 64, m["T"], m["S"], bf16)
-    if cfg_id == 2:
+    if cfg_id in (2, 6):
         return dags.transformer_dag(rng, 12, 3, m["T"], m["S"], bf16)
     if cfg_id == 3:
         return dags.cnn_dag(rng, int(1200 * nodes_scale), m["T"], m["S"], bf16)
