@@ -220,6 +220,24 @@ xrl_status xrl_sample(xrl_ctx* ctx, const float* probs, int32_t num_envs, int32_
  * first error code any kernel recorded since the last call, or XRL_OK. */
 xrl_status xrl_last_device_status(xrl_ctx* ctx, void* stream, int32_t* status);
 
+/* ---- one submission per step ------------------------------------------------------------------- */
+
+/* A step of the paper's size (13-50 candidates of a few hundred to a few thousand operators, 5 attention
+ * layers) is some twenty kernels of 2-15 microseconds each: launched one by one, the host's per-launch cost
+ * (about 6 microseconds) is what bounds the step.  Between xrl_graph_begin and xrl_graph_launch the calls
+ * xrl_encode, xrl_policy_value and xrl_sample on this context do not launch anything: their kernels are
+ * recorded (stream capture on a stream the context owns; the `stream` arguments of those calls are ignored).
+ * xrl_graph_launch turns the record into an executable CUDA graph - the first time by instantiating it, later
+ * by updating the previous executable in place, which works as long as the sequence of kernels is the same
+ * (sizes, pointers and launch shapes may all differ) - and submits it to `stream` with one call.
+ * Results, ordering on `stream` and error reporting are those of the direct calls.
+ * xrl_pack*, xrl_encode_delta (which reads sizes back) and the profiling calls are not recordable:
+ * they return XRL_ERR_STATE between begin and launch; so does a second xrl_graph_begin.  On any error
+ * inside the bracket call xrl_graph_launch all the same (it ends the recording) and discard its result.
+ * Errors: INVALID_ARG, STATE (no recording in progress / profiling enabled), CUDA. */
+xrl_status xrl_graph_begin(xrl_ctx* ctx);
+xrl_status xrl_graph_launch(xrl_ctx* ctx, void* stream);
+
 /* Names of the kernels launched by the last xrl_encode / xrl_policy_value / xrl_pack call on
  * this context and how many launches each call made (HOST outputs, any may be NULL). */
 xrl_status xrl_launch_counts(const xrl_ctx* ctx, int64_t* pack, int64_t* encode, int64_t* heads);

@@ -25,6 +25,7 @@ EXPORTED_SYMBOLS = [
     "xrl_batch_free", "xrl_batch_info", "xrl_batch_export", "xrl_encode", "xrl_debug_node_features",
     "xrl_policy_value", "xrl_sample", "xrl_last_device_status", "xrl_launch_counts", "xrl_version",
     "xrl_profile", "xrl_profile_read", "xrl_pack_csr_static", "xrl_encode_delta", "xrl_delta_rows", "xrl_get_weights",
+    "xrl_graph_begin", "xrl_graph_launch",
 ]
 PROFILE_FAMILIES = ["pack", "node_update", "transform", "aggregate", "readout", "heads", "aggregate_readout"]
 
@@ -84,6 +85,8 @@ def load_library():
         "xrl_delta_rows": [vp, C.POINTER(i64), i32],
         "xrl_pack_csr_static": [i32, i32, i32] + [vp] * 6 + [i32] + [vp] * 8,
         "xrl_profile_read": [vp, C.POINTER(C.c_double), C.POINTER(i64), i32],
+        "xrl_graph_begin": [vp],
+        "xrl_graph_launch": [vp, vp],
     }
     for name, args in sigs.items():
         fn = getattr(lib, name)
@@ -275,6 +278,16 @@ def xrl_last_device_status(ctx, stream=None) -> int:
     return int(s.value)
 
 
+def xrl_graph_begin(ctx):
+    """Start recording the kernels of the following xrl_encode / xrl_policy_value / xrl_sample calls."""
+    _check(load_library().xrl_graph_begin(ctx), "xrl_graph_begin")
+
+
+def xrl_graph_launch(ctx, stream=None):
+    """End the recording and submit the recorded kernels to `stream` with one call."""
+    _check(load_library().xrl_graph_launch(ctx, _stream(stream)), "xrl_graph_launch")
+
+
 def xrl_launch_counts(ctx):
     a, b, c = C.c_int64(), C.c_int64(), C.c_int64()
     _check(load_library().xrl_launch_counts(ctx, C.byref(a), C.byref(b), C.byref(c)), "xrl_launch_counts")
@@ -332,6 +345,7 @@ class Agent:
         self.ctx = xrl_create(self.cfg, device)
         self.batch = None
         self._out = {}
+        self._steps = 0
 
     def close(self):
         if self.ctx is not None:
@@ -381,23 +395,45 @@ class Agent:
         self.batch = xrl_pack(self.ctx, graphs, env_off, self.m["dtype"], batch=self.batch)
         return self.batch
 
-    def forward(self, mask, sample=False, seed=0, step=0, g0=None, base_id=None):
+    # steps with at most this many nodes are submitted as one recorded graph (their kernels are so short
+    # that launching them one by one leaves the GPU waiting for the host)
+    GRAPH_MAX_NODES = 65536
+
+    def forward(self, mask, sample=False, seed=0, step=0, g0=None, base_id=None, graph=None):
         """Encode the packed batch and evaluate the heads.  mask: torch CUDA uint8 [envs, A_max].
-        base_id (torch CUDA int32 [N]) switches to delta encoding of the candidates."""
+        base_id (torch CUDA int32 [N]) switches to delta encoding of the candidates.
+        graph: True submits the kernels as one recorded CUDA graph (xrl_graph_begin / xrl_graph_launch),
+        False launches them one by one, None chooses by batch size (never on a context's first step, which
+        also sets kernel attributes, and never with delta encoding or while profiling)."""
         info = xrl_batch_info(self.batch)
         o = self._buffers(info["num_graphs"], info["num_envs"])
-        if base_id is None:
-            xrl_encode(self.ctx, self.batch, o["emb"], g0)
-        else:
-            xrl_encode_delta(self.ctx, self.batch, base_id, o["emb"], g0)
-        xrl_policy_value(self.ctx, self.batch, o["emb"], mask, o["probs"], o["value"],
-                         o["action"] if sample else None, seed, step)
+        if graph is None:
+            graph = self._steps > 0 and info["num_nodes"] <= self.GRAPH_MAX_NODES
+        recording = False
+        if graph and base_id is None:
+            try:
+                xrl_graph_begin(self.ctx)
+                recording = True
+            except XrlError as e:
+                if e.status != 6:              # XRL_ERR_STATE: profiling is on, launch directly
+                    raise
+        try:
+            if base_id is None:
+                xrl_encode(self.ctx, self.batch, o["emb"], g0)
+            else:
+                xrl_encode_delta(self.ctx, self.batch, base_id, o["emb"], g0)
+            xrl_policy_value(self.ctx, self.batch, o["emb"], mask, o["probs"], o["value"],
+                             o["action"] if sample else None, seed, step)
+        finally:
+            if recording:
+                xrl_graph_launch(self.ctx)
+        self._steps += 1
         return o
 
-    def step(self, batch, mask, sample=False, seed=0, step=0, base_id=None):
+    def step(self, batch, mask, sample=False, seed=0, step=0, base_id=None, graph=None):
         """The whole path for one batch: pack -> encode -> policy/value (-> sample)."""
         self.pack(batch)
-        return self.forward(mask, sample, seed, step, base_id=base_id)
+        return self.forward(mask, sample, seed, step, base_id=base_id, graph=graph)
 
     def device_status(self):
         return xrl_last_device_status(self.ctx)

@@ -80,6 +80,10 @@ struct xrl_ctx {
   DeviceBuf dl_ints, dl_col, dl_scan;
   int32_t* dl_host = nullptr;      // pinned: row counts read back per layer
   int64_t delta_rows[65] = {0};    // rows computed per layer by the last xrl_encode_delta
+  // one submission per step: kernels recorded on cap_stream between xrl_graph_begin and xrl_graph_launch
+  cudaStream_t cap_stream = nullptr;
+  cudaGraphExec_t graph_exec = nullptr;
+  bool capturing = false;
 };
 
 struct xrl_batch {
@@ -204,6 +208,7 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
                        const void* shape, const int32_t* edge_src, const int32_t* edge_dst,
                        const int32_t* env_off, int32_t num_envs, void* stream, xrl_batch** out) {
   if (!ctx || !out || !env_off || num_graphs < 0 || num_envs < 0) return XRL_ERR_INVALID_ARG;
+  if (ctx->capturing) return XRL_ERR_STATE;        // packing synchronises with its staging buffers
   if (!graphs && (where != XRL_MEM_HOST && where != XRL_MEM_DEVICE)) return XRL_ERR_INVALID_ARG;
   if (!graphs && num_graphs > 0 && (!n_nodes || !n_edges)) return XRL_ERR_INVALID_ARG;
   const xrl_model_config& c = ctx->cfg;
@@ -485,6 +490,14 @@ void xrl_destroy(xrl_ctx* ctx) {
   ctx->prof.release();
   ctx->dl_ints.release(); ctx->dl_col.release(); ctx->dl_scan.release();
   if (ctx->dl_host) cudaFreeHost(ctx->dl_host);
+  if (ctx->capturing) {                            // a recording left open: end it, drop the record
+    cudaGraph_t g = nullptr;
+    cudaStreamEndCapture(ctx->cap_stream, &g);
+    if (g) cudaGraphDestroy(g);
+    cudaGetLastError();
+  }
+  if (ctx->graph_exec) cudaGraphExecDestroy(ctx->graph_exec);
+  if (ctx->cap_stream) cudaStreamDestroy(ctx->cap_stream);
   delete ctx;
 }
 
@@ -606,7 +619,7 @@ xrl_status xrl_encode(xrl_ctx* ctx, const xrl_batch* b, const float* g0, float* 
   if (s != XRL_OK) return s;
   if (!graph_emb && b->B > 0) return XRL_ERR_INVALID_ARG;
   XRL_CUDA(cudaSetDevice(ctx->device));
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaStream_t st = ctx->capturing ? ctx->cap_stream : static_cast<cudaStream_t>(stream);
   bool fused = false;
   int n = run_node_layers(ctx, b, ctx->cfg.layers, st, true, &fused);
   if (n < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
@@ -637,6 +650,7 @@ xrl_status xrl_encode_delta(xrl_ctx* ctx, const xrl_batch* b, const int32_t* bas
                             float* graph_emb, void* stream) {
   const xrl_status s = check_batch(ctx, b);
   if (s != XRL_OK) return s;
+  if (ctx->capturing) return XRL_ERR_STATE;        // reads the row counts back between layers
   if (!graph_emb && b->B > 0) return XRL_ERR_INVALID_ARG;
   XRL_CUDA(cudaSetDevice(ctx->device));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -757,6 +771,7 @@ xrl_status xrl_debug_node_features(xrl_ctx* ctx, const xrl_batch* b, int32_t num
   const xrl_status s = check_batch(ctx, b);
   if (s != XRL_OK) return s;
   if (num_layers < 0 || num_layers > ctx->cfg.layers || (!host_out && b->N > 0)) return XRL_ERR_INVALID_ARG;
+  if (ctx->capturing) return XRL_ERR_STATE;
   XRL_CUDA(cudaSetDevice(ctx->device));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (run_node_layers(ctx, b, num_layers, st) < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
@@ -781,7 +796,7 @@ xrl_status xrl_policy_value(xrl_ctx* ctx, const xrl_batch* b, const float* graph
   if (b->num_envs > 0 && (!graph_emb || !probs || !value || (!mask && ctx->cfg.max_actions > 0)))
     return XRL_ERR_INVALID_ARG;
   XRL_CUDA(cudaSetDevice(ctx->device));
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaStream_t st = ctx->capturing ? ctx->cap_stream : static_cast<cudaStream_t>(stream);
   const size_t slot = ctx->prof.begin(st);
   ctx->launches_heads = launch_heads(ctx->dims, ctx->dw, graph_emb, b->d_env_off, mask, b->B, b->num_envs,
                                      ctx->logits.as<float>(), probs, value, action, seed, step,
@@ -796,13 +811,15 @@ xrl_status xrl_sample(xrl_ctx* ctx, const float* probs, int32_t num_envs, int32_
   if (!ctx || num_envs < 0 || num_actions < 1) return XRL_ERR_INVALID_ARG;
   if (num_envs > 0 && (!probs || !action)) return XRL_ERR_INVALID_ARG;
   XRL_CUDA(cudaSetDevice(ctx->device));
-  launch_sample(probs, num_envs, num_actions, seed, step, action, static_cast<cudaStream_t>(stream));
+  launch_sample(probs, num_envs, num_actions, seed, step, action,
+                ctx->capturing ? ctx->cap_stream : static_cast<cudaStream_t>(stream));
   XRL_CUDA(cudaGetLastError());
   return XRL_OK;
 }
 
 xrl_status xrl_last_device_status(xrl_ctx* ctx, void* stream, int32_t* status) {
   if (!ctx || !status) return XRL_ERR_INVALID_ARG;
+  if (ctx->capturing) return XRL_ERR_STATE;
   XRL_CUDA(cudaSetDevice(ctx->device));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   XRL_CUDA(cudaStreamSynchronize(st));
@@ -811,8 +828,50 @@ xrl_status xrl_last_device_status(xrl_ctx* ctx, void* stream, int32_t* status) {
   return XRL_OK;
 }
 
+xrl_status xrl_graph_begin(xrl_ctx* ctx) {
+  if (!ctx) return XRL_ERR_INVALID_ARG;
+  if (ctx->capturing || ctx->prof.on) return XRL_ERR_STATE;     // event timing needs direct launches
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  if (ctx->cap_stream == nullptr)
+    XRL_CUDA(cudaStreamCreateWithFlags(&ctx->cap_stream, cudaStreamNonBlocking));
+  XRL_CUDA(cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeThreadLocal));
+  ctx->capturing = true;
+  return XRL_OK;
+}
+
+xrl_status xrl_graph_launch(xrl_ctx* ctx, void* stream) {
+  if (!ctx) return XRL_ERR_INVALID_ARG;
+  if (!ctx->capturing) return XRL_ERR_STATE;
+  ctx->capturing = false;
+  cudaSetDevice(ctx->device);
+  cudaGraph_t graph = nullptr;
+  if (cudaStreamEndCapture(ctx->cap_stream, &graph) != cudaSuccess || graph == nullptr) {
+    cudaGetLastError();
+    if (graph) cudaGraphDestroy(graph);
+    return XRL_ERR_CUDA;
+  }
+  bool ready = false;
+  if (ctx->graph_exec != nullptr) {                // same kernel sequence as last time: update in place
+    cudaGraphExecUpdateResultInfo info;
+    if (cudaGraphExecUpdate(ctx->graph_exec, graph, &info) == cudaSuccess) {
+      ready = true;
+    } else {
+      cudaGetLastError();
+      cudaGraphExecDestroy(ctx->graph_exec);
+      ctx->graph_exec = nullptr;
+    }
+  }
+  cudaError_t e = cudaSuccess;
+  if (!ready) e = cudaGraphInstantiate(&ctx->graph_exec, graph, 0);
+  if (e == cudaSuccess) e = cudaGraphLaunch(ctx->graph_exec, static_cast<cudaStream_t>(stream));
+  cudaGraphDestroy(graph);
+  if (e != cudaSuccess) { cudaGetLastError(); return XRL_ERR_CUDA; }
+  return XRL_OK;
+}
+
 xrl_status xrl_profile(xrl_ctx* ctx, int32_t enable) {
   if (!ctx) return XRL_ERR_INVALID_ARG;
+  if (ctx->capturing) return XRL_ERR_STATE;
   XRL_CUDA(cudaSetDevice(ctx->device));
   XRL_CUDA(cudaDeviceSynchronize());
   ctx->prof.clear();
@@ -822,6 +881,7 @@ xrl_status xrl_profile(xrl_ctx* ctx, int32_t enable) {
 
 xrl_status xrl_profile_read(xrl_ctx* ctx, double* total_ms, int64_t* launches, int32_t num_families) {
   if (!ctx || !total_ms || !launches || num_families < 0) return XRL_ERR_INVALID_ARG;
+  if (ctx->capturing) return XRL_ERR_STATE;
   XRL_CUDA(cudaSetDevice(ctx->device));
   XRL_CUDA(cudaDeviceSynchronize());
   for (int f = 0; f < num_families; ++f) { total_ms[f] = 0.0; launches[f] = 0; }
