@@ -138,7 +138,13 @@ xrl_status xrl_pack(xrl_ctx* ctx, const xrl_graph* graphs, int32_t num_graphs,
  * kernels directly and must stay valid until the stream has passed the call.  HOST arrays in
  * pageable memory are staged through a pinned buffer before the call returns; HOST arrays that are
  * all page-locked (cudaHostAlloc / cudaHostRegister) are copied asynchronously straight from the
- * caller's memory and must then also stay valid until the stream has passed the call. */
+ * caller's memory and must then also stay valid until the stream has passed the call.
+ * A page-locked batch of 2^20 nodes or more (graphs of at most 16,384 nodes) is copied and packed in
+ * up to 8 ranges of whole graphs on a stream the batch owns, ordered after everything queued on `stream`
+ * so far; xrl_encode then encodes range after range as each arrives (graphs never interact before the
+ * heads), so that the bus transfer of the later ranges overlaps the encoding of the earlier ones.  Every
+ * other consumer of the batch first waits for all ranges; results do not depend on the split except for
+ * the order in which a graph's node features are summed (Eq. 8), i.e. within rounding. */
 xrl_status xrl_pack_flat(xrl_ctx* ctx, int32_t where, int32_t num_graphs, const int32_t* n_nodes,
                          const int32_t* n_edges, const int32_t* op, const void* shape,
                          const int32_t* edge_src, const int32_t* edge_dst, const int32_t* env_off,

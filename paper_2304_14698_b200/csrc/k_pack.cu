@@ -212,13 +212,13 @@ k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ e
              const int32_t* __restrict__ op, const int32_t* __restrict__ edge_src,
              const int32_t* __restrict__ edge_dst, int32_t T, int32_t B, int32_t cap_n,
              int32_t* __restrict__ seg_id, int32_t* __restrict__ rowptr, int32_t* __restrict__ col,
-             int32_t* status) {
+             int32_t* status, int32_t g_first) {
   extern __shared__ __align__(16) int32_t psm[];
   int32_t* deg = psm;                         // [cap_n + 1] in-degree, then exclusive row starts
   int32_t* cur = psm + cap_n + 1;             // [cap_n]     row cursors
   int32_t* wsum = cur + cap_n;                // [kGraphThreads / 32 + 1]
   int2* tmp = reinterpret_cast<int2*>(wsum + kGraphThreads / 32 + 3);   // word 2 cap_n + 20: 8-byte aligned
-  const int32_t g = blockIdx.x;
+  const int32_t g = g_first + blockIdx.x;      // a launch may cover a range of the batch's graphs
   const int32_t nb = node_off[g], n = node_off[g + 1] - nb;
   const int32_t eb = edge_off[g], m = edge_off[g + 1] - eb;
   const int tid = threadIdx.x;
@@ -270,6 +270,9 @@ k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ e
   __syncthreads();
   for (int32_t i = tid; i < n; i += kGraphThreads) rowptr[nb + i] = eb + deg[i];
   if (g == B - 1 && tid == 0) rowptr[nb + n] = eb + deg[n];
+  // the last graph of a partial launch closes its last row itself (the next graph's CTA, which writes the
+  // same value as its first row start, may run much later)
+  else if (blockIdx.x == gridDim.x - 1 && tid == 0) rowptr[nb + n] = edge_off[g + 1];
   // scatter (edge id, global producer) into the rows, slot order as the atomics hand it out
   for (int32_t e0 = tid; e0 < m; e0 += 4 * kGraphThreads) {
     int32_t s[4], t[4];
@@ -333,7 +336,13 @@ size_t scan_workspace_ints(int64_t n) {
   return total + 16;
 }
 
-int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cudaStream_t st) {
+// Graphs small enough for shared memory: one CTA builds the whole CSR of a graph.
+bool pack_per_graph(const PackIn& in) {
+  return in.B > 0 && in.max_n > 0 && in.max_n <= 16384 && pack_graph_smem(in.max_n, in.max_m) <= 160 * 1024;
+}
+
+// Offsets and graph -> environment table: needs the per-graph counts only, not the graphs themselves.
+int launch_pack_offsets(const PackIn& in, const PackOut& out, cudaStream_t st) {
   int launches = 0;
   const int TB = 256;
   launches += exclusive_scan(in.n_nodes, out.node_off, in.B, out.scan_ws, st);
@@ -342,15 +351,25 @@ int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cu
     k_graph_envs<<<(in.B + TB - 1) / TB, TB, 0, st>>>(in.env_off, in.num_envs, in.B, out.graph_env);
     ++launches;
   }
-  // graphs small enough for shared memory: one CTA builds the whole CSR of a graph
-  if (in.B > 0 && in.max_n > 0 && in.max_n <= 16384 && pack_graph_smem(in.max_n, in.max_m) <= 160 * 1024) {
-    static bool attr[64] = {};
-    ensure_dynamic_smem(k_pack_graph, 160 * 1024, attr);
-    k_pack_graph<<<in.B, kGraphThreads, pack_graph_smem(in.max_n, in.max_m), st>>>(
-        out.node_off, out.edge_off, in.op, in.edge_src, in.edge_dst, T, in.B, in.max_n, out.seg_id,
-        out.rowptr, out.col, status);
-    return launches + 1;
-  }
+  return launches;
+}
+
+// CSR, segment ids and validation of graphs [g0, g1) (pack_per_graph(in) must hold; offsets already built).
+int launch_pack_graphs(const PackIn& in, const PackOut& out, int T, int32_t g0, int32_t g1, int32_t* status,
+                       cudaStream_t st) {
+  if (g1 <= g0) return 0;
+  static bool attr[64] = {};
+  ensure_dynamic_smem(k_pack_graph, 160 * 1024, attr);
+  k_pack_graph<<<g1 - g0, kGraphThreads, pack_graph_smem(in.max_n, in.max_m), st>>>(
+      out.node_off, out.edge_off, in.op, in.edge_src, in.edge_dst, T, in.B, in.max_n, out.seg_id,
+      out.rowptr, out.col, status, g0);
+  return 1;
+}
+
+int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cudaStream_t st) {
+  int launches = launch_pack_offsets(in, out, st);
+  const int TB = 256;
+  if (pack_per_graph(in)) return launches + launch_pack_graphs(in, out, T, 0, in.B, status, st);
   if (in.N > 0) {
     k_node_segments<<<(in.N + TB - 1) / TB, TB, 0, st>>>(out.node_off, in.B, in.N, in.op, T,
                                                           out.seg_id, out.deg, status);

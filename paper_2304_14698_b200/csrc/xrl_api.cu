@@ -84,6 +84,8 @@ struct xrl_ctx {
   cudaStream_t cap_stream = nullptr;
   cudaGraphExec_t graph_exec = nullptr;
   bool capturing = false;
+  cudaStream_t last_pipe = nullptr;   // stream of the last batch that was packed range by range (its kernels
+                                      // report bad graphs too: xrl_last_device_status waits for it as well)
 };
 
 struct xrl_batch {
@@ -97,6 +99,16 @@ struct xrl_batch {
   DeviceBuf edge_src, edge_dst, deg, tmp_eid, long_rows, long_count, scan_ws, coarse;
   const int32_t *d_n_nodes = nullptr, *d_n_edges = nullptr, *d_env_off = nullptr,
                 *d_graph_chunk_off = nullptr, *d_chunk_row0 = nullptr, *d_chunk_row1 = nullptr;
+  // Large batches packed from page-locked host memory are copied and packed in `nparts` ranges of whole
+  // graphs on the batch's own stream `pipe`, so that the encoder can start on the first range while the
+  // later ones are still crossing the bus: range p = graphs [part_g[p], part_g[p+1]) = rows
+  // [part_row[p], part_row[p+1]), ready when ev_part[p] has completed.  nparts = 0: packed in one piece
+  // on the caller's stream.
+  static constexpr int kMaxParts = 8;
+  int32_t nparts = 0;
+  int32_t part_g[kMaxParts + 1] = {0}, part_row[kMaxParts + 1] = {0};
+  cudaStream_t pipe = nullptr;
+  cudaEvent_t ev_start = nullptr, ev_meta = nullptr, ev_part[kMaxParts] = {nullptr};
   // pinned host staging (allocated on the first pack from host memory)
   int32_t* h_meta = nullptr;
   size_t h_meta_ints = 0;
@@ -287,7 +299,32 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
   // ---- bulk arrays -------------------------------------------------------------------------------
   const size_t sb = storage_bytes(c.dtype);
   const int32_t *d_src, *d_dst;
-  if (direct) {
+  // page-locked caller memory and a large batch of graphs that the per-graph packer takes: ranges of
+  // graphs are copied and packed one after the other on the batch's own stream (see xrl_batch::nparts)
+  int parts = 0;
+  {
+    const char* ev = getenv("XRL_PIPELINE_MIN_NODES");           // testing aid: pipeline smaller batches too
+    const int64_t min_nodes = ev ? atoll(ev) : (int64_t(1) << 20);
+    PackIn probe{};
+    probe.B = num_graphs; probe.max_n = max_n; probe.max_m = max_m;
+    if (direct && num_graphs >= 2 && N >= min_nodes && min_nodes > 0 && pack_per_graph(probe)) {
+      const int64_t want = N / min_nodes;
+      parts = int(want < 2 ? 2 : (want > xrl_batch::kMaxParts ? xrl_batch::kMaxParts : want));
+      if (parts > num_graphs) parts = num_graphs;
+    }
+  }
+  if (parts > 0 && b->pipe == nullptr) {
+    XRL_CUDA(cudaStreamCreateWithFlags(&b->pipe, cudaStreamNonBlocking));
+    XRL_CUDA(cudaEventCreateWithFlags(&b->ev_start, cudaEventDisableTiming));
+    XRL_CUDA(cudaEventCreateWithFlags(&b->ev_meta, cudaEventDisableTiming));
+    for (int p = 0; p < xrl_batch::kMaxParts; ++p)
+      XRL_CUDA(cudaEventCreateWithFlags(&b->ev_part[p], cudaEventDisableTiming));
+  }
+  b->nparts = 0;
+  if (parts > 0) {
+    d_src = b->edge_src.as<int32_t>();
+    d_dst = b->edge_dst.as<int32_t>();
+  } else if (direct) {
     // page-locked caller memory: copy straight from it, no staging pass
     if (N) {
       XRL_CUDA(cudaMemcpyAsync(b->op.p, op, 4 * size_t(N), cudaMemcpyHostToDevice, st));
@@ -340,7 +377,7 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
     d_src = edge_src;
     d_dst = edge_dst;
   }
-  XRL_CUDA(cudaEventRecord(b->staged, st));
+  if (parts == 0) XRL_CUDA(cudaEventRecord(b->staged, st));
 
   PackIn in;
   in.B = num_graphs; in.num_envs = num_envs; in.N = int32_t(N); in.E = int32_t(E);
@@ -354,10 +391,51 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
   po.deg = b->deg.as<int32_t>(); po.tmp_eid = b->tmp_eid.as<int32_t>();
   po.long_rows = b->long_rows.as<int32_t>(); po.long_count = b->long_count.as<int32_t>();
   po.scan_ws = b->scan_ws.as<int32_t>(); po.coarse = b->coarse.as<int32_t>();
-  {
+  if (parts == 0) {
     const size_t slot = ctx->prof.begin(st);
     ctx->launches_pack = launch_pack(in, po, c.num_op_types, ctx->status.as<int32_t>(), st);
     ctx->prof.end(FAM_PACK, slot, int(ctx->launches_pack), st);
+  } else {
+    // whatever still reads the batch's arrays was queued on the caller's stream before this call
+    XRL_CUDA(cudaEventRecord(b->ev_start, st));
+    XRL_CUDA(cudaStreamWaitEvent(b->pipe, b->ev_start, 0));
+    const size_t slot = ctx->prof.begin(st);
+    int launches = launch_pack_offsets(in, po, st);            // needs the counts only
+    ctx->prof.end(FAM_PACK, slot, launches, st);
+    XRL_CUDA(cudaEventRecord(b->ev_meta, st));
+    XRL_CUDA(cudaStreamWaitEvent(b->pipe, b->ev_meta, 0));
+    // ranges of whole graphs with about N / parts nodes each
+    const char* h_op = reinterpret_cast<const char*>(op);
+    const char* h_shape = reinterpret_cast<const char*>(shape);
+    int32_t g = 0;
+    int64_t row = 0, edge = 0;
+    b->part_g[0] = 0; b->part_row[0] = 0;
+    for (int p = 0; p < parts; ++p) {
+      const int64_t row0 = row, edge0 = edge;
+      const int32_t g0 = g;
+      const int64_t target = (N * int64_t(p + 1)) / parts;
+      while (g < num_graphs && (p == parts - 1 || row < target || g == g0)) { row += n_nodes[g]; edge += n_edges[g]; ++g; }
+      const size_t n = size_t(row - row0), m = size_t(edge - edge0);
+      if (n) {
+        XRL_CUDA(cudaMemcpyAsync(b->op.as<char>() + 4 * size_t(row0), h_op + 4 * size_t(row0), 4 * n,
+                                 cudaMemcpyHostToDevice, b->pipe));
+        XRL_CUDA(cudaMemcpyAsync(b->shape.as<char>() + sb * kS * size_t(row0), h_shape + sb * kS * size_t(row0),
+                                 sb * kS * n, cudaMemcpyHostToDevice, b->pipe));
+      }
+      if (m) {
+        XRL_CUDA(cudaMemcpyAsync(b->edge_src.as<int32_t>() + edge0, edge_src + edge0, 4 * m,
+                                 cudaMemcpyHostToDevice, b->pipe));
+        XRL_CUDA(cudaMemcpyAsync(b->edge_dst.as<int32_t>() + edge0, edge_dst + edge0, 4 * m,
+                                 cudaMemcpyHostToDevice, b->pipe));
+      }
+      launches += launch_pack_graphs(in, po, c.num_op_types, g0, g, ctx->status.as<int32_t>(), b->pipe);
+      XRL_CUDA(cudaEventRecord(b->ev_part[p], b->pipe));
+      b->part_g[p + 1] = g; b->part_row[p + 1] = int32_t(row);
+    }
+    XRL_CUDA(cudaEventRecord(b->staged, b->pipe));
+    b->nparts = parts;
+    ctx->last_pipe = b->pipe;
+    ctx->launches_pack = launches;
   }
   XRL_CUDA(cudaGetLastError());
 
@@ -370,9 +448,9 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
 // With fuse_readout the last of the `layers` attention layers may leave per-graph partial sums in
 // ctx->partial instead of node features in ctx->h; *fused tells whether it did.
 int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t st, bool fuse_readout = false,
-                    bool* fused = nullptr) {
+                    bool* fused = nullptr, int32_t row_begin = 0, int32_t row_end = -1) {
   const Dims& d = ctx->dims;
-  const Window win{0, b->N, 0};
+  const Window win{row_begin, row_end < 0 ? b->N : row_end, 0};   // graphs are independent: any range of whole graphs
   Profiler& pf = ctx->prof;
   size_t slot = pf.begin(st);
   int k = -1;
@@ -415,6 +493,12 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
     n += k;
   }
   return n;
+}
+
+// A batch packed range by range becomes whole for `st` once every range's event has been waited for.
+xrl_status join_parts(const xrl_batch* b, cudaStream_t st) {
+  for (int p = 0; p < b->nparts; ++p) XRL_CUDA(cudaStreamWaitEvent(st, b->ev_part[p], 0));
+  return XRL_OK;
 }
 
 xrl_status check_batch(const xrl_ctx* ctx, const xrl_batch* b) {
@@ -583,6 +667,13 @@ xrl_status xrl_batch_free(xrl_ctx* ctx, xrl_batch* b) {
   if (b->h_meta) cudaFreeHost(b->h_meta);
   if (b->h_bulk) cudaFreeHost(b->h_bulk);
   if (b->staged) cudaEventDestroy(b->staged);
+  if (b->ev_start) cudaEventDestroy(b->ev_start);
+  if (b->ev_meta) cudaEventDestroy(b->ev_meta);
+  for (cudaEvent_t e : b->ev_part) if (e) cudaEventDestroy(e);
+  if (b->pipe) {
+    if (b->ctx->last_pipe == b->pipe) b->ctx->last_pipe = nullptr;
+    cudaStreamDestroy(b->pipe);
+  }
   delete b;
   return XRL_OK;
 }
@@ -604,6 +695,7 @@ xrl_status xrl_batch_export(const xrl_batch* b, int32_t* rowptr, int32_t* col, i
   if (!b->packed) return XRL_ERR_STATE;
   XRL_CUDA(cudaSetDevice(b->ctx->device));
   XRL_CUDA(cudaStreamSynchronize(b->stream));
+  if (b->nparts > 0) XRL_CUDA(cudaStreamSynchronize(b->pipe));
   const size_t N = size_t(b->N), E = size_t(b->E), B = size_t(b->B);
   if (rowptr) XRL_CUDA(cudaMemcpy(rowptr, b->rowptr.p, 4 * (N + 1), cudaMemcpyDeviceToHost));
   if (col && E) XRL_CUDA(cudaMemcpy(col, b->col.p, 4 * E, cudaMemcpyDeviceToHost));
@@ -621,8 +713,22 @@ xrl_status xrl_encode(xrl_ctx* ctx, const xrl_batch* b, const float* g0, float* 
   XRL_CUDA(cudaSetDevice(ctx->device));
   cudaStream_t st = ctx->capturing ? ctx->cap_stream : static_cast<cudaStream_t>(stream);
   bool fused = false;
-  int n = run_node_layers(ctx, b, ctx->cfg.layers, st, true, &fused);
-  if (n < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
+  int n = 0;
+  if (b->nparts > 0) {
+    // packed range by range: encode each range of graphs as soon as it is there (the copies and the packing
+    // of the later ranges run meanwhile on the batch's stream); the per-graph sums follow for all at once
+    if (ctx->capturing) return XRL_ERR_STATE;
+    for (int p = 0; p < b->nparts; ++p) {
+      XRL_CUDA(cudaStreamWaitEvent(st, b->ev_part[p], 0));
+      if (b->part_row[p + 1] == b->part_row[p]) continue;
+      const int k = run_node_layers(ctx, b, ctx->cfg.layers, st, false, nullptr, b->part_row[p], b->part_row[p + 1]);
+      if (k < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
+      n += k;
+    }
+  } else {
+    n = run_node_layers(ctx, b, ctx->cfg.layers, st, true, &fused);
+    if (n < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
+  }
   size_t slot;
   int k;
   if (!fused) {
@@ -654,6 +760,7 @@ xrl_status xrl_encode_delta(xrl_ctx* ctx, const xrl_batch* b, const int32_t* bas
   if (!graph_emb && b->B > 0) return XRL_ERR_INVALID_ARG;
   XRL_CUDA(cudaSetDevice(ctx->device));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  { const xrl_status js = join_parts(b, st); if (js != XRL_OK) return js; }
   const size_t Ncap = size_t(ctx->cfg.max_nodes) + 1, Ecap = size_t(ctx->cfg.max_edges) + 1;
   if (ctx->dl_ints.p == nullptr) {
     XRL_ALLOC(ctx->dl_ints.alloc(4 * (10 * Ncap + 256)));
@@ -774,6 +881,7 @@ xrl_status xrl_debug_node_features(xrl_ctx* ctx, const xrl_batch* b, int32_t num
   if (ctx->capturing) return XRL_ERR_STATE;
   XRL_CUDA(cudaSetDevice(ctx->device));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  { const xrl_status js = join_parts(b, st); if (js != XRL_OK) return js; }
   if (run_node_layers(ctx, b, num_layers, st) < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
   const int64_t n = int64_t(b->N) * ctx->cfg.hidden;
   if (n == 0) return XRL_OK;
@@ -823,6 +931,7 @@ xrl_status xrl_last_device_status(xrl_ctx* ctx, void* stream, int32_t* status) {
   XRL_CUDA(cudaSetDevice(ctx->device));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   XRL_CUDA(cudaStreamSynchronize(st));
+  if (ctx->last_pipe) XRL_CUDA(cudaStreamSynchronize(ctx->last_pipe));
   XRL_CUDA(cudaMemcpy(status, ctx->status.p, 4, cudaMemcpyDeviceToHost));
   XRL_CUDA(cudaMemset(ctx->status.p, 0, 4));
   return XRL_OK;

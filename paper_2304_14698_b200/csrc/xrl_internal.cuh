@@ -115,6 +115,11 @@ struct PackOut {
   int32_t *deg, *tmp_eid /* [2E]: (edge id, producer) pairs */, *long_rows, *long_count, *scan_ws, *coarse;   // scratch
 };
 int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cudaStream_t st);
+// the same in two parts, for packing a batch range by range while its later graphs are still being copied
+bool pack_per_graph(const PackIn& in);
+int launch_pack_offsets(const PackIn& in, const PackOut& out, cudaStream_t st);
+int launch_pack_graphs(const PackIn& in, const PackOut& out, int T, int32_t g0, int32_t g1, int32_t* status,
+                       cudaStream_t st);
 size_t scan_workspace_ints(int64_t n);
 // out[0..n_in] = exclusive prefix sums of in[0..n_in) (n_in + 1 outputs); ws: scan_workspace_ints(n_in) ints
 int launch_exclusive_scan(const int32_t* in, int32_t* out, int32_t n_in, int32_t* ws, cudaStream_t st);
