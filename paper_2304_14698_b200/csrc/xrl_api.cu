@@ -404,7 +404,7 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
     ctx->prof.end(FAM_PACK, slot, launches, st);
     XRL_CUDA(cudaEventRecord(b->ev_meta, st));
     XRL_CUDA(cudaStreamWaitEvent(b->pipe, b->ev_meta, 0));
-    // ranges of whole graphs with about N / parts nodes each
+    // ranges of whole graphs
     const char* h_op = reinterpret_cast<const char*>(op);
     const char* h_shape = reinterpret_cast<const char*>(shape);
     int32_t g = 0;
@@ -413,7 +413,8 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
     for (int p = 0; p < parts; ++p) {
       const int64_t row0 = row, edge0 = edge;
       const int32_t g0 = g;
-      const int64_t target = (N * int64_t(p + 1)) / parts;
+      // the first range is half as long as the others: nothing overlaps its copy
+      const int64_t target = (N * int64_t(2 * p + 1)) / (2 * parts - 1);
       while (g < num_graphs && (p == parts - 1 || row < target || g == g0)) { row += n_nodes[g]; edge += n_edges[g]; ++g; }
       const size_t n = size_t(row - row0), m = size_t(edge - edge0);
       if (n) {
