@@ -144,7 +144,9 @@ xrl_status xrl_pack(xrl_ctx* ctx, const xrl_graph* graphs, int32_t num_graphs,
  * so far; xrl_encode then encodes range after range as each arrives (graphs never interact before the
  * heads), so that the bus transfer of the later ranges overlaps the encoding of the earlier ones.  Every
  * other consumer of the batch first waits for all ranges; results do not depend on the split except for
- * the order in which a graph's node features are summed (Eq. 8), i.e. within rounding. */
+ * the order in which a graph's node features are summed (Eq. 8), i.e. within rounding.  The host arrays of
+ * such a batch are read by that stream: keep them valid until a consumer of the batch queued after this
+ * call (xrl_encode, ...) has completed on its stream, or until xrl_last_device_status has returned. */
 xrl_status xrl_pack_flat(xrl_ctx* ctx, int32_t where, int32_t num_graphs, const int32_t* n_nodes,
                          const int32_t* n_edges, const int32_t* op, const void* shape,
                          const int32_t* edge_src, const int32_t* edge_dst, const int32_t* env_off,

@@ -10,11 +10,23 @@ namespace {
 
 constexpr int kRoThreads = 256;
 
-// sum_k x[k] * W[k * ld + c]: the weight loads are issued eight at a time so that their latencies
-// overlap; the additions keep the order k = 0, 1, 2, ...
+// sum_k x[k] * W[k * ld + c]: the weight loads are issued DEPTH (then eight) at a time so that their
+// latencies overlap; the additions keep the order k = 0, 1, 2, ...  DEPTH = 32 is for launches of few
+// CTAs, which are bound by the latency of these loads; with many CTAs per SM the registers it takes cost
+// more occupancy than the depth gains, and DEPTH = 8 is used.
+template <int DEPTH>
 __device__ __forceinline__ float column_dot(const float* x, int in, const float* __restrict__ W, int ld,
                                             int c, float acc) {
   int k = 0;
+  if (DEPTH > 8) {
+    for (; k + DEPTH <= in; k += DEPTH) {
+      float w[DEPTH];
+#pragma unroll
+      for (int t = 0; t < DEPTH; ++t) w[t] = __ldg(W + size_t(k + t) * ld + c);
+#pragma unroll
+      for (int t = 0; t < DEPTH; ++t) acc = fmaf(x[k + t], w[t], acc);
+    }
+  }
   for (; k + 8 <= in; k += 8) {
     float w[8];
 #pragma unroll
@@ -30,7 +42,7 @@ __device__ __forceinline__ float column_dot(const float* x, int in, const float*
 // than threads the k range is cut into P = blockDim / CP contiguous parts (CP = columns per pass, a power of
 // two), the parts are computed by different thread groups and added in part order.  Every thread of the
 // block calls it; `part` is blockDim floats of scratch; emit(c, y) runs once per column.
-template <typename Emit>
+template <int DEPTH, typename Emit>
 __device__ __forceinline__ void dense_columns(const float* x, int in, const float* __restrict__ W, int ld,
                                               int ncols, const float* __restrict__ bias, float* part, Emit emit) {
   const int nt = blockDim.x, tid = threadIdx.x;
@@ -38,13 +50,13 @@ __device__ __forceinline__ void dense_columns(const float* x, int in, const floa
   while (CP < ncols && CP < nt) CP <<= 1;
   const int P = nt / CP, cl = tid % CP, p = tid / CP;
   if (P == 1) {                                  // as many columns as threads (or more): no split, no barriers
-    for (int c = tid; c < ncols; c += nt) emit(c, column_dot(x, in, W, ld, c, bias[c]));
+    for (int c = tid; c < ncols; c += nt) emit(c, column_dot<DEPTH>(x, in, W, ld, c, bias[c]));
     return;
   }
   const int k0 = int((int64_t(in) * p) / P), k1 = int((int64_t(in) * (p + 1)) / P);
   for (int c0 = 0; c0 < ncols; c0 += CP) {
     const int c = c0 + cl;
-    part[tid] = (c < ncols) ? column_dot(x + k0, k1 - k0, W + size_t(k0) * ld, ld, c, 0.f) : 0.f;
+    part[tid] = (c < ncols) ? column_dot<DEPTH>(x + k0, k1 - k0, W + size_t(k0) * ld, ld, c, 0.f) : 0.f;
     __syncthreads();
     if (p == 0 && c < ncols) {
       float y = bias[c];
@@ -101,6 +113,7 @@ k_readout(const T* __restrict__ h, const int32_t* __restrict__ chunk_row0,
 }
 
 // ---- Eq. 8: emb_g = ReLU(Wg^T [ sum of the graph's chunk sums | g0_g ] + bg) -------------------
+template <int DEPTH>
 __global__ void __launch_bounds__(256)
 k_global_update(const float* __restrict__ partial, const int32_t* __restrict__ graph_chunk_off,
                 const float* __restrict__ g0, const float* __restrict__ Wg,
@@ -116,13 +129,14 @@ k_global_update(const float* __restrict__ partial, const int32_t* __restrict__ g
   }
   for (int t = threadIdx.x; t < Dg; t += blockDim.x) u[H + t] = g0 ? g0[size_t(g) * Dg + t] : 0.f;
   __syncthreads();
-  dense_columns(u, H + Dg, Wg, H, H, bg, part,
+  dense_columns<DEPTH>(u, H + Dg, Wg, H, H, bg, part,
                 [&](int c, float y) { emb[size_t(g) * H + c] = fmaxf(y, 0.f); });
 }
 
 // Eq. 8 from the partial sums written by the aggregate kernel fused with the readout: per graph, the
 // partial of the block in which the graph starts (if it does not start at the block's first row), then
 // the partials of the following 32-row blocks whose first row belongs to the graph, in order.
+template <int DEPTH>
 __global__ void __launch_bounds__(256)
 k_global_update_blocks(const float* __restrict__ partial, const int32_t* __restrict__ node_off,
                        int32_t nblocks, const float* __restrict__ g0, const float* __restrict__ Wg,
@@ -143,7 +157,7 @@ k_global_update_blocks(const float* __restrict__ partial, const int32_t* __restr
   }
   for (int t = threadIdx.x; t < Dg; t += blockDim.x) u[H + t] = g0 ? g0[size_t(g) * Dg + t] : 0.f;
   __syncthreads();
-  dense_columns(u, H + Dg, Wg, H, H, bg, part,
+  dense_columns<DEPTH>(u, H + Dg, Wg, H, H, bg, part,
                 [&](int c, float y) { emb[size_t(g) * H + c] = fmaxf(y, 0.f); });
 }
 
@@ -165,20 +179,22 @@ __device__ float block_sum(float v, float* scratch) {
 // out = w2 . ReLU(Wh^T ReLU(W1^T x + b1) + bh) + b2.  x (length `in`) and y1 (hid floats, used only when
 // hid2 > 0) are in shared memory; all threads return the result.
 struct Mlp { const float *W1, *b1, *Wh, *bh, *w2, *b2; int hid, hid2; };
+template <int DEPTH>
 __device__ float mlp_scalar(const float* x, int in, const Mlp& m, float* y1, float* scratch) {
   float contrib = 0.f;
   if (m.hid2 <= 0) {
-    dense_columns(x, in, m.W1, m.hid, m.hid, m.b1, scratch, [&](int c, float y) { contrib += fmaxf(y, 0.f) * m.w2[c]; });
+    dense_columns<DEPTH>(x, in, m.W1, m.hid, m.hid, m.b1, scratch, [&](int c, float y) { contrib += fmaxf(y, 0.f) * m.w2[c]; });
   } else {
-    dense_columns(x, in, m.W1, m.hid, m.hid, m.b1, scratch, [&](int c, float y) { y1[c] = fmaxf(y, 0.f); });
+    dense_columns<DEPTH>(x, in, m.W1, m.hid, m.hid, m.b1, scratch, [&](int c, float y) { y1[c] = fmaxf(y, 0.f); });
     __syncthreads();
-    dense_columns(y1, m.hid, m.Wh, m.hid2, m.hid2, m.bh, scratch,
+    dense_columns<DEPTH>(y1, m.hid, m.Wh, m.hid2, m.hid2, m.bh, scratch,
                   [&](int c, float y) { contrib += fmaxf(y, 0.f) * m.w2[c]; });
   }
   return block_sum(contrib, scratch) + m.b2[0];
 }
 
 // ---- policy MLP: one scalar score per graph -----------------------------------------------------
+template <int DEPTH>
 __global__ void __launch_bounds__(256)
 k_policy_logit(const float* __restrict__ emb, const Mlp mlp, float* __restrict__ logit, int H) {
   extern __shared__ float sm[];                  // [H] + [blockDim] + [hid]
@@ -188,7 +204,7 @@ k_policy_logit(const float* __restrict__ emb, const Mlp mlp, float* __restrict__
   const int32_t g = blockIdx.x;
   for (int c = threadIdx.x; c < H; c += blockDim.x) x[c] = emb[size_t(g) * H + c];
   __syncthreads();
-  const float v = mlp_scalar(x, H, mlp, y1, scratch);
+  const float v = mlp_scalar<DEPTH>(x, H, mlp, y1, scratch);
   if (threadIdx.x == 0) logit[g] = v;
 }
 
@@ -293,6 +309,7 @@ k_candidate_sum(const float* __restrict__ emb, const int32_t* __restrict__ env_o
 }
 
 // ---- per environment: masked softmax, candidate mean, value MLP, optional draw -----------------
+template <int DEPTH>
 __global__ void __launch_bounds__(1024)
 k_env_policy(const float* __restrict__ emb, const float* __restrict__ logit,
              const float* __restrict__ cand_sum,
@@ -345,7 +362,7 @@ k_env_policy(const float* __restrict__ emb, const float* __restrict__ logit,
   const float nv = block_sum(cnt, scratch);
   for (int c = tid; c < H; c += nt) u[H + c] = nv > 0.f ? cand_sum[size_t(e) * H + c] / nv : 0.f;
   __syncthreads();
-  const float v = mlp_scalar(u, 2 * H, vmlp, y1, scratch);
+  const float v = mlp_scalar<DEPTH>(u, 2 * H, vmlp, y1, scratch);
   if (tid == 0) value[e] = v;
 
   if (action != nullptr) {
@@ -381,6 +398,9 @@ __global__ void k_round_weights(const float* __restrict__ src, T* __restrict__ d
   if (dst_t != nullptr) dst_t[size_t(c) * rows + r] = v;
 }
 
+// Launches with at most a few CTAs per SM are bound by the latency of their weight loads.
+bool few_ctas(int64_t ctas) { return ctas <= 4 * kNumSMs; }
+
 int pow2_threads(int want) {          // power of two in [32, 1024] (block_sum needs a power of two)
   int t = 32;
   while (t < want && t < 1024) t <<= 1;
@@ -409,16 +429,20 @@ int launch_readout(const Dims& d, const void* h, const int32_t* chunk_row0, cons
 int launch_global_update(const Dims& d, const float* partial, const int32_t* graph_chunk_off,
                          const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st) {
   if (B <= 0) return 0;
-  k_global_update<<<B, 256, sizeof(float) * size_t(d.H + d.Dg + 256), st>>>(partial, graph_chunk_off, g0,
-                                                                      w.Wg, w.bg, emb, d.H, d.Dg);
+  const size_t smem = sizeof(float) * size_t(d.H + d.Dg + 256);
+  if (few_ctas(B)) k_global_update<32><<<B, 256, smem, st>>>(partial, graph_chunk_off, g0, w.Wg, w.bg, emb, d.H, d.Dg);
+  else k_global_update<8><<<B, 256, smem, st>>>(partial, graph_chunk_off, g0, w.Wg, w.bg, emb, d.H, d.Dg);
   return 1;
 }
 
 int launch_global_update_blocks(const Dims& d, const float* partial, const int32_t* node_off, int32_t nblocks,
                                 const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st) {
   if (B <= 0) return 0;
-  k_global_update_blocks<<<B, 256, sizeof(float) * size_t(d.H + d.Dg + 256), st>>>(partial, node_off, nblocks, g0,
-                                                                             w.Wg, w.bg, emb, d.H, d.Dg);
+  const size_t smem = sizeof(float) * size_t(d.H + d.Dg + 256);
+  if (few_ctas(B))
+    k_global_update_blocks<32><<<B, 256, smem, st>>>(partial, node_off, nblocks, g0, w.Wg, w.bg, emb, d.H, d.Dg);
+  else
+    k_global_update_blocks<8><<<B, 256, smem, st>>>(partial, node_off, nblocks, g0, w.Wg, w.bg, emb, d.H, d.Dg);
   return 1;
 }
 
@@ -429,15 +453,21 @@ int launch_heads(const Dims& d, const DevWeights& w, const float* emb, const int
   if (B <= 0 || num_envs <= 0) return 0;
   const Mlp pm{w.pW1, w.pb1, w.pWh, w.pbh, w.pw2, w.pb2, d.Hm, d.Hm2};
   const Mlp vm{w.vW1, w.vb1, w.vWh, w.vbh, w.vw2, w.vb2, d.Hm, d.Hm2};
-  k_policy_logit<<<B, 256, sizeof(float) * size_t(d.H + 256 + d.Hm), st>>>(emb, pm, logit_ws, d.H);
+  const size_t psm = sizeof(float) * size_t(d.H + 256 + d.Hm);
+  if (few_ctas(B)) k_policy_logit<32><<<B, 256, psm, st>>>(emb, pm, logit_ws, d.H);
+  else k_policy_logit<8><<<B, 256, psm, st>>>(emb, pm, logit_ws, d.H);
   float* cand_sum = logit_ws + B;                 // [num_envs x H], behind the per-graph logits
   k_candidate_sum<<<dim3(num_envs, (d.H + 31) / 32), 1024, 0, st>>>(emb, env_off, mask, cand_sum, d.H, d.A);
   int want = d.H > d.A + 1 ? d.H : d.A + 1;
   if (want < 256) want = 256;               // enough threads to split the value head's dense map
   const int nt = pow2_threads(want);
   const size_t smem = sizeof(unsigned long long) * size_t(nt + 1) + sizeof(float) * size_t(nt + 2 * d.H + d.Hm);
-  k_env_policy<<<num_envs, nt, smem, st>>>(emb, logit_ws, cand_sum, env_off, mask, vm, probs, value, action,
-                                           d.H, d.A, seed, step, status);
+  if (few_ctas(num_envs))
+    k_env_policy<32><<<num_envs, nt, smem, st>>>(emb, logit_ws, cand_sum, env_off, mask, vm, probs, value, action,
+                                                 d.H, d.A, seed, step, status);
+  else
+    k_env_policy<8><<<num_envs, nt, smem, st>>>(emb, logit_ws, cand_sum, env_off, mask, vm, probs, value, action,
+                                                d.H, d.A, seed, step, status);
   return 3;
 }
 
