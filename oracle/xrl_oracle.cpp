@@ -101,7 +101,8 @@ double stored(const Model& m, float w) { return m.dtype == 1 ? round_bf16(w) : d
 void encode_graph(const Model& m, const Weights& w, int32_t lo, int32_t hi,
                   const int32_t* rowptr, const int32_t* col, const int32_t* op,
                   const float* shape, const double* g_attr, int mode, double* emb,
-                  int dump_layer, double* node_dump, double* alpha_edge, double* alpha_self) {
+                  int dump_layer, double* node_dump, double* alpha_edge, double* alpha_self,
+                  const float* edge_attr, const int32_t* eid) {
   const int S = m.S, T = m.T, H = m.H, K = m.K, d = m.H / m.K;
   const int n = hi - lo;
   const int F0 = 2 * S + T;
@@ -115,15 +116,18 @@ void encode_graph(const Model& m, const Weights& w, int32_t lo, int32_t hi,
   };
 
   // ---- Eq. 6: h'_i = sigma( W ( sum_{j in E_i} e_j  ||  h_i ) ).
-  // The attribute of edge j->i is the shape feature vector of its producer j; the node
-  // attribute is the one-hot operator id followed by the node's own shape features.
+  // The attribute of edge j->i is the shape feature vector of its producer j, or, when the caller
+  // gives attributes per edge (Section 3.3.2 as written: the shape of the tensor the edge carries), the
+  // S values of that edge; the node attribute is the one-hot operator id followed by the node's own
+  // shape features.
   std::vector<double> x(F0), W0s(size_t(F0) * H);
   for (size_t t = 0; t < W0s.size(); ++t) W0s[t] = stored(m, w.W0[t]);
   for (int i = 0; i < n; ++i) {
     const int gi = lo + i;
     for (int s = 0; s < F0; ++s) x[s] = 0.0;
     for (int e = rowptr[gi]; e < rowptr[gi + 1]; ++e)
-      for (int s = 0; s < S; ++s) x[s] += double(shape[size_t(col[e]) * S + s]);
+      for (int s = 0; s < S; ++s)
+        x[s] += edge_attr ? double(edge_attr[size_t(eid[e]) * S + s]) : double(shape[size_t(col[e]) * S + s]);
     x[S + op[gi]] = 1.0;
     for (int s = 0; s < S; ++s) x[S + T + s] = double(shape[size_t(gi) * S + s]);
     for (int c = 0; c < H; ++c) {
@@ -264,7 +268,8 @@ void xo_philox4x32_10(uint32_t k0, uint32_t k1, uint32_t c0, uint32_t c1, uint32
 int xo_pack(int32_t B, const int32_t* n_nodes, const int32_t* n_edges, const int32_t* edge_src,
             const int32_t* edge_dst, int32_t num_envs, const int32_t* env_off,
             int32_t* node_off, int32_t* edge_off, int32_t* seg_id, int32_t* graph_env,
-            int32_t* rowptr, int32_t* col) {
+            int32_t* rowptr, int32_t* col, int32_t* eid) {
+  // eid (optional, [E]): the input edge that ends up in each CSR slot, for attributes that live on edges
   if (B < 0 || num_envs < 0) return XO_INVALID_ARG;
   node_off[0] = 0; edge_off[0] = 0;
   for (int g = 0; g < B; ++g) {
@@ -292,6 +297,7 @@ int xo_pack(int32_t B, const int32_t* n_nodes, const int32_t* n_edges, const int
   for (int g = 0; g < B; ++g)
     for (int e = edge_off[g]; e < edge_off[g + 1]; ++e) {
       const int32_t t = node_off[g] + edge_dst[e];
+      if (eid) eid[cursor[t]] = e;
       col[cursor[t]++] = node_off[g] + edge_src[e];
     }
   return XO_OK;
@@ -305,8 +311,10 @@ int xo_encode(const Model* m, const float* weights, int32_t B, const int32_t* no
               const int32_t* rowptr, const int32_t* col, const int32_t* op, const float* shape,
               const double* g0, int32_t n_sel, const int32_t* sel, int32_t mode,
               int32_t threads, double* graph_emb, int32_t dump_layer, double* node_dump,
-              double* alpha_edge, double* alpha_self) {
+              double* alpha_edge, double* alpha_self, const float* edge_attr, const int32_t* eid) {
+  // edge_attr (optional, [E x S], input edge order) with eid from xo_pack: attributes on edges in Eq. 6
   if (m->H % m->K != 0 || m->L < 0) return XO_INVALID_ARG;
+  if (edge_attr && !eid) return XO_INVALID_ARG;
   const Weights w = slice(*m, weights);
   const int count = sel ? n_sel : B;
   int bad = 0;
@@ -319,7 +327,7 @@ int xo_encode(const Model* m, const float* weights, int32_t B, const int32_t* no
     if (g < 0 || g >= B) { bad = 1; continue; }
     encode_graph(*m, w, node_off[g], node_off[g + 1], rowptr, col, op, shape,
                  g0 ? g0 + size_t(g) * m->Dg : nullptr, mode, graph_emb + size_t(t) * m->H,
-                 dump_layer, node_dump, alpha_edge, alpha_self);
+                 dump_layer, node_dump, alpha_edge, alpha_self, edge_attr, eid);
   }
   (void)threads;
   return bad ? XO_INVALID_ARG : XO_OK;

@@ -60,19 +60,26 @@ def pack(batch):
         "node_off": np.zeros(B + 1, np.int32), "edge_off": np.zeros(B + 1, np.int32),
         "seg_id": np.zeros(N, np.int32), "graph_env": np.zeros(B, np.int32),
         "rowptr": np.zeros(N + 1, np.int32), "col": np.zeros(E, np.int32),
+        "eid": np.zeros(E, np.int32),
     }
     st = lib().xo_pack(
         C.c_int32(B), _p(batch["n_nodes"], _i32p), _p(batch["n_edges"], _i32p),
         _p(batch["edge_src"], _i32p), _p(batch["edge_dst"], _i32p),
         C.c_int32(len(env_off) - 1), _p(env_off, _i32p),
         _p(out["node_off"], _i32p), _p(out["edge_off"], _i32p), _p(out["seg_id"], _i32p),
-        _p(out["graph_env"], _i32p), _p(out["rowptr"], _i32p), _p(out["col"], _i32p))
+        _p(out["graph_env"], _i32p), _p(out["rowptr"], _i32p), _p(out["col"], _i32p),
+        _p(out["eid"], _i32p))
     return int(st), out
 
 
 def encode(m, weights, batch, packed, g0=None, sel=None, mode=0, threads=0, dump_layer=-1,
-           want_nodes=False, want_alpha=False):
-    """Section 3.4 (Eq. 6, Eq. 7 x L, Eq. 8).  Returns dict(emb[, nodes, alpha_edge, alpha_self])."""
+           want_nodes=False, want_alpha=False, edge_attr=None):
+    """Section 3.4 (Eq. 6, Eq. 7 x L, Eq. 8).  Returns dict(emb[, nodes, alpha_edge, alpha_self]).
+    edge_attr ([E x S] float32, input edge order; default batch.get("edge_attr")): attributes on edges in
+    Eq. 6 instead of the producers' shape features."""
+    if edge_attr is None:
+        edge_attr = batch.get("edge_attr")
+    ea = None if edge_attr is None else np.ascontiguousarray(edge_attr, dtype=np.float32)
     B = int(batch["num_graphs"])
     N = int(batch["n_nodes"].sum()); E = int(batch["n_edges"].sum())
     weights = np.ascontiguousarray(weights, dtype=np.float32)
@@ -90,7 +97,8 @@ def encode(m, weights, batch, packed, g0=None, sel=None, mode=0, threads=0, dump
         C.byref(mm), _p(weights, _f32p), C.c_int32(B), _p(packed["node_off"], _i32p),
         _p(packed["rowptr"], _i32p), _p(packed["col"], _i32p), _p(op, _i32p), _p(shape, _f32p),
         _p(g0a, _f64p), C.c_int32(n_out), _p(sel_a, _i32p), C.c_int32(mode), C.c_int32(threads),
-        _p(emb, _f64p), C.c_int32(dump_layer), _p(nodes, _f64p), _p(a_e, _f64p), _p(a_s, _f64p))
+        _p(emb, _f64p), C.c_int32(dump_layer), _p(nodes, _f64p), _p(a_e, _f64p), _p(a_s, _f64p),
+        _p(ea, _f32p), _p(packed["eid"] if ea is not None else None, _i32p))
     if st != 0:
         raise ValueError(f"xo_encode status {st}")
     return {"emb": emb, "nodes": nodes, "alpha_edge": a_e, "alpha_self": a_s}

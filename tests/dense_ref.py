@@ -23,11 +23,20 @@ def adjacency(g):
 
 
 def node_update(g, W, m):
-    """Eq. 6 as X @ W0 + b0 with X = [A @ shape || onehot(op) || shape]."""
+    """Eq. 6 as X @ W0 + b0 with X = [A @ shape || onehot(op) || shape]; with attributes on the edges
+    (g["edge_attr"], one row per edge of the input list) the first block is the incidence matrix (consumer
+    x edge) times the attributes instead."""
     A = adjacency(g)
     shp = g["shape"].astype(np.float64)
     onehot = np.eye(m["T"])[g["op"]]
-    X = np.concatenate([A @ shp, onehot, shp], axis=1)
+    if g.get("edge_attr") is not None:
+        n, ne = len(g["op"]), len(g["edge_dst"])
+        Inc = np.zeros((n, ne))
+        Inc[np.asarray(g["edge_dst"]), np.arange(ne)] = 1.0
+        agg = Inc @ np.asarray(g["edge_attr"], dtype=np.float64)
+    else:
+        agg = A @ shp
+    X = np.concatenate([agg, onehot, shp], axis=1)
     W0 = bf16_round(W["W0"]) if m["dtype"] == "bf16" else W["W0"].astype(np.float64)
     return np.maximum(X @ W0 + W["b0"].astype(np.float64), 0.0)
 

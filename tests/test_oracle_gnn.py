@@ -41,6 +41,47 @@ def test_encoder_matches_dense_bruteforce(xo, dtype):
         np.testing.assert_allclose(out["emb"][gi], want, rtol=1e-12, atol=1e-12)
 
 
+def _shuffle_edges(rng, g):
+    perm = rng.permutation(len(g["edge_src"]))
+    return dict(g, edge_src=g["edge_src"][perm], edge_dst=g["edge_dst"][perm])
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_edge_attributes_match_dense_bruteforce(xo, dtype):
+    """Section 3.3.2 as written: attributes live on the edges.  Edge lists in shuffled order (so that the CSR
+    slots are a non-trivial permutation of the input edges), repeated edges, attributes that differ between
+    the repeats; the expectation sums attributes straight from the input edge list."""
+    m = dict(M_SMALL, dtype=dtype)
+    _, W = configs.make_weights(m, 13)
+    rng = np.random.default_rng(3)
+    graphs = [_shuffle_edges(rng, g) for g in _tiny_graphs(7)]
+    for g in graphs:
+        g["edge_attr"] = dags.tensor_shape_attributes(dags.make_rng(len(g["edge_src"])), len(g["edge_src"]), 8, dtype == "bf16")
+        if dtype == "bf16":
+            g["shape"] = dags.round_to_bf16_grid(g["shape"])
+    b, p, out = _run(xo, m, W, graphs)
+    assert "edge_attr" in b
+    for gi, g in enumerate(graphs):
+        want = dense_ref.encode_graph(g, W, m)
+        np.testing.assert_allclose(out["emb"][gi], want, rtol=1e-12, atol=1e-12)
+        plain = dense_ref.encode_graph({k: v for k, v in g.items() if k != "edge_attr"}, W, m)
+        assert not np.allclose(want, plain)          # the attributes matter
+
+
+def test_edge_attributes_equal_to_the_producers_features_change_nothing(xo):
+    """Edges that carry exactly their producer's shape features reproduce the node-feature reading bit
+    for bit (same values added in the same order)."""
+    m = dict(M_SMALL)
+    _, W = configs.make_weights(m, 14)
+    rng = np.random.default_rng(4)
+    graphs = [_shuffle_edges(rng, g) for g in _tiny_graphs(8)]
+    b, p, base = _run(xo, m, W, graphs)
+    for g in graphs:
+        g["edge_attr"] = g["shape"][g["edge_src"]]
+    b2, p2, out = _run(xo, m, W, graphs)
+    assert np.array_equal(out["emb"], base["emb"])
+
+
 def test_each_stage_matches_dense_bruteforce(xo):
     m = dict(M_SMALL)
     _, W = configs.make_weights(m, 12)

@@ -25,6 +25,17 @@ def _check_against_input(batch, packed):
             want[int(no[g] + d)].append(int(no[g] + s))
     for i in range(no[-1]):
         assert list(col[rowptr[i]:rowptr[i + 1]]) == want.get(i, []), i
+    # eid: the input edge sitting in each CSR slot - a permutation of the edges that agrees with col, with
+    # the row it sits in, and increases inside a row (input order kept)
+    eid = packed["eid"]
+    assert sorted(eid.tolist()) == list(range(int(eo[-1])))
+    g_of_edge = np.repeat(np.arange(B), batch["n_edges"])
+    for i in range(no[-1]):
+        ks = np.arange(rowptr[i], rowptr[i + 1])
+        es = eid[ks]
+        assert np.all(np.diff(es) > 0)
+        assert np.all(no[g_of_edge[es]] + batch["edge_dst"][es] == i)
+        assert np.array_equal(col[ks], no[g_of_edge[es]] + batch["edge_src"][es])
     # env -> graph map
     for e in range(len(batch["env_off"]) - 1):
         assert np.all(packed["graph_env"][batch["env_off"][e]:batch["env_off"][e + 1]] == e)

@@ -198,6 +198,19 @@ def local_rewrite(rng, g, T, bf16=False, max_region=6, max_new=6):
     }
 
 
+def tensor_shape_attributes(rng, num_edges, S=8, bf16=False, M=4096.0):
+    """Per-edge attributes as the paper describes them (Section 3.3.2): the shape of the tensor an edge
+    carries as four dimensions divided by the constant M, ranks below four padded with zeros in the leading
+    positions; the remaining S - 4 columns are zero.  Input data only (no arithmetic of the method)."""
+    a = np.zeros((num_edges, S), dtype=np.float32)
+    rank = rng.integers(1, 5, size=num_edges)
+    dims = np.exp2(rng.uniform(0.0, 12.0, size=(num_edges, 4))).astype(np.int64).clip(1, 4096)
+    for r in range(1, 5):
+        rows = rank == r
+        a[rows, 4 - r:4] = dims[rows, 4 - r:4] / M
+    return round_to_bf16_grid(a) if bf16 else a
+
+
 def flatten(graphs, env_off, A_max, mask=None):
     """Concatenate per-graph arrays into the flat batch both sides consume."""
     env_off = np.asarray(env_off, dtype=np.int32)
@@ -216,7 +229,12 @@ def flatten(graphs, env_off, A_max, mask=None):
             tw = graphs[gi].get("twin")
             if tw is not None:
                 base_id[node_off[gi]:node_off[gi + 1]] = np.where(tw >= 0, tw + node_off[cur], -1)
+    extra = {}
+    if len(graphs) and all(g.get("edge_attr") is not None for g in graphs):      # attributes on the edges
+        extra["edge_attr"] = np.ascontiguousarray(
+            np.concatenate([np.asarray(g["edge_attr"], dtype=np.float32).reshape(-1, S) for g in graphs]))
     return {
+        **extra,
         "base_id": base_id,
         "num_graphs": len(graphs),
         "n_nodes": np.array([len(g["op"]) for g in graphs], dtype=np.int32),
