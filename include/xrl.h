@@ -71,6 +71,10 @@ typedef struct {
                               one-hidden-layer reading                                             */
   int32_t global_dim;      /* Dg: width of the per-graph global attribute (paper: value 0)    */
   int32_t dtype;           /* XRL_FP32, or XRL_BF16 = bf16 storage with fp32 accumulation     */
+  int32_t edge_attributes; /* 0: the attribute of edge j -> i in Eq. 6 is producer j's S shape features
+                              (taken from `shape`); 1: every edge has S attributes of its own, given with
+                              xrl_batch_set_edge_attr after packing - Section 3.3.2 as written, where an
+                              edge carries the shape of its tensor divided by the constant M             */
   int32_t max_actions;     /* A_max: padded number of candidate slots; No-Op is index A_max   */
   int32_t max_graphs;      /* capacity: graphs per batch                                      */
   int32_t max_envs;        /* capacity: environments per batch                                */
@@ -161,6 +165,18 @@ xrl_status xrl_batch_info(const xrl_batch* batch, int64_t* num_nodes, int64_t* n
  * edge_off [B+1], graph_env [B]. */
 xrl_status xrl_batch_export(const xrl_batch* batch, int32_t* rowptr, int32_t* col, int32_t* seg_id,
                             int32_t* node_off, int32_t* edge_off, int32_t* graph_env);
+
+/* Attributes on the edges (contexts created with edge_attributes = 1; Section 3.3.2: "for edges, we use
+ * the corresponding tensor shape as its attributes", padded and divided by a constant).  edge_attr is
+ * [E x S] in the storage type (float, or bf16 bits), one row per edge in the order of the edge lists given
+ * to the pack call, HOST or DEVICE according to `where`; the library brings the rows into the order of the
+ * packed CSR (one gather pass, queued on `stream` after the packing) and Eq. 6 then sums, for each node, the
+ * attributes of its incoming edges in place of its producers' shape features.  Call it after every pack of
+ * the batch and before xrl_encode (which returns XRL_ERR_STATE otherwise).  A HOST array is read before the
+ * call returns.  xrl_encode_delta is not available for such contexts (XRL_ERR_UNSUPPORTED).
+ * Errors: INVALID_ARG, STATE (context without edge attributes, batch not packed, recording), CUDA. */
+xrl_status xrl_batch_set_edge_attr(xrl_ctx* ctx, xrl_batch* batch, int32_t where, const void* edge_attr,
+                                   void* stream);
 
 /* ---- (2) encoder: Section 3.4 ------------------------------------------------------------ */
 

@@ -25,7 +25,7 @@ EXPORTED_SYMBOLS = [
     "xrl_batch_free", "xrl_batch_info", "xrl_batch_export", "xrl_encode", "xrl_debug_node_features",
     "xrl_policy_value", "xrl_sample", "xrl_last_device_status", "xrl_launch_counts", "xrl_version",
     "xrl_profile", "xrl_profile_read", "xrl_pack_csr_static", "xrl_encode_delta", "xrl_delta_rows", "xrl_get_weights",
-    "xrl_graph_begin", "xrl_graph_launch",
+    "xrl_graph_begin", "xrl_graph_launch", "xrl_batch_set_edge_attr",
 ]
 PROFILE_FAMILIES = ["pack", "node_update", "transform", "aggregate", "readout", "heads", "aggregate_readout"]
 
@@ -39,7 +39,8 @@ class XrlError(RuntimeError):
 class _ModelConfig(C.Structure):
     _fields_ = [("num_op_types", C.c_int32), ("num_shape_feats", C.c_int32), ("hidden", C.c_int32),
                 ("heads", C.c_int32), ("layers", C.c_int32), ("mlp_hidden", C.c_int32),
-                ("mlp_hidden2", C.c_int32), ("global_dim", C.c_int32), ("dtype", C.c_int32), ("max_actions", C.c_int32),
+                ("mlp_hidden2", C.c_int32), ("global_dim", C.c_int32), ("dtype", C.c_int32),
+                ("edge_attributes", C.c_int32), ("max_actions", C.c_int32),
                 ("max_graphs", C.c_int32), ("max_envs", C.c_int32), ("max_nodes", C.c_int64),
                 ("max_edges", C.c_int64)]
 
@@ -85,6 +86,7 @@ def load_library():
         "xrl_delta_rows": [vp, C.POINTER(i64), i32],
         "xrl_pack_csr_static": [i32, i32, i32] + [vp] * 6 + [i32] + [vp] * 8,
         "xrl_profile_read": [vp, C.POINTER(C.c_double), C.POINTER(i64), i32],
+        "xrl_batch_set_edge_attr": [vp, vp, i32, vp, vp],
         "xrl_graph_begin": [vp],
         "xrl_graph_launch": [vp, vp],
     }
@@ -120,9 +122,11 @@ def _stream(stream):
 
 def model_config(m, max_graphs, max_envs, max_nodes, max_edges):
     """Build the C config from a dict with keys T, S, H, K, L, Hm, Dg, dtype, A_max and, optionally,
-    Hm2 (second hidden width of the heads' MLPs, default 0 = one hidden layer)."""
+    Hm2 (second hidden width of the heads' MLPs, default 0 = one hidden layer) and edge_attr (True: the
+    model takes Eq. 6's edge attributes from the edges themselves, see xrl_batch_set_edge_attr)."""
     return _ModelConfig(m["T"], m["S"], m["H"], m["K"], m["L"], m["Hm"], int(m.get("Hm2", 0)), m["Dg"],
-                        XRL_BF16 if m["dtype"] in ("bf16", XRL_BF16) else XRL_FP32, m["A_max"],
+                        XRL_BF16 if m["dtype"] in ("bf16", XRL_BF16) else XRL_FP32,
+                        1 if m.get("edge_attr") else 0, m["A_max"],
                         int(max_graphs), int(max_envs), int(max_nodes), int(max_edges))
 
 
@@ -201,6 +205,15 @@ def xrl_pack_flat(ctx, where, n_nodes, n_edges, op, shape, edge_src, edge_dst, e
                                       _np_ptr(env_off), len(env_off) - 1, _stream(stream), C.byref(out))
     _check(st, "xrl_pack_flat")
     return out
+
+
+def xrl_batch_set_edge_attr(ctx, batch, edge_attr, stream=None):
+    """edge_attr: [E, S] in the storage type, rows in the order of the packed edge lists; numpy (HOST;
+    float32, or uint16 bf16 bits) or a torch CUDA tensor (DEVICE)."""
+    on_dev = not isinstance(edge_attr, np.ndarray)
+    ptr = _dev_ptr(edge_attr) if on_dev else _np_ptr(np.ascontiguousarray(edge_attr))
+    _check(load_library().xrl_batch_set_edge_attr(ctx, batch, XRL_MEM_DEVICE if on_dev else XRL_MEM_HOST, ptr,
+                                                  _stream(stream)), "xrl_batch_set_edge_attr")
 
 
 def xrl_batch_free(ctx, batch):
@@ -389,6 +402,9 @@ class Agent:
                                    batch["n_nodes"], batch["n_edges"], batch["op"], shape,
                                    batch["edge_src"], batch["edge_dst"], batch["env_off"],
                                    batch=self.batch)
+        if self.m.get("edge_attr"):
+            ea = batch["edge_attr"]
+            xrl_batch_set_edge_attr(self.ctx, self.batch, ea if on_dev else self.storage_shape(ea))
         return self.batch
 
     def pack_graphs(self, graphs, env_off):

@@ -46,7 +46,7 @@ k_embed_umma(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ 
              const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
              const int32_t* __restrict__ op, const bf16* __restrict__ shape,
              const int32_t* __restrict__ row_list, int row_begin, int rows, int op_pieces, int ksteps,
-             int32_t* status) {
+             int32_t* status, const bf16* __restrict__ eattr) {
   using C = ECfg<H>;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t base = smem_u32(smem);
@@ -177,7 +177,9 @@ k_embed_umma(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ 
         o = __ldg(op + row);
         for (int32_t ed = e0; ed < e1; ++ed) {
           float f[kS];
-          unpack(__ldg(reinterpret_cast<const uint4*>(shape + size_t(__ldg(col + ed)) * kS)), f);
+          // the producer's shape features, or the edge's own attributes (kept in slot order)
+          const bf16* src = eattr ? eattr + size_t(ed) * kS : shape + size_t(__ldg(col + ed)) * kS;
+          unpack(__ldg(reinterpret_cast<const uint4*>(src)), f);
 #pragma unroll
           for (int s = 0; s < kS; ++s) e[s] += f[s];
         }
@@ -240,7 +242,7 @@ __global__ void k_build_w0ext(const bf16* __restrict__ W0, const float* __restri
 template <int H>
 int launch_h(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op,
              const void* shape, const void* w0ext_t, void* h, Window win, const int32_t* row_list,
-             int32_t* status, cudaStream_t st) {
+             int32_t* status, cudaStream_t st, const void* eattr) {
   using C = ECfg<H>;
   static bool attr_set[64] = {};
   if (!ensure_dynamic_smem(k_embed_umma<H>, C::SMEM_BYTES, attr_set)) return -1;
@@ -255,7 +257,8 @@ int launch_h(const Dims& d, const int32_t* rowptr, const int32_t* col, const int
   const int grid = tiles < kNumSMs ? tiles : kNumSMs;
   k_embed_umma<H><<<grid, kThreads, C::SMEM_BYTES, st>>>(mw, mh, rowptr, col, op,
                                                          static_cast<const bf16*>(shape), row_list,
-                                                         win.row_begin, int(rows), op_pieces, ksteps, status);
+                                                         win.row_begin, int(rows), op_pieces, ksteps, status,
+                                                         static_cast<const bf16*>(eattr));
   return 1;
 }
 
@@ -279,10 +282,10 @@ void build_w0ext(const Dims& d, const void* W0_store, const float* b0, void* out
 
 int launch_embed_umma(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op,
                       const void* shape, const void* w0ext_t, void* h, Window win, int32_t* status,
-                      cudaStream_t st, const int32_t* row_list) {
+                      cudaStream_t st, const int32_t* row_list, const void* eattr) {
   if (int64_t(win.row_end) - win.row_begin <= 0) return 0;
-  if (d.H == 256) return launch_h<256>(d, rowptr, col, op, shape, w0ext_t, h, win, row_list, status, st);
-  return launch_h<128>(d, rowptr, col, op, shape, w0ext_t, h, win, row_list, status, st);
+  if (d.H == 256) return launch_h<256>(d, rowptr, col, op, shape, w0ext_t, h, win, row_list, status, st, eattr);
+  return launch_h<128>(d, rowptr, col, op, shape, w0ext_t, h, win, row_list, status, st, eattr);
 }
 
 }  // namespace xrl

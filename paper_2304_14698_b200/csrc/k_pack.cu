@@ -163,20 +163,22 @@ constexpr int kShortRow = 32;
 
 // One thread per row: place each producer at the rank of its edge id among the row's edge ids, which
 // restores the input order whatever order the atomics handed the slots out in.
+// eid (optional): the input edge that lands in each slot, for attributes that live on the edges.
 __global__ void k_row_order(const int32_t* __restrict__ rowptr, const int2* __restrict__ tmp, int32_t N,
                             int32_t* __restrict__ col, int32_t* __restrict__ long_rows,
-                            int32_t* __restrict__ long_count) {
+                            int32_t* __restrict__ long_count, int32_t* __restrict__ eid) {
   const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= N) return;
   const int32_t b = rowptr[i], n = rowptr[i + 1] - b;
   if (n == 0) return;
-  if (n == 1) { col[b] = tmp[b].y; return; }
+  if (n == 1) { col[b] = tmp[b].y; if (eid) eid[b] = tmp[b].x; return; }
   if (n > kShortRow) { long_rows[atomicAdd(long_count, 1)] = i; return; }
   for (int32_t a = 0; a < n; ++a) {
     const int2 ea = tmp[b + a];
     int32_t rank = 0;
     for (int32_t c = 0; c < n; ++c) rank += (tmp[b + c].x < ea.x) ? 1 : 0;
     col[b + rank] = ea.y;
+    if (eid) eid[b + rank] = ea.x;
   }
 }
 
@@ -184,7 +186,7 @@ __global__ void k_row_order(const int32_t* __restrict__ rowptr, const int2* __re
 __global__ void __launch_bounds__(256)
 k_row_order_long(const int32_t* __restrict__ rowptr, const int2* __restrict__ tmp,
                  int32_t* __restrict__ col, const int32_t* __restrict__ long_rows,
-                 const int32_t* __restrict__ long_count) {
+                 const int32_t* __restrict__ long_count, int32_t* __restrict__ eid) {
   const int lane = threadIdx.x & 31;
   const int32_t warps = (gridDim.x * blockDim.x) >> 5;
   const int32_t count = *long_count;
@@ -196,6 +198,7 @@ k_row_order_long(const int32_t* __restrict__ rowptr, const int2* __restrict__ tm
       int32_t rank = 0;
       for (int32_t c = 0; c < n; ++c) rank += (tmp[b + c].x < ea.x) ? 1 : 0;
       col[b + rank] = ea.y;
+      if (eid) eid[b + rank] = ea.x;
     }
   }
 }
@@ -212,7 +215,7 @@ k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ e
              const int32_t* __restrict__ op, const int32_t* __restrict__ edge_src,
              const int32_t* __restrict__ edge_dst, int32_t T, int32_t B, int32_t cap_n,
              int32_t* __restrict__ seg_id, int32_t* __restrict__ rowptr, int32_t* __restrict__ col,
-             int32_t* status, int32_t g_first) {
+             int32_t* status, int32_t g_first, int32_t* __restrict__ eid) {
   extern __shared__ __align__(16) int32_t psm[];
   int32_t* deg = psm;                         // [cap_n + 1] in-degree, then exclusive row starts
   int32_t* cur = psm + cap_n + 1;             // [cap_n]     row cursors
@@ -292,13 +295,14 @@ k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ e
   // rank of each edge id inside its row restores the input order; short rows by one thread ...
   for (int32_t i = tid; i < n; i += kGraphThreads) {
     const int32_t b = deg[i], k = deg[i + 1] - b;
-    if (k == 1) col[eb + b] = tmp[b].y;
+    if (k == 1) { col[eb + b] = tmp[b].y; if (eid) eid[eb + b] = eb + tmp[b].x; }
     else if (k > 1 && k <= kShortRow)
       for (int32_t a = 0; a < k; ++a) {
         const int2 ea = tmp[b + a];
         int32_t rank = 0;
         for (int32_t c = 0; c < k; ++c) rank += (tmp[b + c].x < ea.x) ? 1 : 0;
         col[eb + b + rank] = ea.y;
+        if (eid) eid[eb + b + rank] = eb + ea.x;      // edge ids are local to the graph in here
       }
   }
   // ... long rows by one warp each
@@ -310,6 +314,7 @@ k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ e
       int32_t rank = 0;
       for (int32_t c = 0; c < k; ++c) rank += (tmp[b + c].x < ea.x) ? 1 : 0;
       col[eb + b + rank] = ea.y;
+      if (eid) eid[eb + b + rank] = eb + ea.x;
     }
   }
 }
@@ -319,6 +324,29 @@ size_t pack_graph_smem(int32_t cap_n, int32_t cap_m) {
 }
 
 }  // namespace
+
+// Attributes on the edges, brought from input edge order into CSR slot order: dst[k] = src[eid[k]], rows of
+// `row_bytes` bytes (a multiple of 16), one 16-byte piece per thread.
+namespace {
+__global__ void k_permute_rows(const uint4* __restrict__ src, const int32_t* __restrict__ eid,
+                               uint4* __restrict__ dst, int64_t E, int pieces) {
+  const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= E * pieces) return;
+  const int64_t k = i / pieces;
+  const int p = int(i - k * pieces);
+  dst[i] = __ldg(src + int64_t(__ldg(eid + k)) * pieces + p);
+}
+}  // namespace
+
+int launch_permute_edge_rows(const void* src, const int32_t* eid, void* dst, int64_t E, int row_bytes,
+                             cudaStream_t st) {
+  if (E <= 0) return 0;
+  const int pieces = row_bytes / 16;
+  const int64_t n = E * pieces;
+  k_permute_rows<<<unsigned((n + 255) / 256), 256, 0, st>>>(static_cast<const uint4*>(src), eid,
+                                                             static_cast<uint4*>(dst), E, pieces);
+  return 1;
+}
 
 int launch_exclusive_scan(const int32_t* in, int32_t* out, int32_t n_in, int32_t* ws, cudaStream_t st) {
   return exclusive_scan(in, out, n_in, ws, st);
@@ -362,7 +390,7 @@ int launch_pack_graphs(const PackIn& in, const PackOut& out, int T, int32_t g0, 
   ensure_dynamic_smem(k_pack_graph, 160 * 1024, attr);
   k_pack_graph<<<g1 - g0, kGraphThreads, pack_graph_smem(in.max_n, in.max_m), st>>>(
       out.node_off, out.edge_off, in.op, in.edge_src, in.edge_dst, T, in.B, in.max_n, out.seg_id,
-      out.rowptr, out.col, status, g0);
+      out.rowptr, out.col, status, g0, out.eid);
   return 1;
 }
 
@@ -391,8 +419,8 @@ int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cu
                                                          out.node_off, out.coarse, out.rowptr, in.B, in.E,
                                                          out.deg, tmp);
     k_row_order<<<(in.N + TB - 1) / TB, TB, 0, st>>>(out.rowptr, tmp, in.N, out.col, out.long_rows,
-                                                      out.long_count);
-    k_row_order_long<<<kNumSMs, 256, 0, st>>>(out.rowptr, tmp, out.col, out.long_rows, out.long_count);
+                                                      out.long_count, out.eid);
+    k_row_order_long<<<kNumSMs, 256, 0, st>>>(out.rowptr, tmp, out.col, out.long_rows, out.long_count, out.eid);
     launches += 3;
   }
   return launches;

@@ -21,6 +21,7 @@ __device__ __forceinline__ void load_shape(const bf16* shape, int32_t node, floa
 }
 
 // ---- Eq. 6: h0_i = ReLU(W0^T [ sum_{j->i} shape_j | onehot(op_i) | shape_i ] + b0) -----------
+// (with attributes on the edges, Section 3.3.2 as written, the sum runs over the in-edges' own attributes)
 // The one-hot block of the product is a row lookup of W0; the two shape blocks are a 16 x H
 // dense map kept in shared memory as fp32.
 template <typename T, int LPR, int VPL>
@@ -28,7 +29,7 @@ __global__ void __launch_bounds__(kRowThreads)
 k_embed(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
         const int32_t* __restrict__ op, const T* __restrict__ shape, const T* __restrict__ W0,
         const float* __restrict__ b0, T* __restrict__ h, int H, int Tn, Window win,
-        const int32_t* __restrict__ row_list) {
+        const int32_t* __restrict__ row_list, const T* __restrict__ eattr) {
   constexpr int VEC = VecOf<T>::N;
   constexpr int RPW = 32 / LPR;
   extern __shared__ float smem[];
@@ -57,7 +58,8 @@ k_embed(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
     const int32_t e0 = __ldg(rowptr + row), e1 = __ldg(rowptr + row + 1);
     for (int32_t e = e0; e < e1; ++e) {
       float f[kS];
-      load_shape(shape, __ldg(col + e), f);
+      if (eattr) load_shape(eattr, e, f);            // attributes on the edges, already in slot order
+      else load_shape(shape, __ldg(col + e), f);     // the producer's shape features
 #pragma unroll
       for (int s = 0; s < kS; ++s) x[s] += f[s];
     }
@@ -309,14 +311,14 @@ int row_grid(int64_t rows, int rpw) {
 
 int launch_embed(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op,
                  const void* shape, const DevWeights& w, void* h, Window win, cudaStream_t st,
-                 const int32_t* row_list) {
+                 const int32_t* row_list, const void* eattr) {
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   if (rows <= 0) return 0;
   const size_t smem = sizeof(float) * size_t(2 * kS + 1) * d.H;
 #define CALL(TY_, LPR, VPL)                                                                        \
   k_embed<TY_, LPR, VPL><<<row_grid(rows, 32 / LPR), kRowThreads, smem, st>>>(                     \
       rowptr, col, op, static_cast<const TY_*>(shape), static_cast<const TY_*>(w.W0), w.b0,   \
-      static_cast<TY_*>(h), d.H, d.T, win, row_list)
+      static_cast<TY_*>(h), d.H, d.T, win, row_list, static_cast<const TY_*>(eattr))
   if (d.dtype == XRL_BF16) XRL_ROW_DISPATCH(bf16, d.H, CALL);
   else XRL_ROW_DISPATCH(float, d.H, CALL);
 #undef CALL

@@ -97,6 +97,9 @@ struct xrl_batch {
   DeviceBuf meta;           // n_nodes[B] n_edges[B] env_off[Ne+1] graph_chunk_off[B+1] chunk_row0[] chunk_row1[]
   DeviceBuf node_off, edge_off, seg_id, graph_env, rowptr, col, op, shape;
   DeviceBuf edge_src, edge_dst, deg, tmp_eid, long_rows, long_count, scan_ws, coarse;
+  // contexts with attributes on the edges: slot -> input edge, the attributes as given and in slot order
+  DeviceBuf eid, eattr_in, eattr;
+  bool has_eattr = false;
   const int32_t *d_n_nodes = nullptr, *d_n_edges = nullptr, *d_env_off = nullptr,
                 *d_graph_chunk_off = nullptr, *d_chunk_row0 = nullptr, *d_chunk_row1 = nullptr;
   // Large batches packed from page-locked host memory are copied and packed in `nparts` ranges of whole
@@ -130,7 +133,7 @@ xrl_status check_config(const xrl_model_config& c) {
     return XRL_ERR_INVALID_ARG;
   if (c.num_shape_feats != kS || c.num_op_types > 256) return XRL_ERR_UNSUPPORTED;
   if (c.hidden % 32 != 0 || c.hidden > 512 || (c.hidden / c.heads) % 8 != 0) return XRL_ERR_UNSUPPORTED;
-  if (c.mlp_hidden2 < 0) return XRL_ERR_INVALID_ARG;
+  if (c.mlp_hidden2 < 0 || (c.edge_attributes != 0 && c.edge_attributes != 1)) return XRL_ERR_INVALID_ARG;
   if (c.layers > 64 || c.mlp_hidden > 1024 || c.mlp_hidden2 > 1024 || c.global_dim > 16) return XRL_ERR_UNSUPPORTED;
   if (c.max_actions > (1 << 20)) return XRL_ERR_UNSUPPORTED;
   return XRL_OK;
@@ -179,6 +182,7 @@ xrl_status alloc_batch(xrl_ctx* ctx, xrl_batch** out) {
   A(b->deg, 4 * N); A(b->tmp_eid, 8 * E + 8);
   A(b->long_rows, 4 * (E / 32 + 1)); A(b->long_count, 4); A(b->coarse, 4 * (E / 1024 + 2));
   A(b->scan_ws, 4 * scan_workspace_ints(int64_t(N > B ? N : B) + 1));
+  if (c.edge_attributes) { A(b->eid, 4 * E); A(b->eattr_in, sb * kS * E); A(b->eattr, sb * kS * E); }
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&b->staged, cudaEventDisableTiming);
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -391,6 +395,8 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
   po.deg = b->deg.as<int32_t>(); po.tmp_eid = b->tmp_eid.as<int32_t>();
   po.long_rows = b->long_rows.as<int32_t>(); po.long_count = b->long_count.as<int32_t>();
   po.scan_ws = b->scan_ws.as<int32_t>(); po.coarse = b->coarse.as<int32_t>();
+  po.eid = c.edge_attributes ? b->eid.as<int32_t>() : nullptr;
+  b->has_eattr = false;                          // attributes belong to one packing of the batch
   if (parts == 0) {
     const size_t slot = ctx->prof.begin(st);
     ctx->launches_pack = launch_pack(in, po, c.num_op_types, ctx->status.as<int32_t>(), st);
@@ -453,14 +459,15 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
   const Dims& d = ctx->dims;
   const Window win{row_begin, row_end < 0 ? b->N : row_end, 0};   // graphs are independent: any range of whole graphs
   Profiler& pf = ctx->prof;
+  const void* eattr = b->has_eattr ? b->eattr.p : nullptr;      // attributes on the edges, in slot order
   size_t slot = pf.begin(st);
   int k = -1;
   if (ctx->use_umma_embed)
     k = launch_embed_umma(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), b->op.as<int32_t>(),
-                          b->shape.p, ctx->w0ext.p, ctx->h.p, win, ctx->status.as<int32_t>(), st);
+                          b->shape.p, ctx->w0ext.p, ctx->h.p, win, ctx->status.as<int32_t>(), st, nullptr, eattr);
   if (k < 0)
     k = launch_embed(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), b->op.as<int32_t>(),
-                     b->shape.p, ctx->dw, ctx->h.p, win, st);
+                     b->shape.p, ctx->dw, ctx->h.p, win, st, nullptr, eattr);
   pf.end(FAM_EMBED, slot, k, st);
   int n = k;
   for (int l = 0; l < layers; ++l) {
@@ -505,6 +512,14 @@ xrl_status join_parts(const xrl_batch* b, cudaStream_t st) {
 xrl_status check_batch(const xrl_ctx* ctx, const xrl_batch* b) {
   if (!ctx || !b) return XRL_ERR_INVALID_ARG;
   if (b->ctx != ctx || !b->packed || !ctx->weights_set) return XRL_ERR_STATE;
+  return XRL_OK;
+}
+
+// Encoding additionally needs the edges' attributes where the model takes them from the edges.
+xrl_status check_encodable(const xrl_ctx* ctx, const xrl_batch* b) {
+  const xrl_status s = check_batch(ctx, b);
+  if (s != XRL_OK) return s;
+  if (ctx->cfg.edge_attributes && b->E > 0 && !b->has_eattr) return XRL_ERR_STATE;
   return XRL_OK;
 }
 
@@ -663,7 +678,8 @@ xrl_status xrl_batch_free(xrl_ctx* ctx, xrl_batch* b) {
   cudaDeviceSynchronize();
   DeviceBuf* bufs[] = {&b->meta, &b->node_off, &b->edge_off, &b->seg_id, &b->graph_env, &b->rowptr,
                        &b->col, &b->op, &b->shape, &b->edge_src, &b->edge_dst, &b->deg, &b->tmp_eid,
-                       &b->long_rows, &b->long_count, &b->scan_ws, &b->coarse};
+                       &b->long_rows, &b->long_count, &b->scan_ws, &b->coarse, &b->eid, &b->eattr_in,
+                       &b->eattr};
   for (DeviceBuf* d : bufs) d->release();
   if (b->h_meta) cudaFreeHost(b->h_meta);
   if (b->h_bulk) cudaFreeHost(b->h_bulk);
@@ -707,8 +723,31 @@ xrl_status xrl_batch_export(const xrl_batch* b, int32_t* rowptr, int32_t* col, i
   return XRL_OK;
 }
 
+xrl_status xrl_batch_set_edge_attr(xrl_ctx* ctx, xrl_batch* b, int32_t where, const void* edge_attr,
+                                   void* stream) {
+  if (!ctx || !b || (where != XRL_MEM_HOST && where != XRL_MEM_DEVICE)) return XRL_ERR_INVALID_ARG;
+  if (b->ctx != ctx || !b->packed || !ctx->cfg.edge_attributes || ctx->capturing) return XRL_ERR_STATE;
+  if (!edge_attr && b->E > 0) return XRL_ERR_INVALID_ARG;
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  { const xrl_status js = join_parts(b, st); if (js != XRL_OK) return js; }
+  const size_t row = storage_bytes(ctx->cfg.dtype) * kS, E = size_t(b->E);
+  if (E > 0) {
+    const void* src = edge_attr;
+    if (where == XRL_MEM_HOST) {
+      XRL_CUDA(cudaMemcpyAsync(b->eattr_in.p, edge_attr, row * E, cudaMemcpyHostToDevice, st));
+      if (!pinned(edge_attr)) XRL_CUDA(cudaStreamSynchronize(st));     // the array is read before returning
+      src = b->eattr_in.p;
+    }
+    launch_permute_edge_rows(src, b->eid.as<int32_t>(), b->eattr.p, int64_t(E), int(row), st);
+    XRL_CUDA(cudaGetLastError());
+  }
+  b->has_eattr = true;
+  return XRL_OK;
+}
+
 xrl_status xrl_encode(xrl_ctx* ctx, const xrl_batch* b, const float* g0, float* graph_emb, void* stream) {
-  const xrl_status s = check_batch(ctx, b);
+  const xrl_status s = check_encodable(ctx, b);
   if (s != XRL_OK) return s;
   if (!graph_emb && b->B > 0) return XRL_ERR_INVALID_ARG;
   XRL_CUDA(cudaSetDevice(ctx->device));
@@ -757,6 +796,7 @@ xrl_status xrl_encode_delta(xrl_ctx* ctx, const xrl_batch* b, const int32_t* bas
                             float* graph_emb, void* stream) {
   const xrl_status s = check_batch(ctx, b);
   if (s != XRL_OK) return s;
+  if (ctx->cfg.edge_attributes) return XRL_ERR_UNSUPPORTED;   // the node correspondence ignores edge attributes
   if (ctx->capturing) return XRL_ERR_STATE;        // reads the row counts back between layers
   if (!graph_emb && b->B > 0) return XRL_ERR_INVALID_ARG;
   XRL_CUDA(cudaSetDevice(ctx->device));
@@ -876,7 +916,7 @@ xrl_status xrl_delta_rows(const xrl_ctx* ctx, int64_t* rows, int32_t count) {
 
 xrl_status xrl_debug_node_features(xrl_ctx* ctx, const xrl_batch* b, int32_t num_layers,
                                    float* host_out, void* stream) {
-  const xrl_status s = check_batch(ctx, b);
+  const xrl_status s = check_encodable(ctx, b);
   if (s != XRL_OK) return s;
   if (num_layers < 0 || num_layers > ctx->cfg.layers || (!host_out && b->N > 0)) return XRL_ERR_INVALID_ARG;
   if (ctx->capturing) return XRL_ERR_STATE;

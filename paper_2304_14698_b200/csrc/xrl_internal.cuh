@@ -113,6 +113,7 @@ struct PackIn {
 struct PackOut {
   int32_t *node_off, *edge_off, *seg_id, *graph_env, *rowptr, *col;
   int32_t *deg, *tmp_eid /* [2E]: (edge id, producer) pairs */, *long_rows, *long_count, *scan_ws, *coarse;   // scratch
+  int32_t* eid = nullptr;   // optional output [E]: the input edge in each CSR slot (attributes on edges)
 };
 int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cudaStream_t st);
 // the same in two parts, for packing a batch range by range while its later graphs are still being copied
@@ -121,6 +122,8 @@ int launch_pack_offsets(const PackIn& in, const PackOut& out, cudaStream_t st);
 int launch_pack_graphs(const PackIn& in, const PackOut& out, int T, int32_t g0, int32_t g1, int32_t* status,
                        cudaStream_t st);
 size_t scan_workspace_ints(int64_t n);
+int launch_permute_edge_rows(const void* src, const int32_t* eid, void* dst, int64_t E, int row_bytes,
+                             cudaStream_t st);
 // out[0..n_in] = exclusive prefix sums of in[0..n_in) (n_in + 1 outputs); ws: scan_workspace_ints(n_in) ints
 int launch_exclusive_scan(const int32_t* in, int32_t* out, int32_t n_in, int32_t* ws, cudaStream_t st);
 
@@ -131,9 +134,10 @@ int launch_exclusive_scan(const int32_t* in, int32_t* out, int32_t n_in, int32_t
 // scores) are indexed by (row - win_base), CSR / op / shape arrays by the global row id.
 struct Window { int32_t row_begin, row_end, win_base; };
 
+// eattr (optional, [E x S] storage type, CSR slot order): Eq. 6 sums these instead of the producers' shapes
 int launch_embed(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op,
                  const void* shape, const DevWeights& w, void* h, Window win, cudaStream_t st,
-                 const int32_t* row_list = nullptr);
+                 const int32_t* row_list = nullptr, const void* eattr = nullptr);
 // scores: [N][K] pairs {s_src, s_dst} (float2), both already multiplied by log2(e)
 int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* scores,
                       Window win, cudaStream_t st);
@@ -142,7 +146,7 @@ int embed_umma_kpad(const Dims& d);
 void build_w0ext(const Dims& d, const void* W0_store, const float* b0, void* out, cudaStream_t st);
 int launch_embed_umma(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op,
                       const void* shape, const void* w0ext_t, void* h, Window win, int32_t* status,
-                      cudaStream_t st, const int32_t* row_list = nullptr);
+                      cudaStream_t st, const int32_t* row_list = nullptr, const void* eattr = nullptr);
 bool xform_umma_supported(const Dims& d);
 int launch_xform_umma(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* scores,
                       Window win, int32_t* status, cudaStream_t st);
