@@ -42,6 +42,7 @@ enum { XO_OK = 0, XO_INVALID_ARG = 1, XO_BAD_GRAPH = 2 };
 struct Model {
   int32_t T, S, H, K, L, Hm, Dg, dtype;  // dtype: 0 fp32, 1 bf16 storage
   int32_t Hm2;                           // second hidden width of the heads' MLPs, 0 = one hidden layer
+  int32_t nbr;                           // neighbourhood of Eq. 7: 0 = producers, 1 = producers and consumers
 };
 
 // bfloat16 = the upper 16 bits of an IEEE binary32; round to nearest, ties to even.
@@ -140,7 +141,15 @@ void encode_graph(const Model& m, const Weights& w, int32_t lo, int32_t hi,
   }
   dump(0);
 
-  // ---- Eq. 7, k times: h'_i = sigma( sum_{j in N_i} alpha_ij W h_j ),  N_i = in(i) + {i}.
+  // ---- Eq. 7, k times: h'_i = sigma( sum_{j in N_i} alpha_ij W h_j ),  N_i = in(i) + {i}, or with
+  // nbr = 1 the producers and the consumers of i and i itself ("neighbours of node i" read both ways);
+  // repeated edges count once each, in either direction.
+  std::vector<std::vector<int>> nbl(n);
+  for (int i = 0; i < n; ++i)
+    for (int e = rowptr[lo + i]; e < rowptr[lo + i + 1]; ++e) nbl[i].push_back(col[e] - lo);
+  if (m.nbr == 1)
+    for (int i = 0; i < n; ++i)      // i consumes col[e]: i is a consumer-side neighbour of that producer
+      for (int e = rowptr[lo + i]; e < rowptr[lo + i + 1]; ++e) nbl[col[e] - lo].push_back(i);
   for (int l = 0; l < m.L; ++l) {
     const float* W = w.W[l];
     std::vector<double> Ws(size_t(H) * H);
@@ -169,12 +178,13 @@ void encode_graph(const Model& m, const Weights& w, int32_t lo, int32_t hi,
     for (int i = 0; i < n; ++i) {
       const int gi = lo + i;
       const int e0 = rowptr[gi], e1 = rowptr[gi + 1];
-      const int deg = e1 - e0;
+      const int din = e1 - e0;                          // the first din neighbours are the producers
+      const int deg = int(nbl[i].size());
       std::vector<double> sc(deg + 1), al(deg + 1);
       for (int k = 0; k < K; ++k) {
         double mx = -INFINITY;
         for (int t = 0; t <= deg; ++t) {
-          const int j = (t < deg) ? col[e0 + t] - lo : i;   // last entry is the self term
+          const int j = (t < deg) ? nbl[i][t] : i;   // last entry is the self term
           sc[t] = leaky_relu(s_src[size_t(j) * K + k] + s_dst[size_t(i) * K + k]);
           if (sc[t] > mx) mx = sc[t];
         }
@@ -182,13 +192,13 @@ void encode_graph(const Model& m, const Weights& w, int32_t lo, int32_t hi,
         for (int t = 0; t <= deg; ++t) { al[t] = std::exp(sc[t] - mx); sum += al[t]; }
         for (int t = 0; t <= deg; ++t) al[t] /= sum;
         if (dump_layer == l + 1 && alpha_edge) {
-          for (int t = 0; t < deg; ++t) alpha_edge[size_t(e0 + t) * K + k] = al[t];
+          for (int t = 0; t < din; ++t) alpha_edge[size_t(e0 + t) * K + k] = al[t];
           alpha_self[size_t(gi) * K + k] = al[deg];
         }
         for (int c = k * d; c < (k + 1) * d; ++c) {
           double acc = 0.0;
           for (int t = 0; t <= deg; ++t) {
-            const int j = (t < deg) ? col[e0 + t] - lo : i;
+            const int j = (t < deg) ? nbl[i][t] : i;
             acc += al[t] * z[size_t(j) * H + c];
           }
           acc = relu(acc + double(w.b[l][c]));

@@ -19,7 +19,7 @@ _u8p = C.POINTER(C.c_uint8)
 
 
 class _Model(C.Structure):
-    _fields_ = [(k, C.c_int32) for k in ("T", "S", "H", "K", "L", "Hm", "Dg", "dtype", "Hm2")]
+    _fields_ = [(k, C.c_int32) for k in ("T", "S", "H", "K", "L", "Hm", "Dg", "dtype", "Hm2", "nbr")]
 
 
 def lib():
@@ -38,7 +38,7 @@ def _p(a, t):
 
 def _model(m):
     return _Model(m["T"], m["S"], m["H"], m["K"], m["L"], m["Hm"], m["Dg"],
-                  1 if m["dtype"] == "bf16" else 0, int(m.get("Hm2", 0)))
+                  1 if m["dtype"] == "bf16" else 0, int(m.get("Hm2", 0)), 1 if m.get("both_ways") else 0)
 
 
 def num_threads():

@@ -49,7 +49,8 @@ def gat_layer(g, h, W, l, m, return_alpha=False):
     Wl = W[f"W{l}"]
     Wl = bf16_round(Wl) if m["dtype"] == "bf16" else Wl.astype(np.float64)
     Z = h @ Wl
-    M = adjacency(g) + np.eye(n)
+    A = adjacency(g)
+    M = A + np.eye(n) + (A.T if m.get("both_ways") else 0.0)     # consumers count as neighbours too
     out = np.zeros((n, H))
     alphas = []
     for k in range(K):

@@ -41,6 +41,44 @@ def test_encoder_matches_dense_bruteforce(xo, dtype):
         np.testing.assert_allclose(out["emb"][gi], want, rtol=1e-12, atol=1e-12)
 
 
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_neighbourhood_both_ways_matches_dense_bruteforce(xo, dtype):
+    """Eq. 7 with the consumers of a node among its neighbours: dense row softmax weighted by A + A^T + I
+    (repeated edges count in both directions)."""
+    m = dict(M_SMALL, dtype=dtype, both_ways=True)
+    _, W = configs.make_weights(m, 15)
+    graphs = _tiny_graphs(9)
+    if dtype == "bf16":
+        for g in graphs:
+            g["shape"] = dags.round_to_bf16_grid(g["shape"])
+    b, p, out = _run(xo, m, W, graphs)
+    one_way = dict(m, both_ways=False)
+    for gi, g in enumerate(graphs):
+        want = dense_ref.encode_graph(g, W, m)
+        np.testing.assert_allclose(out["emb"][gi], want, rtol=1e-12, atol=1e-12)
+        assert not np.allclose(want, dense_ref.encode_graph(g, W, one_way))
+
+
+def test_both_ways_on_a_symmetric_graph_doubles_the_multiplicities(xo):
+    """If every edge j -> i comes with its reverse i -> j, reading the neighbourhood both ways only doubles
+    every neighbour's multiplicity: the softmax then weighs neighbours 2 : 1 against the self term, which
+    the one-way reading reproduces when each edge is listed twice."""
+    m = dict(M_SMALL, L=1)
+    _, W = configs.make_weights(m, 16)
+    rng = dags.make_rng(10)
+    g = dags.random_dag(rng, 10, 6, 8, False, window=5)
+    sym = dict(g, edge_src=np.concatenate([g["edge_src"], g["edge_dst"]]).astype(np.int32),
+               edge_dst=np.concatenate([g["edge_dst"], g["edge_src"]]).astype(np.int32))
+    twice = dict(sym, edge_src=np.concatenate([sym["edge_src"]] * 2), edge_dst=np.concatenate([sym["edge_dst"]] * 2))
+    # Eq. 6 sums over in-edges, so compare the attention layer alone: node features after layer 1 given equal h0
+    # is not observable separately; instead zero W0's edge block so that Eq. 6 ignores the edges
+    W = dict(W)
+    W0 = W["W0"].copy(); W0[:8] = 0.0; W["W0"] = W0
+    _, _, a = _run(xo, dict(m, both_ways=True), W, [sym])
+    _, _, b2 = _run(xo, m, W, [twice])
+    np.testing.assert_allclose(a["emb"], b2["emb"], rtol=1e-12, atol=1e-13)
+
+
 def _shuffle_edges(rng, g):
     perm = rng.permutation(len(g["edge_src"]))
     return dict(g, edge_src=g["edge_src"][perm], edge_dst=g["edge_dst"][perm])

@@ -30,6 +30,7 @@ MUTATIONS = [
     ("bf16 truncation instead of rounding", "u += 0x7FFFu + lsb;", "u += 0u * lsb;"),
     ("edge attributes read in CSR slot order", "double(edge_attr[size_t(eid[e]) * S + s])",
      "double(edge_attr[size_t(e) * S + s])"),
+    ("consumers listed under the wrong node", "nbl[col[e] - lo].push_back(i);", "nbl[i].push_back(col[e] - lo);"),
     ("second hidden layer without its ReLU", "out += relu(acc) * double(w2[c]);", "out += acc * double(w2[c]);"),
     ("second hidden layer's bias dropped", "double acc = double(bh[c]);", "double acc = 0.0;"),
     ("second hidden layer reads the first layer transposed", "acc += y1[k] * double(Wh[size_t(k) * hid2 + c]);",
@@ -67,6 +68,19 @@ def _pins_hold(xo):
             want = dense_ref.encode_graph(g, W, m, g0[gi])
             if not np.allclose(out["emb"][gi], want, rtol=1e-10, atol=1e-11):
                 return False
+    # consumers among the neighbours
+    m = dict(T=6, S=8, H=16, K=2, L=2, Hm=8, Dg=1, dtype="fp32", A_max=4, both_ways=True)
+    _, W = configs.make_weights(m, 23)
+    rng = dags.make_rng(12)
+    graphs = [dags.random_dag(rng, 12, 6, 8, False, window=6) for _ in range(3)]
+    b = dags.flatten(graphs, [0, len(graphs)], 4)
+    st, p = xo.pack(b)
+    if st != 0:
+        return False
+    out = xo.encode(m, configs.pack_weights(m, W), b, p)
+    for gi, g in enumerate(graphs):
+        if not np.allclose(out["emb"][gi], dense_ref.encode_graph(g, W, m), rtol=1e-10, atol=1e-11):
+            return False
     # attributes on the edges, edge lists shuffled
     m = dict(T=6, S=8, H=16, K=2, L=1, Hm=8, Dg=1, dtype="fp32", A_max=4)
     _, W = configs.make_weights(m, 19)
