@@ -75,6 +75,12 @@ typedef struct {
                               (taken from `shape`); 1: every edge has S attributes of its own, given with
                               xrl_batch_set_edge_attr after packing - Section 3.3.2 as written, where an
                               edge carries the shape of its tensor divided by the constant M             */
+  int32_t neighbourhood;   /* Eq. 7's neighbours of a node: 0 = its producers (and itself), 1 = its
+                              producers and its consumers (and itself) - "neighbours" read both ways;
+                              Eq. 6 sums over incoming edges either way.  With 1 the packer also
+                              builds the CSR by producer and a merged one (8 more bytes per edge and
+                              node), large batches are not packed range by range, and
+                              xrl_encode_delta is not available (XRL_ERR_UNSUPPORTED)            */
   int32_t max_actions;     /* A_max: padded number of candidate slots; No-Op is index A_max   */
   int32_t max_graphs;      /* capacity: graphs per batch                                      */
   int32_t max_envs;        /* capacity: environments per batch                                */

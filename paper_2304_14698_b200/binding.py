@@ -40,7 +40,7 @@ class _ModelConfig(C.Structure):
     _fields_ = [("num_op_types", C.c_int32), ("num_shape_feats", C.c_int32), ("hidden", C.c_int32),
                 ("heads", C.c_int32), ("layers", C.c_int32), ("mlp_hidden", C.c_int32),
                 ("mlp_hidden2", C.c_int32), ("global_dim", C.c_int32), ("dtype", C.c_int32),
-                ("edge_attributes", C.c_int32), ("max_actions", C.c_int32),
+                ("edge_attributes", C.c_int32), ("neighbourhood", C.c_int32), ("max_actions", C.c_int32),
                 ("max_graphs", C.c_int32), ("max_envs", C.c_int32), ("max_nodes", C.c_int64),
                 ("max_edges", C.c_int64)]
 
@@ -123,10 +123,11 @@ def _stream(stream):
 def model_config(m, max_graphs, max_envs, max_nodes, max_edges):
     """Build the C config from a dict with keys T, S, H, K, L, Hm, Dg, dtype, A_max and, optionally,
     Hm2 (second hidden width of the heads' MLPs, default 0 = one hidden layer) and edge_attr (True: the
-    model takes Eq. 6's edge attributes from the edges themselves, see xrl_batch_set_edge_attr)."""
+    model takes Eq. 6's edge attributes from the edges themselves, see xrl_batch_set_edge_attr) and
+    both_ways (True: Eq. 7's neighbours of a node are its producers and its consumers)."""
     return _ModelConfig(m["T"], m["S"], m["H"], m["K"], m["L"], m["Hm"], int(m.get("Hm2", 0)), m["Dg"],
                         XRL_BF16 if m["dtype"] in ("bf16", XRL_BF16) else XRL_FP32,
-                        1 if m.get("edge_attr") else 0, m["A_max"],
+                        1 if m.get("edge_attr") else 0, 1 if m.get("both_ways") else 0, m["A_max"],
                         int(max_graphs), int(max_envs), int(max_nodes), int(max_edges))
 
 

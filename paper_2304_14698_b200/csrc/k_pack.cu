@@ -348,6 +348,30 @@ int launch_permute_edge_rows(const void* src, const int32_t* eid, void* dst, int
   return 1;
 }
 
+// Neighbourhoods read both ways: row i of the merged CSR = row i of the CSR by consumer (i's producers),
+// then row i of the CSR by producer (i's consumers).  One thread per row copies both pieces.
+namespace {
+__global__ void k_merge_csr(const int32_t* __restrict__ rp_a, const int32_t* __restrict__ col_a,
+                            const int32_t* __restrict__ rp_b, const int32_t* __restrict__ col_b, int32_t N,
+                            int32_t* __restrict__ rp_m, int32_t* __restrict__ col_m) {
+  const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i > N) return;
+  const int32_t a0 = rp_a[i], b0 = rp_b[i];
+  rp_m[i] = a0 + b0;
+  if (i == N) return;
+  const int32_t na = rp_a[i + 1] - a0, nb = rp_b[i + 1] - b0;
+  int32_t* dst = col_m + a0 + b0;
+  for (int32_t t = 0; t < na; ++t) dst[t] = col_a[a0 + t];
+  for (int32_t t = 0; t < nb; ++t) dst[na + t] = col_b[b0 + t];
+}
+}  // namespace
+
+int launch_merge_csr(const int32_t* rp_a, const int32_t* col_a, const int32_t* rp_b, const int32_t* col_b,
+                     int32_t N, int32_t* rp_m, int32_t* col_m, cudaStream_t st) {
+  k_merge_csr<<<(N + 1 + 255) / 256, 256, 0, st>>>(rp_a, col_a, rp_b, col_b, N, rp_m, col_m);
+  return 1;
+}
+
 int launch_exclusive_scan(const int32_t* in, int32_t* out, int32_t n_in, int32_t* ws, cudaStream_t st) {
   return exclusive_scan(in, out, n_in, ws, st);
 }

@@ -100,6 +100,9 @@ struct xrl_batch {
   // contexts with attributes on the edges: slot -> input edge, the attributes as given and in slot order
   DeviceBuf eid, eattr_in, eattr;
   bool has_eattr = false;
+  // contexts whose attention layers read neighbourhoods both ways: CSR by producer, and the merged CSR
+  // (a node's producers, then its consumers) that those layers walk
+  DeviceBuf rowptr_out, col_out, rowptr_nbr, col_nbr;
   const int32_t *d_n_nodes = nullptr, *d_n_edges = nullptr, *d_env_off = nullptr,
                 *d_graph_chunk_off = nullptr, *d_chunk_row0 = nullptr, *d_chunk_row1 = nullptr;
   // Large batches packed from page-locked host memory are copied and packed in `nparts` ranges of whole
@@ -133,7 +136,10 @@ xrl_status check_config(const xrl_model_config& c) {
     return XRL_ERR_INVALID_ARG;
   if (c.num_shape_feats != kS || c.num_op_types > 256) return XRL_ERR_UNSUPPORTED;
   if (c.hidden % 32 != 0 || c.hidden > 512 || (c.hidden / c.heads) % 8 != 0) return XRL_ERR_UNSUPPORTED;
-  if (c.mlp_hidden2 < 0 || (c.edge_attributes != 0 && c.edge_attributes != 1)) return XRL_ERR_INVALID_ARG;
+  if (c.mlp_hidden2 < 0 || (c.edge_attributes != 0 && c.edge_attributes != 1) ||
+      (c.neighbourhood != 0 && c.neighbourhood != 1))
+    return XRL_ERR_INVALID_ARG;
+  if (c.neighbourhood == 1 && c.max_edges >= (int64_t(1) << 30)) return XRL_ERR_INVALID_ARG;   // 2 E entries
   if (c.layers > 64 || c.mlp_hidden > 1024 || c.mlp_hidden2 > 1024 || c.global_dim > 16) return XRL_ERR_UNSUPPORTED;
   if (c.max_actions > (1 << 20)) return XRL_ERR_UNSUPPORTED;
   return XRL_OK;
@@ -183,6 +189,9 @@ xrl_status alloc_batch(xrl_ctx* ctx, xrl_batch** out) {
   A(b->long_rows, 4 * (E / 32 + 1)); A(b->long_count, 4); A(b->coarse, 4 * (E / 1024 + 2));
   A(b->scan_ws, 4 * scan_workspace_ints(int64_t(N > B ? N : B) + 1));
   if (c.edge_attributes) { A(b->eid, 4 * E); A(b->eattr_in, sb * kS * E); A(b->eattr, sb * kS * E); }
+  if (c.neighbourhood) {
+    A(b->rowptr_out, 4 * (N + 1)); A(b->col_out, 4 * E); A(b->rowptr_nbr, 4 * (N + 1)); A(b->col_nbr, 8 * E);
+  }
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&b->staged, cudaEventDisableTiming);
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -311,7 +320,8 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
     const int64_t min_nodes = ev ? atoll(ev) : (int64_t(1) << 20);
     PackIn probe{};
     probe.B = num_graphs; probe.max_n = max_n; probe.max_m = max_m;
-    if (direct && num_graphs >= 2 && N >= min_nodes && min_nodes > 0 && pack_per_graph(probe)) {
+    if (direct && num_graphs >= 2 && N >= min_nodes && min_nodes > 0 && pack_per_graph(probe) &&
+        !c.neighbourhood) {                                       // (the merged CSR is built in one piece)
       const int64_t want = N / min_nodes;
       parts = int(want < 2 ? 2 : (want > xrl_batch::kMaxParts ? xrl_batch::kMaxParts : want));
       if (parts > num_graphs) parts = num_graphs;
@@ -400,6 +410,16 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
   if (parts == 0) {
     const size_t slot = ctx->prof.begin(st);
     ctx->launches_pack = launch_pack(in, po, c.num_op_types, ctx->status.as<int32_t>(), st);
+    if (c.neighbourhood) {
+      // the same packing with the edges reversed gives every node's consumers; then one merged CSR
+      PackIn rin = in;
+      rin.edge_src = in.edge_dst; rin.edge_dst = in.edge_src;
+      PackOut rpo = po;
+      rpo.rowptr = b->rowptr_out.as<int32_t>(); rpo.col = b->col_out.as<int32_t>(); rpo.eid = nullptr;
+      ctx->launches_pack += launch_pack(rin, rpo, c.num_op_types, ctx->status.as<int32_t>(), st);
+      ctx->launches_pack += launch_merge_csr(po.rowptr, po.col, rpo.rowptr, rpo.col, in.N,
+                                             b->rowptr_nbr.as<int32_t>(), b->col_nbr.as<int32_t>(), st);
+    }
     ctx->prof.end(FAM_PACK, slot, int(ctx->launches_pack), st);
   } else {
     // whatever still reads the batch's arrays was queued on the caller's stream before this call
@@ -460,6 +480,9 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
   const Window win{row_begin, row_end < 0 ? b->N : row_end, 0};   // graphs are independent: any range of whole graphs
   Profiler& pf = ctx->prof;
   const void* eattr = b->has_eattr ? b->eattr.p : nullptr;      // attributes on the edges, in slot order
+  // the attention layers walk the producers' CSR, or the merged one when consumers are neighbours too
+  const int32_t* gat_rowptr = ctx->cfg.neighbourhood ? b->rowptr_nbr.as<int32_t>() : b->rowptr.as<int32_t>();
+  const int32_t* gat_col = ctx->cfg.neighbourhood ? b->col_nbr.as<int32_t>() : b->col.as<int32_t>();
   size_t slot = pf.begin(st);
   int k = -1;
   if (ctx->use_umma_embed)
@@ -486,14 +509,14 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
     k = -1;
     bool fused_here = false;
     if (fuse_readout && l == layers - 1) {
-      k = launch_aggregate_tma(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), ctx->Z.p,
+      k = launch_aggregate_tma(d, gat_rowptr, gat_col, ctx->Z.p,
                                ctx->scores.as<float>(), ctx->dw.layer[l].b, ctx->h.p, win, b->N,
                                b->seg_id.as<int32_t>(), ctx->partial.as<float>(),
                                ctx->status.as<int32_t>(), st);
       if (k >= 0) { fused_here = true; if (fused) *fused = true; }
     }
     if (k < 0)
-      k = launch_aggregate(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), ctx->Z.p,
+      k = launch_aggregate(d, gat_rowptr, gat_col, ctx->Z.p,
                            ctx->scores.as<float>(), ctx->dw.layer[l].b,
                            ctx->h.p, win, b->N, ctx->status.as<int32_t>(), st);
     if (k < 0) return -1;
@@ -679,7 +702,7 @@ xrl_status xrl_batch_free(xrl_ctx* ctx, xrl_batch* b) {
   DeviceBuf* bufs[] = {&b->meta, &b->node_off, &b->edge_off, &b->seg_id, &b->graph_env, &b->rowptr,
                        &b->col, &b->op, &b->shape, &b->edge_src, &b->edge_dst, &b->deg, &b->tmp_eid,
                        &b->long_rows, &b->long_count, &b->scan_ws, &b->coarse, &b->eid, &b->eattr_in,
-                       &b->eattr};
+                       &b->eattr, &b->rowptr_out, &b->col_out, &b->rowptr_nbr, &b->col_nbr};
   for (DeviceBuf* d : bufs) d->release();
   if (b->h_meta) cudaFreeHost(b->h_meta);
   if (b->h_bulk) cudaFreeHost(b->h_bulk);
@@ -797,6 +820,7 @@ xrl_status xrl_encode_delta(xrl_ctx* ctx, const xrl_batch* b, const int32_t* bas
   const xrl_status s = check_batch(ctx, b);
   if (s != XRL_OK) return s;
   if (ctx->cfg.edge_attributes) return XRL_ERR_UNSUPPORTED;   // the node correspondence ignores edge attributes
+  if (ctx->cfg.neighbourhood) return XRL_ERR_UNSUPPORTED;     // a rewrite then reaches its producers' side too
   if (ctx->capturing) return XRL_ERR_STATE;        // reads the row counts back between layers
   if (!graph_emb && b->B > 0) return XRL_ERR_INVALID_ARG;
   XRL_CUDA(cudaSetDevice(ctx->device));

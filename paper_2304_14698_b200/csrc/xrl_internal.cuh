@@ -122,6 +122,8 @@ int launch_pack_offsets(const PackIn& in, const PackOut& out, cudaStream_t st);
 int launch_pack_graphs(const PackIn& in, const PackOut& out, int T, int32_t g0, int32_t g1, int32_t* status,
                        cudaStream_t st);
 size_t scan_workspace_ints(int64_t n);
+int launch_merge_csr(const int32_t* rp_a, const int32_t* col_a, const int32_t* rp_b, const int32_t* col_b,
+                     int32_t N, int32_t* rp_m, int32_t* col_m, cudaStream_t st);
 int launch_permute_edge_rows(const void* src, const int32_t* eid, void* dst, int64_t E, int row_bytes,
                              cudaStream_t st);
 // out[0..n_in] = exclusive prefix sums of in[0..n_in) (n_in + 1 outputs); ws: scan_workspace_ints(n_in) ints
