@@ -43,6 +43,12 @@ def _random_case(seed):
     m["A_max"] = A
     batch = dags.flatten(graphs, env_off, A)
     batch["mask"][rng.random(batch["mask"].shape) < 0.2] = 0
+    # every third case or so: attributes on the edges and / or neighbourhoods read both ways
+    if rng.random() < 0.35:
+        m["edge_attr"] = True
+        batch["edge_attr"] = dags.tensor_shape_attributes(grng, int(batch["n_edges"].sum()), 8, dtype == "bf16")
+    if rng.random() < 0.35:
+        m["both_ways"] = True
     batch["model"] = m
     # spoil some hints
     hint = batch["base_id"].copy()
@@ -53,7 +59,7 @@ def _random_case(seed):
     return batch, m, blob, hint, g0
 
 
-@pytest.mark.parametrize("seed", range(24))
+@pytest.mark.parametrize("seed", range(32))
 def test_random_batches(xo, seed):
     import torch
     import paper_2304_14698_b200 as xrl
@@ -72,7 +78,8 @@ def test_random_batches(xo, seed):
             assert np.array_equal(got_pack[k], packed[k]), (seed, k)
         g0d = None if g0 is None else torch.from_numpy(g0.astype(np.float32)).cuda()
         mask = torch.from_numpy(batch["mask"]).cuda()
-        for mode in ("full", "delta"):
+        # delta encoding is defined for the default reading only (producers' features, producers as neighbours)
+        for mode in ("full",) if (m.get("edge_attr") or m.get("both_ways")) else ("full", "delta"):
             bid = torch.from_numpy(hint).cuda() if mode == "delta" else None
             o = ag.forward(mask, sample=True, seed=seed, step=7, g0=g0d, base_id=bid)
             torch.cuda.synchronize()
