@@ -208,9 +208,13 @@ k_row_order_long(const int32_t* __restrict__ rowptr, const int2* __restrict__ tm
 // block scan, a scatter of (edge id, producer) pairs into the rows and the per-row rank restore all stay
 // on chip; global memory sees each edge once on the way in and each output once on the way out.  Rows of
 // graph g occupy col[edge_off[g] .. edge_off[g+1]), so no scan over all nodes is needed.
-constexpr int kGraphThreads = 512;
+// Threads per graph: 1,024 for graphs of thousands of nodes (one CTA per SM fits anyway: more threads hide
+// more latency), 512 for smaller graphs (several CTAs share an SM).
+constexpr int kGraphThreadsMax = 1024;
+inline int graph_threads(int32_t max_n) { return max_n >= 2048 ? 1024 : 512; }
 
-__global__ void __launch_bounds__(kGraphThreads)
+template <int NT>
+__global__ void __launch_bounds__(NT)
 k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ edge_off,
              const int32_t* __restrict__ op, const int32_t* __restrict__ edge_src,
              const int32_t* __restrict__ edge_dst, int32_t T, int32_t B, int32_t cap_n,
@@ -219,14 +223,14 @@ k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ e
   extern __shared__ __align__(16) int32_t psm[];
   int32_t* deg = psm;                         // [cap_n + 1] in-degree, then exclusive row starts
   int32_t* cur = psm + cap_n + 1;             // [cap_n]     row cursors
-  int32_t* wsum = cur + cap_n;                // [kGraphThreads / 32 + 1]
-  int2* tmp = reinterpret_cast<int2*>(wsum + kGraphThreads / 32 + 3);   // word 2 cap_n + 20: 8-byte aligned
+  int32_t* wsum = cur + cap_n;                // [kGraphThreadsMax / 32 + 1]
+  int2* tmp = reinterpret_cast<int2*>(wsum + kGraphThreadsMax / 32 + 3);   // word 2 cap_n + 20: 8-byte aligned
   const int32_t g = g_first + blockIdx.x;      // a launch may cover a range of the batch's graphs
   const int32_t nb = node_off[g], n = node_off[g + 1] - nb;
   const int32_t eb = edge_off[g], m = edge_off[g + 1] - eb;
   const int tid = threadIdx.x;
 
-  for (int32_t i = tid; i < n; i += kGraphThreads) {
+  for (int32_t i = tid; i < n; i += NT) {
     deg[i] = 0;
     cur[i] = 0;
     seg_id[nb + i] = g;
@@ -235,11 +239,11 @@ k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ e
   }
   __syncthreads();
   // edges four at a time per thread: the loads of a batch are issued before any of them is used
-  for (int32_t e0 = tid; e0 < m; e0 += 4 * kGraphThreads) {
+  for (int32_t e0 = tid; e0 < m; e0 += 4 * NT) {
     int32_t s[4], t[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const int32_t e = e0 + u * kGraphThreads;
+      const int32_t e = e0 + u * NT;
       s[u] = e < m ? __ldg(edge_src + eb + e) : 0;
       t[u] = e < m ? __ldg(edge_dst + eb + e) : -2;          // -2: no edge here
     }
@@ -252,7 +256,7 @@ k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ e
   }
   __syncthreads();
   // exclusive scan of deg[0..n): each thread scans a contiguous slice, warp / block offsets on top
-  const int32_t per = (n + kGraphThreads - 1) / kGraphThreads;
+  const int32_t per = (n + NT - 1) / NT;
   const int32_t a0 = min(n, tid * per), a1 = min(n, a0 + per);
   int32_t sum = 0;
   for (int32_t i = a0; i < a1; ++i) sum += deg[i];
@@ -269,31 +273,31 @@ k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ e
   for (int w = 0; w < wid; ++w) wbase += wsum[w];
   int32_t run = wbase + incl - sum;
   for (int32_t i = a0; i < a1; ++i) { const int32_t dgr = deg[i]; deg[i] = run; run += dgr; }
-  if (tid == kGraphThreads - 1) deg[n] = run;          // valid edges of the graph
+  if (tid == NT - 1) deg[n] = run;          // valid edges of the graph
   __syncthreads();
-  for (int32_t i = tid; i < n; i += kGraphThreads) rowptr[nb + i] = eb + deg[i];
+  for (int32_t i = tid; i < n; i += NT) rowptr[nb + i] = eb + deg[i];
   if (g == B - 1 && tid == 0) rowptr[nb + n] = eb + deg[n];
   // the last graph of a partial launch closes its last row itself (the next graph's CTA, which writes the
   // same value as its first row start, may run much later)
   else if (blockIdx.x == gridDim.x - 1 && tid == 0) rowptr[nb + n] = edge_off[g + 1];
   // scatter (edge id, global producer) into the rows, slot order as the atomics hand it out
-  for (int32_t e0 = tid; e0 < m; e0 += 4 * kGraphThreads) {
+  for (int32_t e0 = tid; e0 < m; e0 += 4 * NT) {
     int32_t s[4], t[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const int32_t e = e0 + u * kGraphThreads;
+      const int32_t e = e0 + u * NT;
       s[u] = e < m ? __ldg(edge_src + eb + e) : 0;
       t[u] = e < m ? __ldg(edge_dst + eb + e) : -2;
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       if (t[u] == -2 || s[u] < 0 || s[u] >= n || t[u] < 0 || t[u] >= n || s[u] == t[u]) continue;
-      tmp[deg[t[u]] + atomicAdd(&cur[t[u]], 1)] = make_int2(e0 + u * kGraphThreads, nb + s[u]);
+      tmp[deg[t[u]] + atomicAdd(&cur[t[u]], 1)] = make_int2(e0 + u * NT, nb + s[u]);
     }
   }
   __syncthreads();
   // rank of each edge id inside its row restores the input order; short rows by one thread ...
-  for (int32_t i = tid; i < n; i += kGraphThreads) {
+  for (int32_t i = tid; i < n; i += NT) {
     const int32_t b = deg[i], k = deg[i + 1] - b;
     if (k == 1) { col[eb + b] = tmp[b].y; if (eid) eid[eb + b] = eb + tmp[b].x; }
     else if (k > 1 && k <= kShortRow)
@@ -306,7 +310,7 @@ k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ e
       }
   }
   // ... long rows by one warp each
-  for (int32_t i = wid; i < n; i += kGraphThreads / 32) {
+  for (int32_t i = wid; i < n; i += NT / 32) {
     const int32_t b = deg[i], k = deg[i + 1] - b;
     if (k <= kShortRow) continue;
     for (int32_t a = lane; a < k; a += 32) {
@@ -320,7 +324,7 @@ k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ e
 }
 
 size_t pack_graph_smem(int32_t cap_n, int32_t cap_m) {
-  return 4 * size_t(2 * cap_n + 1 + kGraphThreads / 32 + 3) + 8 * size_t(cap_m) + 16;
+  return 4 * size_t(2 * cap_n + 1 + kGraphThreadsMax / 32 + 3) + 8 * size_t(cap_m) + 16;
 }
 
 }  // namespace
@@ -410,11 +414,19 @@ int launch_pack_offsets(const PackIn& in, const PackOut& out, cudaStream_t st) {
 int launch_pack_graphs(const PackIn& in, const PackOut& out, int T, int32_t g0, int32_t g1, int32_t* status,
                        cudaStream_t st) {
   if (g1 <= g0) return 0;
-  static bool attr[64] = {};
-  ensure_dynamic_smem(k_pack_graph, 160 * 1024, attr);
-  k_pack_graph<<<g1 - g0, kGraphThreads, pack_graph_smem(in.max_n, in.max_m), st>>>(
-      out.node_off, out.edge_off, in.op, in.edge_src, in.edge_dst, T, in.B, in.max_n, out.seg_id,
-      out.rowptr, out.col, status, g0, out.eid);
+  static bool attr512[64] = {}, attr1024[64] = {};
+  const size_t smem = pack_graph_smem(in.max_n, in.max_m);
+  if (graph_threads(in.max_n) == 1024) {
+    ensure_dynamic_smem(k_pack_graph<1024>, 160 * 1024, attr1024);
+    k_pack_graph<1024><<<g1 - g0, 1024, smem, st>>>(out.node_off, out.edge_off, in.op, in.edge_src, in.edge_dst, T,
+                                                    in.B, in.max_n, out.seg_id, out.rowptr, out.col, status, g0,
+                                                    out.eid);
+  } else {
+    ensure_dynamic_smem(k_pack_graph<512>, 160 * 1024, attr512);
+    k_pack_graph<512><<<g1 - g0, 512, smem, st>>>(out.node_off, out.edge_off, in.op, in.edge_src, in.edge_dst, T,
+                                                  in.B, in.max_n, out.seg_id, out.rowptr, out.col, status, g0,
+                                                  out.eid);
+  }
   return 1;
 }
 
