@@ -14,6 +14,9 @@
 //                                   mask, No-Op action; Section 3.3.3 invalid-action masking
 //   xo_sample        Section 3.3.2  the action is drawn from the categorical distribution;
 //                                   random words from Philox4x32-10 (Salmon et al., SC'11)
+//   xo_ppo_grad      Section 3.3.4  Eq. 3 (clipped objective), Eq. 4 (value loss), Eq. 5 (their sum with an
+//                                   entropy term) over a mini-batch, and the gradient with respect to every
+//                                   weight; xo_gae: the generalised advantage estimates it is fed with
 // Readings of what the paper leaves open (activation = ReLU, LeakyReLU slope 0.2 inside the
 // attention score, in-neighbours plus self, heads concatenated, biases, a weight matrix in
 // Eq. 8, per-graph scoring for the policy) are listed in the design notes of the repository.
@@ -245,6 +248,274 @@ double mlp_scalar(const double* x, int in, int hid, int hid2, const float* W1, c
   return out;
 }
 
+// ---- Section 3.3.4: the PPO objective of one mini-batch (Eq. 3, 4, 5) and its gradient ---------------
+// A mini-batch is a packed batch whose environments are stored transitions: environment e holds the state
+// (current graph + candidates), the action that was taken there, the old policy's log-probability of it,
+// its advantage estimate and its value target.
+//   ratio_e = pi(a_e | s_e) / pi_old(a_e | s_e)
+//   L_clip  = - mean_e min(ratio_e A_e, clip(ratio_e, 1 - eps, 1 + eps) A_e)          (Eq. 3)
+//   L_vf    =   mean_e (V(s_e) - R_e)^2                                                (Eq. 4)
+//   L_ent   =   mean_e sum_a pi(a | s_e) log pi(a | s_e)        (minus the entropy, over the valid actions)
+//   J       =   L_clip + c1 L_vf + c2 L_ent                                            (Eq. 5)
+// The gradient is taken by hand, layer by layer in reverse, with respect to every entry of the weight blob
+// (for a bf16 model: with respect to the stored, rounded values).  ReLU'(0) = 0, LeakyReLU'(0) = 0.2, and
+// the derivative of the clipped objective is that of whichever term of the min is the smaller one.
+
+// Forward intermediates of one graph that the reverse pass needs.
+struct GraphTape {
+  int n = 0;
+  std::vector<std::vector<int>> nbl;                 // neighbours of each node (self excluded)
+  std::vector<double> x0;                            // [n x F0] inputs of Eq. 6
+  std::vector<std::vector<double>> h;                // h[l]: [n x H] after Eq. 6 (l = 0) and after layer l
+  std::vector<std::vector<double>> z, s_src, s_dst;  // per layer: [n x H], [n x K], [n x K]
+  std::vector<std::vector<double>> alpha;            // per layer: for node i, head k: deg_i + 1 weights, packed
+  std::vector<size_t> aoff;                          // start of node i's weights inside alpha[l] (times K)
+  std::vector<double> u, emb;                        // Eq. 8 input [H + Dg] and output [H]
+};
+
+void forward_tape(const Model& m, const Weights& w, int32_t lo, int32_t hi, const int32_t* rowptr,
+                  const int32_t* col, const int32_t* op, const float* shape, const double* g_attr,
+                  const float* edge_attr, const int32_t* eid, GraphTape& tp) {
+  const int S = m.S, T = m.T, H = m.H, K = m.K, d = m.H / m.K, F0 = 2 * S + T;
+  const int n = hi - lo;
+  tp.n = n;
+  tp.nbl.assign(n, {});
+  for (int i = 0; i < n; ++i)
+    for (int e = rowptr[lo + i]; e < rowptr[lo + i + 1]; ++e) tp.nbl[i].push_back(col[e] - lo);
+  if (m.nbr == 1)
+    for (int i = 0; i < n; ++i)
+      for (int e = rowptr[lo + i]; e < rowptr[lo + i + 1]; ++e) tp.nbl[col[e] - lo].push_back(i);
+  tp.aoff.assign(n + 1, 0);
+  for (int i = 0; i < n; ++i) tp.aoff[i + 1] = tp.aoff[i] + tp.nbl[i].size() + 1;
+  tp.x0.assign(size_t(n) * F0, 0.0);
+  tp.h.assign(m.L + 1, std::vector<double>(size_t(n) * H));
+  tp.z.assign(m.L, std::vector<double>(size_t(n) * H));
+  tp.s_src.assign(m.L, std::vector<double>(size_t(n) * K));
+  tp.s_dst.assign(m.L, std::vector<double>(size_t(n) * K));
+  tp.alpha.assign(m.L, std::vector<double>(tp.aoff[n] * K));
+  // Eq. 6
+  for (int i = 0; i < n; ++i) {
+    const int gi = lo + i;
+    double* x = &tp.x0[size_t(i) * F0];
+    for (int e = rowptr[gi]; e < rowptr[gi + 1]; ++e)
+      for (int s = 0; s < S; ++s)
+        x[s] += edge_attr ? double(edge_attr[size_t(eid[e]) * S + s]) : double(shape[size_t(col[e]) * S + s]);
+    x[S + op[gi]] = 1.0;
+    for (int s = 0; s < S; ++s) x[S + T + s] = double(shape[size_t(gi) * S + s]);
+    for (int c = 0; c < H; ++c) {
+      double acc = double(w.b0[c]);
+      for (int s = 0; s < F0; ++s) acc += x[s] * stored(m, w.W0[size_t(s) * H + c]);
+      tp.h[0][size_t(i) * H + c] = relu(acc);
+    }
+  }
+  // Eq. 7
+  for (int l = 0; l < m.L; ++l) {
+    const std::vector<double>& hin = tp.h[l];
+    std::vector<double>& z = tp.z[l];
+    for (int i = 0; i < n; ++i)
+      for (int c = 0; c < H; ++c) {
+        double acc = 0.0;
+        for (int k = 0; k < H; ++k) acc += hin[size_t(i) * H + k] * stored(m, w.W[l][size_t(k) * H + c]);
+        z[size_t(i) * H + c] = acc;
+      }
+    for (int i = 0; i < n; ++i)
+      for (int k = 0; k < K; ++k) {
+        double ss = 0.0, sd = 0.0;
+        for (int c = 0; c < d; ++c) {
+          ss += double(w.a_src[l][k * d + c]) * z[size_t(i) * H + k * d + c];
+          sd += double(w.a_dst[l][k * d + c]) * z[size_t(i) * H + k * d + c];
+        }
+        tp.s_src[l][size_t(i) * K + k] = ss;
+        tp.s_dst[l][size_t(i) * K + k] = sd;
+      }
+    for (int i = 0; i < n; ++i) {
+      const int deg = int(tp.nbl[i].size());
+      for (int k = 0; k < K; ++k) {
+        double* al = &tp.alpha[l][(tp.aoff[i]) * K + size_t(k) * (deg + 1)];
+        double mx = -INFINITY;
+        for (int t = 0; t <= deg; ++t) {
+          const int j = (t < deg) ? tp.nbl[i][t] : i;
+          al[t] = leaky_relu(tp.s_src[l][size_t(j) * K + k] + tp.s_dst[l][size_t(i) * K + k]);
+          if (al[t] > mx) mx = al[t];
+        }
+        double sum = 0.0;
+        for (int t = 0; t <= deg; ++t) { al[t] = std::exp(al[t] - mx); sum += al[t]; }
+        for (int t = 0; t <= deg; ++t) al[t] /= sum;
+        for (int c = k * d; c < (k + 1) * d; ++c) {
+          double acc = 0.0;
+          for (int t = 0; t <= deg; ++t) acc += al[t] * z[size_t((t < deg) ? tp.nbl[i][t] : i) * H + c];
+          tp.h[l + 1][size_t(i) * H + c] = relu(acc + double(w.b[l][c]));
+        }
+      }
+    }
+  }
+  // Eq. 8
+  tp.u.assign(H + m.Dg, 0.0);
+  tp.emb.assign(H, 0.0);
+  for (int i = 0; i < n; ++i)
+    for (int c = 0; c < H; ++c) tp.u[c] += tp.h[m.L][size_t(i) * H + c];
+  for (int c = 0; c < m.Dg; ++c) tp.u[H + c] = g_attr ? g_attr[c] : 0.0;
+  for (int c = 0; c < H; ++c) {
+    double acc = double(w.bg[c]);
+    for (int k = 0; k < H + m.Dg; ++k) acc += tp.u[k] * double(w.Wg[size_t(k) * H + c]);
+    tp.emb[c] = relu(acc);
+  }
+}
+
+// Reverse pass of one graph: demb = dJ / d emb of this graph; adds into the blob-shaped gradient `g`
+// (pointers of `gw` address it the way `w` addresses the weights).
+struct GradPtrs {
+  double* W0; double* b0;
+  std::vector<double*> W, a_src, a_dst, b;
+  double* Wg; double* bg;
+  double *pW1, *pb1, *pWh, *pbh, *pw2, *pb2, *vW1, *vb1, *vWh, *vbh, *vw2, *vb2;
+};
+
+void backward_graph(const Model& m, const Weights& w, const GraphTape& tp, const double* demb, GradPtrs& gw) {
+  const int S = m.S, T = m.T, H = m.H, K = m.K, d = m.H / m.K, F0 = 2 * S + T, n = tp.n;
+  // Eq. 8
+  std::vector<double> dpre(H), du(H + m.Dg, 0.0);
+  for (int c = 0; c < H; ++c) dpre[c] = tp.emb[c] > 0.0 ? demb[c] : 0.0;
+  for (int k = 0; k < H + m.Dg; ++k)
+    for (int c = 0; c < H; ++c) {
+      gw.Wg[size_t(k) * H + c] += tp.u[k] * dpre[c];
+      du[k] += double(w.Wg[size_t(k) * H + c]) * dpre[c];
+    }
+  for (int c = 0; c < H; ++c) gw.bg[c] += dpre[c];
+  std::vector<double> dh(size_t(n) * H), dz(size_t(n) * H), dhin(size_t(n) * H);
+  for (int i = 0; i < n; ++i)
+    for (int c = 0; c < H; ++c) dh[size_t(i) * H + c] = du[c];      // the readout is a plain sum
+  // Eq. 7, last layer first
+  for (int l = m.L - 1; l >= 0; --l) {
+    const std::vector<double>& hout = tp.h[l + 1];
+    const std::vector<double>& hin = tp.h[l];
+    const std::vector<double>& z = tp.z[l];
+    std::vector<double> ds_src(size_t(n) * K, 0.0), ds_dst(size_t(n) * K, 0.0);
+    std::fill(dz.begin(), dz.end(), 0.0);
+    for (int i = 0; i < n; ++i) {
+      const int deg = int(tp.nbl[i].size());
+      std::vector<double> dal(deg + 1);
+      for (int k = 0; k < K; ++k) {
+        const double* al = &tp.alpha[l][(tp.aoff[i]) * K + size_t(k) * (deg + 1)];
+        // through ReLU and the bias
+        double dp[512];
+        for (int c = 0; c < d; ++c) {
+          const int cc = k * d + c;
+          dp[c] = hout[size_t(i) * H + cc] > 0.0 ? dh[size_t(i) * H + cc] : 0.0;
+          gw.b[l][cc] += dp[c];
+        }
+        // out = sum_t al[t] z_{j_t}: to the weights and to the gathered rows
+        for (int t = 0; t <= deg; ++t) {
+          const int j = (t < deg) ? tp.nbl[i][t] : i;
+          double acc = 0.0;
+          for (int c = 0; c < d; ++c) {
+            acc += dp[c] * z[size_t(j) * H + k * d + c];
+            dz[size_t(j) * H + k * d + c] += al[t] * dp[c];
+          }
+          dal[t] = acc;
+        }
+        // softmax, then LeakyReLU, then the sum of the two half-scores
+        double dot = 0.0;
+        for (int t = 0; t <= deg; ++t) dot += al[t] * dal[t];
+        for (int t = 0; t <= deg; ++t) {
+          const int j = (t < deg) ? tp.nbl[i][t] : i;
+          const double e = tp.s_src[l][size_t(j) * K + k] + tp.s_dst[l][size_t(i) * K + k];
+          const double de = al[t] * (dal[t] - dot) * (e > 0.0 ? 1.0 : 0.2);
+          ds_src[size_t(j) * K + k] += de;
+          ds_dst[size_t(i) * K + k] += de;
+        }
+      }
+    }
+    // half-scores are dot products of z with the attention vectors
+    for (int i = 0; i < n; ++i)
+      for (int k = 0; k < K; ++k)
+        for (int c = 0; c < d; ++c) {
+          const int cc = k * d + c;
+          const double zs = z[size_t(i) * H + cc];
+          gw.a_src[l][cc] += ds_src[size_t(i) * K + k] * zs;
+          gw.a_dst[l][cc] += ds_dst[size_t(i) * K + k] * zs;
+          dz[size_t(i) * H + cc] += ds_src[size_t(i) * K + k] * double(w.a_src[l][cc]) +
+                                    ds_dst[size_t(i) * K + k] * double(w.a_dst[l][cc]);
+        }
+    // z = h W
+    for (int i = 0; i < n; ++i)
+      for (int k = 0; k < H; ++k) {
+        double acc = 0.0;
+        for (int c = 0; c < H; ++c) {
+          gw.W[l][size_t(k) * H + c] += hin[size_t(i) * H + k] * dz[size_t(i) * H + c];
+          acc += stored(m, w.W[l][size_t(k) * H + c]) * dz[size_t(i) * H + c];
+        }
+        dhin[size_t(i) * H + k] = acc;
+      }
+    dh.swap(dhin);
+  }
+  // Eq. 6
+  for (int i = 0; i < n; ++i)
+    for (int c = 0; c < H; ++c) {
+      const double dp = tp.h[0][size_t(i) * H + c] > 0.0 ? dh[size_t(i) * H + c] : 0.0;
+      gw.b0[c] += dp;
+      for (int s = 0; s < F0; ++s) gw.W0[size_t(s) * H + c] += tp.x0[size_t(i) * F0 + s] * dp;
+    }
+}
+
+// A head's MLP forward keeping its hidden activations, and its reverse pass given d out.
+struct MlpTape { std::vector<double> y1, y2; };
+double mlp_forward_tape(const double* x, int in, int hid, int hid2, const float* W1, const float* b1,
+                        const float* Wh, const float* bh, const float* w2, const float* b2, MlpTape& tp) {
+  tp.y1.assign(hid, 0.0);
+  tp.y2.assign(hid2 > 0 ? hid2 : 0, 0.0);
+  for (int c = 0; c < hid; ++c) {
+    double acc = double(b1[c]);
+    for (int k = 0; k < in; ++k) acc += x[k] * double(W1[size_t(k) * hid + c]);
+    tp.y1[c] = relu(acc);
+  }
+  double out = double(b2[0]);
+  if (hid2 <= 0) {
+    for (int c = 0; c < hid; ++c) out += tp.y1[c] * double(w2[c]);
+    return out;
+  }
+  for (int c = 0; c < hid2; ++c) {
+    double acc = double(bh[c]);
+    for (int k = 0; k < hid; ++k) acc += tp.y1[k] * double(Wh[size_t(k) * hid2 + c]);
+    tp.y2[c] = relu(acc);
+    out += tp.y2[c] * double(w2[c]);
+  }
+  return out;
+}
+void mlp_backward(const double* x, int in, int hid, int hid2, const float* W1, const float* Wh, const float* w2,
+                  const MlpTape& tp, double dout, double* gW1, double* gb1, double* gWh, double* gbh,
+                  double* gw2, double* gb2, double* dx) {
+  gb2[0] += dout;
+  std::vector<double> dy1(hid, 0.0);
+  if (hid2 <= 0) {
+    for (int c = 0; c < hid; ++c) {
+      gw2[c] += tp.y1[c] * dout;
+      dy1[c] = tp.y1[c] > 0.0 ? double(w2[c]) * dout : 0.0;
+    }
+  } else {
+    for (int c = 0; c < hid2; ++c) {
+      gw2[c] += tp.y2[c] * dout;
+      const double da = tp.y2[c] > 0.0 ? double(w2[c]) * dout : 0.0;
+      gbh[c] += da;
+      for (int k = 0; k < hid; ++k) {
+        gWh[size_t(k) * hid2 + c] += tp.y1[k] * da;
+        dy1[k] += double(Wh[size_t(k) * hid2 + c]) * da;
+      }
+    }
+    for (int k = 0; k < hid; ++k)
+      if (!(tp.y1[k] > 0.0)) dy1[k] = 0.0;
+  }
+  for (int c = 0; c < hid; ++c) gb1[c] += dy1[c];
+  for (int k = 0; k < in; ++k) {
+    double acc = 0.0;
+    for (int c = 0; c < hid; ++c) {
+      gW1[size_t(k) * hid + c] += x[k] * dy1[c];
+      acc += double(W1[size_t(k) * hid + c]) * dy1[c];
+    }
+    if (dx) dx[k] += acc;
+  }
+}
+
 inline void mulhilo(uint32_t a, uint32_t b, uint32_t& hi, uint32_t& lo) {
   uint64_t p = uint64_t(a) * uint64_t(b);
   hi = uint32_t(p >> 32);
@@ -418,6 +689,141 @@ int xo_sample(int32_t num_envs, int32_t A1, const float* probs, uint64_t seed, u
       }
     }
     action[e] = act;
+  }
+  return XO_OK;
+}
+
+// Eq. 3-5 over the environments of a packed batch and the gradient of J with respect to the weight blob.
+// action [num_envs] in [0, A_max] (A_max = No-Op) must be a valid action of its environment; logp_old, adv,
+// ret [num_envs]; loss_out[4] = {J, L_clip, L_vf, L_ent}; grad = blob-shaped, double; logp_out (optional,
+// [num_envs]) receives log pi(a_e | s_e) of the current weights.
+int xo_ppo_grad(const Model* m, const float* weights, int32_t B, const int32_t* node_off,
+                const int32_t* rowptr, const int32_t* col, const int32_t* op, const float* shape,
+                const double* g0, const float* edge_attr, const int32_t* eid, int32_t num_envs,
+                const int32_t* env_off, int32_t A_max, const uint8_t* mask, const int32_t* action,
+                const double* logp_old, const double* adv, const double* ret, double eps, double c1,
+                double c2, double* loss_out, double* grad, double* logp_out) {
+  if (m->H % m->K != 0 || m->L < 0 || num_envs <= 0 || m->H / m->K > 512) return XO_INVALID_ARG;
+  if (edge_attr && !eid) return XO_INVALID_ARG;
+  const Weights w = slice(*m, weights);
+  const int H = m->H;
+  // gradient pointers laid out like the blob
+  GradPtrs gw;
+  {
+    double* p = grad;
+    auto take = [&](int64_t nn) { double* q = p; p += nn; return q; };
+    const int last = m->Hm2 > 0 ? m->Hm2 : m->Hm;
+    gw.W0 = take(int64_t(2 * m->S + m->T) * H); gw.b0 = take(H);
+    for (int l = 0; l < m->L; ++l) {
+      gw.W.push_back(take(int64_t(H) * H)); gw.a_src.push_back(take(H));
+      gw.a_dst.push_back(take(H)); gw.b.push_back(take(H));
+    }
+    gw.Wg = take(int64_t(H + m->Dg) * H); gw.bg = take(H);
+    gw.pW1 = take(int64_t(H) * m->Hm); gw.pb1 = take(m->Hm);
+    gw.pWh = take(int64_t(m->Hm) * m->Hm2); gw.pbh = take(m->Hm2);
+    gw.pw2 = take(last); gw.pb2 = take(1);
+    gw.vW1 = take(int64_t(2 * H) * m->Hm); gw.vb1 = take(m->Hm);
+    gw.vWh = take(int64_t(m->Hm) * m->Hm2); gw.vbh = take(m->Hm2);
+    gw.vw2 = take(last); gw.vb2 = take(1);
+    for (double* q = grad; q < p; ++q) *q = 0.0;
+  }
+  // forward of every graph, kept
+  std::vector<GraphTape> tapes(B);
+  for (int g = 0; g < B; ++g)
+    forward_tape(*m, w, node_off[g], node_off[g + 1], rowptr, col, op, shape,
+                 g0 ? g0 + size_t(g) * m->Dg : nullptr, edge_attr, eid, tapes[g]);
+  std::vector<double> demb(size_t(B) * H, 0.0);
+  double Lclip = 0.0, Lvf = 0.0, Lent = 0.0;
+  const double inv_ne = 1.0 / double(num_envs);
+  for (int e = 0; e < num_envs; ++e) {
+    const int cur = env_off[e];
+    const int C = env_off[e + 1] - cur - 1;
+    if (C < 0 || C > A_max) return XO_INVALID_ARG;
+    const int A1 = A_max + 1;
+    // policy logits of the valid actions, their MLP tapes
+    std::vector<double> lg(A1, -INFINITY), pr(A1, 0.0);
+    std::vector<MlpTape> mt(A1);
+    double mx = -INFINITY;
+    for (int a = 0; a < A1; ++a) {
+      const bool valid = (a == A_max) || (a < C && mask[size_t(e) * A_max + a]);
+      if (a < A_max && a >= C && mask[size_t(e) * A_max + a]) return XO_INVALID_ARG;
+      if (!valid) continue;
+      const int g = (a == A_max) ? cur : cur + 1 + a;
+      lg[a] = mlp_forward_tape(tapes[g].emb.data(), H, m->Hm, m->Hm2, w.pW1, w.pb1, w.pWh, w.pbh, w.pw2,
+                               w.pb2, mt[a]);
+      if (lg[a] > mx) mx = lg[a];
+    }
+    double sum = 0.0;
+    for (int a = 0; a < A1; ++a)
+      if (lg[a] != -INFINITY) { pr[a] = std::exp(lg[a] - mx); sum += pr[a]; }
+    for (int a = 0; a < A1; ++a) pr[a] /= sum;
+    const int act = action[e];
+    if (act < 0 || act > A_max || lg[act] == -INFINITY) return XO_INVALID_ARG;
+    const double logp = (lg[act] - mx) - std::log(sum);
+    if (logp_out) logp_out[e] = logp;
+    // Eq. 3
+    const double ratio = std::exp(logp - logp_old[e]);
+    const double clipped = ratio < 1.0 - eps ? 1.0 - eps : (ratio > 1.0 + eps ? 1.0 + eps : ratio);
+    const double t1 = ratio * adv[e], t2 = clipped * adv[e];
+    Lclip += -(t1 <= t2 ? t1 : t2) * inv_ne;
+    const double dlogp = (t1 <= t2) ? -adv[e] * ratio * inv_ne : 0.0;   // the clipped term is flat where it is active
+    // entropy term
+    double plogp = 0.0;
+    for (int a = 0; a < A1; ++a)
+      if (pr[a] > 0.0) plogp += pr[a] * std::log(pr[a]);
+    Lent += plogp * inv_ne;
+    // d J / d logit_b = dlogp (1[b = act] - p_b) + c2 / Ne * p_b (log p_b - sum_a p_a log p_a)
+    for (int a = 0; a < A1; ++a) {
+      if (lg[a] == -INFINITY) continue;
+      double dl = dlogp * ((a == act ? 1.0 : 0.0) - pr[a]);
+      if (pr[a] > 0.0) dl += c2 * inv_ne * pr[a] * (std::log(pr[a]) - plogp);
+      const int g = (a == A_max) ? cur : cur + 1 + a;
+      mlp_backward(tapes[g].emb.data(), H, m->Hm, m->Hm2, w.pW1, w.pWh, w.pw2, mt[a], dl, gw.pW1, gw.pb1,
+                   gw.pWh, gw.pbh, gw.pw2, gw.pb2, &demb[size_t(g) * H]);
+    }
+    // Eq. 4: value head over [ current graph || mean of the valid candidates ]
+    std::vector<double> u(2 * H, 0.0), du(2 * H, 0.0);
+    int nv = 0;
+    for (int c = 0; c < H; ++c) u[c] = tapes[cur].emb[c];
+    for (int a = 0; a < C; ++a)
+      if (mask[size_t(e) * A_max + a]) {
+        ++nv;
+        for (int c = 0; c < H; ++c) u[H + c] += tapes[cur + 1 + a].emb[c];
+      }
+    if (nv > 0)
+      for (int c = 0; c < H; ++c) u[H + c] /= double(nv);
+    MlpTape vt;
+    const double v = mlp_forward_tape(u.data(), 2 * H, m->Hm, m->Hm2, w.vW1, w.vb1, w.vWh, w.vbh, w.vw2,
+                                      w.vb2, vt);
+    Lvf += (v - ret[e]) * (v - ret[e]) * inv_ne;
+    mlp_backward(u.data(), 2 * H, m->Hm, m->Hm2, w.vW1, w.vWh, w.vw2, vt, c1 * 2.0 * (v - ret[e]) * inv_ne,
+                 gw.vW1, gw.vb1, gw.vWh, gw.vbh, gw.vw2, gw.vb2, du.data());
+    for (int c = 0; c < H; ++c) demb[size_t(cur) * H + c] += du[c];
+    if (nv > 0)
+      for (int a = 0; a < C; ++a)
+        if (mask[size_t(e) * A_max + a])
+          for (int c = 0; c < H; ++c) demb[size_t(cur + 1 + a) * H + c] += du[H + c] / double(nv);
+  }
+  for (int g = 0; g < B; ++g) backward_graph(*m, w, tapes[g], &demb[size_t(g) * H], gw);
+  loss_out[0] = Lclip + c1 * Lvf + c2 * Lent;
+  loss_out[1] = Lclip; loss_out[2] = Lvf; loss_out[3] = Lent;
+  return XO_OK;
+}
+
+// Generalised advantage estimation over one trajectory of T steps (the estimator the paper takes its
+// advantages from): delta_t = r_t + gamma V_{t+1} (1 - done_t) - V_t,
+// A_t = delta_t + gamma lambda (1 - done_t) A_{t+1}; value targets R_t = A_t + V_t.  values has T + 1 entries
+// (the last one bootstraps the tail).
+int xo_gae(int32_t T, const double* reward, const double* values, const uint8_t* done, double gamma,
+           double lambda, double* adv, double* ret) {
+  if (T < 0) return XO_INVALID_ARG;
+  double run = 0.0;
+  for (int t = T - 1; t >= 0; --t) {
+    const double nd = done[t] ? 0.0 : 1.0;
+    const double delta = reward[t] + gamma * values[t + 1] * nd - values[t];
+    run = delta + gamma * lambda * nd * run;
+    adv[t] = run;
+    ret[t] = run + values[t];
   }
   return XO_OK;
 }

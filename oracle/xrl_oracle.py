@@ -142,3 +142,56 @@ def forward(m, weights, batch, g0=None, threads=0, mode=0):
     if st != 0:
         raise ValueError(f"xo_policy_value status {st}")
     return {"packed": packed, "emb": enc["emb"], "logits": logits, "probs": probs, "value": value}
+
+
+def ppo_grad(m, weights, batch, packed, action, logp_old, adv, ret, eps=0.2, c1=0.5, c2=0.01, g0=None,
+             mask=None, edge_attr=None):
+    """Section 3.3.4, Eq. 3-5 over the environments of the batch (each a stored transition) and the gradient
+    of J with respect to the weight blob.  Returns dict(loss=[J, L_clip, L_vf, L_ent], grad (float64, blob
+    shaped), logp [num_envs])."""
+    B = int(batch["num_graphs"])
+    weights = np.ascontiguousarray(weights, dtype=np.float32)
+    shape = np.ascontiguousarray(batch["shape"], dtype=np.float32)
+    op = np.ascontiguousarray(batch["op"], dtype=np.int32)
+    env_off = np.ascontiguousarray(batch["env_off"], dtype=np.int32)
+    Ne = len(env_off) - 1
+    A = int(m["A_max"])
+    mask = np.ascontiguousarray(batch["mask"] if mask is None else mask, dtype=np.uint8)
+    if edge_attr is None:
+        edge_attr = batch.get("edge_attr")
+    ea = None if edge_attr is None else np.ascontiguousarray(edge_attr, dtype=np.float32)
+    g0a = None if g0 is None else np.ascontiguousarray(g0, dtype=np.float64)
+    action = np.ascontiguousarray(action, dtype=np.int32)
+    logp_old = np.ascontiguousarray(logp_old, dtype=np.float64)
+    adv = np.ascontiguousarray(adv, dtype=np.float64)
+    ret = np.ascontiguousarray(ret, dtype=np.float64)
+    loss = np.zeros(4)
+    grad = np.zeros(len(weights))
+    logp = np.zeros(Ne)
+    mm = _model(m)
+    st = lib().xo_ppo_grad(
+        C.byref(mm), _p(weights, _f32p), C.c_int32(B), _p(packed["node_off"], _i32p),
+        _p(packed["rowptr"], _i32p), _p(packed["col"], _i32p), _p(op, _i32p), _p(shape, _f32p),
+        _p(g0a, _f64p), _p(ea, _f32p), _p(packed["eid"] if ea is not None else None, _i32p),
+        C.c_int32(Ne), _p(env_off, _i32p), C.c_int32(A), _p(mask, _u8p), _p(action, _i32p),
+        _p(logp_old, _f64p), _p(adv, _f64p), _p(ret, _f64p), C.c_double(eps), C.c_double(c1),
+        C.c_double(c2), _p(loss, _f64p), _p(grad, _f64p), _p(logp, _f64p))
+    if st != 0:
+        raise ValueError(f"xo_ppo_grad status {st}")
+    return {"loss": loss, "grad": grad, "logp": logp}
+
+
+def gae(reward, values, done, gamma, lam):
+    """Generalised advantage estimates of one trajectory: values has len(reward) + 1 entries.  Returns
+    (advantages, value targets)."""
+    reward = np.ascontiguousarray(reward, dtype=np.float64)
+    values = np.ascontiguousarray(values, dtype=np.float64)
+    done = np.ascontiguousarray(done, dtype=np.uint8)
+    T = len(reward)
+    assert len(values) == T + 1 and len(done) == T
+    adv = np.zeros(T); ret = np.zeros(T)
+    st = lib().xo_gae(C.c_int32(T), _p(reward, _f64p), _p(values, _f64p), _p(done, _u8p),
+                      C.c_double(gamma), C.c_double(lam), _p(adv, _f64p), _p(ret, _f64p))
+    if st != 0:
+        raise ValueError(f"xo_gae status {st}")
+    return adv, ret

@@ -127,3 +127,66 @@ def test_planted_mistake_is_caught(xo, tmp_path, name, old, new):
         assert not _pins_hold(xo), f"mutation '{name}' went unnoticed"
     finally:
         xo._lib = saved
+
+
+# ---- the reverse pass of the PPO objective: planted mistakes must break the finite-difference pin ----------
+PPO_MUTATIONS = [
+    ("softmax reverse pass without the mean term", "al[t] * (dal[t] - dot) * (e > 0.0 ? 1.0 : 0.2)",
+     "al[t] * dal[t] * (e > 0.0 ? 1.0 : 0.2)"),
+    ("LeakyReLU slope ignored in the reverse pass", "al[t] * (dal[t] - dot) * (e > 0.0 ? 1.0 : 0.2)",
+     "al[t] * (dal[t] - dot)"),
+    ("a_dst collects the producer-side score gradients", "gw.a_dst[l][cc] += ds_dst[size_t(i) * K + k] * zs;",
+     "gw.a_dst[l][cc] += ds_src[size_t(i) * K + k] * zs;"),
+    ("value loss derivative without its factor 2", "c1 * 2.0 * (v - ret[e]) * inv_ne", "c1 * (v - ret[e]) * inv_ne"),
+    ("candidate mean not divided in the reverse pass", "+= du[H + c] / double(nv);", "+= du[H + c];"),
+    ("entropy gradient with the wrong sign inside", "(std::log(pr[a]) - plogp);", "(std::log(pr[a]) + plogp);"),
+    ("ReLU of Eq. 8 ignored in the reverse pass", "dpre[c] = tp.emb[c] > 0.0 ? demb[c] : 0.0;", "dpre[c] = demb[c];"),
+    ("gathered rows receive unweighted gradients", "dz[size_t(j) * H + k * d + c] += al[t] * dp[c];",
+     "dz[size_t(j) * H + k * d + c] += dp[c];"),
+    ("clipped term treated as if it had a slope", "(t1 <= t2) ? -adv[e] * ratio * inv_ne : 0.0;",
+     "-adv[e] * ratio * inv_ne;"),
+]
+
+
+def _ppo_pin_holds(xo):
+    import test_oracle_ppo as tp
+    m = dict(tp.M, Hm2=5)
+    b = tp._batch(3, m)
+    blob, _ = configs.make_weights(m, 41, readout_scale=0.3)
+    blob = blob.astype(np.float32)
+    st, packed = xo.pack(b)
+    if st != 0:
+        return False
+    ne = len(b["env_off"]) - 1
+    action = np.array([0, m["A_max"]], np.int32)
+    base = xo.forward(m, blob, b)
+    logp_now = np.log(base["probs"][np.arange(ne), action])
+    logp_old = logp_now - np.array([0.05, 0.5])      # second transition: ratio above 1 + eps, clipped (flat)
+    adv = np.array([0.7, 1.3]); ret = np.array([0.3, -0.8])
+    args = (action, logp_old, adv, ret, 0.2, 0.5, 0.05)
+    got = xo.ppo_grad(m, blob, b, packed, *args)
+    J = tp._objective(m, blob, b, *args, xo)
+    if not np.allclose(got["loss"], J, rtol=1e-11, atol=1e-12):
+        return False
+    delta = np.float32(2.0 ** -18)
+    scale = np.abs(got["grad"]).max()
+    for k in range(0, len(blob), 5):
+        wp = blob.copy(); wp[k] += delta
+        wm = blob.copy(); wm[k] -= delta
+        num = (tp._objective(m, wp, b, *args, xo)[0] - tp._objective(m, wm, b, *args, xo)[0]) / (float(wp[k]) - float(wm[k]))
+        if abs(got["grad"][k] - num) > 1e-5 * scale + 1e-4 * abs(num):
+            return False
+    return True
+
+
+@pytest.mark.parametrize("name,old,new", PPO_MUTATIONS, ids=[m[0] for m in PPO_MUTATIONS])
+def test_planted_mistake_in_the_reverse_pass_is_caught(xo, tmp_path, name, old, new):
+    assert _ppo_pin_holds(xo), "the unmodified oracle must pass"
+    mutant = _build(tmp_path, name, old, new)
+    mutant.xo_philox4x32_10.restype = None
+    saved = xo._lib
+    try:
+        xo._lib = mutant
+        assert not _ppo_pin_holds(xo), f"mutation '{name}' went unnoticed"
+    finally:
+        xo._lib = saved
