@@ -260,6 +260,10 @@ double mlp_scalar(const double* x, int in, int hid, int hid2, const float* W1, c
 // The gradient is taken by hand, layer by layer in reverse, with respect to every entry of the weight blob
 // (for a bf16 model: with respect to the stored, rounded values).  ReLU'(0) = 0, LeakyReLU'(0) = 0.2, and
 // the derivative of the clipped objective is that of whichever term of the min is the smaller one.
+// mode 1 ("mirrored", a debugging aid like xo_encode's): the forward pass keeps Z and every layer's output
+// rounded to bf16, as a bf16 model stores them, and the reverse pass runs at those values with the rounding
+// treated as the identity; mode 2 is mode 1 with the half-scores taken from the rounded Z instead of the
+// exact one (the two places an implementation may take them from).  mode 0 is the definition.
 
 // Forward intermediates of one graph that the reverse pass needs.
 struct GraphTape {
@@ -275,9 +279,10 @@ struct GraphTape {
 
 void forward_tape(const Model& m, const Weights& w, int32_t lo, int32_t hi, const int32_t* rowptr,
                   const int32_t* col, const int32_t* op, const float* shape, const double* g_attr,
-                  const float* edge_attr, const int32_t* eid, GraphTape& tp) {
+                  const float* edge_attr, const int32_t* eid, int mode, GraphTape& tp) {
   const int S = m.S, T = m.T, H = m.H, K = m.K, d = m.H / m.K, F0 = 2 * S + T;
   const int n = hi - lo;
+  const bool mirror = (mode != 0 && m.dtype == 1);   // keep Z and the layer outputs as a bf16 model stores them
   tp.n = n;
   tp.nbl.assign(n, {});
   for (int i = 0; i < n; ++i)
@@ -305,7 +310,7 @@ void forward_tape(const Model& m, const Weights& w, int32_t lo, int32_t hi, cons
     for (int c = 0; c < H; ++c) {
       double acc = double(w.b0[c]);
       for (int s = 0; s < F0; ++s) acc += x[s] * stored(m, w.W0[size_t(s) * H + c]);
-      tp.h[0][size_t(i) * H + c] = relu(acc);
+      tp.h[0][size_t(i) * H + c] = mirror ? round_bf16(relu(acc)) : relu(acc);
     }
   }
   // Eq. 7
@@ -316,7 +321,7 @@ void forward_tape(const Model& m, const Weights& w, int32_t lo, int32_t hi, cons
       for (int c = 0; c < H; ++c) {
         double acc = 0.0;
         for (int k = 0; k < H; ++k) acc += hin[size_t(i) * H + k] * stored(m, w.W[l][size_t(k) * H + c]);
-        z[size_t(i) * H + c] = acc;
+        z[size_t(i) * H + c] = (mirror && mode == 2) ? round_bf16(acc) : acc;
       }
     for (int i = 0; i < n; ++i)
       for (int k = 0; k < K; ++k) {
@@ -328,6 +333,8 @@ void forward_tape(const Model& m, const Weights& w, int32_t lo, int32_t hi, cons
         tp.s_src[l][size_t(i) * K + k] = ss;
         tp.s_dst[l][size_t(i) * K + k] = sd;
       }
+    if (mirror)
+      for (auto& v : z) v = round_bf16(v);
     for (int i = 0; i < n; ++i) {
       const int deg = int(tp.nbl[i].size());
       for (int k = 0; k < K; ++k) {
@@ -344,7 +351,8 @@ void forward_tape(const Model& m, const Weights& w, int32_t lo, int32_t hi, cons
         for (int c = k * d; c < (k + 1) * d; ++c) {
           double acc = 0.0;
           for (int t = 0; t <= deg; ++t) acc += al[t] * z[size_t((t < deg) ? tp.nbl[i][t] : i) * H + c];
-          tp.h[l + 1][size_t(i) * H + c] = relu(acc + double(w.b[l][c]));
+          const double out = relu(acc + double(w.b[l][c]));
+          tp.h[l + 1][size_t(i) * H + c] = mirror ? round_bf16(out) : out;
         }
       }
     }
@@ -702,7 +710,7 @@ int xo_ppo_grad(const Model* m, const float* weights, int32_t B, const int32_t* 
                 const double* g0, const float* edge_attr, const int32_t* eid, int32_t num_envs,
                 const int32_t* env_off, int32_t A_max, const uint8_t* mask, const int32_t* action,
                 const double* logp_old, const double* adv, const double* ret, double eps, double c1,
-                double c2, double* loss_out, double* grad, double* logp_out) {
+                double c2, double* loss_out, double* grad, double* logp_out, int32_t mode) {
   if (m->H % m->K != 0 || m->L < 0 || num_envs <= 0 || m->H / m->K > 512) return XO_INVALID_ARG;
   if (edge_attr && !eid) return XO_INVALID_ARG;
   const Weights w = slice(*m, weights);
@@ -731,7 +739,7 @@ int xo_ppo_grad(const Model* m, const float* weights, int32_t B, const int32_t* 
   std::vector<GraphTape> tapes(B);
   for (int g = 0; g < B; ++g)
     forward_tape(*m, w, node_off[g], node_off[g + 1], rowptr, col, op, shape,
-                 g0 ? g0 + size_t(g) * m->Dg : nullptr, edge_attr, eid, tapes[g]);
+                 g0 ? g0 + size_t(g) * m->Dg : nullptr, edge_attr, eid, mode, tapes[g]);
   std::vector<double> demb(size_t(B) * H, 0.0);
   double Lclip = 0.0, Lvf = 0.0, Lent = 0.0;
   const double inv_ne = 1.0 / double(num_envs);

@@ -145,10 +145,11 @@ def forward(m, weights, batch, g0=None, threads=0, mode=0):
 
 
 def ppo_grad(m, weights, batch, packed, action, logp_old, adv, ret, eps=0.2, c1=0.5, c2=0.01, g0=None,
-             mask=None, edge_attr=None):
+             mask=None, edge_attr=None, mirrored=False):
     """Section 3.3.4, Eq. 3-5 over the environments of the batch (each a stored transition) and the gradient
     of J with respect to the weight blob.  Returns dict(loss=[J, L_clip, L_vf, L_ent], grad (float64, blob
-    shaped), logp [num_envs])."""
+    shaped), logp [num_envs]).  mirrored: keep Z and the layer outputs as a bf16 model stores them (debugging
+    aid; the definition is mirrored=False); mirrored=2 also takes the half-scores from the rounded Z."""
     B = int(batch["num_graphs"])
     weights = np.ascontiguousarray(weights, dtype=np.float32)
     shape = np.ascontiguousarray(batch["shape"], dtype=np.float32)
@@ -175,7 +176,7 @@ def ppo_grad(m, weights, batch, packed, action, logp_old, adv, ret, eps=0.2, c1=
         _p(g0a, _f64p), _p(ea, _f32p), _p(packed["eid"] if ea is not None else None, _i32p),
         C.c_int32(Ne), _p(env_off, _i32p), C.c_int32(A), _p(mask, _u8p), _p(action, _i32p),
         _p(logp_old, _f64p), _p(adv, _f64p), _p(ret, _f64p), C.c_double(eps), C.c_double(c1),
-        C.c_double(c2), _p(loss, _f64p), _p(grad, _f64p), _p(logp, _f64p))
+        C.c_double(c2), _p(loss, _f64p), _p(grad, _f64p), _p(logp, _f64p), C.c_int32(int(mirrored)))
     if st != 0:
         raise ValueError(f"xo_ppo_grad status {st}")
     return {"loss": loss, "grad": grad, "logp": logp}

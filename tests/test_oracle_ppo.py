@@ -143,3 +143,25 @@ def test_gae_closed_forms(xo):
     d = r + 0.95 * v[1:] - v[:-1]
     want = [sum((0.95 * 0.8) ** k * d[t + k] for k in range(T - t)) for t in range(T)]
     np.testing.assert_allclose(adv, want, rtol=1e-13)
+
+
+def test_mirrored_mode_is_the_definition_for_fp32_and_close_to_it_for_bf16(xo):
+    """The debugging mode that keeps Z and the layer outputs as a bf16 model stores them changes nothing for
+    an fp32 model and moves a bf16 model's loss and gradient by rounding noise only."""
+    for dtype in ("fp32", "bf16"):
+        m = dict(M, dtype=dtype, H=16, K=2)
+        b = _batch(7, m)
+        blob, _ = configs.make_weights(m, 3, readout_scale=0.3)
+        blob = blob.astype(np.float32)
+        st, packed = xo.pack(b)
+        assert st == 0
+        action = np.array([0, m["A_max"]], np.int32)
+        args = (m, blob, b, packed, action, np.array([-1.0, -0.7]), np.array([0.7, -1.3]), np.array([0.2, -0.4]))
+        exact = xo.ppo_grad(*args)
+        mir = xo.ppo_grad(*args, mirrored=True)
+        if dtype == "fp32":
+            assert np.array_equal(exact["grad"], mir["grad"]) and np.array_equal(exact["loss"], mir["loss"])
+        else:
+            assert not np.array_equal(exact["grad"], mir["grad"])
+            np.testing.assert_allclose(mir["loss"], exact["loss"], rtol=2e-2, atol=1e-3)
+            assert np.linalg.norm(mir["grad"] - exact["grad"]) <= 5e-2 * np.linalg.norm(exact["grad"])
