@@ -246,6 +246,38 @@ xrl_status xrl_policy_value(xrl_ctx* ctx, const xrl_batch* batch, const float* g
 xrl_status xrl_sample(xrl_ctx* ctx, const float* probs, int32_t num_envs, int32_t num_actions,
                       uint64_t seed, uint64_t step, int32_t* action, void* stream);
 
+/* ---- (4) the training step's gradient: Section 3.3.4 -------------------------------------------- */
+
+/* The PPO objective over the environments of a packed batch, each a stored transition (its observation =
+ * the environment's graphs, the action taken, the behaviour policy's log-probability of it, its advantage
+ * estimate and its value target), and the gradient of that objective with respect to every weight:
+ *   ratio_e  = exp(log pi(action_e) - logp_old_e)
+ *   L_clip   = - mean_e min(ratio_e adv_e, clip(ratio_e, 1 - eps, 1 + eps) adv_e)         (Eq. 3)
+ *   L_vf     =   mean_e (value_e - ret_e)^2                                                (Eq. 4)
+ *   L_ent    =   mean_e sum_a p_a log p_a      (minus the policy's entropy)
+ *   J        =   L_clip + c1 L_vf + c2 L_ent                                               (Eq. 5)
+ * The forward pass is that of xrl_encode and xrl_policy_value with every layer's input kept; the reverse
+ * pass runs layer by layer in fp32 (ReLU'(0) = 0, LeakyReLU'(0) = 0.2; where the clipped term of Eq. 3 is
+ * the smaller one its slope is zero).  For a bf16 model the gradient of W0 and of the layer matrices is the
+ * one with respect to the stored (rounded) values.  Sums over rows use floating-point atomics: the last
+ * bits of a gradient may differ from run to run.
+ *   g0        DEVICE fp32 [B x Dg] or NULL            mask      DEVICE u8 [num_envs x A_max]
+ *   action    DEVICE int32 [num_envs]  in [0, A_max], A_max = No-Op; an action the mask excludes raises
+ *                                      XRL_ERR_INVALID_ARG in the device status word (results undefined)
+ *   logp_old, adv, ret   DEVICE fp32 [num_envs]
+ *   loss_out  DEVICE fp32 [4] = { J, L_clip, L_vf, L_ent }
+ *   grad      DEVICE fp32, laid out like the weight blob (xrl_weights_size bytes), overwritten
+ *   logp_out  DEVICE fp32 [num_envs] or NULL: log pi(action_e) under the current weights
+ * The first call allocates the workspace for the context's capacities ((L + 1) copies of the node features
+ * plus three fp32 ones) and therefore synchronises; later calls only enqueue.  Not recordable
+ * (XRL_ERR_STATE between xrl_graph_begin and xrl_graph_launch).  XRL_ERR_UNSUPPORTED when
+ * (2 S + T + 1) x H floats exceed one SM's shared memory (227 KB): W0's gradient is collected there.
+ * Errors: INVALID_ARG, STATE, UNSUPPORTED, ALLOC, CUDA. */
+xrl_status xrl_ppo_grad(xrl_ctx* ctx, const xrl_batch* batch, const float* g0, const uint8_t* mask,
+                        const int32_t* action, const float* logp_old, const float* adv, const float* ret,
+                        float eps, float c1, float c2, float* loss_out, float* grad, float* logp_out,
+                        void* stream);
+
 /* Read and clear the device status word.  Synchronises `stream`.  *status (HOST) receives the
  * first error code any kernel recorded since the last call, or XRL_OK. */
 xrl_status xrl_last_device_status(xrl_ctx* ctx, void* stream, int32_t* status);

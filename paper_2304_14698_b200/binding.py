@@ -25,7 +25,7 @@ EXPORTED_SYMBOLS = [
     "xrl_batch_free", "xrl_batch_info", "xrl_batch_export", "xrl_encode", "xrl_debug_node_features",
     "xrl_policy_value", "xrl_sample", "xrl_last_device_status", "xrl_launch_counts", "xrl_version",
     "xrl_profile", "xrl_profile_read", "xrl_pack_csr_static", "xrl_encode_delta", "xrl_delta_rows", "xrl_get_weights",
-    "xrl_graph_begin", "xrl_graph_launch", "xrl_batch_set_edge_attr",
+    "xrl_graph_begin", "xrl_graph_launch", "xrl_batch_set_edge_attr", "xrl_ppo_grad",
 ]
 PROFILE_FAMILIES = ["pack", "node_update", "transform", "aggregate", "readout", "heads", "aggregate_readout"]
 
@@ -88,6 +88,7 @@ def load_library():
         "xrl_profile_read": [vp, C.POINTER(C.c_double), C.POINTER(i64), i32],
         "xrl_batch_set_edge_attr": [vp, vp, i32, vp, vp],
         "xrl_graph_begin": [vp],
+        "xrl_ppo_grad": [vp] * 8 + [C.c_float] * 3 + [vp] * 4,
         "xrl_graph_launch": [vp, vp],
     }
     for name, args in sigs.items():
@@ -283,6 +284,17 @@ def xrl_sample(ctx, probs, action, seed, step, stream=None):
     _check(load_library().xrl_sample(ctx, _dev_ptr(probs), ne, a1, seed, step, _dev_ptr(action),
                                      _stream(stream)), "xrl_sample")
     return action
+
+
+def xrl_ppo_grad(ctx, batch, mask, action, logp_old, adv, ret, loss_out, grad, eps=0.2, c1=0.5, c2=0.01,
+                 g0=None, logp_out=None, stream=None):
+    """Section 3.3.4: loss_out[4] = {J, L_clip, L_vf, L_ent} and grad (blob-shaped fp32), all device tensors."""
+    st = load_library().xrl_ppo_grad(ctx, batch, _dev_ptr(g0), _dev_ptr(mask), _dev_ptr(action),
+                                     _dev_ptr(logp_old), _dev_ptr(adv), _dev_ptr(ret), C.c_float(eps),
+                                     C.c_float(c1), C.c_float(c2), _dev_ptr(loss_out), _dev_ptr(grad),
+                                     _dev_ptr(logp_out), _stream(stream))
+    _check(st, "xrl_ppo_grad")
+    return loss_out, grad
 
 
 def xrl_last_device_status(ctx, stream=None) -> int:

@@ -1,0 +1,738 @@
+// Reverse pass of the agent's forward path for the PPO objective of the paper's Section 3.3.4
+// (Eq. 3 clipped objective, Eq. 4 value loss, Eq. 5 their sum with an entropy term): the loss over the
+// environments of a mini-batch, then the gradient with respect to every weight, layer by layer backwards
+// through the heads, Eq. 8, the k attention layers of Eq. 7 and Eq. 6.
+//
+// These kernels are the plain, correct version: CUDA cores, fp32 gradients, sums over rows collected with
+// floating-point atomics (so the last bits of a gradient depend on the order in which the hardware serves
+// them).  Activations saved by the forward pass (the input of every layer) are read in their storage type;
+// Z and the half-scores of a layer are recomputed by the forward transform kernel before its reverse pass.
+// ReLU'(0) = 0, LeakyReLU'(0) = 0.2; the clipped objective has the slope of whichever term of its min is
+// the smaller one.
+#include <algorithm>
+
+#include "xrl_internal.cuh"
+
+namespace xrl {
+
+namespace {
+
+__device__ __forceinline__ float lrelu(float x) { return fmaxf(x, 0.2f * x); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+
+// Z rows and half-score pairs of a layer, in either layout (pairs behind the rows, or in their own array).
+template <typename T> struct ZView {
+  const char* z; size_t row_bytes; const float2* pairs; int pair_stride;   // pairs[i * pair_stride + k]
+  __device__ __forceinline__ const T* row(int32_t i) const { return reinterpret_cast<const T*>(z + size_t(i) * row_bytes); }
+  __device__ __forceinline__ float2 pair(int32_t i, int k) const { return pairs[size_t(i) * pair_stride + k]; }
+};
+
+constexpr int kMaxHeads = 64;
+constexpr int kMaxPerLane = 16;          // hidden <= 512
+
+// ---- Eq. 7, reverse: one warp per destination row ---------------------------------------------------
+// in : dh_out [N x H] fp32 (gradient of the layer's output), h_out (its output, for the ReLU), Z / pairs
+// out: dz [N x H] fp32 += alpha * dpre (scattered to the gathered rows, atomics), ds_src [N x K] += (atomics),
+//      ds_dst [N x K] = (own row), db [H] += (atomics, one per CTA and column)
+template <typename T>
+__global__ void __launch_bounds__(256)
+k_aggregate_bwd(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col, ZView<T> zv,
+                const T* __restrict__ h_out, const float* __restrict__ dh_out, float* __restrict__ dz,
+                float* __restrict__ ds_src, float* __restrict__ ds_dst, float* __restrict__ db, int N, int H,
+                int K) {
+  extern __shared__ float sm_db[];                 // [H] per-CTA sums of dpre
+  for (int c = threadIdx.x; c < H; c += blockDim.x) sm_db[c] = 0.f;
+  __syncthreads();
+  const int lane = threadIdx.x & 31;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  const int d = H / K, NF = H / 32;
+  for (int32_t i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < N; i += warps) {
+    float dp[kMaxPerLane];
+#pragma unroll
+    for (int f = 0; f < kMaxPerLane; ++f) {
+      dp[f] = 0.f;
+      if (f < NF) {
+        const int c = lane + 32 * f;
+        dp[f] = to_float(h_out[size_t(i) * H + c]) > 0.f ? dh_out[size_t(i) * H + c] : 0.f;
+        atomicAdd(&sm_db[c], dp[f]);
+      }
+    }
+    const int32_t e0 = rowptr[i], deg = rowptr[i + 1] - e0;
+    // softmax statistics per head (every lane keeps all K heads; K is small)
+    for (int k0 = 0; k0 < K; ++k0) {
+      const float sd = zv.pair(i, k0).y;
+      float mx = -INFINITY;
+      for (int t = lane; t <= deg; t += 32) {
+        const int32_t j = t < deg ? col[e0 + t] : i;
+        mx = fmaxf(mx, lrelu(zv.pair(j, k0).x + sd));
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+      float sum = 0.f;
+      for (int t = lane; t <= deg; t += 32) {
+        const int32_t j = t < deg ? col[e0 + t] : i;
+        sum += exp2f(lrelu(zv.pair(j, k0).x + sd) - mx);
+      }
+      sum = warp_sum(sum);
+      const float inv = 1.f / sum;
+      // dal_t = sum over the head's features of dpre * z_j; dot = sum_t alpha_t dal_t
+      float dot = 0.f;
+      for (int t = 0; t <= deg; ++t) {
+        const int32_t j = t < deg ? col[e0 + t] : i;
+        const T* zj = zv.row(j);
+        float part = 0.f;
+#pragma unroll
+        for (int f = 0; f < kMaxPerLane; ++f)
+          if (f < NF) {
+            const int c = lane + 32 * f;
+            if (c / d == k0) part += dp[f] * to_float(zj[c]);
+          }
+        const float dal = warp_sum(part);
+        const float al = exp2f(lrelu(zv.pair(j, k0).x + sd) - mx) * inv;
+        dot += al * dal;
+      }
+      float dsd = 0.f;
+      for (int t = 0; t <= deg; ++t) {
+        const int32_t j = t < deg ? col[e0 + t] : i;
+        const T* zj = zv.row(j);
+        float part = 0.f;
+#pragma unroll
+        for (int f = 0; f < kMaxPerLane; ++f)
+          if (f < NF) {
+            const int c = lane + 32 * f;
+            if (c / d == k0) part += dp[f] * to_float(zj[c]);
+          }
+        const float dal = warp_sum(part);
+        const float e = zv.pair(j, k0).x + sd;          // (times log2 e: the sign is what matters below)
+        const float al = exp2f(lrelu(e) - mx) * inv;
+        const float de = al * (dal - dot) * (e > 0.f ? 1.f : 0.2f);
+        dsd += de;
+        if (lane == 0) atomicAdd(&ds_src[size_t(j) * K + k0], de);
+#pragma unroll
+        for (int f = 0; f < kMaxPerLane; ++f)
+          if (f < NF) {
+            const int c = lane + 32 * f;
+            if (c / d == k0) atomicAdd(&dz[size_t(j) * H + c], al * dp[f]);
+          }
+      }
+      if (lane == 0) ds_dst[size_t(i) * K + k0] = dsd;
+    }
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < H; c += blockDim.x)
+    if (sm_db[c] != 0.f) atomicAdd(&db[c], sm_db[c]);
+}
+
+// ---- half-scores, reverse: dz += ds_src a_src + ds_dst a_dst; da_src += ds_src z; da_dst += ds_dst z -----
+template <typename T>
+__global__ void __launch_bounds__(256)
+k_scores_bwd(ZView<T> zv, const float* __restrict__ ds_src, const float* __restrict__ ds_dst,
+             const float* __restrict__ a_src, const float* __restrict__ a_dst, float* __restrict__ dz,
+             float* __restrict__ da_src, float* __restrict__ da_dst, int N, int H, int K) {
+  extern __shared__ float sm_da[];                 // [2H]
+  for (int c = threadIdx.x; c < 2 * H; c += blockDim.x) sm_da[c] = 0.f;
+  __syncthreads();
+  const int d = H / K;
+  const int rows_per_cta = (N + gridDim.x - 1) / gridDim.x;
+  const int r0 = blockIdx.x * rows_per_cta, r1 = min(N, r0 + rows_per_cta);
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    const int k = c / d;
+    const float as = a_src[c], ad = a_dst[c];
+    float accs = 0.f, accd = 0.f;
+    for (int i = r0; i < r1; ++i) {
+      const float gs = ds_src[size_t(i) * K + k], gd = ds_dst[size_t(i) * K + k];
+      const float z = to_float(zv.row(i)[c]);
+      dz[size_t(i) * H + c] += gs * as + gd * ad;
+      accs += gs * z;
+      accd += gd * z;
+    }
+    sm_da[c] = accs;
+    sm_da[H + c] = accd;
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    atomicAdd(&da_src[c], sm_da[c]);
+    atomicAdd(&da_dst[c], sm_da[H + c]);
+  }
+}
+
+// ---- dW += A^T B over a range of rows: A [rows x Ka] (storage type), B [rows x Nb] fp32 -------------------
+// 64 x 64 output tile per CTA, the rows cut into chunks along grid.z, partial products added with atomics.
+template <typename TA>
+__global__ void __launch_bounds__(256)
+k_atb(const TA* __restrict__ A, int lda, const float* __restrict__ Bm, int ldb, float* __restrict__ Cout, int ldc,
+      int rows, int Ka, int Nb, int rows_per_chunk) {
+  __shared__ float As[16][64 + 1];
+  __shared__ float Bs[16][64 + 1];
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  const int a0 = blockIdx.x * 64, b0 = blockIdx.y * 64;
+  const int r_begin = blockIdx.z * rows_per_chunk, r_end = min(rows, r_begin + rows_per_chunk);
+  float acc[4][4] = {};
+  for (int r0 = r_begin; r0 < r_end; r0 += 16) {
+    for (int t = tid; t < 16 * 64; t += 256) {
+      const int rr = t >> 6, cc = t & 63;
+      const int r = r0 + rr;
+      As[rr][cc] = (r < r_end && a0 + cc < Ka) ? to_float(A[size_t(r) * lda + a0 + cc]) : 0.f;
+      Bs[rr][cc] = (r < r_end && b0 + cc < Nb) ? Bm[size_t(r) * ldb + b0 + cc] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int rr = 0; rr < 16; ++rr) {
+      float a[4], b[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { a[u] = As[rr][ty * 4 + u]; b[u] = Bs[rr][tx * 4 + u]; }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) acc[u][v] = fmaf(a[u], b[v], acc[u][v]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int u = 0; u < 4; ++u)
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+      const int ka = a0 + ty * 4 + u, nb = b0 + tx * 4 + v;
+      if (ka < Ka && nb < Nb && acc[u][v] != 0.f) atomicAdd(&Cout[size_t(ka) * ldc + nb], acc[u][v]);
+    }
+}
+
+// ---- out = G W^T: G [rows x Hn] fp32, W [Hk x Hn] (storage type, row-major [in x out]) -> out [rows x Hk] ----
+template <typename TW>
+__global__ void __launch_bounds__(256)
+k_gwt(const float* __restrict__ G, const TW* __restrict__ W, float* __restrict__ out, int rows, int Hk, int Hn) {
+  __shared__ float Gs[64][16 + 1];
+  __shared__ float Ws[64][16 + 1];
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  const int r0 = blockIdx.x * 64, k0 = blockIdx.y * 64;
+  float acc[4][4] = {};
+  for (int c0 = 0; c0 < Hn; c0 += 16) {
+    for (int t = tid; t < 64 * 16; t += 256) {
+      const int rr = t >> 4, cc = t & 15;
+      Gs[rr][cc] = (r0 + rr < rows && c0 + cc < Hn) ? G[size_t(r0 + rr) * Hn + c0 + cc] : 0.f;
+      Ws[rr][cc] = (k0 + rr < Hk && c0 + cc < Hn) ? to_float(W[size_t(k0 + rr) * Hn + c0 + cc]) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int cc = 0; cc < 16; ++cc) {
+      float g[4], w[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { g[u] = Gs[ty * 4 + u][cc]; w[u] = Ws[tx * 4 + u][cc]; }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) acc[u][v] = fmaf(g[u], w[v], acc[u][v]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int u = 0; u < 4; ++u)
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+      const int r = r0 + ty * 4 + u, k = k0 + tx * 4 + v;
+      if (r < rows && k < Hk) out[size_t(r) * Hk + k] = acc[u][v];
+    }
+}
+
+// ---- Eq. 6, reverse: dW0 += x^T dpre, db0 += dpre, x_i = [edge sum | one-hot op | own shape] -------------
+// One warp per row builds x's 16 dense entries; a CTA adds its rows' outer products into a shared-memory
+// copy of W0's gradient ([2S + T] x H floats) and adds that to global memory once.
+template <typename T>
+__global__ void __launch_bounds__(256)
+k_embed_bwd(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col, const int32_t* __restrict__ op,
+            const T* __restrict__ shape, const T* __restrict__ eattr, const T* __restrict__ h0,
+            const float* __restrict__ dh0, float* __restrict__ dW0, float* __restrict__ db0, int N, int H, int Tn) {
+  extern __shared__ float acc[];                   // [(2S + T + 1) x H]: dW0 rows, then db0
+  const int F0 = 2 * kS + Tn;
+  for (int t = threadIdx.x; t < (F0 + 1) * H; t += blockDim.x) acc[t] = 0.f;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  const int rows_per_cta = (N + gridDim.x - 1) / gridDim.x;
+  const int r0 = blockIdx.x * rows_per_cta, r1 = min(N, r0 + rows_per_cta);
+  for (int i = r0 + warp; i < r1; i += nw) {
+    float x[2 * kS];
+#pragma unroll
+    for (int s = 0; s < 2 * kS; ++s) x[s] = 0.f;
+    for (int32_t e = rowptr[i]; e < rowptr[i + 1]; ++e) {
+      const T* src = eattr ? eattr + size_t(e) * kS : shape + size_t(col[e]) * kS;
+#pragma unroll
+      for (int s = 0; s < kS; ++s) x[s] += to_float(src[s]);
+    }
+#pragma unroll
+    for (int s = 0; s < kS; ++s) x[kS + s] = to_float(shape[size_t(i) * kS + s]);
+    const int o = op[i];
+    for (int c = lane; c < H; c += 32) {
+      const float dp = to_float(h0[size_t(i) * H + c]) > 0.f ? dh0[size_t(i) * H + c] : 0.f;
+      if (dp == 0.f) continue;
+#pragma unroll
+      for (int s = 0; s < kS; ++s) {
+        atomicAdd(&acc[size_t(s) * H + c], x[s] * dp);
+        atomicAdd(&acc[size_t(kS + Tn + s) * H + c], x[kS + s] * dp);
+      }
+      atomicAdd(&acc[size_t(kS + o) * H + c], dp);
+      atomicAdd(&acc[size_t(F0) * H + c], dp);
+    }
+  }
+  __syncthreads();
+  for (int t = threadIdx.x; t < F0 * H; t += blockDim.x)
+    if (acc[t] != 0.f) atomicAdd(&dW0[t], acc[t]);
+  for (int c = threadIdx.x; c < H; c += blockDim.x)
+    if (acc[size_t(F0) * H + c] != 0.f) atomicAdd(&db0[c], acc[size_t(F0) * H + c]);
+}
+
+// ---- the heads' MLPs: Linear(in, hid), ReLU, [Linear(hid, hid2), ReLU,] Linear(last, 1) ---------------------
+// One CTA per input row.  The forward keeps the hidden activations; the reverse pass turns d(out) into the
+// gradients of the hidden pre-activations (d1, d2) and of the input (dx).  The weights' gradients are
+// products of those per-row buffers (X^T D1, Y1^T D2, ...), taken afterwards by k_atb / k_colsum.
+struct MlpW { const float *W1, *b1, *Wh, *bh, *w2, *b2; int hid, hid2; };
+
+__device__ float block_sum_f(float v, float* scratch) {       // blockDim a power of two
+  scratch[threadIdx.x] = v;
+  __syncthreads();
+  for (int s = blockDim.x >> 1; s > 0; s >>= 1) {
+    if (int(threadIdx.x) < s) scratch[threadIdx.x] += scratch[threadIdx.x + s];
+    __syncthreads();
+  }
+  const float r = scratch[0];
+  __syncthreads();
+  return r;
+}
+
+// x [in], y1 [hid], y2 [hid2] in shared memory; returns the head's output to every thread
+__device__ float mlp_fwd(const float* x, int in, const MlpW& m, float* y1, float* y2, float* scratch) {
+  for (int c = threadIdx.x; c < m.hid; c += blockDim.x) {
+    float acc = m.b1[c];
+    for (int k = 0; k < in; ++k) acc = fmaf(x[k], m.W1[size_t(k) * m.hid + c], acc);
+    y1[c] = fmaxf(acc, 0.f);
+  }
+  __syncthreads();
+  float contrib = 0.f;
+  if (m.hid2 <= 0) {
+    for (int c = threadIdx.x; c < m.hid; c += blockDim.x) contrib += y1[c] * m.w2[c];
+  } else {
+    for (int c = threadIdx.x; c < m.hid2; c += blockDim.x) {
+      float acc = m.bh[c];
+      for (int k = 0; k < m.hid; ++k) acc = fmaf(y1[k], m.Wh[size_t(k) * m.hid2 + c], acc);
+      y2[c] = fmaxf(acc, 0.f);
+      contrib += y2[c] * m.w2[c];
+    }
+  }
+  return block_sum_f(contrib, scratch) + m.b2[0];
+}
+
+// y1, y2, d1, d2, dx in shared memory (dx [in], may be null)
+__device__ void mlp_bwd(int in, const MlpW& m, const float* y1, const float* y2, float dout, float* d1, float* d2,
+                        float* dx) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  if (m.hid2 <= 0) {
+    for (int c = threadIdx.x; c < m.hid; c += blockDim.x) d1[c] = y1[c] > 0.f ? m.w2[c] * dout : 0.f;
+  } else {
+    for (int c = threadIdx.x; c < m.hid2; c += blockDim.x) d2[c] = y2[c] > 0.f ? m.w2[c] * dout : 0.f;
+    __syncthreads();
+    for (int k = warp; k < m.hid; k += nw) {
+      float part = 0.f;
+      for (int c = lane; c < m.hid2; c += 32) part = fmaf(m.Wh[size_t(k) * m.hid2 + c], d2[c], part);
+      part = warp_sum(part);
+      if (lane == 0) d1[k] = y1[k] > 0.f ? part : 0.f;
+    }
+  }
+  __syncthreads();
+  if (dx != nullptr) {
+    for (int k = warp; k < in; k += nw) {
+      float part = 0.f;
+      for (int c = lane; c < m.hid; c += 32) part = fmaf(m.W1[size_t(k) * m.hid + c], d1[c], part);
+      part = warp_sum(part);
+      if (lane == 0) dx[k] = part;
+    }
+  }
+  __syncthreads();
+}
+
+// per-graph sums of the last layer's node features, written as the first H entries of row g of U [B x (H + Dg)];
+// the graph's global attributes fill the rest
+template <typename T>
+__global__ void __launch_bounds__(256)
+k_graph_sum(const T* __restrict__ h, const int32_t* __restrict__ node_off, const float* __restrict__ g0,
+            float* __restrict__ U, int H, int Dg) {
+  const int g = blockIdx.x;
+  const int32_t lo = node_off[g], hi = node_off[g + 1];
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    float s = 0.f;
+    for (int32_t i = lo; i < hi; ++i) s += to_float(h[size_t(i) * H + c]);
+    U[size_t(g) * (H + Dg) + c] = s;
+  }
+  for (int t = threadIdx.x; t < Dg; t += blockDim.x) U[size_t(g) * (H + Dg) + H + t] = g0 ? g0[size_t(g) * Dg + t] : 0.f;
+}
+
+// ---- per graph, forward: Eq. 8 and the policy head ---------------------------------------------------------
+__global__ void __launch_bounds__(256)
+k_graph_fwd(const float* __restrict__ U, const float* __restrict__ Wg, const float* __restrict__ bg, MlpW pm,
+            float* __restrict__ emb, float* __restrict__ py1, float* __restrict__ py2, float* __restrict__ logit,
+            int H, int Dg) {
+  extern __shared__ float sm[];
+  float* scratch = sm;                              // [blockDim]
+  float* uu = scratch + blockDim.x;                 // [H + Dg]
+  float* x = uu + H + Dg;                           // [H]
+  float* y1 = x + H;                                // [hid]
+  float* y2 = y1 + pm.hid;                          // [hid2]
+  const int g = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
+  for (int k = tid; k < H + Dg; k += nt) uu[k] = U[size_t(g) * (H + Dg) + k];
+  __syncthreads();
+  for (int c = tid; c < H; c += nt) {
+    float acc = bg[c];
+    for (int k = 0; k < H + Dg; ++k) acc = fmaf(uu[k], Wg[size_t(k) * H + c], acc);
+    x[c] = fmaxf(acc, 0.f);
+    emb[size_t(g) * H + c] = x[c];
+  }
+  __syncthreads();
+  const float out = mlp_fwd(x, H, pm, y1, y2, scratch);
+  for (int c = tid; c < pm.hid; c += nt) py1[size_t(g) * pm.hid + c] = y1[c];
+  for (int c = tid; c < pm.hid2; c += nt) py2[size_t(g) * pm.hid2 + c] = y2[c];
+  if (tid == 0) logit[g] = out;
+}
+
+// ---- per environment: Eq. 3-5, d J / d logit of its graphs, value head forward and reverse -----------------
+// loss[4] += {J, L_clip, L_vf, L_ent} (atomics); dlogit [B]; demb [B x H] = the value head's share (plain
+// stores: a graph belongs to one environment); the value head's per-row buffers vu [2H], vy1, vy2, vd1, vd2,
+// vdout; logp_out [num_envs].
+struct EnvBufs { float *vu, *vy1, *vy2, *vd1, *vd2, *vdout; };
+
+__global__ void __launch_bounds__(256)
+k_ppo_env(const float* __restrict__ emb, const float* __restrict__ logit, const int32_t* __restrict__ env_off,
+          const uint8_t* __restrict__ mask, const int32_t* __restrict__ action, const float* __restrict__ logp_old,
+          const float* __restrict__ adv, const float* __restrict__ ret, float eps, float c1, float c2, MlpW vm,
+          EnvBufs eb, int H, int A, int num_envs, float* __restrict__ loss, float* __restrict__ dlogit,
+          float* __restrict__ demb, float* __restrict__ logp_out, int32_t* status) {
+  extern __shared__ float sm[];
+  float* scratch = sm;                              // [blockDim]
+  float* u = scratch + blockDim.x;                  // [2H]
+  float* du = u + 2 * H;                            // [2H]
+  float* y1 = du + 2 * H;                           // [hid]
+  float* y2 = y1 + vm.hid;                          // [hid2]
+  float* d1 = y2 + vm.hid2;                         // [hid]
+  float* d2 = d1 + vm.hid;                          // [hid2]
+  const int e = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
+  const int32_t cur = env_off[e];
+  const int32_t C = env_off[e + 1] - cur - 1;
+  const uint8_t* mk = mask + size_t(e) * A;
+  const float inv_ne = 1.f / float(num_envs);
+  auto valid = [&](int a) { return a == A || (a < C && mk[a]); };
+  auto lg = [&](int a) { return logit[a == A ? cur : cur + 1 + a]; };
+  // masked softmax statistics
+  float mx = -INFINITY;
+  for (int a = tid; a <= A; a += nt)
+    if (valid(a)) mx = fmaxf(mx, lg(a));
+  scratch[tid] = mx;
+  __syncthreads();
+  for (int s = nt >> 1; s > 0; s >>= 1) {
+    if (tid < s) scratch[tid] = fmaxf(scratch[tid], scratch[tid + s]);
+    __syncthreads();
+  }
+  mx = scratch[0];
+  __syncthreads();
+  float se = 0.f;
+  for (int a = tid; a <= A; a += nt)
+    if (valid(a)) se += expf(lg(a) - mx);
+  const float sum = block_sum_f(se, scratch);
+  const float lsum = logf(sum);
+  float pl = 0.f;                                   // sum_a p_a log p_a
+  for (int a = tid; a <= A; a += nt)
+    if (valid(a)) { const float lp = lg(a) - mx - lsum; pl += expf(lp) * lp; }
+  const float plogp = block_sum_f(pl, scratch);
+  const int act = action[e];
+  if (act < 0 || act > A || !valid(act)) {          // the same for every thread of the CTA
+    if (tid == 0) raise(status, XRL_ERR_INVALID_ARG);
+    return;
+  }
+  const float logp = lg(act) - mx - lsum;
+  const float ratio = expf(logp - logp_old[e]);
+  const float clipped = fminf(fmaxf(ratio, 1.f - eps), 1.f + eps);
+  const float t1 = ratio * adv[e], t2 = clipped * adv[e];
+  const float dlogp = (t1 <= t2) ? -adv[e] * ratio * inv_ne : 0.f;
+  for (int a = tid; a <= A; a += nt) {
+    if (a < A && a >= C) continue;                  // no graph behind a padded slot
+    const int32_t g = a == A ? cur : cur + 1 + a;
+    float dl = 0.f;
+    if (valid(a)) {
+      const float lp = lg(a) - mx - lsum, p = expf(lp);
+      dl = dlogp * ((a == act ? 1.f : 0.f) - p) + c2 * inv_ne * p * (lp - plogp);
+    }
+    dlogit[g] = dl;
+  }
+  // value head over [ current graph | mean of the valid candidates ]
+  for (int c = tid; c < H; c += nt) u[c] = emb[size_t(cur) * H + c];
+  float cnt = 0.f;
+  for (int a = tid; a < C; a += nt) cnt += mk[a] ? 1.f : 0.f;
+  const float nv = block_sum_f(cnt, scratch);
+  for (int c = tid; c < H; c += nt) {
+    float s = 0.f;
+    for (int a = 0; a < C; ++a)
+      if (mk[a]) s += emb[size_t(cur + 1 + a) * H + c];
+    u[H + c] = nv > 0.f ? s / nv : 0.f;
+  }
+  __syncthreads();
+  const float v = mlp_fwd(u, 2 * H, vm, y1, y2, scratch);
+  const float dv = c1 * 2.f * (v - ret[e]) * inv_ne;
+  mlp_bwd(2 * H, vm, y1, y2, dv, d1, d2, du);
+  for (int c = tid; c < 2 * H; c += nt) eb.vu[size_t(e) * 2 * H + c] = u[c];
+  for (int c = tid; c < vm.hid; c += nt) {
+    eb.vy1[size_t(e) * vm.hid + c] = y1[c];
+    eb.vd1[size_t(e) * vm.hid + c] = d1[c];
+  }
+  for (int c = tid; c < vm.hid2; c += nt) {
+    eb.vy2[size_t(e) * vm.hid2 + c] = y2[c];
+    eb.vd2[size_t(e) * vm.hid2 + c] = d2[c];
+  }
+  for (int c = tid; c < H; c += nt) {
+    demb[size_t(cur) * H + c] = du[c];
+    const float share = nv > 0.f ? du[H + c] / nv : 0.f;
+    for (int a = 0; a < C; ++a) demb[size_t(cur + 1 + a) * H + c] = mk[a] ? share : 0.f;
+  }
+  if (tid == 0) {
+    eb.vdout[e] = dv;
+    const float lc = -(t1 <= t2 ? t1 : t2) * inv_ne, lv = (v - ret[e]) * (v - ret[e]) * inv_ne, le = plogp * inv_ne;
+    atomicAdd(&loss[1], lc); atomicAdd(&loss[2], lv); atomicAdd(&loss[3], le);
+    atomicAdd(&loss[0], lc + c1 * lv + c2 * le);
+    if (logp_out) logp_out[e] = logp;
+  }
+}
+
+// ---- per graph, reverse: policy head, then Eq. 8 -------------------------------------------------------------
+// in : demb (the value head's share), dlogit, emb, py1, py2   out: pd1, pd2, dpre [B x H] (gradient of Eq. 8's
+// pre-activation), dr [B x H] (gradient of the graph's readout sum)
+__global__ void __launch_bounds__(256)
+k_graph_bwd(const float* __restrict__ emb, const float* __restrict__ dlogit, MlpW pm,
+            const float* __restrict__ py1, const float* __restrict__ py2, const float* __restrict__ demb,
+            const float* __restrict__ Wg, float* __restrict__ pd1, float* __restrict__ pd2,
+            float* __restrict__ dpre, float* __restrict__ dr, int H) {
+  extern __shared__ float sm[];
+  float* dx = sm;                                   // [H]
+  float* y1 = dx + H;
+  float* y2 = y1 + pm.hid;
+  float* d1 = y2 + pm.hid2;
+  float* d2 = d1 + pm.hid;
+  const int g = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
+  const int lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
+  for (int c = tid; c < pm.hid; c += nt) y1[c] = py1[size_t(g) * pm.hid + c];
+  for (int c = tid; c < pm.hid2; c += nt) y2[c] = py2[size_t(g) * pm.hid2 + c];
+  __syncthreads();
+  mlp_bwd(H, pm, y1, y2, dlogit[g], d1, d2, dx);
+  for (int c = tid; c < pm.hid; c += nt) pd1[size_t(g) * pm.hid + c] = d1[c];
+  for (int c = tid; c < pm.hid2; c += nt) pd2[size_t(g) * pm.hid2 + c] = d2[c];
+  for (int c = tid; c < H; c += nt) {
+    const float de = demb[size_t(g) * H + c] + dx[c];
+    const float dp = emb[size_t(g) * H + c] > 0.f ? de : 0.f;
+    dx[c] = dp;
+    dpre[size_t(g) * H + c] = dp;
+  }
+  __syncthreads();
+  for (int k = warp; k < H; k += nw) {
+    float part = 0.f;
+    for (int c = lane; c < H; c += 32) part = fmaf(Wg[size_t(k) * H + c], dx[c], part);
+    part = warp_sum(part);
+    if (lane == 0) dr[size_t(g) * H + k] = part;
+  }
+}
+
+// the readout is a plain sum: every node receives its graph's gradient
+__global__ void k_readout_bwd(const float* __restrict__ dr, const int32_t* __restrict__ seg_id,
+                              float* __restrict__ dh, int64_t n_elems, int H) {
+  for (int64_t t = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; t < n_elems; t += int64_t(gridDim.x) * blockDim.x) {
+    const int64_t i = t / H;
+    dh[t] = dr[size_t(seg_id[i]) * H + (t - i * H)];
+  }
+}
+
+// rows per chunk such that the chunks of `rows` fit the grid's y / z extent
+int chunk_rows(int64_t rows, int at_least) {
+  const int64_t need = ((rows + 16383) / 16384 + 15) & ~int64_t(15);
+  return int(std::max<int64_t>(at_least, need));
+}
+
+// out[c] += sum over rows of M[r][c]
+__global__ void __launch_bounds__(256)
+k_colsum(const float* __restrict__ M, int ld, float* __restrict__ out, int rows, int cols, int rows_per_chunk) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= cols) return;
+  const int r0 = blockIdx.y * rows_per_chunk, r1 = min(rows, r0 + rows_per_chunk);
+  float s = 0.f;
+  for (int r = r0; r < r1; ++r) s += M[size_t(r) * ld + c];
+  if (s != 0.f) atomicAdd(&out[c], s);
+}
+
+void atb_f32(const float* A, int lda, const float* Bm, int ldb, float* Cout, int ldc, int rows, int Ka, int Nb,
+             cudaStream_t st) {
+  if (rows <= 0 || Ka <= 0 || Nb <= 0) return;
+  const int chunk = chunk_rows(rows, 1024);
+  dim3 g(unsigned((Ka + 63) / 64), unsigned((Nb + 63) / 64), unsigned((rows + chunk - 1) / chunk));
+  k_atb<float><<<g, 256, 0, st>>>(A, lda, Bm, ldb, Cout, ldc, rows, Ka, Nb, chunk);
+}
+void colsum(const float* M, int ld, float* out, int rows, int cols, cudaStream_t st) {
+  if (rows <= 0 || cols <= 0) return;
+  const int chunk = chunk_rows(rows, 512);
+  dim3 g(unsigned((cols + 255) / 256), unsigned((rows + chunk - 1) / chunk));
+  k_colsum<<<g, 256, 0, st>>>(M, ld, out, rows, cols, chunk);
+}
+
+// weights' gradients of one head from its per-row buffers; returns the launches
+int mlp_weight_grads(const float* X, int in, int rows, int hid, int hid2, const float* Y1, const float* Y2,
+                     const float* D1, const float* D2, const float* dout, float* gW1, float* gb1, float* gWh,
+                     float* gbh, float* gw2, float* gb2, cudaStream_t st) {
+  int n = 0;
+  atb_f32(X, in, D1, hid, gW1, hid, rows, in, hid, st); ++n;
+  colsum(D1, hid, gb1, rows, hid, st); ++n;
+  if (hid2 > 0) {
+    atb_f32(Y1, hid, D2, hid2, gWh, hid2, rows, hid, hid2, st); ++n;
+    colsum(D2, hid2, gbh, rows, hid2, st); ++n;
+    atb_f32(Y2, hid2, dout, 1, gw2, 1, rows, hid2, 1, st); ++n;
+  } else {
+    atb_f32(Y1, hid, dout, 1, gw2, 1, rows, hid, 1, st); ++n;
+  }
+  colsum(dout, 1, gb2, rows, 1, st); ++n;
+  return n;
+}
+
+}  // namespace
+
+// ---- launchers ------------------------------------------------------------------------------------------
+size_t ppo_heads_workspace_floats(const Dims& d, int64_t B, int64_t num_envs) {
+  const size_t H = d.H, Hm = d.Hm, Hm2 = d.Hm2;
+  return size_t(B) * ((H + d.Dg) + 4 * H + 2 + 2 * Hm + 2 * Hm2) + size_t(num_envs) * (2 * H + 2 * Hm + 2 * Hm2 + 1);
+}
+
+// Forward from the saved last-layer features to the logits, Eq. 3-5, and the reverse pass down to the gradient
+// of the last layer's node features (dh [N x H]).  ws: ppo_heads_workspace_floats floats.
+int launch_ppo_heads(const Dims& d, const DevWeights& w, float* grad_base, const float* w_base, const void* hL,
+                     const int32_t* node_off, const int32_t* seg_id, const float* g0, const int32_t* env_off,
+                     const uint8_t* mask, const int32_t* action, const float* logp_old, const float* adv,
+                     const float* ret, float eps, float c1, float c2, int32_t B, int32_t num_envs, int64_t N,
+                     float* ws, float* loss, float* dh, float* logp_out, int32_t* status, cudaStream_t st) {
+  if (B <= 0 || num_envs <= 0) return 0;
+  const size_t H = d.H, Hm = d.Hm, Hm2 = d.Hm2, HU = H + d.Dg;
+  float* p = ws;
+  auto take = [&](size_t n) { float* q = p; p += n; return q; };
+  float* U = take(size_t(B) * HU);
+  float* emb = take(size_t(B) * H);
+  float* demb = take(size_t(B) * H);
+  float* dpre = take(size_t(B) * H);
+  float* dr = take(size_t(B) * H);
+  float* logit = take(B);
+  float* dlogit = take(B);
+  float* py1 = take(size_t(B) * Hm);
+  float* pd1 = take(size_t(B) * Hm);
+  float* py2 = take(size_t(B) * Hm2);
+  float* pd2 = take(size_t(B) * Hm2);
+  EnvBufs eb;
+  eb.vu = take(size_t(num_envs) * 2 * H);
+  eb.vy1 = take(size_t(num_envs) * Hm); eb.vd1 = take(size_t(num_envs) * Hm);
+  eb.vy2 = take(size_t(num_envs) * Hm2); eb.vd2 = take(size_t(num_envs) * Hm2);
+  eb.vdout = take(num_envs);
+  auto gp = [&](const float* q) { return grad_base + (q - w_base); };     // same place in the gradient blob
+  const MlpW vm{w.vW1, w.vb1, w.vWh, w.vbh, w.vw2, w.vb2, d.Hm, d.Hm2};
+  const MlpW pm{w.pW1, w.pb1, w.pWh, w.pbh, w.pw2, w.pb2, d.Hm, d.Hm2};
+  int n = 0;
+  // a bad action leaves its environment's rows unwritten: start them from zero
+  cudaMemsetAsync(demb, 0, sizeof(float) * size_t(B) * H, st);
+  cudaMemsetAsync(dlogit, 0, sizeof(float) * size_t(B), st);
+  cudaMemsetAsync(eb.vu, 0, sizeof(float) * size_t(p - eb.vu), st);
+  if (d.dtype == XRL_BF16)
+    k_graph_sum<bf16><<<B, 256, 0, st>>>(static_cast<const bf16*>(hL), node_off, g0, U, d.H, d.Dg);
+  else
+    k_graph_sum<float><<<B, 256, 0, st>>>(static_cast<const float*>(hL), node_off, g0, U, d.H, d.Dg);
+  ++n;
+  k_graph_fwd<<<B, 256, sizeof(float) * (256 + HU + H + Hm + Hm2), st>>>(U, w.Wg, w.bg, pm, emb, py1, py2, logit,
+                                                                          d.H, d.Dg);
+  ++n;
+  k_ppo_env<<<num_envs, 256, sizeof(float) * (256 + 4 * H + 2 * Hm + 2 * Hm2), st>>>(
+      emb, logit, env_off, mask, action, logp_old, adv, ret, eps, c1, c2, vm, eb, d.H, d.A, num_envs, loss, dlogit,
+      demb, logp_out, status);
+  ++n;
+  k_graph_bwd<<<B, 256, sizeof(float) * (H + 2 * Hm + 2 * Hm2), st>>>(emb, dlogit, pm, py1, py2, demb, w.Wg, pd1,
+                                                                       pd2, dpre, dr, d.H);
+  ++n;
+  atb_f32(U, int(HU), dpre, d.H, gp(w.Wg), d.H, B, int(HU), d.H, st); ++n;
+  colsum(dpre, d.H, gp(w.bg), B, d.H, st); ++n;
+  n += mlp_weight_grads(emb, d.H, B, d.Hm, d.Hm2, py1, py2, pd1, pd2, dlogit, gp(w.pW1), gp(w.pb1), gp(w.pWh),
+                        gp(w.pbh), gp(w.pw2), gp(w.pb2), st);
+  n += mlp_weight_grads(eb.vu, 2 * d.H, num_envs, d.Hm, d.Hm2, eb.vy1, eb.vy2, eb.vd1, eb.vd2, eb.vdout, gp(w.vW1),
+                        gp(w.vb1), gp(w.vWh), gp(w.vbh), gp(w.vw2), gp(w.vb2), st);
+  const int64_t ne = N * d.H;
+  if (ne > 0) {
+    const unsigned grid = unsigned(std::min<int64_t>((ne + 255) / 256, int64_t(kNumSMs) * 64));
+    k_readout_bwd<<<grid, 256, 0, st>>>(dr, seg_id, dh, ne, d.H);
+    ++n;
+  }
+  return n;
+}
+
+// One attention layer backwards: dh_out -> (dW, da_src, da_dst, db) and dh_in.  Z / scores hold the layer's
+// forward transform of h_in; dz [N x H] and ds [2 N K] are scratch.
+int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z, const float* scores,
+                         const void* h_in, const void* h_out, const float* dh_out, float* dh_in, float* dz,
+                         float* ds, const LayerWeights& lw, float* gW, float* ga_src, float* ga_dst, float* gb,
+                         int32_t N, cudaStream_t st) {
+  if (N <= 0) return 0;
+  const int H = d.H, K = d.K;
+  cudaMemsetAsync(dz, 0, sizeof(float) * size_t(N) * H, st);
+  cudaMemsetAsync(ds, 0, sizeof(float) * size_t(N) * K * 2, st);
+  float* ds_src = ds;
+  float* ds_dst = ds + size_t(N) * K;
+  const size_t zrow = z_row_bytes(d);
+  const int grid_rows = int(std::min<int64_t>((int64_t(N) + 7) / 8, int64_t(kNumSMs) * 8));
+  const int grid_cols = int(std::min<int64_t>((int64_t(N) + 255) / 256, int64_t(kNumSMs) * 2));
+  const int chunk = chunk_rows(N, 2048);
+  dim3 g_atb(unsigned((H + 63) / 64), unsigned((H + 63) / 64), unsigned((N + chunk - 1) / chunk));
+  dim3 g_gwt(unsigned((N + 63) / 64), unsigned((H + 63) / 64));
+#define BWD_BODY(TY_)                                                                                          \
+  do {                                                                                                         \
+    ZView<TY_> zv;                                                                                             \
+    zv.z = static_cast<const char*>(Z); zv.row_bytes = zrow;                                                   \
+    zv.pairs = d.zmerged ? reinterpret_cast<const float2*>(static_cast<const char*>(Z) + size_t(H) * sizeof(TY_)) \
+                         : reinterpret_cast<const float2*>(scores);                                          \
+    zv.pair_stride = d.zmerged ? int(zrow / 8) : K;                                                            \
+    k_aggregate_bwd<TY_><<<grid_rows, 256, sizeof(float) * H, st>>>(                                           \
+        rowptr, col, zv, static_cast<const TY_*>(h_out), dh_out, dz, ds_src, ds_dst, gb, N, H, K);             \
+    k_scores_bwd<TY_><<<grid_cols, 256, sizeof(float) * 2 * H, st>>>(zv, ds_src, ds_dst, lw.a_src, lw.a_dst, dz, \
+                                                                     ga_src, ga_dst, N, H, K);                 \
+    k_atb<TY_><<<g_atb, 256, 0, st>>>(static_cast<const TY_*>(h_in), H, dz, H, gW, H, N, H, H, chunk);         \
+    k_gwt<TY_><<<g_gwt, 256, 0, st>>>(dz, static_cast<const TY_*>(lw.W), dh_in, N, H, H);                      \
+  } while (0)
+  if (d.dtype == XRL_BF16) BWD_BODY(bf16); else BWD_BODY(float);
+#undef BWD_BODY
+  return 4;
+}
+
+// W0's gradient is collected per CTA in shared memory: (2S + T + 1) x H floats
+size_t embed_bwd_smem_bytes(const Dims& d) { return sizeof(float) * size_t(2 * kS + d.T + 1) * d.H; }
+
+int launch_embed_bwd(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op, const void* shape,
+                     const void* eattr, const void* h0, const float* dh0, float* gW0, float* gb0, int32_t N,
+                     cudaStream_t st) {
+  if (N <= 0) return 0;
+  const size_t smem = embed_bwd_smem_bytes(d);
+  const int grid = int(std::min<int64_t>((int64_t(N) + 63) / 64, int64_t(kNumSMs)));
+  // the opt-in is the kernel's ceiling for every later launch: ask for all an SM has, once per device
+  constexpr int kSmemCeiling = 227 * 1024;
+  if (smem > size_t(kSmemCeiling)) return -1;
+  if (d.dtype == XRL_BF16) {
+    static bool attr[64] = {};
+    if (!ensure_dynamic_smem(k_embed_bwd<bf16>, kSmemCeiling, attr)) return -1;
+    k_embed_bwd<bf16><<<grid, 256, smem, st>>>(rowptr, col, op, static_cast<const bf16*>(shape),
+                                               static_cast<const bf16*>(eattr), static_cast<const bf16*>(h0), dh0,
+                                               gW0, gb0, N, d.H, d.T);
+  } else {
+    static bool attr[64] = {};
+    if (!ensure_dynamic_smem(k_embed_bwd<float>, kSmemCeiling, attr)) return -1;
+    k_embed_bwd<float><<<grid, 256, smem, st>>>(rowptr, col, op, static_cast<const float*>(shape),
+                                                static_cast<const float*>(eattr), static_cast<const float*>(h0), dh0,
+                                                gW0, gb0, N, d.H, d.T);
+  }
+  return 1;
+}
+
+}  // namespace xrl

@@ -4,6 +4,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
 #include <new>
 #include <vector>
 
@@ -84,6 +85,9 @@ struct xrl_ctx {
   cudaStream_t cap_stream = nullptr;
   cudaGraphExec_t graph_exec = nullptr;
   bool capturing = false;
+  // reverse pass: saved layer inputs and gradient scratch (allocated on the first xrl_ppo_grad)
+  DeviceBuf bw;
+  int64_t launches_backward = 0;
   cudaStream_t last_pipe = nullptr;   // stream of the last batch that was packed range by range (its kernels
                                       // report bad graphs too: xrl_last_device_status waits for it as well)
 };
@@ -474,8 +478,10 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
 // Eq. 6 and the first `layers` attention layers over the whole batch; features end up in ctx->h.
 // With fuse_readout the last of the `layers` attention layers may leave per-graph partial sums in
 // ctx->partial instead of node features in ctx->h; *fused tells whether it did.
+// With `hs` (layers + 1 buffers of N x H storage-type values) every layer's input is kept: Eq. 6 writes hs[0],
+// layer l reads hs[l] and writes hs[l + 1].
 int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t st, bool fuse_readout = false,
-                    bool* fused = nullptr, int32_t row_begin = 0, int32_t row_end = -1) {
+                    bool* fused = nullptr, int32_t row_begin = 0, int32_t row_end = -1, void* const* hs = nullptr) {
   const Dims& d = ctx->dims;
   const Window win{row_begin, row_end < 0 ? b->N : row_end, 0};   // graphs are independent: any range of whole graphs
   Profiler& pf = ctx->prof;
@@ -487,20 +493,22 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
   int k = -1;
   if (ctx->use_umma_embed)
     k = launch_embed_umma(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), b->op.as<int32_t>(),
-                          b->shape.p, ctx->w0ext.p, ctx->h.p, win, ctx->status.as<int32_t>(), st, nullptr, eattr);
+                          b->shape.p, ctx->w0ext.p, hs ? hs[0] : ctx->h.p, win, ctx->status.as<int32_t>(), st, nullptr, eattr);
   if (k < 0)
     k = launch_embed(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), b->op.as<int32_t>(),
-                     b->shape.p, ctx->dw, ctx->h.p, win, st, nullptr, eattr);
+                     b->shape.p, ctx->dw, hs ? hs[0] : ctx->h.p, win, st, nullptr, eattr);
   pf.end(FAM_EMBED, slot, k, st);
   int n = k;
   for (int l = 0; l < layers; ++l) {
+    const void* h_in = hs ? hs[l] : ctx->h.p;
+    void* h_out = hs ? hs[l + 1] : ctx->h.p;
     slot = pf.begin(st);
     k = -1;
     if (ctx->use_umma)
-      k = launch_xform_umma(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), win,
+      k = launch_xform_umma(d, h_in, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), win,
                             ctx->status.as<int32_t>(), st);
     if (k < 0 && !d.zmerged)
-      k = launch_xform_simt(d, ctx->h.p, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), win,
+      k = launch_xform_simt(d, h_in, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), win,
                             st);
     if (k < 0) return -1;                       // merged rows: only the tensor-core transform writes them
     pf.end(FAM_XFORM, slot, k, st);
@@ -510,7 +518,7 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
     bool fused_here = false;
     if (fuse_readout && l == layers - 1) {
       k = launch_aggregate_tma(d, gat_rowptr, gat_col, ctx->Z.p,
-                               ctx->scores.as<float>(), ctx->dw.layer[l].b, ctx->h.p, win, b->N,
+                               ctx->scores.as<float>(), ctx->dw.layer[l].b, h_out, win, b->N,
                                b->seg_id.as<int32_t>(), ctx->partial.as<float>(),
                                ctx->status.as<int32_t>(), st);
       if (k >= 0) { fused_here = true; if (fused) *fused = true; }
@@ -518,7 +526,7 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
     if (k < 0)
       k = launch_aggregate(d, gat_rowptr, gat_col, ctx->Z.p,
                            ctx->scores.as<float>(), ctx->dw.layer[l].b,
-                           ctx->h.p, win, b->N, ctx->status.as<int32_t>(), st);
+                           h_out, win, b->N, ctx->status.as<int32_t>(), st);
     if (k < 0) return -1;
     pf.end(fused_here ? FAM_AGG_READOUT : FAM_AGG, slot, k, st);
     n += k;
@@ -608,7 +616,7 @@ void xrl_destroy(xrl_ctx* ctx) {
   cudaSetDevice(ctx->device);
   cudaDeviceSynchronize();
   DeviceBuf* bufs[] = {&ctx->w0ext, &ctx->w_f32, &ctx->w_store, &ctx->h, &ctx->Z, &ctx->scores,
-                       &ctx->partial, &ctx->logits, &ctx->status};
+                       &ctx->partial, &ctx->logits, &ctx->status, &ctx->bw};
   for (DeviceBuf* d : bufs) d->release();
   ctx->prof.release();
   ctx->dl_ints.release(); ctx->dl_col.release(); ctx->dl_scan.release();
@@ -975,6 +983,85 @@ xrl_status xrl_policy_value(xrl_ctx* ctx, const xrl_batch* b, const float* graph
                                      ctx->logits.as<float>(), probs, value, action, seed, step,
                                      ctx->status.as<int32_t>(), st);
   ctx->prof.end(FAM_HEADS, slot, int(ctx->launches_heads), st);
+  XRL_CUDA(cudaGetLastError());
+  return XRL_OK;
+}
+
+xrl_status xrl_ppo_grad(xrl_ctx* ctx, const xrl_batch* b, const float* g0, const uint8_t* mask,
+                        const int32_t* action, const float* logp_old, const float* adv, const float* ret,
+                        float eps, float c1, float c2, float* loss_out, float* grad, float* logp_out,
+                        void* stream) {
+  const xrl_status s = check_encodable(ctx, b);
+  if (s != XRL_OK) return s;
+  if (ctx->capturing) return XRL_ERR_STATE;
+  if (!loss_out || !grad) return XRL_ERR_INVALID_ARG;
+  if (b->num_envs > 0 && (!action || !logp_old || !adv || !ret || (!mask && ctx->cfg.max_actions > 0)))
+    return XRL_ERR_INVALID_ARG;
+  if (embed_bwd_smem_bytes(ctx->dims) > size_t(227) * 1024) return XRL_ERR_UNSUPPORTED;
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  const Dims& d = ctx->dims;
+  const xrl_model_config& c = ctx->cfg;
+  const int L = c.layers;
+  auto up = [](size_t n) { return (n + 255) & ~size_t(255); };
+  const size_t sb = storage_bytes(c.dtype), Nmax = size_t(c.max_nodes), H = size_t(c.hidden);
+  const size_t h_bytes = up(sb * Nmax * H), f_bytes = up(4 * Nmax * H), ds_bytes = up(8 * Nmax * size_t(c.heads));
+  const size_t heads_bytes = up(4 * ppo_heads_workspace_floats(d, c.max_graphs, c.max_envs));
+  if (!ctx->bw.p) {
+    if (ctx->bw.alloc(size_t(L + 1) * h_bytes + 3 * f_bytes + ds_bytes + heads_bytes) != cudaSuccess) {
+      cudaGetLastError();
+      ctx->bw.p = nullptr;
+      return XRL_ERR_ALLOC;
+    }
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (b->nparts > 0) { const xrl_status j = join_parts(b, st); if (j != XRL_OK) return j; }
+  char* p = ctx->bw.as<char>();
+  void* hs[65];
+  for (int l = 0; l <= L; ++l) { hs[l] = p; p += h_bytes; }
+  float* dh_a = reinterpret_cast<float*>(p); p += f_bytes;
+  float* dh_b = reinterpret_cast<float*>(p); p += f_bytes;
+  float* dz = reinterpret_cast<float*>(p); p += f_bytes;
+  float* ds = reinterpret_cast<float*>(p); p += ds_bytes;
+  float* heads_ws = reinterpret_cast<float*>(p);
+  XRL_CUDA(cudaMemsetAsync(grad, 0, 4 * ctx->weight_floats, st));
+  XRL_CUDA(cudaMemsetAsync(loss_out, 0, 16, st));
+  if (b->B == 0 || b->num_envs == 0) return XRL_OK;
+  int n = run_node_layers(ctx, b, L, st, false, nullptr, 0, -1, hs);
+  if (n < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
+  const float* wb = ctx->w_f32.as<float>();
+  n += launch_ppo_heads(d, ctx->dw, grad, wb, hs[L], b->node_off.as<int32_t>(), b->seg_id.as<int32_t>(), g0,
+                        b->d_env_off, mask, action, logp_old, adv, ret, eps, c1, c2, b->B, b->num_envs, b->N,
+                        heads_ws, loss_out, dh_a, logp_out, ctx->status.as<int32_t>(), st);
+  const int32_t* gat_rowptr = c.neighbourhood ? b->rowptr_nbr.as<int32_t>() : b->rowptr.as<int32_t>();
+  const int32_t* gat_col = c.neighbourhood ? b->col_nbr.as<int32_t>() : b->col.as<int32_t>();
+  const Window win{0, b->N, 0};
+  float* dh_cur = dh_a;
+  float* dh_nxt = dh_b;
+  for (int l = L - 1; l >= 0 && b->N > 0; --l) {
+    // the layer's Z rows and half-scores again, from its saved input
+    int k = -1;
+    if (ctx->use_umma)
+      k = launch_xform_umma(d, hs[l], ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), win,
+                            ctx->status.as<int32_t>(), st);
+    if (k < 0 && !d.zmerged)
+      k = launch_xform_simt(d, hs[l], ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), win, st);
+    if (k < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
+    n += k;
+    const LayerWeights& lw = ctx->dw.layer[l];
+    float* ga_src = grad + (lw.a_src - wb);
+    k = launch_gat_layer_bwd(d, gat_rowptr, gat_col, ctx->Z.p, ctx->scores.as<float>(), hs[l], hs[l + 1], dh_cur,
+                             dh_nxt, dz, ds, lw, ga_src - H * H, ga_src, grad + (lw.a_dst - wb),
+                             grad + (lw.b - wb), b->N, st);
+    if (k < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
+    n += k;
+    std::swap(dh_cur, dh_nxt);
+  }
+  const int k = launch_embed_bwd(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), b->op.as<int32_t>(), b->shape.p,
+                                 b->has_eattr ? b->eattr.p : nullptr, hs[0], dh_cur, grad,
+                                 grad + (ctx->dw.b0 - wb), b->N, st);
+  if (k < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
+  n += k;
+  ctx->launches_backward = n;
   XRL_CUDA(cudaGetLastError());
   return XRL_OK;
 }

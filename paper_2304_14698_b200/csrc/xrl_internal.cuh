@@ -199,6 +199,21 @@ int launch_heads(const Dims& d, const DevWeights& w, const float* emb, const int
                  cudaStream_t st);
 int launch_sample(const float* probs, int32_t num_envs, int32_t A1, uint64_t seed, uint64_t step,
                   int32_t* action, cudaStream_t st);
+// ---- reverse pass (Section 3.3.4) --------------------------------------------------------------------
+size_t ppo_heads_workspace_floats(const Dims& d, int64_t B, int64_t num_envs);
+int launch_ppo_heads(const Dims& d, const DevWeights& w, float* grad_base, const float* w_base, const void* hL,
+                     const int32_t* node_off, const int32_t* seg_id, const float* g0, const int32_t* env_off,
+                     const uint8_t* mask, const int32_t* action, const float* logp_old, const float* adv,
+                     const float* ret, float eps, float c1, float c2, int32_t B, int32_t num_envs, int64_t N,
+                     float* ws, float* loss, float* dh, float* logp_out, int32_t* status, cudaStream_t st);
+int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z, const float* scores,
+                         const void* h_in, const void* h_out, const float* dh_out, float* dh_in, float* dz,
+                         float* ds, const LayerWeights& lw, float* gW, float* ga_src, float* ga_dst, float* gb,
+                         int32_t N, cudaStream_t st);
+size_t embed_bwd_smem_bytes(const Dims& d);
+int launch_embed_bwd(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op, const void* shape,
+                     const void* eattr, const void* h0, const float* dh0, float* gW0, float* gb0, int32_t N,
+                     cudaStream_t st);
 int launch_to_float(const void* src, int dtype, float* dst, int64_t n, cudaStream_t st);
 int launch_round_weights(const float* src, void* dst, void* dst_t, int rows, int cols, int dtype,
                          cudaStream_t st);

@@ -1,0 +1,177 @@
+"""GPU parity of the training step's gradient (Section 3.3.4, Eq. 3-5): the loss terms, the log-probabilities
+and the gradient with respect to every weight tensor against the oracle's reverse pass."""
+import numpy as np
+import pytest
+
+from workloads import configs, dags
+import gpu_util
+from test_gpu_fuzz import _random_case
+
+pytestmark = pytest.mark.gpu
+
+# Per weight tensor: |g - r| <= a max|r| + b |r| for every entry, and ||g - r||_2 <= c ||r||_2 + d ||r_all||_2.
+# "fp32" is the check of the reverse pass itself.  A bf16 model keeps Z and every layer's output in bf16.
+# Against the oracle run at such rounded activations ("mirrored", with the half-scores taken where the
+# transform kernel of that shape takes them: from Z before it is rounded on the tensor cores, hidden 128 and
+# 256, from the stored Z otherwise) what remains are values that fall on the other side of a rounding
+# boundary or of a ReLU's zero.  Against the
+# definition, which keeps everything exact, each term of a gradient sum is off by a fraction of a percent
+# per layer it passed, a ReLU of Eq. 8 or of a head may sit on the other side of zero for one graph, and a
+# sum whose terms cancel (the attention vectors') shows that as a large part of its own, small, norm: there
+# the bound is on norms only, tied to the norm of the whole gradient.
+GRAD_TOL = {"fp32": (1e-3, 1e-3, 1e-3, 0.0), "bf16 mirrored": (3e-2, 2e-2, 3e-2, 0.0),
+            "bf16": (None, None, 0.15, 0.01)}
+
+
+def _check_grad(m, got, want, tol, what):
+    off = 0
+    nall = float(np.linalg.norm(want))
+    for name, shape in configs.weight_layout(m):
+        n = int(np.prod(shape))
+        off += n
+        if n == 0:
+            continue
+        g, r = got[off - n:off], want[off - n:off]
+        if tol[0] is not None:
+            bound = tol[0] * np.abs(r).max() + tol[1] * np.abs(r) + 1e-7
+            err = np.abs(g - r)
+            if (err > bound).any():
+                i = int(np.argmax(err - bound))
+                raise AssertionError(f"{what} {name}: {(err > bound).sum()} of {n} outside tolerance; worst at {i}: "
+                                     f"got {g[i]!r} want {r[i]!r} (max |want| {np.abs(r).max():.3e})")
+        nerr, nref = float(np.linalg.norm(g - r)), float(np.linalg.norm(r))
+        assert nerr <= tol[2] * nref + tol[3] * nall + 1e-6, \
+            f"{what} {name}: ||g - r|| = {nerr:.3e}, ||r|| = {nref:.3e}, ||r_all|| = {nall:.3e}"
+    if tol[3] > 0:
+        assert np.linalg.norm(got - want) <= 0.15 * nall, (what, float(np.linalg.norm(got - want)), nall)
+
+def _transitions(xo, m, blob, batch, packed, seed, g0=None):
+    """Actions, old log-probabilities, advantages and value targets for every environment of the batch."""
+    rng = np.random.default_rng(seed)
+    enc = xo.encode(m, blob, batch, packed, g0=g0)
+    st, _, probs, _ = xo.policy_value(m, blob, batch, enc["emb"])
+    assert st == 0
+    ne = probs.shape[0]
+    action = np.array([rng.choice(np.flatnonzero(probs[e] > 0)) for e in range(ne)], np.int32)
+    logp_now = np.log(probs[np.arange(ne), action])
+    # ratios on both sides of the clipping range and inside it
+    logp_old = logp_now + rng.choice([-0.5, -0.05, 0.03, 0.4], size=ne)
+    adv = rng.normal(size=ne)
+    ret = rng.normal(size=ne)
+    return action, logp_old, adv, ret
+
+
+def _compare(xo, batch, m, blob, g0=None, seed=0, eps=0.2, c1=0.5, c2=0.01):
+    import torch
+    import paper_2304_14698_b200 as xrl
+    st, packed = xo.pack(batch)
+    assert st == 0
+    action, logp_old, adv, ret = _transitions(xo, m, blob, batch, packed, seed, g0)
+    want = xo.ppo_grad(m, blob, batch, packed, action, logp_old, adv, ret, eps, c1, c2, g0=g0)
+    ag = gpu_util.make_agent(batch, slack=2)
+    try:
+        ag.set_weights(blob)
+        ag.pack(batch)
+        f32 = lambda a: torch.from_numpy(np.asarray(a, np.float32)).cuda()
+        loss = torch.full((4,), 7.0, device="cuda")
+        grad = torch.full((len(blob),), 7.0, device="cuda")
+        logp = torch.empty(len(action), device="cuda")
+        g0d = None if g0 is None else f32(g0)
+        for _ in range(2):                 # the second call reuses the workspace and must overwrite, not add
+            xrl.xrl_ppo_grad(ag.ctx, ag.batch, torch.from_numpy(batch["mask"]).cuda(),
+                             torch.from_numpy(action).cuda(), f32(logp_old), f32(adv), f32(ret), loss, grad,
+                             eps=eps, c1=c1, c2=c2, g0=g0d, logp_out=logp)
+        torch.cuda.synchronize()
+        assert ag.device_status() == 0
+        dt = m["dtype"]
+        gpu_util.assert_close(loss.cpu().numpy(), want["loss"], dt, "loss")
+        gpu_util.assert_close(logp.cpu().numpy(), want["logp"], dt, "logp")
+        got = grad.cpu().numpy().astype(np.float64)
+        _check_grad(m, got, want["grad"], GRAD_TOL[dt], "definition")
+        if dt == "bf16":
+            mir = xo.ppo_grad(m, blob, batch, packed, action, logp_old, adv, ret, eps, c1, c2, g0=g0,
+                              mirrored=1 if m["H"] in (128, 256) else 2)
+            _check_grad(m, got, mir["grad"], GRAD_TOL["bf16 mirrored"], "mirrored")
+            np.testing.assert_allclose(loss.cpu().numpy(), mir["loss"], rtol=2e-3, atol=1e-4)
+        # the forward pass of the same context still works afterwards and agrees with the oracle
+        o = ag.forward(torch.from_numpy(batch["mask"]).cuda(), g0=g0d)
+        torch.cuda.synchronize()
+        enc = xo.encode(m, blob, batch, packed, g0=g0)
+        gpu_util.assert_close(o["emb"].cpu().numpy(), enc["emb"], dt, "emb after the gradient")
+    finally:
+        ag.close()
+
+
+def _small_batch(m, seed, envs=(3, 0, 5), nodes=(3, 40), edge_attr=False):
+    rng = dags.make_rng(seed)
+    graphs, env_off = [], [0]
+    for c in envs:
+        for _ in range(c + 1):
+            graphs.append(dags.random_dag(rng, int(rng.integers(*nodes)), m["T"], 8, m["dtype"] == "bf16", window=6))
+        env_off.append(len(graphs))
+    b = dags.flatten(graphs, env_off, m["A_max"])
+    b["mask"][0, 1] = 0
+    if edge_attr:
+        b["edge_attr"] = dags.tensor_shape_attributes(rng, int(b["n_edges"].sum()), 8, m["dtype"] == "bf16")
+    b["model"] = m
+    return b
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("variant", ["plain", "two hidden layers", "edge attributes", "both ways", "no layers",
+                                     "three heads", "hidden 256"])
+def test_gradient_matches_the_oracle(xo, dtype, variant):
+    m = dict(T=12, S=8, H=64, K=4, L=2, Hm=24, Dg=2, dtype=dtype, A_max=6)
+    if variant == "two hidden layers":
+        m["Hm2"] = 9
+    if variant == "edge attributes":
+        m["edge_attr"] = True
+    if variant == "both ways":
+        m["both_ways"] = True
+    if variant == "no layers":
+        m["L"] = 0
+    if variant == "three heads":
+        m.update(H=96, K=3, L=1)
+    if variant == "hidden 256":                      # the tensor-core transform and merged Z rows (bf16)
+        m.update(H=256, K=8, L=3, Hm=64, Hm2=16, T=40)
+    b = _small_batch(m, 11, edge_attr=(variant == "edge attributes"))
+    blob, _ = gpu_util.default_weights(b, 5)
+    rng = np.random.default_rng(2)
+    g0 = rng.normal(size=(b["num_graphs"], m["Dg"]))
+    _compare(xo, b, m, blob, g0=g0, seed=3)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_gradient_on_random_batches(xo, seed):
+    batch, m, blob, _hint, g0 = _random_case(seed)
+    _compare(xo, batch, m, blob, g0=g0, seed=seed)
+
+
+def test_gradient_on_a_step_of_the_papers_size(xo):
+    b = configs.make_batch(6, candidates=5)
+    blob, _ = gpu_util.default_weights(b, 1)
+    _compare(xo, b, b["model"], blob, seed=4)
+
+
+def test_an_action_the_mask_excludes_is_reported(xo):
+    import torch
+    import paper_2304_14698_b200 as xrl
+    m = dict(T=12, S=8, H=64, K=4, L=1, Hm=24, Dg=0, dtype="fp32", A_max=6)
+    b = _small_batch(m, 1)
+    blob, _ = gpu_util.default_weights(b, 5)
+    ag = gpu_util.make_agent(b)
+    try:
+        ag.set_weights(blob)
+        ag.pack(b)
+        ne = len(b["env_off"]) - 1
+        z = torch.zeros(ne, device="cuda")
+        action = torch.full((ne,), m["A_max"], dtype=torch.int32, device="cuda")
+        action[0] = 1                                   # masked out in _small_batch
+        loss = torch.empty(4, device="cuda"); grad = torch.empty(len(blob), device="cuda")
+        xrl.xrl_ppo_grad(ag.ctx, ag.batch, torch.from_numpy(b["mask"]).cuda(), action, z, z, z, loss, grad)
+        assert ag.device_status() == 1
+        with pytest.raises(xrl.XrlError) as e:
+            xrl.xrl_ppo_grad(ag.ctx, ag.batch, torch.from_numpy(b["mask"]).cuda(), action, z, z, z, None, grad)
+        assert e.value.status == 1
+    finally:
+        ag.close()
