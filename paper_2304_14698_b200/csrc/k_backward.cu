@@ -32,7 +32,6 @@ template <typename T> struct ZView {
   __device__ __forceinline__ float2 pair(int32_t i, int k) const { return pairs[size_t(i) * pair_stride + k]; }
 };
 
-constexpr int kMaxHeads = 64;
 constexpr int kMaxPerLane = 16;          // hidden <= 512
 
 // ---- Eq. 7, reverse: one warp per destination row ---------------------------------------------------
@@ -161,6 +160,180 @@ k_scores_bwd(ZView<T> zv, const float* __restrict__ ds_src, const float* __restr
   }
 }
 
+// ---- the same two kernels for the usual shapes: K divides 32 and H = 32 NF, NF in {1, 2, 4, 8, 16} ----------
+// A lane owns NF consecutive features, all of one head (32 / K lanes per head): a head's reductions stay inside
+// its group of lanes, all heads proceed at once, rows move as 4- to 16-byte pieces, and the scattered sums
+// go out as vector atomics.
+template <typename T, int NF> struct alignas((sizeof(T) * NF) >= 16 ? 16 : sizeof(T) * NF) Chunk { T v[NF]; };
+
+template <typename T, int NF>
+__device__ __forceinline__ void load_chunk(const T* p, float (&f)[NF]) {
+  const Chunk<T, NF> c = *reinterpret_cast<const Chunk<T, NF>*>(p);
+#pragma unroll
+  for (int t = 0; t < NF; ++t) f[t] = to_float(c.v[t]);
+}
+template <int NF>
+__device__ __forceinline__ void store_chunk(float* p, const float (&f)[NF]) {
+  Chunk<float, NF> c;
+#pragma unroll
+  for (int t = 0; t < NF; ++t) c.v[t] = f[t];
+  *reinterpret_cast<Chunk<float, NF>*>(p) = c;
+}
+template <int NF>
+__device__ __forceinline__ void atomic_add_chunk(float* p, const float (&v)[NF]) {
+  if constexpr (NF % 4 == 0) {
+#pragma unroll
+    for (int q = 0; q < NF / 4; ++q)
+      atomicAdd(reinterpret_cast<float4*>(p) + q, make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]));
+  } else if constexpr (NF % 2 == 0) {
+#pragma unroll
+    for (int q = 0; q < NF / 2; ++q) atomicAdd(reinterpret_cast<float2*>(p) + q, make_float2(v[2 * q], v[2 * q + 1]));
+  } else {
+#pragma unroll
+    for (int q = 0; q < NF; ++q) atomicAdd(p + q, v[q]);
+  }
+}
+
+template <typename T, int NF>
+__global__ void __launch_bounds__(256)
+k_aggregate_bwd_rows(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col, ZView<T> zv,
+                     const T* __restrict__ h_out, const float* __restrict__ dh_out, float* __restrict__ dz,
+                     float* __restrict__ ds_src, float* __restrict__ ds_dst, float* __restrict__ db, int N, int K) {
+  constexpr int H = 32 * NF;
+  __shared__ float sm_db[H];
+  for (int c = threadIdx.x; c < H; c += blockDim.x) sm_db[c] = 0.f;
+  __syncthreads();
+  const int lane = threadIdx.x & 31;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  const int lph = 32 / K, k = lane / lph;            // lanes per head, this lane's head
+  const bool leader = (lane % lph) == 0;
+  float dbr[NF];
+#pragma unroll
+  for (int f = 0; f < NF; ++f) dbr[f] = 0.f;
+  for (int32_t i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < N; i += warps) {
+    float dp[NF];
+    {
+      float g[NF], ho[NF];
+      load_chunk<float, NF>(dh_out + size_t(i) * H + lane * NF, g);
+      load_chunk<T, NF>(h_out + size_t(i) * H + lane * NF, ho);
+#pragma unroll
+      for (int f = 0; f < NF; ++f) { dp[f] = ho[f] > 0.f ? g[f] : 0.f; dbr[f] += dp[f]; }
+    }
+    bool live = false;
+#pragma unroll
+    for (int f = 0; f < NF; ++f) live = live || dp[f] != 0.f;
+    if (!__any_sync(0xFFFFFFFFu, live)) continue;     // a row whose units are all off: nothing flows (ds is zeroed)
+    const int32_t e0 = rowptr[i], deg = rowptr[i + 1] - e0;
+    const float sd = zv.pair(i, k).y;
+    // softmax statistics of this lane's head over the row's neighbours and the row itself (entry `deg`)
+    float mx = -INFINITY, sum = 0.f;
+    for (int base = 0; base <= deg; base += 32) {
+      const int idx = base + lane;
+      const int32_t cj = idx < deg ? col[e0 + idx] : i;
+      const int cnt = min(32, deg + 1 - base);
+      for (int t = 0; t < cnt; ++t) {
+        const int32_t j = __shfl_sync(0xFFFFFFFFu, cj, t);
+        const float e = lrelu(zv.pair(j, k).x + sd);
+        if (e > mx) { sum = sum * exp2f(mx - e) + 1.f; mx = e; } else { sum += exp2f(e - mx); }
+      }
+    }
+    const float inv = 1.f / sum;
+    float dot = 0.f;
+    for (int base = 0; base <= deg; base += 32) {
+      const int idx = base + lane;
+      const int32_t cj = idx < deg ? col[e0 + idx] : i;
+      const int cnt = min(32, deg + 1 - base);
+      for (int t = 0; t < cnt; ++t) {
+        const int32_t j = __shfl_sync(0xFFFFFFFFu, cj, t);
+        float z[NF];
+        load_chunk<T, NF>(zv.row(j) + lane * NF, z);
+        float part = 0.f;
+#pragma unroll
+        for (int f = 0; f < NF; ++f) part = fmaf(dp[f], z[f], part);
+        for (int o = lph >> 1; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+        const float al = exp2f(lrelu(zv.pair(j, k).x + sd) - mx) * inv;
+        dot = fmaf(al, part, dot);
+      }
+    }
+    float dsd = 0.f;
+    for (int base = 0; base <= deg; base += 32) {
+      const int idx = base + lane;
+      const int32_t cj = idx < deg ? col[e0 + idx] : i;
+      const int cnt = min(32, deg + 1 - base);
+      for (int t = 0; t < cnt; ++t) {
+        const int32_t j = __shfl_sync(0xFFFFFFFFu, cj, t);
+        float z[NF];
+        load_chunk<T, NF>(zv.row(j) + lane * NF, z);
+        float part = 0.f;
+#pragma unroll
+        for (int f = 0; f < NF; ++f) part = fmaf(dp[f], z[f], part);
+        for (int o = lph >> 1; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+        const float e = zv.pair(j, k).x + sd;
+        const float al = exp2f(lrelu(e) - mx) * inv;
+        const float de = al * (part - dot) * (e > 0.f ? 1.f : 0.2f);
+        dsd += de;
+        if (leader && de != 0.f) atomicAdd(&ds_src[size_t(j) * K + k], de);
+        if (live) {
+          float v[NF];
+#pragma unroll
+          for (int f = 0; f < NF; ++f) v[f] = al * dp[f];
+          atomic_add_chunk<NF>(dz + size_t(j) * H + lane * NF, v);
+        }
+      }
+    }
+    if (leader) ds_dst[size_t(i) * K + k] = dsd;
+  }
+#pragma unroll
+  for (int f = 0; f < NF; ++f)
+    if (dbr[f] != 0.f) atomicAdd(&sm_db[lane * NF + f], dbr[f]);
+  __syncthreads();
+  for (int c = threadIdx.x; c < H; c += blockDim.x)
+    if (sm_db[c] != 0.f) atomicAdd(&db[c], sm_db[c]);
+}
+
+template <typename T, int NF>
+__global__ void __launch_bounds__(256)
+k_scores_bwd_rows(ZView<T> zv, const float* __restrict__ ds_src, const float* __restrict__ ds_dst,
+                  const float* __restrict__ a_src, const float* __restrict__ a_dst, float* __restrict__ dz,
+                  float* __restrict__ da_src, float* __restrict__ da_dst, int N, int K) {
+  constexpr int H = 32 * NF;
+  __shared__ float sm_da[2 * H];
+  for (int c = threadIdx.x; c < 2 * H; c += blockDim.x) sm_da[c] = 0.f;
+  __syncthreads();
+  const int lane = threadIdx.x & 31;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  const int k = lane / (32 / K);
+  float as[NF], ad[NF], accs[NF], accd[NF];
+  load_chunk<float, NF>(a_src + lane * NF, as);
+  load_chunk<float, NF>(a_dst + lane * NF, ad);
+#pragma unroll
+  for (int f = 0; f < NF; ++f) { accs[f] = 0.f; accd[f] = 0.f; }
+  for (int32_t i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < N; i += warps) {
+    const float gs = ds_src[size_t(i) * K + k], gd = ds_dst[size_t(i) * K + k];
+    if (gs == 0.f && gd == 0.f) continue;
+    float z[NF], g[NF];
+    load_chunk<T, NF>(zv.row(i) + lane * NF, z);
+    load_chunk<float, NF>(dz + size_t(i) * H + lane * NF, g);
+#pragma unroll
+    for (int f = 0; f < NF; ++f) {
+      g[f] += gs * as[f] + gd * ad[f];
+      accs[f] = fmaf(gs, z[f], accs[f]);
+      accd[f] = fmaf(gd, z[f], accd[f]);
+    }
+    store_chunk<NF>(dz + size_t(i) * H + lane * NF, g);
+  }
+#pragma unroll
+  for (int f = 0; f < NF; ++f) {
+    atomicAdd(&sm_da[lane * NF + f], accs[f]);
+    atomicAdd(&sm_da[H + lane * NF + f], accd[f]);
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    if (sm_da[c] != 0.f) atomicAdd(&da_src[c], sm_da[c]);
+    if (sm_da[H + c] != 0.f) atomicAdd(&da_dst[c], sm_da[H + c]);
+  }
+}
+
 // ---- dW += A^T B over a range of rows: A [rows x Ka] (storage type), B [rows x Nb] fp32 -------------------
 // 64 x 64 output tile per CTA, the rows cut into chunks along grid.z, partial products added with atomics.
 template <typename TA>
@@ -240,8 +413,10 @@ k_gwt(const float* __restrict__ G, const TW* __restrict__ W, float* __restrict__
 }
 
 // ---- Eq. 6, reverse: dW0 += x^T dpre, db0 += dpre, x_i = [edge sum | one-hot op | own shape] -------------
-// One warp per row builds x's 16 dense entries; a CTA adds its rows' outer products into a shared-memory
-// copy of W0's gradient ([2S + T] x H floats) and adds that to global memory once.
+// A CTA takes a range of rows and keeps its share of W0's gradient in shared memory ([2S + T + 1] x H floats,
+// the last row for b0).  A warp takes a row at a time, a lane the columns lane, lane + 32, ...: the sixteen dense
+// entries of x meet dpre in registers (four columns per lane at a time), the one-hot entry is one shared-memory
+// add per column, and the registers are added to shared memory once per pass over the rows.
 template <typename T>
 __global__ void __launch_bounds__(256)
 k_embed_bwd(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col, const int32_t* __restrict__ op,
@@ -254,28 +429,56 @@ k_embed_bwd(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
   const int rows_per_cta = (N + gridDim.x - 1) / gridDim.x;
   const int r0 = blockIdx.x * rows_per_cta, r1 = min(N, r0 + rows_per_cta);
-  for (int i = r0 + warp; i < r1; i += nw) {
-    float x[2 * kS];
+  const int NF = H / 32;
+  constexpr int CU = 4;                            // columns per lane and pass
+  for (int f0 = 0; f0 < NF; f0 += CU) {
+    float a[2 * kS][CU], dbr[CU];
 #pragma unroll
-    for (int s = 0; s < 2 * kS; ++s) x[s] = 0.f;
-    for (int32_t e = rowptr[i]; e < rowptr[i + 1]; ++e) {
-      const T* src = eattr ? eattr + size_t(e) * kS : shape + size_t(col[e]) * kS;
+    for (int u = 0; u < CU; ++u) {
+      dbr[u] = 0.f;
 #pragma unroll
-      for (int s = 0; s < kS; ++s) x[s] += to_float(src[s]);
+      for (int s = 0; s < 2 * kS; ++s) a[s][u] = 0.f;
+    }
+    for (int i = r0 + warp; i < r1; i += nw) {
+      float dp[CU];
+      bool live = false;
+#pragma unroll
+      for (int u = 0; u < CU; ++u) {
+        const int c = lane + 32 * (f0 + u);
+        dp[u] = (f0 + u < NF && to_float(h0[size_t(i) * H + c]) > 0.f) ? dh0[size_t(i) * H + c] : 0.f;
+        live = live || dp[u] != 0.f;
+      }
+      if (!__any_sync(0xFFFFFFFFu, live)) continue;
+      float x[2 * kS];
+#pragma unroll
+      for (int s = 0; s < 2 * kS; ++s) x[s] = 0.f;
+      for (int32_t e = rowptr[i]; e < rowptr[i + 1]; ++e) {
+        float v[kS];
+        load_chunk<T, kS>(eattr ? eattr + size_t(e) * kS : shape + size_t(col[e]) * kS, v);
+#pragma unroll
+        for (int s = 0; s < kS; ++s) x[s] += v[s];
+      }
+      load_chunk<T, kS>(shape + size_t(i) * kS, reinterpret_cast<float(&)[kS]>(x[kS]));
+      const int o = op[i];
+#pragma unroll
+      for (int u = 0; u < CU; ++u) {
+        if (dp[u] == 0.f) continue;
+#pragma unroll
+        for (int s = 0; s < 2 * kS; ++s) a[s][u] = fmaf(x[s], dp[u], a[s][u]);
+        atomicAdd(&acc[size_t(kS + o) * H + lane + 32 * (f0 + u)], dp[u]);
+        dbr[u] += dp[u];
+      }
     }
 #pragma unroll
-    for (int s = 0; s < kS; ++s) x[kS + s] = to_float(shape[size_t(i) * kS + s]);
-    const int o = op[i];
-    for (int c = lane; c < H; c += 32) {
-      const float dp = to_float(h0[size_t(i) * H + c]) > 0.f ? dh0[size_t(i) * H + c] : 0.f;
-      if (dp == 0.f) continue;
+    for (int u = 0; u < CU; ++u) {
+      if (f0 + u >= NF) continue;
+      const int c = lane + 32 * (f0 + u);
 #pragma unroll
       for (int s = 0; s < kS; ++s) {
-        atomicAdd(&acc[size_t(s) * H + c], x[s] * dp);
-        atomicAdd(&acc[size_t(kS + Tn + s) * H + c], x[kS + s] * dp);
+        atomicAdd(&acc[size_t(s) * H + c], a[s][u]);
+        atomicAdd(&acc[size_t(kS + Tn + s) * H + c], a[kS + s][u]);
       }
-      atomicAdd(&acc[size_t(kS + o) * H + c], dp);
-      atomicAdd(&acc[size_t(F0) * H + c], dp);
+      atomicAdd(&acc[size_t(F0) * H + c], dbr[u]);
     }
   }
   __syncthreads();
@@ -688,6 +891,15 @@ int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* co
   const int chunk = chunk_rows(N, 2048);
   dim3 g_atb(unsigned((H + 63) / 64), unsigned((H + 63) / 64), unsigned((N + chunk - 1) / chunk));
   dim3 g_gwt(unsigned((N + 63) / 64), unsigned((H + 63) / 64));
+  const int NF = H / 32;
+  const bool rows_kernels = (32 % K == 0) && (NF == 1 || NF == 2 || NF == 4 || NF == 8 || NF == 16);
+#define BWD_ROWS(TY_, NF_)                                                                                     \
+  do {                                                                                                         \
+    k_aggregate_bwd_rows<TY_, NF_><<<grid_rows, 256, 0, st>>>(rowptr, col, zv, static_cast<const TY_*>(h_out), \
+                                                              dh_out, dz, ds_src, ds_dst, gb, N, K);           \
+    k_scores_bwd_rows<TY_, NF_><<<grid_rows, 256, 0, st>>>(zv, ds_src, ds_dst, lw.a_src, lw.a_dst, dz, ga_src, \
+                                                           ga_dst, N, K);                                      \
+  } while (0)
 #define BWD_BODY(TY_)                                                                                          \
   do {                                                                                                         \
     ZView<TY_> zv;                                                                                             \
@@ -695,14 +907,25 @@ int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* co
     zv.pairs = d.zmerged ? reinterpret_cast<const float2*>(static_cast<const char*>(Z) + size_t(H) * sizeof(TY_)) \
                          : reinterpret_cast<const float2*>(scores);                                          \
     zv.pair_stride = d.zmerged ? int(zrow / 8) : K;                                                            \
-    k_aggregate_bwd<TY_><<<grid_rows, 256, sizeof(float) * H, st>>>(                                           \
-        rowptr, col, zv, static_cast<const TY_*>(h_out), dh_out, dz, ds_src, ds_dst, gb, N, H, K);             \
-    k_scores_bwd<TY_><<<grid_cols, 256, sizeof(float) * 2 * H, st>>>(zv, ds_src, ds_dst, lw.a_src, lw.a_dst, dz, \
-                                                                     ga_src, ga_dst, N, H, K);                 \
+    if (rows_kernels) {                                                                                        \
+      switch (NF) {                                                                                            \
+        case 1: BWD_ROWS(TY_, 1); break;                                                                       \
+        case 2: BWD_ROWS(TY_, 2); break;                                                                       \
+        case 4: BWD_ROWS(TY_, 4); break;                                                                       \
+        case 8: BWD_ROWS(TY_, 8); break;                                                                       \
+        default: BWD_ROWS(TY_, 16); break;                                                                     \
+      }                                                                                                        \
+    } else {                                                                                                   \
+      k_aggregate_bwd<TY_><<<grid_rows, 256, sizeof(float) * H, st>>>(                                         \
+          rowptr, col, zv, static_cast<const TY_*>(h_out), dh_out, dz, ds_src, ds_dst, gb, N, H, K);           \
+      k_scores_bwd<TY_><<<grid_cols, 256, sizeof(float) * 2 * H, st>>>(zv, ds_src, ds_dst, lw.a_src, lw.a_dst, \
+                                                                       dz, ga_src, ga_dst, N, H, K);           \
+    }                                                                                                          \
     k_atb<TY_><<<g_atb, 256, 0, st>>>(static_cast<const TY_*>(h_in), H, dz, H, gW, H, N, H, H, chunk);         \
     k_gwt<TY_><<<g_gwt, 256, 0, st>>>(dz, static_cast<const TY_*>(lw.W), dh_in, N, H, H);                      \
   } while (0)
   if (d.dtype == XRL_BF16) BWD_BODY(bf16); else BWD_BODY(float);
+#undef BWD_ROWS
 #undef BWD_BODY
   return 4;
 }
