@@ -268,7 +268,7 @@ xrl_status xrl_sample(xrl_ctx* ctx, const float* probs, int32_t num_envs, int32_
  *   loss_out  DEVICE fp32 [4] = { J, L_clip, L_vf, L_ent }
  *   grad      DEVICE fp32, laid out like the weight blob (xrl_weights_size bytes), overwritten
  *   logp_out  DEVICE fp32 [num_envs] or NULL: log pi(action_e) under the current weights
- * The first call allocates the workspace for the context's capacities ((L + 1) copies of the node features
+ * The first call allocates the workspace for the context's capacities ((L + 2) copies of the node features
  * plus three fp32 ones) and therefore synchronises; later calls only enqueue.  Not recordable
  * (XRL_ERR_STATE between xrl_graph_begin and xrl_graph_launch).  XRL_ERR_UNSUPPORTED when
  * (2 S + T + 1) x H floats exceed one SM's shared memory (227 KB): W0's gradient is collected there.

@@ -295,7 +295,7 @@ template <typename T, int NF>
 __global__ void __launch_bounds__(256)
 k_scores_bwd_rows(ZView<T> zv, const float* __restrict__ ds_src, const float* __restrict__ ds_dst,
                   const float* __restrict__ a_src, const float* __restrict__ a_dst, float* __restrict__ dz,
-                  float* __restrict__ da_src, float* __restrict__ da_dst, int N, int K) {
+                  bf16* __restrict__ dzb, float* __restrict__ da_src, float* __restrict__ da_dst, int N, int K) {
   constexpr int H = 32 * NF;
   __shared__ float sm_da[2 * H];
   for (int c = threadIdx.x; c < 2 * H; c += blockDim.x) sm_da[c] = 0.f;
@@ -310,17 +310,24 @@ k_scores_bwd_rows(ZView<T> zv, const float* __restrict__ ds_src, const float* __
   for (int f = 0; f < NF; ++f) { accs[f] = 0.f; accd[f] = 0.f; }
   for (int32_t i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < N; i += warps) {
     const float gs = ds_src[size_t(i) * K + k], gd = ds_dst[size_t(i) * K + k];
-    if (gs == 0.f && gd == 0.f) continue;
     float z[NF], g[NF];
-    load_chunk<T, NF>(zv.row(i) + lane * NF, z);
     load_chunk<float, NF>(dz + size_t(i) * H + lane * NF, g);
+    if (gs != 0.f || gd != 0.f) {
+      load_chunk<T, NF>(zv.row(i) + lane * NF, z);
 #pragma unroll
-    for (int f = 0; f < NF; ++f) {
-      g[f] += gs * as[f] + gd * ad[f];
-      accs[f] = fmaf(gs, z[f], accs[f]);
-      accd[f] = fmaf(gd, z[f], accd[f]);
+      for (int f = 0; f < NF; ++f) {
+        g[f] += gs * as[f] + gd * ad[f];
+        accs[f] = fmaf(gs, z[f], accs[f]);
+        accd[f] = fmaf(gd, z[f], accd[f]);
+      }
+      if (dzb == nullptr) store_chunk<NF>(dz + size_t(i) * H + lane * NF, g);
     }
-    store_chunk<NF>(dz + size_t(i) * H + lane * NF, g);
+    if (dzb != nullptr) {                             // the tensor-core products read dz in bf16
+      Chunk<bf16, NF> c;
+#pragma unroll
+      for (int f = 0; f < NF; ++f) c.v[f] = __float2bfloat16(g[f]);
+      *reinterpret_cast<Chunk<bf16, NF>*>(dzb + size_t(i) * H + lane * NF) = c;
+    }
   }
 #pragma unroll
   for (int f = 0; f < NF; ++f) {
@@ -409,6 +416,159 @@ k_gwt(const float* __restrict__ G, const TW* __restrict__ W, float* __restrict__
     for (int v = 0; v < 4; ++v) {
       const int r = r0 + ty * 4 + u, k = k0 + tx * 4 + v;
       if (r < rows && k < Hk) out[size_t(r) * Hk + k] = acc[u][v];
+    }
+}
+
+// ---- the two products of a layer's reverse pass on the tensor cores (bf16 models, H a multiple of 128) --------
+// mma.sync m16n8k16, bf16 operands, fp32 accumulators; a CTA of 8 warps (4 x 2) takes a 128 x 128 tile of the
+// result, a warp 32 x 64.  Operand tiles sit in shared memory in 16-byte pieces whose position within a row is
+// XOR-ed with the row number, so that the eight rows one ldmatrix reads fall into different banks.
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// out [rows x H] fp32 = G [rows x H] bf16 times W^T, W [H x H] bf16 row-major [in x out]: out[r][k] = sum_n G[r][n] W[k][n]
+__global__ void __launch_bounds__(256)
+k_gwt_mma(const bf16* __restrict__ G, const bf16* __restrict__ W, float* __restrict__ out, int rows, int H) {
+  __shared__ __align__(128) bf16 As[128 * 64];      // [row r][64 n], 8 pieces of 16 bytes per row
+  __shared__ __align__(128) bf16 Bs[128 * 64];      // [row k][64 n]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int wm = warp >> 1, wn = warp & 1;
+  const int r0 = blockIdx.x * 128, k0 = blockIdx.y * 128;
+  float acc[2][8][4];
+#pragma unroll
+  for (int a = 0; a < 2; ++a)
+#pragma unroll
+    for (int b = 0; b < 8; ++b)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) acc[a][b][c] = 0.f;
+  const uint32_t as_base = uint32_t(__cvta_generic_to_shared(As)), bs_base = uint32_t(__cvta_generic_to_shared(Bs));
+  for (int n0 = 0; n0 < H; n0 += 64) {
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+      const int idx = tid + 256 * it, row = idx >> 3, ch = idx & 7;
+      uint4 va = make_uint4(0, 0, 0, 0);
+      if (r0 + row < rows) va = *reinterpret_cast<const uint4*>(G + size_t(r0 + row) * H + n0 + ch * 8);
+      const uint4 vb = *reinterpret_cast<const uint4*>(W + size_t(k0 + row) * H + n0 + ch * 8);
+      const int phys = (row * 8 + (ch ^ (row & 7))) * 8;
+      *reinterpret_cast<uint4*>(As + phys) = va;
+      *reinterpret_cast<uint4*>(Bs + phys) = vb;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 64; kk += 16) {
+      uint32_t af[2][4];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        const int row = wm * 32 + mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+        const int ch = (kk >> 3) + (lane >> 4);
+        ldsm_x4(af[mt], as_base + uint32_t((row * 8 + (ch ^ (row & 7))) * 16));
+      }
+#pragma unroll
+      for (int np = 0; np < 4; ++np) {
+        uint32_t bf[4];
+        const int row = wn * 64 + np * 16 + (lane & 7) + (lane >> 4) * 8;
+        const int ch = (kk >> 3) + ((lane >> 3) & 1);
+        ldsm_x4(bf, bs_base + uint32_t((row * 8 + (ch ^ (row & 7))) * 16));
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          mma_bf16(acc[mt][2 * np], af[mt], bf[0], bf[1]);
+          mma_bf16(acc[mt][2 * np + 1], af[mt], bf[2], bf[3]);
+        }
+      }
+    }
+    __syncthreads();
+  }
+  const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+      const int r = r0 + wm * 32 + mt * 16 + g, c = k0 + wn * 64 + nt * 8 + 2 * t;
+      if (r < rows) *reinterpret_cast<float2*>(out + size_t(r) * H + c) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
+      if (r + 8 < rows)
+        *reinterpret_cast<float2*>(out + size_t(r + 8) * H + c) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
+    }
+}
+
+// dW [H x H] fp32 += A^T B over the rows [chunk z], A = h_in [rows x H] bf16, B = dz [rows x H] bf16
+__global__ void __launch_bounds__(256)
+k_atb_mma(const bf16* __restrict__ A, const bf16* __restrict__ Bm, float* __restrict__ dW, int rows, int H,
+          int rows_per_chunk) {
+  __shared__ __align__(128) bf16 As[32 * 128];      // [row r][128 m], 16 pieces of 16 bytes per row
+  __shared__ __align__(128) bf16 Bs[32 * 128];      // [row r][128 n]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int wm = warp >> 1, wn = warp & 1;
+  const int m0 = blockIdx.x * 128, n0 = blockIdx.y * 128;
+  const int r_begin = blockIdx.z * rows_per_chunk, r_end = min(rows, r_begin + rows_per_chunk);
+  float acc[2][8][4];
+#pragma unroll
+  for (int a = 0; a < 2; ++a)
+#pragma unroll
+    for (int b = 0; b < 8; ++b)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) acc[a][b][c] = 0.f;
+  const uint32_t as_base = uint32_t(__cvta_generic_to_shared(As)), bs_base = uint32_t(__cvta_generic_to_shared(Bs));
+  for (int rr = r_begin; rr < r_end; rr += 32) {
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+      const int idx = tid + 256 * it, row = idx >> 4, ch = idx & 15;
+      uint4 va = make_uint4(0, 0, 0, 0), vb = make_uint4(0, 0, 0, 0);
+      if (rr + row < r_end) {
+        va = *reinterpret_cast<const uint4*>(A + size_t(rr + row) * H + m0 + ch * 8);
+        vb = *reinterpret_cast<const uint4*>(Bm + size_t(rr + row) * H + n0 + ch * 8);
+      }
+      const int phys = (row * 16 + (ch ^ (row & 7))) * 8;
+      *reinterpret_cast<uint4*>(As + phys) = va;
+      *reinterpret_cast<uint4*>(Bs + phys) = vb;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 32; kk += 16) {
+      uint32_t af[2][4];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        // the stored rows are the products' k index: transposed 8 x 8 loads give the (m, k) fragments
+        const int row = kk + (lane & 7) + (lane >> 4) * 8;
+        const int ch = ((wm * 32 + mt * 16) >> 3) + ((lane >> 3) & 1);
+        ldsm_x4_trans(af[mt], as_base + uint32_t((row * 16 + (ch ^ (row & 7))) * 16));
+      }
+#pragma unroll
+      for (int np = 0; np < 4; ++np) {
+        uint32_t bf[4];
+        const int row = kk + (lane & 7) + ((lane >> 3) & 1) * 8;
+        const int ch = ((wn * 64 + np * 16) >> 3) + (lane >> 4);
+        ldsm_x4_trans(bf, bs_base + uint32_t((row * 16 + (ch ^ (row & 7))) * 16));
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          mma_bf16(acc[mt][2 * np], af[mt], bf[0], bf[1]);
+          mma_bf16(acc[mt][2 * np + 1], af[mt], bf[2], bf[3]);
+        }
+      }
+    }
+    __syncthreads();
+  }
+  const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+      const int m = m0 + wm * 32 + mt * 16 + g, n = n0 + wn * 64 + nt * 8 + 2 * t;
+      float* o = dW + size_t(m) * H + n;
+      if (acc[mt][nt][0] != 0.f) atomicAdd(o, acc[mt][nt][0]);
+      if (acc[mt][nt][1] != 0.f) atomicAdd(o + 1, acc[mt][nt][1]);
+      if (acc[mt][nt][2] != 0.f) atomicAdd(o + size_t(8) * H, acc[mt][nt][2]);
+      if (acc[mt][nt][3] != 0.f) atomicAdd(o + size_t(8) * H + 1, acc[mt][nt][3]);
     }
 }
 
@@ -877,8 +1037,8 @@ int launch_ppo_heads(const Dims& d, const DevWeights& w, float* grad_base, const
 // forward transform of h_in; dz [N x H] and ds [2 N K] are scratch.
 int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z, const float* scores,
                          const void* h_in, const void* h_out, const float* dh_out, float* dh_in, float* dz,
-                         float* ds, const LayerWeights& lw, float* gW, float* ga_src, float* ga_dst, float* gb,
-                         int32_t N, cudaStream_t st) {
+                         float* ds, void* dz_store, const LayerWeights& lw, float* gW, float* ga_src, float* ga_dst,
+                         float* gb, int32_t N, cudaStream_t st) {
   if (N <= 0) return 0;
   const int H = d.H, K = d.K;
   cudaMemsetAsync(dz, 0, sizeof(float) * size_t(N) * H, st);
@@ -891,14 +1051,23 @@ int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* co
   const int chunk = chunk_rows(N, 2048);
   dim3 g_atb(unsigned((H + 63) / 64), unsigned((H + 63) / 64), unsigned((N + chunk - 1) / chunk));
   dim3 g_gwt(unsigned((N + 63) / 64), unsigned((H + 63) / 64));
+  // tensor-core products: about two waves of CTAs over the rows, chunks of a multiple of 32 rows, at least 512
+  const int tiles = (H / 128) * (H / 128);
+  const int want_chunks = std::max(1, 2 * kNumSMs / std::max(1, tiles));
+  const int chunk_mma = std::max(512, int(((int64_t(N) + want_chunks - 1) / want_chunks + 31) & ~int64_t(31)));
+  dim3 g_atb_mma(unsigned(H / 128), unsigned(H / 128), unsigned((N + chunk_mma - 1) / chunk_mma));
+  dim3 g_gwt_mma(unsigned((N + 127) / 128), unsigned(H / 128));
   const int NF = H / 32;
   const bool rows_kernels = (32 % K == 0) && (NF == 1 || NF == 2 || NF == 4 || NF == 8 || NF == 16);
+  // bf16 models of hidden 128, 256 or 512 take both products on the tensor cores, from a bf16 copy of dz
+  const bool mma = rows_kernels && d.dtype == XRL_BF16 && H % 128 == 0 && dz_store != nullptr;
+  bf16* dzb = mma ? static_cast<bf16*>(dz_store) : nullptr;
 #define BWD_ROWS(TY_, NF_)                                                                                     \
   do {                                                                                                         \
     k_aggregate_bwd_rows<TY_, NF_><<<grid_rows, 256, 0, st>>>(rowptr, col, zv, static_cast<const TY_*>(h_out), \
                                                               dh_out, dz, ds_src, ds_dst, gb, N, K);           \
-    k_scores_bwd_rows<TY_, NF_><<<grid_rows, 256, 0, st>>>(zv, ds_src, ds_dst, lw.a_src, lw.a_dst, dz, ga_src, \
-                                                           ga_dst, N, K);                                      \
+    k_scores_bwd_rows<TY_, NF_><<<grid_rows, 256, 0, st>>>(zv, ds_src, ds_dst, lw.a_src, lw.a_dst, dz, dzb,    \
+                                                           ga_src, ga_dst, N, K);                              \
   } while (0)
 #define BWD_BODY(TY_)                                                                                          \
   do {                                                                                                         \
@@ -921,8 +1090,13 @@ int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* co
       k_scores_bwd<TY_><<<grid_cols, 256, sizeof(float) * 2 * H, st>>>(zv, ds_src, ds_dst, lw.a_src, lw.a_dst, \
                                                                        dz, ga_src, ga_dst, N, H, K);           \
     }                                                                                                          \
-    k_atb<TY_><<<g_atb, 256, 0, st>>>(static_cast<const TY_*>(h_in), H, dz, H, gW, H, N, H, H, chunk);         \
-    k_gwt<TY_><<<g_gwt, 256, 0, st>>>(dz, static_cast<const TY_*>(lw.W), dh_in, N, H, H);                      \
+    if (mma) {                                                                                                 \
+      k_atb_mma<<<g_atb_mma, 256, 0, st>>>(static_cast<const bf16*>(h_in), dzb, gW, N, H, chunk_mma);          \
+      k_gwt_mma<<<g_gwt_mma, 256, 0, st>>>(dzb, static_cast<const bf16*>(lw.W), dh_in, N, H);                  \
+    } else {                                                                                                   \
+      k_atb<TY_><<<g_atb, 256, 0, st>>>(static_cast<const TY_*>(h_in), H, dz, H, gW, H, N, H, H, chunk);       \
+      k_gwt<TY_><<<g_gwt, 256, 0, st>>>(dz, static_cast<const TY_*>(lw.W), dh_in, N, H, H);                    \
+    }                                                                                                          \
   } while (0)
   if (d.dtype == XRL_BF16) BWD_BODY(bf16); else BWD_BODY(float);
 #undef BWD_ROWS

@@ -1007,7 +1007,7 @@ xrl_status xrl_ppo_grad(xrl_ctx* ctx, const xrl_batch* b, const float* g0, const
   const size_t h_bytes = up(sb * Nmax * H), f_bytes = up(4 * Nmax * H), ds_bytes = up(8 * Nmax * size_t(c.heads));
   const size_t heads_bytes = up(4 * ppo_heads_workspace_floats(d, c.max_graphs, c.max_envs));
   if (!ctx->bw.p) {
-    if (ctx->bw.alloc(size_t(L + 1) * h_bytes + 3 * f_bytes + ds_bytes + heads_bytes) != cudaSuccess) {
+    if (ctx->bw.alloc(size_t(L + 2) * h_bytes + 3 * f_bytes + ds_bytes + heads_bytes) != cudaSuccess) {
       cudaGetLastError();
       ctx->bw.p = nullptr;
       return XRL_ERR_ALLOC;
@@ -1018,6 +1018,7 @@ xrl_status xrl_ppo_grad(xrl_ctx* ctx, const xrl_batch* b, const float* g0, const
   char* p = ctx->bw.as<char>();
   void* hs[65];
   for (int l = 0; l <= L; ++l) { hs[l] = p; p += h_bytes; }
+  void* dz_store = p; p += h_bytes;                 // dz in the storage type, for the tensor-core products
   float* dh_a = reinterpret_cast<float*>(p); p += f_bytes;
   float* dh_b = reinterpret_cast<float*>(p); p += f_bytes;
   float* dz = reinterpret_cast<float*>(p); p += f_bytes;
@@ -1050,7 +1051,7 @@ xrl_status xrl_ppo_grad(xrl_ctx* ctx, const xrl_batch* b, const float* g0, const
     const LayerWeights& lw = ctx->dw.layer[l];
     float* ga_src = grad + (lw.a_src - wb);
     k = launch_gat_layer_bwd(d, gat_rowptr, gat_col, ctx->Z.p, ctx->scores.as<float>(), hs[l], hs[l + 1], dh_cur,
-                             dh_nxt, dz, ds, lw, ga_src - H * H, ga_src, grad + (lw.a_dst - wb),
+                             dh_nxt, dz, ds, dz_store, lw, ga_src - H * H, ga_src, grad + (lw.a_dst - wb),
                              grad + (lw.b - wb), b->N, st);
     if (k < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
     n += k;

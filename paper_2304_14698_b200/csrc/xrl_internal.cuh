@@ -208,8 +208,8 @@ int launch_ppo_heads(const Dims& d, const DevWeights& w, float* grad_base, const
                      float* ws, float* loss, float* dh, float* logp_out, int32_t* status, cudaStream_t st);
 int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* col, const void* Z, const float* scores,
                          const void* h_in, const void* h_out, const float* dh_out, float* dh_in, float* dz,
-                         float* ds, const LayerWeights& lw, float* gW, float* ga_src, float* ga_dst, float* gb,
-                         int32_t N, cudaStream_t st);
+                         float* ds, void* dz_store, const LayerWeights& lw, float* gW, float* ga_src, float* ga_dst,
+                         float* gb, int32_t N, cudaStream_t st);
 size_t embed_bwd_smem_bytes(const Dims& d);
 int launch_embed_bwd(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op, const void* shape,
                      const void* eattr, const void* h0, const float* dh0, float* gW0, float* gb0, int32_t N,
