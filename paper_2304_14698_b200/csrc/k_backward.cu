@@ -573,12 +573,14 @@ k_atb_mma(const bf16* __restrict__ A, const bf16* __restrict__ Bm, float* __rest
 }
 
 // ---- Eq. 6, reverse: dW0 += x^T dpre, db0 += dpre, x_i = [edge sum | one-hot op | own shape] -------------
-// A CTA takes a range of rows and keeps its share of W0's gradient in shared memory ([2S + T + 1] x H floats,
-// the last row for b0).  A warp takes a row at a time, a lane the columns lane, lane + 32, ...: the sixteen dense
-// entries of x meet dpre in registers (four columns per lane at a time), the one-hot entry is one shared-memory
-// add per column, and the registers are added to shared memory once per pass over the rows.
+// A CTA of 32 warps takes a range of rows and keeps its share of W0's gradient in shared memory
+// ([2S + T + 1] x H floats, the last row for b0).  A warp owns two columns per lane (lane + 32 f for two
+// consecutive f: a "slice" of 64 columns) and every n-th row of the range, n = the warps that share its slice:
+// the sixteen dense entries of x meet dpre in registers, the one-hot entry is one shared-memory add per
+// column, and the registers are added to shared memory once, at the end.
+constexpr int kEmbedBwdThreads = 1024;
 template <typename T>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kEmbedBwdThreads)
 k_embed_bwd(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col, const int32_t* __restrict__ op,
             const T* __restrict__ shape, const T* __restrict__ eattr, const T* __restrict__ h0,
             const float* __restrict__ dh0, float* __restrict__ dW0, float* __restrict__ db0, int N, int H, int Tn) {
@@ -590,8 +592,11 @@ k_embed_bwd(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
   const int rows_per_cta = (N + gridDim.x - 1) / gridDim.x;
   const int r0 = blockIdx.x * rows_per_cta, r1 = min(N, r0 + rows_per_cta);
   const int NF = H / 32;
-  constexpr int CU = 4;                            // columns per lane and pass
-  for (int f0 = 0; f0 < NF; f0 += CU) {
+  constexpr int CU = 2;                            // columns per lane
+  const int nslices = (NF + CU - 1) / CU, ngroups = max(1, nw / nslices);
+  const int slice = warp % nslices, group = warp / nslices;
+  if (group < ngroups) {                           // (warps beyond nslices x ngroups have nothing to do)
+    const int f0 = slice * CU;
     float a[2 * kS][CU], dbr[CU];
 #pragma unroll
     for (int u = 0; u < CU; ++u) {
@@ -599,7 +604,7 @@ k_embed_bwd(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
 #pragma unroll
       for (int s = 0; s < 2 * kS; ++s) a[s][u] = 0.f;
     }
-    for (int i = r0 + warp; i < r1; i += nw) {
+    for (int i = r0 + group; i < r1; i += ngroups) {
       float dp[CU];
       bool live = false;
 #pragma unroll
@@ -1112,20 +1117,20 @@ int launch_embed_bwd(const Dims& d, const int32_t* rowptr, const int32_t* col, c
                      cudaStream_t st) {
   if (N <= 0) return 0;
   const size_t smem = embed_bwd_smem_bytes(d);
-  const int grid = int(std::min<int64_t>((int64_t(N) + 63) / 64, int64_t(kNumSMs)));
+  const int grid = int(std::min<int64_t>((int64_t(N) + 255) / 256, int64_t(kNumSMs)));
   // the opt-in is the kernel's ceiling for every later launch: ask for all an SM has, once per device
   constexpr int kSmemCeiling = 227 * 1024;
   if (smem > size_t(kSmemCeiling)) return -1;
   if (d.dtype == XRL_BF16) {
     static bool attr[64] = {};
     if (!ensure_dynamic_smem(k_embed_bwd<bf16>, kSmemCeiling, attr)) return -1;
-    k_embed_bwd<bf16><<<grid, 256, smem, st>>>(rowptr, col, op, static_cast<const bf16*>(shape),
+    k_embed_bwd<bf16><<<grid, kEmbedBwdThreads, smem, st>>>(rowptr, col, op, static_cast<const bf16*>(shape),
                                                static_cast<const bf16*>(eattr), static_cast<const bf16*>(h0), dh0,
                                                gW0, gb0, N, d.H, d.T);
   } else {
     static bool attr[64] = {};
     if (!ensure_dynamic_smem(k_embed_bwd<float>, kSmemCeiling, attr)) return -1;
-    k_embed_bwd<float><<<grid, 256, smem, st>>>(rowptr, col, op, static_cast<const float*>(shape),
+    k_embed_bwd<float><<<grid, kEmbedBwdThreads, smem, st>>>(rowptr, col, op, static_cast<const float*>(shape),
                                                 static_cast<const float*>(eattr), static_cast<const float*>(h0), dh0,
                                                 gW0, gb0, N, d.H, d.T);
   }
