@@ -225,60 +225,81 @@ k_aggregate_bwd_rows(const int32_t* __restrict__ rowptr, const int32_t* __restri
     if (!__any_sync(0xFFFFFFFFu, live)) continue;     // a row whose units are all off: nothing flows (ds is zeroed)
     const int32_t e0 = rowptr[i], deg = rowptr[i + 1] - e0;
     const float sd = zv.pair(i, k).y;
-    // softmax statistics of this lane's head over the row's neighbours and the row itself (entry `deg`)
-    float mx = -INFINITY, sum = 0.f;
+    // One sweep over the row's neighbours and the row itself (entry `deg`) takes, per head, the score e_t, the
+    // product dal_t = dpre . z_t, and with a running maximum the sums  sum_t 2^(e_t - mx)  and
+    // sum_t 2^(e_t - mx) dal_t; the first kCache entries keep (e_t, dal_t) in registers for the second sweep,
+    // which turns them into d e_t and the scattered sums (later entries are read and multiplied again).
+    constexpr int kCache = 4;
+    float ce[kCache], cd[kCache];
+    float mx = -INFINITY, sum = 0.f, dotu = 0.f;
+    auto score_and_product = [&](int32_t j, float& eraw, float& dal) {
+      float z[NF];
+      load_chunk<T, NF>(zv.row(j) + lane * NF, z);
+      float part = 0.f;
+#pragma unroll
+      for (int f = 0; f < NF; ++f) part = fmaf(dp[f], z[f], part);
+      for (int o = lph >> 1; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+      dal = part;
+      eraw = zv.pair(j, k).x + sd;
+    };
+    auto accumulate = [&](float eraw, float dal) {
+      const float e = lrelu(eraw);
+      if (e > mx) {
+        const float sc = exp2f(mx - e);
+        sum = fmaf(sum, sc, 1.f); dotu = fmaf(dotu, sc, dal); mx = e;
+      } else {
+        const float w = exp2f(e - mx);
+        sum += w; dotu = fmaf(w, dal, dotu);
+      }
+    };
+    const int32_t c0 = lane < deg ? col[e0 + lane] : i;      // the first 32 entries (the row itself after the last)
+#pragma unroll
+    for (int t = 0; t < kCache; ++t) {
+      ce[t] = 0.f; cd[t] = 0.f;
+      if (t <= deg) {
+        const int32_t j = __shfl_sync(0xFFFFFFFFu, c0, t);
+        score_and_product(j, ce[t], cd[t]);
+        accumulate(ce[t], cd[t]);
+      }
+    }
     for (int base = 0; base <= deg; base += 32) {
       const int idx = base + lane;
-      const int32_t cj = idx < deg ? col[e0 + idx] : i;
+      const int32_t cj = base == 0 ? c0 : (idx < deg ? col[e0 + idx] : i);
       const int cnt = min(32, deg + 1 - base);
-      for (int t = 0; t < cnt; ++t) {
+      for (int t = (base == 0 ? kCache : 0); t < cnt; ++t) {
         const int32_t j = __shfl_sync(0xFFFFFFFFu, cj, t);
-        const float e = lrelu(zv.pair(j, k).x + sd);
-        if (e > mx) { sum = sum * exp2f(mx - e) + 1.f; mx = e; } else { sum += exp2f(e - mx); }
+        float eraw, dal;
+        score_and_product(j, eraw, dal);
+        accumulate(eraw, dal);
       }
     }
     const float inv = 1.f / sum;
-    float dot = 0.f;
-    for (int base = 0; base <= deg; base += 32) {
-      const int idx = base + lane;
-      const int32_t cj = idx < deg ? col[e0 + idx] : i;
-      const int cnt = min(32, deg + 1 - base);
-      for (int t = 0; t < cnt; ++t) {
-        const int32_t j = __shfl_sync(0xFFFFFFFFu, cj, t);
-        float z[NF];
-        load_chunk<T, NF>(zv.row(j) + lane * NF, z);
-        float part = 0.f;
-#pragma unroll
-        for (int f = 0; f < NF; ++f) part = fmaf(dp[f], z[f], part);
-        for (int o = lph >> 1; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
-        const float al = exp2f(lrelu(zv.pair(j, k).x + sd) - mx) * inv;
-        dot = fmaf(al, part, dot);
-      }
-    }
+    const float dot = dotu * inv;
     float dsd = 0.f;
+    auto scatter = [&](int32_t j, float eraw, float dal) {
+      const float al = exp2f(lrelu(eraw) - mx) * inv;
+      const float de = al * (dal - dot) * (eraw > 0.f ? 1.f : 0.2f);
+      dsd += de;
+      if (leader && de != 0.f) atomicAdd(&ds_src[size_t(j) * K + k], de);
+      if (live) {
+        float v[NF];
+#pragma unroll
+        for (int f = 0; f < NF; ++f) v[f] = al * dp[f];
+        atomic_add_chunk<NF>(dz + size_t(j) * H + lane * NF, v);
+      }
+    };
+#pragma unroll
+    for (int t = 0; t < kCache; ++t)
+      if (t <= deg) scatter(__shfl_sync(0xFFFFFFFFu, c0, t), ce[t], cd[t]);
     for (int base = 0; base <= deg; base += 32) {
       const int idx = base + lane;
-      const int32_t cj = idx < deg ? col[e0 + idx] : i;
+      const int32_t cj = base == 0 ? c0 : (idx < deg ? col[e0 + idx] : i);
       const int cnt = min(32, deg + 1 - base);
-      for (int t = 0; t < cnt; ++t) {
+      for (int t = (base == 0 ? kCache : 0); t < cnt; ++t) {
         const int32_t j = __shfl_sync(0xFFFFFFFFu, cj, t);
-        float z[NF];
-        load_chunk<T, NF>(zv.row(j) + lane * NF, z);
-        float part = 0.f;
-#pragma unroll
-        for (int f = 0; f < NF; ++f) part = fmaf(dp[f], z[f], part);
-        for (int o = lph >> 1; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
-        const float e = zv.pair(j, k).x + sd;
-        const float al = exp2f(lrelu(e) - mx) * inv;
-        const float de = al * (part - dot) * (e > 0.f ? 1.f : 0.2f);
-        dsd += de;
-        if (leader && de != 0.f) atomicAdd(&ds_src[size_t(j) * K + k], de);
-        if (live) {
-          float v[NF];
-#pragma unroll
-          for (int f = 0; f < NF; ++f) v[f] = al * dp[f];
-          atomic_add_chunk<NF>(dz + size_t(j) * H + lane * NF, v);
-        }
+        float eraw, dal;
+        score_and_product(j, eraw, dal);
+        scatter(j, eraw, dal);
       }
     }
     if (leader) ds_dst[size_t(i) * K + k] = dsd;
@@ -907,12 +928,14 @@ k_graph_bwd(const float* __restrict__ emb, const float* __restrict__ dlogit, Mlp
   }
 }
 
-// the readout is a plain sum: every node receives its graph's gradient
+// the readout is a plain sum: every node receives its graph's gradient (four columns per thread; H % 4 == 0)
 __global__ void k_readout_bwd(const float* __restrict__ dr, const int32_t* __restrict__ seg_id,
-                              float* __restrict__ dh, int64_t n_elems, int H) {
-  for (int64_t t = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; t < n_elems; t += int64_t(gridDim.x) * blockDim.x) {
-    const int64_t i = t / H;
-    dh[t] = dr[size_t(seg_id[i]) * H + (t - i * H)];
+                              float* __restrict__ dh, int64_t n_quads, int H) {
+  const int q = H >> 2;
+  for (int64_t t = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; t < n_quads; t += int64_t(gridDim.x) * blockDim.x) {
+    const int64_t i = t / q;
+    const int c = int(t - i * q);
+    reinterpret_cast<float4*>(dh)[t] = reinterpret_cast<const float4*>(dr + size_t(seg_id[i]) * H)[c];
   }
 }
 
@@ -968,9 +991,12 @@ int mlp_weight_grads(const float* X, int in, int rows, int hid, int hid2, const 
 }  // namespace
 
 // ---- launchers ------------------------------------------------------------------------------------------
+// every piece of the heads' workspace starts on a 16-byte boundary (some are read as float4)
+static size_t up4(size_t n) { return (n + 3) & ~size_t(3); }
 size_t ppo_heads_workspace_floats(const Dims& d, int64_t B, int64_t num_envs) {
-  const size_t H = d.H, Hm = d.Hm, Hm2 = d.Hm2;
-  return size_t(B) * ((H + d.Dg) + 4 * H + 2 + 2 * Hm + 2 * Hm2) + size_t(num_envs) * (2 * H + 2 * Hm + 2 * Hm2 + 1);
+  const size_t H = d.H, Hm = d.Hm, Hm2 = d.Hm2, b = size_t(B), e = size_t(num_envs);
+  return up4(b * (H + d.Dg)) + 4 * up4(b * H) + 2 * up4(b) + 2 * up4(b * Hm) + 2 * up4(b * Hm2) +
+         up4(e * 2 * H) + 2 * up4(e * Hm) + 2 * up4(e * Hm2) + up4(e);
 }
 
 // Forward from the saved last-layer features to the logits, Eq. 3-5, and the reverse pass down to the gradient
@@ -983,7 +1009,7 @@ int launch_ppo_heads(const Dims& d, const DevWeights& w, float* grad_base, const
   if (B <= 0 || num_envs <= 0) return 0;
   const size_t H = d.H, Hm = d.Hm, Hm2 = d.Hm2, HU = H + d.Dg;
   float* p = ws;
-  auto take = [&](size_t n) { float* q = p; p += n; return q; };
+  auto take = [&](size_t n) { float* q = p; p += up4(n); return q; };
   float* U = take(size_t(B) * HU);
   float* emb = take(size_t(B) * H);
   float* demb = take(size_t(B) * H);
@@ -1029,7 +1055,7 @@ int launch_ppo_heads(const Dims& d, const DevWeights& w, float* grad_base, const
                         gp(w.pbh), gp(w.pw2), gp(w.pb2), st);
   n += mlp_weight_grads(eb.vu, 2 * d.H, num_envs, d.Hm, d.Hm2, eb.vy1, eb.vy2, eb.vd1, eb.vd2, eb.vdout, gp(w.vW1),
                         gp(w.vb1), gp(w.vWh), gp(w.vbh), gp(w.vw2), gp(w.vb2), st);
-  const int64_t ne = N * d.H;
+  const int64_t ne = N * (d.H / 4);
   if (ne > 0) {
     const unsigned grid = unsigned(std::min<int64_t>((ne + 255) / 256, int64_t(kNumSMs) * 64));
     k_readout_bwd<<<grid, 256, 0, st>>>(dr, seg_id, dh, ne, d.H);
