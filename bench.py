@@ -195,6 +195,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-delta", action="store_true")
+    ap.add_argument("--train-step", action="store_true",
+                    help="also time the training step's gradient (Section 3.3.4) on the same batch")
     args = ap.parse_args()
     cfg_id = args.config
     rank, local_rank, world = rank_info()
@@ -319,6 +321,35 @@ def main():
         delta = {"ms_per_step": dms, "rows_per_layer": xrl.xrl_delta_rows(agent.ctx, m["L"]),
                  "kernel_ms_per_step": {f: round(v["ms"] / args.steps, 4) for f, v in dprof.items()}}
 
+    # ---- the training step's gradient on the same packed batch (opt-in: it allocates its own workspace) ------
+    train = None
+    if args.train_step:
+        ne_t = Ne
+        act_d = torch.full((ne_t,), m["A_max"], dtype=torch.int32, device="cuda")     # No-Op: always valid
+        lp_d = torch.full((ne_t,), -1.0, device="cuda")
+        adv_d = torch.ones(ne_t, device="cuda")
+        ret_d = torch.zeros(ne_t, device="cuda")
+        loss_d = torch.empty(4, device="cuda")
+        grad_d = torch.empty(configs.weight_count(m), device="cuda")
+
+        def grad_step():
+            xrl.xrl_ppo_grad(agent.ctx, agent.batch, mask_d, act_d, lp_d, adv_d, ret_d, loss_d, grad_d)
+
+        for _ in range(3):
+            grad_step()
+        torch.cuda.synchronize()
+        barrier()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for _ in range(args.steps):
+            grad_step()
+        t1.record(stream)
+        barrier()
+        assert agent.device_status() == 0
+        tms = t0.elapsed_time(t1) / args.steps
+        train = {"ms_per_step": tms, "unit": "graphs/s",
+                 "note": "xrl_ppo_grad: forward with kept activations, Eq. 3-5, reverse pass to every weight"}
+
     # ---- end to end: host buffers in, results out, through the public call ---------------------------
     e2e = None
     if not args.no_e2e:
@@ -417,6 +448,9 @@ def main():
         delta["unit"] = "graphs/s"
         delta["note"] = "xrl_encode_delta: same outputs, candidates reuse the current graph's unchanged rows"
         line["delta"] = delta
+    if train:
+        train["value"] = tot_graphs / (train["ms_per_step"] * 1e-3)
+        line["train_step"] = train
     if cpu:
         line["cpu_baseline"] = cpu
     if parity:

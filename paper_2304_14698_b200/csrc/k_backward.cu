@@ -232,15 +232,17 @@ k_aggregate_bwd_rows(const int32_t* __restrict__ rowptr, const int32_t* __restri
     constexpr int kCache = 4;
     float ce[kCache], cd[kCache];
     float mx = -INFINITY, sum = 0.f, dotu = 0.f;
-    auto score_and_product = [&](int32_t j, float& eraw, float& dal) {
-      float z[NF];
-      load_chunk<T, NF>(zv.row(j) + lane * NF, z);
+    auto product = [&](const Chunk<T, NF>& zc, float& dal) {
       float part = 0.f;
 #pragma unroll
-      for (int f = 0; f < NF; ++f) part = fmaf(dp[f], z[f], part);
+      for (int f = 0; f < NF; ++f) part = fmaf(dp[f], to_float(zc.v[f]), part);
       for (int o = lph >> 1; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
       dal = part;
+    };
+    auto score_and_product = [&](int32_t j, float& eraw, float& dal) {
+      const Chunk<T, NF> zc = *reinterpret_cast<const Chunk<T, NF>*>(zv.row(j) + lane * NF);
       eraw = zv.pair(j, k).x + sd;
+      product(zc, dal);
     };
     auto accumulate = [&](float eraw, float dal) {
       const float e = lrelu(eraw);
@@ -253,13 +255,23 @@ k_aggregate_bwd_rows(const int32_t* __restrict__ rowptr, const int32_t* __restri
       }
     };
     const int32_t c0 = lane < deg ? col[e0 + lane] : i;      // the first 32 entries (the row itself after the last)
+    {
+      // the first kCache rows are fetched together (entries past the last one repeat it: always a valid row)
+      Chunk<T, NF> zc[kCache];
 #pragma unroll
-    for (int t = 0; t < kCache; ++t) {
-      ce[t] = 0.f; cd[t] = 0.f;
-      if (t <= deg) {
-        const int32_t j = __shfl_sync(0xFFFFFFFFu, c0, t);
-        score_and_product(j, ce[t], cd[t]);
-        accumulate(ce[t], cd[t]);
+      for (int t = 0; t < kCache; ++t) {
+        const int32_t j = __shfl_sync(0xFFFFFFFFu, c0, min(t, deg));
+        zc[t] = *reinterpret_cast<const Chunk<T, NF>*>(zv.row(j) + lane * NF);
+        ce[t] = zv.pair(j, k).x;
+      }
+#pragma unroll
+      for (int t = 0; t < kCache; ++t) {
+        ce[t] += sd;
+        cd[t] = 0.f;
+        if (t <= deg) {
+          product(zc[t], cd[t]);
+          accumulate(ce[t], cd[t]);
+        }
       }
     }
     for (int base = 0; base <= deg; base += 32) {
@@ -459,7 +471,7 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
 }
 
 // out [rows x H] fp32 = G [rows x H] bf16 times W^T, W [H x H] bf16 row-major [in x out]: out[r][k] = sum_n G[r][n] W[k][n]
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 k_gwt_mma(const bf16* __restrict__ G, const bf16* __restrict__ W, float* __restrict__ out, int rows, int H) {
   __shared__ __align__(128) bf16 As[128 * 64];      // [row r][64 n], 8 pieces of 16 bytes per row
   __shared__ __align__(128) bf16 Bs[128 * 64];      // [row k][64 n]
@@ -474,18 +486,28 @@ k_gwt_mma(const bf16* __restrict__ G, const bf16* __restrict__ W, float* __restr
 #pragma unroll
       for (int c = 0; c < 4; ++c) acc[a][b][c] = 0.f;
   const uint32_t as_base = uint32_t(__cvta_generic_to_shared(As)), bs_base = uint32_t(__cvta_generic_to_shared(Bs));
+  // the next tile's pieces travel from global memory to registers while the current tile is multiplied
+  uint4 va[4], vb[4];
+  auto fetch = [&](int n0) {
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+      const int idx = tid + 256 * it, row = idx >> 3, ch = idx & 7;
+      va[it] = make_uint4(0, 0, 0, 0);
+      if (r0 + row < rows) va[it] = *reinterpret_cast<const uint4*>(G + size_t(r0 + row) * H + n0 + ch * 8);
+      vb[it] = *reinterpret_cast<const uint4*>(W + size_t(k0 + row) * H + n0 + ch * 8);
+    }
+  };
+  fetch(0);
   for (int n0 = 0; n0 < H; n0 += 64) {
 #pragma unroll
     for (int it = 0; it < 4; ++it) {
       const int idx = tid + 256 * it, row = idx >> 3, ch = idx & 7;
-      uint4 va = make_uint4(0, 0, 0, 0);
-      if (r0 + row < rows) va = *reinterpret_cast<const uint4*>(G + size_t(r0 + row) * H + n0 + ch * 8);
-      const uint4 vb = *reinterpret_cast<const uint4*>(W + size_t(k0 + row) * H + n0 + ch * 8);
       const int phys = (row * 8 + (ch ^ (row & 7))) * 8;
-      *reinterpret_cast<uint4*>(As + phys) = va;
-      *reinterpret_cast<uint4*>(Bs + phys) = vb;
+      *reinterpret_cast<uint4*>(As + phys) = va[it];
+      *reinterpret_cast<uint4*>(Bs + phys) = vb[it];
     }
     __syncthreads();
+    if (n0 + 64 < H) fetch(n0 + 64);
 #pragma unroll
     for (int kk = 0; kk < 64; kk += 16) {
       uint32_t af[2][4];
@@ -523,7 +545,7 @@ k_gwt_mma(const bf16* __restrict__ G, const bf16* __restrict__ W, float* __restr
 }
 
 // dW [H x H] fp32 += A^T B over the rows [chunk z], A = h_in [rows x H] bf16, B = dz [rows x H] bf16
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 k_atb_mma(const bf16* __restrict__ A, const bf16* __restrict__ Bm, float* __restrict__ dW, int rows, int H,
           int rows_per_chunk) {
   __shared__ __align__(128) bf16 As[32 * 128];      // [row r][128 m], 16 pieces of 16 bytes per row
@@ -540,20 +562,29 @@ k_atb_mma(const bf16* __restrict__ A, const bf16* __restrict__ Bm, float* __rest
 #pragma unroll
       for (int c = 0; c < 4; ++c) acc[a][b][c] = 0.f;
   const uint32_t as_base = uint32_t(__cvta_generic_to_shared(As)), bs_base = uint32_t(__cvta_generic_to_shared(Bs));
+  uint4 va[2], vb[2];
+  auto fetch = [&](int rr) {
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+      const int idx = tid + 256 * it, row = idx >> 4, ch = idx & 15;
+      va[it] = make_uint4(0, 0, 0, 0); vb[it] = make_uint4(0, 0, 0, 0);
+      if (rr + row < r_end) {
+        va[it] = *reinterpret_cast<const uint4*>(A + size_t(rr + row) * H + m0 + ch * 8);
+        vb[it] = *reinterpret_cast<const uint4*>(Bm + size_t(rr + row) * H + n0 + ch * 8);
+      }
+    }
+  };
+  if (r_begin < r_end) fetch(r_begin);
   for (int rr = r_begin; rr < r_end; rr += 32) {
 #pragma unroll
     for (int it = 0; it < 2; ++it) {
       const int idx = tid + 256 * it, row = idx >> 4, ch = idx & 15;
-      uint4 va = make_uint4(0, 0, 0, 0), vb = make_uint4(0, 0, 0, 0);
-      if (rr + row < r_end) {
-        va = *reinterpret_cast<const uint4*>(A + size_t(rr + row) * H + m0 + ch * 8);
-        vb = *reinterpret_cast<const uint4*>(Bm + size_t(rr + row) * H + n0 + ch * 8);
-      }
       const int phys = (row * 16 + (ch ^ (row & 7))) * 8;
-      *reinterpret_cast<uint4*>(As + phys) = va;
-      *reinterpret_cast<uint4*>(Bs + phys) = vb;
+      *reinterpret_cast<uint4*>(As + phys) = va[it];
+      *reinterpret_cast<uint4*>(Bs + phys) = vb[it];
     }
     __syncthreads();
+    if (rr + 32 < r_end) fetch(rr + 32);
 #pragma unroll
     for (int kk = 0; kk < 32; kk += 16) {
       uint32_t af[2][4];
