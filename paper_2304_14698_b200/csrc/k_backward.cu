@@ -624,17 +624,36 @@ k_atb_mma(const bf16* __restrict__ A, const bf16* __restrict__ Bm, float* __rest
     }
 }
 
+// the sixteen dense entries of Eq. 6's input, one thread per node: [sum of the edge attributes | own shape]
+template <typename T>
+__global__ void __launch_bounds__(256)
+k_embed_inputs(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col, const T* __restrict__ shape,
+               const T* __restrict__ eattr, float* __restrict__ xs, int N) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= N) return;
+  float x[2 * kS];
+#pragma unroll
+  for (int s = 0; s < kS; ++s) x[s] = 0.f;
+  for (int32_t e = rowptr[i]; e < rowptr[i + 1]; ++e) {
+    float v[kS];
+    load_chunk<T, kS>(eattr ? eattr + size_t(e) * kS : shape + size_t(col[e]) * kS, v);
+#pragma unroll
+    for (int s = 0; s < kS; ++s) x[s] += v[s];
+  }
+  load_chunk<T, kS>(shape + size_t(i) * kS, reinterpret_cast<float(&)[kS]>(x[kS]));
+  store_chunk<2 * kS>(xs + size_t(i) * 2 * kS, x);
+}
+
 // ---- Eq. 6, reverse: dW0 += x^T dpre, db0 += dpre, x_i = [edge sum | one-hot op | own shape] -------------
 // A CTA of 32 warps takes a range of rows and keeps its share of W0's gradient in shared memory
 // ([2S + T + 1] x H floats, the last row for b0).  A warp owns two columns per lane (lane + 32 f for two
 // consecutive f: a "slice" of 64 columns) and every n-th row of the range, n = the warps that share its slice:
-// the sixteen dense entries of x meet dpre in registers, the one-hot entry is one shared-memory add per
+// the sixteen dense entries of x (computed beforehand by k_embed_inputs) meet dpre in registers, the one-hot entry is one shared-memory add per
 // column, and the registers are added to shared memory once, at the end.
 constexpr int kEmbedBwdThreads = 1024;
 template <typename T>
 __global__ void __launch_bounds__(kEmbedBwdThreads)
-k_embed_bwd(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col, const int32_t* __restrict__ op,
-            const T* __restrict__ shape, const T* __restrict__ eattr, const T* __restrict__ h0,
+k_embed_bwd(const float* __restrict__ xs, const int32_t* __restrict__ op, const T* __restrict__ h0,
             const float* __restrict__ dh0, float* __restrict__ dW0, float* __restrict__ db0, int N, int H, int Tn) {
   extern __shared__ float acc[];                   // [(2S + T + 1) x H]: dW0 rows, then db0
   const int F0 = 2 * kS + Tn;
@@ -667,15 +686,7 @@ k_embed_bwd(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
       }
       if (!__any_sync(0xFFFFFFFFu, live)) continue;
       float x[2 * kS];
-#pragma unroll
-      for (int s = 0; s < 2 * kS; ++s) x[s] = 0.f;
-      for (int32_t e = rowptr[i]; e < rowptr[i + 1]; ++e) {
-        float v[kS];
-        load_chunk<T, kS>(eattr ? eattr + size_t(e) * kS : shape + size_t(col[e]) * kS, v);
-#pragma unroll
-        for (int s = 0; s < kS; ++s) x[s] += v[s];
-      }
-      load_chunk<T, kS>(shape + size_t(i) * kS, reinterpret_cast<float(&)[kS]>(x[kS]));
+      load_chunk<float, 2 * kS>(xs + size_t(i) * 2 * kS, x);      // the same 64 bytes for every lane
       const int o = op[i];
 #pragma unroll
       for (int u = 0; u < CU; ++u) {
@@ -1170,28 +1181,31 @@ int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* co
 size_t embed_bwd_smem_bytes(const Dims& d) { return sizeof(float) * size_t(2 * kS + d.T + 1) * d.H; }
 
 int launch_embed_bwd(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op, const void* shape,
-                     const void* eattr, const void* h0, const float* dh0, float* gW0, float* gb0, int32_t N,
+                     const void* eattr, const void* h0, const float* dh0, float* xs, float* gW0, float* gb0, int32_t N,
                      cudaStream_t st) {
   if (N <= 0) return 0;
   const size_t smem = embed_bwd_smem_bytes(d);
   const int grid = int(std::min<int64_t>((int64_t(N) + 255) / 256, int64_t(kNumSMs)));
+  const unsigned grid_x = unsigned((int64_t(N) + 255) / 256);
   // the opt-in is the kernel's ceiling for every later launch: ask for all an SM has, once per device
   constexpr int kSmemCeiling = 227 * 1024;
   if (smem > size_t(kSmemCeiling)) return -1;
   if (d.dtype == XRL_BF16) {
     static bool attr[64] = {};
     if (!ensure_dynamic_smem(k_embed_bwd<bf16>, kSmemCeiling, attr)) return -1;
-    k_embed_bwd<bf16><<<grid, kEmbedBwdThreads, smem, st>>>(rowptr, col, op, static_cast<const bf16*>(shape),
-                                               static_cast<const bf16*>(eattr), static_cast<const bf16*>(h0), dh0,
-                                               gW0, gb0, N, d.H, d.T);
+    k_embed_inputs<bf16><<<grid_x, 256, 0, st>>>(rowptr, col, static_cast<const bf16*>(shape),
+                                                 static_cast<const bf16*>(eattr), xs, N);
+    k_embed_bwd<bf16><<<grid, kEmbedBwdThreads, smem, st>>>(xs, op, static_cast<const bf16*>(h0), dh0, gW0, gb0, N,
+                                                            d.H, d.T);
   } else {
     static bool attr[64] = {};
     if (!ensure_dynamic_smem(k_embed_bwd<float>, kSmemCeiling, attr)) return -1;
-    k_embed_bwd<float><<<grid, kEmbedBwdThreads, smem, st>>>(rowptr, col, op, static_cast<const float*>(shape),
-                                                static_cast<const float*>(eattr), static_cast<const float*>(h0), dh0,
-                                                gW0, gb0, N, d.H, d.T);
+    k_embed_inputs<float><<<grid_x, 256, 0, st>>>(rowptr, col, static_cast<const float*>(shape),
+                                                  static_cast<const float*>(eattr), xs, N);
+    k_embed_bwd<float><<<grid, kEmbedBwdThreads, smem, st>>>(xs, op, static_cast<const float*>(h0), dh0, gW0, gb0, N,
+                                                             d.H, d.T);
   }
-  return 1;
+  return 2;
 }
 
 }  // namespace xrl

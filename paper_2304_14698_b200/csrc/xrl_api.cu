@@ -1058,7 +1058,7 @@ xrl_status xrl_ppo_grad(xrl_ctx* ctx, const xrl_batch* b, const float* g0, const
     std::swap(dh_cur, dh_nxt);
   }
   const int k = launch_embed_bwd(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), b->op.as<int32_t>(), b->shape.p,
-                                 b->has_eattr ? b->eattr.p : nullptr, hs[0], dh_cur, grad,
+                                 b->has_eattr ? b->eattr.p : nullptr, hs[0], dh_cur, dz, grad,
                                  grad + (ctx->dw.b0 - wb), b->N, st);
   if (k < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
   n += k;
