@@ -738,6 +738,7 @@ __device__ float block_sum_f(float v, float* scratch) {       // blockDim a powe
 __device__ float mlp_fwd(const float* x, int in, const MlpW& m, float* y1, float* y2, float* scratch) {
   for (int c = threadIdx.x; c < m.hid; c += blockDim.x) {
     float acc = m.b1[c];
+#pragma unroll 16
     for (int k = 0; k < in; ++k) acc = fmaf(x[k], m.W1[size_t(k) * m.hid + c], acc);
     y1[c] = fmaxf(acc, 0.f);
   }
@@ -748,6 +749,7 @@ __device__ float mlp_fwd(const float* x, int in, const MlpW& m, float* y1, float
   } else {
     for (int c = threadIdx.x; c < m.hid2; c += blockDim.x) {
       float acc = m.bh[c];
+#pragma unroll 16
       for (int k = 0; k < m.hid; ++k) acc = fmaf(y1[k], m.Wh[size_t(k) * m.hid2 + c], acc);
       y2[c] = fmaxf(acc, 0.f);
       contrib += y2[c] * m.w2[c];
@@ -816,6 +818,7 @@ k_graph_fwd(const float* __restrict__ U, const float* __restrict__ Wg, const flo
   __syncthreads();
   for (int c = tid; c < H; c += nt) {
     float acc = bg[c];
+#pragma unroll 16
     for (int k = 0; k < H + Dg; ++k) acc = fmaf(uu[k], Wg[size_t(k) * H + c], acc);
     x[c] = fmaxf(acc, 0.f);
     emb[size_t(g) * H + c] = x[c];
