@@ -271,7 +271,8 @@ xrl_status xrl_sample(xrl_ctx* ctx, const float* probs, int32_t num_envs, int32_
  * The first call allocates the workspace for the context's capacities ((L + 2) copies of the node features
  * plus three fp32 ones) and therefore synchronises; later calls only enqueue.  Not recordable
  * (XRL_ERR_STATE between xrl_graph_begin and xrl_graph_launch).  XRL_ERR_UNSUPPORTED when
- * (2 S + T + 1) x H floats exceed one SM's shared memory (227 KB): W0's gradient is collected there.
+ * (T + 8) x H floats exceed one SM's shared memory (227 KB): the operator block of W0's gradient and a tile
+ * of eight rows are kept there.
  * Errors: INVALID_ARG, STATE, UNSUPPORTED, ALLOC, CUDA. */
 xrl_status xrl_ppo_grad(xrl_ctx* ctx, const xrl_batch* batch, const float* g0, const uint8_t* mask,
                         const int32_t* action, const float* logp_old, const float* adv, const float* ret,

@@ -645,75 +645,97 @@ k_embed_inputs(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ c
 }
 
 // ---- Eq. 6, reverse: dW0 += x^T dpre, db0 += dpre, x_i = [edge sum | one-hot op | own shape] -------------
-// A CTA of 32 warps takes a range of rows and keeps its share of W0's gradient in shared memory
-// ([2S + T + 1] x H floats, the last row for b0).  A warp owns two columns per lane (lane + 32 f for two
-// consecutive f: a "slice" of 64 columns) and every n-th row of the range, n = the warps that share its slice:
-// the sixteen dense entries of x (computed beforehand by k_embed_inputs) meet dpre in registers, the one-hot entry is one shared-memory add per
-// column, and the registers are added to shared memory once, at the end.
-constexpr int kEmbedBwdThreads = 1024;
+// A CTA takes a range of rows, R at a time: the tile's masked gradients dpre [R x H], its dense inputs
+// [R x 16] (computed beforehand by k_embed_inputs) and its operator ids come into shared memory with wide
+// coalesced loads, eight requested per thread before the first is used; then a thread owns one column and
+// every P-th row of the tile (P threads share a column): the sixteen dense products accumulate in its
+// registers, the one-hot block in the P-th of P shared-memory copies [T x H] of that part of dW0 (a plain add
+// per row and column: nobody else touches that copy's column; shared-memory atomics cost far more here than
+// the adds themselves).  Registers and the copies go to global memory once per CTA.
+constexpr int kEmbedBwdThreads = 512;
 template <typename T>
 __global__ void __launch_bounds__(kEmbedBwdThreads)
 k_embed_bwd(const float* __restrict__ xs, const int32_t* __restrict__ op, const T* __restrict__ h0,
-            const float* __restrict__ dh0, float* __restrict__ dW0, float* __restrict__ db0, int N, int H, int Tn) {
-  extern __shared__ float acc[];                   // [(2S + T + 1) x H]: dW0 rows, then db0
-  const int F0 = 2 * kS + Tn;
-  for (int t = threadIdx.x; t < (F0 + 1) * H; t += blockDim.x) acc[t] = 0.f;
-  __syncthreads();
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+            const float* __restrict__ dh0, float* __restrict__ dW0, float* __restrict__ db0, int N, int H, int Tn,
+            int R, int P) {
+  extern __shared__ float sm_embed[];
+  float* oh = sm_embed;                            // [P][Tn x H]
+  float* dpt = oh + size_t(P) * Tn * H;            // [R x H]
+  float* xt = dpt + size_t(R) * H;                 // [R x 16]
+  int32_t* opt = reinterpret_cast<int32_t*>(xt + size_t(R) * 2 * kS);   // [R]
+  const int tid = threadIdx.x, nt = blockDim.x;
+  for (int t = tid; t < P * Tn * H; t += nt) oh[t] = 0.f;
+  const int part = tid / H, c = tid - part * H;    // threads beyond P x H only help with the loads
+  float* my_oh = oh + size_t(min(part, P - 1)) * Tn * H;
   const int rows_per_cta = (N + gridDim.x - 1) / gridDim.x;
   const int r0 = blockIdx.x * rows_per_cta, r1 = min(N, r0 + rows_per_cta);
-  const int NF = H / 32;
-  constexpr int CU = 2;                            // columns per lane
-  const int nslices = (NF + CU - 1) / CU, ngroups = max(1, nw / nslices);
-  const int slice = warp % nslices, group = warp / nslices;
-  if (group < ngroups) {                           // (warps beyond nslices x ngroups have nothing to do)
-    const int f0 = slice * CU;
-    float a[2 * kS][CU], dbr[CU];
+  const int qpr = H >> 2;                          // 16-byte pieces per row
+  const int step_r = nt / qpr, step_q = nt - step_r * qpr;   // what a stride of nt pieces does to (row, piece)
+  float acc[2 * kS], dbr = 0.f;
 #pragma unroll
-    for (int u = 0; u < CU; ++u) {
-      dbr[u] = 0.f;
+  for (int s = 0; s < 2 * kS; ++s) acc[s] = 0.f;
+  for (int t0 = r0; t0 < r1; t0 += R) {
+    const int rows = min(R, r1 - t0);
+    __syncthreads();                               // the previous tile has been consumed (and oh is zeroed)
+    constexpr int kBatch = 8;
+    int r = tid / qpr, q = tid - r * qpr;
+    while (r < rows) {
+      float4 g[kBatch];
+      Chunk<T, 4> hc[kBatch];
+      int rr[kBatch], qq[kBatch];
 #pragma unroll
-      for (int s = 0; s < 2 * kS; ++s) a[s][u] = 0.f;
+      for (int u = 0; u < kBatch; ++u) {
+        rr[u] = r; qq[u] = q;
+        if (r < rows) {
+          g[u] = *reinterpret_cast<const float4*>(dh0 + size_t(t0 + r) * H + 4 * q);
+          hc[u] = *reinterpret_cast<const Chunk<T, 4>*>(h0 + size_t(t0 + r) * H + 4 * q);
+        }
+        r += step_r; q += step_q;
+        if (q >= qpr) { q -= qpr; ++r; }
+      }
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u)
+        if (rr[u] < rows)
+          *reinterpret_cast<float4*>(dpt + size_t(rr[u]) * H + 4 * qq[u]) =
+              make_float4(to_float(hc[u].v[0]) > 0.f ? g[u].x : 0.f, to_float(hc[u].v[1]) > 0.f ? g[u].y : 0.f,
+                          to_float(hc[u].v[2]) > 0.f ? g[u].z : 0.f, to_float(hc[u].v[3]) > 0.f ? g[u].w : 0.f);
     }
-    for (int i = r0 + group; i < r1; i += ngroups) {
-      float dp[CU];
-      bool live = false;
+    for (int idx = tid; idx < rows * 4; idx += nt)
+      reinterpret_cast<float4*>(xt)[idx] = reinterpret_cast<const float4*>(xs + size_t(t0) * 2 * kS)[idx];
+    for (int idx = tid; idx < rows; idx += nt) opt[idx] = min(max(op[t0 + idx], 0), Tn - 1);   // (pack reports bad ids)
+    __syncthreads();
+    if (part < P) {
+      for (int rw = part; rw < rows; rw += P) {
+        const float dp = dpt[size_t(rw) * H + c];
+        if (dp == 0.f) continue;
+        const float4* xr = reinterpret_cast<const float4*>(xt + size_t(rw) * 2 * kS);
 #pragma unroll
-      for (int u = 0; u < CU; ++u) {
-        const int c = lane + 32 * (f0 + u);
-        dp[u] = (f0 + u < NF && to_float(h0[size_t(i) * H + c]) > 0.f) ? dh0[size_t(i) * H + c] : 0.f;
-        live = live || dp[u] != 0.f;
+        for (int v = 0; v < 4; ++v) {
+          const float4 x = xr[v];
+          acc[4 * v] = fmaf(x.x, dp, acc[4 * v]);
+          acc[4 * v + 1] = fmaf(x.y, dp, acc[4 * v + 1]);
+          acc[4 * v + 2] = fmaf(x.z, dp, acc[4 * v + 2]);
+          acc[4 * v + 3] = fmaf(x.w, dp, acc[4 * v + 3]);
+        }
+        my_oh[size_t(opt[rw]) * H + c] += dp;
+        dbr += dp;
       }
-      if (!__any_sync(0xFFFFFFFFu, live)) continue;
-      float x[2 * kS];
-      load_chunk<float, 2 * kS>(xs + size_t(i) * 2 * kS, x);      // the same 64 bytes for every lane
-      const int o = op[i];
-#pragma unroll
-      for (int u = 0; u < CU; ++u) {
-        if (dp[u] == 0.f) continue;
-#pragma unroll
-        for (int s = 0; s < 2 * kS; ++s) a[s][u] = fmaf(x[s], dp[u], a[s][u]);
-        atomicAdd(&acc[size_t(kS + o) * H + lane + 32 * (f0 + u)], dp[u]);
-        dbr[u] += dp[u];
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < CU; ++u) {
-      if (f0 + u >= NF) continue;
-      const int c = lane + 32 * (f0 + u);
-#pragma unroll
-      for (int s = 0; s < kS; ++s) {
-        atomicAdd(&acc[size_t(s) * H + c], a[s][u]);
-        atomicAdd(&acc[size_t(kS + Tn + s) * H + c], a[kS + s][u]);
-      }
-      atomicAdd(&acc[size_t(F0) * H + c], dbr[u]);
     }
   }
+  if (part < P) {
+#pragma unroll
+    for (int s = 0; s < kS; ++s) {
+      if (acc[s] != 0.f) atomicAdd(&dW0[size_t(s) * H + c], acc[s]);
+      if (acc[kS + s] != 0.f) atomicAdd(&dW0[size_t(kS + Tn + s) * H + c], acc[kS + s]);
+    }
+    if (dbr != 0.f) atomicAdd(&db0[c], dbr);
+  }
   __syncthreads();
-  for (int t = threadIdx.x; t < F0 * H; t += blockDim.x)
-    if (acc[t] != 0.f) atomicAdd(&dW0[t], acc[t]);
-  for (int c = threadIdx.x; c < H; c += blockDim.x)
-    if (acc[size_t(F0) * H + c] != 0.f) atomicAdd(&db0[c], acc[size_t(F0) * H + c]);
+  for (int t = tid; t < Tn * H; t += nt) {
+    float v = 0.f;
+    for (int pp = 0; pp < P; ++pp) v += oh[size_t(pp) * Tn * H + t];
+    if (v != 0.f) atomicAdd(&dW0[size_t(kS) * H + t], v);
+  }
 }
 
 // ---- the heads' MLPs: Linear(in, hid), ReLU, [Linear(hid, hid2), ReLU,] Linear(last, 1) ---------------------
@@ -1180,33 +1202,51 @@ int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* co
   return 4;
 }
 
-// W0's gradient is collected per CTA in shared memory: (2S + T + 1) x H floats
-size_t embed_bwd_smem_bytes(const Dims& d) { return sizeof(float) * size_t(2 * kS + d.T + 1) * d.H; }
+// Eq. 6 in reverse keeps P copies of the one-hot block of W0's gradient ([T x H]) and a tile of R rows in shared
+// memory: as many copies as threads share a column (at most 4), then the largest tile that still fits
+static size_t embed_bwd_bytes(const Dims& d, int R, int P) {
+  return sizeof(float) * (size_t(P) * d.T * d.H + size_t(R) * d.H + size_t(R) * 2 * kS) + sizeof(int32_t) * R;
+}
+static void embed_bwd_shape(const Dims& d, int* R, int* P) {
+  constexpr size_t kCeiling = size_t(227) * 1024;
+  *R = 0; *P = 1;
+  for (int p = std::min(4, std::max(1, kEmbedBwdThreads / d.H)); p >= 1; --p)
+    for (int r = 64; r >= 16; r >>= 1)
+      if (embed_bwd_bytes(d, r, p) <= kCeiling) { *R = r; *P = p; return; }
+  if (embed_bwd_bytes(d, 8, 1) <= kCeiling) *R = 8;
+}
+size_t embed_bwd_smem_bytes(const Dims& d) {
+  int R, P;
+  embed_bwd_shape(d, &R, &P);
+  return embed_bwd_bytes(d, std::max(R, 8), P);
+}
 
 int launch_embed_bwd(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op, const void* shape,
                      const void* eattr, const void* h0, const float* dh0, float* xs, float* gW0, float* gb0, int32_t N,
                      cudaStream_t st) {
   if (N <= 0) return 0;
-  const size_t smem = embed_bwd_smem_bytes(d);
-  const int grid = int(std::min<int64_t>((int64_t(N) + 255) / 256, int64_t(kNumSMs)));
+  int R, P;
+  embed_bwd_shape(d, &R, &P);
+  if (R == 0) return -1;
+  const size_t smem = embed_bwd_bytes(d, R, P);
+  const int grid = int(std::min<int64_t>((int64_t(N) + R - 1) / R, int64_t(kNumSMs)));
   const unsigned grid_x = unsigned((int64_t(N) + 255) / 256);
   // the opt-in is the kernel's ceiling for every later launch: ask for all an SM has, once per device
   constexpr int kSmemCeiling = 227 * 1024;
-  if (smem > size_t(kSmemCeiling)) return -1;
   if (d.dtype == XRL_BF16) {
     static bool attr[64] = {};
     if (!ensure_dynamic_smem(k_embed_bwd<bf16>, kSmemCeiling, attr)) return -1;
     k_embed_inputs<bf16><<<grid_x, 256, 0, st>>>(rowptr, col, static_cast<const bf16*>(shape),
                                                  static_cast<const bf16*>(eattr), xs, N);
     k_embed_bwd<bf16><<<grid, kEmbedBwdThreads, smem, st>>>(xs, op, static_cast<const bf16*>(h0), dh0, gW0, gb0, N,
-                                                            d.H, d.T);
+                                                            d.H, d.T, R, P);
   } else {
     static bool attr[64] = {};
     if (!ensure_dynamic_smem(k_embed_bwd<float>, kSmemCeiling, attr)) return -1;
     k_embed_inputs<float><<<grid_x, 256, 0, st>>>(rowptr, col, static_cast<const float*>(shape),
                                                   static_cast<const float*>(eattr), xs, N);
     k_embed_bwd<float><<<grid, kEmbedBwdThreads, smem, st>>>(xs, op, static_cast<const float*>(h0), dh0, gW0, gb0, N,
-                                                             d.H, d.T);
+                                                             d.H, d.T, R, P);
   }
   return 2;
 }
