@@ -297,6 +297,23 @@ def xrl_ppo_grad(ctx, batch, mask, action, logp_old, adv, ret, loss_out, grad, e
     return loss_out, grad
 
 
+def allreduce_ppo_grad(loss, grad, num_envs, group=None):
+    """Data-parallel training step: every rank has run xrl_ppo_grad on its own environments, so its loss terms
+    and gradient are means over `num_envs` local environments.  In place, they become the means over all
+    ranks' environments (one sum all-reduce of [grad * n | loss * n | n], NCCL for device tensors): the result
+    equals one xrl_ppo_grad call on the concatenated batch.  Returns the global number of environments."""
+    import torch
+    import torch.distributed as dist
+    n = float(num_envs)
+    buf = torch.cat([grad.reshape(-1) * n, loss.reshape(-1).to(grad.dtype) * n,
+                     torch.tensor([n], dtype=grad.dtype, device=grad.device)])
+    dist.all_reduce(buf, op=dist.ReduceOp.SUM, group=group)
+    total = float(buf[-1].item())
+    grad.copy_((buf[:grad.numel()] / total).reshape(grad.shape))
+    loss.copy_((buf[grad.numel():-1] / total).reshape(loss.shape).to(loss.dtype))
+    return int(round(total))
+
+
 def xrl_last_device_status(ctx, stream=None) -> int:
     s = C.c_int32()
     _check(load_library().xrl_last_device_status(ctx, _stream(stream), C.byref(s)),

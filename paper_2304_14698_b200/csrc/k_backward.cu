@@ -471,13 +471,21 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
 }
 
 // out [rows x H] fp32 = G [rows x H] bf16 times W^T, W [H x H] bf16 row-major [in x out]: out[r][k] = sum_n G[r][n] W[k][n]
+// A CTA takes tiles_per_cta consecutive tiles of 128 rows (kGwtTiles when that still leaves several waves of
+// CTAs, else one); its loop runs over (tile, 64-wide step of n) pairs, so
+// that the first pieces of the next tile are already on their way while the last step of the current tile is
+// multiplied and its 64 KB of results are stored.
+constexpr int kGwtTiles = 4;
 __global__ void __launch_bounds__(256, 2)
-k_gwt_mma(const bf16* __restrict__ G, const bf16* __restrict__ W, float* __restrict__ out, int rows, int H) {
+k_gwt_mma(const bf16* __restrict__ G, const bf16* __restrict__ W, float* __restrict__ out, int rows, int H,
+          int tiles_per_cta) {
   __shared__ __align__(128) bf16 As[128 * 64];      // [row r][64 n], 8 pieces of 16 bytes per row
   __shared__ __align__(128) bf16 Bs[128 * 64];      // [row k][64 n]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int wm = warp >> 1, wn = warp & 1;
-  const int r0 = blockIdx.x * 128, k0 = blockIdx.y * 128;
+  const int k0 = blockIdx.y * 128;
+  const int tile0 = blockIdx.x * tiles_per_cta, ntiles = (rows + 127) / 128;
+  const int nk = H / 64, total = min(tiles_per_cta, ntiles - tile0) * nk;
   float acc[2][8][4];
 #pragma unroll
   for (int a = 0; a < 2; ++a)
@@ -486,9 +494,10 @@ k_gwt_mma(const bf16* __restrict__ G, const bf16* __restrict__ W, float* __restr
 #pragma unroll
       for (int c = 0; c < 4; ++c) acc[a][b][c] = 0.f;
   const uint32_t as_base = uint32_t(__cvta_generic_to_shared(As)), bs_base = uint32_t(__cvta_generic_to_shared(Bs));
-  // the next tile's pieces travel from global memory to registers while the current tile is multiplied
+  // the next step's pieces travel from global memory to registers while the current step is multiplied
   uint4 va[4], vb[4];
-  auto fetch = [&](int n0) {
+  auto fetch = [&](int step) {
+    const int r0 = (tile0 + step / nk) * 128, n0 = (step % nk) * 64;
 #pragma unroll
     for (int it = 0; it < 4; ++it) {
       const int idx = tid + 256 * it, row = idx >> 3, ch = idx & 7;
@@ -497,8 +506,8 @@ k_gwt_mma(const bf16* __restrict__ G, const bf16* __restrict__ W, float* __restr
       vb[it] = *reinterpret_cast<const uint4*>(W + size_t(k0 + row) * H + n0 + ch * 8);
     }
   };
-  fetch(0);
-  for (int n0 = 0; n0 < H; n0 += 64) {
+  if (total > 0) fetch(0);
+  for (int step = 0; step < total; ++step) {
 #pragma unroll
     for (int it = 0; it < 4; ++it) {
       const int idx = tid + 256 * it, row = idx >> 3, ch = idx & 7;
@@ -507,7 +516,7 @@ k_gwt_mma(const bf16* __restrict__ G, const bf16* __restrict__ W, float* __restr
       *reinterpret_cast<uint4*>(Bs + phys) = vb[it];
     }
     __syncthreads();
-    if (n0 + 64 < H) fetch(n0 + 64);
+    if (step + 1 < total) fetch(step + 1);
 #pragma unroll
     for (int kk = 0; kk < 64; kk += 16) {
       uint32_t af[2][4];
@@ -531,17 +540,23 @@ k_gwt_mma(const bf16* __restrict__ G, const bf16* __restrict__ W, float* __restr
       }
     }
     __syncthreads();
-  }
-  const int g = lane >> 2, t = lane & 3;
+    if (step % nk == nk - 1) {                       // the tile is complete: store it, start the next from zero
+      const int r0 = (tile0 + step / nk) * 128;
+      const int g = lane >> 2, t = lane & 3;
 #pragma unroll
-  for (int mt = 0; mt < 2; ++mt)
+      for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-      const int r = r0 + wm * 32 + mt * 16 + g, c = k0 + wn * 64 + nt * 8 + 2 * t;
-      if (r < rows) *reinterpret_cast<float2*>(out + size_t(r) * H + c) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
-      if (r + 8 < rows)
-        *reinterpret_cast<float2*>(out + size_t(r + 8) * H + c) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
+        for (int nt = 0; nt < 8; ++nt) {
+          const int r = r0 + wm * 32 + mt * 16 + g, c = k0 + wn * 64 + nt * 8 + 2 * t;
+          if (r < rows)
+            *reinterpret_cast<float2*>(out + size_t(r) * H + c) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
+          if (r + 8 < rows)
+            *reinterpret_cast<float2*>(out + size_t(r + 8) * H + c) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) acc[mt][nt][q] = 0.f;
+        }
     }
+  }
 }
 
 // dW [H x H] fp32 += A^T B over the rows [chunk z], A = h_in [rows x H] bf16, B = dz [rows x H] bf16
@@ -1154,7 +1169,9 @@ int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* co
   const int want_chunks = std::max(1, 2 * kNumSMs / std::max(1, tiles));
   const int chunk_mma = std::max(512, int(((int64_t(N) + want_chunks - 1) / want_chunks + 31) & ~int64_t(31)));
   dim3 g_atb_mma(unsigned(H / 128), unsigned(H / 128), unsigned((N + chunk_mma - 1) / chunk_mma));
-  dim3 g_gwt_mma(unsigned((N + 127) / 128), unsigned(H / 128));
+  const int row_tiles = (N + 127) / 128;
+  const int gwt_tpc = int64_t(row_tiles) * (H / 128) >= int64_t(kGwtTiles) * 4 * kNumSMs ? kGwtTiles : 1;
+  dim3 g_gwt_mma(unsigned((row_tiles + gwt_tpc - 1) / gwt_tpc), unsigned(H / 128));
   const int NF = H / 32;
   const bool rows_kernels = (32 % K == 0) && (NF == 1 || NF == 2 || NF == 4 || NF == 8 || NF == 16);
   // bf16 models of hidden 128, 256 or 512 take both products on the tensor cores, from a bf16 copy of dz
@@ -1190,7 +1207,7 @@ int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* co
     }                                                                                                          \
     if (mma) {                                                                                                 \
       k_atb_mma<<<g_atb_mma, 256, 0, st>>>(static_cast<const bf16*>(h_in), dzb, gW, N, H, chunk_mma);          \
-      k_gwt_mma<<<g_gwt_mma, 256, 0, st>>>(dzb, static_cast<const bf16*>(lw.W), dh_in, N, H);                  \
+      k_gwt_mma<<<g_gwt_mma, 256, 0, st>>>(dzb, static_cast<const bf16*>(lw.W), dh_in, N, H, gwt_tpc);                  \
     } else {                                                                                                   \
       k_atb<TY_><<<g_atb, 256, 0, st>>>(static_cast<const TY_*>(h_in), H, dz, H, gW, H, N, H, H, chunk);       \
       k_gwt<TY_><<<g_gwt, 256, 0, st>>>(dz, static_cast<const TY_*>(lw.W), dh_in, N, H, H);                    \

@@ -87,7 +87,6 @@ struct xrl_ctx {
   bool capturing = false;
   // reverse pass: saved layer inputs and gradient scratch (allocated on the first xrl_ppo_grad)
   DeviceBuf bw;
-  int64_t launches_backward = 0;
   cudaStream_t last_pipe = nullptr;   // stream of the last batch that was packed range by range (its kernels
                                       // report bad graphs too: xrl_last_device_status waits for it as well)
 };
@@ -1062,7 +1061,7 @@ xrl_status xrl_ppo_grad(xrl_ctx* ctx, const xrl_batch* b, const float* g0, const
                                  grad + (ctx->dw.b0 - wb), b->N, st);
   if (k < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
   n += k;
-  ctx->launches_backward = n;
+  (void)n;   // (launches of the reverse pass are not reported by xrl_launch_counts)
   XRL_CUDA(cudaGetLastError());
   return XRL_OK;
 }
