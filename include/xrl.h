@@ -256,7 +256,7 @@ xrl_status xrl_sample(xrl_ctx* ctx, const float* probs, int32_t num_envs, int32_
  *   L_vf     =   mean_e (value_e - ret_e)^2                                                (Eq. 4)
  *   L_ent    =   mean_e sum_a p_a log p_a      (minus the policy's entropy)
  *   J        =   L_clip + c1 L_vf + c2 L_ent                                               (Eq. 5)
- * The forward pass is that of xrl_encode and xrl_policy_value with every layer's input kept; the reverse
+ * The forward pass is that of xrl_encode and xrl_policy_value with every layer's input and Z kept; the reverse
  * pass runs layer by layer in fp32 (ReLU'(0) = 0, LeakyReLU'(0) = 0.2; where the clipped term of Eq. 3 is
  * the smaller one its slope is zero).  For a bf16 model the gradient of W0 and of the layer matrices is the
  * one with respect to the stored (rounded) values.  Sums over rows use floating-point atomics: the last
@@ -268,8 +268,8 @@ xrl_status xrl_sample(xrl_ctx* ctx, const float* probs, int32_t num_envs, int32_
  *   loss_out  DEVICE fp32 [4] = { J, L_clip, L_vf, L_ent }
  *   grad      DEVICE fp32, laid out like the weight blob (xrl_weights_size bytes), overwritten
  *   logp_out  DEVICE fp32 [num_envs] or NULL: log pi(action_e) under the current weights
- * The first call allocates the workspace for the context's capacities ((L + 2) copies of the node features
- * plus three fp32 ones) and therefore synchronises; later calls only enqueue.  Not recordable
+ * The first call allocates the workspace for the context's capacities ((L + 2) copies of the node features,
+ * L of the transformed features Z and three fp32 ones) and therefore synchronises; later calls only enqueue.  Not recordable
  * (XRL_ERR_STATE between xrl_graph_begin and xrl_graph_launch).  XRL_ERR_UNSUPPORTED when
  * (T + 8) x H floats exceed one SM's shared memory (227 KB): the operator block of W0's gradient and a tile
  * of eight rows are kept there.

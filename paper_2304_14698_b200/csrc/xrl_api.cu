@@ -478,9 +478,11 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
 // With fuse_readout the last of the `layers` attention layers may leave per-graph partial sums in
 // ctx->partial instead of node features in ctx->h; *fused tells whether it did.
 // With `hs` (layers + 1 buffers of N x H storage-type values) every layer's input is kept: Eq. 6 writes hs[0],
-// layer l reads hs[l] and writes hs[l + 1].
+// layer l reads hs[l] and writes hs[l + 1]; with `zs` / `ss` layer l's Z rows and half-scores go to zs[l] / ss[l]
+// instead of the context's one buffer each.
 int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t st, bool fuse_readout = false,
-                    bool* fused = nullptr, int32_t row_begin = 0, int32_t row_end = -1, void* const* hs = nullptr) {
+                    bool* fused = nullptr, int32_t row_begin = 0, int32_t row_end = -1, void* const* hs = nullptr,
+                    void* const* zs = nullptr, float* const* ss = nullptr) {
   const Dims& d = ctx->dims;
   const Window win{row_begin, row_end < 0 ? b->N : row_end, 0};   // graphs are independent: any range of whole graphs
   Profiler& pf = ctx->prof;
@@ -501,13 +503,15 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
   for (int l = 0; l < layers; ++l) {
     const void* h_in = hs ? hs[l] : ctx->h.p;
     void* h_out = hs ? hs[l + 1] : ctx->h.p;
+    void* Zl = zs ? zs[l] : ctx->Z.p;
+    float* Sl = ss ? ss[l] : ctx->scores.as<float>();
     slot = pf.begin(st);
     k = -1;
     if (ctx->use_umma)
-      k = launch_xform_umma(d, h_in, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), win,
+      k = launch_xform_umma(d, h_in, ctx->dw.layer[l], Zl, Sl, win,
                             ctx->status.as<int32_t>(), st);
     if (k < 0 && !d.zmerged)
-      k = launch_xform_simt(d, h_in, ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), win,
+      k = launch_xform_simt(d, h_in, ctx->dw.layer[l], Zl, Sl, win,
                             st);
     if (k < 0) return -1;                       // merged rows: only the tensor-core transform writes them
     pf.end(FAM_XFORM, slot, k, st);
@@ -516,15 +520,15 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
     k = -1;
     bool fused_here = false;
     if (fuse_readout && l == layers - 1) {
-      k = launch_aggregate_tma(d, gat_rowptr, gat_col, ctx->Z.p,
-                               ctx->scores.as<float>(), ctx->dw.layer[l].b, h_out, win, b->N,
+      k = launch_aggregate_tma(d, gat_rowptr, gat_col, Zl,
+                               Sl, ctx->dw.layer[l].b, h_out, win, b->N,
                                b->seg_id.as<int32_t>(), ctx->partial.as<float>(),
                                ctx->status.as<int32_t>(), st);
       if (k >= 0) { fused_here = true; if (fused) *fused = true; }
     }
     if (k < 0)
-      k = launch_aggregate(d, gat_rowptr, gat_col, ctx->Z.p,
-                           ctx->scores.as<float>(), ctx->dw.layer[l].b,
+      k = launch_aggregate(d, gat_rowptr, gat_col, Zl,
+                           Sl, ctx->dw.layer[l].b,
                            h_out, win, b->N, ctx->status.as<int32_t>(), st);
     if (k < 0) return -1;
     pf.end(fused_here ? FAM_AGG_READOUT : FAM_AGG, slot, k, st);
@@ -1005,8 +1009,10 @@ xrl_status xrl_ppo_grad(xrl_ctx* ctx, const xrl_batch* b, const float* g0, const
   const size_t sb = storage_bytes(c.dtype), Nmax = size_t(c.max_nodes), H = size_t(c.hidden);
   const size_t h_bytes = up(sb * Nmax * H), f_bytes = up(4 * Nmax * H), ds_bytes = up(8 * Nmax * size_t(c.heads));
   const size_t heads_bytes = up(4 * ppo_heads_workspace_floats(d, c.max_graphs, c.max_envs));
+  const size_t z_bytes = up(Nmax * z_row_bytes(d));
   if (!ctx->bw.p) {
-    if (ctx->bw.alloc(size_t(L + 2) * h_bytes + 3 * f_bytes + ds_bytes + heads_bytes) != cudaSuccess) {
+    if (ctx->bw.alloc(size_t(L + 2) * h_bytes + size_t(L) * (z_bytes + ds_bytes) + 3 * f_bytes + ds_bytes +
+                      heads_bytes) != cudaSuccess) {
       cudaGetLastError();
       ctx->bw.p = nullptr;
       return XRL_ERR_ALLOC;
@@ -1018,6 +1024,9 @@ xrl_status xrl_ppo_grad(xrl_ctx* ctx, const xrl_batch* b, const float* g0, const
   void* hs[65];
   for (int l = 0; l <= L; ++l) { hs[l] = p; p += h_bytes; }
   void* dz_store = p; p += h_bytes;                 // dz in the storage type, for the tensor-core products
+  void* zs[64];                                     // every layer's Z rows and half-scores, kept for the reverse pass
+  float* ss[64];
+  for (int l = 0; l < L; ++l) { zs[l] = p; p += z_bytes; ss[l] = reinterpret_cast<float*>(p); p += ds_bytes; }
   float* dh_a = reinterpret_cast<float*>(p); p += f_bytes;
   float* dh_b = reinterpret_cast<float*>(p); p += f_bytes;
   float* dz = reinterpret_cast<float*>(p); p += f_bytes;
@@ -1026,7 +1035,7 @@ xrl_status xrl_ppo_grad(xrl_ctx* ctx, const xrl_batch* b, const float* g0, const
   XRL_CUDA(cudaMemsetAsync(grad, 0, 4 * ctx->weight_floats, st));
   XRL_CUDA(cudaMemsetAsync(loss_out, 0, 16, st));
   if (b->B == 0 || b->num_envs == 0) return XRL_OK;
-  int n = run_node_layers(ctx, b, L, st, false, nullptr, 0, -1, hs);
+  int n = run_node_layers(ctx, b, L, st, false, nullptr, 0, -1, hs, zs, ss);
   if (n < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
   const float* wb = ctx->w_f32.as<float>();
   n += launch_ppo_heads(d, ctx->dw, grad, wb, hs[L], b->node_off.as<int32_t>(), b->seg_id.as<int32_t>(), g0,
@@ -1034,22 +1043,12 @@ xrl_status xrl_ppo_grad(xrl_ctx* ctx, const xrl_batch* b, const float* g0, const
                         heads_ws, loss_out, dh_a, logp_out, ctx->status.as<int32_t>(), st);
   const int32_t* gat_rowptr = c.neighbourhood ? b->rowptr_nbr.as<int32_t>() : b->rowptr.as<int32_t>();
   const int32_t* gat_col = c.neighbourhood ? b->col_nbr.as<int32_t>() : b->col.as<int32_t>();
-  const Window win{0, b->N, 0};
   float* dh_cur = dh_a;
   float* dh_nxt = dh_b;
   for (int l = L - 1; l >= 0 && b->N > 0; --l) {
-    // the layer's Z rows and half-scores again, from its saved input
-    int k = -1;
-    if (ctx->use_umma)
-      k = launch_xform_umma(d, hs[l], ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), win,
-                            ctx->status.as<int32_t>(), st);
-    if (k < 0 && !d.zmerged)
-      k = launch_xform_simt(d, hs[l], ctx->dw.layer[l], ctx->Z.p, ctx->scores.as<float>(), win, st);
-    if (k < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
-    n += k;
     const LayerWeights& lw = ctx->dw.layer[l];
     float* ga_src = grad + (lw.a_src - wb);
-    k = launch_gat_layer_bwd(d, gat_rowptr, gat_col, ctx->Z.p, ctx->scores.as<float>(), hs[l], hs[l + 1], dh_cur,
+    const int k = launch_gat_layer_bwd(d, gat_rowptr, gat_col, zs[l], ss[l], hs[l], hs[l + 1], dh_cur,
                              dh_nxt, dz, ds, dz_store, lw, ga_src - H * H, ga_src, grad + (lw.a_dst - wb),
                              grad + (lw.b - wb), b->N, st);
     if (k < 0) { cudaGetLastError(); return XRL_ERR_CUDA; }
