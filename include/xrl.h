@@ -279,6 +279,17 @@ xrl_status xrl_ppo_grad(xrl_ctx* ctx, const xrl_batch* batch, const float* g0, c
                         float eps, float c1, float c2, float* loss_out, float* grad, float* logp_out,
                         void* stream);
 
+/* Generalised advantage estimation, the estimator Section 3.3.4 takes its advantages from, for M trajectories of
+ * T steps each, stored step-major:
+ *   delta_t = r_t + gamma V_{t+1} (1 - done_t) - V_t,   A_t = delta_t + gamma lambda (1 - done_t) A_{t+1},
+ *   R_t = A_t + V_t  (the value target of Eq. 4).
+ *   reward DEVICE fp32 [T x M]; values DEVICE fp32 [(T + 1) x M] (the last row bootstraps the tail);
+ *   done DEVICE u8 [T x M] (1 = the episode ended with step t); adv, ret DEVICE fp32 [T x M].
+ * One thread per trajectory.  Needs no context.  Errors: INVALID_ARG, CUDA. */
+xrl_status xrl_gae(int32_t device, int32_t num_steps, int32_t num_trajectories, const float* reward,
+                   const float* values, const uint8_t* done, float gamma, float lambda, float* adv, float* ret,
+                   void* stream);
+
 /* Read and clear the device status word.  Synchronises `stream`.  *status (HOST) receives the
  * first error code any kernel recorded since the last call, or XRL_OK. */
 xrl_status xrl_last_device_status(xrl_ctx* ctx, void* stream, int32_t* status);

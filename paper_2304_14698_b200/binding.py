@@ -25,7 +25,7 @@ EXPORTED_SYMBOLS = [
     "xrl_batch_free", "xrl_batch_info", "xrl_batch_export", "xrl_encode", "xrl_debug_node_features",
     "xrl_policy_value", "xrl_sample", "xrl_last_device_status", "xrl_launch_counts", "xrl_version",
     "xrl_profile", "xrl_profile_read", "xrl_pack_csr_static", "xrl_encode_delta", "xrl_delta_rows", "xrl_get_weights",
-    "xrl_graph_begin", "xrl_graph_launch", "xrl_batch_set_edge_attr", "xrl_ppo_grad",
+    "xrl_graph_begin", "xrl_graph_launch", "xrl_batch_set_edge_attr", "xrl_ppo_grad", "xrl_gae",
 ]
 PROFILE_FAMILIES = ["pack", "node_update", "transform", "aggregate", "readout", "heads", "aggregate_readout"]
 
@@ -89,6 +89,7 @@ def load_library():
         "xrl_batch_set_edge_attr": [vp, vp, i32, vp, vp],
         "xrl_graph_begin": [vp],
         "xrl_ppo_grad": [vp] * 8 + [C.c_float] * 3 + [vp] * 4,
+        "xrl_gae": [i32, i32, i32, vp, vp, vp, C.c_float, C.c_float, vp, vp, vp],
         "xrl_graph_launch": [vp, vp],
     }
     for name, args in sigs.items():
@@ -295,6 +296,19 @@ def xrl_ppo_grad(ctx, batch, mask, action, logp_old, adv, ret, loss_out, grad, e
                                      _dev_ptr(logp_out), _stream(stream))
     _check(st, "xrl_ppo_grad")
     return loss_out, grad
+
+
+def xrl_gae(reward, values, done, gamma, lam, adv=None, ret=None, stream=None):
+    """Generalised advantage estimates of M trajectories, step-major device tensors: reward, done [T x M],
+    values [(T + 1) x M] -> (adv, ret) [T x M]."""
+    import torch
+    T, M = reward.shape
+    adv = torch.empty_like(reward) if adv is None else adv
+    ret = torch.empty_like(reward) if ret is None else ret
+    st = load_library().xrl_gae(reward.device.index or 0, T, M, _dev_ptr(reward), _dev_ptr(values), _dev_ptr(done),
+                                C.c_float(gamma), C.c_float(lam), _dev_ptr(adv), _dev_ptr(ret), _stream(stream))
+    _check(st, "xrl_gae")
+    return adv, ret
 
 
 def allreduce_ppo_grad(loss, grad, num_envs, group=None):

@@ -1070,9 +1070,35 @@ int mlp_weight_grads(const float* X, int in, int rows, int hid, int hid2, const 
   return n;
 }
 
+// Generalised advantage estimates: one thread per trajectory, backwards over its T steps (a first-order
+// recurrence; trajectories are laid out step-major, [T x M], so that the threads of a warp read neighbours)
+__global__ void k_gae(const float* __restrict__ reward, const float* __restrict__ values,
+                      const uint8_t* __restrict__ done, float gamma, float lambda, int T, int M,
+                      float* __restrict__ adv, float* __restrict__ ret) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= M) return;
+  float run = 0.f, vnext = values[size_t(T) * M + j];
+  for (int t = T - 1; t >= 0; --t) {
+    const float nd = done[size_t(t) * M + j] ? 0.f : 1.f;
+    const float v = values[size_t(t) * M + j];
+    const float delta = reward[size_t(t) * M + j] + gamma * vnext * nd - v;
+    run = delta + gamma * lambda * nd * run;
+    adv[size_t(t) * M + j] = run;
+    ret[size_t(t) * M + j] = run + v;
+    vnext = v;
+  }
+}
+
 }  // namespace
 
 // ---- launchers ------------------------------------------------------------------------------------------
+int launch_gae(const float* reward, const float* values, const uint8_t* done, float gamma, float lambda, int32_t T,
+               int32_t M, float* adv, float* ret, cudaStream_t st) {
+  if (T <= 0 || M <= 0) return 0;
+  k_gae<<<unsigned((M + 127) / 128), 128, 0, st>>>(reward, values, done, gamma, lambda, T, M, adv, ret);
+  return 1;
+}
+
 // every piece of the heads' workspace starts on a 16-byte boundary (some are read as float4)
 static size_t up4(size_t n) { return (n + 3) & ~size_t(3); }
 size_t ppo_heads_workspace_floats(const Dims& d, int64_t B, int64_t num_envs) {

@@ -1065,6 +1065,18 @@ xrl_status xrl_ppo_grad(xrl_ctx* ctx, const xrl_batch* b, const float* g0, const
   return XRL_OK;
 }
 
+xrl_status xrl_gae(int32_t device, int32_t num_steps, int32_t num_trajectories, const float* reward,
+                   const float* values, const uint8_t* done, float gamma, float lambda, float* adv, float* ret,
+                   void* stream) {
+  if (num_steps < 0 || num_trajectories < 0) return XRL_ERR_INVALID_ARG;
+  if (num_steps > 0 && num_trajectories > 0 && (!reward || !values || !done || !adv || !ret)) return XRL_ERR_INVALID_ARG;
+  XRL_CUDA(cudaSetDevice(device));
+  launch_gae(reward, values, done, gamma, lambda, num_steps, num_trajectories, adv, ret,
+             static_cast<cudaStream_t>(stream));
+  XRL_CUDA(cudaGetLastError());
+  return XRL_OK;
+}
+
 xrl_status xrl_sample(xrl_ctx* ctx, const float* probs, int32_t num_envs, int32_t num_actions,
                       uint64_t seed, uint64_t step, int32_t* action, void* stream) {
   if (!ctx || num_envs < 0 || num_actions < 1) return XRL_ERR_INVALID_ARG;

@@ -210,6 +210,8 @@ int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* co
                          const void* h_in, const void* h_out, const float* dh_out, float* dh_in, float* dz,
                          float* ds, void* dz_store, const LayerWeights& lw, float* gW, float* ga_src, float* ga_dst,
                          float* gb, int32_t N, cudaStream_t st);
+int launch_gae(const float* reward, const float* values, const uint8_t* done, float gamma, float lambda, int32_t T,
+               int32_t M, float* adv, float* ret, cudaStream_t st);
 size_t embed_bwd_smem_bytes(const Dims& d);
 int launch_embed_bwd(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op, const void* shape,
                      const void* eattr, const void* h0, const float* dh0, float* xs /* scratch [N x 16] */,

@@ -175,3 +175,24 @@ def test_an_action_the_mask_excludes_is_reported(xo):
         assert e.value.status == 1
     finally:
         ag.close()
+
+
+def test_advantage_estimates_match_the_oracle(xo):
+    import torch
+    import paper_2304_14698_b200 as xrl
+    rng = np.random.default_rng(9)
+    T, M = 37, 203
+    reward = rng.normal(size=(T, M)); values = rng.normal(size=(T + 1, M))
+    done = (rng.random((T, M)) < 0.1).astype(np.uint8)
+    done[:, 0] = 0; done[:, 1] = 1                      # a trajectory that never ends, one that ends every step
+    f32 = lambda a: torch.from_numpy(np.asarray(a, np.float32)).cuda()
+    for gamma, lam in ((0.99, 0.95), (1.0, 1.0), (0.9, 0.0)):
+        adv, ret = xrl.xrl_gae(f32(reward), f32(values), torch.from_numpy(done).cuda(), gamma, lam)
+        torch.cuda.synchronize()
+        for j in (0, 1, 2, 57, M - 1):
+            a, r = xo.gae(reward[:, j].astype(np.float32), values[:, j].astype(np.float32), done[:, j], gamma, lam)
+            gpu_util.assert_close(adv[:, j].cpu().numpy(), a, "fp32", f"adv {j}")
+            gpu_util.assert_close(ret[:, j].cpu().numpy(), r, "fp32", f"ret {j}")
+    a0, r0 = xrl.xrl_gae(torch.empty((0, 5), device="cuda"), torch.empty((1, 5), device="cuda"),
+                         torch.empty((0, 5), dtype=torch.uint8, device="cuda"), 0.9, 0.9)
+    assert a0.shape == (0, 5)
