@@ -196,3 +196,32 @@ def test_advantage_estimates_match_the_oracle(xo):
     a0, r0 = xrl.xrl_gae(torch.empty((0, 5), device="cuda"), torch.empty((1, 5), device="cuda"),
                          torch.empty((0, 5), dtype=torch.uint8, device="cuda"), 0.9, 0.9)
     assert a0.shape == (0, 5)
+
+
+def test_gradient_of_a_batch_packed_range_by_range(xo, monkeypatch):
+    """The gradient call joins the ranges of a batch that was copied and packed range by range."""
+    import torch
+    import paper_2304_14698_b200 as xrl
+    from test_gpu_pipeline import _pinned, _pack_pinned
+    monkeypatch.setenv("XRL_PIPELINE_MIN_NODES", "2000")
+    batch = configs.make_batch(3, candidates=15)
+    m = batch["model"]
+    blob, _ = gpu_util.default_weights(batch, 8)
+    st, packed = xo.pack(batch)
+    assert st == 0
+    action, logp_old, adv, ret = _transitions(xo, m, blob, batch, packed, 1)
+    mir = xo.ppo_grad(m, blob, batch, packed, action, logp_old, adv, ret, mirrored=1)
+    ag = gpu_util.make_agent(batch)
+    try:
+        ag.set_weights(blob)
+        keep = _pinned(ag, batch)
+        _pack_pinned(xrl, ag, batch, keep)
+        f32 = lambda a: torch.from_numpy(np.asarray(a, np.float32)).cuda()
+        loss = torch.empty(4, device="cuda"); grad = torch.empty(len(blob), device="cuda")
+        xrl.xrl_ppo_grad(ag.ctx, ag.batch, torch.from_numpy(batch["mask"]).cuda(), torch.from_numpy(action).cuda(),
+                         f32(logp_old), f32(adv), f32(ret), loss, grad)
+        torch.cuda.synchronize()
+        assert ag.device_status() == 0
+        _check_grad(m, grad.cpu().numpy().astype(np.float64), mir["grad"], GRAD_TOL["bf16 mirrored"], "mirrored")
+    finally:
+        ag.close()
