@@ -823,27 +823,36 @@ __device__ void mlp_bwd(int in, const MlpW& m, const float* y1, const float* y2,
   __syncthreads();
 }
 
-// per-graph sums of the last layer's node features, written as the first H entries of row g of U [B x (H + Dg)];
-// the graph's global attributes fill the rest
+// per-graph sums of the last layer's node features into the first H entries of row g of U [B x (H + Dg)] (zeroed
+// beforehand): a CTA takes 64 consecutive rows, a thread a column; a run of rows of one graph is summed in a
+// register and added to U once (atomics: a graph's rows span several CTAs)
 template <typename T>
 __global__ void __launch_bounds__(256)
-k_graph_sum(const T* __restrict__ h, const int32_t* __restrict__ node_off, const float* __restrict__ g0,
-            float* __restrict__ U, int H, int Dg) {
-  const int g = blockIdx.x;
-  const int32_t lo = node_off[g], hi = node_off[g + 1];
+k_graph_sum(const T* __restrict__ h, const int32_t* __restrict__ seg_id, float* __restrict__ U, int N, int H, int HU,
+            int rows_per_cta) {
+  const int r0 = blockIdx.x * rows_per_cta, r1 = min(N, r0 + rows_per_cta);
+  if (r0 >= r1) return;
   for (int c = threadIdx.x; c < H; c += blockDim.x) {
     float s = 0.f;
-    for (int32_t i = lo; i < hi; ++i) s += to_float(h[size_t(i) * H + c]);
-    U[size_t(g) * (H + Dg) + c] = s;
+    int32_t g = seg_id[r0];
+    for (int i = r0; i < r1; ++i) {
+      const int32_t gi = seg_id[i];
+      if (gi != g) {
+        atomicAdd(&U[size_t(g) * HU + c], s);
+        s = 0.f;
+        g = gi;
+      }
+      s += to_float(h[size_t(i) * H + c]);
+    }
+    atomicAdd(&U[size_t(g) * HU + c], s);
   }
-  for (int t = threadIdx.x; t < Dg; t += blockDim.x) U[size_t(g) * (H + Dg) + H + t] = g0 ? g0[size_t(g) * Dg + t] : 0.f;
 }
 
 // ---- per graph, forward: Eq. 8 and the policy head ---------------------------------------------------------
 __global__ void __launch_bounds__(256)
-k_graph_fwd(const float* __restrict__ U, const float* __restrict__ Wg, const float* __restrict__ bg, MlpW pm,
-            float* __restrict__ emb, float* __restrict__ py1, float* __restrict__ py2, float* __restrict__ logit,
-            int H, int Dg) {
+k_graph_fwd(float* __restrict__ U, const float* __restrict__ g0, const float* __restrict__ Wg,
+            const float* __restrict__ bg, MlpW pm, float* __restrict__ emb, float* __restrict__ py1,
+            float* __restrict__ py2, float* __restrict__ logit, int H, int Dg) {
   extern __shared__ float sm[];
   float* scratch = sm;                              // [blockDim]
   float* uu = scratch + blockDim.x;                 // [H + Dg]
@@ -851,7 +860,12 @@ k_graph_fwd(const float* __restrict__ U, const float* __restrict__ Wg, const flo
   float* y1 = x + H;                                // [hid]
   float* y2 = y1 + pm.hid;                          // [hid2]
   const int g = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
-  for (int k = tid; k < H + Dg; k += nt) uu[k] = U[size_t(g) * (H + Dg) + k];
+  for (int k = tid; k < H; k += nt) uu[k] = U[size_t(g) * (H + Dg) + k];
+  for (int k = tid; k < Dg; k += nt) {              // the graph's global attributes complete its row of U
+    const float v = g0 ? g0[size_t(g) * Dg + k] : 0.f;
+    uu[H + k] = v;
+    U[size_t(g) * (H + Dg) + H + k] = v;
+  }
   __syncthreads();
   for (int c = tid; c < H; c += nt) {
     float acc = bg[c];
@@ -1142,12 +1156,18 @@ int launch_ppo_heads(const Dims& d, const DevWeights& w, float* grad_base, const
   cudaMemsetAsync(demb, 0, sizeof(float) * size_t(B) * H, st);
   cudaMemsetAsync(dlogit, 0, sizeof(float) * size_t(B), st);
   cudaMemsetAsync(eb.vu, 0, sizeof(float) * size_t(p - eb.vu), st);
-  if (d.dtype == XRL_BF16)
-    k_graph_sum<bf16><<<B, 256, 0, st>>>(static_cast<const bf16*>(hL), node_off, g0, U, d.H, d.Dg);
-  else
-    k_graph_sum<float><<<B, 256, 0, st>>>(static_cast<const float*>(hL), node_off, g0, U, d.H, d.Dg);
-  ++n;
-  k_graph_fwd<<<B, 256, sizeof(float) * (256 + HU + H + Hm + Hm2), st>>>(U, w.Wg, w.bg, pm, emb, py1, py2, logit,
+  cudaMemsetAsync(U, 0, sizeof(float) * size_t(B) * HU, st);
+  if (N > 0) {
+    const int rows_per_cta = 64;
+    const unsigned grid = unsigned((N + rows_per_cta - 1) / rows_per_cta);
+    if (d.dtype == XRL_BF16)
+      k_graph_sum<bf16><<<grid, 256, 0, st>>>(static_cast<const bf16*>(hL), seg_id, U, int(N), d.H, int(HU), rows_per_cta);
+    else
+      k_graph_sum<float><<<grid, 256, 0, st>>>(static_cast<const float*>(hL), seg_id, U, int(N), d.H, int(HU),
+                                               rows_per_cta);
+    ++n;
+  }
+  k_graph_fwd<<<B, 256, sizeof(float) * (256 + HU + H + Hm + Hm2), st>>>(U, g0, w.Wg, w.bg, pm, emb, py1, py2, logit,
                                                                           d.H, d.Dg);
   ++n;
   k_ppo_env<<<num_envs, 256, sizeof(float) * (256 + 4 * H + 2 * Hm + 2 * Hm2), st>>>(
