@@ -334,6 +334,8 @@ def main():
 
         def grad_step():
             xrl.xrl_ppo_grad(agent.ctx, agent.batch, mask_d, act_d, lp_d, adv_d, ret_d, loss_d, grad_d)
+            if world > 1:                      # data-parallel: means over all ranks' environments
+                xrl.allreduce_ppo_grad(loss_d, grad_d, ne_t)
 
         for _ in range(3):
             grad_step()
@@ -348,7 +350,8 @@ def main():
         assert agent.device_status() == 0
         tms = t0.elapsed_time(t1) / args.steps
         train = {"ms_per_step": tms, "unit": "graphs/s",
-                 "note": "xrl_ppo_grad: forward with kept activations, Eq. 3-5, reverse pass to every weight"}
+                 "note": "xrl_ppo_grad: forward with kept activations, Eq. 3-5, reverse pass to every weight"
+                         + ("; gradient all-reduce over the ranks included" if world > 1 else "")}
 
     # ---- end to end: host buffers in, results out, through the public call ---------------------------
     e2e = None
@@ -400,6 +403,8 @@ def main():
             e2e["s_per_step"] = reduce_over_ranks(e2e["s_per_step"], 0, 0, 0, dist, red_dev)[0]
         if delta:
             delta["ms_per_step"] = reduce_over_ranks(delta["ms_per_step"], 0, 0, 0, dist, red_dev)[0]
+        if train:
+            train["ms_per_step"] = reduce_over_ranks(train["ms_per_step"], 0, 0, 0, dist, red_dev)[0]
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
