@@ -10,6 +10,8 @@
  *     xrl_encode                 Section 3.4    Eq. 6 -> L x Eq. 7 -> Eq. 8
  *     xrl_policy_value           Section 3.3.2  policy / value MLPs, padded action space,
  *                                Section 3.3.3  invalid-action masking, No-Op, sampling
+ *     xrl_ppo_grad, xrl_gae      Section 3.3.4  the training step's objective (Eq. 3-5) and its gradient with
+ *                                               respect to every weight; advantage estimates
  *
  * Conventions
  *  - Plain C ABI.  Every function returns an xrl_status; nothing throws, aborts or traps.
