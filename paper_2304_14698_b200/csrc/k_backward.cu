@@ -483,8 +483,10 @@ k_gwt_mma(const bf16* __restrict__ G, const bf16* __restrict__ W, float* __restr
   __shared__ __align__(128) bf16 Bs[128 * 64];      // [row k][64 n]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int wm = warp >> 1, wn = warp & 1;
-  const int k0 = blockIdx.y * 128;
-  const int tile0 = blockIdx.x * tiles_per_cta, ntiles = (rows + 127) / 128;
+  // consecutive CTAs take the column tiles of the same rows, so that the rows' second reading comes from L2
+  const int ncol = H / 128;
+  const int k0 = int(blockIdx.x % ncol) * 128;
+  const int tile0 = int(blockIdx.x / ncol) * tiles_per_cta, ntiles = (rows + 127) / 128;
   const int nk = H / 64, total = min(tiles_per_cta, ntiles - tile0) * nk;
   float acc[2][8][4];
 #pragma unroll
@@ -1217,7 +1219,7 @@ int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* co
   dim3 g_atb_mma(unsigned(H / 128), unsigned(H / 128), unsigned((N + chunk_mma - 1) / chunk_mma));
   const int row_tiles = (N + 127) / 128;
   const int gwt_tpc = int64_t(row_tiles) * (H / 128) >= int64_t(kGwtTiles) * 4 * kNumSMs ? kGwtTiles : 1;
-  dim3 g_gwt_mma(unsigned((row_tiles + gwt_tpc - 1) / gwt_tpc), unsigned(H / 128));
+  dim3 g_gwt_mma(unsigned((row_tiles + gwt_tpc - 1) / gwt_tpc) * unsigned(H / 128));
   const int NF = H / 32;
   const bool rows_kernels = (32 % K == 0) && (NF == 1 || NF == 2 || NF == 4 || NF == 8 || NF == 16);
   // bf16 models of hidden 128, 256 or 512 take both products on the tensor cores, from a bf16 copy of dz
