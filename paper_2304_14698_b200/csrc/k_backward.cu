@@ -379,13 +379,16 @@ k_scores_bwd_rows(ZView<T> zv, const float* __restrict__ ds_src, const float* __
 template <typename TA>
 __global__ void __launch_bounds__(256)
 k_atb(const TA* __restrict__ A, int lda, const float* __restrict__ Bm, int ldb, float* __restrict__ Cout, int ldc,
-      int rows, int Ka, int Nb, int rows_per_chunk) {
+      int rows, int Ka, int Nb, int rows_per_chunk, float* __restrict__ colsum_out) {
   __shared__ float As[16][64 + 1];
   __shared__ float Bs[16][64 + 1];
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
   const int a0 = blockIdx.x * 64, b0 = blockIdx.y * 64;
   const int r_begin = blockIdx.z * rows_per_chunk, r_end = min(rows, r_begin + rows_per_chunk);
   float acc[4][4] = {};
+  // with colsum_out the first row of CTAs also sums B's columns (the bias gradient that goes with the product)
+  const bool sums = colsum_out != nullptr && blockIdx.x == 0 && ty == 0;
+  float csum[4] = {0.f, 0.f, 0.f, 0.f};
   for (int r0 = r_begin; r0 < r_end; r0 += 16) {
     for (int t = tid; t < 16 * 64; t += 256) {
       const int rr = t >> 6, cc = t & 63;
@@ -403,8 +406,17 @@ k_atb(const TA* __restrict__ A, int lda, const float* __restrict__ Bm, int ldb, 
       for (int u = 0; u < 4; ++u)
 #pragma unroll
         for (int v = 0; v < 4; ++v) acc[u][v] = fmaf(a[u], b[v], acc[u][v]);
+      if (sums) {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) csum[v] += b[v];
+      }
     }
     __syncthreads();
+  }
+  if (sums) {
+#pragma unroll
+    for (int v = 0; v < 4; ++v)
+      if (b0 + tx * 4 + v < Nb && csum[v] != 0.f) atomicAdd(&colsum_out[b0 + tx * 4 + v], csum[v]);
   }
 #pragma unroll
   for (int u = 0; u < 4; ++u)
@@ -758,7 +770,7 @@ k_embed_bwd(const float* __restrict__ xs, const int32_t* __restrict__ op, const 
 // ---- the heads' MLPs: Linear(in, hid), ReLU, [Linear(hid, hid2), ReLU,] Linear(last, 1) ---------------------
 // One CTA per input row.  The forward keeps the hidden activations; the reverse pass turns d(out) into the
 // gradients of the hidden pre-activations (d1, d2) and of the input (dx).  The weights' gradients are
-// products of those per-row buffers (X^T D1, Y1^T D2, ...), taken afterwards by k_atb / k_colsum.
+// products of those per-row buffers (X^T D1, Y1^T D2, ...), taken afterwards by k_atb (which also sums the columns of D for the biases).
 struct MlpW { const float *W1, *b1, *Wh, *bh, *w2, *b2; int hid, hid2; };
 
 __device__ float block_sum_f(float v, float* scratch) {       // blockDim a power of two
@@ -1043,46 +1055,25 @@ int chunk_rows(int64_t rows, int at_least) {
   return int(std::max<int64_t>(at_least, need));
 }
 
-// out[c] += sum over rows of M[r][c]
-__global__ void __launch_bounds__(256)
-k_colsum(const float* __restrict__ M, int ld, float* __restrict__ out, int rows, int cols, int rows_per_chunk) {
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= cols) return;
-  const int r0 = blockIdx.y * rows_per_chunk, r1 = min(rows, r0 + rows_per_chunk);
-  float s = 0.f;
-  for (int r = r0; r < r1; ++r) s += M[size_t(r) * ld + c];
-  if (s != 0.f) atomicAdd(&out[c], s);
-}
-
 void atb_f32(const float* A, int lda, const float* Bm, int ldb, float* Cout, int ldc, int rows, int Ka, int Nb,
-             cudaStream_t st) {
+             cudaStream_t st, float* colsum_out = nullptr) {
   if (rows <= 0 || Ka <= 0 || Nb <= 0) return;
   const int chunk = chunk_rows(rows, 1024);
   dim3 g(unsigned((Ka + 63) / 64), unsigned((Nb + 63) / 64), unsigned((rows + chunk - 1) / chunk));
-  k_atb<float><<<g, 256, 0, st>>>(A, lda, Bm, ldb, Cout, ldc, rows, Ka, Nb, chunk);
+  k_atb<float><<<g, 256, 0, st>>>(A, lda, Bm, ldb, Cout, ldc, rows, Ka, Nb, chunk, colsum_out);
 }
-void colsum(const float* M, int ld, float* out, int rows, int cols, cudaStream_t st) {
-  if (rows <= 0 || cols <= 0) return;
-  const int chunk = chunk_rows(rows, 512);
-  dim3 g(unsigned((cols + 255) / 256), unsigned((rows + chunk - 1) / chunk));
-  k_colsum<<<g, 256, 0, st>>>(M, ld, out, rows, cols, chunk);
-}
-
 // weights' gradients of one head from its per-row buffers; returns the launches
 int mlp_weight_grads(const float* X, int in, int rows, int hid, int hid2, const float* Y1, const float* Y2,
                      const float* D1, const float* D2, const float* dout, float* gW1, float* gb1, float* gWh,
                      float* gbh, float* gw2, float* gb2, cudaStream_t st) {
   int n = 0;
-  atb_f32(X, in, D1, hid, gW1, hid, rows, in, hid, st); ++n;
-  colsum(D1, hid, gb1, rows, hid, st); ++n;
+  atb_f32(X, in, D1, hid, gW1, hid, rows, in, hid, st, gb1); ++n;
   if (hid2 > 0) {
-    atb_f32(Y1, hid, D2, hid2, gWh, hid2, rows, hid, hid2, st); ++n;
-    colsum(D2, hid2, gbh, rows, hid2, st); ++n;
-    atb_f32(Y2, hid2, dout, 1, gw2, 1, rows, hid2, 1, st); ++n;
+    atb_f32(Y1, hid, D2, hid2, gWh, hid2, rows, hid, hid2, st, gbh); ++n;
+    atb_f32(Y2, hid2, dout, 1, gw2, 1, rows, hid2, 1, st, gb2); ++n;
   } else {
-    atb_f32(Y1, hid, dout, 1, gw2, 1, rows, hid, 1, st); ++n;
+    atb_f32(Y1, hid, dout, 1, gw2, 1, rows, hid, 1, st, gb2); ++n;
   }
-  colsum(dout, 1, gb2, rows, 1, st); ++n;
   return n;
 }
 
@@ -1179,8 +1170,7 @@ int launch_ppo_heads(const Dims& d, const DevWeights& w, float* grad_base, const
   k_graph_bwd<<<B, 256, sizeof(float) * (H + 2 * Hm + 2 * Hm2), st>>>(emb, dlogit, pm, py1, py2, demb, w.Wg, pd1,
                                                                        pd2, dpre, dr, d.H);
   ++n;
-  atb_f32(U, int(HU), dpre, d.H, gp(w.Wg), d.H, B, int(HU), d.H, st); ++n;
-  colsum(dpre, d.H, gp(w.bg), B, d.H, st); ++n;
+  atb_f32(U, int(HU), dpre, d.H, gp(w.Wg), d.H, B, int(HU), d.H, st, gp(w.bg)); ++n;
   n += mlp_weight_grads(emb, d.H, B, d.Hm, d.Hm2, py1, py2, pd1, pd2, dlogit, gp(w.pW1), gp(w.pb1), gp(w.pWh),
                         gp(w.pbh), gp(w.pw2), gp(w.pb2), st);
   n += mlp_weight_grads(eb.vu, 2 * d.H, num_envs, d.Hm, d.Hm2, eb.vy1, eb.vy2, eb.vd1, eb.vd2, eb.vdout, gp(w.vW1),
@@ -1257,7 +1247,7 @@ int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* co
       k_atb_mma<<<g_atb_mma, 256, 0, st>>>(static_cast<const bf16*>(h_in), dzb, gW, N, H, chunk_mma);          \
       k_gwt_mma<<<g_gwt_mma, 256, 0, st>>>(dzb, static_cast<const bf16*>(lw.W), dh_in, N, H, gwt_tpc);                  \
     } else {                                                                                                   \
-      k_atb<TY_><<<g_atb, 256, 0, st>>>(static_cast<const TY_*>(h_in), H, dz, H, gW, H, N, H, H, chunk);       \
+      k_atb<TY_><<<g_atb, 256, 0, st>>>(static_cast<const TY_*>(h_in), H, dz, H, gW, H, N, H, H, chunk, nullptr);       \
       k_gwt<TY_><<<g_gwt, 256, 0, st>>>(dz, static_cast<const TY_*>(lw.W), dh_in, N, H, H);                    \
     }                                                                                                          \
   } while (0)
