@@ -1145,11 +1145,9 @@ int launch_ppo_heads(const Dims& d, const DevWeights& w, float* grad_base, const
   const MlpW vm{w.vW1, w.vb1, w.vWh, w.vbh, w.vw2, w.vb2, d.Hm, d.Hm2};
   const MlpW pm{w.pW1, w.pb1, w.pWh, w.pbh, w.pw2, w.pb2, d.Hm, d.Hm2};
   int n = 0;
-  // a bad action leaves its environment's rows unwritten: start them from zero
-  cudaMemsetAsync(demb, 0, sizeof(float) * size_t(B) * H, st);
-  cudaMemsetAsync(dlogit, 0, sizeof(float) * size_t(B), st);
-  cudaMemsetAsync(eb.vu, 0, sizeof(float) * size_t(p - eb.vu), st);
-  cudaMemsetAsync(U, 0, sizeof(float) * size_t(B) * HU, st);
+  // one clearing of everything taken above: the per-graph sums are accumulated with atomics, and a bad action
+  // leaves its environment's rows unwritten
+  cudaMemsetAsync(ws, 0, sizeof(float) * size_t(p - ws), st);
   if (N > 0) {
     const int rows_per_cta = 64;
     const unsigned grid = unsigned((N + rows_per_cta - 1) / rows_per_cta);
