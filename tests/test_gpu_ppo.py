@@ -175,6 +175,17 @@ def test_an_action_the_mask_excludes_is_reported(xo):
         with pytest.raises(xrl.XrlError) as e:
             xrl.xrl_ppo_grad(ag.ctx, ag.batch, torch.from_numpy(b["mask"]).cuda(), action, z, z, z, None, grad)
         assert e.value.status == 1
+        # not recordable: inside a recording bracket the call is refused and nothing is enqueued
+        mask_d = torch.from_numpy(b["mask"]).cuda()     # (copies are not allowed inside the bracket)
+        torch.cuda.synchronize()
+        xrl.xrl_graph_begin(ag.ctx)
+        with pytest.raises(xrl.XrlError) as e:
+            xrl.xrl_ppo_grad(ag.ctx, ag.batch, mask_d, action, z, z, z, loss, grad)
+        assert xrl.STATUS_NAMES[e.value.status] == "XRL_ERR_STATE"
+        try:
+            xrl.xrl_graph_launch(ag.ctx)            # ends the (empty) recording
+        except xrl.XrlError:
+            pass
     finally:
         ag.close()
 
