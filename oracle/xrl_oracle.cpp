@@ -101,6 +101,11 @@ Weights slice(const Model& m, const float* blob) {
 // A weight as the model stores it: Eq. 6 and Eq. 7 matrices live in bf16 when dtype = 1.
 double stored(const Model& m, float w) { return m.dtype == 1 ? round_bf16(w) : double(w); }
 
+// An input feature (a node's shape features, an edge's attributes) as the model stores it: the caller
+// hands over arbitrary reals (Section 3.3.2: tensor shapes divided by a constant); a bf16 model keeps
+// them in bf16, so they are rounded here, once, before anything is computed from them.
+double stored_input(const Model& m, float v) { return m.dtype == 1 ? round_bf16(v) : double(v); }
+
 // Encode one graph (nodes [lo, hi) of the packed batch).  Writes its H-vector to `emb`.
 void encode_graph(const Model& m, const Weights& w, int32_t lo, int32_t hi,
                   const int32_t* rowptr, const int32_t* col, const int32_t* op,
@@ -131,9 +136,9 @@ void encode_graph(const Model& m, const Weights& w, int32_t lo, int32_t hi,
     for (int s = 0; s < F0; ++s) x[s] = 0.0;
     for (int e = rowptr[gi]; e < rowptr[gi + 1]; ++e)
       for (int s = 0; s < S; ++s)
-        x[s] += edge_attr ? double(edge_attr[size_t(eid[e]) * S + s]) : double(shape[size_t(col[e]) * S + s]);
+        x[s] += stored_input(m, edge_attr ? edge_attr[size_t(eid[e]) * S + s] : shape[size_t(col[e]) * S + s]);
     x[S + op[gi]] = 1.0;
-    for (int s = 0; s < S; ++s) x[S + T + s] = double(shape[size_t(gi) * S + s]);
+    for (int s = 0; s < S; ++s) x[S + T + s] = stored_input(m, shape[size_t(gi) * S + s]);
     for (int c = 0; c < H; ++c) {
       double acc = 0.0;
       for (int s = 0; s < F0; ++s) acc += x[s] * W0s[size_t(s) * H + c];
@@ -304,9 +309,9 @@ void forward_tape(const Model& m, const Weights& w, int32_t lo, int32_t hi, cons
     double* x = &tp.x0[size_t(i) * F0];
     for (int e = rowptr[gi]; e < rowptr[gi + 1]; ++e)
       for (int s = 0; s < S; ++s)
-        x[s] += edge_attr ? double(edge_attr[size_t(eid[e]) * S + s]) : double(shape[size_t(col[e]) * S + s]);
+        x[s] += stored_input(m, edge_attr ? edge_attr[size_t(eid[e]) * S + s] : shape[size_t(col[e]) * S + s]);
     x[S + op[gi]] = 1.0;
-    for (int s = 0; s < S; ++s) x[S + T + s] = double(shape[size_t(gi) * S + s]);
+    for (int s = 0; s < S; ++s) x[S + T + s] = stored_input(m, shape[size_t(gi) * S + s]);
     for (int c = 0; c < H; ++c) {
       double acc = double(w.b0[c]);
       for (int s = 0; s < F0; ++s) acc += x[s] * stored(m, w.W0[size_t(s) * H + c]);

@@ -27,13 +27,15 @@ def node_update(g, W, m):
     (g["edge_attr"], one row per edge of the input list) the first block is the incidence matrix (consumer
     x edge) times the attributes instead."""
     A = adjacency(g)
-    shp = g["shape"].astype(np.float64)
+    # a bf16 model stores its input features in bf16: arbitrary reals are rounded once, up front
+    as_stored = bf16_round if m["dtype"] == "bf16" else (lambda a: np.asarray(a, dtype=np.float64))
+    shp = as_stored(g["shape"])
     onehot = np.eye(m["T"])[g["op"]]
     if g.get("edge_attr") is not None:
         n, ne = len(g["op"]), len(g["edge_dst"])
         Inc = np.zeros((n, ne))
         Inc[np.asarray(g["edge_dst"]), np.arange(ne)] = 1.0
-        agg = Inc @ np.asarray(g["edge_attr"], dtype=np.float64)
+        agg = Inc @ as_stored(g["edge_attr"])
     else:
         agg = A @ shp
     X = np.concatenate([agg, onehot, shp], axis=1)

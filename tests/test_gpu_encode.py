@@ -281,3 +281,27 @@ def test_results_are_bitwise_reproducible():
     b = gpu_util.run_gpu(batch, blob, sample=True, seed=3, step=9, where="device")
     for k in ("emb", "probs", "value", "action"):
         assert np.array_equal(a[k], b[k]), k
+
+
+def test_bf16_model_takes_shape_features_off_the_bf16_grid(xo):
+    """Section 3.3.2: shape features are arbitrary reals.  A bf16 model gets float32 features that are not
+    bf16 values, graph by graph through xrl_pack; both sides round them to the storage type on their own."""
+    import torch
+    batch = configs.make_batch(3, candidates=7)
+    m = batch["model"]
+    rng = np.random.default_rng(12)
+    batch["shape"] = (batch["shape"] + rng.uniform(1e-4, 3e-3, size=batch["shape"].shape)).astype(np.float32)
+    assert not np.array_equal(batch["shape"], dags.round_to_bf16_grid(batch["shape"]))
+    blob, _ = gpu_util.default_weights(batch, 1003)
+    want = xo.forward(m, blob, batch)
+    ag = gpu_util.make_agent(batch)
+    try:
+        ag.set_weights(blob)
+        ag.pack_graphs(dags.split(batch), batch["env_off"])
+        o = ag.forward(torch.from_numpy(batch["mask"]).cuda())
+        torch.cuda.synchronize()
+        assert ag.device_status() == 0
+        for k in ("emb", "probs", "value"):
+            gpu_util.assert_close(o[k].cpu().numpy(), want[k], "bf16", k)
+    finally:
+        ag.close()

@@ -41,6 +41,38 @@ def test_encoder_matches_dense_bruteforce(xo, dtype):
         np.testing.assert_allclose(out["emb"][gi], want, rtol=1e-12, atol=1e-12)
 
 
+def test_bf16_model_rounds_its_own_input_features(xo):
+    """Section 3.3.2: shape features and edge attributes are tensor shapes divided by a constant, i.e.
+    arbitrary reals.  A bf16 model stores them in bf16, so features given off the bf16 grid must be rounded
+    (to nearest, ties to even) before Eq. 6 uses them: the dense restatement does its own rounding, the
+    result differs from the unrounded one, and equals what on-grid copies of the same features give."""
+    m = dict(M_SMALL, dtype="bf16")
+    _, W = configs.make_weights(m, 11)
+    graphs = _tiny_graphs(21)
+    rng = np.random.default_rng(4)
+    for g in graphs:
+        g["shape"] = (g["shape"] + rng.uniform(1e-4, 3e-3, size=g["shape"].shape)).astype(np.float32)
+        assert not np.array_equal(g["shape"], dags.round_to_bf16_grid(g["shape"]))
+    _, _, out = _run(xo, m, W, graphs)
+    on_grid = [dict(g, shape=dense_ref.bf16_round(g["shape"]).astype(np.float32)) for g in graphs]
+    _, _, out_grid = _run(xo, m, W, on_grid)
+    np.testing.assert_array_equal(out["emb"], out_grid["emb"])
+    unrounded = dict(m, dtype="fp32")
+    for gi, g in enumerate(graphs):
+        want = dense_ref.encode_graph(g, W, m)
+        np.testing.assert_allclose(out["emb"][gi], want, rtol=1e-12, atol=1e-12)
+        W_r = dict(W, W0=dense_ref.bf16_round(W["W0"]), **{f"W{l}": dense_ref.bf16_round(W[f"W{l}"]) for l in (1, 2)})
+        assert not np.allclose(want, dense_ref.encode_graph(g, W_r, unrounded), rtol=1e-9, atol=1e-12)
+    # the same for attributes that live on the edges
+    eg = [dict(g) for g in graphs]
+    for g in eg:
+        a = dags.tensor_shape_attributes(dags.make_rng(len(g["edge_src"])), len(g["edge_src"]), 8, False)
+        g["edge_attr"] = (a + rng.uniform(1e-4, 3e-3, size=a.shape)).astype(np.float32)
+    _, _, out_e = _run(xo, m, W, eg)
+    for gi, g in enumerate(eg):
+        np.testing.assert_allclose(out_e["emb"][gi], dense_ref.encode_graph(g, W, m), rtol=1e-12, atol=1e-12)
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_neighbourhood_both_ways_matches_dense_bruteforce(xo, dtype):
     """Eq. 7 with the consumers of a node among its neighbours: dense row softmax weighted by A + A^T + I

@@ -21,20 +21,23 @@ MUTATIONS = [
     ("layer bias dropped", "acc = relu(acc + double(w.b[l][c]));", "acc = relu(acc);"),
     ("self term dropped", "for (int t = 0; t <= deg; ++t) { al[t] = std::exp(sc[t] - mx); sum += al[t]; }",
      "for (int t = 0; t <= deg; ++t) { al[t] = (t < deg || deg == 0) ? std::exp(sc[t] - mx) : 0.0; sum += al[t]; }"),
-    ("own shape block dropped", "x[S + T + s] = double(shape[size_t(gi) * S + s]);", "x[S + T + s] = 0.0;"),
-    ("edge aggregate takes the consumer's shape", ": double(shape[size_t(col[e]) * S + s]);",
-     ": double(shape[size_t(gi) * S + s]);"),
+    ("own shape block dropped", "x[S + T + s] = stored_input(m, shape[size_t(gi) * S + s]);", "x[S + T + s] = 0.0;"),
+    ("edge aggregate takes the consumer's shape", ": shape[size_t(col[e]) * S + s]);",
+     ": shape[size_t(gi) * S + s]);"),
     ("readout mean instead of sum", "for (int c = 0; c < m.Dg; ++c) u[H + c] = g_attr ? g_attr[c] : 0.0;",
      "for (int c = 0; c < H; ++c) u[c] /= double(n > 0 ? n : 1);\n  for (int c = 0; c < m.Dg; ++c) u[H + c] = g_attr ? g_attr[c] : 0.0;"),
     ("global attribute ignored", "u[H + c] = g_attr ? g_attr[c] : 0.0;", "u[H + c] = 0.0;"),
     ("bf16 truncation instead of rounding", "u += 0x7FFFu + lsb;", "u += 0u * lsb;"),
-    ("edge attributes read in CSR slot order", "double(edge_attr[size_t(eid[e]) * S + s])",
-     "double(edge_attr[size_t(e) * S + s])"),
+    ("edge attributes read in CSR slot order", "edge_attr ? edge_attr[size_t(eid[e]) * S + s]",
+     "edge_attr ? edge_attr[size_t(e) * S + s]"),
     ("consumers listed under the wrong node", "nbl[col[e] - lo].push_back(i);", "nbl[i].push_back(col[e] - lo);"),
     ("second hidden layer without its ReLU", "out += relu(acc) * double(w2[c]);", "out += acc * double(w2[c]);"),
     ("second hidden layer's bias dropped", "double acc = double(bh[c]);", "double acc = 0.0;"),
     ("second hidden layer reads the first layer transposed", "acc += y1[k] * double(Wh[size_t(k) * hid2 + c]);",
      "acc += y1[k] * double(Wh[size_t(c) * hid + k]);"),
+    ("input features of a bf16 model left unrounded",
+     "double stored_input(const Model& m, float v) { return m.dtype == 1 ? round_bf16(v) : double(v); }",
+     "double stored_input(const Model& m, float v) { return double(v); }"),
     ("masked candidates counted in the value head's mean", "if (mask[size_t(e) * A_max + a]) {\n        ++nv;",
      "{\n        ++nv;"),
 ]
@@ -56,7 +59,8 @@ def _pins_hold(xo):
         m = dict(T=6, S=8, H=16, K=2, L=2, Hm=8, Dg=2, dtype=dtype, A_max=4)
         _, W = configs.make_weights(m, 11)
         rng = dags.make_rng(5)
-        graphs = [dags.random_dag(rng, 12, 6, 8, dtype == "bf16", window=6) for _ in range(4)]
+        # shape features off the bf16 grid: the bf16 model has to round them itself
+        graphs = [dags.random_dag(rng, 12, 6, 8, False, window=6) for _ in range(4)]
         b = dags.flatten(graphs, [0, len(graphs)], 4)
         st, p = xo.pack(b)
         if st != 0:
@@ -81,24 +85,25 @@ def _pins_hold(xo):
     for gi, g in enumerate(graphs):
         if not np.allclose(out["emb"][gi], dense_ref.encode_graph(g, W, m), rtol=1e-10, atol=1e-11):
             return False
-    # attributes on the edges, edge lists shuffled
-    m = dict(T=6, S=8, H=16, K=2, L=1, Hm=8, Dg=1, dtype="fp32", A_max=4)
-    _, W = configs.make_weights(m, 19)
-    rng = dags.make_rng(6)
-    graphs = [dags.random_dag(rng, 12, 6, 8, False, window=6) for _ in range(3)]
-    nrng = np.random.default_rng(8)
-    for g in graphs:
-        perm = nrng.permutation(len(g["edge_src"]))
-        g["edge_src"], g["edge_dst"] = g["edge_src"][perm], g["edge_dst"][perm]
-        g["edge_attr"] = dags.tensor_shape_attributes(rng, len(perm), 8, False)
-    b = dags.flatten(graphs, [0, len(graphs)], 4)
-    st, p = xo.pack(b)
-    if st != 0:
-        return False
-    out = xo.encode(m, configs.pack_weights(m, W), b, p)
-    for gi, g in enumerate(graphs):
-        if not np.allclose(out["emb"][gi], dense_ref.encode_graph(g, W, m), rtol=1e-10, atol=1e-11):
+    # attributes on the edges (off the bf16 grid for the bf16 model too), edge lists shuffled
+    for dtype in ("fp32", "bf16"):
+        m = dict(T=6, S=8, H=16, K=2, L=1, Hm=8, Dg=1, dtype=dtype, A_max=4)
+        _, W = configs.make_weights(m, 19)
+        rng = dags.make_rng(6)
+        graphs = [dags.random_dag(rng, 12, 6, 8, False, window=6) for _ in range(3)]
+        nrng = np.random.default_rng(8)
+        for g in graphs:
+            perm = nrng.permutation(len(g["edge_src"]))
+            g["edge_src"], g["edge_dst"] = g["edge_src"][perm], g["edge_dst"][perm]
+            g["edge_attr"] = dags.tensor_shape_attributes(rng, len(perm), 8, False)
+        b = dags.flatten(graphs, [0, len(graphs)], 4)
+        st, p = xo.pack(b)
+        if st != 0:
             return False
+        out = xo.encode(m, configs.pack_weights(m, W), b, p)
+        for gi, g in enumerate(graphs):
+            if not np.allclose(out["emb"][gi], dense_ref.encode_graph(g, W, m), rtol=1e-10, atol=1e-11):
+                return False
     # heads with two hidden layers (widths 7 and 7) against the brute-force MLP, one candidate masked
     m = dict(T=6, S=8, H=16, K=2, L=0, Hm=7, Hm2=7, Dg=1, dtype="fp32", A_max=3)
     blob, W = configs.make_weights(m, 17)
