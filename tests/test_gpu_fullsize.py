@@ -1,7 +1,9 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py times (device-resident
-inputs, Agent.step).  The packed arrays are compared bit for bit in full; graph embeddings are
-compared on sampled graphs the oracle encodes one by one; the policy is checked through its
-structural properties and through log-probability differences of the sampled graphs."""
+inputs, Agent.step).  For the two largest workloads (the 1,024-action step and the 64-environment
+rollout batch) the oracle runs the whole batch once per module; the packed arrays are then compared bit
+for bit and every graph embedding, every probability of every environment and slot, and every value
+estimate element by element within the bf16 tolerance, for the full encoder and for the delta encoder.
+The draw is exact given the probabilities the GPU reports."""
 import numpy as np
 import pytest
 
@@ -9,6 +11,17 @@ from workloads import configs
 import gpu_util
 
 pytestmark = pytest.mark.gpu
+
+_cache = {}
+
+
+def _reference(xo, cfg_id):
+    """The oracle's whole step on workload `cfg_id` at full size (computed once, kept for the module)."""
+    if cfg_id not in _cache:
+        batch = configs.make_batch(cfg_id)
+        blob, _ = gpu_util.default_weights(batch, 1000 + cfg_id)
+        _cache[cfg_id] = (batch, blob, xo.forward(batch["model"], blob, batch))
+    return _cache[cfg_id]
 
 
 def _run_full(batch, blob, seed, step, delta=False):
@@ -35,63 +48,46 @@ def _run_full(batch, blob, seed, step, delta=False):
         ag.close()
 
 
-def _check(xo, cfg_id, n_sample, delta=False):
-    batch = configs.make_batch(cfg_id)
+def _check(xo, cfg_id, delta=False):
+    batch, blob, want = _reference(xo, cfg_id)
     m = batch["model"]
-    blob, _ = gpu_util.default_weights(batch, 1000 + cfg_id)
     got = _run_full(batch, blob, seed=cfg_id, step=3, delta=delta)
     assert got["status"] == 0
 
-    st, packed = xo.pack(batch)
-    assert st == 0
     for k in ("node_off", "edge_off", "seg_id", "graph_env", "rowptr", "col"):
-        assert np.array_equal(got["packed"][k], packed[k]), k
+        assert np.array_equal(got["packed"][k], want["packed"][k]), k
 
-    rng = np.random.default_rng(cfg_id)
-    env_off = batch["env_off"]
-    e = int(rng.integers(0, len(env_off) - 1))
-    cur = int(env_off[e])
-    C = int(env_off[e + 1]) - cur - 1
-    valid = np.flatnonzero(batch["mask"][e, :C])
-    picks = rng.choice(valid, size=min(n_sample - 1, len(valid)), replace=False)
-    sel = np.array([cur] + [cur + 1 + int(a) for a in picks], dtype=np.int32)
-    want = xo.encode(m, blob, batch, packed, sel=sel)["emb"]
-    gpu_util.assert_close(got["emb"][sel], want, m["dtype"], f"cfg{cfg_id} sampled graph_emb")
+    what = f"workload {cfg_id}{' (delta)' if delta else ''} "
+    gpu_util.assert_close(got["emb"], want["emb"], m["dtype"], what + "graph_emb, every graph")
+    gpu_util.assert_close(got["probs"], want["probs"], m["dtype"], what + "probs, every environment and slot")
+    gpu_util.assert_close(got["value"], want["value"], m["dtype"], what + "value, every environment")
 
     probs = got["probs"]
     A = m["A_max"]
-    full_mask = np.concatenate([batch["mask"], np.ones((len(env_off) - 1, 1), np.uint8)], axis=1)
+    n_env = len(batch["env_off"]) - 1
+    full_mask = np.concatenate([batch["mask"], np.ones((n_env, 1), np.uint8)], axis=1)
     assert np.all(probs[full_mask == 0] == 0.0)
     assert np.all(probs[full_mask == 1] >= 0.0)
     assert np.all(np.abs(probs.sum(axis=1) - 1.0) < 1e-4)
     assert np.all(probs[:, A] > 0)
-    assert np.all(np.isfinite(got["value"]))
-    # log-probability differences against the oracle's logits of the sampled graphs
-    mini = {"env_off": np.array([0, len(sel)], np.int32), "mask": np.ones((1, len(sel) - 1), np.uint8)}
-    st, logits, _, _ = xo.policy_value(dict(m, A_max=len(sel) - 1), blob, mini, want)
-    assert st == 0
-    for i, a in enumerate(picks):
-        lhs = np.log(probs[e, a]) - np.log(probs[e, A])
-        rhs = logits[0, i] - logits[0, -1]
-        assert abs(lhs - rhs) < 5e-2, (a, lhs, rhs)
     # the draw is exact given the probabilities the GPU reports
     assert np.array_equal(got["action"], xo.sample(probs, cfg_id, 3))
 
 
-def test_large_step_full_size(xo):
-    _check(xo, 4, 6)
+def test_large_step_full_size_every_output(xo):
+    _check(xo, 4)
 
 
-def test_rollout_batch_full_size(xo):
-    _check(xo, 5, 6)
+def test_large_step_full_size_delta_encoding_every_output(xo):
+    _check(xo, 4, delta=True)
 
 
-def test_large_step_full_size_delta_encoding(xo):
-    _check(xo, 4, 6, delta=True)
+def test_rollout_batch_full_size_every_output(xo):
+    _check(xo, 5)
 
 
-def test_rollout_batch_full_size_delta_encoding(xo):
-    _check(xo, 5, 6, delta=True)
+def test_rollout_batch_full_size_delta_encoding_every_output(xo):
+    _check(xo, 5, delta=True)
 
 
 def test_cnn_step_full_size_every_output(xo):
