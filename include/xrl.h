@@ -140,7 +140,10 @@ xrl_status xrl_get_weights(const xrl_ctx* ctx, void* host_blob, size_t bytes);
  * shape[N x S].  If *out is NULL a batch sized to the context's capacities is allocated;
  * otherwise the existing batch is re-packed in place with no allocation.
  * Graph validity (ids in range, no self edge, op < T) is checked on the device: a violation
- * sets XRL_ERR_BAD_GRAPH in the device status word and the batch must not be encoded. */
+ * sets XRL_ERR_BAD_GRAPH in the device status word; the offending edges are left out and the slots
+ * they would have taken are filled with a valid node id, so encoding such a batch anyway reads only
+ * inside the arrays (nothing faults), but its results describe no graph the caller gave: read the
+ * status word before trusting them. */
 xrl_status xrl_pack(xrl_ctx* ctx, const xrl_graph* graphs, int32_t num_graphs,
                     const int32_t* env_off, int32_t num_envs, void* stream, xrl_batch** out);
 
@@ -174,8 +177,8 @@ xrl_status xrl_batch_info(const xrl_batch* batch, int64_t* num_nodes, int64_t* n
 xrl_status xrl_batch_export(const xrl_batch* batch, int32_t* rowptr, int32_t* col, int32_t* seg_id,
                             int32_t* node_off, int32_t* edge_off, int32_t* graph_env);
 
-/* Attributes on the edges (contexts created with edge_attributes = 1; Section 3.3.2: "for edges, we use
- * the corresponding tensor shape as its attributes", padded and divided by a constant).  edge_attr is
+/* Attributes on the edges (contexts created with edge_attributes = 1; Section 3.3.2: an edge's attribute is
+ * the shape of the tensor it carries, padded to rank 4 and divided by a constant).  edge_attr is
  * [E x S] in the storage type (float, or bf16 bits), one row per edge in the order of the edge lists given
  * to the pack call, HOST or DEVICE according to `where`; the library brings the rows into the order of the
  * packed CSR (one gather pass, queued on `stream` after the packing) and Eq. 6 then sums, for each node, the
@@ -338,15 +341,18 @@ xrl_status xrl_launch_counts(const xrl_ctx* ctx, int64_t* pack, int64_t* encode,
  * anything larger is refused with XRL_ERR_CAPACITY before any work is queued (the paper's own
  * steps, 13-50 candidates of a few hundred to a few thousand operators, fit).
  *
- * Arguments: n_nodes, n_edges [num_graphs] and env_off [num_envs + 1] are HOST (read before the
- * call returns); op [N], edge_src [E], edge_dst [E] are DEVICE inputs with the meaning they have
+ * Arguments: n_nodes, n_edges [num_graphs] and env_off [num_envs + 1] are HOST; they are validated
+ * before the call returns and copied to the device with an asynchronous copy on `stream` (ordinary
+ * pageable arrays are fully read by then; page-locked arrays must stay unchanged until the stream has
+ * passed the call); op [N], edge_src [E], edge_dst [E] are DEVICE inputs with the meaning they have
  * in xrl_pack_flat; node_off [B+1], edge_off [B+1], seg_id [N], graph_env [B], rowptr [N+1],
  * col [E] and device_status [1] are DEVICE outputs owned by the caller.  device_status receives
  * XRL_OK or XRL_ERR_BAD_GRAPH once the stream has run the work.  `device` is the CUDA device the
  * pointers belong to; the call makes it current.
  *
  * The first call on each device looks up the device address of the built-in array once
- * (cudaGetSymbolAddress); make that first call before you begin any stream capture.  All calls on
+ * (cudaGetSymbolAddress); make that first call before you begin any stream capture, and from one
+ * thread only (first calls on the same device must not run concurrently).  All calls on
  * a device share the one array and it keeps whatever the previous call left there (the kernels
  * re-zero the counters they need), so two calls must never overlap on the GPU: issue them on one
  * stream, or order them with events.  Overlapping calls race and corrupt each other's result. */

@@ -280,6 +280,17 @@ k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ e
   // the last graph of a partial launch closes its last row itself (the next graph's CTA, which writes the
   // same value as its first row start, may run much later)
   else if (blockIdx.x == gridDim.x - 1 && tid == 0) rowptr[nb + n] = edge_off[g + 1];
+  // A malformed graph (already reported through `status`) keeps fewer edges than it was given slots for:
+  // the slots left over sit at the end of the last row before the next graph's rows and nobody writes them.
+  // They get a valid node id (the graph's first node) so that a batch that is encoded although it was
+  // reported bad still reads inside the arrays.
+  if (deg[n] < m) {
+    const int32_t fill = n > 0 ? nb : 0;
+    for (int32_t i = deg[n] + tid; i < m; i += NT) {
+      col[eb + i] = fill;
+      if (eid) eid[eb + i] = eb;
+    }
+  }
   // scatter (edge id, global producer) into the rows, slot order as the atomics hand it out
   for (int32_t e0 = tid; e0 < m; e0 += 4 * NT) {
     int32_t s[4], t[4];

@@ -69,7 +69,9 @@ k_embed(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
 #pragma unroll
       for (int s = 0; s < kS; ++s) x[kS + s] = f[s];
     }
-    const T* lookup = W0 + size_t(kS + __ldg(op + row)) * H;
+    // an operator id outside the table was reported by the packer; clamped here so that nothing is read
+    // outside W0 if the caller encodes such a batch anyway
+    const T* lookup = W0 + size_t(kS + min(max(__ldg(op + row), 0), Tn - 1)) * H;
     T* out = h + size_t(out_row - win.win_base) * H;
 #pragma unroll
     for (int v = 0; v < VPL; ++v) {

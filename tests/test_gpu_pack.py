@@ -103,6 +103,40 @@ def test_pack_reports_bad_graphs_in_the_device_status(xo):
             ag.close()
 
 
+def test_malformed_graph_in_the_middle_leaves_only_valid_indices_and_can_be_encoded_safely(xo):
+    """A bad edge in a graph that is not the last one: its slot stays unused, so the graph's last row spans a
+    slot no edge was written to.  The packed arrays must still hold only valid indices (row pointers
+    monotone, every producer id inside the batch), an operator id outside the table must not index outside
+    the weights, and encoding the batch anyway must come back with the packer's status and finite memory
+    traffic only (nothing to observe but that the calls return and the status is the packer's)."""
+    import torch
+    import paper_2304_14698_b200 as xrl
+    for cfg, kw in [(1, {}), (3, dict(candidates=5))]:
+        base = configs.make_batch(cfg, **kw)
+        b = {kk: (v.copy() if isinstance(v, np.ndarray) else v) for kk, v in base.items()}
+        e_mid = int(b["n_edges"][:2].sum()) + 3                  # an edge of the third graph
+        b["edge_src"][e_mid] = b["edge_dst"][e_mid]              # self edge: dropped by the packer
+        e2 = int(b["n_edges"][:4].sum()) + 1
+        b["edge_dst"][e2] = -5                                   # consumer out of range
+        b["op"][int(b["n_nodes"][:1].sum()) + 2] = 10 ** 6       # operator id far outside the table
+        N, E = int(b["n_nodes"].sum()), int(b["n_edges"].sum())
+        ag = gpu_util.make_agent(b)
+        try:
+            ag.set_weights(gpu_util.default_weights(base, 7)[0])
+            ag.batch = None
+            ag.pack(b)
+            got = xrl.xrl_batch_export(ag.batch)
+            assert np.all(np.diff(got["rowptr"]) >= 0) and got["rowptr"][0] == 0 and got["rowptr"][-1] <= E
+            reach = got["col"][:got["rowptr"][-1]]
+            assert np.all((reach >= 0) & (reach < N))
+            o = ag.forward(torch.from_numpy(b["mask"]).cuda())
+            torch.cuda.synchronize()
+            assert ag.device_status() == 2
+            assert o["emb"].shape[0] == b["num_graphs"]
+        finally:
+            ag.close()
+
+
 def test_pack_argument_and_capacity_errors():
     import paper_2304_14698_b200 as xrl
     b = configs.make_batch(1)
