@@ -21,12 +21,17 @@ namespace {
 
 constexpr int TW = 4;            // warps per CTA
 #ifndef XRL_AGG_GROUPS
-#define XRL_AGG_GROUPS 4
+#define XRL_AGG_GROUPS 2
 #endif
 #ifndef XRL_AGG_CTAS
 #define XRL_AGG_CTAS 5
 #endif
-constexpr int G = XRL_AGG_GROUPS;   // gather groups (of four rows) in flight per warp
+#ifndef XRL_AGG_GATHERS
+#define XRL_AGG_GATHERS 2
+#endif
+constexpr int G = XRL_AGG_GROUPS;   // gather groups in flight per warp
+constexpr int GQ = XRL_AGG_GATHERS; // gathers (of four rows each) per group: one barrier, one wait per group
+constexpr int GV = 4 * GQ;          // vectors (rows) per group
 constexpr int BR = 32;           // destination rows per block
 constexpr int ITEMS = 160;       // list capacity, a multiple of 4
 
@@ -34,11 +39,11 @@ constexpr int ITEMS = 160;       // list capacity, a multiple of 4
 // per group brings both; otherwise the pairs come from a second gather into `sc`.
 template <int K, bool MERGED> struct alignas(128) WarpSmem {
   static constexpr int ROW = MERGED ? 512 + 8 * K : 512;     // bytes per gathered row
-  uint8_t z[G][4][ROW];          // four gathered rows per group
-  float2 sc[MERGED ? 1 : G][4][K];   // their {s_src, s_dst} pairs (separate gather only)
+  uint8_t z[G][GV][ROW];         // the gathered rows of a group
+  float2 sc[MERGED ? 1 : G][GV][K];  // their {s_src, s_dst} pairs (separate gather only)
   unsigned long long bar[G];
   int32_t rp[BR + 1];
-  alignas(16) int32_t item[ITEMS + 4];
+  alignas(16) int32_t item[ITEMS + GV];
 };
 
 __device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, int r0, int r1, int r2,
@@ -88,6 +93,9 @@ __device__ __forceinline__ void fma2(F2& acc, F2 p, F2 z) {
 __device__ __forceinline__ void mul2(F2& acc, F2 p) {
   asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(acc.v) : "l"(p.v));
 }
+__device__ __forceinline__ void add2(F2& acc, F2 x) {
+  asm("add.rn.f32x2 %0, %0, %1;" : "+l"(acc.v) : "l"(x.v));
+}
 
 // Per-lane accumulator of one destination row: NP register pairs.
 template <int VEC> struct Acc { F2 a[VEC / 2]; };
@@ -107,12 +115,13 @@ __device__ __forceinline__ void to_pairs(const uint4& raw, F2 (&z)[2]) {        
 // out = ReLU(acc * inv + bias), stored in the feature type
 __device__ __forceinline__ void finish_row(bf16* dst, const F2 (&acc)[4], float inv, const float (&bs)[8]) {
   uint32_t w[4];
+  const F2 i2 = make_f2(inv, inv);
 #pragma unroll
   for (int t = 0; t < 4; ++t) {
+    F2 o = make_f2(bs[2 * t], bs[2 * t + 1]);
+    fma2(o, acc[t], i2);
     float lo, hi;
-    split_f2(acc[t], lo, hi);
-    lo = fmaf(lo, inv, bs[2 * t]);
-    hi = fmaf(hi, inv, bs[2 * t + 1]);
+    split_f2(o, lo, hi);
     asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(w[t]) : "f"(hi), "f"(lo));   // ReLU inside the rounding
   }
   *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -129,16 +138,18 @@ __device__ __forceinline__ void finish_row(float* dst, const F2 (&acc)[2], float
   *reinterpret_cast<float4*>(dst) = make_float4(o[0], o[1], o[2], o[3]);
 }
 
-// out = ReLU(acc * inv + bias) kept in fp32 (for the fused per-graph readout)
+// out = ReLU(acc * inv + bias) kept in fp32, as register pairs (for the fused per-graph readout)
 template <int NP>
 __device__ __forceinline__ void finish_row_f32(const F2 (&acc)[NP], float inv, const float (&bs)[2 * NP],
-                                               float (&o)[2 * NP]) {
+                                               F2 (&o)[NP]) {
+  const F2 i2 = make_f2(inv, inv);
 #pragma unroll
   for (int t = 0; t < NP; ++t) {
+    F2 v = make_f2(bs[2 * t], bs[2 * t + 1]);
+    fma2(v, acc[t], i2);
     float lo, hi;
-    split_f2(acc[t], lo, hi);
-    o[2 * t] = fmaxf(fmaf(lo, inv, bs[2 * t]), 0.f);
-    o[2 * t + 1] = fmaxf(fmaf(hi, inv, bs[2 * t + 1]), 0.f);
+    split_f2(v, lo, hi);
+    o[t] = make_f2(fmaxf(lo, 0.f), fmaxf(hi, 0.f));
   }
 }
 
@@ -176,8 +187,8 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
   using Smem = WarpSmem<K, MERGED>;
   constexpr uint32_t ZR = Smem::ROW;                  // bytes per gathered row
   constexpr uint32_t SR = MERGED ? ZR : 8 * K;        // distance between consecutive rows' pairs
-  constexpr uint32_t GROUP_BYTES = 4 * 512 + 4 * K * 8;
-  constexpr uint32_t ZG = 4 * ZR, SG = 4 * SR;        // bytes per group in the ring(s)
+  constexpr uint32_t GROUP_BYTES = GV * (512 + K * 8);
+  constexpr uint32_t ZG = GV * ZR, SG = GV * SR;      // bytes per group in the ring(s)
   constexpr int ZS = int(ZR / sizeof(T));             // elements between rows of the Z buffer (slow path)
   extern __shared__ __align__(128) uint8_t tma_smem_raw[];
   Smem& sm = reinterpret_cast<Smem*>(tma_smem_raw)[threadIdx.x >> 5];
@@ -207,13 +218,16 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
   uint32_t slot = 0, par = 0;
   bool alive = true;
 
-  // lane 0: hand group `gi` of the current list (list rows item[4 gi .. 4 gi + 3]) to slot `s`
+  // lane 0: hand group `gi` of the current list (list rows item[GV gi .. GV gi + GV - 1]) to slot `s`
   auto issue = [&](int gi, uint32_t s) {
-    const int4 it = *reinterpret_cast<const int4*>(&sm.item[gi * 4]);
     const uint32_t bar = bar_base + 8 * s;
     mbar_expect_tx(bar, GROUP_BYTES);
-    tma_gather4(z_base + s * ZG, &map_z, it.x, it.y, it.z, it.w, bar);
-    if (!MERGED) tma_gather4(s_base + s * SG, &map_s, it.x, it.y, it.z, it.w, bar);
+#pragma unroll
+    for (int q = 0; q < GQ; ++q) {
+      const int4 it = *reinterpret_cast<const int4*>(&sm.item[gi * GV + q * 4]);
+      tma_gather4(z_base + s * ZG + q * 4 * ZR, &map_z, it.x, it.y, it.z, it.w, bar);
+      if (!MERGED) tma_gather4(s_base + s * SG + q * 4 * SR, &map_s, it.x, it.y, it.z, it.w, bar);
+    }
   };
 
   for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * BR; r0 < win.row_end && alive;
@@ -226,31 +240,35 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
     // fused readout: running per-graph sum of this block's rows
     int32_t myseg = 0, cur_g = -1;
     bool first_seg = true;
-    float rsum[VEC];
+    F2 rsum[NP];
     if (READOUT) {
       myseg = (lane < nr) ? __ldg(seg_id + r0 + lane) : 0;
 #pragma unroll
-      for (int t = 0; t < VEC; ++t) rsum[t] = 0.f;
+      for (int t = 0; t < NP; ++t) rsum[t] = make_f2(0.f, 0.f);
     }
     auto flush = [&]() {
       float* dst = partial + size_t(first_seg ? int32_t(r0 / BR) : nblocks + cur_g) * H + c0;
 #pragma unroll
-      for (int t = 0; t < VEC; t += 4)
-        *reinterpret_cast<float4*>(dst + t) = make_float4(rsum[t], rsum[t + 1], rsum[t + 2], rsum[t + 3]);
+      for (int t = 0; t < NP; t += 2) {
+        float4 v;
+        split_f2(rsum[t], v.x, v.y);
+        split_f2(rsum[t + 1], v.z, v.w);
+        *reinterpret_cast<float4*>(dst + 2 * t) = v;
+      }
     };
-    auto add_row = [&](int row_in_block, const float (&o)[VEC]) {
+    auto add_row = [&](int row_in_block, const F2 (&o)[NP]) {
       const int32_t g = __shfl_sync(0xFFFFFFFFu, myseg, row_in_block);
       if (g != cur_g) {
         if (cur_g >= 0) {
           flush();
           first_seg = false;
 #pragma unroll
-          for (int t = 0; t < VEC; ++t) rsum[t] = 0.f;
+          for (int t = 0; t < NP; ++t) rsum[t] = make_f2(0.f, 0.f);
         }
         cur_g = g;
       }
 #pragma unroll
-      for (int t = 0; t < VEC; ++t) rsum[t] += o[t];
+      for (int t = 0; t < NP; ++t) add2(rsum[t], o[t]);
     };
     int rs = 0;
     while (rs < nr && alive) {
@@ -287,7 +305,7 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
           for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], p2, z[t2]);
         }
         if (READOUT) {
-          float o[VEC];
+          F2 o[NP];
           finish_row_f32<NP>(acc, __fdividef(1.f, l), bs, o);
           add_row(rs, o);
         } else {
@@ -306,16 +324,16 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
                                   : int32_t(r0) + rs + lane - win.win_base;
         for (int t = 0; t < n; ++t) sm.item[pos++] = __ldg(col + eb + e0 + t) - win.win_base;
       }
-      if (lane < 4) sm.item[total + lane] = int32_t(r0) + rs - win.win_base;   // pad the last group
+      if (lane < GV) sm.item[total + lane] = int32_t(r0) + rs - win.win_base;   // pad the last group
       __syncwarp();
-      const int ngroups = (total + 3) >> 2;
+      const int ngroups = (total + GV - 1) / GV;
       if (lane == 0) {
         uint32_t s = slot;
         for (int gi = 0; gi < min(G, ngroups); ++gi) { issue(gi, s); s = (s + 1 == G) ? 0 : s + 1; }
       }
 
       // ---- consume: rows in order, vectors in list order ----------------------------------------------
-      int gi = 0, w = 4;                      // current group of the list, vectors left in it
+      int gi = 0, w = GV;                     // current group of the list, vectors left in it
       uint32_t zp = z_lane + slot * ZG, sp = s_lane + slot * SG;
       if (!wait_all_lanes(bar_base + 8 * slot, par)) alive = false;
       // group finished: refill its slot with group gi + G, move on, wait for the next one
@@ -326,7 +344,7 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
         if (++slot == G) { slot = 0; par ^= 1; }
         zp = z_lane + slot * ZG;
         sp = s_lane + slot * SG;
-        w = 4;
+        w = GV;
         if (gi < ngroups && alive && !wait_all_lanes(bar_base + 8 * slot, par)) alive = false;
       };
       for (int rr = 0; rr < cnt; ++rr) {
@@ -340,7 +358,30 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
         float m = lrelu(sc.x + sd), l = 1.f;
         F2 acc[NP];
         to_pairs(raw, acc);
-        for (int t = 0; t < n; ++t) {
+        int t = 0;
+        // two producers at a time while the row and the group at the ring's head both have two left: one
+        // pointer step, one ring check and one overflow test for the pair, and two independent chains
+        while (n - t >= 2 && w >= 2) {
+          const uint4 raw0 = lds128(zp), raw1 = lds128(zp + ZR);
+          const float2 sc0 = lds64(sp), sc1 = lds64(sp + SR);
+          zp += 2 * ZR; sp += 2 * SR;
+          t += 2;
+          if ((w -= 2) == 0) advance();
+          const float ev0 = lrelu(sc0.x + sd), ev1 = lrelu(sc1.x + sd);
+          const float evm = fmaxf(ev0, ev1);
+          if (evm > m + 32.f) raise_reference<NP>(evm, m, l, acc);
+          const float p0 = fast_exp2(ev0 - m), p1 = fast_exp2(ev1 - m);
+          l += p0 + p1;
+          F2 z0[NP], z1[NP];
+          to_pairs(raw0, z0);
+          to_pairs(raw1, z1);
+          const F2 q0 = make_f2(p0, p0), q1 = make_f2(p1, p1);
+#pragma unroll
+          for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], q0, z0[t2]);
+#pragma unroll
+          for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], q1, z1[t2]);
+        }
+        for (; t < n; ++t) {
           raw = lds128(zp);
           sc = lds64(sp);
           zp += ZR; sp += SR;
@@ -356,14 +397,14 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
           for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], p2, z[t2]);
         }
         if (READOUT) {
-          float o[VEC];
+          F2 o[NP];
           finish_row_f32<NP>(acc, __fdividef(1.f, l), bs, o);
           add_row(rs + rr, o);
         } else {
           finish_row(h_out + size_t(int32_t(r0) + rs + rr - win.win_base) * H + c0, acc, __fdividef(1.f, l), bs);
         }
       }
-      if (w != 4) {                            // the list ended inside a group: retire it without waiting
+      if (w != GV) {                           // the list ended inside a group: retire it without waiting
         __syncwarp();
         if (++slot == G) { slot = 0; par ^= 1; }
       }
