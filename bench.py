@@ -277,16 +277,26 @@ def main():
     elapsed_ms = ev0.elapsed_time(ev1)
     clock_info = clocks.stop()
     launches = xrl.xrl_launch_counts(agent.ctx)
-    # per-family kernel times from a separate pass: the library's event timing needs direct launches,
-    # while the timed steps above may have been submitted as one recorded graph each
-    prof_steps = max(1, min(args.steps, 5))
+    # The same K steps once more with the library's per-family CUDA events recorded inside them (event timing
+    # needs direct launches, while the timed steps above may have been submitted as one recorded graph each):
+    # the family times, the step time of that very pass and the clocks sampled during it belong together, so
+    # that gap_ms = step - sum of families is what the step spends outside its kernels (launch gaps, the
+    # metadata upload, event overhead) and not a difference in clocks between two passes.
+    prof_steps = args.steps
+    clocks_p = ClockSampler(local_rank)
+    clocks_p.start()
     xrl.xrl_profile(agent.ctx, True)
+    barrier()
+    pv0, pv1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    pv0.record(stream)
     for i in range(prof_steps):
         device_step(warmup + i)
+    pv1.record(stream)
+    barrier()
+    prof_ms_per_step = pv0.elapsed_time(pv1) / prof_steps
     prof = xrl.xrl_profile_read(agent.ctx)
     xrl.xrl_profile(agent.ctx, False)
-    for v in prof.values():
-        v["ms"] *= args.steps / prof_steps          # scaled to the timed step count used below
+    clock_info_p = clocks_p.stop()
     status = agent.device_status()
     assert status == 0, f"device status {status}"
     # observed error of the timed configuration against the oracle's embeddings of the sampled graphs
@@ -413,15 +423,32 @@ def main():
     ms_per_step = elapsed_ms / args.steps
     peak, peak_kind = measured_peaks()
     fam_ms = {f: (v["ms"] / args.steps) for f, v in prof.items()}
-    dominant = max(("transform", "aggregate", "aggregate_readout", "node_update", "readout", "pack"),
-                   key=lambda f: fam_ms[f])
     fused = 1 if prof["aggregate_readout"]["launches"] > 0 else 0
     calls = {"pack": 1, "node_update": 1, "transform": m["L"], "aggregate": m["L"] - fused,
              "aggregate_readout": fused, "readout": 1 - fused}       # launches of each kernel family per step
+    # the plain and the readout-fused attention launches are one kernel (two instantiations): the dominant
+    # kernel is chosen by the time of the kernel, the roofline line is that of its plain instantiation and
+    # `families` lists every family's own fraction
+    kernel_of = {"aggregate_readout": "aggregate"}
+    per_kernel = {}
+    for f in ("transform", "aggregate", "aggregate_readout", "node_update", "readout", "pack"):
+        per_kernel[kernel_of.get(f, f)] = per_kernel.get(kernel_of.get(f, f), 0.0) + fam_ms[f]
+    dominant = max(per_kernel, key=per_kernel.get)
+    if dominant == "aggregate" and calls["aggregate"] == 0:
+        dominant = "aggregate_readout"
     dom_ms = fam_ms[dominant] / max(1, calls[dominant])
     alg = algorithmic_bytes(dominant, m, N, E)
     achieved = alg / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
     step_alg = sum(algorithmic_bytes(f, m, N, E) * c for f, c in calls.items())
+    families = {}
+    for f, c in calls.items():
+        if c > 0 and fam_ms[f] > 0:
+            ms = fam_ms[f] / c
+            families[f] = {"launches": c, "launch_ms": round(ms, 4),
+                           "frac": round(algorithmic_bytes(f, m, N, E) / (ms * 1e-3) / 1e9 / peak, 4)}
+    kernels_ms = sum(fam_ms.values())
+    mhz = clock_info.get("sm_mhz")
+    mhz_p = clock_info_p.get("sm_mhz")
     line = {
         "metric": "graphs_encoded_per_s", "value": tot_graphs / (ms_per_step * 1e-3), "unit": "graphs/s",
         "n_gpus": world, "steps": args.steps, "warmup": warmup, "ms_per_step": ms_per_step,
@@ -438,11 +465,18 @@ def main():
         "clocks": clock_info,
         "gpu_launches": int(args.steps * (launches["pack"] + launches["encode"] + launches["heads"])),
         "kernel_ms_per_step": {f: round(v, 4) for f, v in fam_ms.items()},
+        # the pass the family times come from: its own step time, what of it lies outside the kernels, its clocks;
+        # time x clock lets runs under different power caps be compared
+        "profiled_pass": {"ms_per_step": round(prof_ms_per_step, 4), "kernels_ms": round(kernels_ms, 4),
+                          "gap_ms": round(prof_ms_per_step - kernels_ms, 4), "sm_mhz": mhz_p,
+                          "ms_x_ghz": round(prof_ms_per_step * mhz_p / 1e3, 3) if mhz_p else None},
+        "gap_ms": round(ms_per_step - kernels_ms, 4),
+        "ms_x_ghz": round(ms_per_step * mhz / 1e3, 3) if mhz else None,
         "step_hbm_frac": step_alg / (ms_per_step * 1e-3) / 1e9 / peak,
         "roofline": {"kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peak,
                      "peak_source": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
                      "traffic": TRAFFIC.get((cfg_id, dominant)) if args.candidates is None else None,
-                     "algorithmic_bytes": int(alg), "launch_ms": dom_ms},
+                     "algorithmic_bytes": int(alg), "launch_ms": dom_ms, "families": families},
     }
     if e2e:
         line["e2e"] = {"value": tot_graphs / e2e["s_per_step"], "unit": "graphs/s",
@@ -467,8 +501,9 @@ def main():
 
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from the
-# ncu capture summarised under profiles/; filled in once a capture of the current kernel exists.
-TRAFFIC = {(4, "aggregate"): 4.65e9}   # 581.5 MB on the 128-graph capture, scaled by the node count
+# ncu capture summarised under profiles/ (572.6 MB on the 128-graph capture of the current kernel, scaled by
+# the node count: every row is read and written once, so traffic grows in proportion).
+TRAFFIC = {(4, "aggregate"): 4.58e9}
 
 if __name__ == "__main__":
     main()
