@@ -295,6 +295,24 @@ xrl_status xrl_gae(int32_t device, int32_t num_steps, int32_t num_trajectories, 
                    const float* values, const uint8_t* done, float gamma, float lambda, float* adv, float* ret,
                    void* stream);
 
+/* Data-parallel training step (Section 3.3.4: the objective is a mean over the environments of the mini-batch;
+ * the paper leaves training on several devices as future work).  Every rank has run xrl_ppo_grad on its own
+ * environments, so its gradient and loss terms are means over n_r local environments.  The mean over all
+ * ranks' environments is sum_r(n_r x_r) / sum_r(n_r): xrl_grad_weigh writes
+ *   buf = [ grad * n | loss[0..3] * n | n ]         (count + 5 elements)
+ * for the caller's SUM all-reduce of buf (NCCL, gloo, ... - the collective itself is the caller's), and
+ * xrl_grad_unweigh divides the reduced buffer by its last element and writes grad and loss back, which then
+ * equal one xrl_ppo_grad call on the concatenation of all ranks' batches.
+ *   where       XRL_MEM_DEVICE: all pointers DEVICE, work enqueued on `stream` of `device`;
+ *               XRL_MEM_HOST: all pointers HOST, done before the call returns (`device`, `stream` ignored)
+ *   elem_bytes  4 (float, what xrl_ppo_grad produces) or 8 (double)
+ *   total_envs  HOST or NULL: receives sum_r(n_r); for DEVICE buffers a non-NULL pointer synchronises `stream`
+ * Errors: INVALID_ARG, CUDA. */
+xrl_status xrl_grad_weigh(int32_t where, int32_t device, int32_t elem_bytes, const void* grad, int64_t count,
+                          const void* loss, int64_t num_envs, void* buf, void* stream);
+xrl_status xrl_grad_unweigh(int32_t where, int32_t device, int32_t elem_bytes, const void* buf, int64_t count,
+                            void* grad, void* loss, int64_t* total_envs, void* stream);
+
 /* Read and clear the device status word.  Synchronises `stream`.  *status (HOST) receives the
  * first error code any kernel recorded since the last call, or XRL_OK. */
 xrl_status xrl_last_device_status(xrl_ctx* ctx, void* stream, int32_t* status);

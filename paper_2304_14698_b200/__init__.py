@@ -9,5 +9,5 @@ from .binding import (  # noqa: F401
     xrl_batch_free, xrl_batch_info, xrl_batch_export, xrl_encode, xrl_debug_node_features,
     xrl_policy_value, xrl_sample, xrl_last_device_status, xrl_launch_counts, xrl_version,
     xrl_profile, xrl_profile_read, xrl_pack_csr_static, xrl_encode_delta, xrl_delta_rows, xrl_graph_begin,
-    xrl_graph_launch, xrl_batch_set_edge_attr, xrl_ppo_grad, xrl_gae, allreduce_ppo_grad, STATUS_NAMES, EXPORTED_SYMBOLS, PROFILE_FAMILIES,
+    xrl_graph_launch, xrl_batch_set_edge_attr, xrl_ppo_grad, xrl_gae, xrl_grad_weigh, xrl_grad_unweigh, allreduce_ppo_grad, STATUS_NAMES, EXPORTED_SYMBOLS, PROFILE_FAMILIES,
 )

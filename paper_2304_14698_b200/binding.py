@@ -26,6 +26,7 @@ EXPORTED_SYMBOLS = [
     "xrl_policy_value", "xrl_sample", "xrl_last_device_status", "xrl_launch_counts", "xrl_version",
     "xrl_profile", "xrl_profile_read", "xrl_pack_csr_static", "xrl_encode_delta", "xrl_delta_rows", "xrl_get_weights",
     "xrl_graph_begin", "xrl_graph_launch", "xrl_batch_set_edge_attr", "xrl_ppo_grad", "xrl_gae",
+    "xrl_grad_weigh", "xrl_grad_unweigh",
 ]
 PROFILE_FAMILIES = ["pack", "node_update", "transform", "aggregate", "readout", "heads", "aggregate_readout"]
 
@@ -91,6 +92,8 @@ def load_library():
         "xrl_ppo_grad": [vp] * 8 + [C.c_float] * 3 + [vp] * 4,
         "xrl_gae": [i32, i32, i32, vp, vp, vp, C.c_float, C.c_float, vp, vp, vp],
         "xrl_graph_launch": [vp, vp],
+        "xrl_grad_weigh": [i32, i32, i32, vp, i64, vp, i64, vp, vp],
+        "xrl_grad_unweigh": [i32, i32, i32, vp, i64, vp, vp, C.POINTER(i64), vp],
     }
     for name, args in sigs.items():
         fn = getattr(lib, name)
@@ -311,21 +314,45 @@ def xrl_gae(reward, values, done, gamma, lam, adv=None, ret=None, stream=None):
     return adv, ret
 
 
+def _where_ptr(t):
+    """(where, device index, pointer) of a contiguous torch tensor that lives on the CPU or on a CUDA device."""
+    if t.is_cuda:
+        return XRL_MEM_DEVICE, t.device.index or 0, C.c_void_p(t.data_ptr())
+    return XRL_MEM_HOST, 0, C.c_void_p(t.data_ptr())
+
+
+def xrl_grad_weigh(grad, loss, num_envs, buf, stream=None):
+    """buf[count + 5] = [grad * n | loss * n | n] (see include/xrl.h); torch tensors, all on one device or all on
+    the CPU, float32 or float64."""
+    where, dev, gp = _where_ptr(grad)
+    st = _stream(stream) if where == XRL_MEM_DEVICE else None
+    _check(load_library().xrl_grad_weigh(where, dev, grad.element_size(), gp, grad.numel(), _where_ptr(loss)[2],
+                                         int(num_envs), _where_ptr(buf)[2], st), "xrl_grad_weigh")
+    return buf
+
+
+def xrl_grad_unweigh(buf, grad, loss, stream=None) -> int:
+    """grad, loss = buf / buf[-1]; returns the total number of environments (synchronises for device buffers)."""
+    where, dev, gp = _where_ptr(grad)
+    st = _stream(stream) if where == XRL_MEM_DEVICE else None
+    total = C.c_int64()
+    _check(load_library().xrl_grad_unweigh(where, dev, grad.element_size(), _where_ptr(buf)[2], grad.numel(), gp,
+                                           _where_ptr(loss)[2], C.byref(total), st), "xrl_grad_unweigh")
+    return int(total.value)
+
+
 def allreduce_ppo_grad(loss, grad, num_envs, group=None):
     """Data-parallel training step: every rank has run xrl_ppo_grad on its own environments, so its loss terms
     and gradient are means over `num_envs` local environments.  In place, they become the means over all
-    ranks' environments (one sum all-reduce of [grad * n | loss * n | n], NCCL for device tensors): the result
-    equals one xrl_ppo_grad call on the concatenated batch.  Returns the global number of environments."""
+    ranks' environments: xrl_grad_weigh, one sum all-reduce of the buffer (NCCL for device tensors),
+    xrl_grad_unweigh.  The result equals one xrl_ppo_grad call on the concatenated batch.  loss [4] and grad are
+    contiguous torch tensors of one floating type on one device.  Returns the global number of environments."""
     import torch
     import torch.distributed as dist
-    n = float(num_envs)
-    buf = torch.cat([grad.reshape(-1) * n, loss.reshape(-1).to(grad.dtype) * n,
-                     torch.tensor([n], dtype=grad.dtype, device=grad.device)])
+    buf = torch.empty(grad.numel() + 5, dtype=grad.dtype, device=grad.device)
+    xrl_grad_weigh(grad, loss, num_envs, buf)
     dist.all_reduce(buf, op=dist.ReduceOp.SUM, group=group)
-    total = float(buf[-1].item())
-    grad.copy_((buf[:grad.numel()] / total).reshape(grad.shape))
-    loss.copy_((buf[grad.numel():-1] / total).reshape(loss.shape).to(loss.dtype))
-    return int(round(total))
+    return xrl_grad_unweigh(buf, grad, loss)
 
 
 def xrl_last_device_status(ctx, stream=None) -> int:

@@ -3,10 +3,16 @@
 // environments of a mini-batch, then the gradient with respect to every weight, layer by layer backwards
 // through the heads, Eq. 8, the k attention layers of Eq. 7 and Eq. 6.
 //
-// These kernels are the plain, correct version: CUDA cores, fp32 gradients, sums over rows collected with
-// floating-point atomics (so the last bits of a gradient depend on the order in which the hardware serves
-// them).  Activations saved by the forward pass (the input of every layer) are read in their storage type;
-// Z and the half-scores of a layer are recomputed by the forward transform kernel before its reverse pass.
+// What is in this file: the forward pass of xrl_ppo_grad keeps every layer's input, Z rows and half-scores
+// (nothing is recomputed here); the reverse of Eq. 7 runs row-wise kernels (a warp per destination row:
+// k_aggregate_bwd_rows, k_scores_bwd_rows) with generic fallbacks (k_aggregate_bwd, k_scores_bwd) for head
+// counts that do not divide 32; the two dense products of a layer, dW = h_in^T dz and dh_in = dz W^T, run on
+// the tensor cores (mma.sync bf16, fp32 accumulate: k_atb_mma, k_gwt_mma) for bf16 models of hidden 128, 256
+// or 512 and on CUDA-core tiles (k_atb, k_gwt) otherwise.  Gradients are fp32; sums over rows are collected
+// with floating-point atomics, so the last bits of a gradient depend on the order in which the hardware
+// serves them.  Activations saved by the forward pass are read in their storage type.  On the tensor-core
+// path the half-score terms (ds a) are added into the bf16 copy of dz that the products read (`dzb`) only:
+// the fp32 `dz` buffer is then left without them and must not be read afterwards.
 // ReLU'(0) = 0, LeakyReLU'(0) = 0.2; the clipped objective has the slope of whichever term of its min is
 // the smaller one.
 #include <algorithm>
@@ -324,6 +330,8 @@ k_aggregate_bwd_rows(const int32_t* __restrict__ rowptr, const int32_t* __restri
     if (sm_db[c] != 0.f) atomicAdd(&db[c], sm_db[c]);
 }
 
+// dz += ds_src a_src + ds_dst a_dst per row and head, da_src / da_dst += ds z.  With `dzb` (tensor-core
+// products follow) the completed row goes to dzb in bf16 and the fp32 dz is NOT updated.
 template <typename T, int NF>
 __global__ void __launch_bounds__(256)
 k_scores_bwd_rows(ZView<T> zv, const float* __restrict__ ds_src, const float* __restrict__ ds_dst,
@@ -1099,6 +1107,48 @@ __global__ void k_gae(const float* __restrict__ reward, const float* __restrict_
 }  // namespace
 
 // ---- launchers ------------------------------------------------------------------------------------------
+// ---- weights of a rank's means in the data-parallel exchange --------------------------------------------
+// buf = [grad * n | loss[0..3] * n | n] before the caller's sum all-reduce; grad, loss = buf / buf[last] after it.
+namespace {
+template <typename F>
+__global__ void k_grad_weigh(const F* __restrict__ grad, int64_t count, const F* __restrict__ loss, F n,
+                             F* __restrict__ buf) {
+  const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < count) buf[i] = grad[i] * n;
+  else if (i < count + 4) buf[i] = loss[i - count] * n;
+  else if (i == count + 4) buf[i] = n;
+}
+template <typename F>
+__global__ void k_grad_unweigh(const F* __restrict__ buf, int64_t count, F* __restrict__ grad, F* __restrict__ loss) {
+  const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  const F total = buf[count + 4];
+  if (i < count) grad[i] = buf[i] / total;
+  else if (i < count + 4) loss[i - count] = buf[i] / total;
+}
+}  // namespace
+
+int launch_grad_weigh(int elem_bytes, const void* grad, int64_t count, const void* loss, int64_t n, void* buf,
+                      cudaStream_t st) {
+  const unsigned blocks = unsigned((count + 5 + 255) / 256);
+  if (elem_bytes == 8)
+    k_grad_weigh<double><<<blocks, 256, 0, st>>>(static_cast<const double*>(grad), count,
+                                                 static_cast<const double*>(loss), double(n), static_cast<double*>(buf));
+  else
+    k_grad_weigh<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(grad), count,
+                                                static_cast<const float*>(loss), float(n), static_cast<float*>(buf));
+  return 1;
+}
+int launch_grad_unweigh(int elem_bytes, const void* buf, int64_t count, void* grad, void* loss, cudaStream_t st) {
+  const unsigned blocks = unsigned((count + 4 + 255) / 256);
+  if (elem_bytes == 8)
+    k_grad_unweigh<double><<<blocks, 256, 0, st>>>(static_cast<const double*>(buf), count, static_cast<double*>(grad),
+                                                   static_cast<double*>(loss));
+  else
+    k_grad_unweigh<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(buf), count, static_cast<float*>(grad),
+                                                  static_cast<float*>(loss));
+  return 1;
+}
+
 int launch_gae(const float* reward, const float* values, const uint8_t* done, float gamma, float lambda, int32_t T,
                int32_t M, float* adv, float* ret, cudaStream_t st) {
   if (T <= 0 || M <= 0) return 0;

@@ -559,6 +559,28 @@ xrl_status check_encodable(const xrl_ctx* ctx, const xrl_batch* b) {
 
 }  // namespace
 
+namespace {
+template <typename F>
+void grad_weigh_host(const void* grad, int64_t count, const void* loss, int64_t n, void* buf) {
+  const F* g = static_cast<const F*>(grad);
+  const F* l = static_cast<const F*>(loss);
+  F* o = static_cast<F*>(buf);
+  for (int64_t i = 0; i < count; ++i) o[i] = g[i] * F(n);
+  for (int i = 0; i < 4; ++i) o[count + i] = l[i] * F(n);
+  o[count + 4] = F(n);
+}
+template <typename F>
+int64_t grad_unweigh_host(const void* buf, int64_t count, void* grad, void* loss) {
+  const F* b = static_cast<const F*>(buf);
+  F* g = static_cast<F*>(grad);
+  F* l = static_cast<F*>(loss);
+  const F total = b[count + 4];
+  for (int64_t i = 0; i < count; ++i) g[i] = b[i] / total;
+  for (int i = 0; i < 4; ++i) l[i] = b[count + i] / total;
+  return int64_t(total + F(0.5));
+}
+}  // namespace
+
 extern "C" {
 
 const char* xrl_version(void) { return "xrl 0.1 (sm_100a, CUDA C-ABI)"; }
@@ -1074,6 +1096,49 @@ xrl_status xrl_gae(int32_t device, int32_t num_steps, int32_t num_trajectories, 
   launch_gae(reward, values, done, gamma, lambda, num_steps, num_trajectories, adv, ret,
              static_cast<cudaStream_t>(stream));
   XRL_CUDA(cudaGetLastError());
+  return XRL_OK;
+}
+
+xrl_status xrl_grad_weigh(int32_t where, int32_t device, int32_t elem_bytes, const void* grad, int64_t count,
+                          const void* loss, int64_t num_envs, void* buf, void* stream) {
+  if ((where != XRL_MEM_HOST && where != XRL_MEM_DEVICE) || (elem_bytes != 4 && elem_bytes != 8) || count < 0 ||
+      num_envs < 0 || !loss || !buf || (count > 0 && !grad))
+    return XRL_ERR_INVALID_ARG;
+  if (where == XRL_MEM_HOST) {
+    if (elem_bytes == 8) grad_weigh_host<double>(grad, count, loss, num_envs, buf);
+    else grad_weigh_host<float>(grad, count, loss, num_envs, buf);
+    return XRL_OK;
+  }
+  XRL_CUDA(cudaSetDevice(device));
+  launch_grad_weigh(elem_bytes, grad, count, loss, num_envs, buf, static_cast<cudaStream_t>(stream));
+  XRL_CUDA(cudaGetLastError());
+  return XRL_OK;
+}
+
+xrl_status xrl_grad_unweigh(int32_t where, int32_t device, int32_t elem_bytes, const void* buf, int64_t count,
+                            void* grad, void* loss, int64_t* total_envs, void* stream) {
+  if ((where != XRL_MEM_HOST && where != XRL_MEM_DEVICE) || (elem_bytes != 4 && elem_bytes != 8) || count < 0 ||
+      !loss || !buf || (count > 0 && !grad))
+    return XRL_ERR_INVALID_ARG;
+  if (where == XRL_MEM_HOST) {
+    const int64_t total = elem_bytes == 8 ? grad_unweigh_host<double>(buf, count, grad, loss)
+                                          : grad_unweigh_host<float>(buf, count, grad, loss);
+    if (total_envs) *total_envs = total;
+    return XRL_OK;
+  }
+  XRL_CUDA(cudaSetDevice(device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  launch_grad_unweigh(elem_bytes, buf, count, grad, loss, st);
+  XRL_CUDA(cudaGetLastError());
+  if (total_envs) {
+    double t8 = 0.0;
+    float t4 = 0.f;
+    const char* last = static_cast<const char*>(buf) + size_t(count + 4) * size_t(elem_bytes);
+    XRL_CUDA(cudaMemcpyAsync(elem_bytes == 8 ? static_cast<void*>(&t8) : static_cast<void*>(&t4), last,
+                             size_t(elem_bytes), cudaMemcpyDeviceToHost, st));
+    XRL_CUDA(cudaStreamSynchronize(st));
+    *total_envs = int64_t((elem_bytes == 8 ? t8 : double(t4)) + 0.5);
+  }
   return XRL_OK;
 }
 

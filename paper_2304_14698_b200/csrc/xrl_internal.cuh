@@ -212,6 +212,9 @@ int launch_gat_layer_bwd(const Dims& d, const int32_t* rowptr, const int32_t* co
                          float* gb, int32_t N, cudaStream_t st);
 int launch_gae(const float* reward, const float* values, const uint8_t* done, float gamma, float lambda, int32_t T,
                int32_t M, float* adv, float* ret, cudaStream_t st);
+int launch_grad_weigh(int elem_bytes, const void* grad, int64_t count, const void* loss, int64_t n, void* buf,
+                      cudaStream_t st);
+int launch_grad_unweigh(int elem_bytes, const void* buf, int64_t count, void* grad, void* loss, cudaStream_t st);
 size_t embed_bwd_smem_bytes(const Dims& d);
 int launch_embed_bwd(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op, const void* shape,
                      const void* eattr, const void* h0, const float* dh0, float* xs /* scratch [N x 16] */,

@@ -10,20 +10,28 @@ from test_gpu_fuzz import _random_case
 pytestmark = pytest.mark.gpu
 
 # Per weight tensor: |g - r| <= a max|r| + b |r| for every entry, and ||g - r||_2 <= c ||r||_2 + d ||r_all||_2.
-# "fp32" is the check of the reverse pass itself.  A bf16 model keeps Z and every layer's output in bf16.
-# Against the oracle run at such rounded activations ("mirrored", with the half-scores taken where the
-# transform kernel of that shape takes them: from Z before it is rounded on the tensor cores, hidden 128 and
-# 256, from the stored Z otherwise) what remains are values that fall on the other side of a rounding
-# boundary or of a ReLU's zero.  Against the
-# definition, which keeps everything exact, each term of a gradient sum is off by a fraction of a percent
-# per layer it passed, a ReLU of Eq. 8 or of a head may sit on the other side of zero for one graph, and a
-# sum whose terms cancel (the attention vectors') shows that as a large part of its own, small, norm: there
-# the bound is on norms only, tied to the norm of the whole gradient.
+# "fp32" is the check of the reverse pass itself, against the definition.
+# "bf16": a bf16 model keeps Z and every layer's output in bf16 while the definition keeps them exact, so each
+# term of a gradient sum is off by a fraction of a percent per layer it passed.  The pass criterion is still the
+# definition.  Entry by entry: the encoder's matrices and biases (W0, b0, W_l, b_l) within 12 % and the value
+# head within 5 % of the tensor's largest entry (largest observed over the cases below: 10 % and 3 %).  By norms
+# only (15 % of the tensor's own norm plus 1 % of the whole gradient's): Eq. 8 (W_g, b_g) and the policy head,
+# where one hidden unit of one graph whose pre-activation sits within rounding of zero lands on the other side
+# of its ReLU and moves that unit's whole column (batches here have 10-30 graphs), and the attention vectors
+# a_src / a_dst, whose gradients are sums of cancelling terms of size 1e-4 that show the rounding of Z as a
+# large part of their own, small, norm.
+# "bf16 mirrored" (a debugging aid, not the criterion): against the oracle run at the rounded activations, with
+# the half-scores taken where the transform kernel of that shape takes them, what remains are values that fall on
+# the other side of a rounding boundary or of a ReLU's zero.
 GRAD_TOL = {"fp32": (1e-3, 1e-3, 1e-3, 0.0), "bf16 mirrored": (3e-2, 2e-2, 3e-2, 0.0),
-            "bf16": (None, None, 0.15, 0.01)}
+            "bf16": (None, 0.0, 0.15, 0.01)}
+# entry-by-entry bounds of a bf16 model against the definition, by tensor-name prefix (fraction of the largest entry)
+BF16_ENTRYWISE = {"W0": 0.12, "b0": 0.12, "W1": 0.12, "W2": 0.12, "W3": 0.12, "W4": 0.12, "W5": 0.12,
+                  "b1": 0.12, "b2": 0.12, "b3": 0.12, "b4": 0.12, "b5": 0.12,
+                  "vW1": 0.05, "vb1": 0.05, "vWh": 0.05, "vbh": 0.05, "vw2": 0.05}
 
 
-def _check_grad(m, got, want, tol, what):
+def _check_grad(m, got, want, tol, what, entrywise=None):
     off = 0
     nall = float(np.linalg.norm(want))
     for name, shape in configs.weight_layout(m):
@@ -34,8 +42,9 @@ def _check_grad(m, got, want, tol, what):
         g, r = got[off - n:off], want[off - n:off]
         # pb2's gradient is exactly 0 (the softmax ignores a shift of all logits): the GPU's is a sum of fp32 roundings
         floor = 1e-5 if np.abs(r).max() < 1e-12 else 1e-6
-        if tol[0] is not None:
-            bound = tol[0] * np.abs(r).max() + tol[1] * np.abs(r) + floor
+        frac = tol[0] if entrywise is None else entrywise.get(name)
+        if frac is not None:
+            bound = frac * np.abs(r).max() + tol[1] * np.abs(r) + floor
             err = np.abs(g - r)
             if (err > bound).any():
                 i = int(np.argmax(err - bound))
@@ -63,7 +72,7 @@ def _transitions(xo, m, blob, batch, packed, seed, g0=None):
     return action, logp_old, adv, ret
 
 
-def _compare(xo, batch, m, blob, g0=None, seed=0, eps=0.2, c1=0.5, c2=0.01):
+def _compare(xo, batch, m, blob, g0=None, seed=0, eps=0.2, c1=0.5, c2=0.01, mirrored=True):
     import torch
     import paper_2304_14698_b200 as xrl
     st, packed = xo.pack(batch)
@@ -89,8 +98,9 @@ def _compare(xo, batch, m, blob, g0=None, seed=0, eps=0.2, c1=0.5, c2=0.01):
         gpu_util.assert_close(loss.cpu().numpy(), want["loss"], dt, "loss")
         gpu_util.assert_close(logp.cpu().numpy(), want["logp"], dt, "logp")
         got = grad.cpu().numpy().astype(np.float64)
-        _check_grad(m, got, want["grad"], GRAD_TOL[dt], "definition")
-        if dt == "bf16":
+        _check_grad(m, got, want["grad"], GRAD_TOL[dt], "definition",
+                    entrywise=BF16_ENTRYWISE if dt == "bf16" else None)
+        if dt == "bf16" and mirrored:
             mir = xo.ppo_grad(m, blob, batch, packed, action, logp_old, adv, ret, eps, c1, c2, g0=g0,
                               mirrored=1 if m["H"] in (128, 256) else 2)
             _check_grad(m, got, mir["grad"], GRAD_TOL["bf16 mirrored"], "mirrored")
@@ -153,6 +163,38 @@ def test_gradient_on_a_step_of_the_papers_size(xo):
     b = configs.make_batch(6, candidates=5)
     blob, _ = gpu_util.default_weights(b, 1)
     _compare(xo, b, b["model"], blob, seed=4)
+
+
+def test_gradient_on_many_rows_of_the_large_step(xo):
+    """128 k rows of the power-law workload at hidden 256 in bf16: the tensor-core products of the reverse pass
+    run many tiles per CTA and the reverse attention kernel sees the workload's fan-out."""
+    b = configs.make_batch(4, candidates=31)
+    assert int(b["n_nodes"].sum()) > 100_000
+    blob, _ = gpu_util.default_weights(b, 2)
+    _compare(xo, b, b["model"], blob, seed=6, mirrored=False)     # (one run of the oracle's reverse pass: ~2 min)
+
+
+def test_gradient_exchange_weights_on_the_device():
+    """xrl_grad_weigh / xrl_grad_unweigh on device buffers: buf = [grad n | loss n | n], then grad, loss = buf /
+    buf[-1] (here after adding a second rank's buffer by hand)."""
+    import torch
+    import paper_2304_14698_b200 as xrl
+    rng = np.random.default_rng(3)
+    for dtype in (torch.float32, torch.float64):
+        g1, g2 = rng.normal(size=1000), rng.normal(size=1000)
+        l1, l2 = rng.normal(size=4), rng.normal(size=4)
+        bufs = []
+        for g, l, n in ((g1, l1, 3), (g2, l2, 5)):
+            gd, ld = torch.tensor(g, dtype=dtype, device="cuda"), torch.tensor(l, dtype=dtype, device="cuda")
+            buf = torch.empty(1005, dtype=dtype, device="cuda")
+            xrl.xrl_grad_weigh(gd, ld, n, buf)
+            bufs.append(buf)
+        total_buf = bufs[0] + bufs[1]                       # what a sum all-reduce leaves on every rank
+        gd, ld = torch.empty(1000, dtype=dtype, device="cuda"), torch.empty(4, dtype=dtype, device="cuda")
+        assert xrl.xrl_grad_unweigh(total_buf, gd, ld) == 8
+        tol = 1e-6 if dtype == torch.float32 else 1e-14
+        np.testing.assert_allclose(gd.cpu().numpy(), (3 * g1 + 5 * g2) / 8, rtol=tol, atol=tol)
+        np.testing.assert_allclose(ld.cpu().numpy(), (3 * l1 + 5 * l2) / 8, rtol=tol, atol=tol)
 
 
 def test_an_action_the_mask_excludes_is_reported(xo):
