@@ -114,7 +114,7 @@ k_readout(const T* __restrict__ h, const int32_t* __restrict__ chunk_row0,
 
 // ---- Eq. 8: emb_g = ReLU(Wg^T [ sum of the graph's chunk sums | g0_g ] + bg) -------------------
 template <int DEPTH>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 k_global_update(const float* __restrict__ partial, const int32_t* __restrict__ graph_chunk_off,
                 const float* __restrict__ g0, const float* __restrict__ Wg,
                 const float* __restrict__ bg, float* __restrict__ emb, int H, int Dg) {
@@ -137,7 +137,7 @@ k_global_update(const float* __restrict__ partial, const int32_t* __restrict__ g
 // partial of the block in which the graph starts (if it does not start at the block's first row), then
 // the partials of the following 32-row blocks whose first row belongs to the graph, in order.
 template <int DEPTH>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 k_global_update_blocks(const float* __restrict__ partial, const int32_t* __restrict__ node_off,
                        int32_t nblocks, const float* __restrict__ g0, const float* __restrict__ Wg,
                        const float* __restrict__ bg, float* __restrict__ emb, int H, int Dg) {
@@ -195,7 +195,7 @@ __device__ float mlp_scalar(const float* x, int in, const Mlp& m, float* y1, flo
 
 // ---- policy MLP: one scalar score per graph -----------------------------------------------------
 template <int DEPTH>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 k_policy_logit(const float* __restrict__ emb, const Mlp mlp, float* __restrict__ logit, int H) {
   extern __shared__ float sm[];                  // [H] + [blockDim] + [hid]
   float* x = sm;
@@ -400,6 +400,9 @@ __global__ void k_round_weights(const float* __restrict__ src, T* __restrict__ d
 
 // Launches with at most a few CTAs per SM are bound by the latency of their weight loads.
 bool few_ctas(int64_t ctas) { return ctas <= 4 * kNumSMs; }
+// With fewer CTAs than SMs every CTA has an SM to itself and the chain of dependent weight loads of one thread
+// is the whole run time: 1,024 threads cut every column's sum into four parts (dense_columns) instead of one.
+int head_threads(int64_t ctas) { return ctas <= kNumSMs ? 1024 : 256; }
 
 int pow2_threads(int want) {          // power of two in [32, 1024] (block_sum needs a power of two)
   int t = 32;
@@ -429,20 +432,22 @@ int launch_readout(const Dims& d, const void* h, const int32_t* chunk_row0, cons
 int launch_global_update(const Dims& d, const float* partial, const int32_t* graph_chunk_off,
                          const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st) {
   if (B <= 0) return 0;
-  const size_t smem = sizeof(float) * size_t(d.H + d.Dg + 256);
-  if (few_ctas(B)) k_global_update<32><<<B, 256, smem, st>>>(partial, graph_chunk_off, g0, w.Wg, w.bg, emb, d.H, d.Dg);
-  else k_global_update<8><<<B, 256, smem, st>>>(partial, graph_chunk_off, g0, w.Wg, w.bg, emb, d.H, d.Dg);
+  const int nt = head_threads(B);
+  const size_t smem = sizeof(float) * size_t(d.H + d.Dg + nt);
+  if (few_ctas(B)) k_global_update<32><<<B, nt, smem, st>>>(partial, graph_chunk_off, g0, w.Wg, w.bg, emb, d.H, d.Dg);
+  else k_global_update<8><<<B, nt, smem, st>>>(partial, graph_chunk_off, g0, w.Wg, w.bg, emb, d.H, d.Dg);
   return 1;
 }
 
 int launch_global_update_blocks(const Dims& d, const float* partial, const int32_t* node_off, int32_t nblocks,
                                 const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st) {
   if (B <= 0) return 0;
-  const size_t smem = sizeof(float) * size_t(d.H + d.Dg + 256);
+  const int nt = head_threads(B);
+  const size_t smem = sizeof(float) * size_t(d.H + d.Dg + nt);
   if (few_ctas(B))
-    k_global_update_blocks<32><<<B, 256, smem, st>>>(partial, node_off, nblocks, g0, w.Wg, w.bg, emb, d.H, d.Dg);
+    k_global_update_blocks<32><<<B, nt, smem, st>>>(partial, node_off, nblocks, g0, w.Wg, w.bg, emb, d.H, d.Dg);
   else
-    k_global_update_blocks<8><<<B, 256, smem, st>>>(partial, node_off, nblocks, g0, w.Wg, w.bg, emb, d.H, d.Dg);
+    k_global_update_blocks<8><<<B, nt, smem, st>>>(partial, node_off, nblocks, g0, w.Wg, w.bg, emb, d.H, d.Dg);
   return 1;
 }
 
@@ -453,13 +458,15 @@ int launch_heads(const Dims& d, const DevWeights& w, const float* emb, const int
   if (B <= 0 || num_envs <= 0) return 0;
   const Mlp pm{w.pW1, w.pb1, w.pWh, w.pbh, w.pw2, w.pb2, d.Hm, d.Hm2};
   const Mlp vm{w.vW1, w.vb1, w.vWh, w.vbh, w.vw2, w.vb2, d.Hm, d.Hm2};
-  const size_t psm = sizeof(float) * size_t(d.H + 256 + d.Hm);
-  if (few_ctas(B)) k_policy_logit<32><<<B, 256, psm, st>>>(emb, pm, logit_ws, d.H);
-  else k_policy_logit<8><<<B, 256, psm, st>>>(emb, pm, logit_ws, d.H);
+  const int pnt = head_threads(B);
+  const size_t psm = sizeof(float) * size_t(d.H + pnt + d.Hm);
+  if (few_ctas(B)) k_policy_logit<32><<<B, pnt, psm, st>>>(emb, pm, logit_ws, d.H);
+  else k_policy_logit<8><<<B, pnt, psm, st>>>(emb, pm, logit_ws, d.H);
   float* cand_sum = logit_ws + B;                 // [num_envs x H], behind the per-graph logits
   k_candidate_sum<<<dim3(num_envs, (d.H + 31) / 32), 1024, 0, st>>>(emb, env_off, mask, cand_sum, d.H, d.A);
   int want = d.H > d.A + 1 ? d.H : d.A + 1;
   if (want < 256) want = 256;               // enough threads to split the value head's dense map
+  if (num_envs <= kNumSMs) want = 1024;     // (an SM per environment: see head_threads)
   const int nt = pow2_threads(want);
   const size_t smem = sizeof(unsigned long long) * size_t(nt + 1) + sizeof(float) * size_t(nt + 2 * d.H + d.Hm);
   if (few_ctas(num_envs))

@@ -213,22 +213,57 @@ k_row_order_long(const int32_t* __restrict__ rowptr, const int2* __restrict__ tm
 constexpr int kGraphThreadsMax = 1024;
 inline int graph_threads(int32_t max_n) { return max_n >= 2048 ? 1024 : 512; }
 
-template <int NT>
+// OFFSETS = true (small batches, one launch for the whole batch): the CTA also derives its graph's offsets
+// from the per-graph counts itself (a block-wide sum over the graphs before it) and writes node_off[g],
+// edge_off[g] and graph_env[g] (the last graph's CTA the closing entries too), which saves the three tiny
+// launches that otherwise build them first.
+template <int NT, bool OFFSETS>
 __global__ void __launch_bounds__(NT)
-k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ edge_off,
+k_pack_graph(int32_t* __restrict__ node_off, int32_t* __restrict__ edge_off,
              const int32_t* __restrict__ op, const int32_t* __restrict__ edge_src,
              const int32_t* __restrict__ edge_dst, int32_t T, int32_t B, int32_t cap_n,
              int32_t* __restrict__ seg_id, int32_t* __restrict__ rowptr, int32_t* __restrict__ col,
-             int32_t* status, int32_t g_first, int32_t* __restrict__ eid) {
+             int32_t* status, int32_t g_first, int32_t* __restrict__ eid,
+             const int32_t* __restrict__ n_nodes, const int32_t* __restrict__ n_edges,
+             const int32_t* __restrict__ env_off, int32_t num_envs, int32_t* __restrict__ graph_env) {
   extern __shared__ __align__(16) int32_t psm[];
   int32_t* deg = psm;                         // [cap_n + 1] in-degree, then exclusive row starts
   int32_t* cur = psm + cap_n + 1;             // [cap_n]     row cursors
   int32_t* wsum = cur + cap_n;                // [kGraphThreadsMax / 32 + 1]
   int2* tmp = reinterpret_cast<int2*>(wsum + kGraphThreadsMax / 32 + 3);   // word 2 cap_n + 20: 8-byte aligned
   const int32_t g = g_first + blockIdx.x;      // a launch may cover a range of the batch's graphs
-  const int32_t nb = node_off[g], n = node_off[g + 1] - nb;
-  const int32_t eb = edge_off[g], m = edge_off[g + 1] - eb;
   const int tid = threadIdx.x;
+  int32_t nb, n, eb, m;
+  if (OFFSETS) {
+    // nodes and edges of the graphs before this one: per-thread partial sums, then a sum over the block
+    int32_t sn = 0, se = 0;
+    for (int32_t i = tid; i < g; i += NT) { sn += __ldg(n_nodes + i); se += __ldg(n_edges + i); }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      sn += __shfl_xor_sync(0xFFFFFFFFu, sn, o);
+      se += __shfl_xor_sync(0xFFFFFFFFu, se, o);
+    }
+    if ((tid & 31) == 0) wsum[tid >> 5] = sn;
+    __syncthreads();
+    sn = 0;
+    for (int w = 0; w < NT / 32; ++w) sn += wsum[w];
+    __syncthreads();
+    if ((tid & 31) == 0) wsum[tid >> 5] = se;
+    __syncthreads();
+    se = 0;
+    for (int w = 0; w < NT / 32; ++w) se += wsum[w];
+    __syncthreads();
+    nb = sn; eb = se;
+    n = __ldg(n_nodes + g); m = __ldg(n_edges + g);
+    if (tid == 0) {
+      node_off[g] = nb; edge_off[g] = eb;
+      if (g == B - 1) { node_off[B] = nb + n; edge_off[B] = eb + m; }
+      graph_env[g] = upper_segment(env_off, num_envs, g);
+    }
+  } else {
+    nb = node_off[g]; n = node_off[g + 1] - nb;
+    eb = edge_off[g]; m = edge_off[g + 1] - eb;
+  }
 
   for (int32_t i = tid; i < n; i += NT) {
     deg[i] = 0;
@@ -279,7 +314,7 @@ k_pack_graph(const int32_t* __restrict__ node_off, const int32_t* __restrict__ e
   if (g == B - 1 && tid == 0) rowptr[nb + n] = eb + deg[n];
   // the last graph of a partial launch closes its last row itself (the next graph's CTA, which writes the
   // same value as its first row start, may run much later)
-  else if (blockIdx.x == gridDim.x - 1 && tid == 0) rowptr[nb + n] = edge_off[g + 1];
+  else if (blockIdx.x == gridDim.x - 1 && tid == 0) rowptr[nb + n] = eb + m;
   // A malformed graph (already reported through `status`) keeps fewer edges than it was given slots for:
   // the slots left over sit at the end of the last row before the next graph's rows and nobody writes them.
   // They get a valid node id (the graph's first node) so that a batch that is encoded although it was
@@ -421,27 +456,35 @@ int launch_pack_offsets(const PackIn& in, const PackOut& out, cudaStream_t st) {
   return launches;
 }
 
-// CSR, segment ids and validation of graphs [g0, g1) (pack_per_graph(in) must hold; offsets already built).
+// CSR, segment ids and validation of graphs [g0, g1) (pack_per_graph(in) must hold; offsets already built, or
+// with `offsets` built by the same launch, which must then cover the whole batch).
 int launch_pack_graphs(const PackIn& in, const PackOut& out, int T, int32_t g0, int32_t g1, int32_t* status,
-                       cudaStream_t st) {
+                       cudaStream_t st, bool offsets) {
   if (g1 <= g0) return 0;
-  static bool attr512[64] = {}, attr1024[64] = {};
+  static bool attr512[64] = {}, attr1024[64] = {}, attr512o[64] = {}, attr1024o[64] = {};
   const size_t smem = pack_graph_smem(in.max_n, in.max_m);
+#define PACK_GRAPH(NT_, OFF_, ATTR_)                                                                              \
+  do {                                                                                                            \
+    ensure_dynamic_smem(k_pack_graph<NT_, OFF_>, 160 * 1024, ATTR_);                                              \
+    k_pack_graph<NT_, OFF_><<<g1 - g0, NT_, smem, st>>>(out.node_off, out.edge_off, in.op, in.edge_src,           \
+                                                        in.edge_dst, T, in.B, in.max_n, out.seg_id, out.rowptr,   \
+                                                        out.col, status, g0, out.eid, in.n_nodes, in.n_edges,     \
+                                                        in.env_off, in.num_envs, out.graph_env);                  \
+  } while (0)
   if (graph_threads(in.max_n) == 1024) {
-    ensure_dynamic_smem(k_pack_graph<1024>, 160 * 1024, attr1024);
-    k_pack_graph<1024><<<g1 - g0, 1024, smem, st>>>(out.node_off, out.edge_off, in.op, in.edge_src, in.edge_dst, T,
-                                                    in.B, in.max_n, out.seg_id, out.rowptr, out.col, status, g0,
-                                                    out.eid);
+    if (offsets) PACK_GRAPH(1024, true, attr1024o); else PACK_GRAPH(1024, false, attr1024);
   } else {
-    ensure_dynamic_smem(k_pack_graph<512>, 160 * 1024, attr512);
-    k_pack_graph<512><<<g1 - g0, 512, smem, st>>>(out.node_off, out.edge_off, in.op, in.edge_src, in.edge_dst, T,
-                                                  in.B, in.max_n, out.seg_id, out.rowptr, out.col, status, g0,
-                                                  out.eid);
+    if (offsets) PACK_GRAPH(512, true, attr512o); else PACK_GRAPH(512, false, attr512);
   }
+#undef PACK_GRAPH
   return 1;
 }
 
+// Batches of few graphs: the per-graph kernel builds the offsets too (one launch instead of four).
+constexpr int32_t kSelfOffsetGraphs = 2048;
+
 int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cudaStream_t st) {
+  if (pack_per_graph(in) && in.B <= kSelfOffsetGraphs) return launch_pack_graphs(in, out, T, 0, in.B, status, st, true);
   int launches = launch_pack_offsets(in, out, st);
   const int TB = 256;
   if (pack_per_graph(in)) return launches + launch_pack_graphs(in, out, T, 0, in.B, status, st);

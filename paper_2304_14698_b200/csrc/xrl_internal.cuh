@@ -120,7 +120,7 @@ int launch_pack(const PackIn& in, const PackOut& out, int T, int32_t* status, cu
 bool pack_per_graph(const PackIn& in);
 int launch_pack_offsets(const PackIn& in, const PackOut& out, cudaStream_t st);
 int launch_pack_graphs(const PackIn& in, const PackOut& out, int T, int32_t g0, int32_t g1, int32_t* status,
-                       cudaStream_t st);
+                       cudaStream_t st, bool offsets = false);
 size_t scan_workspace_ints(int64_t n);
 int launch_merge_csr(const int32_t* rp_a, const int32_t* col_a, const int32_t* rp_b, const int32_t* col_b,
                      int32_t N, int32_t* rp_m, int32_t* col_m, cudaStream_t st);
