@@ -12,7 +12,19 @@
 
 using namespace xrl;
 
+// NVTX ranges (header-only; no cost unless a profiling tool has attached) around the steps of the path as they
+// are enqueued: pack, Eq. 6, every attention layer's transform and aggregate, readout, Eq. 8, heads, and the
+// training step.  A timeline tool shows them over the kernels they launch.
+#include <nvtx3/nvToolsExt.h>
+
 namespace {
+
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+  NvtxRange(const NvtxRange&) = delete;
+  NvtxRange& operator=(const NvtxRange&) = delete;
+};
 
 constexpr int32_t kReadoutChunkRows = 512;
 
@@ -236,6 +248,7 @@ xrl_status pack_common(xrl_ctx* ctx, const xrl_graph* graphs, int32_t where, int
                        const void* shape, const int32_t* edge_src, const int32_t* edge_dst,
                        const int32_t* env_off, int32_t num_envs, void* stream, xrl_batch** out) {
   if (!ctx || !out || !env_off || num_graphs < 0 || num_envs < 0) return XRL_ERR_INVALID_ARG;
+  NvtxRange nvtx_pack("xrl:pack (Section 3.3.2)");
   if (ctx->capturing) return XRL_ERR_STATE;        // packing synchronises with its staging buffers
   if (!graphs && (where != XRL_MEM_HOST && where != XRL_MEM_DEVICE)) return XRL_ERR_INVALID_ARG;
   if (!graphs && num_graphs > 0 && (!n_nodes || !n_edges)) return XRL_ERR_INVALID_ARG;
@@ -492,6 +505,7 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
   const int32_t* gat_col = ctx->cfg.neighbourhood ? b->col_nbr.as<int32_t>() : b->col.as<int32_t>();
   size_t slot = pf.begin(st);
   int k = -1;
+  nvtxRangePushA("xrl:node update (Eq. 6)");
   if (ctx->use_umma_embed)
     k = launch_embed_umma(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), b->op.as<int32_t>(),
                           b->shape.p, ctx->w0ext.p, hs ? hs[0] : ctx->h.p, win, ctx->status.as<int32_t>(), st, nullptr, eattr);
@@ -499,12 +513,14 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
     k = launch_embed(d, b->rowptr.as<int32_t>(), b->col.as<int32_t>(), b->op.as<int32_t>(),
                      b->shape.p, ctx->dw, hs ? hs[0] : ctx->h.p, win, st, nullptr, eattr);
   pf.end(FAM_EMBED, slot, k, st);
+  nvtxRangePop();
   int n = k;
   for (int l = 0; l < layers; ++l) {
     const void* h_in = hs ? hs[l] : ctx->h.p;
     void* h_out = hs ? hs[l + 1] : ctx->h.p;
     void* Zl = zs ? zs[l] : ctx->Z.p;
     float* Sl = ss ? ss[l] : ctx->scores.as<float>();
+    NvtxRange nvtx_layer("xrl:attention layer (Eq. 7): transform, then score / softmax / aggregate");
     slot = pf.begin(st);
     k = -1;
     if (ctx->use_umma)
@@ -809,6 +825,7 @@ xrl_status xrl_encode(xrl_ctx* ctx, const xrl_batch* b, const float* g0, float* 
   XRL_CUDA(cudaSetDevice(ctx->device));
   cudaStream_t st = ctx->capturing ? ctx->cap_stream : static_cast<cudaStream_t>(stream);
   bool fused = false;
+  NvtxRange nvtx_encode("xrl:encode (Section 3.4)");
   int n = 0;
   if (b->nparts > 0) {
     // packed range by range: encode each range of graphs as soon as it is there (the copies and the packing
@@ -856,6 +873,7 @@ xrl_status xrl_encode_delta(xrl_ctx* ctx, const xrl_batch* b, const int32_t* bas
   if (ctx->cfg.neighbourhood) return XRL_ERR_UNSUPPORTED;     // a rewrite then reaches its producers' side too
   if (ctx->capturing) return XRL_ERR_STATE;        // reads the row counts back between layers
   if (!graph_emb && b->B > 0) return XRL_ERR_INVALID_ARG;
+  NvtxRange nvtx_delta("xrl:encode, delta of the candidates (Section 3.4)");
   XRL_CUDA(cudaSetDevice(ctx->device));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   { const xrl_status js = join_parts(b, st); if (js != XRL_OK) return js; }
@@ -1001,6 +1019,7 @@ xrl_status xrl_policy_value(xrl_ctx* ctx, const xrl_batch* b, const float* graph
   if (s != XRL_OK) return s;
   if (b->num_envs > 0 && (!graph_emb || !probs || !value || (!mask && ctx->cfg.max_actions > 0)))
     return XRL_ERR_INVALID_ARG;
+  NvtxRange nvtx_heads("xrl:policy / value heads, masked softmax, draw (Sections 3.3.2, 3.3.3)");
   XRL_CUDA(cudaSetDevice(ctx->device));
   cudaStream_t st = ctx->capturing ? ctx->cap_stream : static_cast<cudaStream_t>(stream);
   const size_t slot = ctx->prof.begin(st);
@@ -1020,6 +1039,7 @@ xrl_status xrl_ppo_grad(xrl_ctx* ctx, const xrl_batch* b, const float* g0, const
   if (s != XRL_OK) return s;
   if (ctx->capturing) return XRL_ERR_STATE;
   if (!loss_out || !grad) return XRL_ERR_INVALID_ARG;
+  NvtxRange nvtx_grad("xrl:training step gradient (Section 3.3.4, Eq. 3-5)");
   if (b->num_envs > 0 && (!action || !logp_old || !adv || !ret || (!mask && ctx->cfg.max_actions > 0)))
     return XRL_ERR_INVALID_ARG;
   if (embed_bwd_smem_bytes(ctx->dims) > size_t(227) * 1024) return XRL_ERR_UNSUPPORTED;
