@@ -129,6 +129,13 @@ xrl_status xrl_set_weights(xrl_ctx* ctx, const void* host_blob, size_t bytes);
  * together with xrl_set_weights this is the checkpoint / restore of a model.  Synchronous. */
 xrl_status xrl_get_weights(const xrl_ctx* ctx, void* host_blob, size_t bytes);
 
+/* Seeded initial weights in place of xrl_set_weights (the paper names no initialisation; Xavier-uniform is
+ * this library's choice): matrices U(-b, b) with b = sqrt(6 / (fan_in + fan_out)), the attention vectors with
+ * fan (H / heads, 1), the heads' last layers with fan (hidden, 1), every bias U(-0.1, 0.1).  Element i of the
+ * blob is b * ((w >> 8) * 2^-23 - 1), w = first word of Philox4x32-10 with key = seed and counter (i, 0, 0, 1):
+ * reproducible bit for bit from the seed on any device.  Synchronises the device.  Errors: INVALID_ARG, CUDA. */
+xrl_status xrl_init_weights(xrl_ctx* ctx, uint64_t seed);
+
 /* ---- (1) packer: Section 3.3.2, the current graph and its candidates become one meta-graph ---- */
 
 /* graphs[env_off[e]] is the CURRENT graph of environment e and graphs[env_off[e]+1 ..

@@ -14,6 +14,7 @@
 //                                   mask, No-Op action; Section 3.3.3 invalid-action masking
 //   xo_sample        Section 3.3.2  the action is drawn from the categorical distribution;
 //                                   random words from Philox4x32-10 (Salmon et al., SC'11)
+//   xo_init_weights  (no passage: the paper names no initialisation) the library's seeded Xavier-uniform blob
 //   xo_ppo_grad      Section 3.3.4  Eq. 3 (clipped objective), Eq. 4 (value loss), Eq. 5 (their sum with an
 //                                   entropy term) over a mini-batch, and the gradient with respect to every
 //                                   weight; xo_gae: the generalised advantage estimates it is fed with
@@ -839,6 +840,43 @@ int xo_gae(int32_t T, const double* reward, const double* values, const uint8_t*
     ret[t] = run + values[t];
   }
   return XO_OK;
+}
+
+// Seeded initial weights (the paper names no initialisation; Xavier-uniform is the library's documented choice):
+// matrices U(-b, b) with b = sqrt(6 / (fan_in + fan_out)), attention vectors with fan (H / K, 1), the heads' last
+// layers with fan (hidden, 1), biases U(-0.1, 0.1), in blob order.  Element i is b * u_i with
+// u_i = (w >> 8) 2^-23 - 1, w = first word of Philox4x32-10(key = seed, counter = (i, 0, 0, 1)).
+// `out` holds the whole blob; returns the number of elements written.
+int64_t xo_init_weights(const Model* m, uint64_t seed, float* out) {
+  const int64_t S = m->S, T = m->T, H = m->H, Hm = m->Hm, Hm2 = m->Hm2, Dg = m->Dg, d = m->H / m->K;
+  const int64_t last = Hm2 > 0 ? Hm2 : Hm;
+  int64_t off = 0;
+  auto xavier = [](int64_t fan_in, int64_t fan_out) { return float(std::sqrt(6.0 / double(fan_in + fan_out))); };
+  auto fill = [&](int64_t count, float bound) {
+    for (int64_t t = 0; t < count; ++t) {
+      const uint64_t i = uint64_t(off + t);
+      uint32_t w[4];
+      xo_philox4x32_10(uint32_t(seed), uint32_t(seed >> 32), uint32_t(i), uint32_t(i >> 32), 0u, 1u, w);
+      const float u = float(w[0] >> 8) * 1.1920928955078125e-07f - 1.0f;    // both steps are exact in float
+      out[off + t] = bound * u;
+    }
+    off += count;
+  };
+  const float bias = 0.1f;
+  fill((2 * S + T) * H, xavier(2 * S + T, H)); fill(H, bias);
+  for (int l = 0; l < m->L; ++l) {
+    fill(H * H, xavier(H, H));
+    fill(H, xavier(d, 1)); fill(H, xavier(d, 1));
+    fill(H, bias);
+  }
+  fill((H + Dg) * H, xavier(H + Dg, H)); fill(H, bias);
+  for (int head = 0; head < 2; ++head) {
+    const int64_t in = head == 0 ? H : 2 * H;
+    fill(in * Hm, xavier(in, Hm)); fill(Hm, bias);
+    if (Hm2 > 0) { fill(Hm * Hm2, xavier(Hm, Hm2)); fill(Hm2, bias); }
+    fill(last, xavier(last, 1)); fill(1, bias);
+  }
+  return off;
 }
 
 int xo_num_threads(void) {

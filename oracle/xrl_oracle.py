@@ -132,6 +132,20 @@ def sample(probs_f32, seed, step):
     return act
 
 
+def init_weights(m, seed):
+    """The seeded Xavier-uniform weight blob the library's xrl_init_weights defines (float32)."""
+    from workloads import configs
+    n = configs.weight_count(m)
+    out = np.zeros(n, np.float32)
+    fn = lib().xo_init_weights
+    fn.restype = C.c_int64
+    mm = _model(m)
+    wrote = fn(C.byref(mm), C.c_uint64(int(seed)), _p(out, _f32p))
+    if wrote != n:
+        raise ValueError(f"xo_init_weights wrote {wrote} of {n}")
+    return out
+
+
 def forward(m, weights, batch, g0=None, threads=0, mode=0):
     """Whole step: pack -> encode -> heads.  Convenience for tests and the CPU baseline."""
     st, packed = pack(batch)

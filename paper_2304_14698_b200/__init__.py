@@ -5,7 +5,7 @@ arguments.  There is no CPU fallback: importing works without a GPU, creating a 
 """
 from .binding import (  # noqa: F401
     XrlError, Agent, load_library, library_path, model_config,
-    xrl_create, xrl_destroy, xrl_weights_size, xrl_set_weights, xrl_get_weights, xrl_pack, xrl_pack_flat,
+    xrl_create, xrl_destroy, xrl_weights_size, xrl_set_weights, xrl_get_weights, xrl_init_weights, xrl_pack, xrl_pack_flat,
     xrl_batch_free, xrl_batch_info, xrl_batch_export, xrl_encode, xrl_debug_node_features,
     xrl_policy_value, xrl_sample, xrl_last_device_status, xrl_launch_counts, xrl_version,
     xrl_profile, xrl_profile_read, xrl_pack_csr_static, xrl_encode_delta, xrl_delta_rows, xrl_graph_begin,

@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = [
     "xrl_policy_value", "xrl_sample", "xrl_last_device_status", "xrl_launch_counts", "xrl_version",
     "xrl_profile", "xrl_profile_read", "xrl_pack_csr_static", "xrl_encode_delta", "xrl_delta_rows", "xrl_get_weights",
     "xrl_graph_begin", "xrl_graph_launch", "xrl_batch_set_edge_attr", "xrl_ppo_grad", "xrl_gae",
-    "xrl_grad_weigh", "xrl_grad_unweigh",
+    "xrl_grad_weigh", "xrl_grad_unweigh", "xrl_init_weights",
 ]
 PROFILE_FAMILIES = ["pack", "node_update", "transform", "aggregate", "readout", "heads", "aggregate_readout"]
 
@@ -71,6 +71,7 @@ def load_library():
         "xrl_weights_size": [vp, C.POINTER(C.c_size_t)],
         "xrl_set_weights": [vp, vp, C.c_size_t],
         "xrl_get_weights": [vp, vp, C.c_size_t],
+        "xrl_init_weights": [vp, u64],
         "xrl_pack": [vp, C.POINTER(_Graph), i32, vp, i32, vp, C.POINTER(vp)],
         "xrl_pack_flat": [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, i32, vp, C.POINTER(vp)],
         "xrl_batch_free": [vp, vp],
@@ -168,6 +169,11 @@ def xrl_weights_size(ctx) -> int:
 def xrl_set_weights(ctx, blob: np.ndarray):
     blob = np.ascontiguousarray(blob, dtype=np.float32)
     _check(load_library().xrl_set_weights(ctx, _np_ptr(blob), blob.nbytes), "xrl_set_weights")
+
+
+def xrl_init_weights(ctx, seed: int):
+    """Seeded Xavier-uniform weights (see include/xrl.h) in place of xrl_set_weights."""
+    _check(load_library().xrl_init_weights(ctx, int(seed)), "xrl_init_weights")
 
 
 def xrl_get_weights(ctx) -> np.ndarray:

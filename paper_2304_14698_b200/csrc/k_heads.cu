@@ -381,6 +381,20 @@ k_sample(const float* __restrict__ probs, int A1, uint64_t seed, uint64_t step,
   if (threadIdx.x == 0) action[e] = act;
 }
 
+// Seeded initial weights: element i of the blob is bound * u_i, u_i = (w >> 8) * 2^-23 - 1 in [-1, 1) with w the
+// first word of Philox4x32-10(key = seed, counter = (i, 0, 0, 1)); every step is exact in fp32 except the one
+// product, so any IEEE implementation gives the same bits.  (Counter word 3 = 1 keeps this stream apart from
+// the action draws, which use 0.)
+__global__ void k_init_weights(float* __restrict__ blob, int64_t first, int64_t count, float bound, uint32_t k0,
+                               uint32_t k1) {
+  const int64_t t = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (t >= count) return;
+  const uint64_t i = uint64_t(first + t);
+  const U4 r = philox4x32_10(k0, k1, U4{uint32_t(i), uint32_t(i >> 32), 0u, 1u});
+  const float u = __fsub_rn(__fmul_rn(float(r.x >> 8), 1.1920928955078125e-07f), 1.0f);
+  blob[first + t] = __fmul_rn(bound, u);
+}
+
 __global__ void k_to_float_bf16(const bf16* __restrict__ src, float* __restrict__ dst, int64_t n) {
   const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i < n) dst[i] = __bfloat162float(src[i]);
@@ -484,6 +498,13 @@ int launch_sample(const float* probs, int32_t num_envs, int32_t A1, uint64_t see
   const int nt = pow2_threads(A1);
   k_sample<<<num_envs, nt, sizeof(unsigned long long) * size_t(nt + 1), st>>>(probs, A1, seed, step,
                                                                               action);
+  return 1;
+}
+
+int launch_init_weights(float* blob, int64_t first, int64_t count, float bound, uint64_t seed, cudaStream_t st) {
+  if (count <= 0) return 0;
+  k_init_weights<<<unsigned((count + 255) / 256), 256, 0, st>>>(blob, first, count, bound, uint32_t(seed),
+                                                                uint32_t(seed >> 32));
   return 1;
 }
 

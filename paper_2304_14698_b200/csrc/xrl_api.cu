@@ -15,6 +15,7 @@ using namespace xrl;
 // NVTX ranges (header-only; no cost unless a profiling tool has attached) around the steps of the path as they
 // are enqueued: pack, Eq. 6, every attention layer's transform and aggregate, readout, Eq. 8, heads, and the
 // training step.  A timeline tool shows them over the kernels they launch.
+#include <cmath>
 #include <nvtx3/nvToolsExt.h>
 
 namespace {
@@ -679,11 +680,9 @@ xrl_status xrl_weights_size(const xrl_ctx* ctx, size_t* bytes) {
   return XRL_OK;
 }
 
-xrl_status xrl_set_weights(xrl_ctx* ctx, const void* host_blob, size_t bytes) {
-  if (!ctx || !host_blob) return XRL_ERR_INVALID_ARG;
-  if (bytes != 4 * ctx->weight_floats) return XRL_ERR_INVALID_ARG;
-  XRL_CUDA(cudaSetDevice(ctx->device));
-  XRL_CUDA(cudaMemcpy(ctx->w_f32.p, host_blob, bytes, cudaMemcpyHostToDevice));
+// The fp32 blob is in ctx->w_f32: derive the storage-type copies (and transposes) of W0 and the layer matrices
+// and the pointers of every tensor.
+static xrl_status finalize_weights(xrl_ctx* ctx) {
   const xrl_model_config& c = ctx->cfg;
   const size_t H = size_t(c.hidden), Hm = size_t(c.mlp_hidden), Hm2 = size_t(c.mlp_hidden2), Dg = size_t(c.global_dim);
   const size_t last = Hm2 > 0 ? Hm2 : Hm;
@@ -716,6 +715,47 @@ xrl_status xrl_set_weights(xrl_ctx* ctx, const void* host_blob, size_t bytes) {
   XRL_CUDA(cudaGetLastError());
   ctx->weights_set = true;
   return XRL_OK;
+}
+
+xrl_status xrl_set_weights(xrl_ctx* ctx, const void* host_blob, size_t bytes) {
+  if (!ctx || !host_blob) return XRL_ERR_INVALID_ARG;
+  if (bytes != 4 * ctx->weight_floats) return XRL_ERR_INVALID_ARG;
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  XRL_CUDA(cudaMemcpy(ctx->w_f32.p, host_blob, bytes, cudaMemcpyHostToDevice));
+  return finalize_weights(ctx);
+}
+
+xrl_status xrl_init_weights(xrl_ctx* ctx, uint64_t seed) {
+  if (!ctx) return XRL_ERR_INVALID_ARG;
+  XRL_CUDA(cudaSetDevice(ctx->device));
+  const xrl_model_config& c = ctx->cfg;
+  const int64_t H = c.hidden, Hm = c.mlp_hidden, Hm2 = c.mlp_hidden2, Dg = c.global_dim;
+  const int64_t F0 = 2 * kS + c.num_op_types, last = Hm2 > 0 ? Hm2 : Hm, d = H / c.heads;
+  float* blob = ctx->w_f32.as<float>();
+  int64_t off = 0;
+  // Xavier-uniform bound sqrt(6 / (fan_in + fan_out)), taken in double and rounded to float once
+  auto xavier = [](int64_t fan_in, int64_t fan_out) { return float(std::sqrt(6.0 / double(fan_in + fan_out))); };
+  auto fill = [&](int64_t count, float bound) {
+    launch_init_weights(blob, off, count, bound, seed, nullptr);
+    off += count;
+  };
+  const float kBias = 0.1f;
+  fill(F0 * H, xavier(F0, H)); fill(H, kBias);
+  for (int l = 0; l < c.layers; ++l) {
+    fill(H * H, xavier(H, H));
+    fill(H, xavier(d, 1)); fill(H, xavier(d, 1));          // attention vectors: one head's width in, a score out
+    fill(H, kBias);
+  }
+  fill((H + Dg) * H, xavier(H + Dg, H)); fill(H, kBias);
+  for (int head = 0; head < 2; ++head) {                    // policy head (input H), value head (input 2 H)
+    const int64_t in = head == 0 ? H : 2 * H;
+    fill(in * Hm, xavier(in, Hm)); fill(Hm, kBias);
+    if (Hm2 > 0) { fill(Hm * Hm2, xavier(Hm, Hm2)); fill(Hm2, kBias); }
+    fill(last, xavier(last, 1)); fill(1, kBias);
+  }
+  if (size_t(off) != ctx->weight_floats) return XRL_ERR_STATE;
+  XRL_CUDA(cudaGetLastError());
+  return finalize_weights(ctx);
 }
 
 xrl_status xrl_get_weights(const xrl_ctx* ctx, void* host_blob, size_t bytes) {

@@ -219,6 +219,7 @@ size_t embed_bwd_smem_bytes(const Dims& d);
 int launch_embed_bwd(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op, const void* shape,
                      const void* eattr, const void* h0, const float* dh0, float* xs /* scratch [N x 16] */,
                      float* gW0, float* gb0, int32_t N, cudaStream_t st);
+int launch_init_weights(float* blob, int64_t first, int64_t count, float bound, uint64_t seed, cudaStream_t st);
 int launch_to_float(const void* src, int dtype, float* dst, int64_t n, cudaStream_t st);
 int launch_round_weights(const float* src, void* dst, void* dst_t, int rows, int cols, int dtype,
                          cudaStream_t st);

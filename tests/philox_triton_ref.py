@@ -44,6 +44,18 @@ def main():
         for j in range(n):
             cases.append({"seed": seed, "counter": [int(v) for v in ctr[:, j]],
                           "out": [int(v) for v in o[:, j]]})
+    # counters of the form (i, 0, 0, 1): the stream the seeded weight initialisation draws from
+    for seed in [7, 0x0123456789ABCDEF]:
+        ctr = torch.zeros((4, n), dtype=torch.int64)
+        ctr[0] = torch.tensor([0, 1, 2, 3, 1000, 65535, 123456, 2 ** 31 - 1])
+        ctr[3] = 1
+        c32 = ctr.to(torch.int32).contiguous()
+        out = torch.zeros(4 * n, dtype=torch.int32)
+        _kernel[(1,)](out, seed, c32, n)
+        o = out.view(4, n).to(torch.int64) & 0xFFFFFFFF
+        for j in range(n):
+            cases.append({"seed": seed, "counter": [int(v) for v in ctr[:, j]],
+                          "out": [int(v) for v in o[:, j]]})
     print(json.dumps(cases))
 
 

@@ -175,6 +175,36 @@ def test_weights_round_trip():
         ag.close()
 
 
+@pytest.mark.parametrize("cfg", [1, 3, 6])
+def test_seeded_initial_weights_match_the_oracle_bit_for_bit(xo, cfg):
+    """xrl_init_weights: the blob read back equals the oracle's for the same seed, bit for bit, and a step
+    run with it equals the oracle's step with the same blob."""
+    import torch
+    import paper_2304_14698_b200 as xrl
+    batch = configs.make_batch(cfg, candidates=5)
+    m = batch["model"]
+    for seed in (3, 0xFEDCBA9876543210):
+        want = xo.init_weights(m, seed)
+        ag = gpu_util.make_agent(batch)
+        try:
+            xrl.xrl_init_weights(ag.ctx, seed)
+            got = xrl.xrl_get_weights(ag.ctx)
+            assert got.dtype == np.float32 and np.array_equal(got, want)
+            if seed == 3 and m["dtype"] == "fp32":
+                # (plain Xavier weights, without the other tests' readout scaling: sums over hundreds of nodes
+                # saturate the policy and, in bf16, cancel down to the tolerance - the fp32 model's graph
+                # embeddings are the check that the context really runs on the initialised weights)
+                ag.pack(batch)
+                o = ag.forward(torch.from_numpy(batch["mask"]).cuda())
+                torch.cuda.synchronize()
+                assert ag.device_status() == 0
+                st, packed = xo.pack(batch)
+                enc = xo.encode(m, want, batch, packed)
+                gpu_util.assert_close(o["emb"].cpu().numpy(), enc["emb"], m["dtype"], "graph_emb")
+        finally:
+            ag.close()
+
+
 def test_repack_in_place_reuses_the_batch(xo):
     import paper_2304_14698_b200 as xrl
     b1 = configs.make_batch(2, candidates=9, seed=5)
