@@ -161,16 +161,30 @@ k_global_update_blocks(const float* __restrict__ partial, const int32_t* __restr
                 [&](int c, float y) { emb[size_t(g) * H + c] = fmaxf(y, 0.f); });
 }
 
-// Block-wide sum in a fixed order: every thread contributes v, thread 0's tree is the same for
-// the same blockDim.  `scratch` holds blockDim.x floats.
+// Block-wide sum in a fixed order (lanes of a warp by a shuffle tree, then the warps' sums by one warp's
+// shuffle tree): the same for the same blockDim, two barriers.  Every thread contributes v and gets the sum;
+// `scratch` holds at least 32 floats.  blockDim is a multiple of 32.
 __device__ float block_sum(float v, float* scratch) {
-  scratch[threadIdx.x] = v;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  if (lane == 0) scratch[wid] = v;
   __syncthreads();
-  for (int s = blockDim.x >> 1; s > 0; s >>= 1) {
-    if (int(threadIdx.x) < s) scratch[threadIdx.x] += scratch[threadIdx.x + s];
-    __syncthreads();
-  }
-  const float r = scratch[0];
+  float r = lane < nw ? scratch[lane] : 0.f;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) r += __shfl_xor_sync(0xFFFFFFFFu, r, o);
+  __syncthreads();
+  return r;
+}
+__device__ float block_max(float v, float* scratch) {
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+  if (lane == 0) scratch[wid] = v;
+  __syncthreads();
+  float r = lane < nw ? scratch[lane] : -INFINITY;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) r = fmaxf(r, __shfl_xor_sync(0xFFFFFFFFu, r, o));
   __syncthreads();
   return r;
 }
@@ -223,13 +237,14 @@ __device__ U4 philox4x32_10(uint32_t k0, uint32_t k1, U4 c) {
 }
 
 __device__ unsigned long long block_sum_u64(unsigned long long v, unsigned long long* scratch) {
-  scratch[threadIdx.x] = v;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  if (lane == 0) scratch[wid] = v;
   __syncthreads();
-  for (int s = blockDim.x >> 1; s > 0; s >>= 1) {
-    if (int(threadIdx.x) < s) scratch[threadIdx.x] += scratch[threadIdx.x + s];
-    __syncthreads();
-  }
-  const unsigned long long r = scratch[0];
+  unsigned long long r = lane < nw ? scratch[lane] : 0ull;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) r += __shfl_xor_sync(0xFFFFFFFFu, r, o);
   __syncthreads();
   return r;
 }
@@ -337,14 +352,7 @@ k_env_policy(const float* __restrict__ emb, const float* __restrict__ logit,
     }
     if (valid) mx = fmaxf(mx, logit[a == A ? cur : cur + 1 + a]);
   }
-  scratch[tid] = mx;
-  __syncthreads();
-  for (int s = nt >> 1; s > 0; s >>= 1) {
-    if (tid < s) scratch[tid] = fmaxf(scratch[tid], scratch[tid + s]);
-    __syncthreads();
-  }
-  mx = scratch[0];
-  __syncthreads();
+  mx = block_max(mx, scratch);
   float se = 0.f;
   for (int a = tid; a <= A; a += nt) {
     const bool valid = (a == A) || (a < C && mk[a]);
