@@ -32,7 +32,8 @@ constexpr int TW = 4;            // warps per CTA
 constexpr int G = XRL_AGG_GROUPS;   // gather groups in flight per warp
 constexpr int GQ = XRL_AGG_GATHERS; // gathers (of four rows each) per group: one barrier, one wait per group
 constexpr int GV = 4 * GQ;          // vectors (rows) per group
-constexpr int BR = 32;           // destination rows per block
+constexpr int BR = 32;           // destination rows per block (large launches; small ones take 16 or 8, see
+                                 // aggregate_block_shift: with few rows a 32-row block per warp leaves most warps idle)
 constexpr int ITEMS = 160;       // list capacity, a multiple of 4
 
 // MERGED: the rows of Z carry their K {s_src, s_dst} pairs behind the 512 feature bytes, so one gather
@@ -180,7 +181,8 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
                 const T* __restrict__ Z, const float2* __restrict__ scores,
                 const float* __restrict__ bias, T* __restrict__ h_out, Window win,
                 const int32_t* __restrict__ seg_id, float* __restrict__ partial, int32_t nblocks,
-                const int32_t* __restrict__ self_idx, int32_t* status) {
+                const int32_t* __restrict__ self_idx, int32_t* status, int32_t br_shift) {
+  const int br = 1 << br_shift;                       // destination rows per block in this launch (8, 16 or 32)
   constexpr int VEC = VecOf<T>::N;
   constexpr int NP = VEC / 2;
   constexpr int H = 32 * VEC;
@@ -230,9 +232,9 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
     }
   };
 
-  for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * BR; r0 < win.row_end && alive;
-       r0 += int64_t(warps_total) * BR) {
-    const int nr = int(min(int64_t(BR), win.row_end - r0));
+  for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * br; r0 < win.row_end && alive;
+       r0 += int64_t(warps_total) * br) {
+    const int nr = int(min(int64_t(br), win.row_end - r0));
     __syncwarp();
     if (lane < nr) sm.rp[lane] = __ldg(rowptr + r0 + lane);
     if (lane == 0) sm.rp[nr] = __ldg(rowptr + r0 + nr);
@@ -247,7 +249,7 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
       for (int t = 0; t < NP; ++t) rsum[t] = make_f2(0.f, 0.f);
     }
     auto flush = [&]() {
-      float* dst = partial + size_t(first_seg ? int32_t(r0 / BR) : nblocks + cur_g) * H + c0;
+      float* dst = partial + size_t(first_seg ? int32_t(r0 >> br_shift) : nblocks + cur_g) * H + c0;
 #pragma unroll
       for (int t = 0; t < NP; t += 2) {
         float4 v;
@@ -418,6 +420,19 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
   }
 }
 
+}  // namespace
+
+// log2 of the destination rows one warp takes per block: 32, or 16 / 8 when 32-row blocks would not give every
+// resident warp of the grid a block (steps of the paper's size: 15 k rows are 480 blocks of 32 for 2,960 warps).
+int aggregate_block_shift(int64_t rows) {
+  const int64_t warps = int64_t(kNumSMs) * XRL_AGG_CTAS * TW;
+  if ((rows + 31) / 32 >= warps) return 5;
+  if ((rows + 15) / 16 >= warps) return 4;
+  return 3;
+}
+
+namespace {
+
 bool make_row_map(CUtensorMap* m, const void* ptr, CUtensorMapDataType dt, uint32_t elem_bytes,
                   uint64_t rows, uint32_t cols) {
   EncodeTiledFn fn = encode_fn();
@@ -461,12 +476,14 @@ int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const flo
     return -1;
   }
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
-  const int64_t nblocks = (rows + BR - 1) / BR;
-  int64_t nb = (rows + BR * TW - 1) / (BR * TW);
+  const int shift = aggregate_block_shift(rows);
+  const int64_t br = int64_t(1) << shift;
+  const int64_t nblocks = (rows + br - 1) / br;
+  int64_t nb = (rows + br * TW - 1) / (br * TW);
   if (nb > int64_t(kNumSMs) * XRL_AGG_CTAS) nb = int64_t(kNumSMs) * XRL_AGG_CTAS;
   k_aggregate_tma<T, K, READOUT, MERGED><<<int(nb), TW * 32, smem, st>>>(
       mz, ms, rowptr, col, static_cast<const T*>(Z), reinterpret_cast<const float2*>(scores), bias,
-      static_cast<T*>(h_out), win, seg_id, partial, int32_t(nblocks), self_idx, status);
+      static_cast<T*>(h_out), win, seg_id, partial, int32_t(nblocks), self_idx, status, int32_t(shift));
   return 1;
 }
 
@@ -507,7 +524,15 @@ bool aggregate_tma_shape(const Dims& d) {
 }
 
 // Partial-sum slots the fused variant writes for `rows` rows and B graphs.
-int64_t aggregate_readout_slots(int64_t rows, int64_t B) { return (rows + BR - 1) / BR + B; }
-int32_t aggregate_readout_blocks(int64_t rows) { return int32_t((rows + BR - 1) / BR); }
+// (an upper bound over every row count up to `rows`: small launches use smaller blocks, at most 2 x the warps
+// of a full grid of them)
+int64_t aggregate_readout_slots(int64_t rows, int64_t B) {
+  const int64_t full = (rows + BR - 1) / BR, small = 2 * int64_t(kNumSMs) * XRL_AGG_CTAS * TW;
+  return (full > small ? full : small) + B;
+}
+int32_t aggregate_readout_blocks(int64_t rows) {
+  const int shift = aggregate_block_shift(rows);
+  return int32_t((rows + (int64_t(1) << shift) - 1) >> shift);
+}
 
 }  // namespace xrl

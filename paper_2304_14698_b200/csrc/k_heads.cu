@@ -139,7 +139,7 @@ k_global_update(const float* __restrict__ partial, const int32_t* __restrict__ g
 template <int DEPTH>
 __global__ void __launch_bounds__(1024)
 k_global_update_blocks(const float* __restrict__ partial, const int32_t* __restrict__ node_off,
-                       int32_t nblocks, const float* __restrict__ g0, const float* __restrict__ Wg,
+                       int32_t nblocks, int bshift, const float* __restrict__ g0, const float* __restrict__ Wg,
                        const float* __restrict__ bg, float* __restrict__ emb, int H, int Dg) {
   extern __shared__ float u[];                   // [H + Dg], then blockDim floats of scratch
   float* part = u + H + Dg;
@@ -148,9 +148,9 @@ k_global_update_blocks(const float* __restrict__ partial, const int32_t* __restr
   for (int c = threadIdx.x; c < H; c += blockDim.x) {
     float s = 0.f;
     if (end > start) {
-      int32_t b0 = start >> 5;
-      if (start & 31) { s += partial[size_t(nblocks + g) * H + c]; ++b0; }
-      const int32_t b1 = (end - 1) >> 5;
+      int32_t b0 = start >> bshift;
+      if (start & ((1 << bshift) - 1)) { s += partial[size_t(nblocks + g) * H + c]; ++b0; }
+      const int32_t b1 = (end - 1) >> bshift;
       for (int32_t b = b0; b <= b1; ++b) s += partial[size_t(b) * H + c];
     }
     u[c] = s;
@@ -462,14 +462,15 @@ int launch_global_update(const Dims& d, const float* partial, const int32_t* gra
 }
 
 int launch_global_update_blocks(const Dims& d, const float* partial, const int32_t* node_off, int32_t nblocks,
-                                const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st) {
+                                int block_shift, const float* g0, const DevWeights& w, float* emb, int32_t B,
+                                cudaStream_t st) {
   if (B <= 0) return 0;
   const int nt = head_threads(B);
   const size_t smem = sizeof(float) * size_t(d.H + d.Dg + nt);
   if (few_ctas(B))
-    k_global_update_blocks<32><<<B, nt, smem, st>>>(partial, node_off, nblocks, g0, w.Wg, w.bg, emb, d.H, d.Dg);
+    k_global_update_blocks<32><<<B, nt, smem, st>>>(partial, node_off, nblocks, block_shift, g0, w.Wg, w.bg, emb, d.H, d.Dg);
   else
-    k_global_update_blocks<8><<<B, nt, smem, st>>>(partial, node_off, nblocks, g0, w.Wg, w.bg, emb, d.H, d.Dg);
+    k_global_update_blocks<8><<<B, nt, smem, st>>>(partial, node_off, nblocks, block_shift, g0, w.Wg, w.bg, emb, d.H, d.Dg);
   return 1;
 }
 

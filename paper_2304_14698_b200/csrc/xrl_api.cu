@@ -894,7 +894,8 @@ xrl_status xrl_encode(xrl_ctx* ctx, const xrl_batch* b, const float* g0, float* 
   slot = ctx->prof.begin(st);
   if (fused)
     k = launch_global_update_blocks(ctx->dims, ctx->partial.as<float>(), b->node_off.as<int32_t>(),
-                                    aggregate_readout_blocks(b->N), g0, ctx->dw, graph_emb, b->B, st);
+                                    aggregate_readout_blocks(b->N), aggregate_block_shift(b->N), g0, ctx->dw,
+                                    graph_emb, b->B, st);
   else
     k = launch_global_update(ctx->dims, ctx->partial.as<float>(), b->d_graph_chunk_off, g0, ctx->dw,
                              graph_emb, b->B, st);

@@ -162,10 +162,13 @@ int launch_aggregate_tma(const Dims& d, const int32_t* rowptr, const int32_t* co
                          const float* scores, const float* bias, void* h_out, Window win, int64_t buf_rows,
                          const int32_t* seg_id, float* partial, int32_t* status, cudaStream_t st,
                          const int32_t* self_idx = nullptr);
+int aggregate_block_shift(int64_t rows);           // log2(rows per block) the TMA aggregate uses for `rows` rows
 int64_t aggregate_readout_slots(int64_t rows, int64_t B);
 int32_t aggregate_readout_blocks(int64_t rows);
+// block_shift: aggregate_block_shift of the launch that wrote `partial`
 int launch_global_update_blocks(const Dims& d, const float* partial, const int32_t* node_off, int32_t nblocks,
-                                const float* g0, const DevWeights& w, float* emb, int32_t B, cudaStream_t st);
+                                int block_shift, const float* g0, const DevWeights& w, float* emb, int32_t B,
+                                cudaStream_t st);
 int launch_readout(const Dims& d, const void* h, const int32_t* chunk_row0, const int32_t* chunk_row1,
                    int32_t chunk_begin, int32_t chunk_end, float* partial, int32_t win_base,
                    cudaStream_t st, const int32_t* remap = nullptr);
