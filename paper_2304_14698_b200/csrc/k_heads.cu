@@ -145,15 +145,38 @@ k_global_update_blocks(const float* __restrict__ partial, const int32_t* __restr
   float* part = u + H + Dg;
   const int32_t g = blockIdx.x;
   const int32_t start = node_off[g], end = node_off[g + 1];
-  for (int c = threadIdx.x; c < H; c += blockDim.x) {
-    float s = 0.f;
-    if (end > start) {
-      int32_t b0 = start >> bshift;
-      if (start & ((1 << bshift) - 1)) { s += partial[size_t(nblocks + g) * H + c]; ++b0; }
-      const int32_t b1 = (end - 1) >> bshift;
-      for (int32_t b = b0; b <= b1; ++b) s += partial[size_t(b) * H + c];
+  // With more threads than columns the blocks' partial sums are added in P interleaved parts (part p takes the
+  // blocks b0 + p, b0 + p + P, ...), and the parts in order: a fixed order for a given launch shape.
+  const int P = int(blockDim.x) >= 2 * H ? int(blockDim.x) / H : 1;
+  if (P == 1) {
+    for (int c = threadIdx.x; c < H; c += blockDim.x) {
+      float s = 0.f;
+      if (end > start) {
+        int32_t b0 = start >> bshift;
+        if (start & ((1 << bshift) - 1)) { s += partial[size_t(nblocks + g) * H + c]; ++b0; }
+        const int32_t b1 = (end - 1) >> bshift;
+        for (int32_t b = b0; b <= b1; ++b) s += partial[size_t(b) * H + c];
+      }
+      u[c] = s;
     }
-    u[c] = s;
+  } else {
+    const int c = threadIdx.x % H, p = threadIdx.x / H;
+    float s = 0.f;
+    int32_t b0 = 0, b1 = -1;
+    if (end > start) {
+      b0 = start >> bshift;
+      if (start & ((1 << bshift) - 1)) ++b0;
+      b1 = (end - 1) >> bshift;
+    }
+    if (p < P)
+      for (int32_t b = b0 + p; b <= b1; b += P) s += partial[size_t(b) * H + c];
+    part[threadIdx.x] = s;
+    __syncthreads();
+    if (p == 0) {
+      float t = (end > start && (start & ((1 << bshift) - 1))) ? partial[size_t(nblocks + g) * H + c] : 0.f;
+      for (int q = 0; q < P; ++q) t += part[q * H + c];
+      u[c] = t;
+    }
   }
   for (int t = threadIdx.x; t < Dg; t += blockDim.x) u[H + t] = g0 ? g0[size_t(g) * Dg + t] : 0.f;
   __syncthreads();
@@ -220,6 +243,75 @@ k_policy_logit(const float* __restrict__ emb, const Mlp mlp, float* __restrict__
   __syncthreads();
   const float v = mlp_scalar<DEPTH>(x, H, mlp, y1, scratch);
   if (threadIdx.x == 0) logit[g] = v;
+}
+
+// The rest of a head's MLP behind its first layer: y1 = ReLU(W1^T x + b1) is given (hid floats in shared
+// memory); all threads return the result.
+template <int DEPTH>
+__device__ float mlp_tail(const float* y1, const Mlp& m, float* scratch) {
+  float contrib = 0.f;
+  if (m.hid2 <= 0) {
+    for (int c = threadIdx.x; c < m.hid; c += blockDim.x) contrib += y1[c] * m.w2[c];
+  } else {
+    dense_columns<DEPTH>(y1, m.hid, m.Wh, m.hid2, m.hid2, m.bh, scratch,
+                  [&](int c, float y) { contrib += fmaxf(y, 0.f) * m.w2[c]; });
+  }
+  return block_sum(contrib, scratch) + m.b2[0];
+}
+
+// ---- steps of few graphs and environments: policy scores and the value head's first layer in one launch ------
+// CTAs [0, B) are k_policy_logit.  CTAs B + e * VC + ch compute chunk ch (hid / VC columns) of the value head's
+// first layer for environment e: y1[e] = ReLU(W1^T [emb(current) | mean of the valid candidates' emb] + b1), the
+// candidate mean taken inside the CTA (part p of the threads adds candidates p, p + P, ... in order, the parts
+// in order).  The 2H x hid weights are then read by VC CTAs instead of by the one CTA of the environment.
+template <int DEPTH>
+__global__ void __launch_bounds__(1024)
+k_policy_value_hidden(const float* __restrict__ emb, const Mlp pm, float* __restrict__ logit, int H, int32_t B,
+                      const int32_t* __restrict__ env_off, const uint8_t* __restrict__ mask, int A, const Mlp vm,
+                      float* __restrict__ y1v, int VC) {
+  extern __shared__ float sm[];                  // policy: [H] + [blockDim] + [hid]; value: [2H] + [blockDim]
+  const int nt = blockDim.x, tid = threadIdx.x;
+  if (int32_t(blockIdx.x) < B) {
+    float* x = sm;
+    float* scratch = sm + H;
+    float* y1 = scratch + nt;
+    const int32_t g = blockIdx.x;
+    for (int c = tid; c < H; c += nt) x[c] = emb[size_t(g) * H + c];
+    __syncthreads();
+    const float v = mlp_scalar<DEPTH>(x, H, pm, y1, scratch);
+    if (tid == 0) logit[g] = v;
+    return;
+  }
+  float* u = sm;                                 // [2H]
+  float* scratch = sm + 2 * H;                   // [blockDim]
+  const int32_t e = (int32_t(blockIdx.x) - B) / VC, ch = (int32_t(blockIdx.x) - B) % VC;
+  const int32_t cur = env_off[e];
+  const int32_t C = env_off[e + 1] - cur - 1;
+  const uint8_t* mk = mask + size_t(e) * A;
+  float cnt = 0.f;
+  for (int a = tid; a < C && a < A; a += nt) cnt += mk[a] ? 1.f : 0.f;
+  const float nv = block_sum(cnt, scratch);
+  const int P = nt >= 2 * H ? nt / H : 1;
+  {
+    const int c = tid % H, p = tid / H;
+    float s = 0.f;
+    if (p < P && tid < P * H)
+      for (int a = p; a < C && a < A; a += P)
+        if (mk[a]) s += emb[size_t(cur + 1 + a) * H + c];
+    scratch[tid] = s;
+    __syncthreads();
+    if (tid < H) {
+      float t = 0.f;
+      for (int q = 0; q < P; ++q) t += scratch[q * H + tid];
+      u[tid] = emb[size_t(cur) * H + tid];
+      u[H + tid] = nv > 0.f ? t / nv : 0.f;
+    }
+    __syncthreads();
+  }
+  const int CW = (vm.hid + VC - 1) / VC, c_lo = ch * CW, ncols = min(CW, vm.hid - c_lo);
+  if (ncols > 0)
+    dense_columns<DEPTH>(u, 2 * H, vm.W1 + c_lo, vm.hid, ncols, vm.b1 + c_lo, scratch,
+                  [&](int c, float y) { y1v[size_t(e) * vm.hid + c_lo + c] = fmaxf(y, 0.f); });
 }
 
 // ---- Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) -----------------------------------------
@@ -331,7 +423,7 @@ k_env_policy(const float* __restrict__ emb, const float* __restrict__ logit,
              const int32_t* __restrict__ env_off, const uint8_t* __restrict__ mask,
              const Mlp vmlp, float* __restrict__ probs,
              float* __restrict__ value, int32_t* __restrict__ action, int H, int A,
-             uint64_t seed, uint64_t step, int32_t* status) {
+             uint64_t seed, uint64_t step, int32_t* status, const float* __restrict__ y1_pre) {
   extern __shared__ unsigned long long sm64[];   // [nt + 1] u64, then floats
   const int nt = blockDim.x, tid = threadIdx.x;
   float* scratch = reinterpret_cast<float*>(sm64 + nt + 1);   // [nt]
@@ -363,14 +455,22 @@ k_env_policy(const float* __restrict__ emb, const float* __restrict__ logit,
   const float denom = block_sum(se, scratch);
   for (int a = tid; a <= A; a += nt) pr[a] = pr[a] / denom;     // each thread rewrites its own entries
 
-  // value head input: [ emb(current) | mean of emb over the valid candidates ]
-  for (int c = tid; c < H; c += nt) u[c] = emb[size_t(cur) * H + c];
-  float cnt = 0.f;
-  for (int a = tid; a < C; a += nt) cnt += mk[a] ? 1.f : 0.f;
-  const float nv = block_sum(cnt, scratch);
-  for (int c = tid; c < H; c += nt) u[H + c] = nv > 0.f ? cand_sum[size_t(e) * H + c] / nv : 0.f;
-  __syncthreads();
-  const float v = mlp_scalar<DEPTH>(u, 2 * H, vmlp, y1, scratch);
+  float v;
+  if (y1_pre != nullptr) {
+    // the value head's first layer was computed by k_policy_value_hidden: the rest of the MLP
+    for (int c = tid; c < vmlp.hid; c += nt) y1[c] = y1_pre[size_t(e) * vmlp.hid + c];
+    __syncthreads();
+    v = mlp_tail<DEPTH>(y1, vmlp, scratch);
+  } else {
+    // value head input: [ emb(current) | mean of emb over the valid candidates ]
+    for (int c = tid; c < H; c += nt) u[c] = emb[size_t(cur) * H + c];
+    float cnt = 0.f;
+    for (int a = tid; a < C; a += nt) cnt += mk[a] ? 1.f : 0.f;
+    const float nv = block_sum(cnt, scratch);
+    for (int c = tid; c < H; c += nt) u[H + c] = nv > 0.f ? cand_sum[size_t(e) * H + c] / nv : 0.f;
+    __syncthreads();
+    v = mlp_scalar<DEPTH>(u, 2 * H, vmlp, y1, scratch);
+  }
   if (tid == 0) value[e] = v;
 
   if (action != nullptr) {
@@ -481,11 +581,25 @@ int launch_heads(const Dims& d, const DevWeights& w, const float* emb, const int
   if (B <= 0 || num_envs <= 0) return 0;
   const Mlp pm{w.pW1, w.pb1, w.pWh, w.pbh, w.pw2, w.pb2, d.Hm, d.Hm2};
   const Mlp vm{w.vW1, w.vb1, w.vWh, w.vbh, w.vw2, w.vb2, d.Hm, d.Hm2};
+  float* cand_sum = logit_ws + B;                 // [num_envs x H], behind the per-graph logits
+  // Steps of few graphs and environments with a short action space (the paper's own sizes): two launches, the
+  // value head's first layer spread over kValueChunks CTAs per environment next to the policy CTAs.
+  constexpr int kValueChunks = 8;
+  if (B + num_envs * kValueChunks <= kNumSMs && d.A <= 256 && d.Hm <= d.H) {
+    const int nt = 1024;
+    const size_t sm1 = sizeof(float) * size_t(2 * d.H + nt + d.Hm);
+    float* y1v = cand_sum;                        // [num_envs x Hm] (Hm <= H): the candidate sums are not needed here
+    k_policy_value_hidden<32><<<B + num_envs * kValueChunks, nt, sm1, st>>>(emb, pm, logit_ws, d.H, B, env_off, mask,
+                                                                         d.A, vm, y1v, kValueChunks);
+    const size_t smem = sizeof(unsigned long long) * size_t(nt + 1) + sizeof(float) * size_t(nt + 2 * d.H + d.Hm);
+    k_env_policy<32><<<num_envs, nt, smem, st>>>(emb, logit_ws, cand_sum, env_off, mask, vm, probs, value, action,
+                                                 d.H, d.A, seed, step, status, y1v);
+    return 2;
+  }
   const int pnt = head_threads(B);
   const size_t psm = sizeof(float) * size_t(d.H + pnt + d.Hm);
   if (few_ctas(B)) k_policy_logit<32><<<B, pnt, psm, st>>>(emb, pm, logit_ws, d.H);
   else k_policy_logit<8><<<B, pnt, psm, st>>>(emb, pm, logit_ws, d.H);
-  float* cand_sum = logit_ws + B;                 // [num_envs x H], behind the per-graph logits
   k_candidate_sum<<<dim3(num_envs, (d.H + 31) / 32), 1024, 0, st>>>(emb, env_off, mask, cand_sum, d.H, d.A);
   int want = d.H > d.A + 1 ? d.H : d.A + 1;
   if (want < 256) want = 256;               // enough threads to split the value head's dense map
@@ -494,10 +608,10 @@ int launch_heads(const Dims& d, const DevWeights& w, const float* emb, const int
   const size_t smem = sizeof(unsigned long long) * size_t(nt + 1) + sizeof(float) * size_t(nt + 2 * d.H + d.Hm);
   if (few_ctas(num_envs))
     k_env_policy<32><<<num_envs, nt, smem, st>>>(emb, logit_ws, cand_sum, env_off, mask, vm, probs, value, action,
-                                                 d.H, d.A, seed, step, status);
+                                                 d.H, d.A, seed, step, status, nullptr);
   else
     k_env_policy<8><<<num_envs, nt, smem, st>>>(emb, logit_ws, cand_sum, env_off, mask, vm, probs, value, action,
-                                                d.H, d.A, seed, step, status);
+                                                d.H, d.A, seed, step, status, nullptr);
   return 3;
 }
 
