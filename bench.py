@@ -470,9 +470,9 @@ def main():
         "profiled_pass": {"ms_per_step": round(prof_ms_per_step, 4), "kernels_ms": round(kernels_ms, 4),
                           "gap_ms": round(prof_ms_per_step - kernels_ms, 4), "sm_mhz": mhz_p,
                           "ms_x_ghz": round(prof_ms_per_step * mhz_p / 1e3, 3) if mhz_p else None},
-        # (for steps submitted as one recorded graph the timed pass is shorter than the sum of directly launched
-        # kernels: there the profiled pass's own gap is the meaningful one)
-        "gap_ms": round(ms_per_step - kernels_ms, 4) if N > agent.GRAPH_MAX_NODES else None,
+        # the step's time outside its kernels, taken within the profiled pass (the timed pass may run at other
+        # clocks, or as one recorded graph, so its time minus these kernel times would mix two things)
+        "gap_ms": round(prof_ms_per_step - kernels_ms, 4),
         "ms_x_ghz": round(ms_per_step * mhz / 1e3, 3) if mhz else None,
         "step_hbm_frac": step_alg / (ms_per_step * 1e-3) / 1e9 / peak,
         "roofline": {"kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peak,
