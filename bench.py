@@ -73,6 +73,10 @@ def algorithmic_bytes(family, m, N, E):
         return N * (H * b + 4 + 2 * K * 4) + 4 * E + (N // 32 + 1) * H * 4
     if family == "readout":
         return N * H * b
+    if family == "layers_fused":     # all attention layers in one launch: the sum of its layers' bytes
+        L = m["L"]
+        return (L * algorithmic_bytes("transform", m, N, E) + (L - 1) * algorithmic_bytes("aggregate", m, N, E)
+                + algorithmic_bytes("aggregate_readout", m, N, E))
     if family == "pack":             # read edge lists twice + op, write col/seg_id/rowptr/tmp
         return E * (2 * 8 + 4 + 4 + 4) + N * (4 + 4 + 4 + 4)
     return 0
@@ -426,12 +430,15 @@ def main():
     fused = 1 if prof["aggregate_readout"]["launches"] > 0 else 0
     calls = {"pack": 1, "node_update": 1, "transform": m["L"], "aggregate": m["L"] - fused,
              "aggregate_readout": fused, "readout": 1 - fused}       # launches of each kernel family per step
+    if prof["layers_fused"]["launches"] > 0:     # small steps: every attention layer (and the Eq. 8 sum) in one launch
+        calls = {"pack": 1, "node_update": 1, "layers_fused": 1, "transform": 0, "aggregate": 0,
+                 "aggregate_readout": 0, "readout": 0}
     # the plain and the readout-fused attention launches are one kernel (two instantiations): the dominant
     # kernel is chosen by the time of the kernel, the roofline line is that of its plain instantiation and
     # `families` lists every family's own fraction
     kernel_of = {"aggregate_readout": "aggregate"}
     per_kernel = {}
-    for f in ("transform", "aggregate", "aggregate_readout", "node_update", "readout", "pack"):
+    for f in ("transform", "aggregate", "aggregate_readout", "node_update", "readout", "pack", "layers_fused"):
         per_kernel[kernel_of.get(f, f)] = per_kernel.get(kernel_of.get(f, f), 0.0) + fam_ms[f]
     dominant = max(per_kernel, key=per_kernel.get)
     if dominant == "aggregate" and calls["aggregate"] == 0:

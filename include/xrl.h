@@ -395,7 +395,8 @@ xrl_status xrl_pack_csr_static(int32_t device, int32_t num_op_types, int32_t num
 /* Per-step timing of the path's steps with CUDA events on the launching stream (off by
  * default).  Families: 0 pack (Section 3.3.2), 1 node update (Eq. 6), 2 transform and 3
  * score/softmax/aggregate (Eq. 7), 4 readout (Eq. 8 sum), 5 global update + heads, 6 the last
- * aggregate layer when it is fused with the readout.
+ * aggregate layer when it is fused with the readout, 7 all attention layers of a small step when
+ * they run as one launch (then 2, 3 and 6 stay empty).
  * xrl_profile(ctx, 1) starts recording (synchronises the device, drops earlier records);
  * xrl_profile_read synchronises the device, fills total_ms / launches (HOST,
  * [num_families]) with the time and kernel count accumulated per family since the last read,

@@ -28,7 +28,8 @@ EXPORTED_SYMBOLS = [
     "xrl_graph_begin", "xrl_graph_launch", "xrl_batch_set_edge_attr", "xrl_ppo_grad", "xrl_gae",
     "xrl_grad_weigh", "xrl_grad_unweigh", "xrl_init_weights",
 ]
-PROFILE_FAMILIES = ["pack", "node_update", "transform", "aggregate", "readout", "heads", "aggregate_readout"]
+PROFILE_FAMILIES = ["pack", "node_update", "transform", "aggregate", "readout", "heads", "aggregate_readout",
+                    "layers_fused"]
 
 
 class XrlError(RuntimeError):

@@ -46,7 +46,7 @@ size_t storage_bytes(int dtype) { return dtype == XRL_BF16 ? 2 : 4; }
 
 // Optional per-kernel-family timing: CUDA events recorded on the launching stream around every
 // launcher call.  Families index the steps of the path.
-enum { FAM_PACK = 0, FAM_EMBED, FAM_XFORM, FAM_AGG, FAM_READOUT, FAM_HEADS, FAM_AGG_READOUT, FAM_COUNT };
+enum { FAM_PACK = 0, FAM_EMBED, FAM_XFORM, FAM_AGG, FAM_READOUT, FAM_HEADS, FAM_AGG_READOUT, FAM_LAYERS, FAM_COUNT };
 
 struct Profiler {
   bool on = false;
@@ -88,6 +88,8 @@ struct xrl_ctx {
   DeviceBuf w_store;        // storage-type copies of W0 and the layer matrices (+ transposes)
   DevWeights dw;
   DeviceBuf h, Z, scores, partial, logits, status;
+  DeviceBuf Z2;             // second Z buffer of the all-layers kernel for small steps (its row capacity: Z2_rows)
+  int64_t Z2_rows = 0;
   int32_t max_chunks = 0;
   int64_t launches_pack = 0, launches_encode = 0, launches_heads = 0;
   // delta encoding workspace (allocated on the first xrl_encode_delta)
@@ -516,6 +518,20 @@ int run_node_layers(xrl_ctx* ctx, const xrl_batch* b, int layers, cudaStream_t s
   pf.end(FAM_EMBED, slot, k, st);
   nvtxRangePop();
   int n = k;
+  // a small step: all attention layers in one cooperative launch (same arithmetic, same outputs)
+  if (!hs && !zs && !ss && win.row_begin == 0 && win.row_end == b->N && b->N <= ctx->Z2_rows && ctx->use_umma &&
+      layers_coop_supported(d, layers, b->N)) {
+    NvtxRange nvtx_layers("xrl:attention layers (Eq. 7), one launch");
+    slot = pf.begin(st);
+    k = launch_layers_coop(d, ctx->dw, layers, ctx->h.p, ctx->Z.p, ctx->Z2.p, gat_rowptr, gat_col, b->N,
+                           b->seg_id.as<int32_t>(), fuse_readout ? ctx->partial.as<float>() : nullptr,
+                           ctx->status.as<int32_t>(), ctx->status.as<uint32_t>() + 2, st);
+    if (k >= 0) {
+      pf.end(FAM_LAYERS, slot, k, st);
+      if (fuse_readout && fused) *fused = true;
+      return n + k;
+    }
+  }
   for (int l = 0; l < layers; ++l) {
     const void* h_in = hs ? hs[l] : ctx->h.p;
     void* h_out = hs ? hs[l + 1] : ctx->h.p;
@@ -635,6 +651,12 @@ xrl_status xrl_create(const xrl_model_config* cfg, int32_t device, xrl_ctx** out
   A(ctx->w0ext, ctx->use_umma_embed ? 2 * H * size_t(embed_umma_kpad(ctx->dims)) : 0);
   A(ctx->h, sb * N * H);
   A(ctx->Z, N * z_row_bytes(ctx->dims));
+  // XRL_NO_FUSED_LAYERS=1 keeps one launch per transform / attention layer for every size (debugging aid)
+  if (layers_coop_supported(ctx->dims, cfg->layers > 8 ? 8 : (cfg->layers < 1 ? 1 : cfg->layers), 1) &&
+      getenv("XRL_NO_FUSED_LAYERS") == nullptr) {
+    ctx->Z2_rows = int64_t(N < size_t(layers_coop_max_rows()) ? N : size_t(layers_coop_max_rows()));
+    A(ctx->Z2, size_t(ctx->Z2_rows) * z_row_bytes(ctx->dims));
+  }
   A(ctx->scores, 8 * N * size_t(cfg->heads));
   {
     const size_t slots_fused = size_t(aggregate_readout_slots(cfg->max_nodes, cfg->max_graphs));
@@ -642,8 +664,8 @@ xrl_status xrl_create(const xrl_model_config* cfg, int32_t device, xrl_ctx** out
     A(ctx->partial, 4 * slots * H);
   }
   A(ctx->logits, 4 * (size_t(cfg->max_graphs) + size_t(cfg->max_envs) * H));   // logits, then candidate sums
-  A(ctx->status, 4);
-  if (e == cudaSuccess) e = cudaMemset(ctx->status.p, 0, 4);
+  A(ctx->status, 16);          // [0] the device status word; [2], [3] the all-layers kernel's barrier counters
+  if (e == cudaSuccess) e = cudaMemset(ctx->status.p, 0, 16);
   if (e != cudaSuccess) {
     cudaGetLastError();
     xrl_destroy(ctx);
@@ -658,7 +680,7 @@ void xrl_destroy(xrl_ctx* ctx) {
   cudaSetDevice(ctx->device);
   cudaDeviceSynchronize();
   DeviceBuf* bufs[] = {&ctx->w0ext, &ctx->w_f32, &ctx->w_store, &ctx->h, &ctx->Z, &ctx->scores,
-                       &ctx->partial, &ctx->logits, &ctx->status, &ctx->bw};
+                       &ctx->partial, &ctx->logits, &ctx->status, &ctx->bw, &ctx->Z2};
   for (DeviceBuf* d : bufs) d->release();
   ctx->prof.release();
   ctx->dl_ints.release(); ctx->dl_col.release(); ctx->dl_scan.release();

@@ -88,6 +88,9 @@ inline size_t z_row_bytes(const Dims& d) {
   return size_t(d.H) * (d.dtype == XRL_BF16 ? 2 : 4) + (d.zmerged ? size_t(8) * d.K : 0);
 }
 bool aggregate_tma_shape(const Dims& d);
+// all attention layers of a small step in one cooperative launch (bf16, hidden 256, merged Z rows)
+bool layers_coop_supported(const Dims& d, int layers, int64_t rows);
+int64_t layers_coop_max_rows();
 
 // Opt-in to large dynamic shared memory is a per-device function attribute: remember it per device.
 template <typename Kernel>
@@ -162,6 +165,12 @@ int launch_aggregate_tma(const Dims& d, const int32_t* rowptr, const int32_t* co
                          const float* scores, const float* bias, void* h_out, Window win, int64_t buf_rows,
                          const int32_t* seg_id, float* partial, int32_t* status, cudaStream_t st,
                          const int32_t* self_idx = nullptr);
+// h is read and overwritten; Z0 / Z1: two buffers of `rows` merged Z rows; partial != nullptr: the last layer leaves
+// the per-block sums of Eq. 8 instead of node features; sync: two zeroed words only this kernel touches.
+// Returns kernels launched or -1 (not handled / refused).
+int launch_layers_coop(const Dims& d, const DevWeights& dw, int layers, void* h, void* Z0, void* Z1,
+                       const int32_t* rowptr, const int32_t* col, int64_t rows, const int32_t* seg_id,
+                       float* partial, int32_t* status, uint32_t* sync, cudaStream_t st);
 int aggregate_block_shift(int64_t rows);           // log2(rows per block) the TMA aggregate uses for `rows` rows
 int64_t aggregate_readout_slots(int64_t rows, int64_t B);
 int32_t aggregate_readout_blocks(int64_t rows);
