@@ -35,8 +35,9 @@ constexpr int GQ = XRL_AGG_GATHERS; // gathers (of four rows each) per group: on
 
 // One layer per launch: warp w of the grid takes blocks w, w + (warps of the grid), ... of 2^br_shift
 // destination rows (32 in large launches; small ones take 16 or 8, see aggregate_block_shift: with few
-// rows a 32-row block per warp leaves most warps idle).
-template <typename T, int K, bool READOUT, bool MERGED>
+// rows a 32-row block per warp leaves most warps idle).  SEQ: see aggregate_warp; set for the small launches that
+// the all-layers kernel can replace, whose results it must reproduce bit for bit.
+template <typename T, int K, bool READOUT, bool MERGED, bool SEQ>
 __global__ void __launch_bounds__(TW * 32, XRL_AGG_CTAS)
 k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant__ CUtensorMap map_s,
                 const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
@@ -49,7 +50,7 @@ k_aggregate_tma(const __grid_constant__ CUtensorMap map_z, const __grid_constant
   Smem& sm = reinterpret_cast<Smem*>(tma_smem_raw)[threadIdx.x >> 5];
   const int64_t step = int64_t((gridDim.x * blockDim.x) >> 5) << br_shift;
   int64_t next = int64_t(win.row_begin) + (int64_t((blockIdx.x * blockDim.x + threadIdx.x) >> 5) << br_shift);
-  const bool alive = aggregate_warp<T, K, READOUT, MERGED, G, GQ>(
+  const bool alive = aggregate_warp<T, K, READOUT, MERGED, G, GQ, SEQ>(
       &map_z, &map_s, rowptr, col, Z, scores, bias, h_out, win, seg_id, partial, nblocks, self_idx, br_shift, sm,
       [&]() -> int64_t {
         const int64_t r = next;
@@ -88,13 +89,13 @@ bool make_row_map(CUtensorMap* m, const void* ptr, CUtensorMapDataType dt, uint3
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <typename T, int K, bool READOUT, bool MERGED>
-int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const float* scores, const float* bias,
+template <typename T, int K, bool READOUT, bool MERGED, bool SEQ>
+int launch_k_seq(const int32_t* rowptr, const int32_t* col, const void* Z, const float* scores, const float* bias,
              void* h_out, Window win, int64_t buf_rows, const int32_t* seg_id, float* partial,
              const int32_t* self_idx, int32_t* status, cudaStream_t st) {
   static bool attr[64] = {};
   const size_t smem = sizeof(WarpSmem<K, MERGED, G, GQ>) * TW;
-  if (!ensure_dynamic_smem(k_aggregate_tma<T, K, READOUT, MERGED>, int(smem), attr)) return -1;
+  if (!ensure_dynamic_smem(k_aggregate_tma<T, K, READOUT, MERGED, SEQ>, int(smem), attr)) return -1;
   constexpr bool is_bf16 = sizeof(T) == 2;
   CUtensorMap mz, ms;
   if (MERGED) {
@@ -111,10 +112,23 @@ int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const flo
   const int64_t nblocks = (rows + br - 1) / br;
   int64_t nb = (rows + br * TW - 1) / (br * TW);
   if (nb > int64_t(kNumSMs) * XRL_AGG_CTAS) nb = int64_t(kNumSMs) * XRL_AGG_CTAS;
-  k_aggregate_tma<T, K, READOUT, MERGED><<<int(nb), TW * 32, smem, st>>>(
+  k_aggregate_tma<T, K, READOUT, MERGED, SEQ><<<int(nb), TW * 32, smem, st>>>(
       mz, ms, rowptr, col, static_cast<const T*>(Z), reinterpret_cast<const float2*>(scores), bias,
       static_cast<T*>(h_out), win, seg_id, partial, int32_t(nblocks), self_idx, status, int32_t(shift));
   return 1;
+}
+
+
+template <typename T, int K, bool READOUT, bool MERGED>
+int launch_k(const int32_t* rowptr, const int32_t* col, const void* Z, const float* scores, const float* bias,
+             void* h_out, Window win, int64_t buf_rows, const int32_t* seg_id, float* partial,
+             const int32_t* self_idx, int32_t* status, cudaStream_t st) {
+  // launches of fewer than 32 rows per block are the ones the all-layers kernel can stand in for (merged rows only)
+  if (MERGED && aggregate_block_shift(int64_t(win.row_end) - win.row_begin) < 5)
+    return launch_k_seq<T, K, READOUT, MERGED, MERGED>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, seg_id,
+                                                       partial, self_idx, status, st);
+  return launch_k_seq<T, K, READOUT, MERGED, false>(rowptr, col, Z, scores, bias, h_out, win, buf_rows, seg_id,
+                                                    partial, self_idx, status, st);
 }
 
 }  // namespace

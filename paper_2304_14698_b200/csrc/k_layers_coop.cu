@@ -187,11 +187,11 @@ __global__ void __launch_bounds__(kThreads, 1) k_layers_coop(const __grid_consta
       };
       bool alive;
       if (p.partial != nullptr && l == p.layers - 1)
-        alive = aggtma::aggregate_warp<bf16, K, true, true, AG, AGQ>(
+        alive = aggtma::aggregate_warp<bf16, K, true, true, AG, AGQ, true>(
             &p.map_zg[zb], &p.map_zg[zb], p.rowptr, p.col, p.Z[zb], nullptr, p.bias[l], p.h, win, p.seg_id,
             p.partial, p.nblocks, nullptr, p.br_shift, sm, next_block);
       else
-        alive = aggtma::aggregate_warp<bf16, K, false, true, AG, AGQ>(
+        alive = aggtma::aggregate_warp<bf16, K, false, true, AG, AGQ, true>(
             &p.map_zg[zb], &p.map_zg[zb], p.rowptr, p.col, p.Z[zb], nullptr, p.bias[l], p.h, win, p.seg_id,
             nullptr, p.nblocks, nullptr, p.br_shift, sm, next_block);
       if (!alive) {

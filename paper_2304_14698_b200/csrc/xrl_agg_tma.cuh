@@ -158,7 +158,10 @@ __device__ __forceinline__ void raise_reference(float ev, float& m, float& l, F2
 // (k_global_update_blocks adds them per graph in a fixed order; needs row_begin = win_base = 0, and
 // block b = first row >> br_shift).  The ring's barriers are initialised here: call it with no copy of
 // this warp in flight.  Returns false when a wait ran out (the caller reports it).
-template <typename T, int K, bool READOUT, bool MERGED, int G, int GQ, typename NextBlock>
+// SEQ: producers taken two at a time are added exactly as if taken singly (one more addition and compare per
+// pair); without it the pair's weights are summed first and one overflow test serves both, which is faster
+// and equal up to rounding.  Kernels whose results must agree bit for bit use the same setting.
+template <typename T, int K, bool READOUT, bool MERGED, int G, int GQ, bool SEQ, typename NextBlock>
 __device__ __forceinline__ bool aggregate_warp(
     const CUtensorMap* map_z_p, const CUtensorMap* map_s_p, const int32_t* __restrict__ rowptr,
     const int32_t* __restrict__ col, const T* __restrict__ Z, const float2* __restrict__ scores,
@@ -350,29 +353,39 @@ __device__ __forceinline__ bool aggregate_warp(
           t += 2;
           if ((w -= 2) == 0) advance();
           const float ev0 = lrelu(sc0.x + sd), ev1 = lrelu(sc1.x + sd);
-          // (the arithmetic is that of taking the two one after the other, so that a row's result does not
-          // depend on how its producers fall into pairs, i.e. on the ring's geometry)
-          if (fmaxf(ev0, ev1) > m + 32.f) {
-            F2 z[NP];
-            if (ev0 > m + 32.f) raise_reference<NP>(ev0, m, l, acc);
-            const float pa = fast_exp2(ev0 - m);
-            l += pa;
-            to_pairs(raw0, z);
-            const F2 qa = make_f2(pa, pa);
+          float p0, p1;
+          if (SEQ) {
+            // the arithmetic of taking the two one after the other, so that a row's result does not depend on how
+            // its producers fall into pairs, i.e. on the ring's geometry
+            if (fmaxf(ev0, ev1) > m + 32.f) {
+              F2 z[NP];
+              if (ev0 > m + 32.f) raise_reference<NP>(ev0, m, l, acc);
+              const float pa = fast_exp2(ev0 - m);
+              l += pa;
+              to_pairs(raw0, z);
+              const F2 qa = make_f2(pa, pa);
 #pragma unroll
-            for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], qa, z[t2]);
-            if (ev1 > m + 32.f) raise_reference<NP>(ev1, m, l, acc);
-            const float pb = fast_exp2(ev1 - m);
-            l += pb;
-            to_pairs(raw1, z);
-            const F2 qb = make_f2(pb, pb);
+              for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], qa, z[t2]);
+              if (ev1 > m + 32.f) raise_reference<NP>(ev1, m, l, acc);
+              const float pb = fast_exp2(ev1 - m);
+              l += pb;
+              to_pairs(raw1, z);
+              const F2 qb = make_f2(pb, pb);
 #pragma unroll
-            for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], qb, z[t2]);
-            continue;
+              for (int t2 = 0; t2 < NP; ++t2) fma2(acc[t2], qb, z[t2]);
+              continue;
+            }
+            p0 = fast_exp2(ev0 - m);
+            p1 = fast_exp2(ev1 - m);
+            l += p0;
+            l += p1;
+          } else {
+            const float evm = fmaxf(ev0, ev1);
+            if (evm > m + 32.f) raise_reference<NP>(evm, m, l, acc);
+            p0 = fast_exp2(ev0 - m);
+            p1 = fast_exp2(ev1 - m);
+            l += p0 + p1;
           }
-          const float p0 = fast_exp2(ev0 - m), p1 = fast_exp2(ev1 - m);
-          l += p0;
-          l += p1;
           F2 z0[NP], z1[NP];
           to_pairs(raw0, z0);
           to_pairs(raw1, z1);
