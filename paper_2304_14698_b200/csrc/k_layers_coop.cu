@@ -11,8 +11,8 @@
 //               destination rows and gathers the producers' Z rows with the TMA unit.
 // The attention phase reads Z rows of other CTAs' tiles, so a grid-wide barrier separates it from the
 // transform phase (the launch is cooperative, so all CTAs are resident; the barrier is a counter in
-// global memory that every CTA adds to and then polls, with the same time limit as every other wait); the next transform reads only rows this CTA has just
-// written, so a CTA barrier is enough there.  Z alternates between two buffers: a CTA that is already
+// global memory that every CTA adds to and then polls, with a limit like every other wait); the next
+// transform reads only rows this CTA has just written, so a CTA barrier is enough there.  Z alternates between two buffers: a CTA that is already
 // transforming layer l + 1 must not overwrite rows a slower CTA still gathers for layer l.  W of the
 // next layer streams into shared memory during the attention phase, whose gather rings live where the
 // transform's A stages and output staging are.  Tensor memory is allocated once.
