@@ -1,7 +1,9 @@
 // Dense node transform of a graph-attention layer, Z = h W (paper Eq. 7, the "W h_j" term), on
 // the CUDA cores with fp32 accumulation.  This is the path for fp32 storage (whose tolerance a
 // single-pass reduced-precision tensor-core product cannot guarantee) and for hidden sizes the
-// tensor-core kernel is not built for.  The attention half-scores are taken from Z by k_scores.
+// tensor-core kernel is not built for.  The attention half-scores are taken from the accumulators in the
+// kernel's last step when one tile spans all H columns, the storage is fp32 and a head is 4, 8, ... 128 columns
+// wide (SCORES); otherwise from Z by k_scores.
 #include "xrl_internal.cuh"
 
 namespace xrl {
@@ -10,9 +12,25 @@ namespace {
 
 constexpr int BM = 64, BN = 64, BK = 16;
 
-template <typename T>
+// Half-scores of one row's 4-column group held by this thread: partial dot products with the attention
+// vectors, summed over the `g` consecutive lanes that hold the same head of the same row (g a power of two
+// <= 16; those lanes differ in the low bits of the lane id only).  Every lane gets the sums.
+__device__ __forceinline__ void head_partial(const float (&z)[4], const float* __restrict__ a_src,
+                                             const float* __restrict__ a_dst, int c, int g, float& ss, float& sd) {
+  const float4 s = __ldg(reinterpret_cast<const float4*>(a_src + c));
+  const float4 t = __ldg(reinterpret_cast<const float4*>(a_dst + c));
+  ss = fmaf(z[3], s.w, fmaf(z[2], s.z, fmaf(z[1], s.y, z[0] * s.x)));
+  sd = fmaf(z[3], t.w, fmaf(z[2], t.z, fmaf(z[1], t.y, z[0] * t.x)));
+  for (int o = 1; o < g; o <<= 1) {
+    ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+    sd += __shfl_xor_sync(0xFFFFFFFFu, sd, o);
+  }
+}
+
+template <typename T, bool SCORES>
 __global__ void __launch_bounds__(256)
-k_xform_simt(const T* __restrict__ h, const T* __restrict__ W, T* __restrict__ Z, int H, int rows) {
+k_xform_simt(const T* __restrict__ h, const T* __restrict__ W, T* __restrict__ Z, int H, int rows,
+             const float* __restrict__ a_src, const float* __restrict__ a_dst, float2* __restrict__ scores, int K) {
   __shared__ float As[BK][BM + 4];
   __shared__ float Bs[BK][BN + 4];
   const int tid = threadIdx.x;
@@ -60,6 +78,13 @@ k_xform_simt(const T* __restrict__ h, const T* __restrict__ W, T* __restrict__ Z
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int64_t r = row0 + ty * 4 + i;
+    if (SCORES) {                               // (every lane takes part in the shuffles)
+      const int d = H / K, g = d >> 2, c = tx * 4;
+      float ss = 0.f, sd = 0.f;
+      const float z[4] = {acc[i][0], acc[i][1], acc[i][2], acc[i][3]};
+      head_partial(z, a_src, a_dst, c < H ? c : 0, g, ss, sd);
+      if (r < rows && c < H && (tx & (g - 1)) == 0) scores[size_t(r) * K + c / d] = make_float2(ss * kLog2e, sd * kLog2e);
+    }
     if (r >= rows) continue;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -88,9 +113,10 @@ __device__ __forceinline__ void load4<bf16>(const bf16* p, bool ok, float (&v)[4
   v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xFFFF0000u);
 }
 
-template <typename T>
+template <typename T, bool SCORES>
 __global__ void __launch_bounds__(256)
-k_xform_simt128(const T* __restrict__ h, const T* __restrict__ W, T* __restrict__ Z, int H, int rows) {
+k_xform_simt128(const T* __restrict__ h, const T* __restrict__ W, T* __restrict__ Z, int H, int rows,
+                const float* __restrict__ a_src, const float* __restrict__ a_dst, float2* __restrict__ scores, int K) {
   __shared__ __align__(16) float As[TK][TM];
   __shared__ __align__(16) float Bs[TK][TN];
   const int tid = threadIdx.x;
@@ -139,6 +165,28 @@ k_xform_simt128(const T* __restrict__ h, const T* __restrict__ W, T* __restrict_
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const int64_t r = row0 + (i < 4 ? ty * 4 + i : 64 + ty * 4 + (i - 4));
+    if (SCORES) {                               // (every lane takes part in the shuffles)
+      const int d = H / K;
+      float ss[2], sd[2];
+#pragma unroll
+      for (int jg = 0; jg < 2; ++jg) {
+        const int c = jg * 64 + tx * 4;
+        const float z[4] = {acc[i][jg * 4], acc[i][jg * 4 + 1], acc[i][jg * 4 + 2], acc[i][jg * 4 + 3]};
+        head_partial(z, a_src, a_dst, c < H ? c : 0, d >= 64 ? 16 : (d >> 2), ss[jg], sd[jg]);   // (columns >= H hold 0)
+      }
+      if (r < rows) {
+        if (d == 128) {                         // one head over both column groups
+          if (tx == 0) scores[size_t(r) * K] = make_float2((ss[0] + ss[1]) * kLog2e, (sd[0] + sd[1]) * kLog2e);
+        } else {
+          const int g = d >= 64 ? 16 : (d >> 2);
+#pragma unroll
+          for (int jg = 0; jg < 2; ++jg) {
+            const int c = jg * 64 + tx * 4;
+            if (c < H && (tx & (g - 1)) == 0) scores[size_t(r) * K + c / d] = make_float2(ss[jg] * kLog2e, sd[jg] * kLog2e);
+          }
+        }
+      }
+    }
     if (r >= rows) continue;
 #pragma unroll
     for (int jg = 0; jg < 2; ++jg) {
@@ -152,32 +200,58 @@ k_xform_simt128(const T* __restrict__ h, const T* __restrict__ W, T* __restrict_
 
 }  // namespace
 
+// SCORES variant: fp32 storage, one tile across all H columns, heads 4 ... 128 columns wide (a power of two)
+static bool fuse_scores(const Dims& d, int tile_cols, const float* scores) {
+  if (d.dtype != XRL_FP32 || d.zmerged || scores == nullptr || d.H > tile_cols || (d.H & 3) || d.K < 1 || d.H % d.K) return false;
+  const int w = d.H / d.K;
+  return w >= 4 && w <= tile_cols && (w & (w - 1)) == 0;
+}
+
 int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* scores,
                       Window win, cudaStream_t st) {
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   if (rows <= 0) return 0;
   const size_t off = size_t(win.row_begin - win.win_base) * d.H;
+  float2* sc = reinterpret_cast<float2*>(scores) + size_t(win.row_begin - win.win_base) * d.K;
   if (rows >= 8192) {
     dim3 g128(unsigned((rows + TM - 1) / TM), unsigned((d.H + TN - 1) / TN));
-    if (d.dtype == XRL_BF16)
-      k_xform_simt128<bf16><<<g128, 256, 0, st>>>(static_cast<const bf16*>(h) + off,
-                                                  static_cast<const bf16*>(lw.W),
-                                                  static_cast<bf16*>(Z) + off, d.H, int(rows));
-    else
-      k_xform_simt128<float><<<g128, 256, 0, st>>>(static_cast<const float*>(h) + off,
-                                                   static_cast<const float*>(lw.W),
-                                                   static_cast<float*>(Z) + off, d.H, int(rows));
+    if (d.dtype == XRL_BF16) {
+      k_xform_simt128<bf16, false><<<g128, 256, 0, st>>>(static_cast<const bf16*>(h) + off,
+                                                         static_cast<const bf16*>(lw.W),
+                                                         static_cast<bf16*>(Z) + off, d.H, int(rows), nullptr, nullptr,
+                                                         nullptr, d.K);
+    } else if (fuse_scores(d, TN, scores)) {
+      k_xform_simt128<float, true><<<g128, 256, 0, st>>>(static_cast<const float*>(h) + off,
+                                                         static_cast<const float*>(lw.W),
+                                                         static_cast<float*>(Z) + off, d.H, int(rows), lw.a_src, lw.a_dst,
+                                                         sc, d.K);
+      return 1;
+    } else {
+      k_xform_simt128<float, false><<<g128, 256, 0, st>>>(static_cast<const float*>(h) + off,
+                                                          static_cast<const float*>(lw.W),
+                                                          static_cast<float*>(Z) + off, d.H, int(rows), nullptr, nullptr,
+                                                          nullptr, d.K);
+    }
     return 1 + launch_scores(d, Z, lw, scores, win, st);
   }
   dim3 grid(unsigned((rows + BM - 1) / BM), unsigned((d.H + BN - 1) / BN));
-  if (d.dtype == XRL_BF16)
-    k_xform_simt<bf16><<<grid, 256, 0, st>>>(static_cast<const bf16*>(h) + off,
-                                            static_cast<const bf16*>(lw.W),
-                                            static_cast<bf16*>(Z) + off, d.H, int(rows));
-  else
-    k_xform_simt<float><<<grid, 256, 0, st>>>(static_cast<const float*>(h) + off,
-                                             static_cast<const float*>(lw.W),
-                                             static_cast<float*>(Z) + off, d.H, int(rows));
+  if (d.dtype == XRL_BF16) {
+    k_xform_simt<bf16, false><<<grid, 256, 0, st>>>(static_cast<const bf16*>(h) + off,
+                                                   static_cast<const bf16*>(lw.W),
+                                                   static_cast<bf16*>(Z) + off, d.H, int(rows), nullptr, nullptr, nullptr,
+                                                   d.K);
+  } else if (fuse_scores(d, BN, scores)) {
+    k_xform_simt<float, true><<<grid, 256, 0, st>>>(static_cast<const float*>(h) + off,
+                                                   static_cast<const float*>(lw.W),
+                                                   static_cast<float*>(Z) + off, d.H, int(rows), lw.a_src, lw.a_dst, sc,
+                                                   d.K);
+    return 1;
+  } else {
+    k_xform_simt<float, false><<<grid, 256, 0, st>>>(static_cast<const float*>(h) + off,
+                                                    static_cast<const float*>(lw.W),
+                                                    static_cast<float*>(Z) + off, d.H, int(rows), nullptr, nullptr,
+                                                    nullptr, d.K);
+  }
   return 1 + launch_scores(d, Z, lw, scores, win, st);
 }
 
