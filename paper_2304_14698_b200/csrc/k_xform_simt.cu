@@ -198,13 +198,162 @@ k_xform_simt128(const T* __restrict__ h, const T* __restrict__ W, T* __restrict_
   }
 }
 
+
+// ---- fp32 storage, many rows: the product on the tensor cores with every operand split in two ----------------
+// x = hi + lo with hi = tf32(x) and lo = tf32(x - hi); Z = sum hi_a hi_b + hi_a lo_b + lo_a hi_b in fp32
+// accumulators (mma.sync m16n8k8, the small terms first): the dropped lo_a lo_b term is below 2^-22 of the
+// product, i.e. the result is as good as an fp32 FMA chain in another order.  CTA tile 128 rows x 128 columns,
+// 8 warps as 4 (rows) x 2 (columns), warp tile 32 x 64 = 2 x 8 MMA tiles; K advanced 16 at a time; both splits of a
+// slice are made once, when it is written to shared memory (stored k-major: fragment reads are conflict-free
+// with a row stride of 136 words).  Half-scores from the accumulators when a head is 8 ... 64 columns wide.
+constexpr int XM = 128, XN = 128, XK = 16, XS = 136;
+
+__device__ __forceinline__ uint32_t to_tf32(float x) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+               "{%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+template <bool SCORES>
+__global__ void __launch_bounds__(256, 2)
+k_xform_tf32x3(const float* __restrict__ h, const float* __restrict__ W, float* __restrict__ Z, int H, int rows,
+               const float* __restrict__ a_src, const float* __restrict__ a_dst, float2* __restrict__ scores, int K) {
+  extern __shared__ __align__(16) uint32_t xs[];          // A hi, A lo, B hi, B lo: each [XK][XS]
+  uint32_t* Ah = xs;
+  uint32_t* Al = Ah + XK * XS;
+  uint32_t* Bh = Al + XK * XS;
+  uint32_t* Bl = Bh + XK * XS;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int wm = (warp >> 1) * 32, wn = (warp & 1) * 64;  // the warp's tile inside the CTA tile
+  const int64_t row0 = int64_t(blockIdx.x) * XM;
+  const int col0 = blockIdx.y * XN;
+  float acc[2][8][4];
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.f;
+
+  // loads of one slice: A 128 rows x 16 k = 512 float4 (two per thread), B 16 k x 128 columns = 512 float4
+  const int a_row = tid >> 2, a_k = (tid & 3) * 4;        // and a_row + 64
+  const int b_k = tid >> 5, b_c = (tid & 31) * 4;         // and b_k + 8
+  const bool a_ok0 = row0 + a_row < rows, a_ok1 = row0 + a_row + 64 < rows;
+  const bool b_ok = col0 + b_c < H;                       // H is a multiple of 4
+  const float* a_p0 = h + size_t(a_ok0 ? row0 + a_row : 0) * H + a_k;
+  const float* a_p1 = h + size_t(a_ok1 ? row0 + a_row + 64 : 0) * H + a_k;
+  const float* b_p = W + size_t(b_k) * H + (b_ok ? col0 + b_c : 0);
+  const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 ra0 = a_ok0 ? __ldg(reinterpret_cast<const float4*>(a_p0)) : zero4;
+  float4 ra1 = a_ok1 ? __ldg(reinterpret_cast<const float4*>(a_p1)) : zero4;
+  float4 rb0 = b_ok ? __ldg(reinterpret_cast<const float4*>(b_p)) : zero4;
+  float4 rb1 = b_ok ? __ldg(reinterpret_cast<const float4*>(b_p + size_t(8) * H)) : zero4;
+
+  auto split_store = [&](uint32_t* hi, uint32_t* lo, int idx, float x) {
+    const uint32_t hb = to_tf32(x);
+    hi[idx] = hb;
+    lo[idx] = to_tf32(x - __uint_as_float(hb));
+  };
+  for (int k0 = 0; k0 < H; k0 += XK) {
+    {
+      const float a0[4] = {ra0.x, ra0.y, ra0.z, ra0.w}, a1[4] = {ra1.x, ra1.y, ra1.z, ra1.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        split_store(Ah, Al, (a_k + e) * XS + a_row, a0[e]);
+        split_store(Ah, Al, (a_k + e) * XS + a_row + 64, a1[e]);
+      }
+      const float b0[4] = {rb0.x, rb0.y, rb0.z, rb0.w}, b1[4] = {rb1.x, rb1.y, rb1.z, rb1.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        split_store(Bh, Bl, b_k * XS + b_c + e, b0[e]);
+        split_store(Bh, Bl, (b_k + 8) * XS + b_c + e, b1[e]);
+      }
+    }
+    __syncthreads();
+    if (k0 + XK < H) {                                    // next slice in flight during the arithmetic
+      ra0 = a_ok0 ? __ldg(reinterpret_cast<const float4*>(a_p0 + k0 + XK)) : zero4;
+      ra1 = a_ok1 ? __ldg(reinterpret_cast<const float4*>(a_p1 + k0 + XK)) : zero4;
+      rb0 = b_ok ? __ldg(reinterpret_cast<const float4*>(b_p + size_t(k0 + XK) * H)) : zero4;
+      rb1 = b_ok ? __ldg(reinterpret_cast<const float4*>(b_p + size_t(k0 + XK + 8) * H)) : zero4;
+    }
+#pragma unroll
+    for (int ks = 0; ks < XK; ks += 8) {
+      uint32_t ah[2][4], al[2][4];
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const int r = wm + i * 16 + g;
+        // fragment of a 16 x 8 tile: (row g, k t), (row g + 8, k t), (row g, k t + 4), (row g + 8, k t + 4)
+        ah[i][0] = Ah[(ks + t) * XS + r];     ah[i][1] = Ah[(ks + t) * XS + r + 8];
+        ah[i][2] = Ah[(ks + t + 4) * XS + r]; ah[i][3] = Ah[(ks + t + 4) * XS + r + 8];
+        al[i][0] = Al[(ks + t) * XS + r];     al[i][1] = Al[(ks + t) * XS + r + 8];
+        al[i][2] = Al[(ks + t + 4) * XS + r]; al[i][3] = Al[(ks + t + 4) * XS + r + 8];
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int c = wn + j * 8 + g;
+        // fragment of an 8 x 8 tile: (k t, column g), (k t + 4, column g)
+        const uint32_t bh[2] = {Bh[(ks + t) * XS + c], Bh[(ks + t + 4) * XS + c]};
+        const uint32_t bl[2] = {Bl[(ks + t) * XS + c], Bl[(ks + t + 4) * XS + c]};
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          mma_tf32(acc[i][j], al[i], bh);
+          mma_tf32(acc[i][j], ah[i], bl);
+          mma_tf32(acc[i][j], ah[i], bh);
+        }
+      }
+    }
+    __syncthreads();
+  }
+  // accumulator of an MMA tile: (row g, columns 2t, 2t + 1), (row g + 8, columns 2t, 2t + 1)
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const int64_t r = row0 + wm + i * 16 + g + half * 8;
+      if (SCORES) {                             // (every lane takes part in the shuffles)
+        const int d = H / K, tiles = d >> 3;    // MMA tiles per head: 1, 2, 4 or 8
+        float ss = 0.f, sd = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int c = col0 + wn + j * 8 + 2 * t;
+          const int cc = c < H ? c : 0;         // (columns >= H hold 0)
+          const float2 s = __ldg(reinterpret_cast<const float2*>(a_src + cc));
+          const float2 u = __ldg(reinterpret_cast<const float2*>(a_dst + cc));
+          ss = fmaf(acc[i][j][2 * half + 1], s.y, fmaf(acc[i][j][2 * half], s.x, ss));
+          sd = fmaf(acc[i][j][2 * half + 1], u.y, fmaf(acc[i][j][2 * half], u.x, sd));
+          if (((j + 1) & (tiles - 1)) == 0) {   // the head ends with this tile
+            ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1); sd += __shfl_xor_sync(0xFFFFFFFFu, sd, 1);
+            ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2); sd += __shfl_xor_sync(0xFFFFFFFFu, sd, 2);
+            if (t == 0 && r < rows && c < H) scores[size_t(r) * K + c / d] = make_float2(ss * kLog2e, sd * kLog2e);
+            ss = 0.f; sd = 0.f;
+          }
+        }
+      }
+      if (r >= rows) continue;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int c = col0 + wn + j * 8 + 2 * t;
+        if (c < H) *reinterpret_cast<float2*>(Z + size_t(r) * H + c) = make_float2(acc[i][j][2 * half], acc[i][j][2 * half + 1]);
+      }
+    }
+  }
+}
+
 }  // namespace
 
 // SCORES variant: fp32 storage, one tile across all H columns, heads 4 ... 128 columns wide (a power of two)
-static bool fuse_scores(const Dims& d, int tile_cols, const float* scores) {
+static bool fuse_scores(const Dims& d, const LayerWeights& lw, int tile_cols, const float* scores, int min_width = 4) {
   if (d.dtype != XRL_FP32 || d.zmerged || scores == nullptr || d.H > tile_cols || (d.H & 3) || d.K < 1 || d.H % d.K) return false;
+  if ((reinterpret_cast<uintptr_t>(lw.a_src) | reinterpret_cast<uintptr_t>(lw.a_dst)) & 15) return false;   // vector loads
   const int w = d.H / d.K;
-  return w >= 4 && w <= tile_cols && (w & (w - 1)) == 0;
+  return w >= min_width && w <= tile_cols && (w & (w - 1)) == 0;
 }
 
 int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void* Z, float* scores,
@@ -213,6 +362,21 @@ int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void
   if (rows <= 0) return 0;
   const size_t off = size_t(win.row_begin - win.win_base) * d.H;
   float2* sc = reinterpret_cast<float2*>(scores) + size_t(win.row_begin - win.win_base) * d.K;
+  if (rows >= 8192 && d.dtype == XRL_FP32 && d.H % XK == 0) {
+    // fp32 storage: split operands on the tensor cores
+    dim3 gx(unsigned((rows + XM - 1) / XM), unsigned((d.H + XN - 1) / XN));
+    const size_t smem = sizeof(uint32_t) * 4 * XK * XS;
+    const int w = d.H / d.K;
+    if (fuse_scores(d, lw, XN, scores, 8) && w <= 64) {
+      k_xform_tf32x3<true><<<gx, 256, smem, st>>>(static_cast<const float*>(h) + off, static_cast<const float*>(lw.W),
+                                                 static_cast<float*>(Z) + off, d.H, int(rows), lw.a_src, lw.a_dst, sc, d.K);
+      return 1;
+    }
+    k_xform_tf32x3<false><<<gx, 256, smem, st>>>(static_cast<const float*>(h) + off, static_cast<const float*>(lw.W),
+                                                static_cast<float*>(Z) + off, d.H, int(rows), nullptr, nullptr, nullptr,
+                                                d.K);
+    return 1 + launch_scores(d, Z, lw, scores, win, st);
+  }
   if (rows >= 8192) {
     dim3 g128(unsigned((rows + TM - 1) / TM), unsigned((d.H + TN - 1) / TN));
     if (d.dtype == XRL_BF16) {
@@ -220,7 +384,7 @@ int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void
                                                          static_cast<const bf16*>(lw.W),
                                                          static_cast<bf16*>(Z) + off, d.H, int(rows), nullptr, nullptr,
                                                          nullptr, d.K);
-    } else if (fuse_scores(d, TN, scores)) {
+    } else if (fuse_scores(d, lw, TN, scores)) {
       k_xform_simt128<float, true><<<g128, 256, 0, st>>>(static_cast<const float*>(h) + off,
                                                          static_cast<const float*>(lw.W),
                                                          static_cast<float*>(Z) + off, d.H, int(rows), lw.a_src, lw.a_dst,
@@ -240,7 +404,7 @@ int launch_xform_simt(const Dims& d, const void* h, const LayerWeights& lw, void
                                                    static_cast<const bf16*>(lw.W),
                                                    static_cast<bf16*>(Z) + off, d.H, int(rows), nullptr, nullptr, nullptr,
                                                    d.K);
-  } else if (fuse_scores(d, BN, scores)) {
+  } else if (fuse_scores(d, lw, BN, scores)) {
     k_xform_simt<float, true><<<grid, 256, 0, st>>>(static_cast<const float*>(h) + off,
                                                    static_cast<const float*>(lw.W),
                                                    static_cast<float*>(Z) + off, d.H, int(rows), lw.a_src, lw.a_dst, sc,
