@@ -23,7 +23,14 @@ __device__ __forceinline__ void load_shape(const bf16* shape, int32_t node, floa
 // ---- Eq. 6: h0_i = ReLU(W0^T [ sum_{j->i} shape_j | onehot(op_i) | shape_i ] + b0) -----------
 // (with attributes on the edges, Section 3.3.2 as written, the sum runs over the in-edges' own attributes)
 // The one-hot block of the product is a row lookup of W0; the two shape blocks are a 16 x H
-// dense map kept in shared memory as fp32.
+// dense map kept in shared memory as fp32.  A warp takes 8 rows at a time in two phases: first a lane per row
+// gathers the row's sixteen dense inputs (row pointers, producers, their shape features: a chain of dependent
+// loads, 8 chains side by side), then the warp's lanes share each row's columns, reading the inputs back from
+// shared memory; the lookups of W0 for up to four rows are issued before the first is used.
+constexpr int kEmbedWarps = kRowThreads / 32;
+constexpr int kEmbedRows = 8;        // rows a warp takes at a time
+struct EmbedStage { float x[kEmbedRows][2 * kS]; int32_t op[kEmbedRows]; };
+
 template <typename T, int LPR, int VPL>
 __global__ void __launch_bounds__(kRowThreads)
 k_embed(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
@@ -32,9 +39,10 @@ k_embed(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
         const int32_t* __restrict__ row_list, const T* __restrict__ eattr) {
   constexpr int VEC = VecOf<T>::N;
   constexpr int RPW = 32 / LPR;
-  extern __shared__ float smem[];
-  float* Wd = smem;                    // [2*kS][H]
-  float* bs = smem + 2 * kS * H;       // [H]
+  extern __shared__ __align__(16) float smem[];
+  EmbedStage& stg = reinterpret_cast<EmbedStage*>(smem)[threadIdx.x >> 5];
+  float* Wd = smem + kEmbedWarps * (sizeof(EmbedStage) / sizeof(float));   // [2*kS][H]
+  float* bs = Wd + 2 * kS * H;                                             // [H]
   for (int t = threadIdx.x; t < 2 * kS * H; t += blockDim.x) {
     const int s = t / H, c = t - s * H;
     const int src_row = (s < kS) ? s : (kS + Tn + (s - kS));
@@ -47,48 +55,96 @@ k_embed(const int32_t* __restrict__ rowptr, const int32_t* __restrict__ col,
   const int lane = threadIdx.x & 31, sub = lane / LPR, sl = lane % LPR;
   const int warps_total = (gridDim.x * blockDim.x) >> 5;
   const int warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * RPW; r0 < win.row_end;
-       r0 += int64_t(warps_total) * RPW) {
-    const int32_t out_row = int32_t(r0) + sub;
-    if (out_row >= win.row_end) continue;
-    const int32_t row = row_list ? __ldg(row_list + out_row) : out_row;   // listed rows are written densely
-    float x[2 * kS];
+  // fp32 rows with one vector of columns per lane: the lane's 16 x VEC slice of the dense map and its bias stay in registers
+  // (read from shared memory per row, the map makes the kernel wait on shared-memory bandwidth)
+  constexpr bool REGW = VPL == 1 && VEC == 4;
+  float wreg[REGW ? 2 * kS : 1][VEC], breg[VEC];
+  if (REGW && sl < NV) {
 #pragma unroll
-    for (int s = 0; s < kS; ++s) x[s] = 0.f;
-    const int32_t e0 = __ldg(rowptr + row), e1 = __ldg(rowptr + row + 1);
-    for (int32_t e = e0; e < e1; ++e) {
-      float f[kS];
-      if (eattr) load_shape(eattr, e, f);            // attributes on the edges, already in slot order
-      else load_shape(shape, __ldg(col + e), f);     // the producer's shape features
+    for (int s = 0; s < 2 * kS; ++s)
 #pragma unroll
-      for (int s = 0; s < kS; ++s) x[s] += f[s];
+      for (int t = 0; t < VEC; ++t) wreg[REGW ? s : 0][t] = Wd[s * H + sl * VEC + t];
+#pragma unroll
+    for (int t = 0; t < VEC; ++t) breg[t] = bs[sl * VEC + t];
+  }
+  for (int64_t r0 = int64_t(win.row_begin) + int64_t(warp_id) * kEmbedRows; r0 < win.row_end;
+       r0 += int64_t(warps_total) * kEmbedRows) {
+    const int nr = int(min(int64_t(kEmbedRows), win.row_end - r0));
+    __syncwarp();
+    if (lane < nr) {
+      const int32_t out_row = int32_t(r0) + lane;
+      const int32_t row = row_list ? __ldg(row_list + out_row) : out_row;   // listed rows are written densely
+      float x[kS];
+#pragma unroll
+      for (int s = 0; s < kS; ++s) x[s] = 0.f;
+      const int32_t e0 = __ldg(rowptr + row), e1 = __ldg(rowptr + row + 1);
+      for (int32_t e = e0; e < e1; ++e) {
+        float f[kS];
+        if (eattr) load_shape(eattr, e, f);            // attributes on the edges, already in slot order
+        else load_shape(shape, __ldg(col + e), f);     // the producer's shape features
+#pragma unroll
+        for (int s = 0; s < kS; ++s) x[s] += f[s];
+      }
+      float own[kS];
+      load_shape(shape, row, own);
+#pragma unroll
+      for (int s = 0; s < kS; ++s) { stg.x[lane][s] = x[s]; stg.x[lane][kS + s] = own[s]; }
+      // an operator id outside the table was reported by the packer; clamped here so that nothing is read
+      // outside W0 if the caller encodes such a batch anyway
+      stg.op[lane] = min(max(__ldg(op + row), 0), Tn - 1);
     }
-    {
-      float f[kS];
-      load_shape(shape, row, f);
+    __syncwarp();
+    constexpr int U = (VPL >= 4) ? 1 : (VPL == 2 ? 2 : 4);     // rows whose lookups are in flight together
+    for (int rb = sub; rb < nr; rb += RPW * U) {
+      float acc[U][VPL][VEC];
 #pragma unroll
-      for (int s = 0; s < kS; ++s) x[kS + s] = f[s];
-    }
-    // an operator id outside the table was reported by the packer; clamped here so that nothing is read
-    // outside W0 if the caller encodes such a batch anyway
-    const T* lookup = W0 + size_t(kS + min(max(__ldg(op + row), 0), Tn - 1)) * H;
-    T* out = h + size_t(out_row - win.win_base) * H;
+      for (int u = 0; u < U; ++u) {
+        const int rr = rb + u * RPW;
+        if (rr < nr) {
+          const T* lookup = W0 + size_t(kS + stg.op[rr]) * H;
 #pragma unroll
-    for (int v = 0; v < VPL; ++v) {
-      const int vi = v * LPR + sl;
-      if (vi < NV) {
-        const int c0 = vi * VEC;
-        float acc[VEC];
-        load_vec(lookup + c0, acc);
+          for (int v = 0; v < VPL; ++v) {
+            const int vi = v * LPR + sl;
+            if (vi < NV) load_vec(lookup + vi * VEC, acc[u][v]);
+          }
+        }
+      }
 #pragma unroll
-        for (int t = 0; t < VEC; ++t) acc[t] += bs[c0 + t];
+      for (int u = 0; u < U; ++u) {
+        const int rr = rb + u * RPW;
+        if (rr >= nr) continue;
+        float x[2 * kS];
 #pragma unroll
-        for (int s = 0; s < 2 * kS; ++s)
+        for (int s = 0; s < 2 * kS; s += 4) {
+          const float4 v4 = *reinterpret_cast<const float4*>(&stg.x[rr][s]);
+          x[s] = v4.x; x[s + 1] = v4.y; x[s + 2] = v4.z; x[s + 3] = v4.w;
+        }
+        T* out = h + size_t(int32_t(r0) + rr - win.win_base) * H;
 #pragma unroll
-          for (int t = 0; t < VEC; ++t) acc[t] = fmaf(x[s], Wd[s * H + c0 + t], acc[t]);
+        for (int v = 0; v < VPL; ++v) {
+          const int vi = v * LPR + sl;
+          if (vi < NV) {
+            const int c0 = vi * VEC;
+            if (REGW) {
 #pragma unroll
-        for (int t = 0; t < VEC; ++t) acc[t] = fmaxf(acc[t], 0.f);
-        store_vec(out + c0, acc);
+              for (int t = 0; t < VEC; ++t) acc[u][v][t] += breg[t];
+#pragma unroll
+              for (int s = 0; s < 2 * kS; ++s)
+#pragma unroll
+                for (int t = 0; t < VEC; ++t) acc[u][v][t] = fmaf(x[s], wreg[REGW ? s : 0][t], acc[u][v][t]);
+            } else {
+#pragma unroll
+              for (int t = 0; t < VEC; ++t) acc[u][v][t] += bs[c0 + t];
+#pragma unroll
+              for (int s = 0; s < 2 * kS; ++s)
+#pragma unroll
+                for (int t = 0; t < VEC; ++t) acc[u][v][t] = fmaf(x[s], Wd[s * H + c0 + t], acc[u][v][t]);
+            }
+#pragma unroll
+            for (int t = 0; t < VEC; ++t) acc[u][v][t] = fmaxf(acc[u][v][t], 0.f);
+            store_vec(out + c0, acc[u][v]);
+          }
+        }
       }
     }
   }
@@ -311,14 +367,22 @@ int row_grid(int64_t rows, int rpw) {
 
 }  // namespace
 
+// one opt-in record per instantiation of k_embed (ensure_dynamic_smem keeps one flag array per kernel)
+static int embed_slot(size_t elem, int lpr, int vpl) {
+  return (elem == 2 ? 5 : 0) + (lpr == 8 ? 0 : lpr == 16 ? 1 : vpl == 1 ? 2 : vpl == 2 ? 3 : 4);
+}
+
 int launch_embed(const Dims& d, const int32_t* rowptr, const int32_t* col, const int32_t* op,
                  const void* shape, const DevWeights& w, void* h, Window win, cudaStream_t st,
                  const int32_t* row_list, const void* eattr) {
   const int64_t rows = int64_t(win.row_end) - win.row_begin;
   if (rows <= 0) return 0;
-  const size_t smem = sizeof(float) * size_t(2 * kS + 1) * d.H;
+  const size_t smem = sizeof(EmbedStage) * kEmbedWarps + sizeof(float) * size_t(2 * kS + 1) * d.H;
+  static bool attr_set[10][64] = {};
 #define CALL(TY_, LPR, VPL)                                                                        \
-  k_embed<TY_, LPR, VPL><<<row_grid(rows, 32 / LPR), kRowThreads, smem, st>>>(                     \
+  if (smem > 48 * 1024 &&                                                                          \
+      !ensure_dynamic_smem(k_embed<TY_, LPR, VPL>, int(smem), attr_set[embed_slot(sizeof(TY_), LPR, VPL)])) return -1; \
+  k_embed<TY_, LPR, VPL><<<row_grid(rows, kEmbedRows), kRowThreads, smem, st>>>(                           \
       rowptr, col, op, static_cast<const TY_*>(shape), static_cast<const TY_*>(w.W0), w.b0,   \
       static_cast<TY_*>(h), d.H, d.T, win, row_list, static_cast<const TY_*>(eattr))
   if (d.dtype == XRL_BF16) XRL_ROW_DISPATCH(bf16, d.H, CALL);
